@@ -1,0 +1,424 @@
+"""CPU oracle for SWIFT's decoding hot path (arXiv 2410.06916).  TEST INFRASTRUCTURE ONLY.
+
+A plain, slow, obviously-correct restatement of what the path computes, in ordinary PyTorch CPU
+ops (fp64 by default; fp32 for the multi-billion-parameter shapes that do not fit host RAM in
+fp64).  It shares no code with the CUDA library and must never be imported by it: only tests, the
+smoke check and the benchmark's CPU-baseline leg use this file.
+
+What is pinned by tests independent of this file: the decoder forward against the Huggingface LLaMA
+implementation the paper ran (Appendix B.2) and against torch's fused attention; greedy
+losslessness against vanilla decoding (Section 3.1); sampling acceptance by chi-squared and the
+closed-form acceptance rate; matchness (Eq. 3) by brute force; Eq. 5 against the values printed in
+Table 5; Philox against an independent library implementation.
+
+Parity unpinned by the paper (readings, fixed by convention only): RMSNorm eps 1e-5, RoPE theta
+1e4 with rotate-half pairing, argmax tie rule (lowest id), the random-number stream layout.
+
+Notation follows the paper: z in {0,1}^L is the skipped sub-layer set over L = 2*n_blocks sub-layers
+ordered [attn_0, mlp_0, attn_1, ...]; y'_j are draft tokens, p_j their confidence, gamma the context
+window, N_D the maximum draft length, epsilon the early-stop threshold.
+"""
+from __future__ import annotations
+
+import math
+from dataclasses import dataclass, field
+from typing import Dict, List, Optional, Sequence, Tuple
+
+import torch
+
+_MASK32 = 0xFFFFFFFF
+
+
+# =============================================================================== random numbers
+def philox4x32_10(ctr: Sequence[int], key: Sequence[int]) -> Tuple[int, int, int, int]:
+    """Philox4x32-10 (Salmon et al., SC'11): ten rounds of two 32x32->64 multiplies and xors."""
+    c = [int(v) & _MASK32 for v in ctr]
+    k = [int(v) & _MASK32 for v in key]
+    for _ in range(10):
+        prod0 = 0xD2511F53 * c[0]
+        prod1 = 0xCD9E8D57 * c[2]
+        c = [((prod1 >> 32) ^ c[1] ^ k[0]) & _MASK32, prod1 & _MASK32,
+             ((prod0 >> 32) ^ c[3] ^ k[1]) & _MASK32, prod0 & _MASK32]
+        k = [(k[0] + 0x9E3779B9) & _MASK32, (k[1] + 0xBB67AE85) & _MASK32]
+    return tuple(c)
+
+
+# purposes of a random draw inside one decoding round (counter word 2)
+DRAW_DRAFT, DRAW_ACCEPT, DRAW_RESAMPLE, DRAW_BONUS = 0, 1, 2, 3
+
+
+def uniform(seed: int, round_index: int, slot: int, purpose: int) -> float:
+    """u in [0,1): top 24 bits of the first Philox word at counter (round, slot, purpose, 0)."""
+    w = philox4x32_10((round_index, slot, purpose, 0), (seed & _MASK32, (seed >> 32) & _MASK32))
+    return (w[0] >> 8) * (2.0 ** -24)
+
+
+def categorical(weights: torch.Tensor, u: float) -> Tuple[int, float]:
+    """Smallest index i whose running sum (taken in index order) exceeds u * total.
+
+    Returns (i, relative distance of u*total to the nearest edge of bin i) so a comparison with
+    another implementation can exempt draws that sit on a bin edge.
+    """
+    w = weights.to(torch.float64)
+    cs = torch.cumsum(w, 0)
+    total = float(cs[-1])
+    t = u * total
+    i = int(torch.searchsorted(cs, torch.tensor(t, dtype=torch.float64), right=True))
+    i = min(i, w.numel() - 1)
+    while float(w[i]) == 0.0 and i > 0:   # only reachable through rounding at the very top
+        i -= 1
+    lo = float(cs[i - 1]) if i > 0 else 0.0
+    dist = min(t - lo, float(cs[i]) - t) / total
+    return i, dist
+
+
+# =============================================================================== model pieces
+def rmsnorm(x: torch.Tensor, g: torch.Tensor, eps: float) -> torch.Tensor:
+    """x * g / sqrt(mean(x^2) + eps), row-wise."""
+    return x * torch.rsqrt((x * x).mean(dim=-1, keepdim=True) + eps) * g.to(x.dtype)
+
+
+def rope(x: torch.Tensor, positions: torch.Tensor, theta: float) -> torch.Tensor:
+    """Rotary embedding, rotate-half pairing: dim i is paired with dim i + d_h/2.
+
+    x: [M, heads, d_h]; positions: [M] absolute indices from 0.
+    """
+    M, _, dh = x.shape
+    half = dh // 2
+    inv_freq = theta ** (-torch.arange(half, dtype=torch.float64) * 2.0 / dh)
+    ang = positions.to(torch.float64)[:, None] * inv_freq[None, :]          # [M, half]
+    cos, sin = torch.cos(ang).to(x.dtype)[:, None, :], torch.sin(ang).to(x.dtype)[:, None, :]
+    x1, x2 = x[..., :half], x[..., half:]
+    return torch.cat([x1 * cos - x2 * sin, x2 * cos + x1 * sin], dim=-1)
+
+
+def attention(q: torch.Tensor, K: torch.Tensor, V: torch.Tensor, allowed: torch.Tensor) -> torch.Tensor:
+    """softmax(q K^T / sqrt(d_h)) V per head, with an explicit boolean mask.
+
+    q: [M, H, d_h]; K, V: [n, H_kv, d_h]; allowed: [M, n].  Query head h reads KV head h // (H/H_kv).
+    """
+    M, H, dh = q.shape
+    Hkv = K.shape[1]
+    group = H // Hkv
+    out = torch.empty_like(q)
+    for h in range(H):
+        kh, vh = K[:, h // group, :], V[:, h // group, :]
+        s = (q[:, h, :] @ kh.T) / math.sqrt(dh)
+        s = s.masked_fill(~allowed, float("-inf"))
+        out[:, h, :] = torch.softmax(s, dim=-1) @ vh
+    return out
+
+
+def swiglu(gate: torch.Tensor, up: torch.Tensor) -> torch.Tensor:
+    return gate * torch.sigmoid(gate) * up
+
+
+def argmax_lowest(row: torch.Tensor) -> int:
+    """argmax with ties broken towards the lowest token id."""
+    m = row.max()
+    return int(torch.nonzero(row == m)[0])
+
+
+def top2_margin(row: torch.Tensor) -> float:
+    v = torch.topk(row.to(torch.float64), 2).values
+    return float(v[0] - v[1])
+
+
+@dataclass
+class Shape:
+    n_blocks: int
+    d_model: int
+    n_heads: int
+    n_kv_heads: int
+    head_dim: int
+    ffn: int
+    vocab: int
+    rope_theta: float = 10000.0
+    rms_eps: float = 1e-5
+
+    @staticmethod
+    def of(cfg) -> "Shape":
+        return Shape(cfg.n_blocks, cfg.d_model, cfg.n_heads, cfg.n_kv_heads, cfg.head_dim, cfg.ffn,
+                     cfg.vocab, cfg.rope_theta, cfg.rms_eps)
+
+
+# =============================================================================== decoder forward
+class Oracle:
+    """The target model, its KV cache and the committed sequence.
+
+    State after prefill: `tokens` = prompt + generated tokens including the pending token t* (whose
+    K,V are not in the cache yet); `n` = number of cached positions = len(tokens) - 1.
+    """
+
+    def __init__(self, shape: Shape, weights: Dict[str, object], dtype=torch.float64, max_positions: int = 4096):
+        self.s = shape
+        self.w = weights
+        self.dtype = dtype
+        self.max_positions = max_positions
+        s = shape
+        self.K = [torch.zeros(max_positions, s.n_kv_heads, s.head_dim, dtype=dtype) for _ in range(s.n_blocks)]
+        self.V = [torch.zeros(max_positions, s.n_kv_heads, s.head_dim, dtype=dtype) for _ in range(s.n_blocks)]
+        self.tokens: List[int] = []
+        self.n = 0
+
+    # ---- one weight application; weights may be stored in a narrower type and are widened exactly
+    def _lin(self, x: torch.Tensor, W: torch.Tensor) -> torch.Tensor:
+        return x @ W.to(self.dtype).T
+
+    def forward_rows(self, row_tokens: Sequence[int], pos0: int, z: Optional[Sequence[int]] = None,
+                     write_kv: bool = True) -> torch.Tensor:
+        """Logits [M, V] for M new rows at positions pos0..pos0+M-1 under skipped sub-layer set z.
+
+        Every row attends to cached positions [0, pos0) and causally to the new rows.  A skipped
+        sub-layer is the identity on the residual stream (Section 3.1): its norm, projections and,
+        for attention, its K,V computation are all left out.  K,V of the new rows are stored in the
+        cache for non-skipped attention sub-layers when write_kv is set.
+        """
+        s = self.s
+        M = len(row_tokens)
+        z = [0] * (2 * s.n_blocks) if z is None else [int(v) for v in z]
+        assert len(z) == 2 * s.n_blocks and pos0 + M <= self.max_positions
+        pos = torch.arange(pos0, pos0 + M)
+        h = self.w["embed"][torch.tensor(list(row_tokens), dtype=torch.long)].to(self.dtype)
+        # row i may read cache position j < pos0 always, and new row j' <= i
+        allowed = torch.cat([torch.ones(M, pos0, dtype=torch.bool),
+                             torch.tril(torch.ones(M, M, dtype=torch.bool))], dim=1)
+        for b in range(s.n_blocks):
+            wb = self.w["blocks"][b]
+            if not z[2 * b]:
+                x = rmsnorm(h, wb["attn_norm"], s.rms_eps)
+                q = self._lin(x, wb["wq"]).view(M, s.n_heads, s.head_dim)
+                k = self._lin(x, wb["wk"]).view(M, s.n_kv_heads, s.head_dim)
+                v = self._lin(x, wb["wv"]).view(M, s.n_kv_heads, s.head_dim)
+                q, k = rope(q, pos, s.rope_theta), rope(k, pos, s.rope_theta)
+                Kall = torch.cat([self.K[b][:pos0], k], dim=0)
+                Vall = torch.cat([self.V[b][:pos0], v], dim=0)
+                a = attention(q, Kall, Vall, allowed).reshape(M, s.n_heads * s.head_dim)
+                h = h + self._lin(a, wb["wo"])
+                if write_kv:
+                    self.K[b][pos0:pos0 + M] = k
+                    self.V[b][pos0:pos0 + M] = v
+            if not z[2 * b + 1]:
+                x = rmsnorm(h, wb["mlp_norm"], s.rms_eps)
+                h = h + self._lin(swiglu(self._lin(x, wb["wgate"]), self._lin(x, wb["wup"])), wb["wdown"])
+        return self._lin(rmsnorm(h, self.w["final_norm"], s.rms_eps), self.w["lm_head"])
+
+    # ---- the steps of the method ---------------------------------------------------------
+    def prefill(self, prompt: Sequence[int], first_token: Optional[int] = None) -> torch.Tensor:
+        """Full model over the prompt; caches K,V for [0, len(prompt)); t* = argmax of the last row
+        unless the caller supplies it (sampling mode draws it outside).  Returns the logits."""
+        logits = self.forward_rows(prompt, 0)
+        self.n = len(prompt)
+        t = argmax_lowest(logits[-1]) if first_token is None else int(first_token)
+        self.tokens = list(prompt) + [t]
+        return logits
+
+    def draft(self, z: Sequence[int], max_k: int, stop_conf: float = 0.0,
+              sampler=None) -> Tuple[List[int], List[float], List[torch.Tensor]]:
+        """Autoregressive drafting with the layer-skipped model (Eq. 4) and early stopping.
+
+        Step j feeds t* (j = 1) or y'_{j-1} at position n+j-1.  y'_j = argmax of the draft logits,
+        p_j = max softmax (T = 1).  The token that falls below epsilon is kept, then drafting stops.
+        With `sampler(j, probs) -> token`, y'_j is drawn from q_j = softmax(draft logits) instead.
+        Returns (draft tokens, confidences, draft logits rows).
+        """
+        toks, confs, rows = [], [], []
+        inp = self.tokens[-1]
+        for j in range(1, max_k + 1):
+            logit = self.forward_rows([inp], self.n + j - 1, z)[0]
+            prob = torch.softmax(logit.to(torch.float64), dim=-1)
+            y = argmax_lowest(logit) if sampler is None else int(sampler(j, prob))
+            toks.append(y)
+            confs.append(float(prob.max()))
+            rows.append(logit)
+            inp = y
+            if confs[-1] < stop_conf:
+                break
+        return toks, confs, rows
+
+    def verify(self, draft_tokens: Sequence[int]) -> torch.Tensor:
+        """Full model on rows [t*, y'_1..y'_k] at positions n..n+k; K,V written for every layer."""
+        return self.forward_rows([self.tokens[-1]] + list(draft_tokens), self.n)
+
+    def commit(self, accepted: Sequence[int], next_token: int) -> None:
+        """KV rollback: keep positions [0, n + a + 1); positions beyond are dropped (left stale)."""
+        self.n += len(accepted) + 1
+        self.tokens += list(accepted) + [int(next_token)]
+
+    def score_skipsets(self, masks: Sequence[Sequence[int]], gamma: int) -> Tuple[List[float], List[List[int]]]:
+        """matchness (Eq. 2-3) of every candidate z_c on the last gamma generated tokens.
+
+        Rows are the inputs tokens[n-gamma .. n-1] at those positions; their known successors are
+        tokens[n-gamma+1 .. n].  The prefix [0, n-gamma) comes from the target's cache; the window's
+        K,V are the candidate's own and are never stored.
+        """
+        n, T = self.n, self.tokens
+        assert gamma <= n and len(T) == n + 1
+        scores, preds = [], []
+        for z in masks:
+            logits = self.forward_rows(T[n - gamma:n], n - gamma, z, write_kv=False)
+            y = [argmax_lowest(logits[i]) for i in range(gamma)]
+            preds.append(y)
+            scores.append(sum(int(y[i] == T[n - gamma + 1 + i]) for i in range(gamma)) / gamma)
+        return scores, preds
+
+
+# =============================================================================== acceptance
+def accept_greedy(draft_tokens: Sequence[int], target_logits: torch.Tensor) -> Tuple[int, int]:
+    """Greedy verification: a = longest prefix with y'_j == argmax(target row j-1); the next token
+    is the target's argmax on row a (the correction, or the bonus token when a = k)."""
+    a = 0
+    for j, y in enumerate(draft_tokens):
+        if argmax_lowest(target_logits[j]) != int(y):
+            break
+        a += 1
+    return a, argmax_lowest(target_logits[a])
+
+
+def accept_sampling(draft_tokens: Sequence[int], q_rows: Sequence[torch.Tensor], target_logits: torch.Tensor,
+                    temperature: float, seed: int, round_index: int) -> Tuple[int, int, List[dict]]:
+    """Speculative-sampling verification (the acceptance strategy of Appendix B.2, after Leviathan et al.).
+
+    p_j = softmax(target row j-1 / T); q_j = the distribution y'_j was drawn from.  For j = 1..k draw
+    u_j and accept iff u_j * q_j(y'_j) < p_j(y'_j)  (i.e. u < min(1, p/q)).  On the first rejection
+    draw the replacement from max(0, p_j - q_j) renormalised; if nothing is rejected draw a bonus token
+    from p_{k+1}.  Returns (a, next token, per-decision records for boundary-aware comparison).
+    """
+    k = len(draft_tokens)
+    P = torch.softmax(target_logits.to(torch.float64) / temperature, dim=-1)
+    log: List[dict] = []
+    for j in range(1, k + 1):
+        y = int(draft_tokens[j - 1])
+        p, q = P[j - 1], q_rows[j - 1].to(torch.float64)
+        u = uniform(seed, round_index, j, DRAW_ACCEPT)
+        lhs, rhs = u * float(q[y]), float(p[y])
+        log.append({"kind": "accept", "j": j, "u": u, "margin": abs(lhs - rhs) / max(rhs, lhs, 1e-300)})
+        if not lhs < rhs:
+            resid = torch.clamp(p - q, min=0.0)
+            if float(resid.sum()) <= 0.0:      # p == q everywhere: no residual mass, fall back to p
+                resid = p
+            tok, dist = categorical(resid, uniform(seed, round_index, j, DRAW_RESAMPLE))
+            log.append({"kind": "resample", "j": j, "margin": dist})
+            return j - 1, tok, log
+    tok, dist = categorical(P[k], uniform(seed, round_index, k + 1, DRAW_BONUS))
+    log.append({"kind": "bonus", "j": k + 1, "margin": dist})
+    return k, tok, log
+
+
+# =============================================================================== whole runs
+@dataclass
+class GenParams:
+    max_new: int
+    max_draft: int = 8            # N_D
+    stop_conf: float = 0.0        # epsilon
+    mode: str = "greedy"          # or "sampling"
+    temperature: float = 1.0
+    rng_seed: int = 0
+    gamma: int = 32
+    stop_matchness: float = 0.95
+    max_opt_rounds: int = 0       # 0 = skip set fixed
+
+
+@dataclass
+class Round:
+    n_start: int
+    draft: List[int]
+    conf: List[float]
+    draft_margin: List[float]
+    target_argmax: List[int]
+    target_margin: List[float]
+    accepted: int
+    next_token: int
+    decisions: List[dict] = field(default_factory=list)
+    matchness: Optional[List[float]] = None
+    z: Optional[List[int]] = None
+
+
+def vanilla_generate(o: Oracle, prompt: Sequence[int], max_new: int, mode: str = "greedy",
+                     temperature: float = 1.0, rng_seed: int = 0) -> Tuple[List[int], List[float]]:
+    """Plain autoregressive decoding of the full model: the definition SWIFT must reproduce."""
+    logits = o.prefill(prompt)
+    margins = [top2_margin(logits[-1])]
+    if mode == "sampling":
+        p = torch.softmax(logits[-1].to(torch.float64) / temperature, -1)
+        o.tokens[-1] = categorical(p, uniform(rng_seed, 0, 0, DRAW_BONUS))[0]
+    step = 0
+    while len(o.tokens) - len(prompt) < max_new:
+        step += 1
+        row = o.forward_rows([o.tokens[-1]], o.n)[0]
+        margins.append(top2_margin(row))
+        if mode == "sampling":
+            p = torch.softmax(row.to(torch.float64) / temperature, -1)
+            t = categorical(p, uniform(rng_seed, step, 0, DRAW_BONUS))[0]
+        else:
+            t = argmax_lowest(row)
+        o.commit([], t)
+    return o.tokens[len(prompt):], margins
+
+
+def swift_generate(o: Oracle, prompt: Sequence[int], z0: Sequence[int], gp: GenParams,
+                   candidates=None) -> Tuple[List[int], List[Round], dict]:
+    """Draft-then-verify decoding with skipped sub-layer set z (Sections 4.1-4.2).
+
+    Each round: [optionally score candidates on the last gamma generated tokens and keep the best] ->
+    draft at most N_D tokens (stop early below epsilon) -> verify with the full model -> accept ->
+    roll the KV cache back.  Emits exactly gp.max_new tokens: the draft length is capped at
+    remaining - 1, and with one token left a plain full-model step is taken.
+    `candidates(round) -> masks [C, L]` supplies the proposals of one optimisation round.
+    """
+    sampling = gp.mode == "sampling"
+    logits = o.prefill(prompt)
+    if sampling:
+        p = torch.softmax(logits[-1].to(torch.float64) / gp.temperature, -1)
+        o.tokens[-1] = categorical(p, uniform(gp.rng_seed, 0, 0, DRAW_BONUS))[0]
+    z = [int(v) for v in z0]
+    best_score, opt_rounds, optimising = -1.0, 0, gp.max_opt_rounds > 0
+    rounds: List[Round] = []
+    n_prompt = len(prompt)
+    r = 0
+    while len(o.tokens) - n_prompt < gp.max_new:
+        r += 1
+        remaining = gp.max_new - (len(o.tokens) - n_prompt)
+        scores = None
+        if optimising and len(o.tokens) - n_prompt > gp.gamma and candidates is not None:
+            masks = candidates(opt_rounds)
+            scores, _ = o.score_skipsets(masks, gp.gamma)
+            c_best = max(range(len(scores)), key=lambda c: (scores[c], -c))
+            if scores[c_best] > best_score:               # strictly better only
+                best_score, z = scores[c_best], [int(v) for v in masks[c_best]]
+            opt_rounds += 1
+            if best_score > gp.stop_matchness or opt_rounds >= gp.max_opt_rounds:
+                optimising = False
+        k_max = min(gp.max_draft, remaining - 1)
+        q_rows: List[torch.Tensor] = []
+        if k_max > 0:
+            if sampling:
+                def sampler(j, prob, _r=r):
+                    q_rows.append(prob)
+                    return categorical(prob, uniform(gp.rng_seed, _r, j, DRAW_DRAFT))[0]
+                d_tok, d_conf, d_rows = o.draft(z, k_max, gp.stop_conf, sampler)
+            else:
+                d_tok, d_conf, d_rows = o.draft(z, k_max, gp.stop_conf)
+        else:
+            d_tok, d_conf, d_rows = [], [], []
+        tl = o.verify(d_tok)
+        if sampling:
+            a, nxt, dec = accept_sampling(d_tok, q_rows, tl, gp.temperature, gp.rng_seed, r)
+        else:
+            (a, nxt), dec = accept_greedy(d_tok, tl), []
+        rounds.append(Round(o.n, d_tok, d_conf, [top2_margin(x) for x in d_rows],
+                            [argmax_lowest(tl[i]) for i in range(len(d_tok) + 1)],
+                            [top2_margin(tl[i]) for i in range(len(d_tok) + 1)], a, nxt, dec, scores, list(z)))
+        o.commit(d_tok[:a], nxt)
+    out = o.tokens[n_prompt:]
+    n_draft = sum(len(x.draft) for x in rounds)
+    stats = {"rounds": len(rounds), "tokens": len(out), "drafted": n_draft,
+             "accepted": sum(x.accepted for x in rounds),
+             "M": (len(out) - 1) / max(len(rounds), 1),    # tokens per target forward (prefill's token excluded)
+             "alpha": sum(x.accepted for x in rounds) / max(n_draft, 1)}
+    return out, rounds, stats
+
+
+def expected_speedup(M: float, alpha: float, c: float) -> float:
+    """Eq. 5: E(Spd.) = M*alpha / ((M-1)*c + alpha), c = 1 - r the draft/target cost ratio."""
+    return M * alpha / ((M - 1.0) * c + alpha)
