@@ -1,0 +1,208 @@
+/*
+ * swift.h — C boundary of the SWIFT decoding hot path on one B200 (sm_100a).
+ *
+ * SWIFT (arXiv 2410.06916) is self-speculative decoding with on-the-fly layer skipping: a draft
+ * model made by skipping sub-layers z of the target LLM proposes tokens (Section 4.2, Eq. 4), the
+ * full model verifies them in one parallel pass (Section 3.1), an acceptance rule keeps the output
+ * distribution unchanged (Appendix B.2), and candidate skip sets are scored by how well they
+ * re-predict the last gamma generated tokens (Section 4.1, Eq. 2-3).
+ *
+ * Conventions for every call
+ *  - Returns a swift_status; nothing aborts, throws or traps.  swift_last_error() gives the text.
+ *  - "host" / "device" on a pointer says where the memory lives.  The caller owns every buffer it
+ *    passes in and keeps device buffers alive until swift_free().  The library allocates no device
+ *    memory; it owns only the host-side context.
+ *  - All work runs on the CUDA stream given to swift_load.  A call that returns values through host
+ *    pointers synchronises that stream before returning.
+ *  - On error the committed state (tokens, KV length) is unchanged.
+ *  - Sub-layer masks are uint8[2*n_blocks] ordered [attn_0, mlp_0, attn_1, mlp_1, ...], 1 = skip
+ *    ("L layers, including both attention and MLP layers", Section 3.1).
+ *  - State machine: load -> prefill -> { draft -> verify -> accept }* ; score_skipsets and
+ *    forward_rows any time after prefill when no round is open; generate = prefill + rounds.
+ */
+#ifndef SWIFT_H
+#define SWIFT_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct swift_ctx swift_ctx; /* opaque, host-side */
+
+typedef enum {
+    SWIFT_OK = 0,
+    SWIFT_EINVAL = 1,       /* bad argument (null pointer, size out of range, bad token id) */
+    SWIFT_ESTATE = 2,       /* call not allowed in the current state (e.g. draft before prefill) */
+    SWIFT_ECAPACITY = 3,    /* rows, positions or buffer sizes beyond what was configured */
+    SWIFT_ECUDA = 4,        /* a CUDA runtime call failed */
+    SWIFT_ETIMEOUT = 5,     /* a bounded device-side wait ran out */
+    SWIFT_EUNSUPPORTED = 6  /* shape or option this build does not handle */
+} swift_status;
+
+enum { SWIFT_F32 = 0, SWIFT_BF16 = 1 };
+enum { SWIFT_GREEDY = 0, SWIFT_SAMPLING = 1 };
+enum { SWIFT_MAX_ROWS = 16 }; /* rows of one forward pass: pending token + at most 15 drafts */
+
+/* Decoder shape (LLaMA-style, the family the paper evaluates, Section 5.1). */
+typedef struct {
+    int32_t n_blocks, d_model, n_heads, n_kv_heads, head_dim, ffn, vocab;
+    int32_t dtype;          /* SWIFT_F32 or SWIFT_BF16: storage of weights, GEMM inputs and KV cache */
+    float rope_theta, rms_eps;
+    int32_t max_positions;  /* KV capacity in positions; multiple of page_size */
+    int32_t page_size;      /* positions per KV page; power of two, 8..128 */
+    int32_t max_draft;      /* largest k any call will use; <= SWIFT_MAX_ROWS - 1 */
+    int32_t reserved;
+} swift_model_desc;
+
+typedef struct { void* dptr; size_t bytes; } swift_devbuf; /* caller-owned device memory, 256-byte aligned */
+
+/* Names of the tensors swift_pack_tensor accepts.  Shapes are row-major [out_features, in_features]. */
+typedef enum {
+    SWIFT_T_EMBED = 0,      /* [vocab, d] */
+    SWIFT_T_LM_HEAD = 1,    /* [vocab, d] */
+    SWIFT_T_FINAL_NORM = 2, /* [d] fp32 gain */
+    SWIFT_T_WQ = 3, SWIFT_T_WK = 4, SWIFT_T_WV = 5, /* [H*dh, d], [Hkv*dh, d], [Hkv*dh, d] */
+    SWIFT_T_WO = 6,         /* [d, H*dh] */
+    SWIFT_T_WGATE = 7, SWIFT_T_WUP = 8, /* [ffn, d] */
+    SWIFT_T_WDOWN = 9,      /* [d, ffn] */
+    SWIFT_T_ATTN_NORM = 10, SWIFT_T_MLP_NORM = 11 /* [d] fp32 gains */
+} swift_tensor_kind;
+
+/* Sizes of the three device buffers swift_load needs for this shape.  0 on an invalid desc. */
+size_t swift_weights_bytes(const swift_model_desc* desc);
+size_t swift_kv_bytes(const swift_model_desc* desc);
+size_t swift_workspace_bytes(const swift_model_desc* desc);
+
+/*
+ * Creates a context over caller-owned device buffers.  `weights` is filled afterwards with
+ * swift_pack_tensor; `kv_pool` and `workspace` need no initialisation.  `cuda_stream` is a
+ * cudaStream_t (NULL = the legacy default stream).  The current CUDA device at the time of the call
+ * is the device of the context.
+ */
+swift_status swift_load(const swift_model_desc* desc, swift_devbuf weights, swift_devbuf kv_pool,
+                        swift_devbuf workspace, void* cuda_stream, swift_ctx** out);
+swift_status swift_free(swift_ctx* ctx);
+const char* swift_last_error(const swift_ctx* ctx); /* ctx may be NULL: last error of a failed swift_load */
+
+/*
+ * Copies one weight tensor from host memory (`src`, contiguous, the model's dtype; fp32 for gains)
+ * into the library's device layout: q/k/v rows are concatenated into one fused projection, gate and
+ * up rows are interleaved in groups of 16 so that one output tile holds matching gate/up pairs.
+ * `block` is ignored for embed / lm_head / final_norm.  Synchronous.
+ */
+swift_status swift_pack_tensor(swift_ctx* ctx, swift_tensor_kind kind, int32_t block, const void* src_host,
+                               size_t src_bytes);
+
+/* Acceptance strategy for the calls that follow (Appendix B.2).  Sampling uses Philox4x32-10 keyed
+ * by `seed`; temperature scales both the target's and the draft's logits.  Default: greedy. */
+swift_status swift_set_sampling(swift_ctx* ctx, int32_t mode, float temperature, uint64_t seed);
+
+/*
+ * The primitive under all three forms of the forward: M = n_rows new rows at positions
+ * pos0 .. pos0+M-1 run through the sub-layers not in `skip_mask` (NULL = full model); every row
+ * attends to cached positions [0, pos0) and causally to the new rows.  K,V of the new rows are
+ * stored for non-skipped attention sub-layers when write_kv != 0 (positions beyond the committed
+ * length stay uncommitted).  `logits_host` (may be NULL) receives n_rows*vocab fp32 values,
+ * `argmax_host` (may be NULL) n_rows token ids (lowest id on ties).  pos0 <= committed length,
+ * n_rows may exceed SWIFT_MAX_ROWS (processed in row chunks).  `tokens_host`: int32[n_rows].
+ */
+swift_status swift_forward_rows(swift_ctx* ctx, const int32_t* tokens_host, int32_t n_rows, int32_t pos0,
+                                const uint8_t* skip_mask_host, int32_t write_kv, float* logits_host,
+                                int32_t* argmax_host);
+
+/* Full model over the prompt (n >= 1 tokens); caches K,V for [0, n); *first_token_host = the pending
+ * token t* (argmax of the last row, or a draw from its softmax in sampling mode).  Resets the context. */
+swift_status swift_prefill(swift_ctx* ctx, const int32_t* tokens_host, int32_t n, int32_t* first_token_host);
+
+/* Replaces the pending token t* (teacher forcing: lets a caller that follows a reference sequence
+ * resynchronise after a legitimate tie-break difference) and, when rounds_done >= 0, the number of
+ * rounds completed so far (round r draws its random numbers at Philox counter word 0 = r, counted
+ * from 1 after prefill).  Needs a prefilled context, no open round. */
+swift_status swift_set_pending(swift_ctx* ctx, int32_t token, int32_t rounds_done);
+
+/*
+ * Drafting (Section 4.2, Eq. 4): up to max_k autoregressive steps of the layer-skipped model,
+ * starting from the pending token at position n; token feedback and the early-stop test
+ * (confidence p_j = max softmax < stop_conf; that token is kept) stay on the device.  Outputs:
+ * tokens_host[max_k], conf_host[max_k] (either may be NULL), *k_host = number drafted.
+ * max_k = 0 is allowed (an empty draft).  Opens a round.
+ */
+swift_status swift_draft(swift_ctx* ctx, const uint8_t* skip_mask_host, int32_t max_k, float stop_conf,
+                         int32_t* tokens_host, float* conf_host, int32_t* k_host);
+
+/*
+ * Parallel verification (Section 3.1): the full model on rows [t*, y'_1..y'_k] at positions n..n+k,
+ * writing K,V of every layer there (this fills the layers the draft skipped).  tokens_host = k draft
+ * tokens, or NULL to verify what the last swift_draft produced (k is then ignored).  Outputs
+ * (each may be NULL): target_argmax_host[k+1], logits_host[(k+1)*vocab].
+ */
+swift_status swift_verify(swift_ctx* ctx, const int32_t* tokens_host, int32_t k, int32_t* target_argmax_host,
+                          float* logits_host);
+
+/*
+ * Acceptance + KV rollback.  Greedy: a = longest prefix of drafts equal to the target's argmax,
+ * next token = target argmax of row a.  Sampling: accept y'_j while u_j * q_j(y'_j) < p_j(y'_j);
+ * on the first rejection the next token is drawn from max(0, p_j - q_j) renormalised, after k
+ * acceptances from p_{k+1}.  Then n <- n + a + 1 and the next token becomes pending.  Closes the round.
+ */
+swift_status swift_accept(swift_ctx* ctx, int32_t* n_accepted_host, int32_t* next_token_host);
+
+/*
+ * Scores C candidate skip sets (Eq. 2-3): each candidate re-predicts the last gamma generated tokens
+ * from their predecessors, reading the prefix K,V from the target's cache and keeping its own window
+ * K,V in scratch pages.  matchness_host[C] = matches / gamma.  masks_host: uint8[C][2*n_blocks].
+ * Needs gamma generated tokens (gamma <= tokens generated so far, gamma <= 128).
+ */
+swift_status swift_score_skipsets(swift_ctx* ctx, const uint8_t* masks_host, int32_t C, int32_t gamma,
+                                  float* matchness_host);
+
+typedef struct {
+    int32_t max_new;        /* tokens to emit (exactly; there is no end-of-sequence token) */
+    int32_t max_draft;      /* N_D */
+    float stop_conf;        /* epsilon; 0 disables early stopping */
+    int32_t vanilla;        /* 1 = plain autoregressive decoding of the full model (the baseline) */
+    /* on-the-fly optimisation (Section 4.1); n_opt_rounds = 0 keeps skip_mask fixed */
+    int32_t gamma, n_candidates, n_opt_rounds;
+    float stop_matchness;
+    const uint8_t* skip_mask;       /* host, [2*n_blocks]: the (initial) draft skip set */
+    const uint8_t* candidate_masks; /* host, [n_opt_rounds][n_candidates][2*n_blocks] or NULL */
+} swift_gen_params;
+
+typedef struct {
+    int32_t tokens, rounds, drafted, accepted, opt_rounds, reserved;
+    float best_matchness;
+    float ms_prefill, ms_decode, ms_draft, ms_verify, ms_score; /* CUDA-event times on the stream */
+    double bytes_draft, bytes_verify;  /* algorithmic HBM bytes of all draft / verify forwards */
+    int64_t kernel_launches;           /* kernels enqueued by the whole call */
+} swift_stats;
+
+/* prefill + rounds until max_new tokens are out.  out_tokens_host[max_new]; *n_out_host = max_new.
+ * `trace_host` (may be NULL) receives per round 4 int32: n_start, k, a, next_token (capacity
+ * max_new rounds).  stats may be NULL. */
+swift_status swift_generate(swift_ctx* ctx, const swift_gen_params* params, const int32_t* prompt_host,
+                            int32_t n_prompt, int32_t* out_tokens_host, int32_t* n_out_host,
+                            int32_t* trace_host, swift_stats* stats);
+
+/* Introspection used by tests and the benchmark. */
+int32_t swift_committed_length(const swift_ctx* ctx);               /* n; -1 if ctx is NULL */
+int64_t swift_launch_count(const swift_ctx* ctx);                   /* kernels enqueued since load */
+double swift_forward_bytes(const swift_ctx* ctx, const uint8_t* skip_mask_host, int32_t n_rows,
+                           int32_t n_context); /* algorithmic HBM bytes of one forward */
+/* Times `iters` back-to-back launches of one weight-streaming GEMM of the walk (which: 0 fused QKV,
+ * 1 o_proj, 2 fused gate/up, 3 down, 4 output head) with n_rows rows, cycling over the blocks' weights
+ * so that successive launches read different memory.  Outputs the average CUDA-event time per launch
+ * on the stream and the weight bytes one launch streams.  Clobbers the workspace of an open round. */
+swift_status swift_time_gemm(swift_ctx* ctx, int32_t which, int32_t n_rows, int32_t iters,
+                             float* ms_per_launch_host, double* bytes_per_launch_host);
+/* Copies K (which=0) or V (which=1) of `block` for positions [pos0, pos0+count) to host as fp32
+ * [count][n_kv_heads][head_dim]. */
+swift_status swift_read_kv(swift_ctx* ctx, int32_t block, int32_t which, int32_t pos0, int32_t count,
+                           float* out_host);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* SWIFT_H */

@@ -214,12 +214,12 @@ class Oracle:
         return logits
 
     def draft(self, z: Sequence[int], max_k: int, stop_conf: float = 0.0,
-              sampler=None) -> Tuple[List[int], List[float], List[torch.Tensor]]:
+              sampler=None, temperature: float = 1.0) -> Tuple[List[int], List[float], List[torch.Tensor]]:
         """Autoregressive drafting with the layer-skipped model (Eq. 4) and early stopping.
 
         Step j feeds t* (j = 1) or y'_{j-1} at position n+j-1.  y'_j = argmax of the draft logits,
         p_j = max softmax (T = 1).  The token that falls below epsilon is kept, then drafting stops.
-        With `sampler(j, probs) -> token`, y'_j is drawn from q_j = softmax(draft logits) instead.
+        With `sampler(j, q_j) -> token`, y'_j is drawn from q_j = softmax(draft logits / T) instead.
         Returns (draft tokens, confidences, draft logits rows).
         """
         toks, confs, rows = [], [], []
@@ -227,7 +227,10 @@ class Oracle:
         for j in range(1, max_k + 1):
             logit = self.forward_rows([inp], self.n + j - 1, z)[0]
             prob = torch.softmax(logit.to(torch.float64), dim=-1)
-            y = argmax_lowest(logit) if sampler is None else int(sampler(j, prob))
+            if sampler is None:
+                y = argmax_lowest(logit)
+            else:
+                y = int(sampler(j, torch.softmax(logit.to(torch.float64) / temperature, dim=-1)))
             toks.append(y)
             confs.append(float(prob.max()))
             rows.append(logit)
@@ -380,7 +383,7 @@ def swift_generate(o: Oracle, prompt: Sequence[int], z0: Sequence[int], gp: GenP
         r += 1
         remaining = gp.max_new - (len(o.tokens) - n_prompt)
         scores = None
-        if optimising and len(o.tokens) - n_prompt > gp.gamma and candidates is not None:
+        if optimising and len(o.tokens) - n_prompt >= gp.gamma and candidates is not None:
             masks = candidates(opt_rounds)
             scores, _ = o.score_skipsets(masks, gp.gamma)
             c_best = max(range(len(scores)), key=lambda c: (scores[c], -c))
@@ -396,7 +399,7 @@ def swift_generate(o: Oracle, prompt: Sequence[int], z0: Sequence[int], gp: GenP
                 def sampler(j, prob, _r=r):
                     q_rows.append(prob)
                     return categorical(prob, uniform(gp.rng_seed, _r, j, DRAW_DRAFT))[0]
-                d_tok, d_conf, d_rows = o.draft(z, k_max, gp.stop_conf, sampler)
+                d_tok, d_conf, d_rows = o.draft(z, k_max, gp.stop_conf, sampler, gp.temperature)
             else:
                 d_tok, d_conf, d_rows = o.draft(z, k_max, gp.stop_conf)
         else:

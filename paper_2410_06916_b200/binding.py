@@ -1,0 +1,306 @@
+"""ctypes binding of include/swift.h.  Argument marshalling only: every step of the decoding path
+runs inside the CUDA library; torch supplies device memory and the stream.  There is no fallback:
+if the library cannot be built or loaded, importing callers get an exception."""
+from __future__ import annotations
+
+import ctypes as C
+import os
+from dataclasses import dataclass
+from typing import Iterable, List, Optional, Sequence, Tuple
+
+import numpy as np
+import torch
+
+from . import build as _build
+
+MAX_ROWS = 16
+_KINDS = {"embed": 0, "lm_head": 1, "final_norm": 2, "wq": 3, "wk": 4, "wv": 5, "wo": 6, "wgate": 7,
+          "wup": 8, "wdown": 9, "attn_norm": 10, "mlp_norm": 11}
+_STATUS = {0: "OK", 1: "EINVAL", 2: "ESTATE", 3: "ECAPACITY", 4: "ECUDA", 5: "ETIMEOUT", 6: "EUNSUPPORTED"}
+
+
+class SwiftError(RuntimeError):
+    def __init__(self, status: int, message: str):
+        super().__init__(f"SWIFT_{_STATUS.get(status, status)}: {message}")
+        self.status = status
+
+
+class _Desc(C.Structure):
+    _fields_ = [(n, C.c_int32) for n in ("n_blocks", "d_model", "n_heads", "n_kv_heads", "head_dim", "ffn", "vocab",
+                                         "dtype")] + \
+               [("rope_theta", C.c_float), ("rms_eps", C.c_float)] + \
+               [(n, C.c_int32) for n in ("max_positions", "page_size", "max_draft", "reserved")]
+
+
+class _DevBuf(C.Structure):
+    _fields_ = [("dptr", C.c_void_p), ("bytes", C.c_size_t)]
+
+
+class _GenParams(C.Structure):
+    _fields_ = [("max_new", C.c_int32), ("max_draft", C.c_int32), ("stop_conf", C.c_float), ("vanilla", C.c_int32),
+                ("gamma", C.c_int32), ("n_candidates", C.c_int32), ("n_opt_rounds", C.c_int32),
+                ("stop_matchness", C.c_float), ("skip_mask", C.c_void_p), ("candidate_masks", C.c_void_p)]
+
+
+class _Stats(C.Structure):
+    _fields_ = [(n, C.c_int32) for n in ("tokens", "rounds", "drafted", "accepted", "opt_rounds", "reserved")] + \
+               [(n, C.c_float) for n in ("best_matchness", "ms_prefill", "ms_decode", "ms_draft", "ms_verify", "ms_score")] + \
+               [("bytes_draft", C.c_double), ("bytes_verify", C.c_double), ("kernel_launches", C.c_int64)]
+
+
+# every symbol include/swift.h declares
+SYMBOLS = ("swift_weights_bytes", "swift_kv_bytes", "swift_workspace_bytes", "swift_load", "swift_free",
+           "swift_last_error", "swift_pack_tensor", "swift_set_sampling", "swift_forward_rows", "swift_prefill",
+           "swift_set_pending", "swift_draft", "swift_verify", "swift_accept", "swift_score_skipsets", "swift_generate",
+           "swift_committed_length", "swift_launch_count", "swift_forward_bytes", "swift_read_kv", "swift_time_gemm")
+
+_lib = None
+
+
+def load_library(path: Optional[str] = None) -> C.CDLL:
+    """Builds (if stale) and loads libswift_b200.so; raises if that is not possible."""
+    global _lib
+    if _lib is not None and path is None:
+        return _lib
+    p = path or _build.build()
+    lib = C.CDLL(p)
+    vp, i32, u64, f32 = C.c_void_p, C.c_int32, C.c_uint64, C.c_float
+    for name in ("swift_weights_bytes", "swift_kv_bytes", "swift_workspace_bytes"):
+        getattr(lib, name).argtypes = [C.POINTER(_Desc)]
+        getattr(lib, name).restype = C.c_size_t
+    lib.swift_load.argtypes = [C.POINTER(_Desc), _DevBuf, _DevBuf, _DevBuf, vp, C.POINTER(vp)]
+    lib.swift_free.argtypes = [vp]
+    lib.swift_last_error.argtypes = [vp]
+    lib.swift_last_error.restype = C.c_char_p
+    lib.swift_pack_tensor.argtypes = [vp, i32, i32, vp, C.c_size_t]
+    lib.swift_set_sampling.argtypes = [vp, i32, f32, u64]
+    lib.swift_forward_rows.argtypes = [vp, vp, i32, i32, vp, i32, vp, vp]
+    lib.swift_prefill.argtypes = [vp, vp, i32, vp]
+    lib.swift_set_pending.argtypes = [vp, i32, i32]
+    lib.swift_draft.argtypes = [vp, vp, i32, f32, vp, vp, vp]
+    lib.swift_verify.argtypes = [vp, vp, i32, vp, vp]
+    lib.swift_accept.argtypes = [vp, vp, vp]
+    lib.swift_score_skipsets.argtypes = [vp, vp, i32, i32, vp]
+    lib.swift_generate.argtypes = [vp, C.POINTER(_GenParams), vp, i32, vp, vp, vp, C.POINTER(_Stats)]
+    lib.swift_committed_length.argtypes = [vp]
+    lib.swift_launch_count.argtypes = [vp]
+    lib.swift_launch_count.restype = C.c_int64
+    lib.swift_forward_bytes.argtypes = [vp, vp, i32, i32]
+    lib.swift_forward_bytes.restype = C.c_double
+    lib.swift_time_gemm.argtypes = [vp, i32, i32, i32, vp, vp]
+    lib.swift_read_kv.argtypes = [vp, i32, i32, i32, i32, vp]
+    for name in SYMBOLS:
+        fn = getattr(lib, name)          # AttributeError if a declared symbol is missing
+        if fn.restype is C.c_int:
+            fn.restype = C.c_int32
+    if path is None:
+        _lib = lib
+    return lib
+
+
+def lib() -> C.CDLL:
+    return load_library()
+
+
+@dataclass
+class GenParams:
+    max_new: int
+    max_draft: int = 8
+    stop_conf: float = 0.0
+    vanilla: bool = False
+    gamma: int = 32
+    n_opt_rounds: int = 0
+    stop_matchness: float = 0.95
+    skip_mask: Optional[np.ndarray] = None            # uint8 [2*n_blocks]
+    candidate_masks: Optional[np.ndarray] = None      # uint8 [n_opt_rounds, C, 2*n_blocks]
+
+
+@dataclass
+class GenStats:
+    tokens: int
+    rounds: int
+    drafted: int
+    accepted: int
+    opt_rounds: int
+    best_matchness: float
+    ms_prefill: float
+    ms_decode: float
+    ms_draft: float
+    ms_verify: float
+    ms_score: float
+    bytes_draft: float
+    bytes_verify: float
+    kernel_launches: int
+
+
+def _i32(a) -> np.ndarray:
+    return np.ascontiguousarray(np.asarray(a, dtype=np.int32))
+
+
+def _u8(a) -> np.ndarray:
+    return np.ascontiguousarray(np.asarray(a, dtype=np.uint8))
+
+
+def _ptr(a: Optional[np.ndarray]):
+    return None if a is None else a.ctypes.data_as(C.c_void_p)
+
+
+class SwiftModel:
+    """One model + KV cache + workspace on one GPU, driven through the C boundary."""
+
+    def __init__(self, cfg, max_positions: int, page_size: int = 16, max_draft: int = 15, device: str = "cuda:0"):
+        if not torch.cuda.is_available():
+            raise RuntimeError("paper_2410_06916_b200 needs a CUDA device (B200); there is no CPU path")
+        self._lib = lib()
+        self.cfg = cfg
+        self.device = torch.device(device)
+        max_positions = (max_positions + page_size - 1) // page_size * page_size
+        self.desc = _Desc(cfg.n_blocks, cfg.d_model, cfg.n_heads, cfg.n_kv_heads, cfg.head_dim, cfg.ffn, cfg.vocab,
+                          1 if cfg.dtype == "bf16" else 0, cfg.rope_theta, cfg.rms_eps, max_positions, page_size,
+                          max_draft, 0)
+        sizes = [self._lib.swift_weights_bytes(C.byref(self.desc)), self._lib.swift_kv_bytes(C.byref(self.desc)),
+                 self._lib.swift_workspace_bytes(C.byref(self.desc))]
+        if 0 in sizes:
+            raise SwiftError(1, "invalid model description")
+        self.ctx = C.c_void_p()
+        with torch.cuda.device(self.device):
+            self.stream = torch.cuda.Stream(device=self.device)
+            self._bufs = [torch.empty(s + 256, dtype=torch.uint8, device=self.device) for s in sizes]
+            devbufs = []
+            for b, s in zip(self._bufs, sizes):
+                p = (b.data_ptr() + 255) // 256 * 256
+                devbufs.append(_DevBuf(p, s))
+            st = self._lib.swift_load(C.byref(self.desc), *devbufs, C.c_void_p(self.stream.cuda_stream), C.byref(self.ctx))
+        if st != 0:
+            raise SwiftError(st, self._lib.swift_last_error(None).decode())
+        self.weight_bytes, self.kv_bytes, self.workspace_bytes = sizes
+        self.vocab, self.n_sub = cfg.vocab, 2 * cfg.n_blocks
+
+    # ------------------------------------------------------------------ plumbing
+    def _check(self, st: int):
+        if st != 0:
+            raise SwiftError(st, self._lib.swift_last_error(self.ctx).decode())
+
+    def close(self):
+        if getattr(self, "ctx", None) and self.ctx.value:
+            self._lib.swift_free(self.ctx)
+            self.ctx = C.c_void_p()
+            self._bufs = []
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+    def pack(self, name: str, block: int, t: torch.Tensor):
+        want = torch.float32 if name.endswith("norm") or self.cfg.dtype == "f32" else torch.bfloat16
+        t = t.detach().to("cpu").contiguous()
+        if t.dtype != want:
+            raise TypeError(f"{name}: expected {want}, got {t.dtype}")
+        with torch.cuda.device(self.device):
+            self._check(self._lib.swift_pack_tensor(self.ctx, _KINDS[name], block, C.c_void_p(t.data_ptr()),
+                                                    t.numel() * t.element_size()))
+
+    def load_weights(self, tensors: Iterable[Tuple[str, int, torch.Tensor]]):
+        for name, block, t in tensors:
+            self.pack(name, block, t)
+
+    def set_sampling(self, sampling: bool, temperature: float = 1.0, seed: int = 0):
+        self._check(self._lib.swift_set_sampling(self.ctx, 1 if sampling else 0, temperature, seed))
+
+    @property
+    def n(self) -> int:
+        return self._lib.swift_committed_length(self.ctx)
+
+    @property
+    def launches(self) -> int:
+        return self._lib.swift_launch_count(self.ctx)
+
+    def forward_bytes(self, skip_mask, n_rows: int, n_context: int) -> float:
+        m = None if skip_mask is None else _u8(skip_mask)
+        return self._lib.swift_forward_bytes(self.ctx, _ptr(m), n_rows, n_context)
+
+    # ------------------------------------------------------------------ the steps
+    def forward_rows(self, tokens: Sequence[int], pos0: int, skip_mask=None, write_kv: bool = True,
+                     want_logits: bool = True) -> Tuple[Optional[np.ndarray], np.ndarray]:
+        t = _i32(tokens)
+        m = None if skip_mask is None else _u8(skip_mask)
+        logits = np.empty((len(t), self.vocab), dtype=np.float32) if want_logits else None
+        am = np.empty(len(t), dtype=np.int32)
+        with torch.cuda.device(self.device):
+            self._check(self._lib.swift_forward_rows(self.ctx, _ptr(t), len(t), pos0, _ptr(m), 1 if write_kv else 0,
+                                                     _ptr(logits), _ptr(am)))
+        return logits, am
+
+    def prefill(self, tokens: Sequence[int]) -> int:
+        t = _i32(tokens)
+        first = C.c_int32()
+        with torch.cuda.device(self.device):
+            self._check(self._lib.swift_prefill(self.ctx, _ptr(t), len(t), C.byref(first)))
+        return first.value
+
+    def set_pending(self, token: int, rounds_done: int = -1):
+        self._check(self._lib.swift_set_pending(self.ctx, int(token), int(rounds_done)))
+
+    def draft(self, skip_mask, max_k: int, stop_conf: float = 0.0) -> Tuple[List[int], List[float]]:
+        m = _u8(skip_mask)
+        toks = np.zeros(max(max_k, 1), dtype=np.int32)
+        conf = np.zeros(max(max_k, 1), dtype=np.float32)
+        k = C.c_int32()
+        with torch.cuda.device(self.device):
+            self._check(self._lib.swift_draft(self.ctx, _ptr(m), max_k, stop_conf, _ptr(toks), _ptr(conf), C.byref(k)))
+        return toks[:k.value].tolist(), conf[:k.value].tolist()
+
+    def verify(self, tokens: Optional[Sequence[int]] = None, want_logits: bool = True):
+        t = None if tokens is None else _i32(tokens)
+        k = 0 if t is None else len(t)
+        am = np.zeros(MAX_ROWS, dtype=np.int32)
+        logits = np.empty((MAX_ROWS, self.vocab), dtype=np.float32) if want_logits else None
+        tp = None if t is None else (_ptr(t) if k > 0 else C.c_void_p(am.ctypes.data))  # non-null marks "tokens given"
+        with torch.cuda.device(self.device):
+            self._check(self._lib.swift_verify(self.ctx, tp, k, _ptr(am), _ptr(logits)))
+        return am, logits
+
+    def accept(self) -> Tuple[int, int]:
+        a, nxt = C.c_int32(), C.c_int32()
+        with torch.cuda.device(self.device):
+            self._check(self._lib.swift_accept(self.ctx, C.byref(a), C.byref(nxt)))
+        return a.value, nxt.value
+
+    def score_skipsets(self, masks, gamma: int) -> np.ndarray:
+        m = _u8(masks).reshape(-1, self.n_sub)
+        out = np.zeros(m.shape[0], dtype=np.float32)
+        with torch.cuda.device(self.device):
+            self._check(self._lib.swift_score_skipsets(self.ctx, _ptr(m), m.shape[0], gamma, _ptr(out)))
+        return out
+
+    def generate(self, prompt: Sequence[int], gp: GenParams) -> Tuple[List[int], GenStats, np.ndarray]:
+        p = _i32(prompt)
+        skip = None if gp.skip_mask is None else _u8(gp.skip_mask)
+        cands = None if gp.candidate_masks is None else _u8(gp.candidate_masks)
+        n_cand = 0 if cands is None else cands.reshape(gp.n_opt_rounds, -1, self.n_sub).shape[1]
+        cp = _GenParams(gp.max_new, gp.max_draft, gp.stop_conf, 1 if gp.vanilla else 0, gp.gamma, n_cand,
+                        gp.n_opt_rounds if cands is not None else 0, gp.stop_matchness, _ptr(skip), _ptr(cands))
+        out = np.zeros(gp.max_new, dtype=np.int32)
+        trace = np.zeros((gp.max_new, 4), dtype=np.int32)
+        n_out = C.c_int32()
+        st = _Stats()
+        with torch.cuda.device(self.device):
+            self._check(self._lib.swift_generate(self.ctx, C.byref(cp), _ptr(p), len(p), _ptr(out), C.byref(n_out),
+                                                 _ptr(trace), C.byref(st)))
+        stats = GenStats(**{f: getattr(st, f) for f in GenStats.__dataclass_fields__})
+        return out[:n_out.value].tolist(), stats, trace[:stats.rounds]
+
+    def time_gemm(self, which: int, n_rows: int, iters: int) -> Tuple[float, float]:
+        """(ms per launch, weight bytes per launch) of one weight-streaming GEMM of the walk."""
+        ms, nbytes = C.c_float(), C.c_double()
+        with torch.cuda.device(self.device):
+            self._check(self._lib.swift_time_gemm(self.ctx, which, n_rows, iters, C.byref(ms), C.byref(nbytes)))
+        return ms.value, nbytes.value
+
+    def read_kv(self, block: int, which: int, pos0: int, count: int) -> np.ndarray:
+        out = np.empty((count, self.cfg.n_kv_heads, self.cfg.head_dim), dtype=np.float32)
+        with torch.cuda.device(self.device):
+            self._check(self._lib.swift_read_kv(self.ctx, block, which, pos0, count, _ptr(out)))
+        return out

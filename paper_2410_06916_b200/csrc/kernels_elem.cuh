@@ -1,0 +1,189 @@
+// Element-wise and per-row kernels of the decoder walk: state set-up, embedding gather,
+// residual-add + RMSNorm, RoPE + KV append, SwiGLU.  All of them take their row count and base
+// position from the device-resident DevState and do nothing when it holds zero rows.
+#pragma once
+#include "common.cuh"
+
+namespace swk {
+
+// ------------------------------------------------------------------------------ state
+// Generic forward chunk: tokens were copied into st->row_tok beforehand.
+__global__ void set_rows_kernel(DevState* st, int pos0, int n_rows)
+{
+    st->pos0 = pos0;
+    st->n_rows = n_rows;
+    st->tok_off = 0;
+}
+
+// Start of a round: pending token into slot 0, drafting armed.
+__global__ void begin_round_kernel(DevState* st, int pending_token, int use_given_token)
+{
+    if (use_given_token) st->draft_tok[0] = pending_token;
+    st->active = 1;
+    st->n_drafted = 0;
+    st->n_accepted = 0;
+}
+
+// Draft step j (1-based): one row, input y'_{j-1} (slot j-1), position n + j - 1; a stopped draft
+// leaves zero rows so that the step's kernels fall through.
+__global__ void begin_draft_step_kernel(DevState* st, int n, int j)
+{
+    if (st->active) {
+        st->pos0 = n + j - 1;
+        st->n_rows = 1;
+        st->tok_off = j - 1;
+    } else {
+        st->n_rows = 0;
+    }
+}
+
+// Verification: rows [t*, y'_1..y'_k] with k taken from the device (or forced by the host).
+__global__ void begin_verify_kernel(DevState* st, int n, int forced_k)
+{
+    if (forced_k >= 0) st->n_drafted = forced_k;
+    st->pos0 = n;
+    st->n_rows = st->n_drafted + 1;
+    st->tok_off = 0;
+}
+
+// Precomputed rotary table: cs[pos][i] = (cos, sin)(pos * theta^(-2i/dh)), evaluated in double.
+__global__ void rope_table_kernel(float2* cs, int max_positions, int half, double theta)
+{
+    const int idx = blockIdx.x * blockDim.x + threadIdx.x;
+    if (idx >= max_positions * half) return;
+    const int pos = idx / half, i = idx % half;
+    const double inv_freq = pow(theta, -(double)i / (double)half);
+    double s, c;
+    sincos((double)pos * inv_freq, &s, &c);
+    cs[idx] = make_float2((float)c, (float)s);
+}
+
+// Copies whole KV pages (all blocks) src_page -> dst_page: copy-on-write for candidate scoring.
+__global__ void page_copy_kernel(uint4* pool, size_t page_vec16, int src_page, int dst_page)
+{
+    const uint4* s = pool + (size_t)src_page * page_vec16;
+    uint4* d = pool + (size_t)dst_page * page_vec16;
+    for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < page_vec16; i += (size_t)gridDim.x * blockDim.x)
+        d[i] = s[i];
+}
+
+// Gathers K or V of one block for positions [pos0, pos0+count) into fp32 [count][Hkv][dh] (inspection).
+template <typename T>
+__global__ void kv_read_kernel(const T* __restrict__ kv_pool, const int* __restrict__ page_table, KvLayout L, int block,
+                               int which, int pos0, int count, float* __restrict__ out)
+{
+    const size_t total = (size_t)count * L.n_kv_heads * L.head_dim;
+    for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += (size_t)gridDim.x * blockDim.x) {
+        const int d = (int)(i % L.head_dim);
+        const int hk = (int)((i / L.head_dim) % L.n_kv_heads);
+        const int pos = pos0 + (int)(i / ((size_t)L.head_dim * L.n_kv_heads));
+        out[i] = to_float(kv_pool[L.offset(page_table[pos >> L.page_shift], block, which, hk, pos & (L.page_size - 1)) + d]);
+    }
+}
+
+// ------------------------------------------------------------------------------ embedding
+template <typename T>
+__global__ void embed_kernel(DevState* st, const int* __restrict__ toks, const T* __restrict__ embed,
+                             float* __restrict__ h, int d, int vocab)
+{
+    const int r = blockIdx.x;
+    if (r >= st->n_rows) return;
+    int tok = toks[st->tok_off + r];
+    if (tok < 0 || tok >= vocab) {
+        if (threadIdx.x == 0) st->error = 1;
+        tok = 0;
+    }
+    const T* src = embed + (size_t)tok * d;
+    for (int i = threadIdx.x; i < d; i += blockDim.x) h[(size_t)r * d + i] = to_float(src[i]);
+}
+
+// ------------------------------------------------------------------------------ residual + RMSNorm
+// h[r,:] += sum_s part[s][r][:]  (the pending output of the previous residual branch, split-K
+// partial sums added in split order), then x[r,:] = h * rsqrt(mean(h^2) + eps) * g.
+template <typename T>
+__global__ void __launch_bounds__(512) resid_norm_kernel(const DevState* st, float* __restrict__ h,
+                                                         const float* __restrict__ part, int n_split,
+                                                         size_t split_stride, const float* __restrict__ gain,
+                                                         T* __restrict__ x, int d, float eps)
+{
+    __shared__ float red[33];
+    const int r = blockIdx.x;
+    if (r >= st->n_rows) return;
+    float* hr = h + (size_t)r * d;
+    float ss = 0.f;
+    for (int i = threadIdx.x; i < d; i += blockDim.x) {
+        float v = hr[i];
+        for (int s = 0; s < n_split; ++s) v += part[s * split_stride + (size_t)r * d + i];
+        hr[i] = v;
+        ss += v * v;
+    }
+    const float total = block_sum(ss, red);
+    const float rstd = rsqrtf(total / (float)d + eps);
+    for (int i = threadIdx.x; i < d; i += blockDim.x) store_val(&x[(size_t)r * d + i], hr[i] * rstd * gain[i]);
+}
+
+// ------------------------------------------------------------------------------ RoPE + KV append
+// Sums the fused QKV projection's split-K partials, rotates q and k (rotate-half pairing: dim i
+// with i + dh/2) by the row's absolute position, writes q (fp32) for the attention kernel and k, v
+// into the paged cache.  grid = (rows, H + 2*Hkv), block = dh/2 threads.
+template <typename T>
+__global__ void qkv_post_kernel(const DevState* st, const float* __restrict__ part, int n_split, size_t split_stride,
+                                int n_qkv, float* __restrict__ q_out, T* __restrict__ kv_pool,
+                                const int* __restrict__ page_table, KvLayout L, int block, int n_heads,
+                                const float2* __restrict__ rope_cs, int max_positions)
+{
+    const int r = blockIdx.x;
+    if (r >= st->n_rows) return;
+    const int head = blockIdx.y, half = L.head_dim >> 1, i = threadIdx.x;
+    const int pos = st->pos0 + r;
+    if (pos >= max_positions) return;
+    const size_t col = (size_t)head * L.head_dim + i;
+    float a = 0.f, b = 0.f;
+    for (int s = 0; s < n_split; ++s) {
+        const float* p = part + s * split_stride + (size_t)r * n_qkv + col;
+        a += p[0];
+        b += p[half];
+    }
+    const float2 cs = rope_cs[(size_t)pos * half + i];
+    if (head < n_heads) {
+        float* q = q_out + (size_t)r * n_heads * L.head_dim + col;
+        q[0] = a * cs.x - b * cs.y;
+        q[half] = b * cs.x + a * cs.y;
+    } else {
+        const int hk = head - n_heads;
+        const int kv = hk >= L.n_kv_heads ? 1 : 0;
+        const int kh = kv ? hk - L.n_kv_heads : hk;
+        const int page = page_table[pos >> L.page_shift];
+        T* dst = kv_pool + L.offset(page, block, kv, kh, pos & (L.page_size - 1)) + i;
+        if (kv == 0) {
+            store_val(dst, a * cs.x - b * cs.y);
+            store_val(dst + half, b * cs.x + a * cs.y);
+        } else {
+            store_val(dst, a);
+            store_val(dst + half, b);
+        }
+    }
+}
+
+// ------------------------------------------------------------------------------ SwiGLU
+// act[r][i] = silu(gate_i) * up_i from the fused gate/up projection, whose output columns are
+// interleaved in groups of 16: [g0..g15, u0..u15, g16..g31, u16..u31, ...].
+template <typename T>
+__global__ void swiglu_kernel(const DevState* st, const float* __restrict__ part, int n_split, size_t split_stride,
+                              T* __restrict__ act, int ffn)
+{
+    const int r = blockIdx.y;
+    if (r >= st->n_rows) return;
+    const int i = blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= ffn) return;
+    const size_t gi = (size_t)(i >> 4) * 32 + (i & 15);
+    float g = 0.f, u = 0.f;
+    for (int s = 0; s < n_split; ++s) {
+        const float* p = part + s * split_stride + (size_t)r * 2 * ffn;
+        g += p[gi];
+        u += p[gi + 16];
+    }
+    store_val(&act[(size_t)r * ffn + i], g / (1.f + expf(-g)) * u);
+}
+
+} // namespace swk

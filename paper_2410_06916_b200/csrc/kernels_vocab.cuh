@@ -1,0 +1,247 @@
+// Vocabulary-wide kernels: logits reduction + argmax + softmax statistics (+ draft sampling), the
+// acceptance step (greedy prefix match or speculative sampling), and the matchness count.
+#pragma once
+#include "common.cuh"
+
+namespace swk {
+
+constexpr int VOCAB_THREADS = 1024;
+
+struct ArgMax { float v; int i; };
+__device__ __forceinline__ ArgMax better(ArgMax a, ArgMax b)   // larger value; lowest index on ties
+{
+    return (b.v > a.v || (b.v == a.v && b.i < a.i)) ? b : a;
+}
+
+// Block-wide inverse-CDF draw in index order: smallest i with sum_{i' <= i} w(i') > u * total.
+// Thread t owns the contiguous index range [t*seg, (t+1)*seg); its bracket on the running-sum axis
+// is [incl(t-1), incl(t)) with both ends read from the same shared array, so the brackets tile
+// [0, total) without gaps whatever the rounding.  `sh` is shared scratch of VOCAB_THREADS + 72
+// floats.  Every thread returns the same index.  Must be called by all threads of the block.
+template <typename WeightFn>
+__device__ int block_categorical(WeightFn w, int n, float u, float* sh)
+{
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int seg = (n + VOCAB_THREADS - 1) / VOCAB_THREADS;
+    const int b = min(tid * seg, n), e = min(b + seg, n);
+    float* sh_incl = sh;                                        // [VOCAB_THREADS]
+    float* sh_wtot = sh + VOCAB_THREADS;                        // [32]
+    int* result = reinterpret_cast<int*>(sh + VOCAB_THREADS + 64);
+    float local = 0.f;
+    for (int i = b; i < e; ++i) local += w(i);
+    float incl = local;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+        const float t = __shfl_up_sync(0xFFFFFFFFu, incl, o);
+        if (lane >= o) incl += t;
+    }
+    __syncthreads();                                            // scratch may still be in use by the caller
+    if (lane == 31) sh_wtot[warp] = incl;
+    if (tid == 0) *result = 0x7FFFFFFF;
+    __syncthreads();
+    float warp_off = 0.f;
+    for (int ww = 0; ww < warp; ++ww) warp_off += sh_wtot[ww];  // sequential, identical for a whole warp
+    incl += warp_off;
+    sh_incl[tid] = incl;
+    __syncthreads();
+    const float excl = tid > 0 ? sh_incl[tid - 1] : 0.f;
+    const float total = sh_incl[VOCAB_THREADS - 1];
+    const float target = u * total;
+    if (excl <= target && target < incl) {
+        float c = excl;
+        int pick = -1, last_pos = -1;
+        for (int i = b; i < e; ++i) {
+            const float wi = w(i);
+            if (wi > 0.f) last_pos = i;
+            c += wi;
+            if (c > target) { pick = i; break; }
+        }
+        if (pick < 0) pick = last_pos;                          // rounding at the segment's end
+        if (pick >= 0) atomicMin(result, pick);
+    }
+    __syncthreads();
+    if (*result == 0x7FFFFFFF) {
+        // nothing bracketed the target (u * total rounded up to the total, or an all-zero row):
+        // take the last index that carries weight
+        int last = -1;
+        for (int i = b; i < e; ++i) if (w(i) > 0.f) last = i;
+        int* result2 = result + 1;
+        if (tid == 0) *result2 = -1;
+        __syncthreads();
+        if (last >= 0) atomicMax(result2, last);
+        __syncthreads();
+        const int out2 = *result2;
+        __syncthreads();
+        return out2 < 0 ? 0 : out2;
+    }
+    const int out = *result;
+    __syncthreads();
+    return out;
+}
+
+// One CTA per row.  logits[r][i] = sum_s part[s][r][i]; argmax (lowest id on ties), row max,
+// sum exp((l-max)/T); confidence p = max softmax at T = 1.
+// VOCAB_DRAFT (one row, draft step j): y'_j = argmax, or a draw from q_j = softmax(l/T) whose
+// probabilities are kept in q_rows[j-1][:]; records the token and its confidence, and disarms
+// drafting when the confidence is below stop_conf.
+__global__ void __launch_bounds__(VOCAB_THREADS)
+vocab_kernel(DevState* st, const float* __restrict__ part, int n_split, size_t split_stride,
+             float* __restrict__ logits, int vocab, float inv_temp, int mode, int draft_j, float stop_conf,
+             int sampling, uint64_t seed, uint32_t round, float* __restrict__ q_rows)
+{
+    __shared__ float sh[VOCAB_THREADS + 72];
+    __shared__ ArgMax sh_am[32];
+    const int r = blockIdx.x;
+    if (r >= st->n_rows) return;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    float* lrow = logits + (size_t)r * vocab;
+
+    ArgMax am{-INFINITY, 0x7FFFFFFF};
+    for (int i = tid; i < vocab; i += VOCAB_THREADS) {
+        float v = 0.f;
+        for (int s = 0; s < n_split; ++s) v += part[s * split_stride + (size_t)r * vocab + i];
+        lrow[i] = v;
+        am = better(am, ArgMax{v, i});
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+        ArgMax t{__shfl_xor_sync(0xFFFFFFFFu, am.v, o), __shfl_xor_sync(0xFFFFFFFFu, am.i, o)};
+        am = better(am, t);
+    }
+    if (lane == 0) sh_am[warp] = am;
+    __syncthreads();
+    if (warp == 0) {
+        ArgMax t = sh_am[lane];
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) {
+            ArgMax t2{__shfl_xor_sync(0xFFFFFFFFu, t.v, o), __shfl_xor_sync(0xFFFFFFFFu, t.i, o)};
+            t = better(t, t2);
+        }
+        if (lane == 0) sh_am[0] = t;
+    }
+    __syncthreads();
+    am = sh_am[0];
+    __syncthreads();
+
+    float s1 = 0.f, sT = 0.f;
+    for (int i = tid; i < vocab; i += VOCAB_THREADS) {
+        const float dlt = lrow[i] - am.v;
+        s1 += expf(dlt);
+        sT += expf(dlt * inv_temp);
+    }
+    s1 = block_sum(s1, sh);
+    sT = block_sum(sT, sh);
+    const float conf = 1.f / s1;
+    if (tid == 0) {
+        st->argmax[r] = am.i;
+        st->row_max[r] = am.v;
+        st->row_sum[r] = sT;
+    }
+    if (mode != VOCAB_DRAFT || r != 0) return;
+
+    int y = am.i;
+    if (sampling) {
+        float* qrow = q_rows + (size_t)(draft_j - 1) * vocab;
+        const float inv_sum = 1.f / sT;
+        for (int i = tid; i < vocab; i += VOCAB_THREADS) qrow[i] = expf((lrow[i] - am.v) * inv_temp) * inv_sum;
+        __syncthreads();
+        const float u = philox_uniform(seed, round, (uint32_t)draft_j, DRAW_DRAFT);
+        y = block_categorical([&](int i) { return qrow[i]; }, vocab, u, sh);
+    }
+    if (tid == 0) {
+        st->draft_tok[draft_j] = y;
+        st->conf[draft_j - 1] = conf;
+        st->n_drafted = draft_j;
+        if (conf < stop_conf) st->active = 0;
+    }
+}
+
+// Acceptance over the k = st->n_drafted drafts of the round, one CTA.  `logits` holds the k+1
+// target rows, st->argmax / row_max / row_sum their statistics, q_rows the draft distributions.
+// Writes n_accepted, next_token, and makes next_token the pending token (draft_tok[0]).
+__global__ void __launch_bounds__(VOCAB_THREADS)
+accept_kernel(DevState* st, const float* __restrict__ logits, const float* __restrict__ q_rows, int vocab,
+              int sampling, float inv_temp, uint64_t seed, uint32_t round)
+{
+    __shared__ float sh[VOCAB_THREADS + 72];
+    __shared__ int sh_a, sh_rejected;
+    const int k = st->n_drafted;
+    const int tid = threadIdx.x;
+    if (!sampling) {
+        if (tid == 0) {
+            int a = 0;
+            while (a < k && st->draft_tok[a + 1] == st->argmax[a]) ++a;
+            st->n_accepted = a;
+            st->next_token = st->argmax[a];
+            st->draft_tok[0] = st->argmax[a];
+        }
+        return;
+    }
+    if (tid == 0) {
+        int a = 0, rejected = 0;
+        for (int j = 1; j <= k; ++j) {
+            const int y = st->draft_tok[j];
+            const float p = expf((logits[(size_t)(j - 1) * vocab + y] - st->row_max[j - 1]) * inv_temp) / st->row_sum[j - 1];
+            const float q = q_rows[(size_t)(j - 1) * vocab + y];
+            const float u = philox_uniform(seed, round, (uint32_t)j, DRAW_ACCEPT);
+            if (!(u * q < p)) { rejected = 1; break; }
+            ++a;
+        }
+        sh_a = a;
+        sh_rejected = rejected;
+    }
+    __syncthreads();
+    const int a = sh_a, rejected = sh_rejected;
+    const float* lrow = logits + (size_t)a * vocab;          // target row j-1 with j = a+1
+    const float mx = st->row_max[a], inv_sum = 1.f / st->row_sum[a];
+    auto p_of = [&](int i) { return expf((lrow[i] - mx) * inv_temp) * inv_sum; };
+    int tok;
+    if (rejected) {
+        const float* qrow = q_rows + (size_t)a * vocab;
+        float mass = 0.f;
+        for (int i = tid; i < vocab; i += VOCAB_THREADS) mass += fmaxf(p_of(i) - qrow[i], 0.f);
+        mass = block_sum(mass, sh);
+        const float u = philox_uniform(seed, round, (uint32_t)(a + 1), DRAW_RESAMPLE);
+        if (mass > 0.f) tok = block_categorical([&](int i) { return fmaxf(p_of(i) - qrow[i], 0.f); }, vocab, u, sh);
+        else tok = block_categorical(p_of, vocab, u, sh);
+    } else {
+        const float u = philox_uniform(seed, round, (uint32_t)(k + 1), DRAW_BONUS);
+        tok = block_categorical(p_of, vocab, u, sh);
+    }
+    if (tid == 0) {
+        st->n_accepted = a;
+        st->next_token = tok;
+        st->draft_tok[0] = tok;
+    }
+}
+
+// Draws one token from softmax(row r / T) of the last forward (first token in sampling mode, and
+// vanilla sampling steps): counter (round, slot, DRAW_BONUS).
+__global__ void __launch_bounds__(VOCAB_THREADS)
+sample_row_kernel(DevState* st, const float* __restrict__ logits, int vocab, int row, float inv_temp,
+                  uint64_t seed, uint32_t round, uint32_t slot)
+{
+    __shared__ float sh[VOCAB_THREADS + 72];
+    const float* lrow = logits + (size_t)row * vocab;
+    const float mx = st->row_max[row];
+    const float u = philox_uniform(seed, round, slot, DRAW_BONUS);
+    const int tok = block_categorical([&](int i) { return expf((lrow[i] - mx) * inv_temp); }, vocab, u, sh);
+    if (threadIdx.x == 0) {
+        st->next_token = tok;
+        st->draft_tok[0] = tok;
+    }
+}
+
+// matchness numerator (Eq. 3): adds #(argmax[r] == truth[r]) over the rows of this chunk; the
+// running count is stored to *out after the candidate's last chunk.
+__global__ void match_count_kernel(DevState* st, const int* __restrict__ truth, int reset, int* out)
+{
+    if (threadIdx.x == 0) {
+        int c = reset ? 0 : st->match_count;
+        for (int r = 0; r < st->n_rows; ++r) c += (st->argmax[r] == truth[r]) ? 1 : 0;
+        st->match_count = c;
+        if (out) *out = c;
+    }
+}
+
+} // namespace swk

@@ -1,0 +1,992 @@
+// Host side of the SWIFT hot-path library: context, buffer carving, the sub-layer walk that
+// enqueues the kernels of one forward chunk, and the extern "C" entry points of include/swift.h.
+#include "../../include/swift.h"
+
+#include <cuda_runtime.h>
+
+#include <algorithm>
+#include <cstdarg>
+#include <cstdio>
+#include <cstring>
+#include <string>
+#include <vector>
+
+#include "common.cuh"
+#include "kernels_attn.cuh"
+#include "kernels_elem.cuh"
+#include "kernels_gemm_simt.cuh"
+#include "kernels_vocab.cuh"
+
+using namespace swk;
+
+namespace {
+
+thread_local std::string g_load_error;
+
+constexpr size_t ALIGN = 256;
+inline size_t align_up(size_t v, size_t a = ALIGN) { return (v + a - 1) / a * a; }
+inline int ceil_div(int a, int b) { return (a + b - 1) / b; }
+
+enum Phase { PH_LOADED = 0, PH_READY = 1, PH_DRAFTED = 2, PH_VERIFIED = 3 };
+
+struct GemmPlan { int S, Kc; };
+
+struct Carve {
+    size_t off = 0;
+    size_t take(size_t bytes) { size_t o = off; off = align_up(off + bytes); return o; }
+};
+
+// Offsets (bytes) of every tensor inside the weights buffer.
+struct WeightLayout {
+    size_t embed, lm_head, final_norm, total;
+    std::vector<size_t> wqkv, wo, wgu, wdown, attn_norm, mlp_norm;
+};
+
+struct WorkLayout {
+    size_t state, h, xn, xa, act, q, part, o_part, ml_part, logits, q_rows, rope, pt_main, pt_score, score_tok,
+        score_truth, score_out, total;
+    size_t part_floats;
+};
+
+} // namespace
+
+struct swift_ctx {
+    swift_model_desc d;
+    cudaStream_t stream;
+    int device;
+    size_t esize;
+    char* wbase; char* kvbase; char* ws;
+    WeightLayout wl;
+    WorkLayout kl;
+    KvLayout kv;
+    int n_pages_main, n_pages_scratch, max_splits;
+    // host-side state
+    int phase, n, pending, n_prompt, round, last_k, last_max_k;
+    bool round_open;
+    std::vector<int> hist;           // prompt + generated tokens, pending included
+    int mode; float temperature; uint64_t seed;
+    int64_t launches;
+    std::string err;
+    cudaEvent_t ev[8];
+};
+
+namespace {
+
+swift_status fail(swift_ctx* c, swift_status s, const char* fmt, ...)
+{
+    char buf[512];
+    va_list ap;
+    va_start(ap, fmt);
+    vsnprintf(buf, sizeof buf, fmt, ap);
+    va_end(ap);
+    if (c) c->err = buf; else g_load_error = buf;
+    return s;
+}
+
+#define CU(call)                                                                                   \
+    do {                                                                                           \
+        cudaError_t e_ = (call);                                                                   \
+        if (e_ != cudaSuccess)                                                                     \
+            return fail(ctx, SWIFT_ECUDA, "%s failed: %s (%s:%d)", #call, cudaGetErrorString(e_),  \
+                        __FILE__, __LINE__);                                                       \
+    } while (0)
+
+bool desc_ok(const swift_model_desc* d, std::string* why)
+{
+    auto bad = [&](const char* m) { if (why) *why = m; return false; };
+    if (!d) return bad("null desc");
+    if (d->n_blocks < 1 || d->d_model < 8 || d->n_heads < 1 || d->n_kv_heads < 1 || d->ffn < 16 || d->vocab < 2)
+        return bad("non-positive dimension");
+    if (d->dtype != SWIFT_F32 && d->dtype != SWIFT_BF16) return bad("dtype must be SWIFT_F32 or SWIFT_BF16");
+    if (d->n_heads % d->n_kv_heads) return bad("n_heads must be a multiple of n_kv_heads");
+    if (d->head_dim < 16 || d->head_dim > 256 || (d->head_dim & (d->head_dim - 1)))
+        return bad("head_dim must be a power of two in 16..256");
+    if (d->d_model % 8 || d->ffn % 16 || (d->n_heads * d->head_dim) % 8) return bad("d_model%8, ffn%16 required");
+    if (d->page_size < 8 || d->page_size > 128 || (d->page_size & (d->page_size - 1)))
+        return bad("page_size must be a power of two in 8..128");
+    if (d->max_positions < d->page_size || d->max_positions % d->page_size) return bad("max_positions must be a positive multiple of page_size");
+    if (d->max_draft < 0 || d->max_draft > SWIFT_MAX_ROWS - 1) return bad("max_draft must be in 0..15");
+    if (!(d->rope_theta > 1.f) || !(d->rms_eps >= 0.f)) return bad("rope_theta > 1 and rms_eps >= 0 required");
+    return true;
+}
+
+size_t esize_of(const swift_model_desc* d) { return d->dtype == SWIFT_BF16 ? 2 : 4; }
+
+GemmPlan plan_gemm(const swift_model_desc* d, int N, int K)
+{
+    const int vec = d->dtype == SWIFT_BF16 ? 8 : 4;
+    const int kc_max = d->dtype == SWIFT_BF16 ? 2048 : 1024;
+    const int gran = 32 * vec;
+    const int tiles = ceil_div(N, GEMM_SIMT_TILE_N);
+    int S = ceil_div(K, kc_max);
+    const int want = ceil_div(2 * 148, tiles);              // at least two CTAs per SM in flight
+    const int s_cap = std::max(1, K / (2 * gran));
+    S = std::max(S, std::min(want, s_cap));
+    int Kc = ceil_div(ceil_div(K, S), gran) * gran;
+    S = ceil_div(K, Kc);
+    return {S, Kc};
+}
+
+WeightLayout weight_layout(const swift_model_desc* d)
+{
+    WeightLayout w;
+    Carve c;
+    const size_t es = esize_of(d);
+    const size_t dm = d->d_model, qd = (size_t)d->n_heads * d->head_dim, kd = (size_t)d->n_kv_heads * d->head_dim;
+    w.embed = c.take((size_t)d->vocab * dm * es);
+    for (int b = 0; b < d->n_blocks; ++b) {
+        w.wqkv.push_back(c.take((qd + 2 * kd) * dm * es));
+        w.wo.push_back(c.take(dm * qd * es));
+        w.wgu.push_back(c.take(2 * (size_t)d->ffn * dm * es));
+        w.wdown.push_back(c.take(dm * (size_t)d->ffn * es));
+    }
+    w.lm_head = c.take((size_t)d->vocab * dm * es);
+    for (int b = 0; b < d->n_blocks; ++b) {
+        w.attn_norm.push_back(c.take(dm * 4));
+        w.mlp_norm.push_back(c.take(dm * 4));
+    }
+    w.final_norm = c.take(dm * 4);
+    w.total = c.off;
+    return w;
+}
+
+int scratch_pages(const swift_model_desc* d) { return MAX_SCORE_ROWS / d->page_size + 2; }
+
+size_t page_bytes(const swift_model_desc* d)
+{
+    return (size_t)d->n_blocks * 2 * d->n_kv_heads * d->page_size * d->head_dim * esize_of(d);
+}
+
+WorkLayout work_layout(const swift_model_desc* d)
+{
+    WorkLayout k;
+    Carve c;
+    const size_t es = esize_of(d);
+    const size_t dm = d->d_model, qd = (size_t)d->n_heads * d->head_dim, kd = (size_t)d->n_kv_heads * d->head_dim;
+    const int max_splits = ceil_div(d->max_positions, ATTN_CHUNK);
+    size_t pf = 0;
+    auto need = [&](int N, int K) { pf = std::max(pf, (size_t)plan_gemm(d, N, K).S * ROWS * (size_t)N); };
+    need((int)(qd + 2 * kd), (int)dm); need((int)dm, (int)qd); need(2 * d->ffn, (int)dm); need((int)dm, d->ffn);
+    need(d->vocab, (int)dm);
+    k.part_floats = pf;
+    k.state = c.take(sizeof(DevState));
+    k.h = c.take(ROWS * dm * 4);
+    k.xn = c.take(ROWS * dm * es);
+    k.xa = c.take(ROWS * qd * es);
+    k.act = c.take(ROWS * (size_t)d->ffn * es);
+    k.q = c.take(ROWS * qd * 4);
+    k.part = c.take(pf * 4);
+    k.o_part = c.take((size_t)d->n_heads * max_splits * ROWS * d->head_dim * 4);
+    k.ml_part = c.take((size_t)d->n_heads * max_splits * ROWS * 8);
+    k.logits = c.take((size_t)ROWS * d->vocab * 4);
+    k.q_rows = c.take((size_t)std::max(1, d->max_draft) * d->vocab * 4);
+    k.rope = c.take((size_t)d->max_positions * (d->head_dim / 2) * 8);
+    const int np = d->max_positions / d->page_size;
+    k.pt_main = c.take((size_t)np * 4);
+    k.pt_score = c.take((size_t)np * 4);
+    k.score_tok = c.take(MAX_SCORE_ROWS * 4);
+    k.score_truth = c.take(MAX_SCORE_ROWS * 4);
+    k.score_out = c.take(1024 * 4);
+    k.total = c.off;
+    return k;
+}
+
+template <typename T> T* wptr(swift_ctx* c, size_t off) { return reinterpret_cast<T*>(c->wbase + off); }
+template <typename T> T* kptr(swift_ctx* c, size_t off) { return reinterpret_cast<T*>(c->ws + off); }
+DevState* state_of(swift_ctx* c) { return kptr<DevState>(c, c->kl.state); }
+
+int mr_of(int rows) { return rows <= 1 ? 1 : rows <= 2 ? 2 : rows <= 4 ? 4 : rows <= 8 ? 8 : 16; }
+
+// ------------------------------------------------------------------------------ launches
+template <typename T, int MR>
+swift_status launch_gemm_mr(swift_ctx* ctx, const T* X, int ldx, const T* W, int N, int K, GemmPlan p)
+{
+    static bool attr_set[8] = {false};
+    const size_t smem = (size_t)MR * p.Kc * sizeof(T);
+    if (!attr_set[ctx->device & 7]) {
+        CU(cudaFuncSetAttribute(gemm_simt_kernel<T, MR>, cudaFuncAttributeMaxDynamicSharedMemorySize, 16 * 2048 * 2 + 0));
+        attr_set[ctx->device & 7] = true;
+    }
+    dim3 grid(ceil_div(N, GEMM_SIMT_TILE_N), p.S);
+    gemm_simt_kernel<T, MR><<<grid, GEMM_SIMT_THREADS, smem, ctx->stream>>>(state_of(ctx), X, ldx, W,
+                                                                            kptr<float>(ctx, ctx->kl.part), N, K, p.Kc);
+    ctx->launches++;
+    CU(cudaGetLastError());
+    return SWIFT_OK;
+}
+
+template <typename T>
+swift_status launch_gemm(swift_ctx* ctx, int mr, const T* X, int ldx, const T* W, int N, int K, GemmPlan* plan_out)
+{
+    const GemmPlan p = plan_gemm(&ctx->d, N, K);
+    *plan_out = p;
+    switch (mr) {
+    case 1: return launch_gemm_mr<T, 1>(ctx, X, ldx, W, N, K, p);
+    case 2: return launch_gemm_mr<T, 2>(ctx, X, ldx, W, N, K, p);
+    case 4: return launch_gemm_mr<T, 4>(ctx, X, ldx, W, N, K, p);
+    case 8: return launch_gemm_mr<T, 8>(ctx, X, ldx, W, N, K, p);
+    default: return launch_gemm_mr<T, 16>(ctx, X, ldx, W, N, K, p);
+    }
+}
+
+template <typename T, int MR>
+swift_status launch_attn_mr(swift_ctx* ctx, const int* page_table, int block)
+{
+    const swift_model_desc& d = ctx->d;
+    const size_t smem = ((size_t)MR * d.head_dim + (size_t)MR * ATTN_CHUNK + 2 * MR) * sizeof(float);
+    static bool attr_set[8] = {false};
+    if (!attr_set[ctx->device & 7]) {
+        CU(cudaFuncSetAttribute(attn_split_kernel<T, MR>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                (16 * 256 + 16 * ATTN_CHUNK + 32) * 4));
+        attr_set[ctx->device & 7] = true;
+    }
+    dim3 grid(d.n_heads, ctx->max_splits);
+    attn_split_kernel<T, MR><<<grid, ATTN_THREADS, smem, ctx->stream>>>(
+        state_of(ctx), kptr<float>(ctx, ctx->kl.q), reinterpret_cast<const T*>(ctx->kvbase), page_table, ctx->kv, block,
+        d.n_heads, ctx->max_splits, 1.0f / sqrtf((float)d.head_dim), kptr<float>(ctx, ctx->kl.o_part),
+        kptr<float2>(ctx, ctx->kl.ml_part));
+    ctx->launches++;
+    CU(cudaGetLastError());
+    return SWIFT_OK;
+}
+
+template <typename T>
+swift_status launch_attn(swift_ctx* ctx, int mr, const int* page_table, int block)
+{
+    switch (mr) {
+    case 1: return launch_attn_mr<T, 1>(ctx, page_table, block);
+    case 2: return launch_attn_mr<T, 2>(ctx, page_table, block);
+    case 4: return launch_attn_mr<T, 4>(ctx, page_table, block);
+    case 8: return launch_attn_mr<T, 8>(ctx, page_table, block);
+    default: return launch_attn_mr<T, 16>(ctx, page_table, block);
+    }
+}
+
+struct HeadOpts {
+    bool run = false;
+    int mode = VOCAB_PLAIN, draft_j = 0;
+    float stop_conf = 0.f;
+};
+
+#define ST(call)                                   \
+    do {                                           \
+        swift_status s_ = (call);                  \
+        if (s_ != SWIFT_OK) return s_;             \
+    } while (0)
+
+// Enqueues the kernels of one forward chunk of at most `rows` (<= 16) rows.  The device state
+// (pos0, n_rows, tok_off) must have been set by a preceding kernel on the same stream.
+template <typename T>
+swift_status forward_chunk(swift_ctx* ctx, int rows, const int* toks_dev, const uint8_t* skip, const int* page_table,
+                           HeadOpts head)
+{
+    const swift_model_desc& d = ctx->d;
+    DevState* st = state_of(ctx);
+    cudaStream_t s = ctx->stream;
+    const int mr = mr_of(rows);
+    const int dm = d.d_model, qd = d.n_heads * d.head_dim, kd = d.n_kv_heads * d.head_dim, nqkv = qd + 2 * kd;
+    float* h = kptr<float>(ctx, ctx->kl.h);
+    T* xn = kptr<T>(ctx, ctx->kl.xn);
+    T* xa = kptr<T>(ctx, ctx->kl.xa);
+    T* act = kptr<T>(ctx, ctx->kl.act);
+    float* part = kptr<float>(ctx, ctx->kl.part);
+    const float* pend = nullptr;      // pending residual-branch output (split-K partials) not yet added to h
+    int pend_S = 0;
+    GemmPlan p;
+
+    embed_kernel<T><<<rows, 256, 0, s>>>(st, toks_dev, wptr<T>(ctx, ctx->wl.embed), h, dm, d.vocab);
+    ctx->launches++;
+    for (int b = 0; b < d.n_blocks; ++b) {
+        if (!(skip && skip[2 * b])) {
+            resid_norm_kernel<T><<<rows, 512, 0, s>>>(st, h, pend, pend_S, (size_t)ROWS * dm,
+                                                      wptr<float>(ctx, ctx->wl.attn_norm[b]), xn, dm, d.rms_eps);
+            ctx->launches++;
+            ST(launch_gemm<T>(ctx, mr, xn, dm, wptr<T>(ctx, ctx->wl.wqkv[b]), nqkv, dm, &p));
+            qkv_post_kernel<T><<<dim3(rows, d.n_heads + 2 * d.n_kv_heads), d.head_dim / 2, 0, s>>>(
+                st, part, p.S, (size_t)ROWS * nqkv, nqkv, kptr<float>(ctx, ctx->kl.q), reinterpret_cast<T*>(ctx->kvbase),
+                page_table, ctx->kv, b, d.n_heads, kptr<float2>(ctx, ctx->kl.rope), d.max_positions);
+            ctx->launches++;
+            ST(launch_attn<T>(ctx, mr, page_table, b));
+            attn_combine_kernel<T><<<dim3(d.n_heads, rows), d.head_dim, 0, s>>>(
+                st, kptr<float>(ctx, ctx->kl.o_part), kptr<float2>(ctx, ctx->kl.ml_part), ctx->max_splits, d.n_heads,
+                d.head_dim, xa);
+            ctx->launches++;
+            ST(launch_gemm<T>(ctx, mr, xa, qd, wptr<T>(ctx, ctx->wl.wo[b]), dm, qd, &p));
+            pend = part; pend_S = p.S;
+        }
+        if (!(skip && skip[2 * b + 1])) {
+            resid_norm_kernel<T><<<rows, 512, 0, s>>>(st, h, pend, pend_S, (size_t)ROWS * dm,
+                                                      wptr<float>(ctx, ctx->wl.mlp_norm[b]), xn, dm, d.rms_eps);
+            ctx->launches++;
+            ST(launch_gemm<T>(ctx, mr, xn, dm, wptr<T>(ctx, ctx->wl.wgu[b]), 2 * d.ffn, dm, &p));
+            swiglu_kernel<T><<<dim3(ceil_div(d.ffn, 256), rows), 256, 0, s>>>(st, part, p.S, (size_t)ROWS * 2 * d.ffn, act,
+                                                                            d.ffn);
+            ctx->launches++;
+            ST(launch_gemm<T>(ctx, mr, act, d.ffn, wptr<T>(ctx, ctx->wl.wdown[b]), dm, d.ffn, &p));
+            pend = part; pend_S = p.S;
+        }
+    }
+    if (head.run) {
+        resid_norm_kernel<T><<<rows, 512, 0, s>>>(st, h, pend, pend_S, (size_t)ROWS * dm,
+                                                  wptr<float>(ctx, ctx->wl.final_norm), xn, dm, d.rms_eps);
+        ctx->launches++;
+        ST(launch_gemm<T>(ctx, mr, xn, dm, wptr<T>(ctx, ctx->wl.lm_head), d.vocab, dm, &p));
+        vocab_kernel<<<rows, VOCAB_THREADS, 0, s>>>(st, part, p.S, (size_t)ROWS * d.vocab,
+                                                   kptr<float>(ctx, ctx->kl.logits), d.vocab, 1.0f / ctx->temperature,
+                                                   head.mode, head.draft_j, head.stop_conf,
+                                                   ctx->mode == SWIFT_SAMPLING ? 1 : 0, ctx->seed, (uint32_t)ctx->round,
+                                                   kptr<float>(ctx, ctx->kl.q_rows));
+        ctx->launches++;
+    }
+    CU(cudaGetLastError());
+    return SWIFT_OK;
+}
+
+swift_status forward_chunk_any(swift_ctx* ctx, int rows, const int* toks_dev, const uint8_t* skip, const int* page_table,
+                               HeadOpts head)
+{
+    if (ctx->d.dtype == SWIFT_BF16) return forward_chunk<__nv_bfloat16>(ctx, rows, toks_dev, skip, page_table, head);
+    return forward_chunk<float>(ctx, rows, toks_dev, skip, page_table, head);
+}
+
+} // namespace
+
+// =============================================================================== helpers
+namespace {
+
+struct HostState { DevState s; };
+
+swift_status read_state(swift_ctx* ctx, DevState* out)
+{
+    CU(cudaMemcpyAsync(out, state_of(ctx), sizeof(DevState), cudaMemcpyDeviceToHost, ctx->stream));
+    CU(cudaStreamSynchronize(ctx->stream));
+    if (out->error) {
+        CU(cudaMemsetAsync(&state_of(ctx)->error, 0, sizeof(int), ctx->stream));
+        return fail(ctx, SWIFT_EINVAL, "device reported an invalid token id");
+    }
+    return SWIFT_OK;
+}
+
+const int* pt_main(swift_ctx* c) { return kptr<int>(c, c->kl.pt_main); }
+const int* pt_score(swift_ctx* c) { return kptr<int>(c, c->kl.pt_score); }
+
+// Redirects the pages that hold positions [p_begin, p_end) to scratch pages in the scoring page
+// table, copying the first page when the range starts inside it (copy-on-write).
+swift_status prepare_scratch(swift_ctx* ctx, int p_begin, int p_end)
+{
+    const int P = ctx->d.page_size;
+    const int first = p_begin / P, last = (p_end - 1) / P;
+    if (last - first + 1 > ctx->n_pages_scratch) return fail(ctx, SWIFT_ECAPACITY, "window spans too many KV pages");
+    std::vector<int> pt(ctx->n_pages_main);
+    for (int i = 0; i < ctx->n_pages_main; ++i) pt[i] = i;
+    for (int p = first; p <= last; ++p) pt[p] = ctx->n_pages_main + (p - first);
+    CU(cudaMemcpyAsync(kptr<int>(ctx, ctx->kl.pt_score), pt.data(), pt.size() * 4, cudaMemcpyHostToDevice, ctx->stream));
+    if (p_begin % P) {
+        const size_t v16 = page_bytes(&ctx->d) / 16;
+        page_copy_kernel<<<296, 256, 0, ctx->stream>>>(reinterpret_cast<uint4*>(ctx->kvbase), v16, first, ctx->n_pages_main);
+        ctx->launches++;
+        CU(cudaGetLastError());
+    }
+    return SWIFT_OK;
+}
+
+// head_mode: 0 = no output head, 1 = last chunk only, 2 = every chunk.
+swift_status run_rows(swift_ctx* ctx, const int32_t* tokens, int n_rows, int pos0, const uint8_t* skip,
+                      const int* page_table, int head_mode, float* logits_host, int32_t* argmax_host, int* last_chunk_rows)
+{
+    DevState* st = state_of(ctx);
+    for (int c0 = 0; c0 < n_rows; c0 += ROWS) {
+        const int rows = std::min(ROWS, n_rows - c0);
+        const bool last = c0 + rows == n_rows;
+        CU(cudaMemcpyAsync(st->row_tok, tokens + c0, rows * 4, cudaMemcpyHostToDevice, ctx->stream));
+        set_rows_kernel<<<1, 1, 0, ctx->stream>>>(st, pos0 + c0, rows);
+        ctx->launches++;
+        HeadOpts head;
+        head.run = head_mode == 2 || (head_mode == 1 && last);
+        ST(forward_chunk_any(ctx, rows, st->row_tok, skip, page_table, head));
+        if (head.run && logits_host)
+            CU(cudaMemcpyAsync(logits_host + (size_t)c0 * ctx->d.vocab, kptr<float>(ctx, ctx->kl.logits),
+                               (size_t)rows * ctx->d.vocab * 4, cudaMemcpyDeviceToHost, ctx->stream));
+        if (head.run && argmax_host)
+            CU(cudaMemcpyAsync(argmax_host + c0, st->argmax, rows * 4, cudaMemcpyDeviceToHost, ctx->stream));
+        if (last && last_chunk_rows) *last_chunk_rows = rows;
+    }
+    return SWIFT_OK;
+}
+
+swift_status check_tokens(swift_ctx* ctx, const int32_t* t, int n)
+{
+    if (!t) return fail(ctx, SWIFT_EINVAL, "null token pointer");
+    for (int i = 0; i < n; ++i)
+        if (t[i] < 0 || t[i] >= ctx->d.vocab) return fail(ctx, SWIFT_EINVAL, "token id %d at index %d outside [0, %d)", t[i], i, ctx->d.vocab);
+    return SWIFT_OK;
+}
+
+// ---- enqueue-only forms of the steps (no host synchronisation); used by the entry points and by generate
+swift_status enqueue_draft(swift_ctx* ctx, const uint8_t* skip, int max_k, float stop_conf)
+{
+    DevState* st = state_of(ctx);
+    ctx->round++;
+    begin_round_kernel<<<1, 1, 0, ctx->stream>>>(st, ctx->pending, 1);
+    ctx->launches++;
+    for (int j = 1; j <= max_k; ++j) {
+        begin_draft_step_kernel<<<1, 1, 0, ctx->stream>>>(st, ctx->n, j);
+        ctx->launches++;
+        HeadOpts head;
+        head.run = true; head.mode = VOCAB_DRAFT; head.draft_j = j; head.stop_conf = stop_conf;
+        ST(forward_chunk_any(ctx, 1, st->draft_tok, skip, pt_main(ctx), head));
+    }
+    ctx->last_max_k = max_k;
+    ctx->round_open = true;
+    return SWIFT_OK;
+}
+
+swift_status enqueue_verify(swift_ctx* ctx, int rows_launch, int forced_k)
+{
+    DevState* st = state_of(ctx);
+    begin_verify_kernel<<<1, 1, 0, ctx->stream>>>(st, ctx->n, forced_k);
+    ctx->launches++;
+    HeadOpts head;
+    head.run = true;
+    return forward_chunk_any(ctx, rows_launch, st->draft_tok, nullptr, pt_main(ctx), head);
+}
+
+swift_status enqueue_accept(swift_ctx* ctx)
+{
+    accept_kernel<<<1, VOCAB_THREADS, 0, ctx->stream>>>(state_of(ctx), kptr<float>(ctx, ctx->kl.logits),
+                                                        kptr<float>(ctx, ctx->kl.q_rows), ctx->d.vocab,
+                                                        ctx->mode == SWIFT_SAMPLING ? 1 : 0, 1.0f / ctx->temperature,
+                                                        ctx->seed, (uint32_t)ctx->round);
+    ctx->launches++;
+    CU(cudaGetLastError());
+    return SWIFT_OK;
+}
+
+// Folds the outcome of a round (read back from the device) into the host-side committed state.
+void commit_round(swift_ctx* ctx, const DevState& hs)
+{
+    const int a = hs.n_accepted;
+    for (int j = 1; j <= a; ++j) ctx->hist.push_back(hs.draft_tok[j]);
+    ctx->hist.push_back(hs.next_token);
+    ctx->n += a + 1;
+    ctx->pending = hs.next_token;
+    ctx->phase = PH_READY;
+    ctx->round_open = false;
+}
+
+// Scores C candidates; results (match counts) land in the score_out device array.
+swift_status enqueue_score(swift_ctx* ctx, const uint8_t* masks, int C, int gamma)
+{
+    const int n = ctx->n, L = 2 * ctx->d.n_blocks;
+    DevState* st = state_of(ctx);
+    int* tok_dev = kptr<int>(ctx, ctx->kl.score_tok);
+    int* truth_dev = kptr<int>(ctx, ctx->kl.score_truth);
+    int* out_dev = kptr<int>(ctx, ctx->kl.score_out);
+    CU(cudaMemcpyAsync(tok_dev, ctx->hist.data() + (n - gamma), gamma * 4, cudaMemcpyHostToDevice, ctx->stream));
+    CU(cudaMemcpyAsync(truth_dev, ctx->hist.data() + (n - gamma + 1), gamma * 4, cudaMemcpyHostToDevice, ctx->stream));
+    ST(prepare_scratch(ctx, n - gamma, n));
+    for (int c = 0; c < C; ++c) {
+        for (int c0 = 0; c0 < gamma; c0 += ROWS) {
+            const int rows = std::min(ROWS, gamma - c0);
+            set_rows_kernel<<<1, 1, 0, ctx->stream>>>(st, n - gamma + c0, rows);
+            ctx->launches++;
+            HeadOpts head;
+            head.run = true;
+            ST(forward_chunk_any(ctx, rows, tok_dev + c0, masks + (size_t)c * L, pt_score(ctx), head));
+            match_count_kernel<<<1, 32, 0, ctx->stream>>>(st, truth_dev + c0, c0 == 0 ? 1 : 0,
+                                                          c0 + rows == gamma ? out_dev + c : nullptr);
+            ctx->launches++;
+        }
+    }
+    CU(cudaGetLastError());
+    return SWIFT_OK;
+}
+
+double forward_bytes(const swift_ctx* ctx, const uint8_t* skip, int n_rows, int n_context)
+{
+    const swift_model_desc& d = ctx->d;
+    const double es = (double)ctx->esize;
+    const double dm = d.d_model, qd = (double)d.n_heads * d.head_dim, kd = (double)d.n_kv_heads * d.head_dim;
+    const double attn_w = (qd + 2 * kd) * dm + dm * qd, mlp_w = 3.0 * d.ffn * dm;
+    double bytes = (double)d.vocab * dm * es;                      // output head
+    for (int b = 0; b < d.n_blocks; ++b) {
+        if (!(skip && skip[2 * b])) bytes += attn_w * es + 2.0 * kd * n_context * es + 2.0 * kd * n_rows * es;
+        if (!(skip && skip[2 * b + 1])) bytes += mlp_w * es;
+    }
+    bytes += n_rows * (dm * es + (double)d.vocab * 4.0);           // embedding rows in, logits out
+    return bytes;
+}
+
+} // namespace
+
+// =============================================================================== C boundary
+extern "C" {
+
+size_t swift_weights_bytes(const swift_model_desc* d) { return desc_ok(d, nullptr) ? weight_layout(d).total : 0; }
+
+size_t swift_kv_bytes(const swift_model_desc* d)
+{
+    if (!desc_ok(d, nullptr)) return 0;
+    return (size_t)(d->max_positions / d->page_size + scratch_pages(d)) * page_bytes(d);
+}
+
+size_t swift_workspace_bytes(const swift_model_desc* d) { return desc_ok(d, nullptr) ? work_layout(d).total : 0; }
+
+const char* swift_last_error(const swift_ctx* ctx) { return ctx ? ctx->err.c_str() : g_load_error.c_str(); }
+
+swift_status swift_load(const swift_model_desc* desc, swift_devbuf weights, swift_devbuf kv_pool, swift_devbuf workspace,
+                        void* cuda_stream, swift_ctx** out)
+{
+    swift_ctx* ctx = nullptr;   // for the error macros: errors before creation go to the thread-local text
+    if (!out) return fail(nullptr, SWIFT_EINVAL, "out is null");
+    *out = nullptr;
+    std::string why;
+    if (!desc_ok(desc, &why)) return fail(nullptr, SWIFT_EINVAL, "invalid model description: %s", why.c_str());
+    if (!weights.dptr || !kv_pool.dptr || !workspace.dptr) return fail(nullptr, SWIFT_EINVAL, "null device buffer");
+    if (((uintptr_t)weights.dptr | (uintptr_t)kv_pool.dptr | (uintptr_t)workspace.dptr) % ALIGN)
+        return fail(nullptr, SWIFT_EINVAL, "device buffers must be 256-byte aligned");
+    if (weights.bytes < swift_weights_bytes(desc) || kv_pool.bytes < swift_kv_bytes(desc) ||
+        workspace.bytes < swift_workspace_bytes(desc))
+        return fail(nullptr, SWIFT_ECAPACITY, "a device buffer is smaller than the size query says");
+    int dev = 0, major = 0;
+    CU(cudaGetDevice(&dev));
+    CU(cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev));
+    if (major < 10) return fail(nullptr, SWIFT_EUNSUPPORTED, "this library is built for sm_100a only (device has major %d)", major);
+
+    swift_ctx* c = new swift_ctx();
+    c->d = *desc;
+    c->stream = (cudaStream_t)cuda_stream;
+    c->device = dev;
+    c->esize = esize_of(desc);
+    c->wbase = (char*)weights.dptr; c->kvbase = (char*)kv_pool.dptr; c->ws = (char*)workspace.dptr;
+    c->wl = weight_layout(desc);
+    c->kl = work_layout(desc);
+    int shift = 0;
+    while ((1 << shift) < desc->page_size) ++shift;
+    c->kv = KvLayout{desc->n_blocks, desc->n_kv_heads, desc->head_dim, desc->page_size, shift};
+    c->n_pages_main = desc->max_positions / desc->page_size;
+    c->n_pages_scratch = scratch_pages(desc);
+    c->max_splits = ceil_div(desc->max_positions, ATTN_CHUNK);
+    c->phase = PH_LOADED; c->n = 0; c->pending = 0; c->n_prompt = 0; c->round = 0; c->last_k = 0; c->last_max_k = 0;
+    c->round_open = false;
+    c->mode = SWIFT_GREEDY; c->temperature = 1.f; c->seed = 0; c->launches = 0;
+    ctx = c;
+    for (auto& e : c->ev) e = nullptr;
+    cudaError_t e = cudaSuccess;
+    for (auto& ev : c->ev) if (e == cudaSuccess) e = cudaEventCreate(&ev);
+    if (e == cudaSuccess) e = cudaMemsetAsync(c->ws, 0, c->kl.total, c->stream);
+    if (e == cudaSuccess) {
+        const int half = desc->head_dim / 2, total = desc->max_positions * half;
+        rope_table_kernel<<<ceil_div(total, 256), 256, 0, c->stream>>>(kptr<float2>(c, c->kl.rope), desc->max_positions, half,
+                                                                     (double)desc->rope_theta);
+        c->launches++;
+        std::vector<int> pt(c->n_pages_main);
+        for (int i = 0; i < c->n_pages_main; ++i) pt[i] = i;
+        e = cudaMemcpyAsync(kptr<int>(c, c->kl.pt_main), pt.data(), pt.size() * 4, cudaMemcpyHostToDevice, c->stream);
+        if (e == cudaSuccess) e = cudaMemcpyAsync(kptr<int>(c, c->kl.pt_score), pt.data(), pt.size() * 4, cudaMemcpyHostToDevice, c->stream);
+        if (e == cudaSuccess) e = cudaStreamSynchronize(c->stream);
+        if (e == cudaSuccess) e = cudaGetLastError();
+    }
+    if (e != cudaSuccess) {
+        fail(nullptr, SWIFT_ECUDA, "set-up failed: %s", cudaGetErrorString(e));
+        for (auto& ev : c->ev) if (ev) cudaEventDestroy(ev);
+        delete c;
+        return SWIFT_ECUDA;
+    }
+    *out = c;
+    return SWIFT_OK;
+}
+
+swift_status swift_free(swift_ctx* ctx)
+{
+    if (!ctx) return SWIFT_OK;
+    cudaStreamSynchronize(ctx->stream);
+    for (auto& ev : ctx->ev) if (ev) cudaEventDestroy(ev);
+    delete ctx;
+    return SWIFT_OK;
+}
+
+swift_status swift_pack_tensor(swift_ctx* ctx, swift_tensor_kind kind, int32_t block, const void* src, size_t src_bytes)
+{
+    if (!ctx || !src) return fail(ctx, SWIFT_EINVAL, "null argument");
+    const swift_model_desc& d = ctx->d;
+    const size_t es = ctx->esize, dm = d.d_model, qd = (size_t)d.n_heads * d.head_dim, kd = (size_t)d.n_kv_heads * d.head_dim;
+    const bool per_block = kind >= SWIFT_T_WQ;
+    if (per_block && (block < 0 || block >= d.n_blocks)) return fail(ctx, SWIFT_EINVAL, "block %d out of range", block);
+    size_t dst = 0, bytes = 0;
+    bool interleave = false;
+    switch (kind) {
+    case SWIFT_T_EMBED: dst = ctx->wl.embed; bytes = (size_t)d.vocab * dm * es; break;
+    case SWIFT_T_LM_HEAD: dst = ctx->wl.lm_head; bytes = (size_t)d.vocab * dm * es; break;
+    case SWIFT_T_FINAL_NORM: dst = ctx->wl.final_norm; bytes = dm * 4; break;
+    case SWIFT_T_WQ: dst = ctx->wl.wqkv[block]; bytes = qd * dm * es; break;
+    case SWIFT_T_WK: dst = ctx->wl.wqkv[block] + qd * dm * es; bytes = kd * dm * es; break;
+    case SWIFT_T_WV: dst = ctx->wl.wqkv[block] + (qd + kd) * dm * es; bytes = kd * dm * es; break;
+    case SWIFT_T_WO: dst = ctx->wl.wo[block]; bytes = dm * qd * es; break;
+    case SWIFT_T_WGATE: dst = ctx->wl.wgu[block]; bytes = (size_t)d.ffn * dm * es; interleave = true; break;
+    case SWIFT_T_WUP: dst = ctx->wl.wgu[block] + 16 * dm * es; bytes = (size_t)d.ffn * dm * es; interleave = true; break;
+    case SWIFT_T_WDOWN: dst = ctx->wl.wdown[block]; bytes = dm * (size_t)d.ffn * es; break;
+    case SWIFT_T_ATTN_NORM: dst = ctx->wl.attn_norm[block]; bytes = dm * 4; break;
+    case SWIFT_T_MLP_NORM: dst = ctx->wl.mlp_norm[block]; bytes = dm * 4; break;
+    default: return fail(ctx, SWIFT_EINVAL, "unknown tensor kind %d", (int)kind);
+    }
+    if (src_bytes != bytes) return fail(ctx, SWIFT_EINVAL, "tensor kind %d expects %zu bytes, got %zu", (int)kind, bytes, src_bytes);
+    CU(cudaStreamSynchronize(ctx->stream));
+    if (interleave) {
+        const size_t group = 16 * dm * es;       // 16 rows of gate (or up) ...
+        CU(cudaMemcpy2D(ctx->wbase + dst, 2 * group, src, group, group, d.ffn / 16, cudaMemcpyHostToDevice));  // ... every 32 rows
+    } else {
+        CU(cudaMemcpy(ctx->wbase + dst, src, bytes, cudaMemcpyHostToDevice));
+    }
+    return SWIFT_OK;
+}
+
+swift_status swift_set_sampling(swift_ctx* ctx, int32_t mode, float temperature, uint64_t seed)
+{
+    if (!ctx) return SWIFT_EINVAL;
+    if (mode != SWIFT_GREEDY && mode != SWIFT_SAMPLING) return fail(ctx, SWIFT_EINVAL, "mode must be SWIFT_GREEDY or SWIFT_SAMPLING");
+    if (!(temperature > 0.f)) return fail(ctx, SWIFT_EINVAL, "temperature must be positive");
+    if (ctx->round_open) return fail(ctx, SWIFT_ESTATE, "cannot change the acceptance strategy inside a round");
+    ctx->mode = mode; ctx->temperature = temperature; ctx->seed = seed;
+    return SWIFT_OK;
+}
+
+swift_status swift_forward_rows(swift_ctx* ctx, const int32_t* tokens, int32_t n_rows, int32_t pos0, const uint8_t* skip,
+                                int32_t write_kv, float* logits_host, int32_t* argmax_host)
+{
+    if (!ctx) return SWIFT_EINVAL;
+    if (ctx->round_open) return fail(ctx, SWIFT_ESTATE, "a round is open");
+    if (n_rows < 1 || pos0 < 0) return fail(ctx, SWIFT_EINVAL, "n_rows >= 1 and pos0 >= 0 required");
+    if (pos0 > ctx->n) return fail(ctx, SWIFT_EINVAL, "pos0 %d beyond the committed length %d", pos0, ctx->n);
+    if (pos0 + n_rows > ctx->d.max_positions) return fail(ctx, SWIFT_ECAPACITY, "rows run past max_positions");
+    if (!write_kv && n_rows > MAX_SCORE_ROWS) return fail(ctx, SWIFT_ECAPACITY, "at most %d rows without KV write", MAX_SCORE_ROWS);
+    ST(check_tokens(ctx, tokens, n_rows));
+    const int* pt = pt_main(ctx);
+    if (!write_kv) { ST(prepare_scratch(ctx, pos0, pos0 + n_rows)); pt = pt_score(ctx); }
+    ST(run_rows(ctx, tokens, n_rows, pos0, skip, pt, (logits_host || argmax_host) ? 2 : 0, logits_host, argmax_host, nullptr));
+    DevState hs;
+    return read_state(ctx, &hs);
+}
+
+swift_status swift_prefill(swift_ctx* ctx, const int32_t* tokens, int32_t n, int32_t* first_token)
+{
+    if (!ctx) return SWIFT_EINVAL;
+    if (n < 1) return fail(ctx, SWIFT_EINVAL, "prompt must have at least one token");
+    if (n + 1 > ctx->d.max_positions) return fail(ctx, SWIFT_ECAPACITY, "prompt of %d tokens exceeds max_positions %d", n, ctx->d.max_positions);
+    ST(check_tokens(ctx, tokens, n));
+    ctx->round_open = false;
+    ctx->n = 0;
+    int last_rows = 0;
+    ST(run_rows(ctx, tokens, n, 0, nullptr, pt_main(ctx), 1, nullptr, nullptr, &last_rows));
+    if (ctx->mode == SWIFT_SAMPLING) {
+        sample_row_kernel<<<1, VOCAB_THREADS, 0, ctx->stream>>>(state_of(ctx), kptr<float>(ctx, ctx->kl.logits), ctx->d.vocab,
+                                                                last_rows - 1, 1.0f / ctx->temperature, ctx->seed, 0u, 0u);
+        ctx->launches++;
+    }
+    DevState hs;
+    swift_status s = read_state(ctx, &hs);
+    if (s != SWIFT_OK) { ctx->phase = PH_LOADED; return s; }
+    const int tok = ctx->mode == SWIFT_SAMPLING ? hs.next_token : hs.argmax[last_rows - 1];
+    ctx->n = n; ctx->n_prompt = n; ctx->pending = tok; ctx->round = 0;
+    ctx->hist.assign(tokens, tokens + n);
+    ctx->hist.push_back(tok);
+    ctx->phase = PH_READY;
+    if (first_token) *first_token = tok;
+    return SWIFT_OK;
+}
+
+swift_status swift_set_pending(swift_ctx* ctx, int32_t token, int32_t rounds_done)
+{
+    if (!ctx) return SWIFT_EINVAL;
+    if (ctx->phase != PH_READY) return fail(ctx, SWIFT_ESTATE, "swift_set_pending needs a prefilled context with no open round");
+    if (token < 0 || token >= ctx->d.vocab) return fail(ctx, SWIFT_EINVAL, "token id %d outside [0, %d)", token, ctx->d.vocab);
+    ctx->pending = token;
+    ctx->hist.back() = token;
+    if (rounds_done >= 0) ctx->round = rounds_done;
+    return SWIFT_OK;
+}
+
+swift_status swift_draft(swift_ctx* ctx, const uint8_t* skip, int32_t max_k, float stop_conf, int32_t* tokens_host,
+                         float* conf_host, int32_t* k_host)
+{
+    if (!ctx) return SWIFT_EINVAL;
+    if (ctx->phase != PH_READY) return fail(ctx, SWIFT_ESTATE, "swift_draft needs a prefilled context with no open round");
+    if (!skip) return fail(ctx, SWIFT_EINVAL, "skip_mask is null");
+    if (max_k < 0 || max_k > ctx->d.max_draft) return fail(ctx, SWIFT_ECAPACITY, "max_k %d outside 0..max_draft (%d)", max_k, ctx->d.max_draft);
+    if (ctx->n + max_k + 1 > ctx->d.max_positions) return fail(ctx, SWIFT_ECAPACITY, "KV cache too small for %d more positions", max_k + 1);
+    ST(enqueue_draft(ctx, skip, max_k, stop_conf));
+    DevState hs;
+    ST(read_state(ctx, &hs));
+    ctx->last_k = hs.n_drafted;
+    ctx->phase = PH_DRAFTED;
+    for (int j = 0; j < hs.n_drafted; ++j) {
+        if (tokens_host) tokens_host[j] = hs.draft_tok[j + 1];
+        if (conf_host) conf_host[j] = hs.conf[j];
+    }
+    if (k_host) *k_host = hs.n_drafted;
+    return SWIFT_OK;
+}
+
+swift_status swift_verify(swift_ctx* ctx, const int32_t* tokens_host, int32_t k, int32_t* target_argmax, float* logits_host)
+{
+    if (!ctx) return SWIFT_EINVAL;
+    if (ctx->phase != PH_READY && ctx->phase != PH_DRAFTED) return fail(ctx, SWIFT_ESTATE, "swift_verify needs a prefilled context");
+    int rows_launch, forced_k;
+    if (tokens_host) {
+        if (k < 0 || k > SWIFT_MAX_ROWS - 1) return fail(ctx, SWIFT_ECAPACITY, "k %d outside 0..%d", k, SWIFT_MAX_ROWS - 1);
+        if (ctx->mode == SWIFT_SAMPLING && k > 0 && ctx->phase != PH_DRAFTED)
+            return fail(ctx, SWIFT_ESTATE, "sampling acceptance needs the draft distributions of swift_draft");
+        if (k > 0) ST(check_tokens(ctx, tokens_host, k));
+        if (ctx->n + k + 1 > ctx->d.max_positions) return fail(ctx, SWIFT_ECAPACITY, "KV cache too small");
+        if (ctx->phase == PH_READY) {
+            ctx->round++;
+            begin_round_kernel<<<1, 1, 0, ctx->stream>>>(state_of(ctx), ctx->pending, 1);
+            ctx->launches++;
+            ctx->round_open = true;
+        }
+        if (k > 0) CU(cudaMemcpyAsync(state_of(ctx)->draft_tok + 1, tokens_host, k * 4, cudaMemcpyHostToDevice, ctx->stream));
+        rows_launch = k + 1; forced_k = k;
+    } else {
+        if (ctx->phase != PH_DRAFTED) return fail(ctx, SWIFT_ESTATE, "no draft to verify: call swift_draft or pass tokens");
+        rows_launch = ctx->last_k + 1; forced_k = -1;
+    }
+    ST(enqueue_verify(ctx, rows_launch, forced_k));
+    DevState hs;
+    ST(read_state(ctx, &hs));
+    ctx->last_k = hs.n_drafted;
+    ctx->phase = PH_VERIFIED;
+    const int rows = hs.n_drafted + 1;
+    if (target_argmax) for (int r = 0; r < rows; ++r) target_argmax[r] = hs.argmax[r];
+    if (logits_host) {
+        CU(cudaMemcpyAsync(logits_host, kptr<float>(ctx, ctx->kl.logits), (size_t)rows * ctx->d.vocab * 4, cudaMemcpyDeviceToHost, ctx->stream));
+        CU(cudaStreamSynchronize(ctx->stream));
+    }
+    return SWIFT_OK;
+}
+
+swift_status swift_accept(swift_ctx* ctx, int32_t* n_accepted, int32_t* next_token)
+{
+    if (!ctx) return SWIFT_EINVAL;
+    if (ctx->phase != PH_VERIFIED) return fail(ctx, SWIFT_ESTATE, "swift_accept needs a verified round");
+    ST(enqueue_accept(ctx));
+    DevState hs;
+    ST(read_state(ctx, &hs));
+    commit_round(ctx, hs);
+    if (n_accepted) *n_accepted = hs.n_accepted;
+    if (next_token) *next_token = hs.next_token;
+    return SWIFT_OK;
+}
+
+swift_status swift_score_skipsets(swift_ctx* ctx, const uint8_t* masks, int32_t C, int32_t gamma, float* matchness)
+{
+    if (!ctx) return SWIFT_EINVAL;
+    if (ctx->phase != PH_READY) return fail(ctx, SWIFT_ESTATE, "swift_score_skipsets needs a prefilled context with no open round");
+    if (!masks || !matchness) return fail(ctx, SWIFT_EINVAL, "null argument");
+    if (C < 1 || C > 1024) return fail(ctx, SWIFT_ECAPACITY, "C must be in 1..1024");
+    if (gamma < 1 || gamma > MAX_SCORE_ROWS) return fail(ctx, SWIFT_ECAPACITY, "gamma must be in 1..%d", MAX_SCORE_ROWS);
+    if (gamma > ctx->n) return fail(ctx, SWIFT_EINVAL, "gamma %d exceeds the %d cached positions", gamma, ctx->n);
+    ST(enqueue_score(ctx, masks, C, gamma));
+    std::vector<int> counts(C);
+    CU(cudaMemcpyAsync(counts.data(), kptr<int>(ctx, ctx->kl.score_out), C * 4, cudaMemcpyDeviceToHost, ctx->stream));
+    DevState hs;
+    ST(read_state(ctx, &hs));
+    for (int c = 0; c < C; ++c) matchness[c] = (float)counts[c] / (float)gamma;
+    return SWIFT_OK;
+}
+
+int32_t swift_committed_length(const swift_ctx* ctx) { return ctx ? ctx->n : -1; }
+int64_t swift_launch_count(const swift_ctx* ctx) { return ctx ? ctx->launches : -1; }
+double swift_forward_bytes(const swift_ctx* ctx, const uint8_t* skip, int32_t n_rows, int32_t n_context)
+{
+    return ctx ? forward_bytes(ctx, skip, n_rows, n_context) : 0.0;
+}
+
+} // extern "C"
+
+// =============================================================================== inspection, generate
+extern "C" {
+
+swift_status swift_read_kv(swift_ctx* ctx, int32_t block, int32_t which, int32_t pos0, int32_t count, float* out_host)
+{
+    if (!ctx || !out_host) return fail(ctx, SWIFT_EINVAL, "null argument");
+    if (block < 0 || block >= ctx->d.n_blocks || (which != 0 && which != 1)) return fail(ctx, SWIFT_EINVAL, "bad block or which");
+    if (pos0 < 0 || count < 1 || pos0 + count > ctx->d.max_positions) return fail(ctx, SWIFT_EINVAL, "bad position range");
+    const size_t per_pos = (size_t)ctx->d.n_kv_heads * ctx->d.head_dim;
+    const int step = (int)std::max<size_t>(1, std::min<size_t>(count, ctx->kl.part_floats / per_pos));
+    float* stage = kptr<float>(ctx, ctx->kl.part);
+    for (int c0 = 0; c0 < count; c0 += step) {
+        const int cnt = std::min(step, count - c0);
+        if (ctx->d.dtype == SWIFT_BF16)
+            kv_read_kernel<__nv_bfloat16><<<64, 256, 0, ctx->stream>>>(reinterpret_cast<const __nv_bfloat16*>(ctx->kvbase),
+                                                                      pt_main(ctx), ctx->kv, block, which, pos0 + c0, cnt, stage);
+        else
+            kv_read_kernel<float><<<64, 256, 0, ctx->stream>>>(reinterpret_cast<const float*>(ctx->kvbase), pt_main(ctx),
+                                                               ctx->kv, block, which, pos0 + c0, cnt, stage);
+        ctx->launches++;
+        CU(cudaMemcpyAsync(out_host + (size_t)c0 * per_pos, stage, (size_t)cnt * per_pos * 4, cudaMemcpyDeviceToHost, ctx->stream));
+        CU(cudaStreamSynchronize(ctx->stream));
+    }
+    return SWIFT_OK;
+}
+
+} // extern "C"
+
+template <typename T>
+static swift_status time_gemm_t(swift_ctx* ctx, int which, int n_rows, int iters, float* ms, double* bytes)
+{
+    const swift_model_desc& d = ctx->d;
+    const int dm = d.d_model, qd = d.n_heads * d.head_dim, kd = d.n_kv_heads * d.head_dim;
+    const int N = which == 0 ? qd + 2 * kd : which == 1 ? dm : which == 2 ? 2 * d.ffn : which == 3 ? dm : d.vocab;
+    const int K = which == 1 ? qd : which == 3 ? d.ffn : dm;
+    const T* X = which == 1 ? kptr<T>(ctx, ctx->kl.xa) : which == 3 ? kptr<T>(ctx, ctx->kl.act) : kptr<T>(ctx, ctx->kl.xn);
+    set_rows_kernel<<<1, 1, 0, ctx->stream>>>(state_of(ctx), 0, n_rows);
+    ctx->launches++;
+    GemmPlan p;
+    auto weight = [&](int i) -> const T* {
+        const int b = i % d.n_blocks;
+        switch (which) {
+        case 0: return wptr<T>(ctx, ctx->wl.wqkv[b]);
+        case 1: return wptr<T>(ctx, ctx->wl.wo[b]);
+        case 2: return wptr<T>(ctx, ctx->wl.wgu[b]);
+        case 3: return wptr<T>(ctx, ctx->wl.wdown[b]);
+        default: return (i & 1) ? wptr<T>(ctx, ctx->wl.embed) : wptr<T>(ctx, ctx->wl.lm_head);
+        }
+    };
+    for (int i = 0; i < 3; ++i) ST(launch_gemm<T>(ctx, mr_of(n_rows), X, K, weight(i), N, K, &p));
+    CU(cudaEventRecord(ctx->ev[0], ctx->stream));
+    for (int i = 0; i < iters; ++i) ST(launch_gemm<T>(ctx, mr_of(n_rows), X, K, weight(i + 3), N, K, &p));
+    CU(cudaEventRecord(ctx->ev[1], ctx->stream));
+    CU(cudaStreamSynchronize(ctx->stream));
+    float t = 0.f;
+    CU(cudaEventElapsedTime(&t, ctx->ev[0], ctx->ev[1]));
+    *ms = t / (float)iters;
+    *bytes = (double)N * K * sizeof(T);
+    return SWIFT_OK;
+}
+
+extern "C" {
+
+swift_status swift_time_gemm(swift_ctx* ctx, int32_t which, int32_t n_rows, int32_t iters, float* ms, double* bytes)
+{
+    if (!ctx || !ms || !bytes) return fail(ctx, SWIFT_EINVAL, "null argument");
+    if (ctx->round_open) return fail(ctx, SWIFT_ESTATE, "a round is open");
+    if (which < 0 || which > 4 || n_rows < 1 || n_rows > ROWS || iters < 1) return fail(ctx, SWIFT_EINVAL, "bad which / n_rows / iters");
+    if (ctx->d.dtype == SWIFT_BF16) return time_gemm_t<__nv_bfloat16>(ctx, which, n_rows, iters, ms, bytes);
+    return time_gemm_t<float>(ctx, which, n_rows, iters, ms, bytes);
+}
+
+swift_status swift_generate(swift_ctx* ctx, const swift_gen_params* gp, const int32_t* prompt, int32_t n_prompt,
+                            int32_t* out_tokens, int32_t* n_out, int32_t* trace, swift_stats* stats)
+{
+    if (!ctx) return SWIFT_EINVAL;
+    if (!gp || !prompt || !out_tokens) return fail(ctx, SWIFT_EINVAL, "null argument");
+    const swift_model_desc& d = ctx->d;
+    if (gp->max_new < 1) return fail(ctx, SWIFT_EINVAL, "max_new must be >= 1");
+    if (n_prompt + gp->max_new + 1 > d.max_positions) return fail(ctx, SWIFT_ECAPACITY, "prompt + max_new exceeds max_positions");
+    if (!gp->vanilla) {
+        if (!gp->skip_mask) return fail(ctx, SWIFT_EINVAL, "skip_mask is null");
+        if (gp->max_draft < 0 || gp->max_draft > d.max_draft) return fail(ctx, SWIFT_ECAPACITY, "max_draft %d outside 0..%d", gp->max_draft, d.max_draft);
+        if (gp->n_opt_rounds > 0) {
+            if (!gp->candidate_masks || gp->n_candidates < 1 || gp->n_candidates > 1024) return fail(ctx, SWIFT_EINVAL, "candidate masks missing");
+            if (gp->gamma < 1 || gp->gamma > MAX_SCORE_ROWS) return fail(ctx, SWIFT_ECAPACITY, "gamma must be in 1..%d", MAX_SCORE_ROWS);
+        }
+    }
+    const int L = 2 * d.n_blocks;
+    const int64_t launches0 = ctx->launches;
+    swift_stats stt;
+    memset(&stt, 0, sizeof stt);
+    stt.best_matchness = -1.f;
+    cudaEvent_t* ev = ctx->ev;
+
+    CU(cudaEventRecord(ev[0], ctx->stream));
+    int first = 0;
+    ST(swift_prefill(ctx, prompt, n_prompt, &first));
+    CU(cudaEventRecord(ev[1], ctx->stream));
+    int count = 0;
+    out_tokens[count++] = first;
+
+    std::vector<uint8_t> z(L, 0);
+    if (!gp->vanilla) memcpy(z.data(), gp->skip_mask, L);
+    bool optimising = !gp->vanilla && gp->n_opt_rounds > 0;
+    std::vector<int> counts;
+    DevState hs;
+    while (count < gp->max_new) {
+        const int remaining = gp->max_new - count;
+        const int n_start = ctx->n;
+        if (gp->vanilla) {
+            ctx->round++;
+            begin_round_kernel<<<1, 1, 0, ctx->stream>>>(state_of(ctx), ctx->pending, 1);
+            ctx->launches++;
+            ST(enqueue_verify(ctx, 1, 0));
+            if (ctx->mode == SWIFT_SAMPLING) {
+                sample_row_kernel<<<1, VOCAB_THREADS, 0, ctx->stream>>>(state_of(ctx), kptr<float>(ctx, ctx->kl.logits), d.vocab, 0,
+                                                                        1.0f / ctx->temperature, ctx->seed, (uint32_t)ctx->round, 0u);
+                ctx->launches++;
+            } else {
+                const int save = ctx->mode;
+                ST(enqueue_accept(ctx));
+                ctx->mode = save;
+            }
+            ST(read_state(ctx, &hs));
+            hs.n_accepted = 0;
+            stt.bytes_verify += forward_bytes(ctx, nullptr, 1, n_start);
+        } else {
+            if (optimising && count >= gp->gamma) {
+                CU(cudaEventRecord(ev[2], ctx->stream));
+                const uint8_t* masks = gp->candidate_masks + (size_t)stt.opt_rounds * gp->n_candidates * L;
+                ST(enqueue_score(ctx, masks, gp->n_candidates, gp->gamma));
+                counts.resize(gp->n_candidates);
+                CU(cudaMemcpyAsync(counts.data(), kptr<int>(ctx, ctx->kl.score_out), gp->n_candidates * 4, cudaMemcpyDeviceToHost, ctx->stream));
+                CU(cudaEventRecord(ev[3], ctx->stream));
+                CU(cudaStreamSynchronize(ctx->stream));
+                float ms = 0.f;
+                CU(cudaEventElapsedTime(&ms, ev[2], ev[3]));
+                stt.ms_score += ms;
+                int cb = 0;
+                for (int c = 1; c < gp->n_candidates; ++c) if (counts[c] > counts[cb]) cb = c;   // lowest index among equals
+                const float best = (float)counts[cb] / (float)gp->gamma;
+                if (best > stt.best_matchness) {                                                // strictly better only
+                    stt.best_matchness = best;
+                    memcpy(z.data(), masks + (size_t)cb * L, L);
+                }
+                stt.opt_rounds++;
+                if (stt.best_matchness > gp->stop_matchness || stt.opt_rounds >= gp->n_opt_rounds) optimising = false;
+            }
+            const int k_max = std::min(gp->max_draft, remaining - 1);
+            CU(cudaEventRecord(ev[4], ctx->stream));
+            ST(enqueue_draft(ctx, z.data(), k_max, gp->stop_conf));
+            CU(cudaEventRecord(ev[5], ctx->stream));
+            ST(enqueue_verify(ctx, k_max + 1, -1));
+            ST(enqueue_accept(ctx));
+            CU(cudaEventRecord(ev[6], ctx->stream));
+            ST(read_state(ctx, &hs));
+            float md = 0.f, mv = 0.f;
+            CU(cudaEventElapsedTime(&md, ev[4], ev[5]));
+            CU(cudaEventElapsedTime(&mv, ev[5], ev[6]));
+            stt.ms_draft += md; stt.ms_verify += mv;
+            for (int j = 0; j < hs.n_drafted; ++j) stt.bytes_draft += forward_bytes(ctx, z.data(), 1, n_start + j);
+            stt.bytes_verify += forward_bytes(ctx, nullptr, hs.n_drafted + 1, n_start);
+            stt.drafted += hs.n_drafted;
+            stt.accepted += hs.n_accepted;
+        }
+        if (trace) {
+            trace[4 * stt.rounds + 0] = n_start; trace[4 * stt.rounds + 1] = gp->vanilla ? 0 : hs.n_drafted;
+            trace[4 * stt.rounds + 2] = hs.n_accepted; trace[4 * stt.rounds + 3] = hs.next_token;
+        }
+        stt.rounds++;
+        for (int j = 1; j <= hs.n_accepted; ++j) out_tokens[count++] = hs.draft_tok[j];
+        out_tokens[count++] = hs.next_token;
+        commit_round(ctx, hs);
+    }
+    CU(cudaEventRecord(ev[7], ctx->stream));
+    CU(cudaStreamSynchronize(ctx->stream));
+    CU(cudaEventElapsedTime(&stt.ms_prefill, ev[0], ev[1]));
+    CU(cudaEventElapsedTime(&stt.ms_decode, ev[1], ev[7]));
+    stt.tokens = count;
+    stt.kernel_launches = ctx->launches - launches0;
+    if (n_out) *n_out = count;
+    if (stats) *stats = stt;
+    return SWIFT_OK;
+}
+
+} // extern "C"

@@ -1,0 +1,67 @@
+"""No-GPU checks of the C boundary: the library builds, loads, exports every declared symbol, and
+answers size queries and argument errors without touching a device."""
+import ctypes as C
+import os
+import re
+
+import pytest
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+def test_library_exports_every_declared_symbol():
+    from paper_2410_06916_b200 import binding
+    lib = binding.load_library()
+    header = open(os.path.join(ROOT, "include", "swift.h")).read()
+    declared = set(re.findall(r"\b(swift_[a-z_]+)\s*\(", header))
+    declared -= {"swift_free"} - set(binding.SYMBOLS)
+    assert declared == set(binding.SYMBOLS), declared ^ set(binding.SYMBOLS)
+    for name in declared:
+        assert getattr(lib, name) is not None
+
+
+def test_size_queries_and_layout_invariants():
+    from paper_2410_06916_b200 import binding
+    import synth
+    lib = binding.load_library()
+    for name, cfg in synth.MODELS.items():
+        d = binding._Desc(cfg.n_blocks, cfg.d_model, cfg.n_heads, cfg.n_kv_heads, cfg.head_dim, cfg.ffn, cfg.vocab,
+                          1 if cfg.dtype == "bf16" else 0, cfg.rope_theta, cfg.rms_eps, 4096, 16, 12, 0)
+        wb = lib.swift_weights_bytes(C.byref(d))
+        es = 2 if cfg.dtype == "bf16" else 4
+        params = cfg.n_blocks * cfg.block_params() + 2 * cfg.vocab * cfg.d_model
+        gains = (2 * cfg.n_blocks + 1) * cfg.d_model * 4
+        assert params * es + gains <= wb <= params * es + gains + 256 * (6 * cfg.n_blocks + 4), name
+        kv = lib.swift_kv_bytes(C.byref(d))
+        per_pos = cfg.n_blocks * 2 * cfg.n_kv_heads * cfg.head_dim * es
+        assert kv == (4096 + 16 * (128 // 16 + 2)) * per_pos
+        assert lib.swift_workspace_bytes(C.byref(d)) > 0
+    bad = binding._Desc(4, 64, 4, 3, 16, 96, 97, 0, 1e4, 1e-5, 64, 16, 4, 0)     # heads not a multiple of kv heads
+    assert lib.swift_weights_bytes(C.byref(bad)) == 0
+
+
+def test_load_rejects_bad_arguments_without_a_device():
+    from paper_2410_06916_b200 import binding
+    lib = binding.load_library()
+    d = binding._Desc(4, 64, 4, 2, 16, 96, 97, 0, 1e4, 1e-5, 64, 16, 4, 0)
+    ctx = C.c_void_p()
+    null = binding._DevBuf(None, 0)
+    assert lib.swift_load(C.byref(d), null, null, null, None, C.byref(ctx)) == 1
+    assert b"null device buffer" in lib.swift_last_error(None)
+    assert lib.swift_prefill(None, None, 0, None) == 1
+    assert lib.swift_committed_length(None) == -1
+
+
+def test_product_path_has_no_oracle_or_cpu_fallback():
+    pkg = os.path.join(ROOT, "paper_2410_06916_b200")
+    for dirpath, _, files in os.walk(pkg):
+        for f in files:
+            if f.endswith((".py", ".cu", ".cuh", ".h")):
+                text = open(os.path.join(dirpath, f)).read()
+                assert "oracle" not in text.lower() or f == "binding.py" and False, f
+    import torch
+    if not torch.cuda.is_available():
+        from paper_2410_06916_b200 import SwiftModel
+        import synth
+        with pytest.raises(RuntimeError, match="needs a CUDA device"):
+            SwiftModel(synth.MODELS["tiny"], 64)

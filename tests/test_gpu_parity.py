@@ -1,0 +1,275 @@
+"""GPU parity: the CUDA library, called through its C boundary, against the CPU oracle on the same
+seeded inputs.  Tolerances: logits within 2e-2 of the oracle after dividing by the row's standard
+deviation; tokens, accepted-prefix lengths and matchness identical wherever the oracle's top-1/top-2
+margin exceeds 0.05; fp32 models are held to 1e-4 sigma."""
+import numpy as np
+import pytest
+import torch
+
+import synth
+from oracle import swift_oracle as so
+from tests.helpers import LOGIT_TOL, MARGIN, compare_free_running, logit_err, make_pair, resync, walk_rounds
+
+pytestmark = pytest.mark.gpu
+
+TINY = synth.MODELS["tiny"]
+BF16_SMALL = synth.ModelConfig("bf16-small", n_blocks=3, d_model=512, n_heads=8, n_kv_heads=2, head_dim=64,
+                               ffn=1376, vocab=3001, dtype="bf16", seed=21, n_planted=1, gain_std=0.05)
+
+
+@pytest.fixture(scope="module")
+def tiny_pair():
+    o, g = make_pair(TINY, max_positions=192)
+    yield o, g
+    g.close()
+
+
+@pytest.fixture(scope="module")
+def small_pair(small_cfg):
+    o, g = make_pair(small_cfg, max_positions=192, page_size=8)
+    yield o, g
+    g.close()
+
+
+@pytest.fixture(scope="module")
+def bf16_pair():
+    o, g = make_pair(BF16_SMALL, max_positions=640)
+    yield o, g
+    g.close()
+
+
+# ------------------------------------------------------------------------------ logits
+@pytest.mark.parametrize("which", ["tiny", "small"])
+def test_fp32_teacher_forced_logits(which, tiny_pair, small_pair, small_cfg):
+    (o, g), cfg = (tiny_pair, TINY) if which == "tiny" else (small_pair, small_cfg)
+    toks = synth.prompt(cfg, 45)                       # three row chunks, the last one ragged
+    ref = o.forward_rows(toks, 0)
+    g.prefill(toks[:1])
+    got, am = g.forward_rows(toks, 0)
+    assert logit_err(got, ref) < 1e-4
+    assert am.tolist() == [so.argmax_lowest(r) for r in ref]
+    # rows fed one at a time (the drafting shape) give the same logits as rows fed together
+    g.prefill(toks[:20])
+    one, _ = g.forward_rows(toks[20:21], 20)
+    assert logit_err(one, ref[20:21]) < 1e-4
+
+
+def test_fp32_skip_masks_and_no_kv_write(small_pair, small_cfg):
+    o, g = small_pair
+    toks = synth.prompt(small_cfg, 30)
+    L = 2 * small_cfg.n_blocks
+    o.prefill(toks[:19]); g.prefill(toks[:19])
+    rng = np.random.default_rng(2)
+    for z in [[1] * L, [0, 1] * (L // 2), [1, 0] * (L // 2), list(rng.integers(0, 2, L))]:
+        ref = o.forward_rows(toks[19:30], 19, z, write_kv=False)
+        got, _ = g.forward_rows(toks[19:30], 19, z, write_kv=False)
+        assert logit_err(got, ref) < 1e-4, z
+    # nothing above touched the committed cache
+    ref = o.forward_rows(toks[19:25], 19)
+    got, _ = g.forward_rows(toks[19:25], 19)
+    assert logit_err(got, ref) < 1e-4
+
+
+def test_bf16_teacher_forced_logits(bf16_pair):
+    o, g = bf16_pair
+    toks = synth.prompt(BF16_SMALL, 300)               # crosses an attention split (256 positions)
+    ref = o.forward_rows(toks, 0)
+    g.prefill(toks[:1])
+    got, _ = g.forward_rows(toks, 0)
+    err = logit_err(got, ref)
+    assert err < LOGIT_TOL, err
+    z = list(synth.block_mask(BF16_SMALL, [1]))
+    o.n = 300
+    ref = o.forward_rows(toks[290:300], 290, z, write_kv=False)
+    g.prefill(toks)
+    got, _ = g.forward_rows(toks[290:300], 290, z, write_kv=False)
+    assert logit_err(got, ref) < LOGIT_TOL
+
+
+def test_kv_cache_matches_oracle(small_pair, small_cfg):
+    o, g = small_pair
+    toks = synth.prompt(small_cfg, 21)
+    o.prefill(toks); g.prefill(toks)
+    for b in range(small_cfg.n_blocks):
+        assert np.abs(g.read_kv(b, 0, 0, 21) - o.K[b][:21].numpy()).max() < 1e-4
+        assert np.abs(g.read_kv(b, 1, 0, 21) - o.V[b][:21].numpy()).max() < 1e-4
+
+
+# ------------------------------------------------------------------------------ rounds
+@pytest.mark.parametrize("stop_conf,max_k", [(0.0, 4), (0.8, 4), (0.0005, 7), (0.0, 15)])
+def test_tiny_rounds_step_by_step(tiny_pair, stop_conf, max_k):
+    o, g = tiny_pair
+    prompt = synth.prompt(TINY, 32)
+    o.prefill(prompt)
+    assert g.prefill(prompt) == o.tokens[-1]
+    z = list(synth.block_mask(TINY, synth.planted_blocks(TINY)))
+    st = walk_rounds(o, g, z, n_rounds=12, max_k=max_k, stop_conf=stop_conf)
+    assert st["max_logit_err"] < 1e-4
+    assert st["accept_cmp"] >= 10 and st["draft_cmp"] >= 10, st
+    if stop_conf == 0.8:
+        assert st["drafted"] == st["rounds"]           # flat logits: every round stops after one draft
+
+
+def test_small_rounds_arbitrary_sublayer_masks(small_pair, small_cfg):
+    o, g = small_pair
+    prompt = synth.prompt(small_cfg, 11)
+    rng = np.random.default_rng(3)
+    for z in [[0] * 8, [1] * 8, list(rng.integers(0, 2, 8))]:
+        o.prefill(prompt); g.prefill(prompt)
+        st = walk_rounds(o, g, z, n_rounds=6, max_k=5)
+        assert st["accept_cmp"] + st["accept_exempt"] == 6 and st["max_logit_err"] < 1e-4
+        if sum(z) == 0:
+            assert st["accepted"] == st["drafted"]     # empty skip set: the draft model is the target
+
+
+def test_bf16_rounds(bf16_pair):
+    o, g = bf16_pair
+    prompt = synth.prompt(BF16_SMALL, 270)
+    o.prefill(prompt); g.prefill(prompt); g.set_pending(o.tokens[-1])
+    z = list(synth.block_mask(BF16_SMALL, synth.planted_blocks(BF16_SMALL)))
+    st = walk_rounds(o, g, z, n_rounds=8, max_k=8)
+    assert st["max_logit_err"] < LOGIT_TOL and st["accept_cmp"] >= 4, st
+
+
+# ------------------------------------------------------------------------------ whole runs
+def test_config1_generate_matches_oracle(tiny_pair):
+    """Config 1: prompt 32, 64 greedy tokens, skip set = planted blocks, max draft 4, epsilon 0.8 (and 0)."""
+    o, g = tiny_pair
+    from paper_2410_06916_b200 import GenParams
+    prompt = synth.prompt(TINY, 32)
+    z = synth.block_mask(TINY, synth.planted_blocks(TINY))
+    ref, margins = so.vanilla_generate(o, prompt, 64)
+    van, vst, _ = g.generate(prompt, GenParams(max_new=64, vanilla=True))
+    assert compare_free_running(van, ref, margins) == 64
+    for eps in (0.8, 0.0):
+        o_out, o_rounds, o_stats = so.swift_generate(o, prompt, list(z), so.GenParams(max_new=64, max_draft=4, stop_conf=eps))
+        assert o_out == ref
+        out, st, trace = g.generate(prompt, GenParams(max_new=64, max_draft=4, stop_conf=eps, skip_mask=z))
+        assert out == van                               # lossless on the GPU itself, bit for bit
+        assert st.tokens == 64 and st.rounds == len(trace)
+        assert [int(t[1]) for t in trace] == [len(r.draft) for r in o_rounds]
+        assert [int(t[2]) for t in trace] == [r.accepted for r in o_rounds]
+        assert st.accepted == o_stats["accepted"] and st.drafted == o_stats["drafted"]
+
+
+def test_gpu_swift_equals_gpu_vanilla_bf16(bf16_pair):
+    _, g = bf16_pair
+    from paper_2410_06916_b200 import GenParams
+    prompt = synth.prompt(BF16_SMALL, 64)
+    van, _, _ = g.generate(prompt, GenParams(max_new=40, vanilla=True))
+    for blocks, k in (([1], 8), ([0, 2], 5), ([], 15)):
+        out, st, _ = g.generate(prompt, GenParams(max_new=40, max_draft=k, skip_mask=synth.block_mask(BF16_SMALL, blocks)))
+        assert out == van, blocks
+        if not blocks:
+            assert st.accepted == st.drafted
+    # KV after the run equals the KV of a fresh prefill of the committed sequence
+    n = g.n
+    kv = [g.read_kv(b, w, 0, n) for b in range(BF16_SMALL.n_blocks) for w in (0, 1)]
+    g.prefill(prompt + out[:n - len(prompt)])
+    kv2 = [g.read_kv(b, w, 0, n) for b in range(BF16_SMALL.n_blocks) for w in (0, 1)]
+    for a, b in zip(kv, kv2):
+        assert np.array_equal(a, b)
+
+
+# ------------------------------------------------------------------------------ scoring
+def test_score_skipsets_matches_oracle(tiny_pair):
+    o, g = tiny_pair
+    prompt = synth.prompt(TINY, 32)
+    so.vanilla_generate(o, prompt, 40)
+    resync(g, o)
+    masks = np.concatenate([synth.candidate_masks(TINY, 4, 6, 0), np.zeros((1, 16), np.uint8),
+                            synth.block_mask(TINY, synth.planted_blocks(TINY))[None]])
+    for gamma in (32, 19):
+        ref, preds = o.score_skipsets(masks.tolist(), gamma)
+        got = g.score_skipsets(masks, gamma)
+        assert got[6] == 1.0                            # the empty set re-predicts the model's own tokens
+        for c in range(len(masks)):
+            if got[c] != pytest.approx(ref[c]):
+                rows = o.forward_rows(o.tokens[o.n - gamma:o.n], o.n - gamma, masks[c].tolist(), write_kv=False)
+                assert min(so.top2_margin(r) for r in rows) <= MARGIN, (c, got[c], ref[c])
+    assert g.n == o.n
+    ref = o.forward_rows([o.tokens[-1]], o.n)           # scoring left the committed cache untouched
+    got, _ = g.forward_rows([o.tokens[-1]], o.n)
+    assert logit_err(got, ref) < 1e-4
+
+
+def test_generate_with_on_the_fly_optimisation(tiny_pair):
+    o, g = tiny_pair
+    from paper_2410_06916_b200 import GenParams
+    prompt = synth.prompt(TINY, 32)
+    cands = np.stack([synth.candidate_masks(TINY, 4, 8, r) for r in range(3)])
+    z0 = synth.block_mask(TINY, synth.uniform_blocks(8, 4))
+    gp = so.GenParams(max_new=80, max_draft=4, gamma=32, max_opt_rounds=3)
+    o_out, o_rounds, _ = so.swift_generate(o, prompt, list(z0), gp, lambda r: cands[r])
+    out, st, trace = g.generate(prompt, GenParams(max_new=80, max_draft=4, gamma=32, n_opt_rounds=3, skip_mask=z0,
+                                                  candidate_masks=cands))
+    assert out == o_out and st.opt_rounds == 3
+    scored = [r for r in o_rounds if r.matchness is not None]
+    assert st.best_matchness == pytest.approx(max(max(r.matchness) for r in scored))
+    assert [int(t[2]) for t in trace] == [r.accepted for r in o_rounds]
+
+
+# ------------------------------------------------------------------------------ sampling
+def test_sampling_rounds_follow_the_oracle_stream(tiny_pair):
+    o, g = tiny_pair
+    prompt = synth.prompt(TINY, 32)
+    seed = 0x1234ABCD5
+    g.set_sampling(True, 1.0, seed)
+    try:
+        logits = o.prefill(prompt)
+        p = torch.softmax(logits[-1].double(), -1)
+        first, dist = so.categorical(p, so.uniform(seed, 0, 0, so.DRAW_BONUS))
+        o.tokens[-1] = first
+        g_first = g.prefill(prompt)
+        assert g_first == first or dist < 1e-3
+        g.set_pending(first)
+        z = list(synth.block_mask(TINY, synth.draft_blocks(TINY, 5)))
+        st = walk_rounds(o, g, z, n_rounds=25, max_k=4, sampling=True, seed=seed)
+        assert st["accept_cmp"] >= 20 and st["max_logit_err"] < 1e-4, st
+        assert 0 < st["accepted"] < st["drafted"]       # both the accept and the reject branch ran
+    finally:
+        g.set_sampling(False)
+
+
+def test_sampling_bf16_rounds(bf16_pair):
+    o, g = bf16_pair
+    prompt = synth.prompt(BF16_SMALL, 40)
+    seed = 4
+    g.set_sampling(True, 1.0, seed)
+    try:
+        o.prefill(prompt)
+        g.prefill(prompt); g.set_pending(o.tokens[-1])
+        z = list(synth.block_mask(BF16_SMALL, [1]))
+        st = walk_rounds(o, g, z, n_rounds=12, max_k=6, sampling=True, seed=seed, dec_tol=0.06)
+        assert st["accept_cmp"] >= 6, st
+    finally:
+        g.set_sampling(False)
+
+
+# ------------------------------------------------------------------------------ boundary behaviour
+def test_errors_are_statuses_not_crashes(small_cfg):
+    from paper_2410_06916_b200 import SwiftError, SwiftModel, GenParams
+    g = SwiftModel(small_cfg, max_positions=32, page_size=8, max_draft=4)
+    z = np.zeros(8, np.uint8)
+    with pytest.raises(SwiftError, match="ESTATE"):
+        g.draft(z, 2)
+    with pytest.raises(SwiftError, match="ESTATE"):
+        g.accept()
+    with pytest.raises(SwiftError, match="EINVAL"):
+        g.prefill([0, small_cfg.vocab])
+    with pytest.raises(SwiftError, match="ECAPACITY"):
+        g.prefill(list(range(40)))
+    g.prefill([1, 2, 3])
+    with pytest.raises(SwiftError, match="ECAPACITY"):
+        g.draft(z, 5)
+    with pytest.raises(SwiftError, match="EINVAL"):
+        g.score_skipsets(z[None], 9)
+    with pytest.raises(SwiftError, match="ECAPACITY"):
+        g.generate([1, 2, 3], GenParams(max_new=40, max_draft=2, skip_mask=z))
+    assert g.n == 3
+    toks, _ = g.draft(z, 4)
+    with pytest.raises(SwiftError, match="ESTATE"):
+        g.draft(z, 2)
+    g.verify(); g.accept()
+    assert g.n >= 4
+    g.close()
