@@ -1,0 +1,268 @@
+#!/usr/bin/env python
+"""Benchmark of the SWIFT decoding hot path on B200.
+
+One step = one complete run of the workload through the C boundary: prefill of the synthetic prompt,
+then draft / verify / accept rounds until max_new tokens are out (all with host buffers in and out).
+`value` is decode tokens/s with everything resident in HBM (CUDA-event time of the decode part, on the
+library's stream); `e2e` is tokens/s of the whole call (prefill and host<->device copies included) by
+the host clock.  Inputs are synthetic LLaMA-shaped models (see synth/), far larger than L2, so no L2
+flush is needed between steps.  Multi-GPU: replicas only (batch-1 decoding is one dependent chain);
+each rank decodes its own sequence on its own GPU and `value` sums them.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+import numpy as np  # noqa: E402
+import torch  # noqa: E402
+
+import synth  # noqa: E402
+
+METRIC = "batch-1 decode tokens/s (SWIFT self-speculative decoding)"
+UNIT = "tokens/s"
+PAPER_CONTEXT = "paper: 1.3x-1.6x over vanilla on 4x RTX A6000, FP16, HF transformers (context only)"
+
+
+def peaks():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        d = json.load(open(p))
+        return float(d["hbm_gbs"]), "measured"
+    return 6650.0, "fallback"
+
+
+class ClockSampler:
+    """Samples SM clocks and throttle reasons with nvidia-smi while the timed region runs."""
+    Q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+         "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index, self.rows, self.proc = index, [], None
+
+    def __enter__(self):
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", f"--id={self.index}", f"--query-gpu={self.Q}",
+                                          "--format=csv,noheader,nounits", "-lms", "200"],
+                                         stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.thread = threading.Thread(target=self._read, daemon=True)
+            self.thread.start()
+        except OSError:
+            self.proc = None
+        return self
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.rows.append([x.strip() for x in line.split(",")])
+
+    def __exit__(self, *a):
+        if self.proc:
+            self.proc.terminate()
+            try:
+                self.proc.wait(timeout=5)
+            except subprocess.TimeoutExpired:
+                self.proc.kill()
+
+    def summary(self):
+        sm, mx, reasons = [], 0.0, set()
+        for r in self.rows:
+            try:
+                sm.append(float(r[0])); mx = max(mx, float(r[1]))
+            except (ValueError, IndexError):
+                continue
+            for name, v in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"), r[3:7]):
+                if v.lower().startswith("active"):
+                    reasons.add(name)
+        return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": mx or None, "reasons": sorted(reasons),
+                "samples": len(sm)}
+
+
+def workload(name: str):
+    model_name, run = synth.RUNS[name]
+    cfg = synth.MODELS[model_name]
+    z = synth.block_mask(cfg, synth.draft_blocks(cfg, run.n_skip_blocks))
+    return cfg, run, z
+
+
+def oracle_sample(cfg, run, z, weights, n_ctx=16, k=2):
+    """The CPU oracle, as it stands, on a bounded slice of the workload: a short prefill, then one
+    vanilla step and one SWIFT round (k drafts + verify + accept).  Returns tokens/s of both."""
+    from oracle import swift_oracle as so
+    dtype = torch.float64 if cfg.dtype == "f32" else torch.float32
+    o = so.Oracle(so.Shape.of(cfg), weights, dtype=dtype, max_positions=n_ctx + k + 8)
+    prompt = synth.prompt(cfg, n_ctx)
+    o.prefill(prompt)
+    t0 = time.perf_counter()
+    row = o.forward_rows([o.tokens[-1]], o.n)[0]
+    o.commit([], so.argmax_lowest(row))
+    t1 = time.perf_counter()
+    d_tok, _, _ = o.draft(list(z), k)
+    tl = o.verify(d_tok)
+    a, nxt = so.accept_greedy(d_tok, tl)
+    o.commit(d_tok[:a], nxt)
+    t2 = time.perf_counter()
+    return {"vanilla": 1.0 / (t1 - t0), "swift": (a + 1) / (t2 - t1), "seconds": t2 - t0, "accepted": a, "k": k}
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=3)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="c2", choices=sorted(synth.RUNS))
+    ap.add_argument("--max-new", type=int, default=0, help="override the number of generated tokens")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+
+    cfg, run, z = workload(args.workload)
+    max_new = args.max_new or run.max_new
+    hbm_peak, peak_kind = peaks()
+    sampling = run.mode == "sampling"
+    desc = (f"{args.workload}: {cfg.name}-shaped decoder ({cfg.n_blocks} blocks, d {cfg.d_model}, {cfg.dtype}), "
+            f"prompt {run.prompt_len}, {max_new} {run.mode} tokens, {run.n_skip_blocks} blocks skipped, max draft {run.max_draft}")
+
+    if args.impl == "reference":
+        if rank != 0:
+            return
+        torch.set_num_threads(os.cpu_count() or 1)
+        small = cfg if cfg.n_blocks * cfg.block_params() < 16e9 else cfg.with_blocks(8)
+        zz = z if small is cfg else synth.block_mask(small, synth.draft_blocks(small, max(1, run.n_skip_blocks * 8 // cfg.n_blocks)))
+        w = synth.make_weights(small)
+        vals = []
+        for i in range(args.warmup + args.steps):
+            s = oracle_sample(small, run, zz, w)
+            if i >= args.warmup:
+                vals.append(s)
+        v = statistics.mean(x["swift"] for x in vals) * (small.n_blocks / cfg.n_blocks if small is not cfg else 1.0)
+        sample = "per step: prefill of 16 tokens, then one vanilla step and one SWIFT round of 2 drafts + verify + accept" + \
+                 ("" if small is cfg else f"; on an 8-block copy of the model, scaled by depth (extrapolated)")
+        print(json.dumps({"impl": "reference", "metric": METRIC, "value": v, "unit": UNIT, "n_gpus": 0, "steps": args.steps,
+                          "warmup": args.warmup, "ms_per_step": 1e3 * statistics.mean(x["seconds"] for x in vals),
+                          "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+                          "config": {"workload": desc},
+                          "cpu_baseline": {"value": v, "unit": UNIT, "cores": torch.get_num_threads(), "kind": "oracle", "sample": sample},
+                          "e2e": {"value": v, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}))
+        return
+
+    from paper_2410_06916_b200 import GenParams, SwiftModel
+    torch.cuda.set_device(local)
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    weights = synth.make_weights(cfg) if cfg.n_blocks * cfg.block_params() < 40e9 else None
+    model = SwiftModel(cfg, max_positions=run.prompt_len + max_new + 32, max_draft=run.max_draft, device=f"cuda:{local}")
+    if weights is not None:
+        model.load_weights((n, -1, weights[n]) for n in ("embed", "lm_head", "final_norm"))
+        model.load_weights((n, b, t) for b, wb in enumerate(weights["blocks"]) for n, t in wb.items())
+    else:
+        model.load_weights(synth.iter_tensors(cfg))
+    if sampling:
+        model.set_sampling(True, run.temperature, run.rng_seed)
+    prompt = synth.prompt(cfg, run.prompt_len, stream=rank)
+    cands = None
+    if run.optimise:
+        cands = np.stack([synth.candidate_masks(cfg, run.n_skip_blocks, run.n_candidates, r) for r in range(run.max_opt_rounds)])
+        z = synth.block_mask(cfg, synth.uniform_blocks(cfg.n_blocks, run.n_skip_blocks))
+    gp = GenParams(max_new=max_new, max_draft=run.max_draft, stop_conf=run.stop_conf, skip_mask=z, gamma=run.gamma,
+                   n_opt_rounds=run.max_opt_rounds if run.optimise else 0, stop_matchness=run.stop_matchness, candidate_masks=cands)
+
+    def barrier():
+        torch.cuda.synchronize()
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    for _ in range(args.warmup):
+        model.generate(prompt, gp)
+    launches0 = model.launches
+    stats = []
+    barrier()
+    with ClockSampler(local) as clk:
+        t0 = time.perf_counter()
+        for _ in range(args.steps):
+            stats.append(model.generate(prompt, gp)[1])
+        torch.cuda.synchronize()
+        wall = time.perf_counter() - t0
+    barrier()
+    launches = model.launches - launches0
+    dec_ms = sum(s.ms_decode for s in stats)
+    tot_ms = sum(s.ms_decode + s.ms_prefill for s in stats)
+    if world > 1:
+        t = torch.tensor([dec_ms, tot_ms, wall], device="cuda", dtype=torch.float64)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        dec_ms, tot_ms, wall = t.tolist()
+    tokens = sum(s.tokens - 1 for s in stats)            # the first token comes out of prefill
+    value = world * tokens / (dec_ms * 1e-3)
+    e2e = world * sum(s.tokens for s in stats) / wall
+
+    # vanilla decoding of the same model for the comparison the metric names
+    swift_tokens = model.generate(prompt, gp)[0]
+    model.generate(prompt[:64], GenParams(max_new=8, vanilla=True))
+    if sampling:
+        model.set_sampling(False)
+    v_tokens, vst, _ = model.generate(prompt, GenParams(max_new=max_new, vanilla=True))
+    vanilla = (vst.tokens - 1) / (vst.ms_decode * 1e-3)
+    lossless = None if sampling else (swift_tokens == v_tokens)   # greedy SWIFT must reproduce vanilla decoding
+
+    s0 = stats[-1]
+    n_ctx = run.prompt_len + max_new // 2
+    fw = {"draft_gbs": sum(s.bytes_draft for s in stats) / max(sum(s.ms_draft for s in stats), 1e-9) * 1e-6,
+          "verify_gbs": sum(s.bytes_verify for s in stats) / max(sum(s.ms_verify for s in stats), 1e-9) * 1e-6,
+          "vanilla_gbs": vst.bytes_verify / (vst.ms_decode * 1e-3) * 1e-9,
+          "draft_bytes": model.forward_bytes(z, 1, n_ctx), "verify_bytes": model.forward_bytes(None, run.max_draft + 1, n_ctx)}
+    fw["draft_frac"], fw["verify_frac"], fw["vanilla_frac"] = (fw[k] / hbm_peak for k in ("draft_gbs", "verify_gbs", "vanilla_gbs"))
+
+    # dominant kernel: the weight-streaming GEMM (largest instance: fused gate/up), timed alone with CUDA events
+    g_ms, g_bytes = model.time_gemm(2, run.max_draft + 1, 200)
+    g1_ms, _ = model.time_gemm(2, 1, 200)
+    achieved = g_bytes / (g_ms * 1e-3) * 1e-9
+    roofline = {"bound": "hbm", "kernel": "skinny GEMM, fused gate/up projection, %d rows" % (run.max_draft + 1),
+                "achieved": achieved, "peak": hbm_peak, "peak_kind": f"{peak_kind} copy bandwidth (burst)", "unit": "GB/s",
+                "frac": achieved / hbm_peak, "traffic": None, "bytes_per_launch": g_bytes, "ms_per_launch": g_ms,
+                "one_row_frac": g_bytes / (g1_ms * 1e-3) * 1e-9 / hbm_peak}
+
+    out = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
+           "ms_per_step": tot_ms / args.steps, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+           "dtype": "bf16" if cfg.dtype == "bf16" else "f32", "data": "synthetic",
+           "config": {"workload": desc, "l2": "inputs (weights) far larger than L2; no flush", "parallelism": "replicas only",
+                      "e2e_note": "whole swift_generate call incl. prefill and host copies, host clock", "context": PAPER_CONTEXT},
+           "vanilla_tokens_per_s": vanilla, "swift_equals_vanilla": lossless, "speedup_vs_vanilla": value / world / vanilla,
+           "M": (s0.tokens - 1) / s0.rounds, "alpha": s0.accepted / max(s0.drafted, 1), "rounds": s0.rounds,
+           "ms_prefill": s0.ms_prefill, "forwards": fw, "roofline": roofline,
+           "e2e": {"value": e2e, "unit": UNIT, "h2d_bytes_per_step": 4 * run.prompt_len, "d2h_bytes_per_step": 448 * (s0.rounds + 1)},
+           "gpu_launches": launches, "clocks": clk.summary()}
+
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        small = cfg if weights is not None and cfg.n_blocks * cfg.block_params() < 16e9 else cfg.with_blocks(8)
+        zz = z if small is cfg else synth.block_mask(small, synth.draft_blocks(small, max(1, run.n_skip_blocks * 8 // cfg.n_blocks)))
+        w = weights if small is cfg else synth.make_weights(small)
+        model.close()
+        torch.set_num_threads(os.cpu_count() or 1)
+        s = oracle_sample(small, run, zz, w)
+        scale = 1.0 if small is cfg else small.n_blocks / cfg.n_blocks
+        out["cpu_baseline"] = {"value": s["swift"] * scale, "unit": UNIT, "cores": torch.get_num_threads(), "kind": "oracle",
+                               "vanilla_value": s["vanilla"] * scale,
+                               "sample": "prefill of 16 tokens, then one vanilla step and one SWIFT round of 2 drafts + verify "
+                                         "+ accept (%.1f s of CPU work)%s" % (s["seconds"], "" if small is cfg else
+                                                                               "; 8-block copy scaled by depth (extrapolated)")}
+    if rank == 0:
+        print(json.dumps(out))
+    if world > 1:
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

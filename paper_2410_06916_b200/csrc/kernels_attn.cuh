@@ -100,10 +100,9 @@ attn_split_kernel(const DevState* st, const float* __restrict__ q, const T* __re
 }
 
 // grid = (H, rows), block = dh threads.  Combines the splits in chunk order.
-template <typename T>
 __global__ void attn_combine_kernel(const DevState* st, const float* __restrict__ o_part,
                                     const float2* __restrict__ ml_part, int max_splits, int n_heads, int dh,
-                                    T* __restrict__ out)
+                                    float* __restrict__ out)
 {
     const int r = blockIdx.y;
     if (r >= st->n_rows) return;
@@ -119,7 +118,7 @@ __global__ void attn_combine_kernel(const DevState* st, const float* __restrict_
         num += w * o_part[(((size_t)h * max_splits + s) * ROWS + r) * dh + d];
         den += w * ml.y;
     }
-    store_val(&out[((size_t)r * n_heads + h) * dh + d], num / den);
+    out[((size_t)r * n_heads + h) * dh + d] = num / den;
 }
 
 } // namespace swk

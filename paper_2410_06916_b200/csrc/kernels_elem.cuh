@@ -100,11 +100,10 @@ __global__ void embed_kernel(DevState* st, const int* __restrict__ toks, const T
 // ------------------------------------------------------------------------------ residual + RMSNorm
 // h[r,:] += sum_s part[s][r][:]  (the pending output of the previous residual branch, split-K
 // partial sums added in split order), then x[r,:] = h * rsqrt(mean(h^2) + eps) * g.
-template <typename T>
 __global__ void __launch_bounds__(512) resid_norm_kernel(const DevState* st, float* __restrict__ h,
                                                          const float* __restrict__ part, int n_split,
                                                          size_t split_stride, const float* __restrict__ gain,
-                                                         T* __restrict__ x, int d, float eps)
+                                                         float* __restrict__ x, int d, float eps)
 {
     __shared__ float red[33];
     const int r = blockIdx.x;
@@ -119,7 +118,7 @@ __global__ void __launch_bounds__(512) resid_norm_kernel(const DevState* st, flo
     }
     const float total = block_sum(ss, red);
     const float rstd = rsqrtf(total / (float)d + eps);
-    for (int i = threadIdx.x; i < d; i += blockDim.x) store_val(&x[(size_t)r * d + i], hr[i] * rstd * gain[i]);
+    for (int i = threadIdx.x; i < d; i += blockDim.x) x[(size_t)r * d + i] = hr[i] * rstd * gain[i];
 }
 
 // ------------------------------------------------------------------------------ RoPE + KV append
@@ -168,9 +167,8 @@ __global__ void qkv_post_kernel(const DevState* st, const float* __restrict__ pa
 // ------------------------------------------------------------------------------ SwiGLU
 // act[r][i] = silu(gate_i) * up_i from the fused gate/up projection, whose output columns are
 // interleaved in groups of 16: [g0..g15, u0..u15, g16..g31, u16..u31, ...].
-template <typename T>
 __global__ void swiglu_kernel(const DevState* st, const float* __restrict__ part, int n_split, size_t split_stride,
-                              T* __restrict__ act, int ffn)
+                              float* __restrict__ act, int ffn)
 {
     const int r = blockIdx.y;
     if (r >= st->n_rows) return;
@@ -183,7 +181,7 @@ __global__ void swiglu_kernel(const DevState* st, const float* __restrict__ part
         g += p[gi];
         u += p[gi + 16];
     }
-    store_val(&act[(size_t)r * ffn + i], g / (1.f + expf(-g)) * u);
+    act[(size_t)r * ffn + i] = g / (1.f + expf(-g)) * u;
 }
 
 } // namespace swk

@@ -12,11 +12,12 @@ constexpr int GEMM_SIMT_THREADS = 256;
 constexpr int GEMM_SIMT_R = 4;                                   // weight rows per warp
 constexpr int GEMM_SIMT_TILE_N = (GEMM_SIMT_THREADS / 32) * GEMM_SIMT_R;
 
-// grid = (ceil(N / 32), n_split); dynamic smem = MR * Kc * sizeof(T).
+// Activations X are fp32 (nothing but the weights and the KV cache is ever rounded to bf16); weights
+// are T.  grid = (ceil(N / 32), n_split); dynamic smem = MR * Kc * 4 bytes.
 // Kc is a multiple of 32 * VEC; K a multiple of VEC; X rows are ldx elements apart (16-byte aligned).
 template <typename T, int MR>
 __global__ void __launch_bounds__(GEMM_SIMT_THREADS)
-gemm_simt_kernel(const DevState* st, const T* __restrict__ X, int ldx, const T* __restrict__ W,
+gemm_simt_kernel(const DevState* st, const float* __restrict__ X, int ldx, const T* __restrict__ W,
                  float* __restrict__ Ypart, int N, int K, int Kc)
 {
     constexpr int VEC = Vec<T>::N;
@@ -24,7 +25,7 @@ gemm_simt_kernel(const DevState* st, const T* __restrict__ X, int ldx, const T* 
     const int n_rows = min(st->n_rows, MR);
     if (n_rows == 0) return;
     extern __shared__ __align__(16) unsigned char smem_raw[];
-    T* xs = reinterpret_cast<T*>(smem_raw);                      // [MR][Kc]
+    float* xs = reinterpret_cast<float*>(smem_raw);              // [MR][Kc]
 
     const int k0 = blockIdx.y * Kc;
     const int klen = min(Kc, K - k0);
@@ -33,10 +34,10 @@ gemm_simt_kernel(const DevState* st, const T* __restrict__ X, int ldx, const T* 
 
     // stage the X rows of this K range (rows beyond n_rows are zero)
     for (int m = 0; m < MR; ++m) {
-        for (int kk = tid * VEC; kk < klen; kk += GEMM_SIMT_THREADS * VEC) {
-            uint4 v = make_uint4(0u, 0u, 0u, 0u);
-            if (m < n_rows) v = *reinterpret_cast<const uint4*>(X + (size_t)m * ldx + k0 + kk);
-            *reinterpret_cast<uint4*>(xs + (size_t)m * Kc + kk) = v;
+        for (int kk = tid * 4; kk < klen; kk += GEMM_SIMT_THREADS * 4) {
+            float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
+            if (m < n_rows) v = *reinterpret_cast<const float4*>(X + (size_t)m * ldx + k0 + kk);
+            *reinterpret_cast<float4*>(xs + (size_t)m * Kc + kk) = v;
         }
     }
     __syncthreads();
@@ -61,7 +62,11 @@ gemm_simt_kernel(const DevState* st, const T* __restrict__ X, int ldx, const T* 
 #pragma unroll
         for (int m = 0; m < MR; ++m) {
             float x[VEC];
-            load_vec(xs + (size_t)m * Kc + kk, x);
+#pragma unroll
+            for (int e = 0; e < VEC; e += 4) {
+                const float4 v = *reinterpret_cast<const float4*>(xs + (size_t)m * Kc + kk + e);
+                x[e] = v.x; x[e + 1] = v.y; x[e + 2] = v.z; x[e + 3] = v.w;
+            }
 #pragma unroll
             for (int rr = 0; rr < R; ++rr)
 #pragma unroll

@@ -115,7 +115,7 @@ size_t esize_of(const swift_model_desc* d) { return d->dtype == SWIFT_BF16 ? 2 :
 GemmPlan plan_gemm(const swift_model_desc* d, int N, int K)
 {
     const int vec = d->dtype == SWIFT_BF16 ? 8 : 4;
-    const int kc_max = d->dtype == SWIFT_BF16 ? 2048 : 1024;
+    const int kc_max = 1024;                                // 16 rows x 1024 fp32 = 64 KB of shared memory
     const int gran = 32 * vec;
     const int tiles = ceil_div(N, GEMM_SIMT_TILE_N);
     int S = ceil_div(K, kc_max);
@@ -171,9 +171,9 @@ WorkLayout work_layout(const swift_model_desc* d)
     k.part_floats = pf;
     k.state = c.take(sizeof(DevState));
     k.h = c.take(ROWS * dm * 4);
-    k.xn = c.take(ROWS * dm * es);
-    k.xa = c.take(ROWS * qd * es);
-    k.act = c.take(ROWS * (size_t)d->ffn * es);
+    k.xn = c.take(ROWS * dm * 4);
+    k.xa = c.take(ROWS * qd * 4);
+    k.act = c.take(ROWS * (size_t)d->ffn * 4);
     k.q = c.take(ROWS * qd * 4);
     k.part = c.take(pf * 4);
     k.o_part = c.take((size_t)d->n_heads * max_splits * ROWS * d->head_dim * 4);
@@ -199,12 +199,12 @@ int mr_of(int rows) { return rows <= 1 ? 1 : rows <= 2 ? 2 : rows <= 4 ? 4 : row
 
 // ------------------------------------------------------------------------------ launches
 template <typename T, int MR>
-swift_status launch_gemm_mr(swift_ctx* ctx, const T* X, int ldx, const T* W, int N, int K, GemmPlan p)
+swift_status launch_gemm_mr(swift_ctx* ctx, const float* X, int ldx, const T* W, int N, int K, GemmPlan p)
 {
     static bool attr_set[8] = {false};
-    const size_t smem = (size_t)MR * p.Kc * sizeof(T);
+    const size_t smem = (size_t)MR * p.Kc * sizeof(float);
     if (!attr_set[ctx->device & 7]) {
-        CU(cudaFuncSetAttribute(gemm_simt_kernel<T, MR>, cudaFuncAttributeMaxDynamicSharedMemorySize, 16 * 2048 * 2 + 0));
+        CU(cudaFuncSetAttribute(gemm_simt_kernel<T, MR>, cudaFuncAttributeMaxDynamicSharedMemorySize, 16 * 1024 * 4));
         attr_set[ctx->device & 7] = true;
     }
     dim3 grid(ceil_div(N, GEMM_SIMT_TILE_N), p.S);
@@ -216,7 +216,7 @@ swift_status launch_gemm_mr(swift_ctx* ctx, const T* X, int ldx, const T* W, int
 }
 
 template <typename T>
-swift_status launch_gemm(swift_ctx* ctx, int mr, const T* X, int ldx, const T* W, int N, int K, GemmPlan* plan_out)
+swift_status launch_gemm(swift_ctx* ctx, int mr, const float* X, int ldx, const T* W, int N, int K, GemmPlan* plan_out)
 {
     const GemmPlan p = plan_gemm(&ctx->d, N, K);
     *plan_out = p;
@@ -286,9 +286,9 @@ swift_status forward_chunk(swift_ctx* ctx, int rows, const int* toks_dev, const 
     const int mr = mr_of(rows);
     const int dm = d.d_model, qd = d.n_heads * d.head_dim, kd = d.n_kv_heads * d.head_dim, nqkv = qd + 2 * kd;
     float* h = kptr<float>(ctx, ctx->kl.h);
-    T* xn = kptr<T>(ctx, ctx->kl.xn);
-    T* xa = kptr<T>(ctx, ctx->kl.xa);
-    T* act = kptr<T>(ctx, ctx->kl.act);
+    float* xn = kptr<float>(ctx, ctx->kl.xn);
+    float* xa = kptr<float>(ctx, ctx->kl.xa);
+    float* act = kptr<float>(ctx, ctx->kl.act);
     float* part = kptr<float>(ctx, ctx->kl.part);
     const float* pend = nullptr;      // pending residual-branch output (split-K partials) not yet added to h
     int pend_S = 0;
@@ -298,7 +298,7 @@ swift_status forward_chunk(swift_ctx* ctx, int rows, const int* toks_dev, const 
     ctx->launches++;
     for (int b = 0; b < d.n_blocks; ++b) {
         if (!(skip && skip[2 * b])) {
-            resid_norm_kernel<T><<<rows, 512, 0, s>>>(st, h, pend, pend_S, (size_t)ROWS * dm,
+            resid_norm_kernel<<<rows, 512, 0, s>>>(st, h, pend, pend_S, (size_t)ROWS * dm,
                                                       wptr<float>(ctx, ctx->wl.attn_norm[b]), xn, dm, d.rms_eps);
             ctx->launches++;
             ST(launch_gemm<T>(ctx, mr, xn, dm, wptr<T>(ctx, ctx->wl.wqkv[b]), nqkv, dm, &p));
@@ -307,7 +307,7 @@ swift_status forward_chunk(swift_ctx* ctx, int rows, const int* toks_dev, const 
                 page_table, ctx->kv, b, d.n_heads, kptr<float2>(ctx, ctx->kl.rope), d.max_positions);
             ctx->launches++;
             ST(launch_attn<T>(ctx, mr, page_table, b));
-            attn_combine_kernel<T><<<dim3(d.n_heads, rows), d.head_dim, 0, s>>>(
+            attn_combine_kernel<<<dim3(d.n_heads, rows), d.head_dim, 0, s>>>(
                 st, kptr<float>(ctx, ctx->kl.o_part), kptr<float2>(ctx, ctx->kl.ml_part), ctx->max_splits, d.n_heads,
                 d.head_dim, xa);
             ctx->launches++;
@@ -315,11 +315,11 @@ swift_status forward_chunk(swift_ctx* ctx, int rows, const int* toks_dev, const 
             pend = part; pend_S = p.S;
         }
         if (!(skip && skip[2 * b + 1])) {
-            resid_norm_kernel<T><<<rows, 512, 0, s>>>(st, h, pend, pend_S, (size_t)ROWS * dm,
+            resid_norm_kernel<<<rows, 512, 0, s>>>(st, h, pend, pend_S, (size_t)ROWS * dm,
                                                       wptr<float>(ctx, ctx->wl.mlp_norm[b]), xn, dm, d.rms_eps);
             ctx->launches++;
             ST(launch_gemm<T>(ctx, mr, xn, dm, wptr<T>(ctx, ctx->wl.wgu[b]), 2 * d.ffn, dm, &p));
-            swiglu_kernel<T><<<dim3(ceil_div(d.ffn, 256), rows), 256, 0, s>>>(st, part, p.S, (size_t)ROWS * 2 * d.ffn, act,
+            swiglu_kernel<<<dim3(ceil_div(d.ffn, 256), rows), 256, 0, s>>>(st, part, p.S, (size_t)ROWS * 2 * d.ffn, act,
                                                                             d.ffn);
             ctx->launches++;
             ST(launch_gemm<T>(ctx, mr, act, d.ffn, wptr<T>(ctx, ctx->wl.wdown[b]), dm, d.ffn, &p));
@@ -327,7 +327,7 @@ swift_status forward_chunk(swift_ctx* ctx, int rows, const int* toks_dev, const 
         }
     }
     if (head.run) {
-        resid_norm_kernel<T><<<rows, 512, 0, s>>>(st, h, pend, pend_S, (size_t)ROWS * dm,
+        resid_norm_kernel<<<rows, 512, 0, s>>>(st, h, pend, pend_S, (size_t)ROWS * dm,
                                                   wptr<float>(ctx, ctx->wl.final_norm), xn, dm, d.rms_eps);
         ctx->launches++;
         ST(launch_gemm<T>(ctx, mr, xn, dm, wptr<T>(ctx, ctx->wl.lm_head), d.vocab, dm, &p));
@@ -838,7 +838,7 @@ static swift_status time_gemm_t(swift_ctx* ctx, int which, int n_rows, int iters
     const int dm = d.d_model, qd = d.n_heads * d.head_dim, kd = d.n_kv_heads * d.head_dim;
     const int N = which == 0 ? qd + 2 * kd : which == 1 ? dm : which == 2 ? 2 * d.ffn : which == 3 ? dm : d.vocab;
     const int K = which == 1 ? qd : which == 3 ? d.ffn : dm;
-    const T* X = which == 1 ? kptr<T>(ctx, ctx->kl.xa) : which == 3 ? kptr<T>(ctx, ctx->kl.act) : kptr<T>(ctx, ctx->kl.xn);
+    const float* X = which == 1 ? kptr<float>(ctx, ctx->kl.xa) : which == 3 ? kptr<float>(ctx, ctx->kl.act) : kptr<float>(ctx, ctx->kl.xn);
     set_rows_kernel<<<1, 1, 0, ctx->stream>>>(state_of(ctx), 0, n_rows);
     ctx->launches++;
     GemmPlan p;

@@ -102,12 +102,15 @@ class RunConfig:
     stop_matchness: float = 0.95
 
 
-# The five benchmark shapes.  Seeds other than the first are this repository's choice.
+# The five benchmark shapes.  Seeds other than the first are this repository's choice: the lowest
+# seed whose planted set leaves the first three blocks alone.  With N(0, 0.02) everywhere the token
+# embedding is small (0.02 per element) next to a block's output (order 1), so a planted block at the
+# very start still contributes as much as the embedding itself and skipping it is not "nearly free".
 MODELS: Dict[str, ModelConfig] = {
     "tiny": ModelConfig("tiny", 8, 256, 4, 4, 64, 688, 2048, "f32", seed=0, n_planted=4),
-    "7b": ModelConfig("7b", 32, 4096, 32, 32, 128, 11008, 32000, "bf16", seed=1, n_planted=14),
-    "13b": ModelConfig("13b", 40, 5120, 40, 40, 128, 13824, 32000, "bf16", seed=2, n_planted=18),
-    "70b": ModelConfig("70b", 80, 8192, 64, 8, 128, 28672, 32000, "bf16", seed=3, n_planted=36),
+    "7b": ModelConfig("7b", 32, 4096, 32, 32, 128, 11008, 32000, "bf16", seed=2, n_planted=14),
+    "13b": ModelConfig("13b", 40, 5120, 40, 40, 128, 13824, 32000, "bf16", seed=3, n_planted=18),
+    "70b": ModelConfig("70b", 80, 8192, 64, 8, 128, 28672, 32000, "bf16", seed=6, n_planted=36),
 }
 RUNS: Dict[str, Tuple[str, RunConfig]] = {
     "c1": ("tiny", RunConfig(32, 64, 4, stop_conf=0.8, n_skip_blocks=4)),

