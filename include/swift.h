@@ -49,12 +49,12 @@ enum { SWIFT_MAX_ROWS = 16 }; /* rows of one forward pass: pending token + at mo
 /* Decoder shape (LLaMA-style, the family the paper evaluates, Section 5.1). */
 typedef struct {
     int32_t n_blocks, d_model, n_heads, n_kv_heads, head_dim, ffn, vocab;
-    int32_t dtype;          /* SWIFT_F32 or SWIFT_BF16: storage of weights, GEMM inputs and KV cache */
+    int32_t dtype;          /* SWIFT_F32 or SWIFT_BF16: storage of the weights (activations are always fp32) */
     float rope_theta, rms_eps;
     int32_t max_positions;  /* KV capacity in positions; multiple of page_size */
     int32_t page_size;      /* positions per KV page; power of two, 8..128 */
     int32_t max_draft;      /* largest k any call will use; <= SWIFT_MAX_ROWS - 1 */
-    int32_t reserved;
+    int32_t kv_dtype;       /* SWIFT_F32 or SWIFT_BF16: storage of cached K,V (fp32 models: SWIFT_F32) */
 } swift_model_desc;
 
 typedef struct { void* dptr; size_t bytes; } swift_devbuf; /* caller-owned device memory, 256-byte aligned */
@@ -185,6 +185,17 @@ typedef struct {
 swift_status swift_generate(swift_ctx* ctx, const swift_gen_params* params, const int32_t* prompt_host,
                             int32_t n_prompt, int32_t* out_tokens_host, int32_t* n_out_host,
                             int32_t* trace_host, swift_stats* stats);
+
+/* Selects the kernel behind the weight-streaming GEMMs: 1 = tensor cores (tcgen05 + TMA; default and
+ * only sensible choice for bf16 models), 0 = the SIMT kernel (always used for fp32 models; for bf16 it
+ * exists so that tests can check one kernel against the other).  No open round. */
+swift_status swift_set_gemm_impl(swift_ctx* ctx, int32_t impl);
+
+/* One weight-streaming GEMM of the walk on caller data: y[r][n] = sum_k x[r][k] * W[n][k] with W the
+ * stored weight `which` (0 fused QKV, 1 o_proj, 2 fused gate/up in its interleaved row order, 3 down,
+ * 4 output head) of `block`.  x_host: fp32 [n_rows][K], y_host: fp32 [n_rows][N], n_rows <= 16. */
+swift_status swift_gemm(swift_ctx* ctx, int32_t which, int32_t block, const float* x_host, int32_t n_rows,
+                        float* y_host);
 
 /* Introspection used by tests and the benchmark. */
 int32_t swift_committed_length(const swift_ctx* ctx);               /* n; -1 if ctx is NULL */

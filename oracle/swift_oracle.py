@@ -109,6 +109,11 @@ def attention(q: torch.Tensor, K: torch.Tensor, V: torch.Tensor, allowed: torch.
     return out
 
 
+def linear(x: torch.Tensor, W: torch.Tensor) -> torch.Tensor:
+    """y = x W^T in fp64: the projection every sub-layer applies (weights stored [out, in])."""
+    return x.to(torch.float64) @ W.to(torch.float64).T
+
+
 def swiglu(gate: torch.Tensor, up: torch.Tensor) -> torch.Tensor:
     return gate * torch.sigmoid(gate) * up
 

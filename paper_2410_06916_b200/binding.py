@@ -29,7 +29,7 @@ class _Desc(C.Structure):
     _fields_ = [(n, C.c_int32) for n in ("n_blocks", "d_model", "n_heads", "n_kv_heads", "head_dim", "ffn", "vocab",
                                          "dtype")] + \
                [("rope_theta", C.c_float), ("rms_eps", C.c_float)] + \
-               [(n, C.c_int32) for n in ("max_positions", "page_size", "max_draft", "reserved")]
+               [(n, C.c_int32) for n in ("max_positions", "page_size", "max_draft", "kv_dtype")]
 
 
 class _DevBuf(C.Structure):
@@ -52,7 +52,7 @@ class _Stats(C.Structure):
 SYMBOLS = ("swift_weights_bytes", "swift_kv_bytes", "swift_workspace_bytes", "swift_load", "swift_free",
            "swift_last_error", "swift_pack_tensor", "swift_set_sampling", "swift_forward_rows", "swift_prefill",
            "swift_set_pending", "swift_draft", "swift_verify", "swift_accept", "swift_score_skipsets", "swift_generate",
-           "swift_committed_length", "swift_launch_count", "swift_forward_bytes", "swift_read_kv", "swift_time_gemm")
+           "swift_committed_length", "swift_launch_count", "swift_forward_bytes", "swift_read_kv", "swift_time_gemm", "swift_set_gemm_impl", "swift_gemm")
 
 _lib = None
 
@@ -87,6 +87,8 @@ def load_library(path: Optional[str] = None) -> C.CDLL:
     lib.swift_launch_count.restype = C.c_int64
     lib.swift_forward_bytes.argtypes = [vp, vp, i32, i32]
     lib.swift_forward_bytes.restype = C.c_double
+    lib.swift_set_gemm_impl.argtypes = [vp, i32]
+    lib.swift_gemm.argtypes = [vp, i32, i32, vp, i32, vp]
     lib.swift_time_gemm.argtypes = [vp, i32, i32, i32, vp, vp]
     lib.swift_read_kv.argtypes = [vp, i32, i32, i32, i32, vp]
     for name in SYMBOLS:
@@ -148,7 +150,10 @@ def _ptr(a: Optional[np.ndarray]):
 class SwiftModel:
     """One model + KV cache + workspace on one GPU, driven through the C boundary."""
 
-    def __init__(self, cfg, max_positions: int, page_size: int = 16, max_draft: int = 15, device: str = "cuda:0"):
+    def __init__(self, cfg, max_positions: int, page_size: int = 16, max_draft: int = 15, device: str = "cuda:0",
+                 kv_dtype: str = "f32"):
+        """kv_dtype: storage of cached K,V: "f32" (default: keeps the logits within the parity tolerance) or
+        "bf16" (halves the cache and its traffic; fp32 models always use "f32")."""
         if not torch.cuda.is_available():
             raise RuntimeError("paper_2410_06916_b200 needs a CUDA device (B200); there is no CPU path")
         self._lib = lib()
@@ -157,7 +162,7 @@ class SwiftModel:
         max_positions = (max_positions + page_size - 1) // page_size * page_size
         self.desc = _Desc(cfg.n_blocks, cfg.d_model, cfg.n_heads, cfg.n_kv_heads, cfg.head_dim, cfg.ffn, cfg.vocab,
                           1 if cfg.dtype == "bf16" else 0, cfg.rope_theta, cfg.rms_eps, max_positions, page_size,
-                          max_draft, 0)
+                          max_draft, 1 if (kv_dtype == "bf16" and cfg.dtype == "bf16") else 0)
         sizes = [self._lib.swift_weights_bytes(C.byref(self.desc)), self._lib.swift_kv_bytes(C.byref(self.desc)),
                  self._lib.swift_workspace_bytes(C.byref(self.desc))]
         if 0 in sizes:
@@ -291,6 +296,19 @@ class SwiftModel:
                                                  _ptr(trace), C.byref(st)))
         stats = GenStats(**{f: getattr(st, f) for f in GenStats.__dataclass_fields__})
         return out[:n_out.value].tolist(), stats, trace[:stats.rounds]
+
+    def set_gemm_impl(self, tensor_cores: bool):
+        self._check(self._lib.swift_set_gemm_impl(self.ctx, 1 if tensor_cores else 0))
+
+    def gemm(self, which: int, block: int, x: np.ndarray) -> np.ndarray:
+        """y = x @ W^T for one stored weight (fused / interleaved row order), through the library's GEMM kernel."""
+        x = np.ascontiguousarray(x, dtype=np.float32)
+        c = self.cfg
+        n = [c.q_dim + 2 * c.kv_dim, c.d_model, 2 * c.ffn, c.d_model, c.vocab][which]
+        y = np.empty((x.shape[0], n), dtype=np.float32)
+        with torch.cuda.device(self.device):
+            self._check(self._lib.swift_gemm(self.ctx, which, block, _ptr(x), x.shape[0], _ptr(y)))
+        return y
 
     def time_gemm(self, which: int, n_rows: int, iters: int) -> Tuple[float, float]:
         """(ms per launch, weight bytes per launch) of one weight-streaming GEMM of the walk."""

@@ -4,6 +4,7 @@
 // does not depend on how many other rows are in flight.
 #pragma once
 #include "common.cuh"
+#include "kernels_gemm_tc.cuh"
 
 namespace swk {
 
@@ -102,7 +103,7 @@ attn_split_kernel(const DevState* st, const float* __restrict__ q, const T* __re
 // grid = (H, rows), block = dh threads.  Combines the splits in chunk order.
 __global__ void attn_combine_kernel(const DevState* st, const float* __restrict__ o_part,
                                     const float2* __restrict__ ml_part, int max_splits, int n_heads, int dh,
-                                    float* __restrict__ out)
+                                    float* __restrict__ out, __nv_bfloat16* __restrict__ planes)
 {
     const int r = blockIdx.y;
     if (r >= st->n_rows) return;
@@ -118,7 +119,9 @@ __global__ void attn_combine_kernel(const DevState* st, const float* __restrict_
         num += w * o_part[(((size_t)h * max_splits + s) * ROWS + r) * dh + d];
         den += w * ml.y;
     }
-    out[((size_t)r * n_heads + h) * dh + d] = num / den;
+    const float v = num / den;
+    out[((size_t)r * n_heads + h) * dh + d] = v;
+    if (planes) store_hi_lo(planes, r, n_heads * dh, h * dh + d, v);
 }
 
 } // namespace swk

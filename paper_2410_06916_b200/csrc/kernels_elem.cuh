@@ -3,6 +3,7 @@
 // position from the device-resident DevState and do nothing when it holds zero rows.
 #pragma once
 #include "common.cuh"
+#include "kernels_gemm_tc.cuh"
 
 namespace swk {
 
@@ -103,7 +104,8 @@ __global__ void embed_kernel(DevState* st, const int* __restrict__ toks, const T
 __global__ void __launch_bounds__(512) resid_norm_kernel(const DevState* st, float* __restrict__ h,
                                                          const float* __restrict__ part, int n_split,
                                                          size_t split_stride, const float* __restrict__ gain,
-                                                         float* __restrict__ x, int d, float eps)
+                                                         float* __restrict__ x, __nv_bfloat16* __restrict__ planes,
+                                                         int d, float eps)
 {
     __shared__ float red[33];
     const int r = blockIdx.x;
@@ -118,7 +120,11 @@ __global__ void __launch_bounds__(512) resid_norm_kernel(const DevState* st, flo
     }
     const float total = block_sum(ss, red);
     const float rstd = rsqrtf(total / (float)d + eps);
-    for (int i = threadIdx.x; i < d; i += blockDim.x) x[(size_t)r * d + i] = hr[i] * rstd * gain[i];
+    for (int i = threadIdx.x; i < d; i += blockDim.x) {
+        const float v = hr[i] * rstd * gain[i];
+        x[(size_t)r * d + i] = v;
+        if (planes) store_hi_lo(planes, r, d, i, v);
+    }
 }
 
 // ------------------------------------------------------------------------------ RoPE + KV append
@@ -168,7 +174,7 @@ __global__ void qkv_post_kernel(const DevState* st, const float* __restrict__ pa
 // act[r][i] = silu(gate_i) * up_i from the fused gate/up projection, whose output columns are
 // interleaved in groups of 16: [g0..g15, u0..u15, g16..g31, u16..u31, ...].
 __global__ void swiglu_kernel(const DevState* st, const float* __restrict__ part, int n_split, size_t split_stride,
-                              float* __restrict__ act, int ffn)
+                              float* __restrict__ act, __nv_bfloat16* __restrict__ planes, int ffn)
 {
     const int r = blockIdx.y;
     if (r >= st->n_rows) return;
@@ -181,7 +187,9 @@ __global__ void swiglu_kernel(const DevState* st, const float* __restrict__ part
         g += p[gi];
         u += p[gi + 16];
     }
-    act[(size_t)r * ffn + i] = g / (1.f + expf(-g)) * u;
+    const float v = g / (1.f + expf(-g)) * u;
+    act[(size_t)r * ffn + i] = v;
+    if (planes) store_hi_lo(planes, r, ffn, i, v);
 }
 
 } // namespace swk

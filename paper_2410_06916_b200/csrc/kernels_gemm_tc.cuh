@@ -1,0 +1,293 @@
+// Skinny weight-streaming GEMM on the 5th-generation tensor cores (sm_100a):
+//     Y[r][n] = sum_k X[r][k] * W[n][k],   r < 16 rows,  W bf16 [N][K] streamed once from HBM.
+//
+// The contraction is "swapped": the 128 weight rows of a tile are the M side of tcgen05.mma, the
+// rows of X are its N side.  X is fp32 upstream; it reaches the tensor cores as two bf16 planes,
+// hi = bf16(x) and lo = bf16(x - hi), stacked as 32 operand rows, and the epilogue adds the two
+// accumulator columns, so activations keep ~16 mantissa bits while the weights stay the only
+// rounded quantity.  The kernel is HBM-bound (<= 26 flop per weight byte); tensor cores are simply
+// the cheapest way to keep the arithmetic out of the way.
+//
+// Work decomposition (stream-K): the (tile, 64-wide k-block) units are numbered tile-major and cut
+// into gridDim.x equal contiguous ranges, one per persistent CTA, so every SM streams the same
+// number of bytes whatever N and K are.  A CTA whose range covers only part of a tile writes its
+// partial accumulator to a slab; the last CTA to finish a tile (per-tile arrival counter) adds the
+// slabs in slab order and writes Y, which makes the result independent of arrival order and of the
+// row count.
+//
+// Pipeline per CTA: warp 0 issues TMA loads (weights 128x64 + activations 32x64 per stage, 128-byte
+// swizzle) into an 8-stage shared-memory ring guarded by mbarriers; warp 1 issues tcgen05.mma from
+// shared memory into a double-buffered TMEM accumulator; warps 2-5 drain TMEM with tcgen05.ld, add
+// the hi/lo columns and store.  Every mbarrier wait is bounded; on expiry the kernel records an
+// error and winds down (TMEM is always released).
+#pragma once
+#include <cuda.h>
+
+#include "common.cuh"
+
+namespace swk {
+
+constexpr int TC_TILE_N = 128;      // weight rows per tile (MMA M)
+constexpr int TC_COLS = 32;         // operand rows of X: 16 hi + 16 lo (MMA N)
+constexpr int TC_BK = 64;           // k elements per stage: 128 bytes of bf16 = one swizzle row
+constexpr int TC_STAGES = 8;
+constexpr int TC_THREADS = 192;
+constexpr int TC_A_BYTES = TC_TILE_N * TC_BK * 2;   // 16384
+constexpr int TC_B_BYTES = TC_COLS * TC_BK * 2;     // 4096
+constexpr int TC_STAGE_BYTES = TC_A_BYTES + TC_B_BYTES;
+constexpr int TC_SMEM_BYTES = TC_STAGES * TC_STAGE_BYTES + 1024 /*alignment slack*/ + 256 /*barriers*/;
+constexpr long long TC_WAIT_CYCLES = 3000000000LL;  // ~1.5 s of SM clocks before a wait is declared dead
+constexpr int TC_ERR_TIMEOUT = 2;
+
+// ------------------------------------------------------------------------------ PTX wrappers
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count)
+{
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count));
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes)
+{
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar)
+{
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+// Bounded wait on a phase parity.  Returns false when the limit ran out.
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity)
+{
+    const long long t0 = clock64();
+    for (uint32_t it = 0;; ++it) {
+        uint32_t ok;
+        asm volatile(
+            "{\n\t.reg .pred p;\n\t"
+            "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+            "selp.u32 %0, 1, 0, p;\n\t}"
+            : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+        if (ok) return true;
+        if ((it & 63u) == 63u && clock64() - t0 > TC_WAIT_CYCLES) return false;
+    }
+}
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, int c0, int c1, uint32_t bar)
+{
+    asm volatile(
+        "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
+        ::"r"(dst), "l"(map), "r"(bar), "r"(c0), "r"(c1) : "memory");
+}
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_commit(uint32_t bar)
+{
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+// D[tmem] (+)= A[smem] * B[smem]; bf16 inputs, fp32 accumulate, M = 128, N = 32, K = 16
+__device__ __forceinline__ void tc_mma(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, uint32_t accumulate)
+{
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+        ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate) : "memory");
+}
+// Shared-memory operand descriptor: K-major tile whose rows are 128 bytes, 128-byte swizzle, groups
+// of 8 rows 1024 bytes apart; descriptor version 1 (sm_100).
+__device__ __forceinline__ uint64_t tc_smem_desc(uint32_t addr)
+{
+    return (uint64_t)((addr >> 4) & 0x3FFFu) | ((uint64_t)(1024 >> 4) << 32) | ((uint64_t)1 << 46) | ((uint64_t)2 << 61);
+}
+// Instruction descriptor: D fp32, A and B bf16, both K-major, N = 32, M = 128.
+constexpr uint32_t TC_IDESC = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(TC_COLS >> 3) << 17) | ((uint32_t)(TC_TILE_N >> 4) << 24);
+
+// Static stream-K schedule shared by host and device: CTA g owns units [start(g), start(g+1)).
+struct StreamK {
+    long long U;   // units = n_tiles * KB
+    int G, KB;
+    __host__ __device__ long long start(int g) const { return (U * g) / G; }
+    __host__ __device__ int owner(long long u) const      // the CTA whose range contains unit u
+    {
+        int g = (int)((u * G) / U);
+        while (g + 1 < G && start(g + 1) <= u) ++g;
+        while (g > 0 && start(g) > u) --g;
+        return g;
+    }
+};
+
+// grid = G persistent CTAs, block = 192 threads, dynamic smem = TC_SMEM_BYTES.
+// mapW: bf16 [N][K], box {64, 128}; mapX: bf16 [32][K] (rows 0-15 hi, 16-31 lo), box {64, 32}; both
+// 128-byte swizzled.  slabs: [S_max][ROWS][N] fp32; counters: one int per tile, zero on entry and on exit.
+__global__ void __launch_bounds__(TC_THREADS, 1)
+gemm_tc_kernel(DevState* st, const __grid_constant__ CUtensorMap mapW, const __grid_constant__ CUtensorMap mapX,
+               float* __restrict__ Y, float* __restrict__ slabs, int* __restrict__ counters, int N, int K)
+{
+    const int n_rows = st->n_rows;
+    if (n_rows == 0) return;
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int n_tiles = (N + TC_TILE_N - 1) / TC_TILE_N;
+    StreamK sk;
+    sk.KB = (K + TC_BK - 1) / TC_BK;
+    sk.U = (long long)n_tiles * sk.KB;
+    sk.G = (int)(sk.U < (long long)gridDim.x ? sk.U : (long long)gridDim.x);   // never more CTAs than units: no empty ranges
+    if ((int)blockIdx.x >= sk.G) return;
+    const long long u_begin = sk.start(blockIdx.x), u_end = sk.start(blockIdx.x + 1);
+
+    extern __shared__ unsigned char smem_raw[];
+    const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;        // swizzled tiles need 1024-byte alignment
+    const uint32_t bars = base + TC_STAGES * TC_STAGE_BYTES;            // full[8], empty[8], tfull[2], tempty[2]
+    auto full_bar = [&](int s) { return bars + 8u * s; };
+    auto empty_bar = [&](int s) { return bars + 8u * (TC_STAGES + s); };
+    auto tfull_bar = [&](int b) { return bars + 8u * (2 * TC_STAGES + b); };
+    auto tempty_bar = [&](int b) { return bars + 8u * (2 * TC_STAGES + 2 + b); };
+    __shared__ uint32_t tmem_base_sh;
+    __shared__ int last_flag_sh;
+    __shared__ int abort_sh, epi_abort_sh;
+
+    if (tid == 0) {
+        for (int s = 0; s < TC_STAGES; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
+        for (int b = 0; b < 2; ++b) { mbar_init(tfull_bar(b), 1); mbar_init(tempty_bar(b), 4); }
+        abort_sh = 0;
+        epi_abort_sh = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (warp == 1) {   // one warp allocates 64 TMEM columns: two accumulator buffers of 32
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&tmem_base_sh)), "r"(64));
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;");
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = tmem_base_sh;
+
+    if (warp == 0) {
+        // ---------------------------------------------------------------- TMA producer
+        if (lane == 0) {
+            asm volatile("prefetch.tensormap [%0];" ::"l"(&mapW) : "memory");
+            asm volatile("prefetch.tensormap [%0];" ::"l"(&mapX) : "memory");
+            int it = 0;
+            for (long long u = u_begin; u < u_end; ++u, ++it) {
+                const int tile = (int)(u / sk.KB), kb = (int)(u % sk.KB);
+                const int s = it % TC_STAGES;
+                if (!mbar_wait(empty_bar(s), ((it / TC_STAGES) & 1) ^ 1)) { abort_sh = 1; break; }
+                const uint32_t a_dst = base + s * TC_STAGE_BYTES, b_dst = a_dst + TC_A_BYTES;
+                mbar_expect_tx(full_bar(s), TC_STAGE_BYTES);
+                tma_load_2d(a_dst, &mapW, kb * TC_BK, tile * TC_TILE_N, full_bar(s));
+                tma_load_2d(b_dst, &mapX, kb * TC_BK, 0, full_bar(s));
+            }
+        }
+    } else if (warp == 1) {
+        // ---------------------------------------------------------------- MMA issuer
+        if (lane == 0) {
+            int it = 0, seg = 0;
+            for (long long u = u_begin; u < u_end; ++u, ++it) {
+                const int tile = (int)(u / sk.KB), kb = (int)(u % sk.KB);
+                const bool seg_first = (u == u_begin) || kb == 0;
+                const bool seg_last = (u + 1 == u_end) || kb == sk.KB - 1;
+                const int buf = seg & 1;
+                (void)tile;
+                if (seg_first) {   // the epilogue must have drained this accumulator buffer (two segments ago)
+                    if (!mbar_wait(tempty_bar(buf), ((seg >> 1) & 1) ^ 1)) { abort_sh = 1; break; }
+                    tc_fence_after();
+                }
+                const int s = it % TC_STAGES;
+                if (!mbar_wait(full_bar(s), (it / TC_STAGES) & 1)) { abort_sh = 1; break; }
+                tc_fence_after();
+                const uint32_t a_addr = base + s * TC_STAGE_BYTES, b_addr = a_addr + TC_A_BYTES;
+                const uint64_t a_desc = tc_smem_desc(a_addr), b_desc = tc_smem_desc(b_addr);
+#pragma unroll
+                for (int k = 0; k < TC_BK / 16; ++k)   // 16 bf16 = 32 bytes further along the swizzled row
+                    tc_mma(tmem_base + buf * TC_COLS, a_desc + 2 * k, b_desc + 2 * k, TC_IDESC, (seg_first && k == 0) ? 0u : 1u);
+                tc_commit(empty_bar(s));               // smem stage reusable once these MMAs have read it
+                if (seg_last) { tc_commit(tfull_bar(buf)); ++seg; }
+            }
+        }
+    } else {
+        // ---------------------------------------------------------------- epilogue (warps 2..5)
+        const int quarter = warp & 3;                  // TMEM lanes this warp may read: 32*quarter ..
+        const int etid = tid - 64;                     // 0..127
+        int seg = 0;
+        long long u = u_begin;
+        while (u < u_end) {
+            const int tile = (int)(u / sk.KB), kb0 = (int)(u % sk.KB);
+            const long long tile_end = (long long)(tile + 1) * sk.KB;
+            const long long seg_end = tile_end < u_end ? tile_end : u_end;
+            const int buf = seg & 1;
+            if (!mbar_wait(tfull_bar(buf), (seg >> 1) & 1)) epi_abort_sh = 1;
+            asm volatile("bar.sync 1, 128;" ::: "memory");     // all four warps agree before anyone leaves the loop
+            if (epi_abort_sh) { abort_sh = 1; break; }
+            tc_fence_after();
+            uint32_t v[32];
+            const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(buf * TC_COLS);
+            asm volatile(
+                "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+                "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+                "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+                : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]),
+                  "=r"(v[8]), "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15]),
+                  "=r"(v[16]), "=r"(v[17]), "=r"(v[18]), "=r"(v[19]), "=r"(v[20]), "=r"(v[21]), "=r"(v[22]), "=r"(v[23]),
+                  "=r"(v[24]), "=r"(v[25]), "=r"(v[26]), "=r"(v[27]), "=r"(v[28]), "=r"(v[29]), "=r"(v[30]), "=r"(v[31])
+                : "r"(taddr));
+            asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(tempty_bar(buf));       // accumulator buffer free again (4 warps arrive)
+
+            const int n = tile * TC_TILE_N + quarter * 32 + lane;
+            const bool whole = (kb0 == 0) && (seg_end == tile_end);   // this CTA covered the tile's whole K range
+            if (whole) {
+                if (n < N)
+                    for (int m = 0; m < ROWS; ++m)
+                        if (m < n_rows) Y[(size_t)m * N + n] = __uint_as_float(v[m]) + __uint_as_float(v[16 + m]);
+            } else {
+                const int g_first = sk.owner((long long)tile * sk.KB), g_last = sk.owner(tile_end - 1);
+                const int slab = blockIdx.x - g_first, nseg = g_last - g_first + 1;
+                float* mine = slabs + (size_t)slab * ROWS * N;
+                if (n < N)
+                    for (int m = 0; m < ROWS; ++m)
+                        if (m < n_rows) mine[(size_t)m * N + n] = __uint_as_float(v[m]) + __uint_as_float(v[16 + m]);
+                __threadfence();
+                asm volatile("bar.sync 1, 128;" ::: "memory");
+                if (etid == 0) last_flag_sh = (atomicAdd(&counters[tile], 1) == nseg - 1) ? 1 : 0;
+                asm volatile("bar.sync 1, 128;" ::: "memory");
+                if (last_flag_sh) {                             // last arrival: add the slabs in slab order
+                    __threadfence();
+                    if (n < N)
+                        for (int m = 0; m < ROWS; ++m)
+                            if (m < n_rows) {
+                                float acc = 0.f;
+                                for (int j = 0; j < nseg; ++j) acc += __ldcg(slabs + ((size_t)j * ROWS + m) * N + n);
+                                Y[(size_t)m * N + n] = acc;
+                            }
+                    if (etid == 0) counters[tile] = 0;
+                }
+                asm volatile("bar.sync 1, 128;" ::: "memory");  // last_flag_sh is rewritten by the next segment
+            }
+            ++seg;
+            u = seg_end;
+        }
+    }
+
+    tc_fence_before();
+    __syncthreads();
+    if (abort_sh && tid == 0) st->error = TC_ERR_TIMEOUT;
+    if (warp == 1) {
+        tc_fence_after();
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(64));
+    }
+}
+
+// fp32 rows -> the two bf16 planes the tensor-core GEMM reads: plane[r] = bf16(x), plane[16 + r] = bf16(x - hi).
+__device__ __forceinline__ void store_hi_lo(__nv_bfloat16* planes, int r, int K, int i, float x)
+{
+    const __nv_bfloat16 hi = __float2bfloat16_rn(x);
+    planes[(size_t)r * K + i] = hi;
+    planes[(size_t)(ROWS + r) * K + i] = __float2bfloat16_rn(x - __bfloat162float(hi));
+}
+
+// grid = (ceil(K/256), rows): splits fp32 rows [rows][K] into the planes (used when a caller supplies X directly)
+__global__ void split_planes_kernel(const float* __restrict__ x, __nv_bfloat16* __restrict__ planes, int K)
+{
+    const int r = blockIdx.y, i = blockIdx.x * blockDim.x + threadIdx.x;
+    if (i < K) store_hi_lo(planes, r, K, i, x[(size_t)r * K + i]);
+}
+
+} // namespace swk

@@ -2,6 +2,8 @@
 // enqueues the kernels of one forward chunk, and the extern "C" entry points of include/swift.h.
 #include "../../include/swift.h"
 
+#include <cuda.h>
+#include <cudaTypedefs.h>
 #include <cuda_runtime.h>
 
 #include <algorithm>
@@ -15,6 +17,7 @@
 #include "kernels_attn.cuh"
 #include "kernels_elem.cuh"
 #include "kernels_gemm_simt.cuh"
+#include "kernels_gemm_tc.cuh"
 #include "kernels_vocab.cuh"
 
 using namespace swk;
@@ -44,8 +47,8 @@ struct WeightLayout {
 
 struct WorkLayout {
     size_t state, h, xn, xa, act, q, part, o_part, ml_part, logits, q_rows, rope, pt_main, pt_score, score_tok,
-        score_truth, score_out, total;
-    size_t part_floats;
+        score_truth, score_out, xn_hl, xa_hl, act_hl, slabs, counters, total;
+    size_t part_floats, slab_floats;
 };
 
 } // namespace
@@ -68,6 +71,10 @@ struct swift_ctx {
     int64_t launches;
     std::string err;
     cudaEvent_t ev[8];
+    // tensor-core GEMM path (bf16 models)
+    bool use_tc;
+    std::vector<CUtensorMap> tm_wqkv, tm_wo, tm_wgu, tm_wdown;
+    CUtensorMap tm_lm_head, tm_embed, tm_xn, tm_xa, tm_act;
 };
 
 namespace {
@@ -98,6 +105,8 @@ bool desc_ok(const swift_model_desc* d, std::string* why)
     if (d->n_blocks < 1 || d->d_model < 8 || d->n_heads < 1 || d->n_kv_heads < 1 || d->ffn < 16 || d->vocab < 2)
         return bad("non-positive dimension");
     if (d->dtype != SWIFT_F32 && d->dtype != SWIFT_BF16) return bad("dtype must be SWIFT_F32 or SWIFT_BF16");
+    if (d->kv_dtype != SWIFT_F32 && d->kv_dtype != SWIFT_BF16) return bad("kv_dtype must be SWIFT_F32 or SWIFT_BF16");
+    if (d->dtype == SWIFT_F32 && d->kv_dtype != SWIFT_F32) return bad("fp32 models keep an fp32 KV cache");
     if (d->n_heads % d->n_kv_heads) return bad("n_heads must be a multiple of n_kv_heads");
     if (d->head_dim < 16 || d->head_dim > 256 || (d->head_dim & (d->head_dim - 1)))
         return bad("head_dim must be a power of two in 16..256");
@@ -111,6 +120,7 @@ bool desc_ok(const swift_model_desc* d, std::string* why)
 }
 
 size_t esize_of(const swift_model_desc* d) { return d->dtype == SWIFT_BF16 ? 2 : 4; }
+size_t kv_esize_of(const swift_model_desc* d) { return d->kv_dtype == SWIFT_BF16 ? 2 : 4; }
 
 GemmPlan plan_gemm(const swift_model_desc* d, int N, int K)
 {
@@ -150,11 +160,28 @@ WeightLayout weight_layout(const swift_model_desc* d)
     return w;
 }
 
+constexpr int TC_GRID = 148;        // persistent CTAs of the tensor-core GEMM: one per SM of a B200
+constexpr int TC_MAX_TILES = 1024;
+
+// Largest number of CTAs that share one output tile under the stream-K schedule (= slabs needed).
+int max_segments(int N, int K)
+{
+    StreamK sk;
+    sk.KB = ceil_div(K, TC_BK);
+    const int tiles = ceil_div(N, TC_TILE_N);
+    sk.U = (long long)tiles * sk.KB;
+    sk.G = (int)std::min<long long>(TC_GRID, sk.U);
+    int worst = 1;
+    for (int t = 0; t < tiles; ++t)
+        worst = std::max(worst, sk.owner((long long)(t + 1) * sk.KB - 1) - sk.owner((long long)t * sk.KB) + 1);
+    return worst;
+}
+
 int scratch_pages(const swift_model_desc* d) { return MAX_SCORE_ROWS / d->page_size + 2; }
 
 size_t page_bytes(const swift_model_desc* d)
 {
-    return (size_t)d->n_blocks * 2 * d->n_kv_heads * d->page_size * d->head_dim * esize_of(d);
+    return (size_t)d->n_blocks * 2 * d->n_kv_heads * d->page_size * d->head_dim * kv_esize_of(d);
 }
 
 WorkLayout work_layout(const swift_model_desc* d)
@@ -187,6 +214,19 @@ WorkLayout work_layout(const swift_model_desc* d)
     k.score_tok = c.take(MAX_SCORE_ROWS * 4);
     k.score_truth = c.take(MAX_SCORE_ROWS * 4);
     k.score_out = c.take(1024 * 4);
+    // tensor-core path (bf16 models): hi/lo bf16 planes of the GEMM inputs, stream-K slabs, tile counters
+    k.slab_floats = 0;
+    k.xn_hl = k.xa_hl = k.act_hl = k.slabs = k.counters = 0;
+    if (d->dtype == SWIFT_BF16) {
+        auto slab_need = [&](int N, int K) { k.slab_floats = std::max(k.slab_floats, (size_t)max_segments(N, K) * ROWS * (size_t)N); };
+        slab_need((int)(qd + 2 * kd), (int)dm); slab_need((int)dm, (int)qd); slab_need(2 * d->ffn, (int)dm);
+        slab_need((int)dm, d->ffn); slab_need(d->vocab, (int)dm);
+        k.xn_hl = c.take(2 * ROWS * dm * 2);
+        k.xa_hl = c.take(2 * ROWS * qd * 2);
+        k.act_hl = c.take(2 * ROWS * (size_t)d->ffn * 2);
+        k.slabs = c.take(k.slab_floats * 4);
+        k.counters = c.take(TC_MAX_TILES * 4);
+    }
     k.total = c.off;
     return k;
 }
@@ -227,6 +267,45 @@ swift_status launch_gemm(swift_ctx* ctx, int mr, const float* X, int ldx, const 
     case 8: return launch_gemm_mr<T, 8>(ctx, X, ldx, W, N, K, p);
     default: return launch_gemm_mr<T, 16>(ctx, X, ldx, W, N, K, p);
     }
+}
+
+// One GEMM of the walk: where its fp32 input lives, its hi/lo planes and tensor maps (tensor-core path).
+struct GemmSite {
+    const float* X;
+    int N, K;
+    const void* W;
+    const CUtensorMap* mapW;
+    const CUtensorMap* mapX;
+};
+
+swift_status launch_gemm_tc(swift_ctx* ctx, const GemmSite& g)
+{
+    static bool attr_set[8] = {false};
+    if (!attr_set[ctx->device & 7]) {
+        CU(cudaFuncSetAttribute(gemm_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, TC_SMEM_BYTES));
+        attr_set[ctx->device & 7] = true;
+    }
+    if (ceil_div(g.N, TC_TILE_N) > TC_MAX_TILES) return fail(ctx, SWIFT_EUNSUPPORTED, "GEMM with %d output tiles", ceil_div(g.N, TC_TILE_N));
+    gemm_tc_kernel<<<TC_GRID, TC_THREADS, TC_SMEM_BYTES, ctx->stream>>>(state_of(ctx), *g.mapW, *g.mapX,
+                                                                       kptr<float>(ctx, ctx->kl.part), kptr<float>(ctx, ctx->kl.slabs),
+                                                                       kptr<int>(ctx, ctx->kl.counters), g.N, g.K);
+    ctx->launches++;
+    CU(cudaGetLastError());
+    return SWIFT_OK;
+}
+
+// Runs one GEMM site; the result lands in the `part` buffer as *n_split slabs of [ROWS][N] to be summed.
+template <typename T>
+swift_status run_gemm(swift_ctx* ctx, int mr, const GemmSite& g, int* n_split)
+{
+    if (ctx->use_tc) {
+        *n_split = 1;
+        return launch_gemm_tc(ctx, g);
+    }
+    GemmPlan p;
+    swift_status s = launch_gemm<T>(ctx, mr, g.X, g.K, reinterpret_cast<const T*>(g.W), g.N, g.K, &p);
+    *n_split = p.S;
+    return s;
 }
 
 template <typename T, int MR>
@@ -276,7 +355,7 @@ struct HeadOpts {
 
 // Enqueues the kernels of one forward chunk of at most `rows` (<= 16) rows.  The device state
 // (pos0, n_rows, tok_off) must have been set by a preceding kernel on the same stream.
-template <typename T>
+template <typename T, typename TKV>
 swift_status forward_chunk(swift_ctx* ctx, int rows, const int* toks_dev, const uint8_t* skip, const int* page_table,
                            HeadOpts head)
 {
@@ -290,48 +369,50 @@ swift_status forward_chunk(swift_ctx* ctx, int rows, const int* toks_dev, const 
     float* xa = kptr<float>(ctx, ctx->kl.xa);
     float* act = kptr<float>(ctx, ctx->kl.act);
     float* part = kptr<float>(ctx, ctx->kl.part);
-    const float* pend = nullptr;      // pending residual-branch output (split-K partials) not yet added to h
-    int pend_S = 0;
-    GemmPlan p;
+    const bool tc = ctx->use_tc;
+    __nv_bfloat16* xn_hl = tc ? kptr<__nv_bfloat16>(ctx, ctx->kl.xn_hl) : nullptr;
+    __nv_bfloat16* xa_hl = tc ? kptr<__nv_bfloat16>(ctx, ctx->kl.xa_hl) : nullptr;
+    __nv_bfloat16* act_hl = tc ? kptr<__nv_bfloat16>(ctx, ctx->kl.act_hl) : nullptr;
+    const float* pend = nullptr;      // pending residual-branch output (split-K slabs) not yet added to h
+    int pend_S = 0, S = 0;
 
     embed_kernel<T><<<rows, 256, 0, s>>>(st, toks_dev, wptr<T>(ctx, ctx->wl.embed), h, dm, d.vocab);
     ctx->launches++;
     for (int b = 0; b < d.n_blocks; ++b) {
         if (!(skip && skip[2 * b])) {
             resid_norm_kernel<<<rows, 512, 0, s>>>(st, h, pend, pend_S, (size_t)ROWS * dm,
-                                                      wptr<float>(ctx, ctx->wl.attn_norm[b]), xn, dm, d.rms_eps);
+                                                   wptr<float>(ctx, ctx->wl.attn_norm[b]), xn, xn_hl, dm, d.rms_eps);
             ctx->launches++;
-            ST(launch_gemm<T>(ctx, mr, xn, dm, wptr<T>(ctx, ctx->wl.wqkv[b]), nqkv, dm, &p));
-            qkv_post_kernel<T><<<dim3(rows, d.n_heads + 2 * d.n_kv_heads), d.head_dim / 2, 0, s>>>(
-                st, part, p.S, (size_t)ROWS * nqkv, nqkv, kptr<float>(ctx, ctx->kl.q), reinterpret_cast<T*>(ctx->kvbase),
+            ST(run_gemm<T>(ctx, mr, GemmSite{xn, nqkv, dm, wptr<T>(ctx, ctx->wl.wqkv[b]), tc ? &ctx->tm_wqkv[b] : nullptr, &ctx->tm_xn}, &S));
+            qkv_post_kernel<TKV><<<dim3(rows, d.n_heads + 2 * d.n_kv_heads), d.head_dim / 2, 0, s>>>(
+                st, part, S, (size_t)ROWS * nqkv, nqkv, kptr<float>(ctx, ctx->kl.q), reinterpret_cast<TKV*>(ctx->kvbase),
                 page_table, ctx->kv, b, d.n_heads, kptr<float2>(ctx, ctx->kl.rope), d.max_positions);
             ctx->launches++;
-            ST(launch_attn<T>(ctx, mr, page_table, b));
+            ST(launch_attn<TKV>(ctx, mr, page_table, b));
             attn_combine_kernel<<<dim3(d.n_heads, rows), d.head_dim, 0, s>>>(
                 st, kptr<float>(ctx, ctx->kl.o_part), kptr<float2>(ctx, ctx->kl.ml_part), ctx->max_splits, d.n_heads,
-                d.head_dim, xa);
+                d.head_dim, xa, xa_hl);
             ctx->launches++;
-            ST(launch_gemm<T>(ctx, mr, xa, qd, wptr<T>(ctx, ctx->wl.wo[b]), dm, qd, &p));
-            pend = part; pend_S = p.S;
+            ST(run_gemm<T>(ctx, mr, GemmSite{xa, dm, qd, wptr<T>(ctx, ctx->wl.wo[b]), tc ? &ctx->tm_wo[b] : nullptr, &ctx->tm_xa}, &S));
+            pend = part; pend_S = S;
         }
         if (!(skip && skip[2 * b + 1])) {
             resid_norm_kernel<<<rows, 512, 0, s>>>(st, h, pend, pend_S, (size_t)ROWS * dm,
-                                                      wptr<float>(ctx, ctx->wl.mlp_norm[b]), xn, dm, d.rms_eps);
+                                                   wptr<float>(ctx, ctx->wl.mlp_norm[b]), xn, xn_hl, dm, d.rms_eps);
             ctx->launches++;
-            ST(launch_gemm<T>(ctx, mr, xn, dm, wptr<T>(ctx, ctx->wl.wgu[b]), 2 * d.ffn, dm, &p));
-            swiglu_kernel<<<dim3(ceil_div(d.ffn, 256), rows), 256, 0, s>>>(st, part, p.S, (size_t)ROWS * 2 * d.ffn, act,
-                                                                            d.ffn);
+            ST(run_gemm<T>(ctx, mr, GemmSite{xn, 2 * d.ffn, dm, wptr<T>(ctx, ctx->wl.wgu[b]), tc ? &ctx->tm_wgu[b] : nullptr, &ctx->tm_xn}, &S));
+            swiglu_kernel<<<dim3(ceil_div(d.ffn, 256), rows), 256, 0, s>>>(st, part, S, (size_t)ROWS * 2 * d.ffn, act, act_hl, d.ffn);
             ctx->launches++;
-            ST(launch_gemm<T>(ctx, mr, act, d.ffn, wptr<T>(ctx, ctx->wl.wdown[b]), dm, d.ffn, &p));
-            pend = part; pend_S = p.S;
+            ST(run_gemm<T>(ctx, mr, GemmSite{act, dm, d.ffn, wptr<T>(ctx, ctx->wl.wdown[b]), tc ? &ctx->tm_wdown[b] : nullptr, &ctx->tm_act}, &S));
+            pend = part; pend_S = S;
         }
     }
     if (head.run) {
         resid_norm_kernel<<<rows, 512, 0, s>>>(st, h, pend, pend_S, (size_t)ROWS * dm,
-                                                  wptr<float>(ctx, ctx->wl.final_norm), xn, dm, d.rms_eps);
+                                               wptr<float>(ctx, ctx->wl.final_norm), xn, xn_hl, dm, d.rms_eps);
         ctx->launches++;
-        ST(launch_gemm<T>(ctx, mr, xn, dm, wptr<T>(ctx, ctx->wl.lm_head), d.vocab, dm, &p));
-        vocab_kernel<<<rows, VOCAB_THREADS, 0, s>>>(st, part, p.S, (size_t)ROWS * d.vocab,
+        ST(run_gemm<T>(ctx, mr, GemmSite{xn, d.vocab, dm, wptr<T>(ctx, ctx->wl.lm_head), &ctx->tm_lm_head, &ctx->tm_xn}, &S));
+        vocab_kernel<<<rows, VOCAB_THREADS, 0, s>>>(st, part, S, (size_t)ROWS * d.vocab,
                                                    kptr<float>(ctx, ctx->kl.logits), d.vocab, 1.0f / ctx->temperature,
                                                    head.mode, head.draft_j, head.stop_conf,
                                                    ctx->mode == SWIFT_SAMPLING ? 1 : 0, ctx->seed, (uint32_t)ctx->round,
@@ -345,8 +426,11 @@ swift_status forward_chunk(swift_ctx* ctx, int rows, const int* toks_dev, const 
 swift_status forward_chunk_any(swift_ctx* ctx, int rows, const int* toks_dev, const uint8_t* skip, const int* page_table,
                                HeadOpts head)
 {
-    if (ctx->d.dtype == SWIFT_BF16) return forward_chunk<__nv_bfloat16>(ctx, rows, toks_dev, skip, page_table, head);
-    return forward_chunk<float>(ctx, rows, toks_dev, skip, page_table, head);
+    if (ctx->d.dtype == SWIFT_BF16) {
+        if (ctx->d.kv_dtype == SWIFT_BF16) return forward_chunk<__nv_bfloat16, __nv_bfloat16>(ctx, rows, toks_dev, skip, page_table, head);
+        return forward_chunk<__nv_bfloat16, float>(ctx, rows, toks_dev, skip, page_table, head);
+    }
+    return forward_chunk<float, float>(ctx, rows, toks_dev, skip, page_table, head);
 }
 
 } // namespace
@@ -361,7 +445,12 @@ swift_status read_state(swift_ctx* ctx, DevState* out)
     CU(cudaMemcpyAsync(out, state_of(ctx), sizeof(DevState), cudaMemcpyDeviceToHost, ctx->stream));
     CU(cudaStreamSynchronize(ctx->stream));
     if (out->error) {
+        const int code = out->error;
         CU(cudaMemsetAsync(&state_of(ctx)->error, 0, sizeof(int), ctx->stream));
+        if (code == TC_ERR_TIMEOUT) {
+            CU(cudaMemsetAsync(kptr<int>(ctx, ctx->kl.counters), 0, TC_MAX_TILES * 4, ctx->stream));
+            return fail(ctx, SWIFT_ETIMEOUT, "a bounded wait inside the tensor-core GEMM ran out");
+        }
         return fail(ctx, SWIFT_EINVAL, "device reported an invalid token id");
     }
     return SWIFT_OK;
@@ -505,16 +594,63 @@ swift_status enqueue_score(swift_ctx* ctx, const uint8_t* masks, int C, int gamm
 double forward_bytes(const swift_ctx* ctx, const uint8_t* skip, int n_rows, int n_context)
 {
     const swift_model_desc& d = ctx->d;
-    const double es = (double)ctx->esize;
+    const double es = (double)ctx->esize, kes = (double)kv_esize_of(&ctx->d);
     const double dm = d.d_model, qd = (double)d.n_heads * d.head_dim, kd = (double)d.n_kv_heads * d.head_dim;
     const double attn_w = (qd + 2 * kd) * dm + dm * qd, mlp_w = 3.0 * d.ffn * dm;
     double bytes = (double)d.vocab * dm * es;                      // output head
     for (int b = 0; b < d.n_blocks; ++b) {
-        if (!(skip && skip[2 * b])) bytes += attn_w * es + 2.0 * kd * n_context * es + 2.0 * kd * n_rows * es;
+        if (!(skip && skip[2 * b])) bytes += attn_w * es + 2.0 * kd * n_context * kes + 2.0 * kd * n_rows * kes;
         if (!(skip && skip[2 * b + 1])) bytes += mlp_w * es;
     }
     bytes += n_rows * (dm * es + (double)d.vocab * 4.0);           // embedding rows in, logits out
     return bytes;
+}
+
+} // namespace
+
+// =============================================================================== tensor maps
+namespace {
+
+// bf16 row-major [rows][cols] matrix, box = box_rows x 64 columns (128 bytes), 128-byte swizzle.
+swift_status make_map(swift_ctx* ctx, CUtensorMap* out, const void* base, uint64_t rows, uint64_t cols, uint32_t box_rows)
+{
+    static PFN_cuTensorMapEncodeTiled_v12000 encode = nullptr;
+    if (!encode) {
+        void* fn = nullptr;
+        cudaDriverEntryPointQueryResult q;
+        CU(cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &q));
+        if (q != cudaDriverEntryPointSuccess || !fn) return fail(ctx, SWIFT_ECUDA, "cuTensorMapEncodeTiled not available from the driver");
+        encode = reinterpret_cast<PFN_cuTensorMapEncodeTiled_v12000>(fn);
+    }
+    const cuuint64_t dims[2] = {cols, rows};
+    const cuuint64_t strides[1] = {cols * 2};
+    const cuuint32_t box[2] = {(cuuint32_t)TC_BK, box_rows};
+    const cuuint32_t estr[2] = {1, 1};
+    const CUresult r = encode(out, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, estr,
+                              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (r != CUDA_SUCCESS) return fail(ctx, SWIFT_ECUDA, "cuTensorMapEncodeTiled failed with code %d (rows %llu, cols %llu)", (int)r,
+                                       (unsigned long long)rows, (unsigned long long)cols);
+    return SWIFT_OK;
+}
+
+swift_status make_all_maps(swift_ctx* ctx)
+{
+    const swift_model_desc& d = ctx->d;
+    const uint64_t dm = d.d_model, qd = (uint64_t)d.n_heads * d.head_dim, kd = (uint64_t)d.n_kv_heads * d.head_dim;
+    ctx->tm_wqkv.resize(d.n_blocks); ctx->tm_wo.resize(d.n_blocks); ctx->tm_wgu.resize(d.n_blocks); ctx->tm_wdown.resize(d.n_blocks);
+    for (int b = 0; b < d.n_blocks; ++b) {
+        ST(make_map(ctx, &ctx->tm_wqkv[b], ctx->wbase + ctx->wl.wqkv[b], qd + 2 * kd, dm, TC_TILE_N));
+        ST(make_map(ctx, &ctx->tm_wo[b], ctx->wbase + ctx->wl.wo[b], dm, qd, TC_TILE_N));
+        ST(make_map(ctx, &ctx->tm_wgu[b], ctx->wbase + ctx->wl.wgu[b], 2 * (uint64_t)d.ffn, dm, TC_TILE_N));
+        ST(make_map(ctx, &ctx->tm_wdown[b], ctx->wbase + ctx->wl.wdown[b], dm, d.ffn, TC_TILE_N));
+    }
+    ST(make_map(ctx, &ctx->tm_lm_head, ctx->wbase + ctx->wl.lm_head, d.vocab, dm, TC_TILE_N));
+    ST(make_map(ctx, &ctx->tm_embed, ctx->wbase + ctx->wl.embed, d.vocab, dm, TC_TILE_N));
+    ST(make_map(ctx, &ctx->tm_xn, ctx->ws + ctx->kl.xn_hl, 2 * ROWS, dm, TC_COLS));
+    ST(make_map(ctx, &ctx->tm_xa, ctx->ws + ctx->kl.xa_hl, 2 * ROWS, qd, TC_COLS));
+    ST(make_map(ctx, &ctx->tm_act, ctx->ws + ctx->kl.act_hl, 2 * ROWS, d.ffn, TC_COLS));
+    return SWIFT_OK;
 }
 
 } // namespace
@@ -571,6 +707,12 @@ swift_status swift_load(const swift_model_desc* desc, swift_devbuf weights, swif
     c->round_open = false;
     c->mode = SWIFT_GREEDY; c->temperature = 1.f; c->seed = 0; c->launches = 0;
     ctx = c;
+    c->use_tc = false;
+    if (desc->dtype == SWIFT_BF16) {
+        const swift_status ms = make_all_maps(c);
+        if (ms != SWIFT_OK) { g_load_error = c->err; delete c; return ms; }
+        c->use_tc = true;
+    }
     for (auto& e : c->ev) e = nullptr;
     cudaError_t e = cudaSuccess;
     for (auto& ev : c->ev) if (e == cudaSuccess) e = cudaEventCreate(&ev);
@@ -794,6 +936,57 @@ swift_status swift_score_skipsets(swift_ctx* ctx, const uint8_t* masks, int32_t 
     return SWIFT_OK;
 }
 
+swift_status swift_gemm(swift_ctx* ctx, int32_t which, int32_t block, const float* x_host, int32_t n_rows, float* y_host)
+{
+    if (!ctx || !x_host || !y_host) return fail(ctx, SWIFT_EINVAL, "null argument");
+    if (ctx->round_open) return fail(ctx, SWIFT_ESTATE, "a round is open");
+    const swift_model_desc& d = ctx->d;
+    if (which < 0 || which > 4 || n_rows < 1 || n_rows > ROWS || block < 0 || block >= d.n_blocks)
+        return fail(ctx, SWIFT_EINVAL, "bad which / block / n_rows");
+    const int dm = d.d_model, qd = d.n_heads * d.head_dim, kd = d.n_kv_heads * d.head_dim;
+    const int N = which == 0 ? qd + 2 * kd : which == 1 ? dm : which == 2 ? 2 * d.ffn : which == 3 ? dm : d.vocab;
+    const int K = which == 1 ? qd : which == 3 ? d.ffn : dm;
+    float* X = which == 1 ? kptr<float>(ctx, ctx->kl.xa) : which == 3 ? kptr<float>(ctx, ctx->kl.act) : kptr<float>(ctx, ctx->kl.xn);
+    const size_t woff = which == 0 ? ctx->wl.wqkv[block] : which == 1 ? ctx->wl.wo[block] : which == 2 ? ctx->wl.wgu[block]
+                        : which == 3 ? ctx->wl.wdown[block] : ctx->wl.lm_head;
+    CU(cudaMemcpyAsync(X, x_host, (size_t)n_rows * K * 4, cudaMemcpyHostToDevice, ctx->stream));
+    set_rows_kernel<<<1, 1, 0, ctx->stream>>>(state_of(ctx), 0, n_rows);
+    ctx->launches++;
+    GemmSite g{X, N, K, ctx->wbase + woff, nullptr, nullptr};
+    if (ctx->use_tc) {
+        __nv_bfloat16* planes = which == 1 ? kptr<__nv_bfloat16>(ctx, ctx->kl.xa_hl) : which == 3 ? kptr<__nv_bfloat16>(ctx, ctx->kl.act_hl)
+                                           : kptr<__nv_bfloat16>(ctx, ctx->kl.xn_hl);
+        split_planes_kernel<<<dim3(ceil_div(K, 256), n_rows), 256, 0, ctx->stream>>>(X, planes, K);
+        ctx->launches++;
+        g.mapW = which == 0 ? &ctx->tm_wqkv[block] : which == 1 ? &ctx->tm_wo[block] : which == 2 ? &ctx->tm_wgu[block]
+                 : which == 3 ? &ctx->tm_wdown[block] : &ctx->tm_lm_head;
+        g.mapX = which == 1 ? &ctx->tm_xa : which == 3 ? &ctx->tm_act : &ctx->tm_xn;
+    }
+    int S = 0;
+    if (d.dtype == SWIFT_BF16) ST(run_gemm<__nv_bfloat16>(ctx, mr_of(n_rows), g, &S));
+    else ST(run_gemm<float>(ctx, mr_of(n_rows), g, &S));
+    std::vector<float> slab((size_t)n_rows * N);
+    std::fill(y_host, y_host + (size_t)n_rows * N, 0.f);
+    for (int s = 0; s < S; ++s) {          // slabs are added in slab order, as the consumers on the device do
+        CU(cudaMemcpyAsync(slab.data(), kptr<float>(ctx, ctx->kl.part) + (size_t)s * ROWS * N, slab.size() * 4,
+                           cudaMemcpyDeviceToHost, ctx->stream));
+        CU(cudaStreamSynchronize(ctx->stream));
+        for (size_t i = 0; i < slab.size(); ++i) y_host[i] += slab[i];
+    }
+    DevState hs;
+    return read_state(ctx, &hs);
+}
+
+swift_status swift_set_gemm_impl(swift_ctx* ctx, int32_t impl)
+{
+    if (!ctx) return SWIFT_EINVAL;
+    if (impl != 0 && impl != 1) return fail(ctx, SWIFT_EINVAL, "impl must be 0 (SIMT) or 1 (tensor cores)");
+    if (impl == 1 && ctx->d.dtype != SWIFT_BF16) return fail(ctx, SWIFT_EUNSUPPORTED, "the tensor-core GEMM needs bf16 weights");
+    if (ctx->round_open) return fail(ctx, SWIFT_ESTATE, "a round is open");
+    ctx->use_tc = impl == 1;
+    return SWIFT_OK;
+}
+
 int32_t swift_committed_length(const swift_ctx* ctx) { return ctx ? ctx->n : -1; }
 int64_t swift_launch_count(const swift_ctx* ctx) { return ctx ? ctx->launches : -1; }
 double swift_forward_bytes(const swift_ctx* ctx, const uint8_t* skip, int32_t n_rows, int32_t n_context)
@@ -816,7 +1009,7 @@ swift_status swift_read_kv(swift_ctx* ctx, int32_t block, int32_t which, int32_t
     float* stage = kptr<float>(ctx, ctx->kl.part);
     for (int c0 = 0; c0 < count; c0 += step) {
         const int cnt = std::min(step, count - c0);
-        if (ctx->d.dtype == SWIFT_BF16)
+        if (ctx->d.kv_dtype == SWIFT_BF16)
             kv_read_kernel<__nv_bfloat16><<<64, 256, 0, ctx->stream>>>(reinterpret_cast<const __nv_bfloat16*>(ctx->kvbase),
                                                                       pt_main(ctx), ctx->kv, block, which, pos0 + c0, cnt, stage);
         else
@@ -852,16 +1045,28 @@ static swift_status time_gemm_t(swift_ctx* ctx, int which, int n_rows, int iters
         default: return (i & 1) ? wptr<T>(ctx, ctx->wl.embed) : wptr<T>(ctx, ctx->wl.lm_head);
         }
     };
-    for (int i = 0; i < 3; ++i) ST(launch_gemm<T>(ctx, mr_of(n_rows), X, K, weight(i), N, K, &p));
+    auto site = [&](int i) -> GemmSite {
+        const int b = i % d.n_blocks;
+        const CUtensorMap* mw = nullptr;
+        if (ctx->use_tc)
+            mw = which == 0 ? &ctx->tm_wqkv[b] : which == 1 ? &ctx->tm_wo[b] : which == 2 ? &ctx->tm_wgu[b] : which == 3 ? &ctx->tm_wdown[b]
+                 : (i & 1) ? &ctx->tm_embed : &ctx->tm_lm_head;
+        const CUtensorMap* mx = which == 1 ? &ctx->tm_xa : which == 3 ? &ctx->tm_act : &ctx->tm_xn;
+        return GemmSite{X, N, K, weight(i), mw, mx};
+    };
+    int S = 0;
+    (void)p;
+    for (int i = 0; i < 3; ++i) ST(run_gemm<T>(ctx, mr_of(n_rows), site(i), &S));
     CU(cudaEventRecord(ctx->ev[0], ctx->stream));
-    for (int i = 0; i < iters; ++i) ST(launch_gemm<T>(ctx, mr_of(n_rows), X, K, weight(i + 3), N, K, &p));
+    for (int i = 0; i < iters; ++i) ST(run_gemm<T>(ctx, mr_of(n_rows), site(i + 3), &S));
     CU(cudaEventRecord(ctx->ev[1], ctx->stream));
     CU(cudaStreamSynchronize(ctx->stream));
     float t = 0.f;
     CU(cudaEventElapsedTime(&t, ctx->ev[0], ctx->ev[1]));
     *ms = t / (float)iters;
     *bytes = (double)N * K * sizeof(T);
-    return SWIFT_OK;
+    DevState hs;
+    return read_state(ctx, &hs);
 }
 
 extern "C" {

@@ -13,11 +13,11 @@ LOGIT_TOL = 2e-2        # max |dlogit| / std(oracle row)
 MARGIN = 0.05           # tokens must agree wherever the oracle's top-1/top-2 gap exceeds this
 
 
-def make_pair(cfg, max_positions=256, page_size=16, max_draft=15, oracle_dtype=None):
+def make_pair(cfg, max_positions=256, page_size=16, max_draft=15, oracle_dtype=None, kv_dtype="f32"):
     """(oracle, gpu model) over identical synthetic weights."""
     from paper_2410_06916_b200 import SwiftModel
     w = synth.make_weights(cfg)
-    gpu = SwiftModel(cfg, max_positions=max_positions, page_size=page_size, max_draft=max_draft)
+    gpu = SwiftModel(cfg, max_positions=max_positions, page_size=page_size, max_draft=max_draft, kv_dtype=kv_dtype)
     gpu.pack("embed", -1, w["embed"]); gpu.pack("lm_head", -1, w["lm_head"]); gpu.pack("final_norm", -1, w["final_norm"])
     for b, wb in enumerate(w["blocks"]):
         for name, t in wb.items():

@@ -95,27 +95,67 @@ def test_kv_cache_matches_oracle(small_pair, small_cfg):
         assert np.abs(g.read_kv(b, 1, 0, 21) - o.V[b][:21].numpy()).max() < 1e-4
 
 
-@pytest.mark.parametrize("shape", ["7b", "13b"])
-def test_full_width_bf16_forward(shape):
+@pytest.mark.parametrize("shape,rows", [("13b", 1), ("13b", 9), ("13b", 16), ("7b", 13), ("odd", 5)])
+def test_weight_streaming_gemm_kernels(shape, rows):
+    """The skinny GEMM alone, tensor-core and SIMT kernels, at the real projection shapes of the 13B / 7B
+    models (and an odd shape with ragged tiles in N and K) against the oracle's fp64 projection."""
+    if shape == "odd":
+        cfg = synth.ModelConfig("odd", n_blocks=1, d_model=520, n_heads=5, n_kv_heads=5, head_dim=64, ffn=1392, vocab=777,
+                                dtype="bf16", seed=9, n_planted=0)
+    else:
+        cfg = synth.MODELS[shape].with_blocks(1, n_planted=0)
+    from paper_2410_06916_b200 import SwiftModel
+    g = SwiftModel(cfg, max_positions=64)
+    try:
+        w = {n: synth.make_tensor(cfg, n, 0, planted=False) for n in ("wq", "wk", "wv", "wo", "wgate", "wup", "wdown")}
+        w["lm_head"] = synth.make_tensor(cfg, "lm_head")
+        for n, t in w.items():
+            g.pack(n, 0 if n != "lm_head" else -1, t)
+        F = cfg.ffn
+        il = torch.stack([w["wgate"].view(F // 16, 16, -1), w["wup"].view(F // 16, 16, -1)], 1).reshape(2 * F, -1)
+        mats = [torch.cat([w["wq"], w["wk"], w["wv"]]), w["wo"], il, w["wdown"], w["lm_head"]]
+        gen = torch.Generator().manual_seed(rows)
+        for which, W in enumerate(mats):
+            x = torch.randn(rows, W.shape[1], generator=gen) * (1.0 + which)
+            ref = so.linear(x, W).numpy()
+            scale = float(np.sqrt((ref ** 2).mean()))
+            g.set_gemm_impl(True)
+            y_tc = g.gemm(which, 0, x.numpy())
+            g.set_gemm_impl(False)
+            y_simt = g.gemm(which, 0, x.numpy())
+            assert np.abs(y_simt - ref).max() < 2e-5 * scale * np.sqrt(W.shape[1] / 512), which
+            assert np.abs(y_tc - ref).max() < 1e-4 * scale, (which, float(np.abs(y_tc - ref).max()), scale)
+            if rows > 1:                                         # row-count invariance of the tensor-core kernel
+                g.set_gemm_impl(True)
+                assert np.array_equal(g.gemm(which, 0, x.numpy()[:1]), y_tc[:1])
+    finally:
+        g.close()
+
+
+@pytest.mark.parametrize("shape,kv", [("7b", "f32"), ("13b", "f32"), ("13b", "bf16")])
+def test_full_width_bf16_forward(shape, kv):
     """Two blocks at the real 7B / 13B widths and vocabulary, in the launch shapes the benchmark uses:
     one row (drafting, vanilla) and nine rows (verification of 8 drafts), behind a prefix that spans an
     attention split, full model and layer-skipped."""
     cfg = synth.MODELS[shape].with_blocks(2, n_planted=1)
-    o, g = make_pair(cfg, max_positions=320)
+    o, g = make_pair(cfg, max_positions=320, kv_dtype=kv)
+    tol = LOGIT_TOL if kv == "f32" else 3 * LOGIT_TOL      # a bf16 cache costs accuracy: measured, not a parity claim
     try:
         toks = synth.prompt(cfg, 290)
         ref = o.forward_rows(toks[:280], 0)[-3:]
         g.prefill(toks[:280])
         assert g.n == 280
         got, _ = g.forward_rows(toks[277:280], 277)              # recompute the last three rows over the cached prefix
-        assert logit_err(got, ref) < LOGIT_TOL
+        err = logit_err(got, ref)
+        print(f"{shape} kv={kv}: teacher-forced logits off by {err:.2e} sigma")
+        assert err < tol, err
         o.n = 280
         for z in (None, list(synth.block_mask(cfg, [1])), [1, 0, 0, 1]):
             ref9 = o.forward_rows(toks[280:289], 280, z, write_kv=False)
             got9, _ = g.forward_rows(toks[280:289], 280, z, write_kv=False)
             err9 = logit_err(got9, ref9)
             got1, _ = g.forward_rows(toks[280:281], 280, z, write_kv=False)
-            assert err9 < LOGIT_TOL and logit_err(got1, ref9[:1]) < LOGIT_TOL, (z, err9)
+            assert err9 < tol and logit_err(got1, ref9[:1]) < tol, (z, err9)
             assert np.array_equal(got1[0], got9[0])              # row-count invariance, bit for bit
     finally:
         g.close()
