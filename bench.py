@@ -113,6 +113,22 @@ def oracle_sample(cfg, run, z, weights, n_ctx=16, k=2):
     return {"vanilla": 1.0 / (t1 - t0), "swift": (a + 1) / (t2 - t1), "seconds": t2 - t0, "accepted": a, "k": k}
 
 
+def micro(cfg, run, args, hbm_peak):
+    """Each GEMM shape of the walk, alone, on a 4-block copy of the model (weights still several times L2)."""
+    from paper_2410_06916_b200 import SwiftModel
+    small = cfg.with_blocks(4)
+    model = SwiftModel(small, max_positions=64, max_draft=run.max_draft, kv_dtype=args.kv_dtype)
+    model.load_weights(synth.iter_tensors(small))
+    names = ["qkv", "o_proj", "gate_up", "down", "lm_head"]
+    out = {"micro": small.name, "peak_gbs": hbm_peak, "gemms": {}}
+    for which, name in enumerate(names):
+        for rows in (1, run.max_draft + 1):
+            ms, nbytes = model.time_gemm(which, rows, args.micro_iters)
+            out["gemms"][f"{name}/{rows}"] = {"us": round(ms * 1e3, 2), "MB": round(nbytes / 1e6, 1),
+                                              "gbs": round(nbytes / ms * 1e-6, 1), "frac": round(nbytes / ms * 1e-6 / hbm_peak, 3)}
+    print(json.dumps(out))
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -121,13 +137,21 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="c2", choices=sorted(synth.RUNS))
     ap.add_argument("--max-new", type=int, default=0, help="override the number of generated tokens")
+    ap.add_argument("--prompt-len", type=int, default=0, help="override the prompt length (profiling runs)")
+    ap.add_argument("--kv-dtype", default="f32", choices=["f32", "bf16"], help="storage of cached K,V")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--micro", action="store_true",
+                    help="time each weight-streaming GEMM of the model alone on a few-block copy (profiling aid); prints one JSON line")
+    ap.add_argument("--micro-iters", type=int, default=40)
     args = ap.parse_args()
     rank = int(os.environ.get("RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
     local = int(os.environ.get("LOCAL_RANK", "0"))
 
     cfg, run, z = workload(args.workload)
+    if args.prompt_len:
+        import dataclasses
+        run = dataclasses.replace(run, prompt_len=args.prompt_len)
     max_new = args.max_new or run.max_new
     hbm_peak, peak_kind = peaks()
     sampling = run.mode == "sampling"
@@ -159,11 +183,15 @@ def main():
 
     from paper_2410_06916_b200 import GenParams, SwiftModel
     torch.cuda.set_device(local)
+    if args.micro:
+        micro(cfg, run, args, hbm_peak)
+        return
     if world > 1:
         import torch.distributed as dist
         dist.init_process_group("nccl", device_id=torch.device("cuda", local))
     weights = synth.make_weights(cfg) if cfg.n_blocks * cfg.block_params() < 40e9 else None
-    model = SwiftModel(cfg, max_positions=run.prompt_len + max_new + 32, max_draft=run.max_draft, device=f"cuda:{local}")
+    model = SwiftModel(cfg, max_positions=run.prompt_len + max_new + 32, max_draft=run.max_draft, device=f"cuda:{local}",
+                       kv_dtype=args.kv_dtype)
     if weights is not None:
         model.load_weights((n, -1, weights[n]) for n in ("embed", "lm_head", "final_norm"))
         model.load_weights((n, b, t) for b, wb in enumerate(weights["blocks"]) for n, t in wb.items())
@@ -237,7 +265,7 @@ def main():
     out = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
            "ms_per_step": tot_ms / args.steps, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
            "dtype": "bf16" if cfg.dtype == "bf16" else "f32", "data": "synthetic",
-           "config": {"workload": desc, "l2": "inputs (weights) far larger than L2; no flush", "parallelism": "replicas only",
+           "config": {"workload": desc, "l2": "inputs (weights) far larger than L2; no flush", "parallelism": "replicas only", "kv_cache": args.kv_dtype,
                       "e2e_note": "whole swift_generate call incl. prefill and host copies, host clock", "context": PAPER_CONTEXT},
            "vanilla_tokens_per_s": vanilla, "swift_equals_vanilla": lossless, "speedup_vs_vanilla": value / world / vanilla,
            "M": (s0.tokens - 1) / s0.rounds, "alpha": s0.accepted / max(s0.drafted, 1), "rounds": s0.rounds,
