@@ -33,7 +33,11 @@ struct DevState {
     float row_max[ROWS];   // per-row max logit
     float row_sum[ROWS];   // per-row sum exp((l - max) / T)
     int match_count;       // score_skipsets: matches of the current candidate
-    int pad[7];
+    int draft_j;           // index (1-based) of the draft step in flight
+    int round;             // round counter = Philox counter word 0
+    float stop_conf;       // early-stop threshold of this round
+    unsigned seed_lo, seed_hi;
+    int pad[2];
 };
 
 template <typename T> struct Vec;

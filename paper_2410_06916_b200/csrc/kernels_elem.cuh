@@ -17,9 +17,14 @@ __global__ void set_rows_kernel(DevState* st, int pos0, int n_rows)
 }
 
 // Start of a round: pending token into slot 0, drafting armed.
-__global__ void begin_round_kernel(DevState* st, int pending_token, int use_given_token)
+__global__ void begin_round_kernel(DevState* st, int pending_token, int use_given_token, int round, float stop_conf,
+                                   unsigned seed_lo, unsigned seed_hi)
 {
     if (use_given_token) st->draft_tok[0] = pending_token;
+    st->round = round;
+    st->stop_conf = stop_conf;
+    st->seed_lo = seed_lo;
+    st->seed_hi = seed_hi;
     st->active = 1;
     st->n_drafted = 0;
     st->n_accepted = 0;
@@ -29,6 +34,7 @@ __global__ void begin_round_kernel(DevState* st, int pending_token, int use_give
 // leaves zero rows so that the step's kernels fall through.
 __global__ void begin_draft_step_kernel(DevState* st, int n, int j)
 {
+    st->draft_j = j;
     if (st->active) {
         st->pos0 = n + j - 1;
         st->n_rows = 1;

@@ -250,13 +250,19 @@ gemm_tc_kernel(DevState* st, const __grid_constant__ CUtensorMap mapW, const __g
                 asm volatile("bar.sync 1, 128;" ::: "memory");
                 if (last_flag_sh) {                             // last arrival: add the slabs in slab order
                     __threadfence();
-                    if (n < N)
+                    if (n < N) {
+                        float acc[ROWS];
+#pragma unroll
+                        for (int m = 0; m < ROWS; ++m) acc[m] = 0.f;
+                        for (int j = 0; j < nseg; ++j) {            // slab order; the 16 row loads of a slab are independent
+#pragma unroll
+                            for (int m = 0; m < ROWS; ++m)
+                                if (m < n_rows) acc[m] += __ldcg(slabs + ((size_t)j * ROWS + m) * N + n);
+                        }
+#pragma unroll
                         for (int m = 0; m < ROWS; ++m)
-                            if (m < n_rows) {
-                                float acc = 0.f;
-                                for (int j = 0; j < nseg; ++j) acc += __ldcg(slabs + ((size_t)j * ROWS + m) * N + n);
-                                Y[(size_t)m * N + n] = acc;
-                            }
+                            if (m < n_rows) Y[(size_t)m * N + n] = acc[m];
+                    }
                     if (etid == 0) counters[tile] = 0;
                 }
                 asm volatile("bar.sync 1, 128;" ::: "memory");  // last_flag_sh is rewritten by the next segment

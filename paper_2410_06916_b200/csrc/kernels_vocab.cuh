@@ -86,8 +86,7 @@ __device__ int block_categorical(WeightFn w, int n, float u, float* sh)
 // drafting when the confidence is below stop_conf.
 __global__ void __launch_bounds__(VOCAB_THREADS)
 vocab_kernel(DevState* st, const float* __restrict__ part, int n_split, size_t split_stride,
-             float* __restrict__ logits, int vocab, float inv_temp, int mode, int draft_j, float stop_conf,
-             int sampling, uint64_t seed, uint32_t round, float* __restrict__ q_rows)
+             float* __restrict__ logits, int vocab, float inv_temp, int mode, int sampling, float* __restrict__ q_rows)
 {
     __shared__ float sh[VOCAB_THREADS + 72];
     __shared__ ArgMax sh_am[32];
@@ -139,6 +138,12 @@ vocab_kernel(DevState* st, const float* __restrict__ part, int n_split, size_t s
     }
     if (mode != VOCAB_DRAFT || r != 0) return;
 
+    // step index, threshold and random-number coordinates come from the control block, so that one
+    // captured launch sequence serves every draft step of every round
+    const int draft_j = st->draft_j;
+    const float stop_conf = st->stop_conf;
+    const uint64_t seed = ((uint64_t)st->seed_hi << 32) | st->seed_lo;
+    const uint32_t round = (uint32_t)st->round;
     int y = am.i;
     if (sampling) {
         float* qrow = q_rows + (size_t)(draft_j - 1) * vocab;

@@ -51,6 +51,8 @@ struct WorkLayout {
     size_t part_floats, slab_floats;
 };
 
+struct FwdGraph;
+
 } // namespace
 
 struct swift_ctx {
@@ -71,6 +73,10 @@ struct swift_ctx {
     int64_t launches;
     std::string err;
     cudaEvent_t ev[8];
+    // captured forwards
+    bool use_graphs;
+    std::vector<FwdGraph>* graphs;
+    uint64_t graph_clock;
     // tensor-core GEMM path (bf16 models)
     bool use_tc;
     std::vector<CUtensorMap> tm_wqkv, tm_wo, tm_wgu, tm_wdown;
@@ -241,12 +247,7 @@ int mr_of(int rows) { return rows <= 1 ? 1 : rows <= 2 ? 2 : rows <= 4 ? 4 : row
 template <typename T, int MR>
 swift_status launch_gemm_mr(swift_ctx* ctx, const float* X, int ldx, const T* W, int N, int K, GemmPlan p)
 {
-    static bool attr_set[8] = {false};
     const size_t smem = (size_t)MR * p.Kc * sizeof(float);
-    if (!attr_set[ctx->device & 7]) {
-        CU(cudaFuncSetAttribute(gemm_simt_kernel<T, MR>, cudaFuncAttributeMaxDynamicSharedMemorySize, 16 * 1024 * 4));
-        attr_set[ctx->device & 7] = true;
-    }
     dim3 grid(ceil_div(N, GEMM_SIMT_TILE_N), p.S);
     gemm_simt_kernel<T, MR><<<grid, GEMM_SIMT_THREADS, smem, ctx->stream>>>(state_of(ctx), X, ldx, W,
                                                                             kptr<float>(ctx, ctx->kl.part), N, K, p.Kc);
@@ -280,11 +281,6 @@ struct GemmSite {
 
 swift_status launch_gemm_tc(swift_ctx* ctx, const GemmSite& g)
 {
-    static bool attr_set[8] = {false};
-    if (!attr_set[ctx->device & 7]) {
-        CU(cudaFuncSetAttribute(gemm_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, TC_SMEM_BYTES));
-        attr_set[ctx->device & 7] = true;
-    }
     if (ceil_div(g.N, TC_TILE_N) > TC_MAX_TILES) return fail(ctx, SWIFT_EUNSUPPORTED, "GEMM with %d output tiles", ceil_div(g.N, TC_TILE_N));
     gemm_tc_kernel<<<TC_GRID, TC_THREADS, TC_SMEM_BYTES, ctx->stream>>>(state_of(ctx), *g.mapW, *g.mapX,
                                                                        kptr<float>(ctx, ctx->kl.part), kptr<float>(ctx, ctx->kl.slabs),
@@ -313,12 +309,6 @@ swift_status launch_attn_mr(swift_ctx* ctx, const int* page_table, int block)
 {
     const swift_model_desc& d = ctx->d;
     const size_t smem = ((size_t)MR * d.head_dim + (size_t)MR * ATTN_CHUNK + 2 * MR) * sizeof(float);
-    static bool attr_set[8] = {false};
-    if (!attr_set[ctx->device & 7]) {
-        CU(cudaFuncSetAttribute(attn_split_kernel<T, MR>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                (16 * 256 + 16 * ATTN_CHUNK + 32) * 4));
-        attr_set[ctx->device & 7] = true;
-    }
     dim3 grid(d.n_heads, ctx->max_splits);
     attn_split_kernel<T, MR><<<grid, ATTN_THREADS, smem, ctx->stream>>>(
         state_of(ctx), kptr<float>(ctx, ctx->kl.q), reinterpret_cast<const T*>(ctx->kvbase), page_table, ctx->kv, block,
@@ -343,8 +333,7 @@ swift_status launch_attn(swift_ctx* ctx, int mr, const int* page_table, int bloc
 
 struct HeadOpts {
     bool run = false;
-    int mode = VOCAB_PLAIN, draft_j = 0;
-    float stop_conf = 0.f;
+    int mode = VOCAB_PLAIN;
 };
 
 #define ST(call)                                   \
@@ -414,8 +403,7 @@ swift_status forward_chunk(swift_ctx* ctx, int rows, const int* toks_dev, const 
         ST(run_gemm<T>(ctx, mr, GemmSite{xn, d.vocab, dm, wptr<T>(ctx, ctx->wl.lm_head), &ctx->tm_lm_head, &ctx->tm_xn}, &S));
         vocab_kernel<<<rows, VOCAB_THREADS, 0, s>>>(st, part, S, (size_t)ROWS * d.vocab,
                                                    kptr<float>(ctx, ctx->kl.logits), d.vocab, 1.0f / ctx->temperature,
-                                                   head.mode, head.draft_j, head.stop_conf,
-                                                   ctx->mode == SWIFT_SAMPLING ? 1 : 0, ctx->seed, (uint32_t)ctx->round,
+                                                   head.mode, ctx->mode == SWIFT_SAMPLING ? 1 : 0,
                                                    kptr<float>(ctx, ctx->kl.q_rows));
         ctx->launches++;
     }
@@ -431,6 +419,71 @@ swift_status forward_chunk_any(swift_ctx* ctx, int rows, const int* toks_dev, co
         return forward_chunk<__nv_bfloat16, float>(ctx, rows, toks_dev, skip, page_table, head);
     }
     return forward_chunk<float, float>(ctx, rows, toks_dev, skip, page_table, head);
+}
+
+// A forward chunk depends on the host only through (rows, skip mask, page table, token source, head
+// options, sampling settings); everything else it reads from the device control block.  So its launch
+// sequence is captured once into a CUDA graph and replayed: one graph launch instead of several
+// hundred kernel launches per forward.
+struct FwdKey {
+    int rows, head_run, head_mode, sampling, use_tc;
+    float temperature;
+    const void* toks;
+    const void* page_table;
+    std::vector<uint8_t> mask;
+    bool operator==(const FwdKey& o) const
+    {
+        return rows == o.rows && head_run == o.head_run && head_mode == o.head_mode && sampling == o.sampling &&
+               use_tc == o.use_tc && temperature == o.temperature && toks == o.toks && page_table == o.page_table && mask == o.mask;
+    }
+};
+struct FwdGraph {
+    FwdKey key;
+    cudaGraphExec_t exec;
+    int64_t launches;
+    uint64_t last_use;
+};
+
+swift_status forward_cached(swift_ctx* ctx, int rows, const int* toks_dev, const uint8_t* skip, const int* page_table,
+                            HeadOpts head)
+{
+    if (!ctx->use_graphs) return forward_chunk_any(ctx, rows, toks_dev, skip, page_table, head);
+    const int L = 2 * ctx->d.n_blocks;
+    FwdKey key{rows, head.run ? 1 : 0, head.mode, ctx->mode, ctx->use_tc ? 1 : 0, ctx->temperature, toks_dev, page_table,
+               skip ? std::vector<uint8_t>(skip, skip + L) : std::vector<uint8_t>()};
+    auto& cache = *ctx->graphs;
+    ctx->graph_clock++;
+    for (auto& g : cache)
+        if (g.key == key) {
+            g.last_use = ctx->graph_clock;
+            CU(cudaGraphLaunch(g.exec, ctx->stream));
+            ctx->launches += g.launches;
+            return SWIFT_OK;
+        }
+    // capture a new one
+    const int64_t before = ctx->launches;
+    cudaGraph_t graph = nullptr;
+    CU(cudaStreamBeginCapture(ctx->stream, cudaStreamCaptureModeThreadLocal));
+    const swift_status fs = forward_chunk_any(ctx, rows, toks_dev, skip, page_table, head);
+    const cudaError_t ce = cudaStreamEndCapture(ctx->stream, &graph);
+    if (fs != SWIFT_OK) { if (graph) cudaGraphDestroy(graph); return fs; }
+    if (ce != cudaSuccess) return fail(ctx, SWIFT_ECUDA, "stream capture failed: %s", cudaGetErrorString(ce));
+    cudaGraphExec_t exec = nullptr;
+    const cudaError_t ie = cudaGraphInstantiate(&exec, graph, 0);
+    cudaGraphDestroy(graph);
+    if (ie != cudaSuccess) return fail(ctx, SWIFT_ECUDA, "graph instantiation failed: %s", cudaGetErrorString(ie));
+    const int64_t n_launch = ctx->launches - before;
+    ctx->launches = before;
+    if (cache.size() >= 24) {             // evict the least recently used graph
+        size_t victim = 0;
+        for (size_t i = 1; i < cache.size(); ++i) if (cache[i].last_use < cache[victim].last_use) victim = i;
+        cudaGraphExecDestroy(cache[victim].exec);
+        cache.erase(cache.begin() + victim);
+    }
+    cache.push_back(FwdGraph{key, exec, n_launch, ctx->graph_clock});
+    CU(cudaGraphLaunch(exec, ctx->stream));
+    ctx->launches += n_launch;
+    return SWIFT_OK;
 }
 
 } // namespace
@@ -492,7 +545,7 @@ swift_status run_rows(swift_ctx* ctx, const int32_t* tokens, int n_rows, int pos
         ctx->launches++;
         HeadOpts head;
         head.run = head_mode == 2 || (head_mode == 1 && last);
-        ST(forward_chunk_any(ctx, rows, st->row_tok, skip, page_table, head));
+        ST(forward_cached(ctx, rows, st->row_tok, skip, page_table, head));
         if (head.run && logits_host)
             CU(cudaMemcpyAsync(logits_host + (size_t)c0 * ctx->d.vocab, kptr<float>(ctx, ctx->kl.logits),
                                (size_t)rows * ctx->d.vocab * 4, cudaMemcpyDeviceToHost, ctx->stream));
@@ -511,19 +564,25 @@ swift_status check_tokens(swift_ctx* ctx, const int32_t* t, int n)
     return SWIFT_OK;
 }
 
+void launch_begin_round(swift_ctx* ctx, float stop_conf)
+{
+    begin_round_kernel<<<1, 1, 0, ctx->stream>>>(state_of(ctx), ctx->pending, 1, ctx->round, stop_conf, (unsigned)ctx->seed,
+                                                 (unsigned)(ctx->seed >> 32));
+    ctx->launches++;
+}
+
 // ---- enqueue-only forms of the steps (no host synchronisation); used by the entry points and by generate
 swift_status enqueue_draft(swift_ctx* ctx, const uint8_t* skip, int max_k, float stop_conf)
 {
     DevState* st = state_of(ctx);
     ctx->round++;
-    begin_round_kernel<<<1, 1, 0, ctx->stream>>>(st, ctx->pending, 1);
-    ctx->launches++;
+    launch_begin_round(ctx, stop_conf);
     for (int j = 1; j <= max_k; ++j) {
         begin_draft_step_kernel<<<1, 1, 0, ctx->stream>>>(st, ctx->n, j);
         ctx->launches++;
         HeadOpts head;
-        head.run = true; head.mode = VOCAB_DRAFT; head.draft_j = j; head.stop_conf = stop_conf;
-        ST(forward_chunk_any(ctx, 1, st->draft_tok, skip, pt_main(ctx), head));
+        head.run = true; head.mode = VOCAB_DRAFT;
+        ST(forward_cached(ctx, 1, st->draft_tok, skip, pt_main(ctx), head));
     }
     ctx->last_max_k = max_k;
     ctx->round_open = true;
@@ -537,7 +596,7 @@ swift_status enqueue_verify(swift_ctx* ctx, int rows_launch, int forced_k)
     ctx->launches++;
     HeadOpts head;
     head.run = true;
-    return forward_chunk_any(ctx, rows_launch, st->draft_tok, nullptr, pt_main(ctx), head);
+    return forward_cached(ctx, rows_launch, st->draft_tok, nullptr, pt_main(ctx), head);
 }
 
 swift_status enqueue_accept(swift_ctx* ctx)
@@ -610,6 +669,33 @@ double forward_bytes(const swift_ctx* ctx, const uint8_t* skip, int n_rows, int 
 
 // =============================================================================== tensor maps
 namespace {
+
+template <typename T, int MR>
+cudaError_t set_attrs_mr()
+{
+    cudaError_t e = cudaFuncSetAttribute(gemm_simt_kernel<T, MR>, cudaFuncAttributeMaxDynamicSharedMemorySize, 16 * 1024 * 4);
+    if (e == cudaSuccess)
+        e = cudaFuncSetAttribute(attn_split_kernel<T, MR>, cudaFuncAttributeMaxDynamicSharedMemorySize, (16 * 256 + 16 * ATTN_CHUNK + 32) * 4);
+    return e;
+}
+template <typename T>
+cudaError_t set_attrs()
+{
+    cudaError_t e = set_attrs_mr<T, 1>();
+    if (e == cudaSuccess) e = set_attrs_mr<T, 2>();
+    if (e == cudaSuccess) e = set_attrs_mr<T, 4>();
+    if (e == cudaSuccess) e = set_attrs_mr<T, 8>();
+    if (e == cudaSuccess) e = set_attrs_mr<T, 16>();
+    return e;
+}
+// Opt-in shared-memory sizes of every kernel, set once per device before anything is captured.
+cudaError_t init_kernel_attrs()
+{
+    cudaError_t e = set_attrs<float>();
+    if (e == cudaSuccess) e = set_attrs<__nv_bfloat16>();
+    if (e == cudaSuccess) e = cudaFuncSetAttribute(gemm_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, TC_SMEM_BYTES);
+    return e;
+}
 
 // bf16 row-major [rows][cols] matrix, box = box_rows x 64 columns (128 bytes), 128-byte swizzle.
 swift_status make_map(swift_ctx* ctx, CUtensorMap* out, const void* base, uint64_t rows, uint64_t cols, uint32_t box_rows)
@@ -710,11 +796,14 @@ swift_status swift_load(const swift_model_desc* desc, swift_devbuf weights, swif
     c->use_tc = false;
     if (desc->dtype == SWIFT_BF16) {
         const swift_status ms = make_all_maps(c);
-        if (ms != SWIFT_OK) { g_load_error = c->err; delete c; return ms; }
+        if (ms != SWIFT_OK) { g_load_error = c->err; delete c; return ms; }   // (graphs not allocated yet)
         c->use_tc = true;
     }
     for (auto& e : c->ev) e = nullptr;
-    cudaError_t e = cudaSuccess;
+    c->use_graphs = true;
+    c->graphs = new std::vector<FwdGraph>();
+    c->graph_clock = 0;
+    cudaError_t e = init_kernel_attrs();
     for (auto& ev : c->ev) if (e == cudaSuccess) e = cudaEventCreate(&ev);
     if (e == cudaSuccess) e = cudaMemsetAsync(c->ws, 0, c->kl.total, c->stream);
     if (e == cudaSuccess) {
@@ -732,6 +821,7 @@ swift_status swift_load(const swift_model_desc* desc, swift_devbuf weights, swif
     if (e != cudaSuccess) {
         fail(nullptr, SWIFT_ECUDA, "set-up failed: %s", cudaGetErrorString(e));
         for (auto& ev : c->ev) if (ev) cudaEventDestroy(ev);
+        delete c->graphs;
         delete c;
         return SWIFT_ECUDA;
     }
@@ -744,6 +834,8 @@ swift_status swift_free(swift_ctx* ctx)
     if (!ctx) return SWIFT_OK;
     cudaStreamSynchronize(ctx->stream);
     for (auto& ev : ctx->ev) if (ev) cudaEventDestroy(ev);
+    for (auto& g : *ctx->graphs) cudaGraphExecDestroy(g.exec);
+    delete ctx->graphs;
     delete ctx;
     return SWIFT_OK;
 }
@@ -882,8 +974,7 @@ swift_status swift_verify(swift_ctx* ctx, const int32_t* tokens_host, int32_t k,
         if (ctx->n + k + 1 > ctx->d.max_positions) return fail(ctx, SWIFT_ECAPACITY, "KV cache too small");
         if (ctx->phase == PH_READY) {
             ctx->round++;
-            begin_round_kernel<<<1, 1, 0, ctx->stream>>>(state_of(ctx), ctx->pending, 1);
-            ctx->launches++;
+            launch_begin_round(ctx, 0.f);
             ctx->round_open = true;
         }
         if (k > 0) CU(cudaMemcpyAsync(state_of(ctx)->draft_tok + 1, tokens_host, k * 4, cudaMemcpyHostToDevice, ctx->stream));
@@ -1120,8 +1211,7 @@ swift_status swift_generate(swift_ctx* ctx, const swift_gen_params* gp, const in
         const int n_start = ctx->n;
         if (gp->vanilla) {
             ctx->round++;
-            begin_round_kernel<<<1, 1, 0, ctx->stream>>>(state_of(ctx), ctx->pending, 1);
-            ctx->launches++;
+            launch_begin_round(ctx, 0.f);
             ST(enqueue_verify(ctx, 1, 0));
             if (ctx->mode == SWIFT_SAMPLING) {
                 sample_row_kernel<<<1, VOCAB_THREADS, 0, ctx->stream>>>(state_of(ctx), kptr<float>(ctx, ctx->kl.logits), d.vocab, 0,
