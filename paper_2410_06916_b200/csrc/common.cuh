@@ -40,6 +40,15 @@ struct DevState {
     int pad[2];
 };
 
+// Programmatic dependent launch.  Every kernel of a forward is launched with programmatic stream
+// serialisation: it may start while its predecessor is still running, so it (a) lets its own successor
+// start early and (b) waits for the predecessor's completion and memory before touching anything the
+// predecessor produced.  Every thread calls pdl_wait() on every path, or the chain of completions
+// would be broken for the kernels that follow.  Without the launch attribute both are no-ops.
+__device__ __forceinline__ void pdl_trigger() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void pdl_enter() { pdl_trigger(); pdl_wait(); }
+
 template <typename T> struct Vec;
 template <> struct Vec<float> { static constexpr int N = 4; };
 template <> struct Vec<__nv_bfloat16> { static constexpr int N = 8; };

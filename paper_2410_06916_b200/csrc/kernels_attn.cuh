@@ -18,6 +18,7 @@ attn_split_kernel(const DevState* st, const float* __restrict__ q, const T* __re
                   const int* __restrict__ page_table, KvLayout L, int block, int n_heads, int max_splits,
                   float scale, float* __restrict__ o_part, float2* __restrict__ ml_part)
 {
+    pdl_enter();
     constexpr int VEC = Vec<T>::N;
     const int n_rows = min(st->n_rows, MR);
     if (n_rows == 0) return;
@@ -105,6 +106,7 @@ __global__ void attn_combine_kernel(const DevState* st, const float* __restrict_
                                     const float2* __restrict__ ml_part, int max_splits, int n_heads, int dh,
                                     float* __restrict__ out, __nv_bfloat16* __restrict__ planes)
 {
+    pdl_enter();
     const int r = blockIdx.y;
     if (r >= st->n_rows) return;
     const int h = blockIdx.x, d = threadIdx.x;

@@ -93,6 +93,7 @@ template <typename T>
 __global__ void embed_kernel(DevState* st, const int* __restrict__ toks, const T* __restrict__ embed,
                              float* __restrict__ h, int d, int vocab)
 {
+    pdl_enter();
     const int r = blockIdx.x;
     if (r >= st->n_rows) return;
     int tok = toks[st->tok_off + r];
@@ -113,6 +114,7 @@ __global__ void __launch_bounds__(512) resid_norm_kernel(const DevState* st, flo
                                                          float* __restrict__ x, __nv_bfloat16* __restrict__ planes,
                                                          int d, float eps)
 {
+    pdl_enter();
     __shared__ float red[33];
     const int r = blockIdx.x;
     if (r >= st->n_rows) return;
@@ -143,6 +145,7 @@ __global__ void qkv_post_kernel(const DevState* st, const float* __restrict__ pa
                                 const int* __restrict__ page_table, KvLayout L, int block, int n_heads,
                                 const float2* __restrict__ rope_cs, int max_positions)
 {
+    pdl_enter();
     const int r = blockIdx.x;
     if (r >= st->n_rows) return;
     const int head = blockIdx.y, half = L.head_dim >> 1, i = threadIdx.x;
@@ -182,6 +185,7 @@ __global__ void qkv_post_kernel(const DevState* st, const float* __restrict__ pa
 __global__ void swiglu_kernel(const DevState* st, const float* __restrict__ part, int n_split, size_t split_stride,
                               float* __restrict__ act, __nv_bfloat16* __restrict__ planes, int ffn)
 {
+    pdl_enter();
     const int r = blockIdx.y;
     if (r >= st->n_rows) return;
     const int i = blockIdx.x * blockDim.x + threadIdx.x;

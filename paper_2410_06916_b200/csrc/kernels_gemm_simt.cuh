@@ -20,6 +20,7 @@ __global__ void __launch_bounds__(GEMM_SIMT_THREADS)
 gemm_simt_kernel(const DevState* st, const float* __restrict__ X, int ldx, const T* __restrict__ W,
                  float* __restrict__ Ypart, int N, int K, int Kc)
 {
+    pdl_enter();
     constexpr int VEC = Vec<T>::N;
     constexpr int R = GEMM_SIMT_R;
     const int n_rows = min(st->n_rows, MR);

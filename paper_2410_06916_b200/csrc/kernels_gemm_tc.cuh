@@ -30,7 +30,7 @@ namespace swk {
 constexpr int TC_TILE_N = 128;      // weight rows per tile (MMA M)
 constexpr int TC_COLS = 32;         // operand rows of X: 16 hi + 16 lo (MMA N)
 constexpr int TC_BK = 64;           // k elements per stage: 128 bytes of bf16 = one swizzle row
-constexpr int TC_STAGES = 8;
+constexpr int TC_STAGES = 5;       // 100 KB of shared memory: two CTAs (successive GEMMs) fit on one SM
 constexpr int TC_THREADS = 192;
 constexpr int TC_A_BYTES = TC_TILE_N * TC_BK * 2;   // 16384
 constexpr int TC_B_BYTES = TC_COLS * TC_BK * 2;     // 4096
@@ -120,15 +120,14 @@ __global__ void __launch_bounds__(TC_THREADS, 1)
 gemm_tc_kernel(DevState* st, const __grid_constant__ CUtensorMap mapW, const __grid_constant__ CUtensorMap mapX,
                float* __restrict__ Y, float* __restrict__ slabs, int* __restrict__ counters, int N, int K)
 {
-    const int n_rows = st->n_rows;
-    if (n_rows == 0) return;
+    pdl_trigger();
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int n_tiles = (N + TC_TILE_N - 1) / TC_TILE_N;
     StreamK sk;
     sk.KB = (K + TC_BK - 1) / TC_BK;
     sk.U = (long long)n_tiles * sk.KB;
     sk.G = (int)(sk.U < (long long)gridDim.x ? sk.U : (long long)gridDim.x);   // never more CTAs than units: no empty ranges
-    if ((int)blockIdx.x >= sk.G) return;
+    if ((int)blockIdx.x >= sk.G) { pdl_wait(); return; }
     const long long u_begin = sk.start(blockIdx.x), u_end = sk.start(blockIdx.x + 1);
 
     extern __shared__ unsigned char smem_raw[];
@@ -163,8 +162,22 @@ gemm_tc_kernel(DevState* st, const __grid_constant__ CUtensorMap mapW, const __g
         if (lane == 0) {
             asm volatile("prefetch.tensormap [%0];" ::"l"(&mapW) : "memory");
             asm volatile("prefetch.tensormap [%0];" ::"l"(&mapX) : "memory");
-            int it = 0;
-            for (long long u = u_begin; u < u_end; ++u, ++it) {
+            // Weights do not depend on the preceding kernel: the first ring-full is requested before
+            // waiting for it, so that HBM is already streaming when the activations become valid.
+            const int n_pre = (int)((u_end - u_begin) < TC_STAGES ? (u_end - u_begin) : TC_STAGES);
+            for (int i = 0; i < n_pre; ++i) {
+                const long long u = u_begin + i;
+                mbar_expect_tx(full_bar(i), TC_STAGE_BYTES);
+                tma_load_2d(base + i * TC_STAGE_BYTES, &mapW, (int)(u % sk.KB) * TC_BK, (int)(u / sk.KB) * TC_TILE_N, full_bar(i));
+            }
+            pdl_wait();
+            for (int i = 0; i < n_pre; ++i)
+                tma_load_2d(base + i * TC_STAGE_BYTES + TC_A_BYTES, &mapX, (int)((u_begin + i) % sk.KB) * TC_BK, 0, full_bar(i));
+            if (st->n_rows == 0) {                      // nothing to compute: let the requested tiles land, then leave
+                for (int i = 0; i < n_pre; ++i) mbar_wait(full_bar(i), 0);
+            } else {
+            int it = n_pre;
+            for (long long u = u_begin + n_pre; u < u_end; ++u, ++it) {
                 const int tile = (int)(u / sk.KB), kb = (int)(u % sk.KB);
                 const int s = it % TC_STAGES;
                 if (!mbar_wait(empty_bar(s), ((it / TC_STAGES) & 1) ^ 1)) { abort_sh = 1; break; }
@@ -173,10 +186,14 @@ gemm_tc_kernel(DevState* st, const __grid_constant__ CUtensorMap mapW, const __g
                 tma_load_2d(a_dst, &mapW, kb * TC_BK, tile * TC_TILE_N, full_bar(s));
                 tma_load_2d(b_dst, &mapX, kb * TC_BK, 0, full_bar(s));
             }
+            }
+        } else {
+            pdl_wait();
         }
     } else if (warp == 1) {
         // ---------------------------------------------------------------- MMA issuer
-        if (lane == 0) {
+        pdl_wait();
+        if (lane == 0 && st->n_rows != 0) {
             int it = 0, seg = 0;
             for (long long u = u_begin; u < u_end; ++u, ++it) {
                 const int tile = (int)(u / sk.KB), kb = (int)(u % sk.KB);
@@ -202,10 +219,12 @@ gemm_tc_kernel(DevState* st, const __grid_constant__ CUtensorMap mapW, const __g
         }
     } else {
         // ---------------------------------------------------------------- epilogue (warps 2..5)
+        pdl_wait();
+        const int n_rows = st->n_rows;
         const int quarter = warp & 3;                  // TMEM lanes this warp may read: 32*quarter ..
         const int etid = tid - 64;                     // 0..127
         int seg = 0;
-        long long u = u_begin;
+        long long u = n_rows != 0 ? u_begin : u_end;
         while (u < u_end) {
             const int tile = (int)(u / sk.KB), kb0 = (int)(u % sk.KB);
             const long long tile_end = (long long)(tile + 1) * sk.KB;

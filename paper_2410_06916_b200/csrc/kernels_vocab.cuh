@@ -88,6 +88,7 @@ __global__ void __launch_bounds__(VOCAB_THREADS)
 vocab_kernel(DevState* st, const float* __restrict__ part, int n_split, size_t split_stride,
              float* __restrict__ logits, int vocab, float inv_temp, int mode, int sampling, float* __restrict__ q_rows)
 {
+    pdl_enter();
     __shared__ float sh[VOCAB_THREADS + 72];
     __shared__ ArgMax sh_am[32];
     const int r = blockIdx.x;

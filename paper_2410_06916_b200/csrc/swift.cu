@@ -73,8 +73,8 @@ struct swift_ctx {
     int64_t launches;
     std::string err;
     cudaEvent_t ev[8];
-    // captured forwards
-    bool use_graphs;
+    // captured forwards; programmatic dependent launch between the kernels of a forward
+    bool use_graphs, use_pdl;
     std::vector<FwdGraph>* graphs;
     uint64_t graph_clock;
     // tensor-core GEMM path (bf16 models)
@@ -244,15 +244,31 @@ DevState* state_of(swift_ctx* c) { return kptr<DevState>(c, c->kl.state); }
 int mr_of(int rows) { return rows <= 1 ? 1 : rows <= 2 ? 2 : rows <= 4 ? 4 : rows <= 8 ? 8 : 16; }
 
 // ------------------------------------------------------------------------------ launches
+// Launch with programmatic stream serialisation (see pdl_enter in common.cuh).
+template <typename... KArgs, typename... Args>
+cudaError_t launch_k(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, swift_ctx* ctx, Args&&... args)
+{
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid;
+    cfg.blockDim = block;
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = ctx->stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = ctx->use_pdl ? 1 : 0;
+    ctx->launches++;
+    return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
+}
+
 template <typename T, int MR>
 swift_status launch_gemm_mr(swift_ctx* ctx, const float* X, int ldx, const T* W, int N, int K, GemmPlan p)
 {
     const size_t smem = (size_t)MR * p.Kc * sizeof(float);
     dim3 grid(ceil_div(N, GEMM_SIMT_TILE_N), p.S);
-    gemm_simt_kernel<T, MR><<<grid, GEMM_SIMT_THREADS, smem, ctx->stream>>>(state_of(ctx), X, ldx, W,
-                                                                            kptr<float>(ctx, ctx->kl.part), N, K, p.Kc);
-    ctx->launches++;
-    CU(cudaGetLastError());
+    CU(launch_k(gemm_simt_kernel<T, MR>, grid, dim3(GEMM_SIMT_THREADS), smem, ctx, (const DevState*)state_of(ctx), X, ldx, W,
+                kptr<float>(ctx, ctx->kl.part), N, K, p.Kc));
     return SWIFT_OK;
 }
 
@@ -282,11 +298,8 @@ struct GemmSite {
 swift_status launch_gemm_tc(swift_ctx* ctx, const GemmSite& g)
 {
     if (ceil_div(g.N, TC_TILE_N) > TC_MAX_TILES) return fail(ctx, SWIFT_EUNSUPPORTED, "GEMM with %d output tiles", ceil_div(g.N, TC_TILE_N));
-    gemm_tc_kernel<<<TC_GRID, TC_THREADS, TC_SMEM_BYTES, ctx->stream>>>(state_of(ctx), *g.mapW, *g.mapX,
-                                                                       kptr<float>(ctx, ctx->kl.part), kptr<float>(ctx, ctx->kl.slabs),
-                                                                       kptr<int>(ctx, ctx->kl.counters), g.N, g.K);
-    ctx->launches++;
-    CU(cudaGetLastError());
+    CU(launch_k(gemm_tc_kernel, dim3(TC_GRID), dim3(TC_THREADS), (size_t)TC_SMEM_BYTES, ctx, state_of(ctx), *g.mapW, *g.mapX,
+                kptr<float>(ctx, ctx->kl.part), kptr<float>(ctx, ctx->kl.slabs), kptr<int>(ctx, ctx->kl.counters), g.N, g.K));
     return SWIFT_OK;
 }
 
@@ -310,12 +323,10 @@ swift_status launch_attn_mr(swift_ctx* ctx, const int* page_table, int block)
     const swift_model_desc& d = ctx->d;
     const size_t smem = ((size_t)MR * d.head_dim + (size_t)MR * ATTN_CHUNK + 2 * MR) * sizeof(float);
     dim3 grid(d.n_heads, ctx->max_splits);
-    attn_split_kernel<T, MR><<<grid, ATTN_THREADS, smem, ctx->stream>>>(
-        state_of(ctx), kptr<float>(ctx, ctx->kl.q), reinterpret_cast<const T*>(ctx->kvbase), page_table, ctx->kv, block,
-        d.n_heads, ctx->max_splits, 1.0f / sqrtf((float)d.head_dim), kptr<float>(ctx, ctx->kl.o_part),
-        kptr<float2>(ctx, ctx->kl.ml_part));
-    ctx->launches++;
-    CU(cudaGetLastError());
+    CU(launch_k(attn_split_kernel<T, MR>, grid, dim3(ATTN_THREADS), smem, ctx, (const DevState*)state_of(ctx),
+                (const float*)kptr<float>(ctx, ctx->kl.q), reinterpret_cast<const T*>(ctx->kvbase), page_table, ctx->kv, block,
+                d.n_heads, ctx->max_splits, 1.0f / sqrtf((float)d.head_dim), kptr<float>(ctx, ctx->kl.o_part),
+                kptr<float2>(ctx, ctx->kl.ml_part)));
     return SWIFT_OK;
 }
 
@@ -365,47 +376,40 @@ swift_status forward_chunk(swift_ctx* ctx, int rows, const int* toks_dev, const 
     const float* pend = nullptr;      // pending residual-branch output (split-K slabs) not yet added to h
     int pend_S = 0, S = 0;
 
-    embed_kernel<T><<<rows, 256, 0, s>>>(st, toks_dev, wptr<T>(ctx, ctx->wl.embed), h, dm, d.vocab);
-    ctx->launches++;
+    CU(launch_k(embed_kernel<T>, dim3(rows), dim3(256), 0, ctx, st, toks_dev, (const T*)wptr<T>(ctx, ctx->wl.embed), h, dm, d.vocab));
     for (int b = 0; b < d.n_blocks; ++b) {
         if (!(skip && skip[2 * b])) {
-            resid_norm_kernel<<<rows, 512, 0, s>>>(st, h, pend, pend_S, (size_t)ROWS * dm,
-                                                   wptr<float>(ctx, ctx->wl.attn_norm[b]), xn, xn_hl, dm, d.rms_eps);
-            ctx->launches++;
+            CU(launch_k(resid_norm_kernel, dim3(rows), dim3(512), 0, ctx, (const DevState*)st, h, pend, pend_S, (size_t)ROWS * dm,
+                        (const float*)wptr<float>(ctx, ctx->wl.attn_norm[b]), xn, xn_hl, dm, d.rms_eps));
             ST(run_gemm<T>(ctx, mr, GemmSite{xn, nqkv, dm, wptr<T>(ctx, ctx->wl.wqkv[b]), tc ? &ctx->tm_wqkv[b] : nullptr, &ctx->tm_xn}, &S));
-            qkv_post_kernel<TKV><<<dim3(rows, d.n_heads + 2 * d.n_kv_heads), d.head_dim / 2, 0, s>>>(
-                st, part, S, (size_t)ROWS * nqkv, nqkv, kptr<float>(ctx, ctx->kl.q), reinterpret_cast<TKV*>(ctx->kvbase),
-                page_table, ctx->kv, b, d.n_heads, kptr<float2>(ctx, ctx->kl.rope), d.max_positions);
-            ctx->launches++;
+            CU(launch_k(qkv_post_kernel<TKV>, dim3(rows, d.n_heads + 2 * d.n_kv_heads), dim3(d.head_dim / 2), 0, ctx,
+                        (const DevState*)st, (const float*)part, S, (size_t)ROWS * nqkv, nqkv, kptr<float>(ctx, ctx->kl.q),
+                        reinterpret_cast<TKV*>(ctx->kvbase), page_table, ctx->kv, b, d.n_heads,
+                        (const float2*)kptr<float2>(ctx, ctx->kl.rope), d.max_positions));
             ST(launch_attn<TKV>(ctx, mr, page_table, b));
-            attn_combine_kernel<<<dim3(d.n_heads, rows), d.head_dim, 0, s>>>(
-                st, kptr<float>(ctx, ctx->kl.o_part), kptr<float2>(ctx, ctx->kl.ml_part), ctx->max_splits, d.n_heads,
-                d.head_dim, xa, xa_hl);
-            ctx->launches++;
+            CU(launch_k(attn_combine_kernel, dim3(d.n_heads, rows), dim3(d.head_dim), 0, ctx, (const DevState*)st,
+                        (const float*)kptr<float>(ctx, ctx->kl.o_part), (const float2*)kptr<float2>(ctx, ctx->kl.ml_part),
+                        ctx->max_splits, d.n_heads, d.head_dim, xa, xa_hl));
             ST(run_gemm<T>(ctx, mr, GemmSite{xa, dm, qd, wptr<T>(ctx, ctx->wl.wo[b]), tc ? &ctx->tm_wo[b] : nullptr, &ctx->tm_xa}, &S));
             pend = part; pend_S = S;
         }
         if (!(skip && skip[2 * b + 1])) {
-            resid_norm_kernel<<<rows, 512, 0, s>>>(st, h, pend, pend_S, (size_t)ROWS * dm,
-                                                   wptr<float>(ctx, ctx->wl.mlp_norm[b]), xn, xn_hl, dm, d.rms_eps);
-            ctx->launches++;
+            CU(launch_k(resid_norm_kernel, dim3(rows), dim3(512), 0, ctx, (const DevState*)st, h, pend, pend_S, (size_t)ROWS * dm,
+                        (const float*)wptr<float>(ctx, ctx->wl.mlp_norm[b]), xn, xn_hl, dm, d.rms_eps));
             ST(run_gemm<T>(ctx, mr, GemmSite{xn, 2 * d.ffn, dm, wptr<T>(ctx, ctx->wl.wgu[b]), tc ? &ctx->tm_wgu[b] : nullptr, &ctx->tm_xn}, &S));
-            swiglu_kernel<<<dim3(ceil_div(d.ffn, 256), rows), 256, 0, s>>>(st, part, S, (size_t)ROWS * 2 * d.ffn, act, act_hl, d.ffn);
-            ctx->launches++;
+            CU(launch_k(swiglu_kernel, dim3(ceil_div(d.ffn, 256), rows), dim3(256), 0, ctx, (const DevState*)st, (const float*)part, S,
+                        (size_t)ROWS * 2 * d.ffn, act, act_hl, d.ffn));
             ST(run_gemm<T>(ctx, mr, GemmSite{act, dm, d.ffn, wptr<T>(ctx, ctx->wl.wdown[b]), tc ? &ctx->tm_wdown[b] : nullptr, &ctx->tm_act}, &S));
             pend = part; pend_S = S;
         }
     }
     if (head.run) {
-        resid_norm_kernel<<<rows, 512, 0, s>>>(st, h, pend, pend_S, (size_t)ROWS * dm,
-                                               wptr<float>(ctx, ctx->wl.final_norm), xn, xn_hl, dm, d.rms_eps);
-        ctx->launches++;
+        CU(launch_k(resid_norm_kernel, dim3(rows), dim3(512), 0, ctx, (const DevState*)st, h, pend, pend_S, (size_t)ROWS * dm,
+                    (const float*)wptr<float>(ctx, ctx->wl.final_norm), xn, xn_hl, dm, d.rms_eps));
         ST(run_gemm<T>(ctx, mr, GemmSite{xn, d.vocab, dm, wptr<T>(ctx, ctx->wl.lm_head), &ctx->tm_lm_head, &ctx->tm_xn}, &S));
-        vocab_kernel<<<rows, VOCAB_THREADS, 0, s>>>(st, part, S, (size_t)ROWS * d.vocab,
-                                                   kptr<float>(ctx, ctx->kl.logits), d.vocab, 1.0f / ctx->temperature,
-                                                   head.mode, ctx->mode == SWIFT_SAMPLING ? 1 : 0,
-                                                   kptr<float>(ctx, ctx->kl.q_rows));
-        ctx->launches++;
+        CU(launch_k(vocab_kernel, dim3(rows), dim3(VOCAB_THREADS), 0, ctx, st, (const float*)part, S, (size_t)ROWS * d.vocab,
+                    kptr<float>(ctx, ctx->kl.logits), d.vocab, 1.0f / ctx->temperature, head.mode,
+                    ctx->mode == SWIFT_SAMPLING ? 1 : 0, kptr<float>(ctx, ctx->kl.q_rows)));
     }
     CU(cudaGetLastError());
     return SWIFT_OK;
@@ -426,7 +430,7 @@ swift_status forward_chunk_any(swift_ctx* ctx, int rows, const int* toks_dev, co
 // sequence is captured once into a CUDA graph and replayed: one graph launch instead of several
 // hundred kernel launches per forward.
 struct FwdKey {
-    int rows, head_run, head_mode, sampling, use_tc;
+    int rows, head_run, head_mode, sampling, use_tc, use_pdl;
     float temperature;
     const void* toks;
     const void* page_table;
@@ -434,7 +438,7 @@ struct FwdKey {
     bool operator==(const FwdKey& o) const
     {
         return rows == o.rows && head_run == o.head_run && head_mode == o.head_mode && sampling == o.sampling &&
-               use_tc == o.use_tc && temperature == o.temperature && toks == o.toks && page_table == o.page_table && mask == o.mask;
+               use_tc == o.use_tc && use_pdl == o.use_pdl && temperature == o.temperature && toks == o.toks && page_table == o.page_table && mask == o.mask;
     }
 };
 struct FwdGraph {
@@ -449,7 +453,7 @@ swift_status forward_cached(swift_ctx* ctx, int rows, const int* toks_dev, const
 {
     if (!ctx->use_graphs) return forward_chunk_any(ctx, rows, toks_dev, skip, page_table, head);
     const int L = 2 * ctx->d.n_blocks;
-    FwdKey key{rows, head.run ? 1 : 0, head.mode, ctx->mode, ctx->use_tc ? 1 : 0, ctx->temperature, toks_dev, page_table,
+    FwdKey key{rows, head.run ? 1 : 0, head.mode, ctx->mode, ctx->use_tc ? 1 : 0, ctx->use_pdl ? 1 : 0, ctx->temperature, toks_dev, page_table,
                skip ? std::vector<uint8_t>(skip, skip + L) : std::vector<uint8_t>()};
     auto& cache = *ctx->graphs;
     ctx->graph_clock++;
@@ -800,7 +804,8 @@ swift_status swift_load(const swift_model_desc* desc, swift_devbuf weights, swif
         c->use_tc = true;
     }
     for (auto& e : c->ev) e = nullptr;
-    c->use_graphs = true;
+    c->use_graphs = getenv("SWIFT_NO_GRAPHS") == nullptr;
+    c->use_pdl = getenv("SWIFT_NO_PDL") == nullptr;
     c->graphs = new std::vector<FwdGraph>();
     c->graph_clock = 0;
     cudaError_t e = init_kernel_attrs();
