@@ -7,7 +7,7 @@
 namespace swk {
 
 constexpr int ROWS = 16;          // rows of one forward chunk (pending token + up to 15 drafts)
-constexpr int ATTN_CHUNK = 256;   // KV positions per attention split; anchored at multiples of this
+constexpr int ATTN_CHUNK = 64;    // KV positions per attention split; anchored at multiples of this
 constexpr int MAX_SCORE_ROWS = 128;
 
 // purposes of a random draw inside one decoding round (Philox counter word 2)

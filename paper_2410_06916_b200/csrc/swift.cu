@@ -321,7 +321,7 @@ template <typename T, int MR>
 swift_status launch_attn_mr(swift_ctx* ctx, const int* page_table, int block)
 {
     const swift_model_desc& d = ctx->d;
-    const size_t smem = ((size_t)MR * d.head_dim + (size_t)MR * ATTN_CHUNK + 2 * MR) * sizeof(float);
+    const size_t smem = 2 * (size_t)ATTN_CHUNK * d.head_dim * sizeof(T) + ((size_t)MR * d.head_dim + 3 * (size_t)MR * ATTN_CHUNK) * sizeof(float);
     dim3 grid(d.n_heads, ctx->max_splits);
     CU(launch_k(attn_split_kernel<T, MR>, grid, dim3(ATTN_THREADS), smem, ctx, (const DevState*)state_of(ctx),
                 (const float*)kptr<float>(ctx, ctx->kl.q), reinterpret_cast<const T*>(ctx->kvbase), page_table, ctx->kv, block,
@@ -508,6 +508,7 @@ swift_status read_state(swift_ctx* ctx, DevState* out)
             CU(cudaMemsetAsync(kptr<int>(ctx, ctx->kl.counters), 0, TC_MAX_TILES * 4, ctx->stream));
             return fail(ctx, SWIFT_ETIMEOUT, "a bounded wait inside the tensor-core GEMM ran out");
         }
+        if (code == 3) return fail(ctx, SWIFT_ETIMEOUT, "a bounded wait inside the attention kernel ran out");
         return fail(ctx, SWIFT_EINVAL, "device reported an invalid token id");
     }
     return SWIFT_OK;
@@ -679,7 +680,8 @@ cudaError_t set_attrs_mr()
 {
     cudaError_t e = cudaFuncSetAttribute(gemm_simt_kernel<T, MR>, cudaFuncAttributeMaxDynamicSharedMemorySize, 16 * 1024 * 4);
     if (e == cudaSuccess)
-        e = cudaFuncSetAttribute(attn_split_kernel<T, MR>, cudaFuncAttributeMaxDynamicSharedMemorySize, (16 * 256 + 16 * ATTN_CHUNK + 32) * 4);
+        e = cudaFuncSetAttribute(attn_split_kernel<T, MR>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                 (int)(2 * ATTN_CHUNK * 256 * sizeof(T) + (MR * 256 + 3 * MR * ATTN_CHUNK) * 4));
     return e;
 }
 template <typename T>
