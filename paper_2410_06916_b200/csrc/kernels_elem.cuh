@@ -105,6 +105,34 @@ __global__ void embed_kernel(DevState* st, const int* __restrict__ toks, const T
     for (int i = threadIdx.x; i < d; i += blockDim.x) h[(size_t)r * d + i] = to_float(src[i]);
 }
 
+// Embedding gather for the fused tensor-core walk: besides h it stores the hi/lo planes of h * gain
+// (gain of the first RMSNorm that will see this row) and the row's sum of squares as "tile 0".
+template <typename T>
+__global__ void embed_fused_kernel(DevState* st, const int* __restrict__ toks, const T* __restrict__ embed,
+                                   float* __restrict__ h, const float* __restrict__ gain, __nv_bfloat16* __restrict__ planes,
+                                   float* __restrict__ sumsq_out, int d, int vocab)
+{
+    pdl_enter();
+    __shared__ float red[33];
+    const int r = blockIdx.x;
+    if (r >= st->n_rows) return;
+    int tok = toks[st->tok_off + r];
+    if (tok < 0 || tok >= vocab) {
+        if (threadIdx.x == 0) st->error = 1;
+        tok = 0;
+    }
+    const T* src = embed + (size_t)tok * d;
+    float ss = 0.f;
+    for (int i = threadIdx.x; i < d; i += blockDim.x) {
+        const float v = to_float(src[i]);
+        h[(size_t)r * d + i] = v;
+        if (gain) store_hi_lo(planes, r, d, i, v * gain[i]);
+        ss += v * v;
+    }
+    const float total = block_sum(ss, red);
+    if (threadIdx.x == 0) sumsq_out[r] = total;
+}
+
 // ------------------------------------------------------------------------------ residual + RMSNorm
 // h[r,:] += sum_s part[s][r][:]  (the pending output of the previous residual branch, split-K
 // partial sums added in split order), then x[r,:] = h * rsqrt(mean(h^2) + eps) * g.

@@ -113,12 +113,144 @@ struct StreamK {
     }
 };
 
+// fp32 rows -> the two bf16 planes the tensor-core GEMM reads: plane[r] = bf16(x), plane[16 + r] = bf16(x - hi).
+__device__ __forceinline__ void store_hi_lo(__nv_bfloat16* planes, int r, int K, int i, float x)
+{
+    const __nv_bfloat16 hi = __float2bfloat16_rn(x);
+    planes[(size_t)r * K + i] = hi;
+    planes[(size_t)(ROWS + r) * K + i] = __float2bfloat16_rn(x - __bfloat162float(hi));
+}
+
+// What the epilogue does with a finished output tile.  The element-wise steps of the decoder walk are
+// folded in here so that a block of the model is four GEMM launches plus the attention pair:
+//   EPI_PLAIN : Y = acc * rstd                                    (output head; rstd = 1 without a norm)
+//   EPI_QKV   : acc * rstd -> RoPE on q and k -> q buffer (fp32) and K,V into the paged cache
+//   EPI_SWIGLU: acc * rstd -> silu(gate) * up -> hi/lo planes of the down projection's input
+//   EPI_RESID : h += acc; hi/lo planes of h * gain_next; per-tile sums of h^2 for the next RMSNorm
+// RMSNorm is split around the GEMM that follows it: the producer (EPI_RESID, or the embedding gather)
+// stores h * gain and the row's sum of squares in per-tile pieces; the consumer multiplies its
+// accumulators by rstd = rsqrt(sum / d + eps), which is the same product in a different order.
+enum { EPI_PLAIN = 0, EPI_QKV = 1, EPI_SWIGLU = 2, EPI_RESID = 3 };
+
+struct EpiParams {
+    // consumer side of the norm
+    const float* sumsq_in;   // [n_sumsq_tiles][ROWS] or null (no norm in front of this GEMM)
+    int n_sumsq_tiles;
+    float inv_d, eps;
+    // EPI_RESID
+    float* h;                       // [ROWS][N] residual stream
+    const float* gain_next;         // [N] gain of the next RMSNorm, or null when nothing follows
+    __nv_bfloat16* planes_out;      // [2*ROWS][N]
+    float* sumsq_out;               // [n_tiles][ROWS]
+    // EPI_SWIGLU
+    __nv_bfloat16* act_planes;      // [2*ROWS][ffn]
+    int ffn;
+    // EPI_QKV
+    float* q_out;                   // [ROWS][n_heads*dh]
+    void* kv_pool;
+    const int* page_table;
+    KvLayout L;
+    int block, n_heads, max_positions;
+    const float2* rope_cs;
+};
+
+template <int EPI, typename TKV>
+__device__ __forceinline__ void tc_finalize(const EpiParams& ep, const DevState* st, float (&val)[ROWS], int n_rows, int tile,
+                                            int quarter, int lane, int etid, int N, float* Y, const float* rstd_sh,
+                                            float* stage_sh)
+{
+    const int l = quarter * 32 + lane;                 // row of the tile
+    const int n = tile * TC_TILE_N + l;
+    if (EPI != EPI_RESID) {
+#pragma unroll
+        for (int m = 0; m < ROWS; ++m) val[m] *= rstd_sh[m];
+    }
+    if (EPI == EPI_PLAIN) {
+        if (n < N) {
+#pragma unroll
+            for (int m = 0; m < ROWS; ++m)
+                if (m < n_rows) Y[(size_t)m * N + n] = val[m];
+        }
+    } else if (EPI == EPI_SWIGLU) {
+        // rows come in groups of 32: 16 gate rows then the 16 matching up rows
+        const int i = (n >> 5) * 16 + (lane & 15);
+#pragma unroll
+        for (int m = 0; m < ROWS; ++m) {
+            const float up = __shfl_down_sync(0xFFFFFFFFu, val[m], 16);
+            if (lane < 16 && m < n_rows && i < ep.ffn) {
+                const float g = val[m];
+                store_hi_lo(ep.act_planes, m, ep.ffn, i, g / (1.f + expf(-g)) * up);
+            }
+        }
+    } else if (EPI == EPI_RESID) {
+        float sq[ROWS];
+#pragma unroll
+        for (int m = 0; m < ROWS; ++m) {
+            sq[m] = 0.f;
+            if (n < N && m < n_rows) {
+                const float hn = ep.h[(size_t)m * N + n] + val[m];
+                ep.h[(size_t)m * N + n] = hn;
+                if (ep.gain_next) store_hi_lo(ep.planes_out, m, N, n, hn * ep.gain_next[n]);
+                sq[m] = hn * hn;
+            }
+        }
+        if (ep.gain_next) {                            // uniform over the grid
+#pragma unroll
+            for (int m = 0; m < ROWS; ++m) {
+                const float w = warp_sum(sq[m]);
+                if (lane == 0) stage_sh[quarter * ROWS + m] = w;
+            }
+            asm volatile("bar.sync 1, 128;" ::: "memory");
+            if (etid < ROWS)
+                ep.sumsq_out[(size_t)tile * ROWS + etid] =
+                    (stage_sh[etid] + stage_sh[ROWS + etid]) + (stage_sh[2 * ROWS + etid] + stage_sh[3 * ROWS + etid]);
+            asm volatile("bar.sync 1, 128;" ::: "memory");
+        }
+    } else {   // EPI_QKV
+        // exchange through shared memory: the RoPE partner of row l sits dh/2 rows away in the same tile
+#pragma unroll
+        for (int m = 0; m < ROWS; ++m) stage_sh[m * TC_TILE_N + l] = val[m];
+        asm volatile("bar.sync 1, 128;" ::: "memory");
+        const int dh = ep.L.head_dim, half = dh >> 1;
+        const int gh = n / dh, i = n - gh * dh;        // global head index (q heads, then k heads, then v heads), dim
+        const int lp = i < half ? l + half : l - half;
+        const int pos0 = st->pos0;
+        TKV* pool = reinterpret_cast<TKV*>(ep.kv_pool);
+        if (n < N) {
+#pragma unroll
+            for (int m = 0; m < ROWS; ++m) {
+                const int pos = pos0 + m;
+                if (m < n_rows && pos < ep.max_positions) {
+                    const float a = val[m], b = stage_sh[m * TC_TILE_N + lp];
+                    float out = a;
+                    if (gh < ep.n_heads + ep.L.n_kv_heads) {      // q or k: rotate
+                        const float2 cs = ep.rope_cs[(size_t)pos * half + (i < half ? i : i - half)];
+                        out = i < half ? a * cs.x - b * cs.y : a * cs.x + b * cs.y;
+                    }
+                    if (gh < ep.n_heads) {
+                        ep.q_out[(size_t)m * ep.n_heads * dh + n] = out;
+                    } else {
+                        const int hk = gh - ep.n_heads;
+                        const int kv = hk >= ep.L.n_kv_heads ? 1 : 0;
+                        const int kh = kv ? hk - ep.L.n_kv_heads : hk;
+                        const int page = ep.page_table[pos >> ep.L.page_shift];
+                        store_val(pool + ep.L.offset(page, ep.block, kv, kh, pos & (ep.L.page_size - 1)) + i, out);
+                    }
+                }
+            }
+        }
+        asm volatile("bar.sync 1, 128;" ::: "memory");   // staging buffer is reused by the next tile
+    }
+}
+
 // grid = G persistent CTAs, block = 192 threads, dynamic smem = TC_SMEM_BYTES.
 // mapW: bf16 [N][K], box {64, 128}; mapX: bf16 [32][K] (rows 0-15 hi, 16-31 lo), box {64, 32}; both
 // 128-byte swizzled.  slabs: [S_max][ROWS][N] fp32; counters: one int per tile, zero on entry and on exit.
+template <int EPI, typename TKV>
 __global__ void __launch_bounds__(TC_THREADS, 1)
 gemm_tc_kernel(DevState* st, const __grid_constant__ CUtensorMap mapW, const __grid_constant__ CUtensorMap mapX,
-               float* __restrict__ Y, float* __restrict__ slabs, int* __restrict__ counters, int N, int K)
+               float* __restrict__ Y, float* __restrict__ slabs, int* __restrict__ counters, int N, int K,
+               const __grid_constant__ EpiParams ep)
 {
     pdl_trigger();
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -140,6 +272,8 @@ gemm_tc_kernel(DevState* st, const __grid_constant__ CUtensorMap mapW, const __g
     __shared__ uint32_t tmem_base_sh;
     __shared__ int last_flag_sh;
     __shared__ int abort_sh, epi_abort_sh;
+    __shared__ float rstd_sh[ROWS];
+    __shared__ float stage_sh[EPI == EPI_QKV ? ROWS * TC_TILE_N : 4 * ROWS];
 
     if (tid == 0) {
         for (int s = 0; s < TC_STAGES; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
@@ -225,6 +359,16 @@ gemm_tc_kernel(DevState* st, const __grid_constant__ CUtensorMap mapW, const __g
         const int etid = tid - 64;                     // 0..127
         int seg = 0;
         long long u = n_rows != 0 ? u_begin : u_end;
+        if (etid < ROWS) {                             // rstd of the RMSNorm in front of this GEMM (1 when there is none)
+            float r = 1.f;
+            if (EPI != EPI_RESID && ep.sumsq_in) {
+                float ss = 0.f;
+                for (int t = 0; t < ep.n_sumsq_tiles; ++t) ss += ep.sumsq_in[(size_t)t * ROWS + etid];
+                r = rsqrtf(ss * ep.inv_d + ep.eps);
+            }
+            rstd_sh[etid] = r;
+        }
+        asm volatile("bar.sync 1, 128;" ::: "memory");
         while (u < u_end) {
             const int tile = (int)(u / sk.KB), kb0 = (int)(u % sk.KB);
             const long long tile_end = (long long)(tile + 1) * sk.KB;
@@ -252,36 +396,34 @@ gemm_tc_kernel(DevState* st, const __grid_constant__ CUtensorMap mapW, const __g
 
             const int n = tile * TC_TILE_N + quarter * 32 + lane;
             const bool whole = (kb0 == 0) && (seg_end == tile_end);   // this CTA covered the tile's whole K range
+            float val[ROWS];
+#pragma unroll
+            for (int m = 0; m < ROWS; ++m) val[m] = __uint_as_float(v[m]) + __uint_as_float(v[16 + m]);
             if (whole) {
-                if (n < N)
-                    for (int m = 0; m < ROWS; ++m)
-                        if (m < n_rows) Y[(size_t)m * N + n] = __uint_as_float(v[m]) + __uint_as_float(v[16 + m]);
+                tc_finalize<EPI, TKV>(ep, st, val, n_rows, tile, quarter, lane, etid, N, Y, rstd_sh, stage_sh);
             } else {
                 const int g_first = sk.owner((long long)tile * sk.KB), g_last = sk.owner(tile_end - 1);
                 const int slab = blockIdx.x - g_first, nseg = g_last - g_first + 1;
                 float* mine = slabs + (size_t)slab * ROWS * N;
                 if (n < N)
                     for (int m = 0; m < ROWS; ++m)
-                        if (m < n_rows) mine[(size_t)m * N + n] = __uint_as_float(v[m]) + __uint_as_float(v[16 + m]);
+                        if (m < n_rows) mine[(size_t)m * N + n] = val[m];
                 __threadfence();
                 asm volatile("bar.sync 1, 128;" ::: "memory");
                 if (etid == 0) last_flag_sh = (atomicAdd(&counters[tile], 1) == nseg - 1) ? 1 : 0;
                 asm volatile("bar.sync 1, 128;" ::: "memory");
                 if (last_flag_sh) {                             // last arrival: add the slabs in slab order
                     __threadfence();
-                    if (n < N) {
-                        float acc[ROWS];
 #pragma unroll
-                        for (int m = 0; m < ROWS; ++m) acc[m] = 0.f;
+                    for (int m = 0; m < ROWS; ++m) val[m] = 0.f;
+                    if (n < N) {
                         for (int j = 0; j < nseg; ++j) {            // slab order; the 16 row loads of a slab are independent
 #pragma unroll
                             for (int m = 0; m < ROWS; ++m)
-                                if (m < n_rows) acc[m] += __ldcg(slabs + ((size_t)j * ROWS + m) * N + n);
+                                if (m < n_rows) val[m] += __ldcg(slabs + ((size_t)j * ROWS + m) * N + n);
                         }
-#pragma unroll
-                        for (int m = 0; m < ROWS; ++m)
-                            if (m < n_rows) Y[(size_t)m * N + n] = acc[m];
                     }
+                    tc_finalize<EPI, TKV>(ep, st, val, n_rows, tile, quarter, lane, etid, N, Y, rstd_sh, stage_sh);
                     if (etid == 0) counters[tile] = 0;
                 }
                 asm volatile("bar.sync 1, 128;" ::: "memory");  // last_flag_sh is rewritten by the next segment
@@ -298,14 +440,6 @@ gemm_tc_kernel(DevState* st, const __grid_constant__ CUtensorMap mapW, const __g
         tc_fence_after();
         asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(64));
     }
-}
-
-// fp32 rows -> the two bf16 planes the tensor-core GEMM reads: plane[r] = bf16(x), plane[16 + r] = bf16(x - hi).
-__device__ __forceinline__ void store_hi_lo(__nv_bfloat16* planes, int r, int K, int i, float x)
-{
-    const __nv_bfloat16 hi = __float2bfloat16_rn(x);
-    planes[(size_t)r * K + i] = hi;
-    planes[(size_t)(ROWS + r) * K + i] = __float2bfloat16_rn(x - __bfloat162float(hi));
 }
 
 // grid = (ceil(K/256), rows): splits fp32 rows [rows][K] into the planes (used when a caller supplies X directly)

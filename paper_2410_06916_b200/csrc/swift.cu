@@ -47,7 +47,7 @@ struct WeightLayout {
 
 struct WorkLayout {
     size_t state, h, xn, xa, act, q, part, o_part, ml_part, logits, q_rows, rope, pt_main, pt_score, score_tok,
-        score_truth, score_out, xn_hl, xa_hl, act_hl, slabs, counters, total;
+        score_truth, score_out, xn_hl, xa_hl, act_hl, slabs, counters, sumsq, total;
     size_t part_floats, slab_floats;
 };
 
@@ -74,7 +74,7 @@ struct swift_ctx {
     std::string err;
     cudaEvent_t ev[8];
     // captured forwards; programmatic dependent launch between the kernels of a forward
-    bool use_graphs, use_pdl;
+    bool use_graphs, use_pdl, fuse;
     std::vector<FwdGraph>* graphs;
     uint64_t graph_clock;
     // tensor-core GEMM path (bf16 models)
@@ -222,7 +222,7 @@ WorkLayout work_layout(const swift_model_desc* d)
     k.score_out = c.take(1024 * 4);
     // tensor-core path (bf16 models): hi/lo bf16 planes of the GEMM inputs, stream-K slabs, tile counters
     k.slab_floats = 0;
-    k.xn_hl = k.xa_hl = k.act_hl = k.slabs = k.counters = 0;
+    k.xn_hl = k.xa_hl = k.act_hl = k.slabs = k.counters = k.sumsq = 0;
     if (d->dtype == SWIFT_BF16) {
         auto slab_need = [&](int N, int K) { k.slab_floats = std::max(k.slab_floats, (size_t)max_segments(N, K) * ROWS * (size_t)N); };
         slab_need((int)(qd + 2 * kd), (int)dm); slab_need((int)dm, (int)qd); slab_need(2 * d->ffn, (int)dm);
@@ -232,6 +232,7 @@ WorkLayout work_layout(const swift_model_desc* d)
         k.act_hl = c.take(2 * ROWS * (size_t)d->ffn * 2);
         k.slabs = c.take(k.slab_floats * 4);
         k.counters = c.take(TC_MAX_TILES * 4);
+        k.sumsq = c.take((size_t)std::max(1, ceil_div((int)dm, TC_TILE_N)) * ROWS * 4);
     }
     k.total = c.off;
     return k;
@@ -295,11 +296,12 @@ struct GemmSite {
     const CUtensorMap* mapX;
 };
 
-swift_status launch_gemm_tc(swift_ctx* ctx, const GemmSite& g)
+template <int EPI, typename TKV>
+swift_status launch_gemm_tc(swift_ctx* ctx, const GemmSite& g, const EpiParams& ep)
 {
     if (ceil_div(g.N, TC_TILE_N) > TC_MAX_TILES) return fail(ctx, SWIFT_EUNSUPPORTED, "GEMM with %d output tiles", ceil_div(g.N, TC_TILE_N));
-    CU(launch_k(gemm_tc_kernel, dim3(TC_GRID), dim3(TC_THREADS), (size_t)TC_SMEM_BYTES, ctx, state_of(ctx), *g.mapW, *g.mapX,
-                kptr<float>(ctx, ctx->kl.part), kptr<float>(ctx, ctx->kl.slabs), kptr<int>(ctx, ctx->kl.counters), g.N, g.K));
+    CU(launch_k(gemm_tc_kernel<EPI, TKV>, dim3(TC_GRID), dim3(TC_THREADS), (size_t)TC_SMEM_BYTES, ctx, state_of(ctx), *g.mapW, *g.mapX,
+                kptr<float>(ctx, ctx->kl.part), kptr<float>(ctx, ctx->kl.slabs), kptr<int>(ctx, ctx->kl.counters), g.N, g.K, ep));
     return SWIFT_OK;
 }
 
@@ -309,7 +311,9 @@ swift_status run_gemm(swift_ctx* ctx, int mr, const GemmSite& g, int* n_split)
 {
     if (ctx->use_tc) {
         *n_split = 1;
-        return launch_gemm_tc(ctx, g);
+        EpiParams ep;
+        memset(&ep, 0, sizeof ep);
+        return launch_gemm_tc<EPI_PLAIN, float>(ctx, g, ep);
     }
     GemmPlan p;
     swift_status s = launch_gemm<T>(ctx, mr, g.X, g.K, reinterpret_cast<const T*>(g.W), g.N, g.K, &p);
@@ -415,9 +419,85 @@ swift_status forward_chunk(swift_ctx* ctx, int rows, const int* toks_dev, const 
     return SWIFT_OK;
 }
 
+// The same walk on the tensor-core path, with the element-wise steps folded into the GEMM epilogues:
+// per block  QKV GEMM (+RMSNorm scale, RoPE, KV append) -> attention split -> combine -> o_proj GEMM
+// (+residual, next norm's planes) -> gate/up GEMM (+RMSNorm scale, SwiGLU) -> down GEMM (+residual ...).
+template <typename TKV>
+swift_status forward_chunk_fused(swift_ctx* ctx, int rows, const int* toks_dev, const uint8_t* skip, const int* page_table,
+                                 HeadOpts head)
+{
+    typedef __nv_bfloat16 T;
+    const swift_model_desc& d = ctx->d;
+    DevState* st = state_of(ctx);
+    const int mr = mr_of(rows);
+    const int dm = d.d_model, qd = d.n_heads * d.head_dim, kd = d.n_kv_heads * d.head_dim, nqkv = qd + 2 * kd;
+    float* h = kptr<float>(ctx, ctx->kl.h);
+    float* xa = kptr<float>(ctx, ctx->kl.xa);
+    __nv_bfloat16* xn_hl = kptr<__nv_bfloat16>(ctx, ctx->kl.xn_hl);
+    __nv_bfloat16* xa_hl = kptr<__nv_bfloat16>(ctx, ctx->kl.xa_hl);
+    __nv_bfloat16* act_hl = kptr<__nv_bfloat16>(ctx, ctx->kl.act_hl);
+    float* sumsq = kptr<float>(ctx, ctx->kl.sumsq);
+
+    std::vector<int> kept;                       // sub-layers that run, in walk order
+    for (int sl = 0; sl < 2 * d.n_blocks; ++sl)
+        if (!(skip && skip[sl])) kept.push_back(sl);
+    auto gain_of = [&](size_t k) -> const float* {   // gain of the RMSNorm in front of kept[k]; past the end: the final norm
+        if (k < kept.size()) return wptr<float>(ctx, (kept[k] & 1) ? ctx->wl.mlp_norm[kept[k] >> 1] : ctx->wl.attn_norm[kept[k] >> 1]);
+        return head.run ? wptr<float>(ctx, ctx->wl.final_norm) : nullptr;
+    };
+    EpiParams base;
+    memset(&base, 0, sizeof base);
+    base.inv_d = 1.0f / (float)dm;
+    base.eps = d.rms_eps;
+    base.sumsq_in = sumsq;
+    int n_tiles_in = 1;                          // the embedding gather writes one "tile" of sums
+
+    CU(launch_k(embed_fused_kernel<T>, dim3(rows), dim3(256), 0, ctx, st, toks_dev, (const T*)wptr<T>(ctx, ctx->wl.embed), h,
+                gain_of(0), xn_hl, sumsq, dm, d.vocab));
+    const int d_tiles = ceil_div(dm, TC_TILE_N);
+    for (size_t k = 0; k < kept.size(); ++k) {
+        const int b = kept[k] >> 1;
+        EpiParams resid = base;
+        resid.h = h; resid.gain_next = gain_of(k + 1); resid.planes_out = xn_hl; resid.sumsq_out = sumsq;
+        if (!(kept[k] & 1)) {
+            EpiParams ep = base;
+            ep.n_sumsq_tiles = n_tiles_in;
+            ep.q_out = kptr<float>(ctx, ctx->kl.q); ep.kv_pool = ctx->kvbase; ep.page_table = page_table; ep.L = ctx->kv;
+            ep.block = b; ep.n_heads = d.n_heads; ep.max_positions = d.max_positions; ep.rope_cs = kptr<float2>(ctx, ctx->kl.rope);
+            ST((launch_gemm_tc<EPI_QKV, TKV>(ctx, GemmSite{nullptr, nqkv, dm, nullptr, &ctx->tm_wqkv[b], &ctx->tm_xn}, ep)));
+            ST(launch_attn<TKV>(ctx, mr, page_table, b));
+            CU(launch_k(attn_combine_kernel, dim3(d.n_heads, rows), dim3(d.head_dim), 0, ctx, (const DevState*)st,
+                        (const float*)kptr<float>(ctx, ctx->kl.o_part), (const float2*)kptr<float2>(ctx, ctx->kl.ml_part),
+                        ctx->max_splits, d.n_heads, d.head_dim, xa, xa_hl));
+            ST((launch_gemm_tc<EPI_RESID, float>(ctx, GemmSite{nullptr, dm, qd, nullptr, &ctx->tm_wo[b], &ctx->tm_xa}, resid)));
+        } else {
+            EpiParams ep = base;
+            ep.n_sumsq_tiles = n_tiles_in;
+            ep.act_planes = act_hl; ep.ffn = d.ffn;
+            ST((launch_gemm_tc<EPI_SWIGLU, float>(ctx, GemmSite{nullptr, 2 * d.ffn, dm, nullptr, &ctx->tm_wgu[b], &ctx->tm_xn}, ep)));
+            ST((launch_gemm_tc<EPI_RESID, float>(ctx, GemmSite{nullptr, dm, d.ffn, nullptr, &ctx->tm_wdown[b], &ctx->tm_act}, resid)));
+        }
+        n_tiles_in = d_tiles;
+    }
+    if (head.run) {
+        EpiParams ep = base;
+        ep.n_sumsq_tiles = n_tiles_in;
+        ST((launch_gemm_tc<EPI_PLAIN, float>(ctx, GemmSite{nullptr, d.vocab, dm, nullptr, &ctx->tm_lm_head, &ctx->tm_xn}, ep)));
+        CU(launch_k(vocab_kernel, dim3(rows), dim3(VOCAB_THREADS), 0, ctx, st, (const float*)kptr<float>(ctx, ctx->kl.part), 1,
+                    (size_t)ROWS * d.vocab, kptr<float>(ctx, ctx->kl.logits), d.vocab, 1.0f / ctx->temperature, head.mode,
+                    ctx->mode == SWIFT_SAMPLING ? 1 : 0, kptr<float>(ctx, ctx->kl.q_rows)));
+    }
+    CU(cudaGetLastError());
+    return SWIFT_OK;
+}
+
 swift_status forward_chunk_any(swift_ctx* ctx, int rows, const int* toks_dev, const uint8_t* skip, const int* page_table,
                                HeadOpts head)
 {
+    if (ctx->use_tc && ctx->fuse) {
+        if (ctx->d.kv_dtype == SWIFT_BF16) return forward_chunk_fused<__nv_bfloat16>(ctx, rows, toks_dev, skip, page_table, head);
+        return forward_chunk_fused<float>(ctx, rows, toks_dev, skip, page_table, head);
+    }
     if (ctx->d.dtype == SWIFT_BF16) {
         if (ctx->d.kv_dtype == SWIFT_BF16) return forward_chunk<__nv_bfloat16, __nv_bfloat16>(ctx, rows, toks_dev, skip, page_table, head);
         return forward_chunk<__nv_bfloat16, float>(ctx, rows, toks_dev, skip, page_table, head);
@@ -430,7 +510,7 @@ swift_status forward_chunk_any(swift_ctx* ctx, int rows, const int* toks_dev, co
 // sequence is captured once into a CUDA graph and replayed: one graph launch instead of several
 // hundred kernel launches per forward.
 struct FwdKey {
-    int rows, head_run, head_mode, sampling, use_tc, use_pdl;
+    int rows, head_run, head_mode, sampling, use_tc, use_pdl, fuse;
     float temperature;
     const void* toks;
     const void* page_table;
@@ -438,7 +518,7 @@ struct FwdKey {
     bool operator==(const FwdKey& o) const
     {
         return rows == o.rows && head_run == o.head_run && head_mode == o.head_mode && sampling == o.sampling &&
-               use_tc == o.use_tc && use_pdl == o.use_pdl && temperature == o.temperature && toks == o.toks && page_table == o.page_table && mask == o.mask;
+               use_tc == o.use_tc && use_pdl == o.use_pdl && fuse == o.fuse && temperature == o.temperature && toks == o.toks && page_table == o.page_table && mask == o.mask;
     }
 };
 struct FwdGraph {
@@ -453,7 +533,7 @@ swift_status forward_cached(swift_ctx* ctx, int rows, const int* toks_dev, const
 {
     if (!ctx->use_graphs) return forward_chunk_any(ctx, rows, toks_dev, skip, page_table, head);
     const int L = 2 * ctx->d.n_blocks;
-    FwdKey key{rows, head.run ? 1 : 0, head.mode, ctx->mode, ctx->use_tc ? 1 : 0, ctx->use_pdl ? 1 : 0, ctx->temperature, toks_dev, page_table,
+    FwdKey key{rows, head.run ? 1 : 0, head.mode, ctx->mode, ctx->use_tc ? 1 : 0, ctx->use_pdl ? 1 : 0, ctx->fuse ? 1 : 0, ctx->temperature, toks_dev, page_table,
                skip ? std::vector<uint8_t>(skip, skip + L) : std::vector<uint8_t>()};
     auto& cache = *ctx->graphs;
     ctx->graph_clock++;
@@ -699,7 +779,11 @@ cudaError_t init_kernel_attrs()
 {
     cudaError_t e = set_attrs<float>();
     if (e == cudaSuccess) e = set_attrs<__nv_bfloat16>();
-    if (e == cudaSuccess) e = cudaFuncSetAttribute(gemm_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, TC_SMEM_BYTES);
+    if (e == cudaSuccess) e = cudaFuncSetAttribute(gemm_tc_kernel<EPI_PLAIN, float>, cudaFuncAttributeMaxDynamicSharedMemorySize, TC_SMEM_BYTES);
+    if (e == cudaSuccess) e = cudaFuncSetAttribute(gemm_tc_kernel<EPI_RESID, float>, cudaFuncAttributeMaxDynamicSharedMemorySize, TC_SMEM_BYTES);
+    if (e == cudaSuccess) e = cudaFuncSetAttribute(gemm_tc_kernel<EPI_SWIGLU, float>, cudaFuncAttributeMaxDynamicSharedMemorySize, TC_SMEM_BYTES);
+    if (e == cudaSuccess) e = cudaFuncSetAttribute(gemm_tc_kernel<EPI_QKV, float>, cudaFuncAttributeMaxDynamicSharedMemorySize, TC_SMEM_BYTES);
+    if (e == cudaSuccess) e = cudaFuncSetAttribute(gemm_tc_kernel<EPI_QKV, __nv_bfloat16>, cudaFuncAttributeMaxDynamicSharedMemorySize, TC_SMEM_BYTES);
     return e;
 }
 
@@ -808,6 +892,7 @@ swift_status swift_load(const swift_model_desc* desc, swift_devbuf weights, swif
     for (auto& e : c->ev) e = nullptr;
     c->use_graphs = getenv("SWIFT_NO_GRAPHS") == nullptr;
     c->use_pdl = getenv("SWIFT_NO_PDL") == nullptr;
+    c->fuse = getenv("SWIFT_NO_FUSE") == nullptr && desc->head_dim <= TC_TILE_N;
     c->graphs = new std::vector<FwdGraph>();
     c->graph_clock = 0;
     cudaError_t e = init_kernel_attrs();
