@@ -143,6 +143,8 @@ def main():
     ap.add_argument("--micro", action="store_true",
                     help="time each weight-streaming GEMM of the model alone on a few-block copy (profiling aid); prints one JSON line")
     ap.add_argument("--micro-iters", type=int, default=40)
+    ap.add_argument("--micro-forward", action="store_true",
+                    help="a few decode rounds on a 4-block copy of the model at the workload's context length (profiling aid)")
     args = ap.parse_args()
     rank = int(os.environ.get("RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
@@ -185,6 +187,19 @@ def main():
     torch.cuda.set_device(local)
     if args.micro:
         micro(cfg, run, args, hbm_peak)
+        return
+    if args.micro_forward:
+        small = cfg.with_blocks(4)
+        zz = synth.block_mask(small, synth.draft_blocks(small, 2))
+        model = SwiftModel(small, max_positions=run.prompt_len + 64, max_draft=run.max_draft, kv_dtype=args.kv_dtype)
+        model.load_weights(synth.iter_tensors(small))
+        prompt = synth.prompt(small, run.prompt_len)
+        outs = {}
+        for name, gp in (("vanilla", GenParams(max_new=4, vanilla=True)),
+                         ("swift", GenParams(max_new=2 * (run.max_draft + 1) + 1, max_draft=run.max_draft, skip_mask=zz))):
+            _, st, _ = model.generate(prompt, gp)
+            outs[name] = {"ms_decode": st.ms_decode, "tokens": st.tokens, "rounds": st.rounds, "launches": st.kernel_launches}
+        print(json.dumps({"micro_forward": small.name, "prompt": run.prompt_len, **outs}))
         return
     if world > 1:
         import torch.distributed as dist

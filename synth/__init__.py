@@ -116,6 +116,7 @@ RUNS: Dict[str, Tuple[str, RunConfig]] = {
     "c1": ("tiny", RunConfig(32, 64, 4, stop_conf=0.8, n_skip_blocks=4)),
     "c2": ("7b", RunConfig(512, 256, 8, n_skip_blocks=14)),
     "c3": ("13b", RunConfig(1024, 512, 8, n_skip_blocks=18, optimise=True)),
+    "c3-fixed": ("13b", RunConfig(1024, 512, 8, n_skip_blocks=18)),     # config 3's shape with the planted set held fixed
     "c4": ("13b", RunConfig(1024, 512, 8, n_skip_blocks=20, mode="sampling", rng_seed=4)),
     "c5": ("70b", RunConfig(2048, 512, 12, n_skip_blocks=36)),
 }
