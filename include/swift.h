@@ -213,6 +213,38 @@ swift_status swift_time_gemm(swift_ctx* ctx, int32_t which, int32_t n_rows, int3
 swift_status swift_read_kv(swift_ctx* ctx, int32_t block, int32_t which, int32_t pos0, int32_t count,
                            float* out_host);
 
+/*
+ * swift_gemm_static — the paper has no counterpart to this call; it exists for integration reasons only.
+ *
+ * y[r][n] = sum_k x[r][k] * w[n][k] for n_rows <= 16 rows, the same skinny weight-streaming product the
+ * decoder walk is made of, for callers that are not allowed to allocate device memory: plug-ins that
+ * run inside a host application which owns the allocator and hands them ready-made tensors, code that
+ * runs at a point where a cudaMalloc (an implicit device synchronisation, and a lock other threads may
+ * hold) is unacceptable.  The split-K partial sums and a small control block live in an array built into
+ * the library image (SWIFT_STATIC_SCRATCH_BYTES per GPU that loads the library, held until the process
+ * exits), so the call allocates nothing: no cudaMalloc, no cudaFree, no allocating library routine.
+ *
+ *  w_dev   device, row-major [N][K], SWIFT_F32 or SWIFT_BF16 (w_dtype), 16-byte aligned, K % 4 == 0
+ *          (fp32) or K % 8 == 0 (bf16)
+ *  x_dev   device, fp32 [n_rows][K], 16-byte aligned;   y_dev   device, fp32 [n_rows][N]
+ *  All three stay the caller's.  The work is enqueued on cuda_stream (a cudaStream_t; NULL = default
+ *  stream) and the call returns without synchronising.
+ *
+ * Limit: ceil(K / 512) * 16 * N * 4 + 1024 bytes must fit in SWIFT_STATIC_SCRATCH_BYTES, otherwise
+ * SWIFT_ECAPACITY is returned and nothing is enqueued.  swift_gemm_static_error() gives the text of the
+ * calling thread's last failure.
+ *
+ * The first call on each device looks the array's device address up (cudaGetSymbolAddress, with that
+ * device current); make that first call outside any stream capture.  All calls on a device share the one
+ * array and it keeps whatever the previous call left: each call re-initialises the control block and
+ * overwrites every partial sum it later reads, but two calls whose kernels overlap on the GPU (different
+ * streams, or concurrent host threads) race on it.  Serialise them.
+ */
+enum { SWIFT_STATIC_SCRATCH_BYTES = 8 * 1024 * 1024 };
+swift_status swift_gemm_static(const void* w_dev, int32_t w_dtype, int32_t N, int32_t K, const float* x_dev,
+                               int32_t n_rows, float* y_dev, void* cuda_stream);
+const char* swift_gemm_static_error(void);
+
 #ifdef __cplusplus
 }
 #endif

@@ -52,7 +52,8 @@ class _Stats(C.Structure):
 SYMBOLS = ("swift_weights_bytes", "swift_kv_bytes", "swift_workspace_bytes", "swift_load", "swift_free",
            "swift_last_error", "swift_pack_tensor", "swift_set_sampling", "swift_forward_rows", "swift_prefill",
            "swift_set_pending", "swift_draft", "swift_verify", "swift_accept", "swift_score_skipsets", "swift_generate",
-           "swift_committed_length", "swift_launch_count", "swift_forward_bytes", "swift_read_kv", "swift_time_gemm", "swift_set_gemm_impl", "swift_gemm")
+           "swift_committed_length", "swift_launch_count", "swift_forward_bytes", "swift_read_kv", "swift_time_gemm", "swift_set_gemm_impl", "swift_gemm", "swift_gemm_static",
+           "swift_gemm_static_error")
 
 _lib = None
 
@@ -88,6 +89,9 @@ def load_library(path: Optional[str] = None) -> C.CDLL:
     lib.swift_forward_bytes.argtypes = [vp, vp, i32, i32]
     lib.swift_forward_bytes.restype = C.c_double
     lib.swift_set_gemm_impl.argtypes = [vp, i32]
+    lib.swift_gemm_static.argtypes = [vp, i32, i32, i32, vp, i32, vp, vp]
+    lib.swift_gemm_static_error.argtypes = []
+    lib.swift_gemm_static_error.restype = C.c_char_p
     lib.swift_gemm.argtypes = [vp, i32, i32, vp, i32, vp]
     lib.swift_time_gemm.argtypes = [vp, i32, i32, i32, vp, vp]
     lib.swift_read_kv.argtypes = [vp, i32, i32, i32, i32, vp]
@@ -133,6 +137,27 @@ class GenStats:
     bytes_draft: float
     bytes_verify: float
     kernel_launches: int
+
+
+STATIC_SCRATCH_BYTES = 8 * 1024 * 1024
+
+
+def gemm_static(w: torch.Tensor, x: torch.Tensor, y: torch.Tensor, stream: Optional[torch.cuda.Stream] = None) -> None:
+    """y = x @ w.T through swift_gemm_static: w [N, K] fp32 or bf16, x [rows <= 16, K] fp32, y [rows, N] fp32, all
+    contiguous CUDA tensors the caller made beforehand.  The call itself allocates nothing (its scratch is an
+    array inside the library) and only enqueues work on `stream` (default: the current stream)."""
+    if not (w.is_cuda and x.is_cuda and y.is_cuda and w.is_contiguous() and x.is_contiguous() and y.is_contiguous()):
+        raise ValueError("w, x, y must be contiguous CUDA tensors")
+    if x.dtype != torch.float32 or y.dtype != torch.float32 or w.dtype not in (torch.float32, torch.bfloat16):
+        raise TypeError("x, y fp32; w fp32 or bf16")
+    if w.dim() != 2 or x.dim() != 2 or x.shape[1] != w.shape[1] or tuple(y.shape) != (x.shape[0], w.shape[0]):
+        raise ValueError("shape mismatch")
+    s = stream if stream is not None else torch.cuda.current_stream(w.device)
+    with torch.cuda.device(w.device):
+        st = lib().swift_gemm_static(C.c_void_p(w.data_ptr()), 1 if w.dtype == torch.bfloat16 else 0, w.shape[0], w.shape[1],
+                                     C.c_void_p(x.data_ptr()), x.shape[0], C.c_void_p(y.data_ptr()), C.c_void_p(s.cuda_stream))
+    if st != 0:
+        raise SwiftError(st, lib().swift_gemm_static_error().decode())
 
 
 def _i32(a) -> np.ndarray:
