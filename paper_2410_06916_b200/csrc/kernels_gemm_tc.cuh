@@ -188,7 +188,7 @@ __device__ __forceinline__ void tc_finalize(const EpiParams& ep, const DevState*
         for (int m = 0; m < ROWS; ++m) {
             sq[m] = 0.f;
             if (n < N && m < n_rows) {
-                const float hn = ep.h[(size_t)m * N + n] + val[m];
+                const float hn = __ldcg(ep.h + (size_t)m * N + n) + val[m];   // L2: another SM may have written it earlier in this kernel
                 ep.h[(size_t)m * N + n] = hn;
                 if (ep.gain_next) store_hi_lo(ep.planes_out, m, N, n, hn * ep.gain_next[n]);
                 sq[m] = hn * hn;
@@ -311,8 +311,8 @@ gemm_tc_kernel(DevState* st, const __grid_constant__ CUtensorMap mapW, const __g
                 for (int i = 0; i < n_pre; ++i) mbar_wait(full_bar(i), 0);
             } else {
             int it = n_pre;
-            for (long long u = u_begin + n_pre; u < u_end; ++u, ++it) {
-                const int tile = (int)(u / sk.KB), kb = (int)(u % sk.KB);
+            int tile = (int)((u_begin + n_pre) / sk.KB), kb = (int)((u_begin + n_pre) % sk.KB);
+            for (long long u = u_begin + n_pre; u < u_end; ++u, ++it, (++kb == sk.KB ? (kb = 0, ++tile) : 0)) {
                 const int s = it % TC_STAGES;
                 if (!mbar_wait(empty_bar(s), ((it / TC_STAGES) & 1) ^ 1)) { abort_sh = 1; break; }
                 const uint32_t a_dst = base + s * TC_STAGE_BYTES, b_dst = a_dst + TC_A_BYTES;
@@ -329,12 +329,11 @@ gemm_tc_kernel(DevState* st, const __grid_constant__ CUtensorMap mapW, const __g
         pdl_wait();
         if (lane == 0 && st->n_rows != 0) {
             int it = 0, seg = 0;
-            for (long long u = u_begin; u < u_end; ++u, ++it) {
-                const int tile = (int)(u / sk.KB), kb = (int)(u % sk.KB);
+            int kb = (int)(u_begin % sk.KB);
+            for (long long u = u_begin; u < u_end; ++u, ++it, (++kb == sk.KB ? (kb = 0) : 0)) {
                 const bool seg_first = (u == u_begin) || kb == 0;
                 const bool seg_last = (u + 1 == u_end) || kb == sk.KB - 1;
                 const int buf = seg & 1;
-                (void)tile;
                 if (seg_first) {   // the epilogue must have drained this accumulator buffer (two segments ago)
                     if (!mbar_wait(tempty_bar(buf), ((seg >> 1) & 1) ^ 1)) { abort_sh = 1; break; }
                     tc_fence_after();

@@ -452,6 +452,16 @@ swift_status forward_chunk_fused(swift_ctx* ctx, int rows, const int* toks_dev, 
     base.sumsq_in = sumsq;
     int n_tiles_in = 1;                          // the embedding gather writes one "tile" of sums
 
+    auto gemm = [&](int epi, const CUtensorMap* mw, const CUtensorMap* mx, int N, int K, const EpiParams& ep) -> swift_status {
+        const GemmSite g{nullptr, N, K, nullptr, mw, mx};
+        switch (epi) {
+        case EPI_QKV: return launch_gemm_tc<EPI_QKV, TKV>(ctx, g, ep);
+        case EPI_SWIGLU: return launch_gemm_tc<EPI_SWIGLU, float>(ctx, g, ep);
+        case EPI_RESID: return launch_gemm_tc<EPI_RESID, float>(ctx, g, ep);
+        default: return launch_gemm_tc<EPI_PLAIN, float>(ctx, g, ep);
+        }
+    };
+
     CU(launch_k(embed_fused_kernel<T>, dim3(rows), dim3(256), 0, ctx, st, toks_dev, (const T*)wptr<T>(ctx, ctx->wl.embed), h,
                 gain_of(0), xn_hl, sumsq, dm, d.vocab));
     const int d_tiles = ceil_div(dm, TC_TILE_N);
@@ -464,25 +474,25 @@ swift_status forward_chunk_fused(swift_ctx* ctx, int rows, const int* toks_dev, 
             ep.n_sumsq_tiles = n_tiles_in;
             ep.q_out = kptr<float>(ctx, ctx->kl.q); ep.kv_pool = ctx->kvbase; ep.page_table = page_table; ep.L = ctx->kv;
             ep.block = b; ep.n_heads = d.n_heads; ep.max_positions = d.max_positions; ep.rope_cs = kptr<float2>(ctx, ctx->kl.rope);
-            ST((launch_gemm_tc<EPI_QKV, TKV>(ctx, GemmSite{nullptr, nqkv, dm, nullptr, &ctx->tm_wqkv[b], &ctx->tm_xn}, ep)));
+            ST(gemm(EPI_QKV, &ctx->tm_wqkv[b], &ctx->tm_xn, nqkv, dm, ep));
             ST(launch_attn<TKV>(ctx, mr, page_table, b));
             CU(launch_k(attn_combine_kernel, dim3(d.n_heads, rows), dim3(d.head_dim), 0, ctx, (const DevState*)st,
                         (const float*)kptr<float>(ctx, ctx->kl.o_part), (const float2*)kptr<float2>(ctx, ctx->kl.ml_part),
                         ctx->max_splits, d.n_heads, d.head_dim, xa, xa_hl));
-            ST((launch_gemm_tc<EPI_RESID, float>(ctx, GemmSite{nullptr, dm, qd, nullptr, &ctx->tm_wo[b], &ctx->tm_xa}, resid)));
+            ST(gemm(EPI_RESID, &ctx->tm_wo[b], &ctx->tm_xa, dm, qd, resid));
         } else {
             EpiParams ep = base;
             ep.n_sumsq_tiles = n_tiles_in;
             ep.act_planes = act_hl; ep.ffn = d.ffn;
-            ST((launch_gemm_tc<EPI_SWIGLU, float>(ctx, GemmSite{nullptr, 2 * d.ffn, dm, nullptr, &ctx->tm_wgu[b], &ctx->tm_xn}, ep)));
-            ST((launch_gemm_tc<EPI_RESID, float>(ctx, GemmSite{nullptr, dm, d.ffn, nullptr, &ctx->tm_wdown[b], &ctx->tm_act}, resid)));
+            ST(gemm(EPI_SWIGLU, &ctx->tm_wgu[b], &ctx->tm_xn, 2 * d.ffn, dm, ep));
+            ST(gemm(EPI_RESID, &ctx->tm_wdown[b], &ctx->tm_act, dm, d.ffn, resid));
         }
         n_tiles_in = d_tiles;
     }
     if (head.run) {
         EpiParams ep = base;
         ep.n_sumsq_tiles = n_tiles_in;
-        ST((launch_gemm_tc<EPI_PLAIN, float>(ctx, GemmSite{nullptr, d.vocab, dm, nullptr, &ctx->tm_lm_head, &ctx->tm_xn}, ep)));
+        ST(gemm(EPI_PLAIN, &ctx->tm_lm_head, &ctx->tm_xn, d.vocab, dm, ep));
         CU(launch_k(vocab_kernel, dim3(rows), dim3(VOCAB_THREADS), 0, ctx, st, (const float*)kptr<float>(ctx, ctx->kl.part), 1,
                     (size_t)ROWS * d.vocab, kptr<float>(ctx, ctx->kl.logits), d.vocab, 1.0f / ctx->temperature, head.mode,
                     ctx->mode == SWIFT_SAMPLING ? 1 : 0, kptr<float>(ctx, ctx->kl.q_rows)));
@@ -891,7 +901,7 @@ swift_status swift_load(const swift_model_desc* desc, swift_devbuf weights, swif
     }
     for (auto& e : c->ev) e = nullptr;
     c->use_graphs = getenv("SWIFT_NO_GRAPHS") == nullptr;
-    c->use_pdl = getenv("SWIFT_NO_PDL") == nullptr;
+    c->use_pdl = getenv("SWIFT_PDL") != nullptr;   // programmatic dependent launch: measured neutral to slightly negative on whole forwards, so opt-in
     c->fuse = getenv("SWIFT_NO_FUSE") == nullptr && desc->head_dim <= TC_TILE_N;
     c->graphs = new std::vector<FwdGraph>();
     c->graph_clock = 0;
