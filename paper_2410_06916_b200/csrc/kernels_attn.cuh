@@ -150,12 +150,26 @@ attn_split_kernel(const DevState* st, const float* __restrict__ q, const T* __re
     }
     __syncthreads();
 
-    // phase 3: out[r][d] = sum_j p[r][j] * V[j][d]; one thread per d
+    // phase 3: out[r][d] = sum_j p[r][j] * V[j][d]; one thread per d, positions taken four at a time so that
+    // one 16-byte read of p feeds four multiply-adds (same summation order as one at a time)
+    const int len4 = len & ~3;
     for (int d = tid; d < dh; d += ATTN_THREADS) {
         float acc[MR];
 #pragma unroll
         for (int r = 0; r < MR; ++r) acc[r] = 0.f;
-        for (int j = 0; j < len; ++j) {
+        for (int j = 0; j < len4; j += 4) {
+            const float v0 = to_float(Vs[(size_t)j * dh + d]), v1 = to_float(Vs[(size_t)(j + 1) * dh + d]);
+            const float v2 = to_float(Vs[(size_t)(j + 2) * dh + d]), v3 = to_float(Vs[(size_t)(j + 3) * dh + d]);
+#pragma unroll
+            for (int r = 0; r < MR; ++r) {
+                const float4 p4 = *reinterpret_cast<const float4*>(ps + r * ATTN_CHUNK + j);
+                acc[r] = fmaf(p4.x, v0, acc[r]);
+                acc[r] = fmaf(p4.y, v1, acc[r]);
+                acc[r] = fmaf(p4.z, v2, acc[r]);
+                acc[r] = fmaf(p4.w, v3, acc[r]);
+            }
+        }
+        for (int j = len4; j < len; ++j) {
             const float v = to_float(Vs[(size_t)j * dh + d]);
 #pragma unroll
             for (int r = 0; r < MR; ++r) acc[r] = fmaf(ps[r * ATTN_CHUNK + j], v, acc[r]);

@@ -243,6 +243,7 @@ template <typename T> T* kptr(swift_ctx* c, size_t off) { return reinterpret_cas
 DevState* state_of(swift_ctx* c) { return kptr<DevState>(c, c->kl.state); }
 
 int mr_of(int rows) { return rows <= 1 ? 1 : rows <= 2 ? 2 : rows <= 4 ? 4 : rows <= 8 ? 8 : 16; }
+int attn_mr_of(int rows) { return rows > 8 && rows <= 12 ? 12 : mr_of(rows); }   // 9 rows = a verification of 8 drafts
 
 // ------------------------------------------------------------------------------ launches
 // Launch with programmatic stream serialisation (see pdl_enter in common.cuh).
@@ -342,6 +343,7 @@ swift_status launch_attn(swift_ctx* ctx, int mr, const int* page_table, int bloc
     case 2: return launch_attn_mr<T, 2>(ctx, page_table, block);
     case 4: return launch_attn_mr<T, 4>(ctx, page_table, block);
     case 8: return launch_attn_mr<T, 8>(ctx, page_table, block);
+    case 12: return launch_attn_mr<T, 12>(ctx, page_table, block);
     default: return launch_attn_mr<T, 16>(ctx, page_table, block);
     }
 }
@@ -365,7 +367,6 @@ swift_status forward_chunk(swift_ctx* ctx, int rows, const int* toks_dev, const 
 {
     const swift_model_desc& d = ctx->d;
     DevState* st = state_of(ctx);
-    cudaStream_t s = ctx->stream;
     const int mr = mr_of(rows);
     const int dm = d.d_model, qd = d.n_heads * d.head_dim, kd = d.n_kv_heads * d.head_dim, nqkv = qd + 2 * kd;
     float* h = kptr<float>(ctx, ctx->kl.h);
@@ -390,7 +391,7 @@ swift_status forward_chunk(swift_ctx* ctx, int rows, const int* toks_dev, const 
                         (const DevState*)st, (const float*)part, S, (size_t)ROWS * nqkv, nqkv, kptr<float>(ctx, ctx->kl.q),
                         reinterpret_cast<TKV*>(ctx->kvbase), page_table, ctx->kv, b, d.n_heads,
                         (const float2*)kptr<float2>(ctx, ctx->kl.rope), d.max_positions));
-            ST(launch_attn<TKV>(ctx, mr, page_table, b));
+            ST(launch_attn<TKV>(ctx, attn_mr_of(rows), page_table, b));
             CU(launch_k(attn_combine_kernel, dim3(d.n_heads, rows), dim3(d.head_dim), 0, ctx, (const DevState*)st,
                         (const float*)kptr<float>(ctx, ctx->kl.o_part), (const float2*)kptr<float2>(ctx, ctx->kl.ml_part),
                         ctx->max_splits, d.n_heads, d.head_dim, xa, xa_hl));
@@ -475,7 +476,7 @@ swift_status forward_chunk_fused(swift_ctx* ctx, int rows, const int* toks_dev, 
             ep.q_out = kptr<float>(ctx, ctx->kl.q); ep.kv_pool = ctx->kvbase; ep.page_table = page_table; ep.L = ctx->kv;
             ep.block = b; ep.n_heads = d.n_heads; ep.max_positions = d.max_positions; ep.rope_cs = kptr<float2>(ctx, ctx->kl.rope);
             ST(gemm(EPI_QKV, &ctx->tm_wqkv[b], &ctx->tm_xn, nqkv, dm, ep));
-            ST(launch_attn<TKV>(ctx, mr, page_table, b));
+            ST(launch_attn<TKV>(ctx, attn_mr_of(rows), page_table, b));
             CU(launch_k(attn_combine_kernel, dim3(d.n_heads, rows), dim3(d.head_dim), 0, ctx, (const DevState*)st,
                         (const float*)kptr<float>(ctx, ctx->kl.o_part), (const float2*)kptr<float2>(ctx, ctx->kl.ml_part),
                         ctx->max_splits, d.n_heads, d.head_dim, xa, xa_hl));
@@ -777,7 +778,9 @@ cudaError_t set_attrs_mr()
 template <typename T>
 cudaError_t set_attrs()
 {
-    cudaError_t e = set_attrs_mr<T, 1>();
+    cudaError_t e = cudaFuncSetAttribute(attn_split_kernel<T, 12>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                         (int)(2 * ATTN_CHUNK * 256 * sizeof(T) + (12 * 256 + 3 * 12 * ATTN_CHUNK) * 4));
+    if (e == cudaSuccess) e = set_attrs_mr<T, 1>();
     if (e == cudaSuccess) e = set_attrs_mr<T, 2>();
     if (e == cudaSuccess) e = set_attrs_mr<T, 4>();
     if (e == cudaSuccess) e = set_attrs_mr<T, 8>();
