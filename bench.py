@@ -86,6 +86,18 @@ class ClockSampler:
                 "samples": len(sm)}
 
 
+def aggregate_replicas(tokens: int, decode_ms: float, total_ms: float, wall_s: float, world: int, device=None):
+    """Whole-job numbers of N independent replicas: every rank decoded `tokens` tokens of its own sequence; the job
+    takes as long as its slowest rank (max over ranks), and its throughput is all ranks' tokens over that time.
+    Returns (decode tokens/s, max decode ms, max total ms, max wall s).  Uses the default process group when world > 1."""
+    if world > 1:
+        import torch.distributed as dist
+        t = torch.tensor([decode_ms, total_ms, wall_s], dtype=torch.float64, device=device)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        decode_ms, total_ms, wall_s = t.tolist()
+    return world * tokens / (decode_ms * 1e-3), decode_ms, total_ms, wall_s
+
+
 def workload(name: str):
     model_name, run = synth.RUNS[name]
     cfg = synth.MODELS[model_name]
@@ -243,12 +255,8 @@ def main():
     launches = model.launches - launches0
     dec_ms = sum(s.ms_decode for s in stats)
     tot_ms = sum(s.ms_decode + s.ms_prefill for s in stats)
-    if world > 1:
-        t = torch.tensor([dec_ms, tot_ms, wall], device="cuda", dtype=torch.float64)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        dec_ms, tot_ms, wall = t.tolist()
     tokens = sum(s.tokens - 1 for s in stats)            # the first token comes out of prefill
-    value = world * tokens / (dec_ms * 1e-3)
+    value, dec_ms, tot_ms, wall = aggregate_replicas(tokens, dec_ms, tot_ms, wall, world, device="cuda")
     e2e = world * sum(s.tokens for s in stats) / wall
 
     # vanilla decoding of the same model for the comparison the metric names
