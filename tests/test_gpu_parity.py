@@ -132,11 +132,11 @@ def test_weight_streaming_gemm_kernels(shape, rows):
         g.close()
 
 
-@pytest.mark.parametrize("shape,kv", [("7b", "f32"), ("13b", "f32"), ("13b", "bf16")])
+@pytest.mark.parametrize("shape,kv", [("7b", "f32"), ("13b", "f32"), ("13b", "bf16"), ("70b", "f32")])
 def test_full_width_bf16_forward(shape, kv):
-    """Two blocks at the real 7B / 13B widths and vocabulary, in the launch shapes the benchmark uses:
-    one row (drafting, vanilla) and nine rows (verification of 8 drafts), behind a prefix that spans an
-    attention split, full model and layer-skipped."""
+    """Two blocks at the real 7B / 13B / 70B (grouped-query, 8 query heads per KV head) widths and vocabulary, in
+    the launch shapes the benchmark uses: one row (drafting, vanilla) and nine rows (verification of 8 drafts),
+    behind a prefix that spans several attention chunks, full model and layer-skipped."""
     cfg = synth.MODELS[shape].with_blocks(2, n_planted=1)
     o, g = make_pair(cfg, max_positions=320, kv_dtype=kv)
     tol = LOGIT_TOL if kv == "f32" else 3 * LOGIT_TOL      # a bf16 cache costs accuracy: measured, not a parity claim
