@@ -280,9 +280,12 @@ def main():
     g_ms, g_bytes = model.time_gemm(2, run.max_draft + 1, 200)
     g1_ms, _ = model.time_gemm(2, 1, 200)
     achieved = g_bytes / (g_ms * 1e-3) * 1e-9
+    # DRAM bytes per launch of that kernel from the ncu capture summarised in profiles/gemm_tc_7b_gate_up_9rows.md
+    # (7B widths, 9 rows); other shapes have no capture of their own
+    traffic = 186.4e6 if (cfg.name == "7b" and run.max_draft == 8) else None
     roofline = {"bound": "hbm", "kernel": "skinny GEMM, fused gate/up projection, %d rows" % (run.max_draft + 1),
                 "achieved": achieved, "peak": hbm_peak, "peak_kind": f"{peak_kind} copy bandwidth (burst)", "unit": "GB/s",
-                "frac": achieved / hbm_peak, "traffic": None, "bytes_per_launch": g_bytes, "ms_per_launch": g_ms,
+                "frac": achieved / hbm_peak, "traffic": traffic, "bytes_per_launch": g_bytes, "ms_per_launch": g_ms,
                 "one_row_frac": g_bytes / (g1_ms * 1e-3) * 1e-9 / hbm_peak}
 
     out = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,

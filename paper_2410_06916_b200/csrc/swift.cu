@@ -563,6 +563,17 @@ swift_status forward_cached(swift_ctx* ctx, int rows, const int* toks_dev, const
     const cudaError_t ce = cudaStreamEndCapture(ctx->stream, &graph);
     if (fs != SWIFT_OK) { if (graph) cudaGraphDestroy(graph); return fs; }
     if (ce != cudaSuccess) return fail(ctx, SWIFT_ECUDA, "stream capture failed: %s", cudaGetErrorString(ce));
+    if (getenv("SWIFT_DEBUG_GRAPH")) {       // how many of the captured dependencies are programmatic (PDL) edges
+        size_t n_nodes = 0, n_edges = 0;
+        cudaGraphGetNodes(graph, nullptr, &n_nodes);
+        cudaGraphGetEdges_v2(graph, nullptr, nullptr, nullptr, &n_edges);
+        std::vector<cudaGraphNode_t> from(n_edges), to(n_edges);
+        std::vector<cudaGraphEdgeData> data(n_edges);
+        size_t n_prog = 0;
+        if (n_edges && cudaGraphGetEdges_v2(graph, from.data(), to.data(), data.data(), &n_edges) == cudaSuccess)
+            for (size_t i = 0; i < n_edges; ++i) n_prog += data[i].type == cudaGraphDependencyTypeProgrammatic ? 1 : 0;
+        fprintf(stderr, "[swift] captured forward: %zu nodes, %zu edges, %zu programmatic\n", n_nodes, n_edges, n_prog);
+    }
     cudaGraphExec_t exec = nullptr;
     const cudaError_t ie = cudaGraphInstantiate(&exec, graph, 0);
     cudaGraphDestroy(graph);
