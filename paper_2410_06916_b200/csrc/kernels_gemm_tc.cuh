@@ -99,6 +99,16 @@ __device__ __forceinline__ uint64_t tc_smem_desc(uint32_t addr)
 // Instruction descriptor: D fp32, A and B bf16, both K-major, N = 32, M = 128.
 constexpr uint32_t TC_IDESC = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(TC_COLS >> 3) << 17) | ((uint32_t)(TC_TILE_N >> 4) << 24);
 
+// Arrival on a counter that both publishes this CTA's earlier stores and, for the CTA that turns out to be
+// last, acquires everybody else's: one acq_rel atomic at GPU scope instead of fence + atomic + fence.
+// Stores of the CTA's other threads are covered through the CTA barrier that precedes it (cumulativity).
+__device__ __forceinline__ int atom_add_acq_rel_gpu(int* p, int v)
+{
+    int old;
+    asm volatile("atom.acq_rel.gpu.global.add.s32 %0, [%1], %2;" : "=r"(old) : "l"(p), "r"(v) : "memory");
+    return old;
+}
+
 // Static stream-K schedule shared by host and device: CTA g owns units [start(g), start(g+1)).
 struct StreamK {
     long long U;   // units = n_tiles * KB
@@ -281,6 +291,16 @@ gemm_tc_kernel(DevState* st, const __grid_constant__ CUtensorMap mapW, const __g
         abort_sh = 0;
         epi_abort_sh = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        // Weights depend on nothing: this thread (the TMA producer) requests the first ring-full right away,
+        // before the block-wide set-up barrier and before waiting for the preceding kernel, so that HBM is
+        // already streaming while TMEM is allocated and when the activations become valid.
+        asm volatile("prefetch.tensormap [%0];" ::"l"(&mapW) : "memory");
+        const int n_pre0 = (int)((u_end - u_begin) < TC_STAGES ? (u_end - u_begin) : TC_STAGES);
+        for (int i = 0; i < n_pre0; ++i) {
+            const long long u = u_begin + i;
+            mbar_expect_tx(full_bar(i), TC_STAGE_BYTES);
+            tma_load_2d(base + i * TC_STAGE_BYTES, &mapW, (int)(u % sk.KB) * TC_BK, (int)(u / sk.KB) * TC_TILE_N, full_bar(i));
+        }
     }
     if (warp == 1) {   // one warp allocates 64 TMEM columns: two accumulator buffers of 32
         asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&tmem_base_sh)), "r"(64));
@@ -294,16 +314,8 @@ gemm_tc_kernel(DevState* st, const __grid_constant__ CUtensorMap mapW, const __g
     if (warp == 0) {
         // ---------------------------------------------------------------- TMA producer
         if (lane == 0) {
-            asm volatile("prefetch.tensormap [%0];" ::"l"(&mapW) : "memory");
             asm volatile("prefetch.tensormap [%0];" ::"l"(&mapX) : "memory");
-            // Weights do not depend on the preceding kernel: the first ring-full is requested before
-            // waiting for it, so that HBM is already streaming when the activations become valid.
-            const int n_pre = (int)((u_end - u_begin) < TC_STAGES ? (u_end - u_begin) : TC_STAGES);
-            for (int i = 0; i < n_pre; ++i) {
-                const long long u = u_begin + i;
-                mbar_expect_tx(full_bar(i), TC_STAGE_BYTES);
-                tma_load_2d(base + i * TC_STAGE_BYTES, &mapW, (int)(u % sk.KB) * TC_BK, (int)(u / sk.KB) * TC_TILE_N, full_bar(i));
-            }
+            const int n_pre = (int)((u_end - u_begin) < TC_STAGES ? (u_end - u_begin) : TC_STAGES);   // weights already requested
             pdl_wait();
             for (int i = 0; i < n_pre; ++i)
                 tma_load_2d(base + i * TC_STAGE_BYTES + TC_A_BYTES, &mapX, (int)((u_begin + i) % sk.KB) * TC_BK, 0, full_bar(i));
@@ -407,12 +419,10 @@ gemm_tc_kernel(DevState* st, const __grid_constant__ CUtensorMap mapW, const __g
                 if (n < N)
                     for (int m = 0; m < ROWS; ++m)
                         if (m < n_rows) mine[(size_t)m * N + n] = val[m];
-                __threadfence();
                 asm volatile("bar.sync 1, 128;" ::: "memory");
-                if (etid == 0) last_flag_sh = (atomicAdd(&counters[tile], 1) == nseg - 1) ? 1 : 0;
+                if (etid == 0) last_flag_sh = (atom_add_acq_rel_gpu(&counters[tile], 1) == nseg - 1) ? 1 : 0;
                 asm volatile("bar.sync 1, 128;" ::: "memory");
                 if (last_flag_sh) {                             // last arrival: add the slabs in slab order
-                    __threadfence();
 #pragma unroll
                     for (int m = 0; m < ROWS; ++m) val[m] = 0.f;
                     if (n < N) {
