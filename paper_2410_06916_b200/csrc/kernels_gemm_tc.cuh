@@ -16,7 +16,7 @@
 // row count.
 //
 // Pipeline per CTA: warp 0 issues TMA loads (weights 128x64 + activations 32x64 per stage, 128-byte
-// swizzle) into an 8-stage shared-memory ring guarded by mbarriers; warp 1 issues tcgen05.mma from
+// swizzle) into a 9-stage shared-memory ring guarded by mbarriers; warp 1 issues tcgen05.mma from
 // shared memory into a double-buffered TMEM accumulator; warps 2-5 drain TMEM with tcgen05.ld, add
 // the hi/lo columns and store.  Every mbarrier wait is bounded; on expiry the kernel records an
 // error and winds down (TMEM is always released).
@@ -30,7 +30,7 @@ namespace swk {
 constexpr int TC_TILE_N = 128;      // weight rows per tile (MMA M)
 constexpr int TC_COLS = 32;         // operand rows of X: 16 hi + 16 lo (MMA N)
 constexpr int TC_BK = 64;           // k elements per stage: 128 bytes of bf16 = one swizzle row
-constexpr int TC_STAGES = 5;       // 100 KB of shared memory: two CTAs (successive GEMMs) fit on one SM
+constexpr int TC_STAGES = 9;        // 144 KB of weight tiles in flight per SM: HBM latency (~2 us) x 44 GB/s per SM needs ~90 KB
 constexpr int TC_THREADS = 192;
 constexpr int TC_A_BYTES = TC_TILE_N * TC_BK * 2;   // 16384
 constexpr int TC_B_BYTES = TC_COLS * TC_BK * 2;     // 4096
