@@ -167,8 +167,11 @@ struct EpiParams {
 template <int EPI, typename TKV>
 __device__ __forceinline__ void tc_finalize(const EpiParams& ep, const DevState* st, float (&val)[ROWS], int n_rows, int tile,
                                             int quarter, int lane, int etid, int N, float* Y, const float* rstd_sh,
-                                            float* stage_sh)
+                                            float* stage_sh, const float (&h_pre)[ROWS], float gain_pre,
+                                            const float2* rope_sh, const int* page_sh)
 {
+    // h_pre / gain_pre (EPI_RESID) and rope_sh / page_sh (EPI_QKV) were fetched while the accumulator was still
+    // being computed, so that nothing here waits for a round trip to L2 before it can store.
     const int l = quarter * 32 + lane;                 // row of the tile
     const int n = tile * TC_TILE_N + l;
     if (EPI != EPI_RESID) {
@@ -198,9 +201,9 @@ __device__ __forceinline__ void tc_finalize(const EpiParams& ep, const DevState*
         for (int m = 0; m < ROWS; ++m) {
             sq[m] = 0.f;
             if (n < N && m < n_rows) {
-                const float hn = __ldcg(ep.h + (size_t)m * N + n) + val[m];   // L2: another SM may have written it earlier in this kernel
+                const float hn = h_pre[m] + val[m];
                 ep.h[(size_t)m * N + n] = hn;
-                if (ep.gain_next) store_hi_lo(ep.planes_out, m, N, n, hn * ep.gain_next[n]);
+                if (ep.gain_next) store_hi_lo(ep.planes_out, m, N, n, hn * gain_pre);
                 sq[m] = hn * hn;
             }
         }
@@ -234,7 +237,7 @@ __device__ __forceinline__ void tc_finalize(const EpiParams& ep, const DevState*
                     const float a = val[m], b = stage_sh[m * TC_TILE_N + lp];
                     float out = a;
                     if (gh < ep.n_heads + ep.L.n_kv_heads) {      // q or k: rotate
-                        const float2 cs = ep.rope_cs[(size_t)pos * half + (i < half ? i : i - half)];
+                        const float2 cs = rope_sh[m * (TC_TILE_N / 2) + (i < half ? i : i - half)];
                         out = i < half ? a * cs.x - b * cs.y : a * cs.x + b * cs.y;
                     }
                     if (gh < ep.n_heads) {
@@ -243,8 +246,7 @@ __device__ __forceinline__ void tc_finalize(const EpiParams& ep, const DevState*
                         const int hk = gh - ep.n_heads;
                         const int kv = hk >= ep.L.n_kv_heads ? 1 : 0;
                         const int kh = kv ? hk - ep.L.n_kv_heads : hk;
-                        const int page = ep.page_table[pos >> ep.L.page_shift];
-                        store_val(pool + ep.L.offset(page, ep.block, kv, kh, pos & (ep.L.page_size - 1)) + i, out);
+                        store_val(pool + ep.L.offset(page_sh[m], ep.block, kv, kh, pos & (ep.L.page_size - 1)) + i, out);
                     }
                 }
             }
@@ -284,6 +286,8 @@ gemm_tc_kernel(DevState* st, const __grid_constant__ CUtensorMap mapW, const __g
     __shared__ int abort_sh, epi_abort_sh;
     __shared__ float rstd_sh[ROWS];
     __shared__ float stage_sh[EPI == EPI_QKV ? ROWS * TC_TILE_N : 4 * ROWS];
+    __shared__ float2 rope_sh[EPI == EPI_QKV ? ROWS * (TC_TILE_N / 2) : 1];   // (cos, sin) of the rows' positions
+    __shared__ int page_sh[ROWS];                                              // KV page of each row's position
 
     if (tid == 0) {
         for (int s = 0; s < TC_STAGES; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
@@ -379,12 +383,31 @@ gemm_tc_kernel(DevState* st, const __grid_constant__ CUtensorMap mapW, const __g
             }
             rstd_sh[etid] = r;
         }
+        if (EPI == EPI_QKV) {
+            const int half = ep.L.head_dim >> 1, pos0 = st->pos0;
+            for (int idx = etid; idx < ROWS * half; idx += 128) {
+                const int m = idx / half, j = idx - m * half, pos = pos0 + m;
+                if (m < n_rows && pos < ep.max_positions) rope_sh[m * (TC_TILE_N / 2) + j] = ep.rope_cs[(size_t)pos * half + j];
+            }
+            if (etid < ROWS) {
+                const int pos = pos0 + etid;
+                page_sh[etid] = (etid < n_rows && pos < ep.max_positions) ? ep.page_table[pos >> ep.L.page_shift] : 0;
+            }
+        }
         asm volatile("bar.sync 1, 128;" ::: "memory");
         while (u < u_end) {
             const int tile = (int)(u / sk.KB), kb0 = (int)(u % sk.KB);
             const long long tile_end = (long long)(tile + 1) * sk.KB;
             const long long seg_end = tile_end < u_end ? tile_end : u_end;
             const int buf = seg & 1;
+            float h_pre[ROWS];
+            float gain_pre = 0.f;
+            if (EPI == EPI_RESID) {                     // this tile's slice of the residual stream, requested early
+                const int n_pre = tile * TC_TILE_N + quarter * 32 + lane;
+#pragma unroll
+                for (int m = 0; m < ROWS; ++m) h_pre[m] = (n_pre < N && m < n_rows) ? __ldcg(ep.h + (size_t)m * N + n_pre) : 0.f;
+                if (ep.gain_next && n_pre < N) gain_pre = ep.gain_next[n_pre];
+            }
             if (!mbar_wait(tfull_bar(buf), (seg >> 1) & 1)) epi_abort_sh = 1;
             asm volatile("bar.sync 1, 128;" ::: "memory");     // all four warps agree before anyone leaves the loop
             if (epi_abort_sh) { abort_sh = 1; break; }
@@ -411,7 +434,7 @@ gemm_tc_kernel(DevState* st, const __grid_constant__ CUtensorMap mapW, const __g
 #pragma unroll
             for (int m = 0; m < ROWS; ++m) val[m] = __uint_as_float(v[m]) + __uint_as_float(v[16 + m]);
             if (whole) {
-                tc_finalize<EPI, TKV>(ep, st, val, n_rows, tile, quarter, lane, etid, N, Y, rstd_sh, stage_sh);
+                tc_finalize<EPI, TKV>(ep, st, val, n_rows, tile, quarter, lane, etid, N, Y, rstd_sh, stage_sh, h_pre, gain_pre, rope_sh, page_sh);
             } else {
                 const int g_first = sk.owner((long long)tile * sk.KB), g_last = sk.owner(tile_end - 1);
                 const int slab = blockIdx.x - g_first, nseg = g_last - g_first + 1;
@@ -432,7 +455,7 @@ gemm_tc_kernel(DevState* st, const __grid_constant__ CUtensorMap mapW, const __g
                                 if (m < n_rows) val[m] += __ldcg(slabs + ((size_t)j * ROWS + m) * N + n);
                         }
                     }
-                    tc_finalize<EPI, TKV>(ep, st, val, n_rows, tile, quarter, lane, etid, N, Y, rstd_sh, stage_sh);
+                    tc_finalize<EPI, TKV>(ep, st, val, n_rows, tile, quarter, lane, etid, N, Y, rstd_sh, stage_sh, h_pre, gain_pre, rope_sh, page_sh);
                     if (etid == 0) counters[tile] = 0;
                 }
                 asm volatile("bar.sync 1, 128;" ::: "memory");  // last_flag_sh is rewritten by the next segment
