@@ -295,16 +295,20 @@ gemm_tc_kernel(DevState* st, const __grid_constant__ CUtensorMap mapW, const __g
         abort_sh = 0;
         epi_abort_sh = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-        // Weights depend on nothing: this thread (the TMA producer) requests the first ring-full right away,
-        // before the block-wide set-up barrier and before waiting for the preceding kernel, so that HBM is
-        // already streaming while TMEM is allocated and when the activations become valid.
+        // This thread is the TMA producer.  It requests the first ring-full right away, before the block-wide
+        // set-up barrier: the weight tiles first (they depend on nothing, so they may even precede the wait for
+        // the preceding kernel), then, once that kernel's results are visible, the matching activation tiles.
         asm volatile("prefetch.tensormap [%0];" ::"l"(&mapW) : "memory");
+        asm volatile("prefetch.tensormap [%0];" ::"l"(&mapX) : "memory");
         const int n_pre0 = (int)((u_end - u_begin) < TC_STAGES ? (u_end - u_begin) : TC_STAGES);
         for (int i = 0; i < n_pre0; ++i) {
             const long long u = u_begin + i;
             mbar_expect_tx(full_bar(i), TC_STAGE_BYTES);
             tma_load_2d(base + i * TC_STAGE_BYTES, &mapW, (int)(u % sk.KB) * TC_BK, (int)(u / sk.KB) * TC_TILE_N, full_bar(i));
         }
+        pdl_wait();
+        for (int i = 0; i < n_pre0; ++i)
+            tma_load_2d(base + i * TC_STAGE_BYTES + TC_A_BYTES, &mapX, (int)((u_begin + i) % sk.KB) * TC_BK, 0, full_bar(i));
     }
     if (warp == 1) {   // one warp allocates 64 TMEM columns: two accumulator buffers of 32
         asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&tmem_base_sh)), "r"(64));
@@ -318,11 +322,7 @@ gemm_tc_kernel(DevState* st, const __grid_constant__ CUtensorMap mapW, const __g
     if (warp == 0) {
         // ---------------------------------------------------------------- TMA producer
         if (lane == 0) {
-            asm volatile("prefetch.tensormap [%0];" ::"l"(&mapX) : "memory");
-            const int n_pre = (int)((u_end - u_begin) < TC_STAGES ? (u_end - u_begin) : TC_STAGES);   // weights already requested
-            pdl_wait();
-            for (int i = 0; i < n_pre; ++i)
-                tma_load_2d(base + i * TC_STAGE_BYTES + TC_A_BYTES, &mapX, (int)((u_begin + i) % sk.KB) * TC_BK, 0, full_bar(i));
+            const int n_pre = (int)((u_end - u_begin) < TC_STAGES ? (u_end - u_begin) : TC_STAGES);   // already requested above
             if (st->n_rows == 0) {                      // nothing to compute: let the requested tiles land, then leave
                 for (int i = 0; i < n_pre; ++i) mbar_wait(full_bar(i), 0);
             } else {
