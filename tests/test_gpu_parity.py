@@ -343,3 +343,81 @@ def test_errors_are_statuses_not_crashes(small_cfg):
     g.verify(); g.accept()
     assert g.n >= 4
     g.close()
+
+
+# ------------------------------------------------------------------------------ edge cases
+@pytest.mark.parametrize("page_size", [8, 128])
+def test_page_sizes_and_ragged_windows(small_cfg, page_size):
+    """Pages smaller and larger than an attention chunk; a scoring window that starts in the middle of a page."""
+    o, g = make_pair(small_cfg, max_positions=256, page_size=page_size)
+    try:
+        prompt = synth.prompt(small_cfg, 70)
+        so.vanilla_generate(o, prompt, 30)
+        resync(g, o)
+        masks = np.array([[0] * 8, [1, 0, 0, 1, 0, 0, 1, 0], [1] * 8], dtype=np.uint8)
+        for gamma in (29, 7):
+            ref, _ = o.score_skipsets(masks.tolist(), gamma)
+            got = g.score_skipsets(masks, gamma)
+            assert got[0] == 1.0
+            for c in range(3):
+                if got[c] != pytest.approx(ref[c]):
+                    rows = o.forward_rows(o.tokens[o.n - gamma:o.n], o.n - gamma, masks[c].tolist(), write_kv=False)
+                    assert min(so.top2_margin(r) for r in rows) <= MARGIN
+        st = walk_rounds(o, g, [0, 1, 0, 0, 1, 0, 0, 0], n_rounds=5, max_k=6)
+        assert st["max_logit_err"] < 1e-4 and st["accept_cmp"] + st["accept_exempt"] == 5
+    finally:
+        g.close()
+
+
+def test_degenerate_lengths(tiny_pair):
+    """One-token prompt, a single generated token, an empty draft, and a run that ends inside a round."""
+    o, g = tiny_pair
+    from paper_2410_06916_b200 import GenParams
+    z = synth.block_mask(TINY, synth.planted_blocks(TINY))
+    for prompt, max_new, k in (([7], 1, 4), ([7], 2, 4), (synth.prompt(TINY, 3), 7, 15), (synth.prompt(TINY, 17), 5, 0)):
+        ref, margins = so.vanilla_generate(o, prompt, max_new)
+        out, st, _ = g.generate(prompt, GenParams(max_new=max_new, max_draft=k, skip_mask=z))
+        assert len(out) == max_new and compare_free_running(out, ref, margins) == max_new
+        van, _, _ = g.generate(prompt, GenParams(max_new=max_new, vanilla=True))
+        assert van == out
+    # an explicitly empty draft followed by verification is one vanilla step
+    o.prefill([5, 6, 7]); g.prefill([5, 6, 7])
+    toks, conf = g.draft(z, 0)
+    assert toks == [] and conf == []
+    am, logits = g.verify()
+    ref = o.forward_rows([o.tokens[-1]], o.n)
+    assert logit_err(logits[:1], ref) < 1e-4
+    a, nxt = g.accept()
+    assert a == 0 and nxt == so.argmax_lowest(ref[0])
+
+
+def test_sampling_with_temperature(tiny_pair):
+    """Temperature scales the target's and the draft's logits alike; confidence stays at temperature 1."""
+    o, g = tiny_pair
+    prompt = synth.prompt(TINY, 20)
+    seed, T = 77, 0.6
+    g.set_sampling(True, T, seed)
+    try:
+        o.prefill(prompt)
+        g.prefill(prompt); g.set_pending(o.tokens[-1])
+        z = list(synth.block_mask(TINY, synth.planted_blocks(TINY)))
+        st = walk_rounds(o, g, z, n_rounds=15, max_k=5, sampling=True, temperature=T, seed=seed)
+        assert st["accept_cmp"] >= 12 and st["max_logit_err"] < 1e-4, st
+    finally:
+        g.set_sampling(False)
+
+
+def test_cache_fills_to_capacity(small_cfg):
+    """Generation that ends exactly at max_positions, and one token more is refused without side effects."""
+    from paper_2410_06916_b200 import GenParams, SwiftError
+    o, g = make_pair(small_cfg, max_positions=64, page_size=16, max_draft=4)
+    try:
+        prompt = synth.prompt(small_cfg, 40)
+        z = np.array([0, 1, 0, 0, 0, 0, 1, 0], dtype=np.uint8)
+        ref, margins = so.vanilla_generate(o, prompt, 23)
+        out, _, _ = g.generate(prompt, GenParams(max_new=23, max_draft=4, skip_mask=z))       # 40 + 23 + 1 = 64
+        assert compare_free_running(out, ref, margins) == 23
+        with pytest.raises(SwiftError, match="ECAPACITY"):
+            g.generate(prompt, GenParams(max_new=24, max_draft=4, skip_mask=z))
+    finally:
+        g.close()
