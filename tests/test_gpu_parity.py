@@ -421,3 +421,32 @@ def test_cache_fills_to_capacity(small_cfg):
             g.generate(prompt, GenParams(max_new=24, max_draft=4, skip_mask=z))
     finally:
         g.close()
+
+
+@pytest.mark.slow
+def test_full_depth_7b_against_oracle_and_losslessness():
+    """Config 2 at full size (32 blocks, 13 GB of weights), in the launch configuration the benchmark times:
+    teacher-forced logits of the last prompt rows against the oracle, then SWIFT == vanilla on the GPU."""
+    import psutil
+    if psutil.virtual_memory().available < 64 * 2 ** 30:
+        pytest.skip("needs 64 GB of host memory for the oracle's fp32 copy of the weights")
+    from paper_2410_06916_b200 import GenParams
+    cfg = synth.MODELS["7b"]
+    o, g = make_pair(cfg, max_positions=256, max_draft=8)
+    try:
+        prompt = synth.prompt(cfg, 48)
+        ref = o.forward_rows(prompt, 0)
+        g.prefill(prompt[:1])
+        got, am = g.forward_rows(prompt, 0)
+        err = logit_err(got[-8:], ref[-8:])
+        print(f"7B full depth: teacher-forced logits off by {err:.2e} sigma")
+        assert err < LOGIT_TOL
+        for i in range(40, 48):
+            if so.top2_margin(ref[i]) > MARGIN:
+                assert int(am[i]) == so.argmax_lowest(ref[i])
+        z = synth.block_mask(cfg, synth.draft_blocks(cfg, 14))
+        van, _, _ = g.generate(prompt, GenParams(max_new=48, vanilla=True))
+        out, st, _ = g.generate(prompt, GenParams(max_new=48, max_draft=8, skip_mask=z))
+        assert out == van and st.accepted > 0
+    finally:
+        g.close()
