@@ -181,6 +181,231 @@ attn_split_kernel(const DevState* st, const float* __restrict__ q, const T* __re
     if (tid < n_rows) ml_part[((size_t)h * max_splits + s) * ROWS + tid] = make_float2(row_m[tid], row_l[tid]);
 }
 
+// ---------------------------------------------------------------------------------------------
+// Streaming form for head_dim == 128: no shared-memory staging of K and V; every byte of the cache is
+// loaded once, straight into registers, by coalesced warp loads with many rows in flight per warp.
+// grid = (H, max_splits), block = 128.  Warp w owns positions [16w, 16w + 16) of the chunk and takes
+// them in two batches of eight.  Within a batch, with lane = 8 * pg + dl:
+//   K : lane holds elements {32c + 4dl .. +3, c = 0..3} of rows pg and pg + 4 (eight lanes per row),
+//       so a score is a 16-term chain per lane followed by a three-level xor tree over dl.  The tree is
+//       "packed": while a lane holds an even number of sums it keeps one half and hands the other to
+//       its partner, which yields the same additions as the full butterfly at a fraction of the
+//       shuffles and leaves every (row, position) score in one owner lane (times replication);
+//   softmax: the owner lanes do the running max / exponentials / sums, trees over the position lanes;
+//   V : lane holds elements [4 lane, 4 lane + 4) of all eight rows; probabilities and rescale factors
+//       reach all lanes through a small per-warp shared array.
+// Finally the four warps' partial results are merged in warp order.  A query row's arithmetic does not
+// depend on MR or on how many other rows are present: masked positions enter with probability exactly
+// 0 and a rescale factor of exactly 1 where nothing is visible yet.
+// Same outputs as attn_split_kernel: o_part[h][s][r][dh] (unnormalised) and ml_part[h][s][r].
+constexpr int ATTN_BATCH = 8;
+
+template <typename T>
+__device__ __forceinline__ float4 load_row4(const T* p);
+template <>
+__device__ __forceinline__ float4 load_row4<float>(const float* p)
+{
+    return __ldg(reinterpret_cast<const float4*>(p));
+}
+template <>
+__device__ __forceinline__ float4 load_row4<__nv_bfloat16>(const __nv_bfloat16* p)
+{
+    const uint2 u = __ldg(reinterpret_cast<const uint2*>(p));
+    float4 f;
+    f.x = __uint_as_float(u.x << 16);
+    f.y = __uint_as_float(u.x & 0xFFFF0000u);
+    f.z = __uint_as_float(u.y << 16);
+    f.w = __uint_as_float(u.y & 0xFFFF0000u);
+    return f;
+}
+
+// One level of the xor tree over N per-lane sums.  Even N: the lane with `upper` clear keeps sums
+// [0, N/2) and adds the partner's copies of them, the other lane keeps [N/2, N); N/2 sums remain, in
+// v[0 .. N/2).  Odd N: plain butterfly, N sums remain.
+template <int N>
+__device__ __forceinline__ void fold_level(float* v, int off, bool upper)
+{
+    if constexpr (N % 2 == 0) {
+        constexpr int H = N / 2;
+#pragma unroll
+        for (int i = 0; i < H; ++i) {
+            const float keep = upper ? v[i + H] : v[i];
+            const float send = upper ? v[i] : v[i + H];
+            v[i] = keep + __shfl_xor_sync(0xffffffffu, send, off);
+        }
+    } else {
+#pragma unroll
+        for (int i = 0; i < N; ++i) v[i] += __shfl_xor_sync(0xffffffffu, v[i], off);
+    }
+}
+__host__ __device__ constexpr int folded(int n) { return n % 2 == 0 ? n / 2 : n; }
+
+template <typename T, int MR>
+__global__ void __launch_bounds__(ATTN_THREADS, MR == 1 ? 5 : (MR <= 12 ? 3 : 2))
+attn_stream_kernel(const DevState* st, const float* __restrict__ q, const T* __restrict__ kv_pool,
+                   const int* __restrict__ page_table, KvLayout L, int block, int n_heads, int max_splits,
+                   float scale, float* __restrict__ o_part, float2* __restrict__ ml_part)
+{
+    pdl_enter();
+    constexpr int DH = 128, NW = ATTN_THREADS / 32, PER_WARP = ATTN_CHUNK / NW;
+    static_assert(PER_WARP == 2 * ATTN_BATCH, "two batches per warp");
+    constexpr int N1 = MR, N2 = folded(N1), N3 = folded(N2);       // sums per lane after each tree level
+    const int n_rows = min(st->n_rows, MR);
+    if (n_rows == 0) return;
+    const int pos0 = st->pos0;
+    const int total = pos0 + n_rows;
+    const int h = blockIdx.x, s = blockIdx.y;
+    const int c0 = s * ATTN_CHUNK;
+    if (c0 >= total) return;
+    const int len = min(ATTN_CHUNK, total - c0);
+    const int kvh = h / (n_heads / L.n_kv_heads);
+    const int tid = threadIdx.x, lane = tid & 31, w = tid >> 5;
+    const int pg = lane >> 3, dl = lane & 7;
+    const bool b2 = (lane >> 2) & 1, b1 = (lane >> 1) & 1, b0 = lane & 1;
+    // what this lane owns after the tree: position pi of the batch and rows [row_base, row_base + N3)
+    const int pi = pg + (b2 ? 4 : 0);
+    int row_base = 0;
+    if (N1 % 2 == 0) row_base += b1 ? N2 : 0;
+    if (N2 % 2 == 0) row_base += b0 ? N3 : 0;
+
+    __shared__ float4 q_sh[MR][32];
+    __shared__ __align__(16) float part_acc[NW][MR][DH];
+    __shared__ float2 part_ml[NW][MR];
+    __shared__ __align__(16) float p_sh[NW][MR][ATTN_BATCH];
+    __shared__ float corr_sh[NW][MR];
+
+    for (int i = tid; i < MR * 32; i += ATTN_THREADS) {
+        const int r = i >> 5, c = i & 31;
+        float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
+        if (r < n_rows) {
+            v = *reinterpret_cast<const float4*>(q + ((size_t)r * n_heads + h) * DH + c * 4);
+            v.x *= scale; v.y *= scale; v.z *= scale; v.w *= scale;
+        }
+        q_sh[r][c] = v;
+    }
+    __syncthreads();
+
+    float m_own[N3], l_own[N3];
+#pragma unroll
+    for (int t = 0; t < N3; ++t) { m_own[t] = -INFINITY; l_own[t] = 0.f; }
+    float4 acc[MR];
+#pragma unroll
+    for (int r = 0; r < MR; ++r) acc[r] = make_float4(0.f, 0.f, 0.f, 0.f);
+    const size_t v_off = (size_t)L.n_kv_heads * L.page_size * DH;      // from a K row to the V row of the same slot
+
+#pragma unroll 1
+    for (int b = 0; b < 2; ++b) {
+        const int j0 = w * PER_WARP + b * ATTN_BATCH;
+        if (j0 >= len) break;
+        // rows past the end re-read the last one (finite values); they are masked below
+        float4 kx[2][4], vx[ATTN_BATCH];
+#pragma unroll
+        for (int sl = 0; sl < 2; ++sl) {
+            const int pos = c0 + min(j0 + pg + 4 * sl, len - 1);
+            const int page = __ldg(page_table + (pos >> L.page_shift));
+            const T* kp = kv_pool + L.offset(page, block, 0, kvh, pos & (L.page_size - 1)) + dl * 4;
+#pragma unroll
+            for (int c = 0; c < 4; ++c) kx[sl][c] = load_row4<T>(kp + 32 * c);
+        }
+#pragma unroll
+        for (int i = 0; i < ATTN_BATCH; ++i) {
+            const int pos = c0 + min(j0 + i, len - 1);
+            const int page = __ldg(page_table + (pos >> L.page_shift));
+            vx[i] = load_row4<T>(kv_pool + L.offset(page, block, 0, kvh, pos & (L.page_size - 1)) + v_off + lane * 4);
+        }
+
+        // partial scores: sc[sl * MR + r] over this lane's 16 elements
+        float sc[2 * MR];
+#pragma unroll
+        for (int r = 0; r < MR; ++r) {
+            float s0 = 0.f, s1 = 0.f;
+            if (r < n_rows) {
+#pragma unroll
+                for (int c = 0; c < 4; ++c) {
+                    const float4 q4 = q_sh[r][8 * c + dl];
+                    s0 = fmaf(kx[0][c].x, q4.x, s0); s0 = fmaf(kx[0][c].y, q4.y, s0);
+                    s0 = fmaf(kx[0][c].z, q4.z, s0); s0 = fmaf(kx[0][c].w, q4.w, s0);
+                    s1 = fmaf(kx[1][c].x, q4.x, s1); s1 = fmaf(kx[1][c].y, q4.y, s1);
+                    s1 = fmaf(kx[1][c].z, q4.z, s1); s1 = fmaf(kx[1][c].w, q4.w, s1);
+                }
+            }
+            sc[r] = s0; sc[MR + r] = s1;
+        }
+        fold_level<2 * MR>(sc, 4, b2);          // -> N1 = MR sums: all rows, position pi
+        fold_level<N1>(sc, 2, b1);              // -> N2
+        fold_level<N2>(sc, 1, b0);              // -> N3 sums: rows row_base .., position pi
+
+        __syncwarp();                           // previous batch's readers of p_sh are done
+#pragma unroll
+        for (int t = 0; t < N3; ++t) {
+            const int r = row_base + t;
+            float x = sc[t];
+            if (c0 + j0 + pi > pos0 + r) x = -INFINITY;                // causal mask; also covers positions past the end
+            float bm = x;
+            bm = fmaxf(bm, __shfl_xor_sync(0xffffffffu, bm, 4));
+            bm = fmaxf(bm, __shfl_xor_sync(0xffffffffu, bm, 8));
+            bm = fmaxf(bm, __shfl_xor_sync(0xffffffffu, bm, 16));
+            const float mn = fmaxf(m_own[t], bm);
+            float corr = 1.f, p = 0.f;
+            if (mn != -INFINITY) {
+                corr = (m_own[t] == -INFINITY) ? 0.f : expf(m_own[t] - mn);
+                p = (x == -INFINITY) ? 0.f : expf(x - mn);
+            }
+            float ps = p;
+            ps += __shfl_xor_sync(0xffffffffu, ps, 4);
+            ps += __shfl_xor_sync(0xffffffffu, ps, 8);
+            ps += __shfl_xor_sync(0xffffffffu, ps, 16);
+            l_own[t] = fmaf(l_own[t], corr, ps);
+            m_own[t] = mn;
+            p_sh[w][r][pi] = p;
+            if (pi == 0) corr_sh[w][r] = corr;
+        }
+        __syncwarp();
+
+#pragma unroll
+        for (int r = 0; r < MR; ++r) {
+            if (r < n_rows) {
+                const float corr = corr_sh[w][r];
+                const float4 pa = *reinterpret_cast<const float4*>(&p_sh[w][r][0]);
+                const float4 pb = *reinterpret_cast<const float4*>(&p_sh[w][r][4]);
+                const float pp[ATTN_BATCH] = {pa.x, pa.y, pa.z, pa.w, pb.x, pb.y, pb.z, pb.w};
+                float4 a = acc[r];
+                a.x *= corr; a.y *= corr; a.z *= corr; a.w *= corr;
+#pragma unroll
+                for (int i = 0; i < ATTN_BATCH; ++i) {
+                    a.x = fmaf(pp[i], vx[i].x, a.x); a.y = fmaf(pp[i], vx[i].y, a.y);
+                    a.z = fmaf(pp[i], vx[i].z, a.z); a.w = fmaf(pp[i], vx[i].w, a.w);
+                }
+                acc[r] = a;
+            }
+        }
+    }
+
+#pragma unroll
+    for (int r = 0; r < MR; ++r)
+        if (r < n_rows) *reinterpret_cast<float4*>(&part_acc[w][r][lane * 4]) = acc[r];
+    if (pi == 0) {
+#pragma unroll
+        for (int t = 0; t < N3; ++t) part_ml[w][row_base + t] = make_float2(m_own[t], l_own[t]);
+    }
+    __syncthreads();
+    for (int r = 0; r < n_rows; ++r) {                      // thread d merges the four warps in warp order
+        float M = -INFINITY;
+#pragma unroll
+        for (int ww = 0; ww < NW; ++ww) M = fmaxf(M, part_ml[ww][r].x);
+        float num = 0.f, den = 0.f;
+#pragma unroll
+        for (int ww = 0; ww < NW; ++ww) {
+            const float2 ml = part_ml[ww][r];
+            const float wt = (ml.x == -INFINITY) ? 0.f : expf(ml.x - M);
+            num = fmaf(wt, part_acc[ww][r][tid], num);
+            den = fmaf(wt, ml.y, den);
+        }
+        o_part[(((size_t)h * max_splits + s) * ROWS + r) * DH + tid] = num;
+        if (tid == 0) ml_part[((size_t)h * max_splits + s) * ROWS + r] = make_float2(M, den);
+    }
+}
+
 // grid = (H, rows), block = dh threads.  Combines the splits in chunk order.
 __global__ void attn_combine_kernel(const DevState* st, const float* __restrict__ o_part,
                                     const float2* __restrict__ ml_part, int max_splits, int n_heads, int dh,

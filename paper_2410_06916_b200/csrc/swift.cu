@@ -328,6 +328,13 @@ swift_status launch_attn_mr(swift_ctx* ctx, const int* page_table, int block)
     const swift_model_desc& d = ctx->d;
     const size_t smem = 2 * (size_t)ATTN_CHUNK * d.head_dim * sizeof(T) + ((size_t)MR * d.head_dim + 3 * (size_t)MR * ATTN_CHUNK) * sizeof(float);
     dim3 grid(d.n_heads, ctx->max_splits);
+    if (d.head_dim == 128) {
+        CU(launch_k(attn_stream_kernel<T, MR>, grid, dim3(ATTN_THREADS), 0, ctx, (const DevState*)state_of(ctx),
+                    (const float*)kptr<float>(ctx, ctx->kl.q), reinterpret_cast<const T*>(ctx->kvbase), page_table, ctx->kv,
+                    block, d.n_heads, ctx->max_splits, 1.0f / sqrtf((float)d.head_dim), kptr<float>(ctx, ctx->kl.o_part),
+                    kptr<float2>(ctx, ctx->kl.ml_part)));
+        return SWIFT_OK;
+    }
     CU(launch_k(attn_split_kernel<T, MR>, grid, dim3(ATTN_THREADS), smem, ctx, (const DevState*)state_of(ctx),
                 (const float*)kptr<float>(ctx, ctx->kl.q), reinterpret_cast<const T*>(ctx->kvbase), page_table, ctx->kv, block,
                 d.n_heads, ctx->max_splits, 1.0f / sqrtf((float)d.head_dim), kptr<float>(ctx, ctx->kl.o_part),
