@@ -51,7 +51,7 @@ typedef struct {
     int32_t n_blocks, d_model, n_heads, n_kv_heads, head_dim, ffn, vocab;
     int32_t dtype;          /* SWIFT_F32 or SWIFT_BF16: storage of the weights (activations are always fp32) */
     float rope_theta, rms_eps;
-    int32_t max_positions;  /* KV capacity in positions; multiple of page_size */
+    int32_t max_positions;  /* KV capacity in positions; multiple of page_size, at most 262144 */
     int32_t page_size;      /* positions per KV page; power of two, 8..128 */
     int32_t max_draft;      /* largest k any call will use; <= SWIFT_MAX_ROWS - 1 */
     int32_t kv_dtype;       /* SWIFT_F32 or SWIFT_BF16: storage of cached K,V (fp32 models: SWIFT_F32) */

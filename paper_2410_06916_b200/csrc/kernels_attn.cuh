@@ -406,7 +406,10 @@ attn_stream_kernel(const DevState* st, const float* __restrict__ q, const T* __r
     }
 }
 
-// grid = (H, rows), block = dh threads.  Combines the splits in chunk order.
+// grid = (H, rows), block = dh threads, dynamic smem = 2 * max_splits floats.  Combines the splits in chunk
+// order.  The (m, l) pairs are fetched once per block, spread over the threads, and the partial outputs are
+// read eight splits at a time with independent loads, so the kernel costs a few trips to L2 rather than one
+// per split; the sums themselves still run over the splits in ascending order.
 __global__ void attn_combine_kernel(const DevState* st, const float* __restrict__ o_part,
                                     const float2* __restrict__ ml_part, int max_splits, int n_heads, int dh,
                                     float* __restrict__ out, __nv_bfloat16* __restrict__ planes)
@@ -417,14 +420,47 @@ __global__ void attn_combine_kernel(const DevState* st, const float* __restrict_
     const int h = blockIdx.x, d = threadIdx.x;
     const int total = st->pos0 + st->n_rows;
     const int n_splits = (total + ATTN_CHUNK - 1) / ATTN_CHUNK;
+    extern __shared__ float comb_sh[];
+    float* w_sh = comb_sh;                    // [n_splits] exp(m_s - M), 0 for empty splits
+    float* l_sh = comb_sh + max_splits;       // [n_splits]
+    __shared__ float wmax_sh[32];
+    const size_t base = (size_t)h * max_splits;
+
+    float mx = -INFINITY;
+    for (int s = d; s < n_splits; s += blockDim.x) {
+        const float2 ml = ml_part[(base + s) * ROWS + r];
+        w_sh[s] = ml.x;
+        l_sh[s] = ml.y;
+        mx = fmaxf(mx, ml.x);
+    }
+    mx = warp_max(mx);
+    if ((d & 31) == 0) wmax_sh[d >> 5] = mx;
+    __syncthreads();
     float M = -INFINITY;
-    for (int s = 0; s < n_splits; ++s) M = fmaxf(M, ml_part[((size_t)h * max_splits + s) * ROWS + r].x);
+    for (int wi = 0; wi < (int)(blockDim.x + 31) / 32; ++wi) M = fmaxf(M, wmax_sh[wi]);
+    for (int s = d; s < n_splits; s += blockDim.x) {
+        const float m = w_sh[s];
+        w_sh[s] = (m == -INFINITY) ? 0.f : expf(m - M);
+    }
+    __syncthreads();
+
     float num = 0.f, den = 0.f;
-    for (int s = 0; s < n_splits; ++s) {
-        const float2 ml = ml_part[((size_t)h * max_splits + s) * ROWS + r];
-        const float w = (ml.x == -INFINITY) ? 0.f : expf(ml.x - M);
-        num += w * o_part[(((size_t)h * max_splits + s) * ROWS + r) * dh + d];
-        den += w * ml.y;
+    const float* op = o_part + (base * ROWS + r) * dh + d;
+    const size_t stride = (size_t)ROWS * dh;
+    int s = 0;
+    for (; s + 8 <= n_splits; s += 8) {
+        float o[8];
+#pragma unroll
+        for (int i = 0; i < 8; ++i) o[i] = __ldcg(op + (size_t)(s + i) * stride);
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+            num = fmaf(w_sh[s + i], o[i], num);
+            den = fmaf(w_sh[s + i], l_sh[s + i], den);
+        }
+    }
+    for (; s < n_splits; ++s) {
+        num = fmaf(w_sh[s], __ldcg(op + (size_t)s * stride), num);
+        den = fmaf(w_sh[s], l_sh[s], den);
     }
     const float v = num / den;
     out[((size_t)r * n_heads + h) * dh + d] = v;

@@ -120,6 +120,7 @@ bool desc_ok(const swift_model_desc* d, std::string* why)
     if (d->page_size < 8 || d->page_size > 128 || (d->page_size & (d->page_size - 1)))
         return bad("page_size must be a power of two in 8..128");
     if (d->max_positions < d->page_size || d->max_positions % d->page_size) return bad("max_positions must be a positive multiple of page_size");
+    if (d->max_positions > 262144) return bad("max_positions is limited to 262144 (the split-combine step keeps one weight per 64 positions in shared memory)");
     if (d->max_draft < 0 || d->max_draft > SWIFT_MAX_ROWS - 1) return bad("max_draft must be in 0..15");
     if (!(d->rope_theta > 1.f) || !(d->rms_eps >= 0.f)) return bad("rope_theta > 1 and rms_eps >= 0 required");
     return true;
@@ -399,7 +400,7 @@ swift_status forward_chunk(swift_ctx* ctx, int rows, const int* toks_dev, const 
                         reinterpret_cast<TKV*>(ctx->kvbase), page_table, ctx->kv, b, d.n_heads,
                         (const float2*)kptr<float2>(ctx, ctx->kl.rope), d.max_positions));
             ST(launch_attn<TKV>(ctx, attn_mr_of(rows), page_table, b));
-            CU(launch_k(attn_combine_kernel, dim3(d.n_heads, rows), dim3(d.head_dim), 0, ctx, (const DevState*)st,
+            CU(launch_k(attn_combine_kernel, dim3(d.n_heads, rows), dim3(d.head_dim), 2 * (size_t)ctx->max_splits * sizeof(float), ctx, (const DevState*)st,
                         (const float*)kptr<float>(ctx, ctx->kl.o_part), (const float2*)kptr<float2>(ctx, ctx->kl.ml_part),
                         ctx->max_splits, d.n_heads, d.head_dim, xa, xa_hl));
             ST(run_gemm<T>(ctx, mr, GemmSite{xa, dm, qd, wptr<T>(ctx, ctx->wl.wo[b]), tc ? &ctx->tm_wo[b] : nullptr, &ctx->tm_xa}, &S));
@@ -484,7 +485,7 @@ swift_status forward_chunk_fused(swift_ctx* ctx, int rows, const int* toks_dev, 
             ep.block = b; ep.n_heads = d.n_heads; ep.max_positions = d.max_positions; ep.rope_cs = kptr<float2>(ctx, ctx->kl.rope);
             ST(gemm(EPI_QKV, &ctx->tm_wqkv[b], &ctx->tm_xn, nqkv, dm, ep));
             ST(launch_attn<TKV>(ctx, attn_mr_of(rows), page_table, b));
-            CU(launch_k(attn_combine_kernel, dim3(d.n_heads, rows), dim3(d.head_dim), 0, ctx, (const DevState*)st,
+            CU(launch_k(attn_combine_kernel, dim3(d.n_heads, rows), dim3(d.head_dim), 2 * (size_t)ctx->max_splits * sizeof(float), ctx, (const DevState*)st,
                         (const float*)kptr<float>(ctx, ctx->kl.o_part), (const float2*)kptr<float2>(ctx, ctx->kl.ml_part),
                         ctx->max_splits, d.n_heads, d.head_dim, xa, xa_hl));
             ST(gemm(EPI_RESID, &ctx->tm_wo[b], &ctx->tm_xa, dm, qd, resid));
