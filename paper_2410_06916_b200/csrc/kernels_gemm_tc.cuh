@@ -34,6 +34,7 @@ constexpr int TC_STAGES = 9;        // 144 KB of weight tiles in flight per SM: 
 constexpr int TC_THREADS = 192;
 constexpr int TC_A_BYTES = TC_TILE_N * TC_BK * 2;   // 16384
 constexpr int TC_B_BYTES = TC_COLS * TC_BK * 2;     // 4096
+constexpr int TC_PRE = 1;           // tiles requested before the set-up barrier (see the producer's comment)
 constexpr int TC_STAGE_BYTES = TC_A_BYTES + TC_B_BYTES;
 constexpr int TC_SMEM_BYTES = TC_STAGES * TC_STAGE_BYTES + 1024 /*alignment slack*/ + 256 /*barriers*/;
 constexpr long long TC_WAIT_CYCLES = 3000000000LL;  // ~1.5 s of SM clocks before a wait is declared dead
@@ -113,7 +114,11 @@ __device__ __forceinline__ int atom_add_acq_rel_gpu(int* p, int v)
 struct StreamK {
     long long U;   // units = n_tiles * KB
     int G, KB;
-    __host__ __device__ long long start(int g) const { return (U * g) / G; }
+    __host__ __device__ long long start(int g) const
+    {
+        if (U < (1ll << 31) / (G + 1)) return (long long)((unsigned)U * (unsigned)g / (unsigned)G);   // same value, 32-bit divide
+        return (U * g) / G;
+    }
     __host__ __device__ int owner(long long u) const      // the CTA whose range contains unit u
     {
         int g = (int)((u * G) / U);
@@ -290,25 +295,29 @@ gemm_tc_kernel(DevState* st, const __grid_constant__ CUtensorMap mapW, const __g
     __shared__ int page_sh[ROWS];                                              // KV page of each row's position
 
     if (tid == 0) {
-        for (int s = 0; s < TC_STAGES; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
+        // This thread is the TMA producer.  It requests its first weight tiles right away, before the block-wide
+        // set-up barrier and even before the wait for the preceding kernel (weights depend on nothing), then,
+        // once that kernel's results are visible, the matching activation tiles.  Only TC_PRE tiles go out here:
+        // a full ring from every CTA at once queues some 20 MB in front of each CTA's first tile, and the first
+        // tile then arrives microseconds later than it does behind a short queue.
+        asm volatile("prefetch.tensormap [%0];" ::"l"(&mapW) : "memory");
+        asm volatile("prefetch.tensormap [%0];" ::"l"(&mapX) : "memory");
+        for (int s = 0; s < TC_PRE; ++s) mbar_init(full_bar(s), 1);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        const int n_pre0 = (int)((u_end - u_begin) < TC_PRE ? (u_end - u_begin) : TC_PRE);
+        int tile0 = (int)(u_begin / sk.KB), kb0 = (int)(u_begin - (long long)tile0 * sk.KB);
+        for (int i = 0, t = tile0, k = kb0; i < n_pre0; ++i, (++k == sk.KB ? (k = 0, ++t) : 0)) {
+            mbar_expect_tx(full_bar(i), TC_STAGE_BYTES);
+            tma_load_2d(base + i * TC_STAGE_BYTES, &mapW, k * TC_BK, t * TC_TILE_N, full_bar(i));
+        }
+        for (int s = 0; s < TC_STAGES; ++s) { if (s >= TC_PRE) mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
         for (int b = 0; b < 2; ++b) { mbar_init(tfull_bar(b), 1); mbar_init(tempty_bar(b), 4); }
         abort_sh = 0;
         epi_abort_sh = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-        // This thread is the TMA producer.  It requests the first ring-full right away, before the block-wide
-        // set-up barrier: the weight tiles first (they depend on nothing, so they may even precede the wait for
-        // the preceding kernel), then, once that kernel's results are visible, the matching activation tiles.
-        asm volatile("prefetch.tensormap [%0];" ::"l"(&mapW) : "memory");
-        asm volatile("prefetch.tensormap [%0];" ::"l"(&mapX) : "memory");
-        const int n_pre0 = (int)((u_end - u_begin) < TC_STAGES ? (u_end - u_begin) : TC_STAGES);
-        for (int i = 0; i < n_pre0; ++i) {
-            const long long u = u_begin + i;
-            mbar_expect_tx(full_bar(i), TC_STAGE_BYTES);
-            tma_load_2d(base + i * TC_STAGE_BYTES, &mapW, (int)(u % sk.KB) * TC_BK, (int)(u / sk.KB) * TC_TILE_N, full_bar(i));
-        }
         pdl_wait();
-        for (int i = 0; i < n_pre0; ++i)
-            tma_load_2d(base + i * TC_STAGE_BYTES + TC_A_BYTES, &mapX, (int)((u_begin + i) % sk.KB) * TC_BK, 0, full_bar(i));
+        for (int i = 0, k = kb0; i < n_pre0; ++i, (++k == sk.KB ? (k = 0) : 0))
+            tma_load_2d(base + i * TC_STAGE_BYTES + TC_A_BYTES, &mapX, k * TC_BK, 0, full_bar(i));
     }
     if (warp == 1) {   // one warp allocates 64 TMEM columns: two accumulator buffers of 32
         asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&tmem_base_sh)), "r"(64));
@@ -322,7 +331,7 @@ gemm_tc_kernel(DevState* st, const __grid_constant__ CUtensorMap mapW, const __g
     if (warp == 0) {
         // ---------------------------------------------------------------- TMA producer
         if (lane == 0) {
-            const int n_pre = (int)((u_end - u_begin) < TC_STAGES ? (u_end - u_begin) : TC_STAGES);   // already requested above
+            const int n_pre = (int)((u_end - u_begin) < TC_PRE ? (u_end - u_begin) : TC_PRE);   // already requested above
             if (st->n_rows == 0) {                      // nothing to compute: let the requested tiles land, then leave
                 for (int i = 0; i < n_pre; ++i) mbar_wait(full_bar(i), 0);
             } else {
