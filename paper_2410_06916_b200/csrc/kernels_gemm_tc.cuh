@@ -110,6 +110,22 @@ __device__ __forceinline__ int atom_add_acq_rel_gpu(int* p, int v)
     return old;
 }
 
+// A 4-byte read whose value nobody uses: it pulls the address translation (and the line) of a location this
+// thread is going to store to later, so that the store at the end of the tile does not wait for a page walk.
+__device__ __forceinline__ void touch_global(const void* p)
+{
+    unsigned v;
+    const unsigned long long a = reinterpret_cast<unsigned long long>(p) & ~3ull;   // the word that holds *p
+    asm volatile("ld.global.cg.b32 %0, [%1];" : "=r"(v) : "l"(a) : "memory");
+}
+
+__device__ __forceinline__ int ld_acquire_gpu(const int* p)
+{
+    int v;
+    asm volatile("ld.acquire.gpu.global.s32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
+    return v;
+}
+
 // Static stream-K schedule shared by host and device: CTA g owns units [start(g), start(g+1)).
 struct StreamK {
     long long U;   // units = n_tiles * KB
@@ -170,7 +186,7 @@ struct EpiParams {
 };
 
 template <int EPI, typename TKV>
-__device__ __forceinline__ void tc_finalize(const EpiParams& ep, const DevState* st, float (&val)[ROWS], int n_rows, int tile,
+__device__ __forceinline__ void tc_finalize(const EpiParams& ep, int pos0, float (&val)[ROWS], int n_rows, int tile,
                                             int quarter, int lane, int etid, int N, float* Y, const float* rstd_sh,
                                             float* stage_sh, const float (&h_pre)[ROWS], float gain_pre,
                                             const float2* rope_sh, const int* page_sh)
@@ -201,27 +217,29 @@ __device__ __forceinline__ void tc_finalize(const EpiParams& ep, const DevState*
             }
         }
     } else if (EPI == EPI_RESID) {
-        float sq[ROWS];
+        // Rows go through shared memory so that the per-row work can be a rolled loop over the rows that exist:
+        // a draft step has one, and the epilogue of the last tile is executed once, from cold instruction caches.
 #pragma unroll
-        for (int m = 0; m < ROWS; ++m) {
-            sq[m] = 0.f;
-            if (n < N && m < n_rows) {
-                const float hn = h_pre[m] + val[m];
+        for (int m = 0; m < ROWS; ++m) stage_sh[m * TC_TILE_N + l] = h_pre[m] + val[m];   // read back by this thread only
+        float* sums_sh = stage_sh + ROWS * TC_TILE_N;
+#pragma unroll 1
+        for (int m = 0; m < n_rows; ++m) {
+            float hn = 0.f;
+            if (n < N) {
+                hn = stage_sh[m * TC_TILE_N + l];
                 ep.h[(size_t)m * N + n] = hn;
                 if (ep.gain_next) store_hi_lo(ep.planes_out, m, N, n, hn * gain_pre);
-                sq[m] = hn * hn;
+            }
+            if (ep.gain_next) {                        // uniform over the grid
+                const float w = warp_sum(hn * hn);
+                if (lane == 0) sums_sh[quarter * ROWS + m] = w;
             }
         }
-        if (ep.gain_next) {                            // uniform over the grid
-#pragma unroll
-            for (int m = 0; m < ROWS; ++m) {
-                const float w = warp_sum(sq[m]);
-                if (lane == 0) stage_sh[quarter * ROWS + m] = w;
-            }
+        if (ep.gain_next) {
             asm volatile("bar.sync 1, 128;" ::: "memory");
             if (etid < ROWS)
-                ep.sumsq_out[(size_t)tile * ROWS + etid] =
-                    (stage_sh[etid] + stage_sh[ROWS + etid]) + (stage_sh[2 * ROWS + etid] + stage_sh[3 * ROWS + etid]);
+                ep.sumsq_out[(size_t)tile * ROWS + etid] = etid < n_rows ?
+                    (sums_sh[etid] + sums_sh[ROWS + etid]) + (sums_sh[2 * ROWS + etid] + sums_sh[3 * ROWS + etid]) : 0.f;
             asm volatile("bar.sync 1, 128;" ::: "memory");
         }
     } else {   // EPI_QKV
@@ -232,14 +250,13 @@ __device__ __forceinline__ void tc_finalize(const EpiParams& ep, const DevState*
         const int dh = ep.L.head_dim, half = dh >> 1;
         const int gh = n / dh, i = n - gh * dh;        // global head index (q heads, then k heads, then v heads), dim
         const int lp = i < half ? l + half : l - half;
-        const int pos0 = st->pos0;
         TKV* pool = reinterpret_cast<TKV*>(ep.kv_pool);
         if (n < N) {
-#pragma unroll
-            for (int m = 0; m < ROWS; ++m) {
+#pragma unroll 1
+            for (int m = 0; m < n_rows; ++m) {         // rolled on purpose: one row per draft step, and far less code to fetch
                 const int pos = pos0 + m;
-                if (m < n_rows && pos < ep.max_positions) {
-                    const float a = val[m], b = stage_sh[m * TC_TILE_N + lp];
+                if (pos < ep.max_positions) {
+                    const float a = stage_sh[m * TC_TILE_N + l], b = stage_sh[m * TC_TILE_N + lp];
                     float out = a;
                     if (gh < ep.n_heads + ep.L.n_kv_heads) {      // q or k: rotate
                         const float2 cs = rope_sh[m * (TC_TILE_N / 2) + (i < half ? i : i - half)];
@@ -287,10 +304,10 @@ gemm_tc_kernel(DevState* st, const __grid_constant__ CUtensorMap mapW, const __g
     auto tfull_bar = [&](int b) { return bars + 8u * (2 * TC_STAGES + b); };
     auto tempty_bar = [&](int b) { return bars + 8u * (2 * TC_STAGES + 2 + b); };
     __shared__ uint32_t tmem_base_sh;
-    __shared__ int last_flag_sh;
+    __shared__ int last_flag_sh, peek_sh;
     __shared__ int abort_sh, epi_abort_sh;
     __shared__ float rstd_sh[ROWS];
-    __shared__ float stage_sh[EPI == EPI_QKV ? ROWS * TC_TILE_N : 4 * ROWS];
+    __shared__ float stage_sh[EPI == EPI_QKV ? ROWS * TC_TILE_N : EPI == EPI_RESID ? ROWS * TC_TILE_N + 4 * ROWS : 4 * ROWS];
     __shared__ float2 rope_sh[EPI == EPI_QKV ? ROWS * (TC_TILE_N / 2) : 1];   // (cos, sin) of the rows' positions
     __shared__ int page_sh[ROWS];                                              // KV page of each row's position
 
@@ -379,6 +396,7 @@ gemm_tc_kernel(DevState* st, const __grid_constant__ CUtensorMap mapW, const __g
         // ---------------------------------------------------------------- epilogue (warps 2..5)
         pdl_wait();
         const int n_rows = st->n_rows;
+        const int pos0_epi = st->pos0;                 // read once here rather than in every tile's epilogue
         const int quarter = warp & 3;                  // TMEM lanes this warp may read: 32*quarter ..
         const int etid = tid - 64;                     // 0..127
         int seg = 0;
@@ -393,7 +411,7 @@ gemm_tc_kernel(DevState* st, const __grid_constant__ CUtensorMap mapW, const __g
             rstd_sh[etid] = r;
         }
         if (EPI == EPI_QKV) {
-            const int half = ep.L.head_dim >> 1, pos0 = st->pos0;
+            const int half = ep.L.head_dim >> 1, pos0 = pos0_epi;
             for (int idx = etid; idx < ROWS * half; idx += 128) {
                 const int m = idx / half, j = idx - m * half, pos = pos0 + m;
                 if (m < n_rows && pos < ep.max_positions) rope_sh[m * (TC_TILE_N / 2) + j] = ep.rope_cs[(size_t)pos * half + j];
@@ -409,6 +427,53 @@ gemm_tc_kernel(DevState* st, const __grid_constant__ CUtensorMap mapW, const __g
             const long long tile_end = (long long)(tile + 1) * sk.KB;
             const long long seg_end = tile_end < u_end ? tile_end : u_end;
             const int buf = seg & 1;
+            const int n = tile * TC_TILE_N + quarter * 32 + lane;
+            const bool whole = (kb0 == 0) && (seg_end == tile_end);   // this CTA covered the tile's whole K range
+            // A shared tile whose other segments have all arrived already (the usual case when they sit at the start
+            // of their CTAs' ranges and this one at the end of its own) needs no slab of ours and no arrival: their
+            // slabs are fetched now, while the accumulator is still being computed, and added in slab order below.
+            int slab = 0, nseg = 1;
+            bool fast = false;
+            float pre[2][ROWS];
+            if (!whole) {
+                const int g_first = sk.owner((long long)tile * sk.KB), g_last = sk.owner(tile_end - 1);
+                slab = blockIdx.x - g_first;
+                nseg = g_last - g_first + 1;
+                if (etid == 0) peek_sh = ld_acquire_gpu(&counters[tile]);
+                asm volatile("bar.sync 1, 128;" ::: "memory");
+                fast = nseg <= 3 && peek_sh == nseg - 1;
+                if (fast) {
+#pragma unroll
+                    for (int jj = 0; jj < 2; ++jj) {
+                        const int j = jj < slab ? jj : jj + 1;          // the other segments' slabs, in slab order
+#pragma unroll
+                        for (int m = 0; m < ROWS; ++m)
+                            pre[jj][m] = (j < nseg && n < N && m < n_rows) ? __ldcg(slabs + ((size_t)j * ROWS + m) * N + n) : 0.f;
+                    }
+                }
+            }
+            if (n < N) {                                 // where this tile's results will go (row 0 stands for all rows)
+                if (EPI == EPI_PLAIN) {
+                    touch_global(Y + n);
+                } else if (EPI == EPI_SWIGLU) {
+                    if ((n >> 5) * 16 + (lane & 15) < ep.ffn) touch_global(ep.act_planes + (n >> 5) * 16 + (lane & 15));
+                } else if (EPI == EPI_RESID) {
+                    if (ep.gain_next) touch_global(ep.planes_out + n);
+                    if (ep.gain_next && lane == 0) touch_global(ep.sumsq_out + (size_t)tile * ROWS);
+                } else {
+                    const int dh = ep.L.head_dim;
+                    const int gh = n / dh, i = n - gh * dh;
+                    if (gh < ep.n_heads) {
+                        touch_global(ep.q_out + n);
+                    } else if (pos0_epi < ep.max_positions) {
+                        const int hk = gh - ep.n_heads;
+                        const int kv = hk >= ep.L.n_kv_heads ? 1 : 0;
+                        const int kh = kv ? hk - ep.L.n_kv_heads : hk;
+                        touch_global(reinterpret_cast<TKV*>(ep.kv_pool) +
+                                     ep.L.offset(page_sh[0], ep.block, kv, kh, pos0_epi & (ep.L.page_size - 1)) + i);
+                    }
+                }
+            }
             float h_pre[ROWS];
             float gain_pre = 0.f;
             if (EPI == EPI_RESID) {                     // this tile's slice of the residual stream, requested early
@@ -437,16 +502,27 @@ gemm_tc_kernel(DevState* st, const __grid_constant__ CUtensorMap mapW, const __g
             __syncwarp();
             if (lane == 0) mbar_arrive(tempty_bar(buf));       // accumulator buffer free again (4 warps arrive)
 
-            const int n = tile * TC_TILE_N + quarter * 32 + lane;
-            const bool whole = (kb0 == 0) && (seg_end == tile_end);   // this CTA covered the tile's whole K range
             float val[ROWS];
 #pragma unroll
             for (int m = 0; m < ROWS; ++m) val[m] = __uint_as_float(v[m]) + __uint_as_float(v[16 + m]);
             if (whole) {
-                tc_finalize<EPI, TKV>(ep, st, val, n_rows, tile, quarter, lane, etid, N, Y, rstd_sh, stage_sh, h_pre, gain_pre, rope_sh, page_sh);
+                tc_finalize<EPI, TKV>(ep, pos0_epi, val, n_rows, tile, quarter, lane, etid, N, Y, rstd_sh, stage_sh, h_pre, gain_pre, rope_sh, page_sh);
+            } else if (fast) {
+                // same additions as the last-arrival path below: 0 + slab 0 + slab 1 (+ slab 2), ours taken from registers
+                float acc[ROWS];
+#pragma unroll
+                for (int m = 0; m < ROWS; ++m) {
+                    const float s0 = slab == 0 ? val[m] : pre[0][m];
+                    const float s1 = slab == 1 ? val[m] : (slab == 0 ? pre[0][m] : pre[1][m]);
+                    float a = 0.f + s0;
+                    a += s1;
+                    if (nseg == 3) a += (slab == 2 ? val[m] : pre[1][m]);
+                    acc[m] = a;
+                }
+                tc_finalize<EPI, TKV>(ep, pos0_epi, acc, n_rows, tile, quarter, lane, etid, N, Y, rstd_sh, stage_sh, h_pre, gain_pre, rope_sh, page_sh);
+                if (etid == 0) counters[tile] = 0;
+                asm volatile("bar.sync 1, 128;" ::: "memory");  // peek_sh is rewritten by the next segment
             } else {
-                const int g_first = sk.owner((long long)tile * sk.KB), g_last = sk.owner(tile_end - 1);
-                const int slab = blockIdx.x - g_first, nseg = g_last - g_first + 1;
                 float* mine = slabs + (size_t)slab * ROWS * N;
                 if (n < N)
                     for (int m = 0; m < ROWS; ++m)
@@ -458,16 +534,24 @@ gemm_tc_kernel(DevState* st, const __grid_constant__ CUtensorMap mapW, const __g
 #pragma unroll
                     for (int m = 0; m < ROWS; ++m) val[m] = 0.f;
                     if (n < N) {
-                        for (int j = 0; j < nseg; ++j) {            // slab order; the 16 row loads of a slab are independent
+                        for (int j0 = 0; j0 < nseg; j0 += 2) {      // two slabs' loads in flight at a time
 #pragma unroll
-                            for (int m = 0; m < ROWS; ++m)
-                                if (m < n_rows) val[m] += __ldcg(slabs + ((size_t)j * ROWS + m) * N + n);
+                            for (int jj = 0; jj < 2; ++jj)
+#pragma unroll
+                                for (int m = 0; m < ROWS; ++m)
+                                    pre[jj][m] = (j0 + jj < nseg && m < n_rows) ? __ldcg(slabs + ((size_t)(j0 + jj) * ROWS + m) * N + n) : 0.f;
+#pragma unroll
+                            for (int m = 0; m < ROWS; ++m) val[m] += pre[0][m];
+                            if (j0 + 1 < nseg) {
+#pragma unroll
+                                for (int m = 0; m < ROWS; ++m) val[m] += pre[1][m];
+                            }
                         }
                     }
-                    tc_finalize<EPI, TKV>(ep, st, val, n_rows, tile, quarter, lane, etid, N, Y, rstd_sh, stage_sh, h_pre, gain_pre, rope_sh, page_sh);
+                    tc_finalize<EPI, TKV>(ep, pos0_epi, val, n_rows, tile, quarter, lane, etid, N, Y, rstd_sh, stage_sh, h_pre, gain_pre, rope_sh, page_sh);
                     if (etid == 0) counters[tile] = 0;
                 }
-                asm volatile("bar.sync 1, 128;" ::: "memory");  // last_flag_sh is rewritten by the next segment
+                asm volatile("bar.sync 1, 128;" ::: "memory");  // last_flag_sh and peek_sh are rewritten by the next segment
             }
             ++seg;
             u = seg_end;
