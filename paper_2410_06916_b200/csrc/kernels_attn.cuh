@@ -184,7 +184,8 @@ attn_split_kernel(const DevState* st, const float* __restrict__ q, const T* __re
 // ---------------------------------------------------------------------------------------------
 // Streaming form for head_dim == 128: no shared-memory staging of K and V; every byte of the cache is
 // loaded once, straight into registers, by coalesced warp loads with many rows in flight per warp.
-// grid = (H, max_splits), block = 128.  Warp w owns positions [16w, 16w + 16) of the chunk and takes
+// grid = (H, max_splits, row groups), block = 128.  A CTA takes MR consecutive rows of the forward chunk
+// (blockIdx.z picks the group).  Warp w owns positions [16w, 16w + 16) of the chunk and takes
 // them in two batches of eight.  Within a batch, with lane = 8 * pg + dl:
 //   K : lane holds elements {32c + 4dl .. +3, c = 0..3} of rows pg and pg + 4 (eight lanes per row),
 //       so a score is a 16-term chain per lane followed by a three-level xor tree over dl.  The tree is
@@ -250,10 +251,13 @@ attn_stream_kernel(const DevState* st, const float* __restrict__ q, const T* __r
     constexpr int DH = 128, NW = ATTN_THREADS / 32, PER_WARP = ATTN_CHUNK / NW;
     static_assert(PER_WARP == 2 * ATTN_BATCH, "two batches per warp");
     constexpr int N1 = MR, N2 = folded(N1), N3 = folded(N2);       // sums per lane after each tree level
-    const int n_rows = min(st->n_rows, MR);
-    if (n_rows == 0) return;
-    const int pos0 = st->pos0;
-    const int total = pos0 + n_rows;
+    // blockIdx.z selects a group of MR consecutive rows of the forward chunk; everything below is relative to it
+    const int row0 = blockIdx.z * MR;
+    const int n_rows = min(st->n_rows - row0, MR);
+    if (n_rows <= 0) return;
+    const int pos0 = st->pos0 + row0;                       // position of the group's first row
+    const int total = pos0 + n_rows;                        // positions visible to the group's last row
+    q += (size_t)row0 * n_heads * 128;
     const int h = blockIdx.x, s = blockIdx.y;
     const int c0 = s * ATTN_CHUNK;
     if (c0 >= total) return;
@@ -401,8 +405,8 @@ attn_stream_kernel(const DevState* st, const float* __restrict__ q, const T* __r
             num = fmaf(wt, part_acc[ww][r][tid], num);
             den = fmaf(wt, ml.y, den);
         }
-        o_part[(((size_t)h * max_splits + s) * ROWS + r) * DH + tid] = num;
-        if (tid == 0) ml_part[((size_t)h * max_splits + s) * ROWS + r] = make_float2(M, den);
+        o_part[(((size_t)h * max_splits + s) * ROWS + row0 + r) * DH + tid] = num;
+        if (tid == 0) ml_part[((size_t)h * max_splits + s) * ROWS + row0 + r] = make_float2(M, den);
     }
 }
 
@@ -418,8 +422,9 @@ __global__ void attn_combine_kernel(const DevState* st, const float* __restrict_
     const int r = blockIdx.y;
     if (r >= st->n_rows) return;
     const int h = blockIdx.x, d = threadIdx.x;
-    const int total = st->pos0 + st->n_rows;
-    const int n_splits = (total + ATTN_CHUNK - 1) / ATTN_CHUNK;
+    // row r sees positions <= pos0 + r: later splits hold nothing for it (and, when the rows were processed in
+    // groups, were not written for it at all)
+    const int n_splits = (st->pos0 + r + 1 + ATTN_CHUNK - 1) / ATTN_CHUNK;
     extern __shared__ float comb_sh[];
     float* w_sh = comb_sh;                    // [n_splits] exp(m_s - M), 0 for empty splits
     float* l_sh = comb_sh + max_splits;       // [n_splits]

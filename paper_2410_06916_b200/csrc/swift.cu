@@ -75,6 +75,7 @@ struct swift_ctx {
     cudaEvent_t ev[8];
     // captured forwards; programmatic dependent launch between the kernels of a forward
     bool use_graphs, use_pdl, fuse;
+    int attn_rows_per_cta;
     std::vector<FwdGraph>* graphs;
     uint64_t graph_clock;
     // tensor-core GEMM path (bf16 models)
@@ -324,12 +325,13 @@ swift_status run_gemm(swift_ctx* ctx, int mr, const GemmSite& g, int* n_split)
 }
 
 template <typename T, int MR>
-swift_status launch_attn_mr(swift_ctx* ctx, const int* page_table, int block)
+swift_status launch_attn_mr(swift_ctx* ctx, const int* page_table, int block, int groups = 1)
 {
     const swift_model_desc& d = ctx->d;
     const size_t smem = 2 * (size_t)ATTN_CHUNK * d.head_dim * sizeof(T) + ((size_t)MR * d.head_dim + 3 * (size_t)MR * ATTN_CHUNK) * sizeof(float);
     dim3 grid(d.n_heads, ctx->max_splits);
     if (d.head_dim == 128) {
+        grid.z = groups;
         CU(launch_k(attn_stream_kernel<T, MR>, grid, dim3(ATTN_THREADS), 0, ctx, (const DevState*)state_of(ctx),
                     (const float*)kptr<float>(ctx, ctx->kl.q), reinterpret_cast<const T*>(ctx->kvbase), page_table, ctx->kv,
                     block, d.n_heads, ctx->max_splits, 1.0f / sqrtf((float)d.head_dim), kptr<float>(ctx, ctx->kl.o_part),
@@ -344,15 +346,23 @@ swift_status launch_attn_mr(swift_ctx* ctx, const int* page_table, int block)
 }
 
 template <typename T>
-swift_status launch_attn(swift_ctx* ctx, int mr, const int* page_table, int block)
+swift_status launch_attn(swift_ctx* ctx, int rows, const int* page_table, int block)
 {
+    // The streaming kernel (head_dim 128) takes the rows in groups of at most attn_rows_per_cta, one group per
+    // grid.z slice: fewer rows per CTA means fewer registers and more CTAs in flight.
+    int mr = attn_mr_of(rows), groups = 1;
+    if (ctx->d.head_dim == 128 && rows > ctx->attn_rows_per_cta) {
+        mr = ctx->attn_rows_per_cta;
+        groups = ceil_div(rows, mr);
+    }
     switch (mr) {
-    case 1: return launch_attn_mr<T, 1>(ctx, page_table, block);
-    case 2: return launch_attn_mr<T, 2>(ctx, page_table, block);
-    case 4: return launch_attn_mr<T, 4>(ctx, page_table, block);
-    case 8: return launch_attn_mr<T, 8>(ctx, page_table, block);
-    case 12: return launch_attn_mr<T, 12>(ctx, page_table, block);
-    default: return launch_attn_mr<T, 16>(ctx, page_table, block);
+    case 1: return launch_attn_mr<T, 1>(ctx, page_table, block, groups);
+    case 2: return launch_attn_mr<T, 2>(ctx, page_table, block, groups);
+    case 4: return launch_attn_mr<T, 4>(ctx, page_table, block, groups);
+    case 6: return launch_attn_mr<T, 6>(ctx, page_table, block, groups);
+    case 8: return launch_attn_mr<T, 8>(ctx, page_table, block, groups);
+    case 12: return launch_attn_mr<T, 12>(ctx, page_table, block, groups);
+    default: return launch_attn_mr<T, 16>(ctx, page_table, block, groups);
     }
 }
 
@@ -399,7 +409,7 @@ swift_status forward_chunk(swift_ctx* ctx, int rows, const int* toks_dev, const 
                         (const DevState*)st, (const float*)part, S, (size_t)ROWS * nqkv, nqkv, kptr<float>(ctx, ctx->kl.q),
                         reinterpret_cast<TKV*>(ctx->kvbase), page_table, ctx->kv, b, d.n_heads,
                         (const float2*)kptr<float2>(ctx, ctx->kl.rope), d.max_positions));
-            ST(launch_attn<TKV>(ctx, attn_mr_of(rows), page_table, b));
+            ST(launch_attn<TKV>(ctx, rows, page_table, b));
             CU(launch_k(attn_combine_kernel, dim3(d.n_heads, rows), dim3(d.head_dim), 2 * (size_t)ctx->max_splits * sizeof(float), ctx, (const DevState*)st,
                         (const float*)kptr<float>(ctx, ctx->kl.o_part), (const float2*)kptr<float2>(ctx, ctx->kl.ml_part),
                         ctx->max_splits, d.n_heads, d.head_dim, xa, xa_hl));
@@ -484,7 +494,7 @@ swift_status forward_chunk_fused(swift_ctx* ctx, int rows, const int* toks_dev, 
             ep.q_out = kptr<float>(ctx, ctx->kl.q); ep.kv_pool = ctx->kvbase; ep.page_table = page_table; ep.L = ctx->kv;
             ep.block = b; ep.n_heads = d.n_heads; ep.max_positions = d.max_positions; ep.rope_cs = kptr<float2>(ctx, ctx->kl.rope);
             ST(gemm(EPI_QKV, &ctx->tm_wqkv[b], &ctx->tm_xn, nqkv, dm, ep));
-            ST(launch_attn<TKV>(ctx, attn_mr_of(rows), page_table, b));
+            ST(launch_attn<TKV>(ctx, rows, page_table, b));
             CU(launch_k(attn_combine_kernel, dim3(d.n_heads, rows), dim3(d.head_dim), 2 * (size_t)ctx->max_splits * sizeof(float), ctx, (const DevState*)st,
                         (const float*)kptr<float>(ctx, ctx->kl.o_part), (const float2*)kptr<float2>(ctx, ctx->kl.ml_part),
                         ctx->max_splits, d.n_heads, d.head_dim, xa, xa_hl));
@@ -923,6 +933,11 @@ swift_status swift_load(const swift_model_desc* desc, swift_devbuf weights, swif
     }
     for (auto& e : c->ev) e = nullptr;
     c->use_graphs = getenv("SWIFT_NO_GRAPHS") == nullptr;
+    {
+        const char* e = getenv("SWIFT_ATTN_ROWS");           // rows per attention CTA: 1, 2, 4, 6, 8, 12 or 16
+        const int v = e ? atoi(e) : 16;
+        c->attn_rows_per_cta = (v == 1 || v == 2 || v == 4 || v == 6 || v == 8 || v == 12) ? v : 16;
+    }
     c->use_pdl = getenv("SWIFT_PDL") != nullptr;   // programmatic dependent launch: measured neutral to slightly negative on whole forwards, so opt-in
     c->fuse = getenv("SWIFT_NO_FUSE") == nullptr && desc->head_dim <= TC_TILE_N;
     c->graphs = new std::vector<FwdGraph>();
