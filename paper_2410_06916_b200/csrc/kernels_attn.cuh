@@ -181,6 +181,65 @@ attn_split_kernel(const DevState* st, const float* __restrict__ q, const T* __re
     if (tid < n_rows) ml_part[((size_t)h * max_splits + s) * ROWS + tid] = make_float2(row_m[tid], row_l[tid]);
 }
 
+// Merges the splits of one (head, row) in chunk order; called by all blockDim.x = dh threads of a block.
+// comb_sh: 2 * max_splits floats, wmax_sh: 32 floats of shared memory.  The (m, l) pairs are fetched once per
+// block, spread over the threads, and the partial outputs are read eight splits at a time with independent
+// loads, so this costs a few trips to L2 rather than one per split; the sums themselves run over the splits
+// in ascending order.
+__device__ __forceinline__ void combine_row(int pos0, int r, int h, const float* __restrict__ o_part,
+                                            const float2* __restrict__ ml_part, int max_splits, int n_heads, int dh,
+                                            float* __restrict__ out, __nv_bfloat16* __restrict__ planes,
+                                            float* comb_sh, float* wmax_sh)
+{
+    const int d = threadIdx.x;
+    // row r sees positions <= pos0 + r: later splits hold nothing for it (and, when the rows were processed in
+    // groups, were not written for it at all)
+    const int n_splits = (pos0 + r + 1 + ATTN_CHUNK - 1) / ATTN_CHUNK;
+    float* w_sh = comb_sh;                    // [n_splits] exp(m_s - M), 0 for empty splits
+    float* l_sh = comb_sh + max_splits;       // [n_splits]
+    const size_t base = (size_t)h * max_splits;
+
+    float mx = -INFINITY;
+    for (int s = d; s < n_splits; s += blockDim.x) {
+        const float2 ml = __ldcg(ml_part + (base + s) * ROWS + r);
+        w_sh[s] = ml.x;
+        l_sh[s] = ml.y;
+        mx = fmaxf(mx, ml.x);
+    }
+    mx = warp_max(mx);
+    if ((d & 31) == 0) wmax_sh[d >> 5] = mx;
+    __syncthreads();
+    float M = -INFINITY;
+    for (int wi = 0; wi < (int)(blockDim.x + 31) / 32; ++wi) M = fmaxf(M, wmax_sh[wi]);
+    for (int s = d; s < n_splits; s += blockDim.x) {
+        const float m = w_sh[s];
+        w_sh[s] = (m == -INFINITY) ? 0.f : expf(m - M);
+    }
+    __syncthreads();
+
+    float num = 0.f, den = 0.f;
+    const float* op = o_part + (base * ROWS + r) * dh + d;
+    const size_t stride = (size_t)ROWS * dh;
+    int s = 0;
+    for (; s + 8 <= n_splits; s += 8) {
+        float o[8];
+#pragma unroll
+        for (int i = 0; i < 8; ++i) o[i] = __ldcg(op + (size_t)(s + i) * stride);
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+            num = fmaf(w_sh[s + i], o[i], num);
+            den = fmaf(w_sh[s + i], l_sh[s + i], den);
+        }
+    }
+    for (; s < n_splits; ++s) {
+        num = fmaf(w_sh[s], __ldcg(op + (size_t)s * stride), num);
+        den = fmaf(w_sh[s], l_sh[s], den);
+    }
+    const float v = num / den;
+    out[((size_t)r * n_heads + h) * dh + d] = v;
+    if (planes) store_hi_lo(planes, r, n_heads * dh, h * dh + d, v);
+}
+
 // ---------------------------------------------------------------------------------------------
 // Streaming form for head_dim == 128: no shared-memory staging of K and V; every byte of the cache is
 // loaded once, straight into registers, by coalesced warp loads with many rows in flight per warp.
@@ -245,7 +304,8 @@ template <typename T, int MR>
 __global__ void __launch_bounds__(ATTN_THREADS, MR == 1 ? 5 : (MR <= 12 ? 3 : 2))
 attn_stream_kernel(const DevState* st, const float* __restrict__ q, const T* __restrict__ kv_pool,
                    const int* __restrict__ page_table, KvLayout L, int block, int n_heads, int max_splits,
-                   float scale, float* __restrict__ o_part, float2* __restrict__ ml_part)
+                   float scale, float* __restrict__ o_part, float2* __restrict__ ml_part,
+                   int* __restrict__ head_counters, float* __restrict__ out, __nv_bfloat16* __restrict__ planes)
 {
     pdl_enter();
     constexpr int DH = 128, NW = ATTN_THREADS / 32, PER_WARP = ATTN_CHUNK / NW;
@@ -408,12 +468,31 @@ attn_stream_kernel(const DevState* st, const float* __restrict__ q, const T* __r
         o_part[(((size_t)h * max_splits + s) * ROWS + row0 + r) * DH + tid] = num;
         if (tid == 0) ml_part[((size_t)h * max_splits + s) * ROWS + row0 + r] = make_float2(M, den);
     }
+
+    // One-row forwards (draft and vanilla steps) merge the chunks here instead of in a launch of their own: every
+    // CTA of the head arrives on a counter once its partial result is stored, and the last one to arrive runs the
+    // same merge the combine kernel runs (zero on entry, zero again on exit; dynamic smem = 2 * max_splits floats).
+    if constexpr (MR == 1) {
+        if (head_counters) {
+            __shared__ int last_sh;
+            __shared__ float wmax_sh[32];
+            extern __shared__ float comb_sh[];
+            __syncthreads();                                    // this CTA's stores precede its arrival
+            if (tid == 0) {
+                const int n_chunks = (total + ATTN_CHUNK - 1) / ATTN_CHUNK;
+                last_sh = atom_add_acq_rel_gpu(&head_counters[h], 1) == n_chunks - 1;
+            }
+            __syncthreads();
+            if (last_sh) {
+                combine_row(pos0, 0, h, o_part, ml_part, max_splits, n_heads, DH, out, planes, comb_sh, wmax_sh);
+                if (tid == 0) head_counters[h] = 0;
+            }
+        }
+    }
 }
 
 // grid = (H, rows), block = dh threads, dynamic smem = 2 * max_splits floats.  Combines the splits in chunk
-// order.  The (m, l) pairs are fetched once per block, spread over the threads, and the partial outputs are
-// read eight splits at a time with independent loads, so the kernel costs a few trips to L2 rather than one
-// per split; the sums themselves still run over the splits in ascending order.
+// order (combine_row above).
 __global__ void attn_combine_kernel(const DevState* st, const float* __restrict__ o_part,
                                     const float2* __restrict__ ml_part, int max_splits, int n_heads, int dh,
                                     float* __restrict__ out, __nv_bfloat16* __restrict__ planes)
@@ -421,55 +500,9 @@ __global__ void attn_combine_kernel(const DevState* st, const float* __restrict_
     pdl_enter();
     const int r = blockIdx.y;
     if (r >= st->n_rows) return;
-    const int h = blockIdx.x, d = threadIdx.x;
-    // row r sees positions <= pos0 + r: later splits hold nothing for it (and, when the rows were processed in
-    // groups, were not written for it at all)
-    const int n_splits = (st->pos0 + r + 1 + ATTN_CHUNK - 1) / ATTN_CHUNK;
     extern __shared__ float comb_sh[];
-    float* w_sh = comb_sh;                    // [n_splits] exp(m_s - M), 0 for empty splits
-    float* l_sh = comb_sh + max_splits;       // [n_splits]
     __shared__ float wmax_sh[32];
-    const size_t base = (size_t)h * max_splits;
-
-    float mx = -INFINITY;
-    for (int s = d; s < n_splits; s += blockDim.x) {
-        const float2 ml = ml_part[(base + s) * ROWS + r];
-        w_sh[s] = ml.x;
-        l_sh[s] = ml.y;
-        mx = fmaxf(mx, ml.x);
-    }
-    mx = warp_max(mx);
-    if ((d & 31) == 0) wmax_sh[d >> 5] = mx;
-    __syncthreads();
-    float M = -INFINITY;
-    for (int wi = 0; wi < (int)(blockDim.x + 31) / 32; ++wi) M = fmaxf(M, wmax_sh[wi]);
-    for (int s = d; s < n_splits; s += blockDim.x) {
-        const float m = w_sh[s];
-        w_sh[s] = (m == -INFINITY) ? 0.f : expf(m - M);
-    }
-    __syncthreads();
-
-    float num = 0.f, den = 0.f;
-    const float* op = o_part + (base * ROWS + r) * dh + d;
-    const size_t stride = (size_t)ROWS * dh;
-    int s = 0;
-    for (; s + 8 <= n_splits; s += 8) {
-        float o[8];
-#pragma unroll
-        for (int i = 0; i < 8; ++i) o[i] = __ldcg(op + (size_t)(s + i) * stride);
-#pragma unroll
-        for (int i = 0; i < 8; ++i) {
-            num = fmaf(w_sh[s + i], o[i], num);
-            den = fmaf(w_sh[s + i], l_sh[s + i], den);
-        }
-    }
-    for (; s < n_splits; ++s) {
-        num = fmaf(w_sh[s], __ldcg(op + (size_t)s * stride), num);
-        den = fmaf(w_sh[s], l_sh[s], den);
-    }
-    const float v = num / den;
-    out[((size_t)r * n_heads + h) * dh + d] = v;
-    if (planes) store_hi_lo(planes, r, n_heads * dh, h * dh + d, v);
+    combine_row(st->pos0, r, blockIdx.x, o_part, ml_part, max_splits, n_heads, dh, out, planes, comb_sh, wmax_sh);
 }
 
 } // namespace swk

@@ -47,7 +47,7 @@ struct WeightLayout {
 
 struct WorkLayout {
     size_t state, h, xn, xa, act, q, part, o_part, ml_part, logits, q_rows, rope, pt_main, pt_score, score_tok,
-        score_truth, score_out, xn_hl, xa_hl, act_hl, slabs, counters, sumsq, total;
+        score_truth, score_out, attn_counters, xn_hl, xa_hl, act_hl, slabs, counters, sumsq, total;
     size_t part_floats, slab_floats;
 };
 
@@ -74,7 +74,7 @@ struct swift_ctx {
     std::string err;
     cudaEvent_t ev[8];
     // captured forwards; programmatic dependent launch between the kernels of a forward
-    bool use_graphs, use_pdl, fuse;
+    bool use_graphs, use_pdl, fuse, fuse_combine;
     int attn_rows_per_cta;
     std::vector<FwdGraph>* graphs;
     uint64_t graph_clock;
@@ -222,6 +222,7 @@ WorkLayout work_layout(const swift_model_desc* d)
     k.score_tok = c.take(MAX_SCORE_ROWS * 4);
     k.score_truth = c.take(MAX_SCORE_ROWS * 4);
     k.score_out = c.take(1024 * 4);
+    k.attn_counters = c.take((size_t)d->n_heads * 4);
     // tensor-core path (bf16 models): hi/lo bf16 planes of the GEMM inputs, stream-K slabs, tile counters
     k.slab_floats = 0;
     k.xn_hl = k.xa_hl = k.act_hl = k.slabs = k.counters = k.sumsq = 0;
@@ -325,17 +326,19 @@ swift_status run_gemm(swift_ctx* ctx, int mr, const GemmSite& g, int* n_split)
 }
 
 template <typename T, int MR>
-swift_status launch_attn_mr(swift_ctx* ctx, const int* page_table, int block, int groups = 1)
+swift_status launch_attn_mr(swift_ctx* ctx, const int* page_table, int block, int groups, float* fused_out, __nv_bfloat16* fused_planes)
 {
     const swift_model_desc& d = ctx->d;
     const size_t smem = 2 * (size_t)ATTN_CHUNK * d.head_dim * sizeof(T) + ((size_t)MR * d.head_dim + 3 * (size_t)MR * ATTN_CHUNK) * sizeof(float);
     dim3 grid(d.n_heads, ctx->max_splits);
     if (d.head_dim == 128) {
         grid.z = groups;
-        CU(launch_k(attn_stream_kernel<T, MR>, grid, dim3(ATTN_THREADS), 0, ctx, (const DevState*)state_of(ctx),
-                    (const float*)kptr<float>(ctx, ctx->kl.q), reinterpret_cast<const T*>(ctx->kvbase), page_table, ctx->kv,
-                    block, d.n_heads, ctx->max_splits, 1.0f / sqrtf((float)d.head_dim), kptr<float>(ctx, ctx->kl.o_part),
-                    kptr<float2>(ctx, ctx->kl.ml_part)));
+        const bool fused = MR == 1 && fused_out != nullptr;       // one-row forwards merge the chunks in the same launch
+        CU(launch_k(attn_stream_kernel<T, MR>, grid, dim3(ATTN_THREADS), fused ? 2 * (size_t)ctx->max_splits * sizeof(float) : 0, ctx,
+                    (const DevState*)state_of(ctx), (const float*)kptr<float>(ctx, ctx->kl.q), reinterpret_cast<const T*>(ctx->kvbase),
+                    page_table, ctx->kv, block, d.n_heads, ctx->max_splits, 1.0f / sqrtf((float)d.head_dim),
+                    kptr<float>(ctx, ctx->kl.o_part), kptr<float2>(ctx, ctx->kl.ml_part),
+                    fused ? kptr<int>(ctx, ctx->kl.attn_counters) : (int*)nullptr, fused_out, fused_planes));
         return SWIFT_OK;
     }
     CU(launch_k(attn_split_kernel<T, MR>, grid, dim3(ATTN_THREADS), smem, ctx, (const DevState*)state_of(ctx),
@@ -345,25 +348,37 @@ swift_status launch_attn_mr(swift_ctx* ctx, const int* page_table, int block, in
     return SWIFT_OK;
 }
 
+// Attention of one block for the forward chunk's rows: split kernel + merge of the splits into `out` (fp32 rows)
+// and, when given, the hi/lo planes the next GEMM reads.
 template <typename T>
-swift_status launch_attn(swift_ctx* ctx, int rows, const int* page_table, int block)
+swift_status launch_attn(swift_ctx* ctx, int rows, const int* page_table, int block, float* out, __nv_bfloat16* planes)
 {
+    const swift_model_desc& d = ctx->d;
     // The streaming kernel (head_dim 128) takes the rows in groups of at most attn_rows_per_cta, one group per
     // grid.z slice: fewer rows per CTA means fewer registers and more CTAs in flight.
     int mr = attn_mr_of(rows), groups = 1;
-    if (ctx->d.head_dim == 128 && rows > ctx->attn_rows_per_cta) {
+    if (d.head_dim == 128 && rows > ctx->attn_rows_per_cta) {
         mr = ctx->attn_rows_per_cta;
         groups = ceil_div(rows, mr);
     }
+    const bool fused = d.head_dim == 128 && rows == 1 && ctx->fuse_combine;
+    float* fo = fused ? out : nullptr;
+    __nv_bfloat16* fp = fused ? planes : nullptr;
+    swift_status s;
     switch (mr) {
-    case 1: return launch_attn_mr<T, 1>(ctx, page_table, block, groups);
-    case 2: return launch_attn_mr<T, 2>(ctx, page_table, block, groups);
-    case 4: return launch_attn_mr<T, 4>(ctx, page_table, block, groups);
-    case 6: return launch_attn_mr<T, 6>(ctx, page_table, block, groups);
-    case 8: return launch_attn_mr<T, 8>(ctx, page_table, block, groups);
-    case 12: return launch_attn_mr<T, 12>(ctx, page_table, block, groups);
-    default: return launch_attn_mr<T, 16>(ctx, page_table, block, groups);
+    case 1: s = launch_attn_mr<T, 1>(ctx, page_table, block, groups, fo, fp); break;
+    case 2: s = launch_attn_mr<T, 2>(ctx, page_table, block, groups, fo, fp); break;
+    case 4: s = launch_attn_mr<T, 4>(ctx, page_table, block, groups, fo, fp); break;
+    case 6: s = launch_attn_mr<T, 6>(ctx, page_table, block, groups, fo, fp); break;
+    case 8: s = launch_attn_mr<T, 8>(ctx, page_table, block, groups, fo, fp); break;
+    case 12: s = launch_attn_mr<T, 12>(ctx, page_table, block, groups, fo, fp); break;
+    default: s = launch_attn_mr<T, 16>(ctx, page_table, block, groups, fo, fp); break;
     }
+    if (s != SWIFT_OK || fused) return s;
+    CU(launch_k(attn_combine_kernel, dim3(d.n_heads, rows), dim3(d.head_dim), 2 * (size_t)ctx->max_splits * sizeof(float), ctx,
+                (const DevState*)state_of(ctx), (const float*)kptr<float>(ctx, ctx->kl.o_part),
+                (const float2*)kptr<float2>(ctx, ctx->kl.ml_part), ctx->max_splits, d.n_heads, d.head_dim, out, planes));
+    return SWIFT_OK;
 }
 
 struct HeadOpts {
@@ -409,10 +424,7 @@ swift_status forward_chunk(swift_ctx* ctx, int rows, const int* toks_dev, const 
                         (const DevState*)st, (const float*)part, S, (size_t)ROWS * nqkv, nqkv, kptr<float>(ctx, ctx->kl.q),
                         reinterpret_cast<TKV*>(ctx->kvbase), page_table, ctx->kv, b, d.n_heads,
                         (const float2*)kptr<float2>(ctx, ctx->kl.rope), d.max_positions));
-            ST(launch_attn<TKV>(ctx, rows, page_table, b));
-            CU(launch_k(attn_combine_kernel, dim3(d.n_heads, rows), dim3(d.head_dim), 2 * (size_t)ctx->max_splits * sizeof(float), ctx, (const DevState*)st,
-                        (const float*)kptr<float>(ctx, ctx->kl.o_part), (const float2*)kptr<float2>(ctx, ctx->kl.ml_part),
-                        ctx->max_splits, d.n_heads, d.head_dim, xa, xa_hl));
+            ST(launch_attn<TKV>(ctx, rows, page_table, b, xa, xa_hl));
             ST(run_gemm<T>(ctx, mr, GemmSite{xa, dm, qd, wptr<T>(ctx, ctx->wl.wo[b]), tc ? &ctx->tm_wo[b] : nullptr, &ctx->tm_xa}, &S));
             pend = part; pend_S = S;
         }
@@ -494,10 +506,7 @@ swift_status forward_chunk_fused(swift_ctx* ctx, int rows, const int* toks_dev, 
             ep.q_out = kptr<float>(ctx, ctx->kl.q); ep.kv_pool = ctx->kvbase; ep.page_table = page_table; ep.L = ctx->kv;
             ep.block = b; ep.n_heads = d.n_heads; ep.max_positions = d.max_positions; ep.rope_cs = kptr<float2>(ctx, ctx->kl.rope);
             ST(gemm(EPI_QKV, &ctx->tm_wqkv[b], &ctx->tm_xn, nqkv, dm, ep));
-            ST(launch_attn<TKV>(ctx, rows, page_table, b));
-            CU(launch_k(attn_combine_kernel, dim3(d.n_heads, rows), dim3(d.head_dim), 2 * (size_t)ctx->max_splits * sizeof(float), ctx, (const DevState*)st,
-                        (const float*)kptr<float>(ctx, ctx->kl.o_part), (const float2*)kptr<float2>(ctx, ctx->kl.ml_part),
-                        ctx->max_splits, d.n_heads, d.head_dim, xa, xa_hl));
+            ST(launch_attn<TKV>(ctx, rows, page_table, b, xa, xa_hl));
             ST(gemm(EPI_RESID, &ctx->tm_wo[b], &ctx->tm_xa, dm, qd, resid));
         } else {
             EpiParams ep = base;
@@ -938,6 +947,7 @@ swift_status swift_load(const swift_model_desc* desc, swift_devbuf weights, swif
         const int v = e ? atoi(e) : 16;
         c->attn_rows_per_cta = (v == 1 || v == 2 || v == 4 || v == 6 || v == 8 || v == 12) ? v : 16;
     }
+    c->fuse_combine = getenv("SWIFT_NO_FUSE_COMBINE") == nullptr;
     c->use_pdl = getenv("SWIFT_PDL") != nullptr;   // programmatic dependent launch: measured neutral to slightly negative on whole forwards, so opt-in
     c->fuse = getenv("SWIFT_NO_FUSE") == nullptr && desc->head_dim <= TC_TILE_N;
     c->graphs = new std::vector<FwdGraph>();
