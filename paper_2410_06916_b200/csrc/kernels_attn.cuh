@@ -199,6 +199,14 @@ __device__ __forceinline__ void combine_row(int pos0, int r, int h, const float*
     float* l_sh = comb_sh + max_splits;       // [n_splits]
     const size_t base = (size_t)h * max_splits;
 
+    // the first 16 splits' partial outputs are requested before anything else: they do not depend on the weights
+    constexpr int CB = 16;
+    const float* op = o_part + (base * ROWS + r) * dh + d;
+    const size_t stride = (size_t)ROWS * dh;
+    float o[CB];
+#pragma unroll
+    for (int i = 0; i < CB; ++i) o[i] = i < n_splits ? __ldcg(op + (size_t)i * stride) : 0.f;
+
     float mx = -INFINITY;
     for (int s = d; s < n_splits; s += blockDim.x) {
         const float2 ml = __ldcg(ml_part + (base + s) * ROWS + r);
@@ -218,22 +226,18 @@ __device__ __forceinline__ void combine_row(int pos0, int r, int h, const float*
     __syncthreads();
 
     float num = 0.f, den = 0.f;
-    const float* op = o_part + (base * ROWS + r) * dh + d;
-    const size_t stride = (size_t)ROWS * dh;
-    int s = 0;
-    for (; s + 8 <= n_splits; s += 8) {
-        float o[8];
+    for (int s0 = 0; s0 < n_splits; s0 += CB) {
+        if (s0 > 0) {
 #pragma unroll
-        for (int i = 0; i < 8; ++i) o[i] = __ldcg(op + (size_t)(s + i) * stride);
-#pragma unroll
-        for (int i = 0; i < 8; ++i) {
-            num = fmaf(w_sh[s + i], o[i], num);
-            den = fmaf(w_sh[s + i], l_sh[s + i], den);
+            for (int i = 0; i < CB; ++i) o[i] = s0 + i < n_splits ? __ldcg(op + (size_t)(s0 + i) * stride) : 0.f;
         }
-    }
-    for (; s < n_splits; ++s) {
-        num = fmaf(w_sh[s], __ldcg(op + (size_t)s * stride), num);
-        den = fmaf(w_sh[s], l_sh[s], den);
+#pragma unroll
+        for (int i = 0; i < CB; ++i) {
+            if (s0 + i < n_splits) {
+                num = fmaf(w_sh[s0 + i], o[i], num);
+                den = fmaf(w_sh[s0 + i], l_sh[s0 + i], den);
+            }
+        }
     }
     const float v = num / den;
     out[((size_t)r * n_heads + h) * dh + d] = v;

@@ -206,16 +206,20 @@ __device__ __forceinline__ void tc_finalize(const EpiParams& ep, int pos0, float
                 if (m < n_rows) Y[(size_t)m * N + n] = val[m];
         }
     } else if (EPI == EPI_SWIGLU) {
-        // rows come in groups of 32: 16 gate rows then the 16 matching up rows
+        // rows come in groups of 32: 16 gate rows then the 16 matching up rows (same warp); staged through shared
+        // memory so that the loop over the forward's rows can stay rolled
         const int i = (n >> 5) * 16 + (lane & 15);
 #pragma unroll
-        for (int m = 0; m < ROWS; ++m) {
-            const float up = __shfl_down_sync(0xFFFFFFFFu, val[m], 16);
-            if (lane < 16 && m < n_rows && i < ep.ffn) {
-                const float g = val[m];
+        for (int m = 0; m < ROWS; ++m) stage_sh[m * TC_TILE_N + l] = val[m];
+        __syncwarp();
+        if (lane < 16 && i < ep.ffn) {
+#pragma unroll 1
+            for (int m = 0; m < n_rows; ++m) {
+                const float g = stage_sh[m * TC_TILE_N + l], up = stage_sh[m * TC_TILE_N + l + 16];
                 store_hi_lo(ep.act_planes, m, ep.ffn, i, g / (1.f + expf(-g)) * up);
             }
         }
+        __syncwarp();                                  // the staging rows are rewritten by the next tile
     } else if (EPI == EPI_RESID) {
         // Rows go through shared memory so that the per-row work can be a rolled loop over the rows that exist:
         // a draft step has one, and the epilogue of the last tile is executed once, from cold instruction caches.
@@ -307,7 +311,7 @@ gemm_tc_kernel(DevState* st, const __grid_constant__ CUtensorMap mapW, const __g
     __shared__ int last_flag_sh, peek_sh;
     __shared__ int abort_sh, epi_abort_sh;
     __shared__ float rstd_sh[ROWS];
-    __shared__ float stage_sh[EPI == EPI_QKV ? ROWS * TC_TILE_N : EPI == EPI_RESID ? ROWS * TC_TILE_N + 4 * ROWS : 4 * ROWS];
+    __shared__ float stage_sh[EPI == EPI_PLAIN ? 4 * ROWS : ROWS * TC_TILE_N + 4 * ROWS];
     __shared__ float2 rope_sh[EPI == EPI_QKV ? ROWS * (TC_TILE_N / 2) : 1];   // (cos, sin) of the rows' positions
     __shared__ int page_sh[ROWS];                                              // KV page of each row's position
 
