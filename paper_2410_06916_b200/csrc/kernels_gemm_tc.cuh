@@ -331,16 +331,19 @@ gemm_tc_kernel(DevState* st, const __grid_constant__ CUtensorMap mapW, const __g
             mbar_expect_tx(full_bar(i), TC_STAGE_BYTES);
             tma_load_2d(base + i * TC_STAGE_BYTES, &mapW, k * TC_BK, t * TC_TILE_N, full_bar(i));
         }
-        for (int s = 0; s < TC_STAGES; ++s) { if (s >= TC_PRE) mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
-        for (int b = 0; b < 2; ++b) { mbar_init(tfull_bar(b), 1); mbar_init(tempty_bar(b), 4); }
-        abort_sh = 0;
-        epi_abort_sh = 0;
-        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         pdl_wait();
         for (int i = 0, k = kb0; i < n_pre0; ++i, (++k == sk.KB ? (k = 0) : 0))
             tma_load_2d(base + i * TC_STAGE_BYTES + TC_A_BYTES, &mapX, k * TC_BK, 0, full_bar(i));
     }
-    if (warp == 1) {   // one warp allocates 64 TMEM columns: two accumulator buffers of 32
+    if (warp == 1) {   // this warp sets up the remaining barriers and allocates 64 TMEM columns: two accumulator buffers of 32
+        if (lane == 0) {
+            for (int s = 0; s < TC_STAGES; ++s) { if (s >= TC_PRE) mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
+            for (int b = 0; b < 2; ++b) { mbar_init(tfull_bar(b), 1); mbar_init(tempty_bar(b), 4); }
+            abort_sh = 0;
+            epi_abort_sh = 0;
+            asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        }
+        __syncwarp();
         asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&tmem_base_sh)), "r"(64));
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;");
     }
