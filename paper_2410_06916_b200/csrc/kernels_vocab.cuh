@@ -96,12 +96,37 @@ vocab_kernel(DevState* st, const float* __restrict__ part, int n_split, size_t s
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     float* lrow = logits + (size_t)r * vocab;
 
+    // Vocabularies of up to VOCAB_THREADS * VPT entries with a single slab (the tensor-core path) stay in
+    // registers: all of a thread's loads are in flight together and nothing is read back from memory for the
+    // second pass.  Same per-thread order of operations as the general loops.
+    constexpr int VPT = 32;
+    const bool in_regs = n_split == 1 && vocab <= VOCAB_THREADS * VPT;
+    float vr[VPT];
     ArgMax am{-INFINITY, 0x7FFFFFFF};
-    for (int i = tid; i < vocab; i += VOCAB_THREADS) {
-        float v = 0.f;
-        for (int s = 0; s < n_split; ++s) v += part[s * split_stride + (size_t)r * vocab + i];
-        lrow[i] = v;
-        am = better(am, ArgMax{v, i});
+    if (in_regs) {
+        const float* prow = part + (size_t)r * vocab;
+#pragma unroll
+        for (int k = 0; k < VPT; ++k) {
+            const int i = tid + k * VOCAB_THREADS;
+            vr[k] = i < vocab ? __ldcg(prow + i) : 0.f;
+        }
+#pragma unroll
+        for (int k = 0; k < VPT; ++k) {
+            const int i = tid + k * VOCAB_THREADS;
+            if (i < vocab) {
+                const float v = 0.f + vr[k];
+                vr[k] = v;
+                lrow[i] = v;
+                am = better(am, ArgMax{v, i});
+            }
+        }
+    } else {
+        for (int i = tid; i < vocab; i += VOCAB_THREADS) {
+            float v = 0.f;
+            for (int s = 0; s < n_split; ++s) v += part[s * split_stride + (size_t)r * vocab + i];
+            lrow[i] = v;
+            am = better(am, ArgMax{v, i});
+        }
     }
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) {
@@ -124,10 +149,21 @@ vocab_kernel(DevState* st, const float* __restrict__ part, int n_split, size_t s
     __syncthreads();
 
     float s1 = 0.f, sT = 0.f;
-    for (int i = tid; i < vocab; i += VOCAB_THREADS) {
-        const float dlt = lrow[i] - am.v;
-        s1 += expf(dlt);
-        sT += expf(dlt * inv_temp);
+    if (in_regs) {
+#pragma unroll
+        for (int k = 0; k < VPT; ++k) {
+            if (tid + k * VOCAB_THREADS < vocab) {
+                const float dlt = vr[k] - am.v;
+                s1 += expf(dlt);
+                sT += expf(dlt * inv_temp);
+            }
+        }
+    } else {
+        for (int i = tid; i < vocab; i += VOCAB_THREADS) {
+            const float dlt = lrow[i] - am.v;
+            s1 += expf(dlt);
+            sT += expf(dlt * inv_temp);
+        }
     }
     s1 = block_sum(s1, sh);
     sT = block_sum(sT, sh);
