@@ -123,6 +123,7 @@ __global__ void embed_fused_kernel(DevState* st, const int* __restrict__ toks, c
     }
     const T* src = embed + (size_t)tok * d;
     float ss = 0.f;
+#pragma unroll 4
     for (int i = threadIdx.x; i < d; i += blockDim.x) {
         const float v = to_float(src[i]);
         h[(size_t)r * d + i] = v;

@@ -226,7 +226,7 @@ __device__ __forceinline__ void tc_finalize(const EpiParams& ep, int pos0, float
 #pragma unroll
         for (int m = 0; m < ROWS; ++m) stage_sh[m * TC_TILE_N + l] = h_pre[m] + val[m];   // read back by this thread only
         float* sums_sh = stage_sh + ROWS * TC_TILE_N;
-#pragma unroll 1
+#pragma unroll 2                                       // two rows' shuffle chains in flight; still compact code
         for (int m = 0; m < n_rows; ++m) {
             float hn = 0.f;
             if (n < N) {

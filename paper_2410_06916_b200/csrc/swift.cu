@@ -493,7 +493,7 @@ swift_status forward_chunk_fused(swift_ctx* ctx, int rows, const int* toks_dev, 
         }
     };
 
-    CU(launch_k(embed_fused_kernel<T>, dim3(rows), dim3(256), 0, ctx, st, toks_dev, (const T*)wptr<T>(ctx, ctx->wl.embed), h,
+    CU(launch_k(embed_fused_kernel<T>, dim3(rows), dim3(1024), 0, ctx, st, toks_dev, (const T*)wptr<T>(ctx, ctx->wl.embed), h,
                 gain_of(0), xn_hl, sumsq, dm, d.vocab));
     const int d_tiles = ceil_div(dm, TC_TILE_N);
     for (size_t k = 0; k < kept.size(); ++k) {
