@@ -34,6 +34,7 @@ constexpr int TC_STAGES = 9;        // 144 KB of weight tiles in flight per SM: 
 constexpr int TC_THREADS = 192;
 constexpr int TC_A_BYTES = TC_TILE_N * TC_BK * 2;   // 16384
 constexpr int TC_B_BYTES = TC_COLS * TC_BK * 2;     // 4096
+constexpr int TC_NEXT_TILES = 2;     // tiles of the next GEMM each CTA prefetches into L2 at the end of its loads
 constexpr int TC_PRE = 1;           // tiles requested before the set-up barrier (see the producer's comment)
 constexpr int TC_STAGE_BYTES = TC_A_BYTES + TC_B_BYTES;
 constexpr int TC_SMEM_BYTES = TC_STAGES * TC_STAGE_BYTES + 1024 /*alignment slack*/ + 256 /*barriers*/;
@@ -183,6 +184,9 @@ struct EpiParams {
     KvLayout L;
     int block, n_heads, max_positions;
     const float2* rope_cs;
+    // any epilogue: shape of the GEMM that runs next on this stream (0 = none): each CTA asks for the first
+    // weight tiles it will need there to be brought into L2 while this launch drains
+    int next_N, next_K;
 };
 
 template <int EPI, typename TKV>
@@ -288,7 +292,7 @@ template <int EPI, typename TKV>
 __global__ void __launch_bounds__(TC_THREADS, 1)
 gemm_tc_kernel(DevState* st, const __grid_constant__ CUtensorMap mapW, const __grid_constant__ CUtensorMap mapX,
                float* __restrict__ Y, float* __restrict__ slabs, int* __restrict__ counters, int N, int K,
-               const __grid_constant__ EpiParams ep)
+               const __grid_constant__ EpiParams ep, const __grid_constant__ CUtensorMap mapNext)
 {
     pdl_trigger();
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -315,6 +319,9 @@ gemm_tc_kernel(DevState* st, const __grid_constant__ CUtensorMap mapW, const __g
     __shared__ float2 rope_sh[EPI == EPI_QKV ? ROWS * (TC_TILE_N / 2) : 1];   // (cos, sin) of the rows' positions
     __shared__ int page_sh[ROWS];                                              // KV page of each row's position
 
+    // The producer and the MMA warp need the row count before they can start; they read it here, ahead of the
+    // set-up barrier, so that the trip to L2 overlaps the rest of the set-up.
+    int n_rows_early = 0;
     if (tid == 0) {
         // This thread is the TMA producer.  It requests its first weight tiles right away, before the block-wide
         // set-up barrier and even before the wait for the preceding kernel (weights depend on nothing), then,
@@ -332,6 +339,7 @@ gemm_tc_kernel(DevState* st, const __grid_constant__ CUtensorMap mapW, const __g
             tma_load_2d(base + i * TC_STAGE_BYTES, &mapW, k * TC_BK, t * TC_TILE_N, full_bar(i));
         }
         pdl_wait();
+        n_rows_early = st->n_rows;
         for (int i = 0, k = kb0; i < n_pre0; ++i, (++k == sk.KB ? (k = 0) : 0))
             tma_load_2d(base + i * TC_STAGE_BYTES + TC_A_BYTES, &mapX, k * TC_BK, 0, full_bar(i));
     }
@@ -344,6 +352,8 @@ gemm_tc_kernel(DevState* st, const __grid_constant__ CUtensorMap mapW, const __g
             asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         }
         __syncwarp();
+        pdl_wait();
+        n_rows_early = st->n_rows;
         asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&tmem_base_sh)), "r"(64));
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;");
     }
@@ -356,7 +366,7 @@ gemm_tc_kernel(DevState* st, const __grid_constant__ CUtensorMap mapW, const __g
         // ---------------------------------------------------------------- TMA producer
         if (lane == 0) {
             const int n_pre = (int)((u_end - u_begin) < TC_PRE ? (u_end - u_begin) : TC_PRE);   // already requested above
-            if (st->n_rows == 0) {                      // nothing to compute: let the requested tiles land, then leave
+            if (n_rows_early == 0) {                    // nothing to compute: let the requested tiles land, then leave
                 for (int i = 0; i < n_pre; ++i) mbar_wait(full_bar(i), 0);
             } else {
             int it = n_pre;
@@ -370,13 +380,26 @@ gemm_tc_kernel(DevState* st, const __grid_constant__ CUtensorMap mapW, const __g
                 tma_load_2d(b_dst, &mapX, kb * TC_BK, 0, full_bar(s));
             }
             }
+            if (ep.next_K > 0) {                        // everything of this launch is requested: now the next one's start
+                StreamK nk;
+                nk.KB = (ep.next_K + TC_BK - 1) / TC_BK;
+                nk.U = (long long)((ep.next_N + TC_TILE_N - 1) / TC_TILE_N) * nk.KB;
+                nk.G = (int)(nk.U < (long long)gridDim.x ? nk.U : (long long)gridDim.x);
+                if ((int)blockIdx.x < nk.G) {
+                    const long long u0 = nk.start(blockIdx.x), u1 = nk.start(blockIdx.x + 1);
+                    int t = (int)(u0 / nk.KB), k = (int)(u0 - (long long)t * nk.KB);
+                    for (int i = 0; i < TC_NEXT_TILES && u0 + i < u1; ++i, (++k == nk.KB ? (k = 0, ++t) : 0))
+                        asm volatile("cp.async.bulk.prefetch.tensor.2d.L2.global [%0, {%1, %2}];"
+                                     ::"l"(&mapNext), "r"(k * TC_BK), "r"(t * TC_TILE_N) : "memory");
+                }
+            }
         } else {
             pdl_wait();
         }
     } else if (warp == 1) {
         // ---------------------------------------------------------------- MMA issuer
         pdl_wait();
-        if (lane == 0 && st->n_rows != 0) {
+        if (lane == 0 && n_rows_early != 0) {
             int it = 0, seg = 0;
             int kb = (int)(u_begin % sk.KB);
             for (long long u = u_begin; u < u_end; ++u, ++it, (++kb == sk.KB ? (kb = 0) : 0)) {

@@ -74,7 +74,7 @@ struct swift_ctx {
     std::string err;
     cudaEvent_t ev[8];
     // captured forwards; programmatic dependent launch between the kernels of a forward
-    bool use_graphs, use_pdl, fuse, fuse_combine;
+    bool use_graphs, use_pdl, fuse, fuse_combine, prefetch_next;
     int attn_rows_per_cta;
     std::vector<FwdGraph>* graphs;
     uint64_t graph_clock;
@@ -301,11 +301,12 @@ struct GemmSite {
 };
 
 template <int EPI, typename TKV>
-swift_status launch_gemm_tc(swift_ctx* ctx, const GemmSite& g, const EpiParams& ep)
+swift_status launch_gemm_tc(swift_ctx* ctx, const GemmSite& g, const EpiParams& ep, const CUtensorMap* next_map = nullptr)
 {
     if (ceil_div(g.N, TC_TILE_N) > TC_MAX_TILES) return fail(ctx, SWIFT_EUNSUPPORTED, "GEMM with %d output tiles", ceil_div(g.N, TC_TILE_N));
     CU(launch_k(gemm_tc_kernel<EPI, TKV>, dim3(TC_GRID), dim3(TC_THREADS), (size_t)TC_SMEM_BYTES, ctx, state_of(ctx), *g.mapW, *g.mapX,
-                kptr<float>(ctx, ctx->kl.part), kptr<float>(ctx, ctx->kl.slabs), kptr<int>(ctx, ctx->kl.counters), g.N, g.K, ep));
+                kptr<float>(ctx, ctx->kl.part), kptr<float>(ctx, ctx->kl.slabs), kptr<int>(ctx, ctx->kl.counters), g.N, g.K, ep,
+                next_map ? *next_map : *g.mapW));
     return SWIFT_OK;
 }
 
@@ -483,13 +484,36 @@ swift_status forward_chunk_fused(swift_ctx* ctx, int rows, const int* toks_dev, 
     base.sumsq_in = sumsq;
     int n_tiles_in = 1;                          // the embedding gather writes one "tile" of sums
 
-    auto gemm = [&](int epi, const CUtensorMap* mw, const CUtensorMap* mx, int N, int K, const EpiParams& ep) -> swift_status {
+    // the weight matrices in the order this forward streams them: each GEMM prefetches the start of the next one
+    struct NextW { const CUtensorMap* map; int N, K; };
+    std::vector<NextW> order;
+    for (int sl : kept) {
+        const int b = sl >> 1;
+        if (!(sl & 1)) {
+            order.push_back({&ctx->tm_wqkv[b], nqkv, dm});
+            order.push_back({&ctx->tm_wo[b], dm, qd});
+        } else {
+            order.push_back({&ctx->tm_wgu[b], 2 * d.ffn, dm});
+            order.push_back({&ctx->tm_wdown[b], dm, d.ffn});
+        }
+    }
+    if (head.run) order.push_back({&ctx->tm_lm_head, d.vocab, dm});
+    size_t gemm_index = 0;
+    auto gemm = [&](int epi, const CUtensorMap* mw, const CUtensorMap* mx, int N, int K, const EpiParams& ep_in) -> swift_status {
+        EpiParams ep = ep_in;
+        const CUtensorMap* next_map = nullptr;
+        ++gemm_index;
+        if (ctx->prefetch_next && gemm_index < order.size()) {
+            next_map = order[gemm_index].map;
+            ep.next_N = order[gemm_index].N;
+            ep.next_K = order[gemm_index].K;
+        }
         const GemmSite g{nullptr, N, K, nullptr, mw, mx};
         switch (epi) {
-        case EPI_QKV: return launch_gemm_tc<EPI_QKV, TKV>(ctx, g, ep);
-        case EPI_SWIGLU: return launch_gemm_tc<EPI_SWIGLU, float>(ctx, g, ep);
-        case EPI_RESID: return launch_gemm_tc<EPI_RESID, float>(ctx, g, ep);
-        default: return launch_gemm_tc<EPI_PLAIN, float>(ctx, g, ep);
+        case EPI_QKV: return launch_gemm_tc<EPI_QKV, TKV>(ctx, g, ep, next_map);
+        case EPI_SWIGLU: return launch_gemm_tc<EPI_SWIGLU, float>(ctx, g, ep, next_map);
+        case EPI_RESID: return launch_gemm_tc<EPI_RESID, float>(ctx, g, ep, next_map);
+        default: return launch_gemm_tc<EPI_PLAIN, float>(ctx, g, ep, next_map);
         }
     };
 
@@ -948,6 +972,7 @@ swift_status swift_load(const swift_model_desc* desc, swift_devbuf weights, swif
         c->attn_rows_per_cta = (v == 1 || v == 2 || v == 4 || v == 6 || v == 8 || v == 12) ? v : 16;
     }
     c->fuse_combine = getenv("SWIFT_NO_FUSE_COMBINE") == nullptr;
+    c->prefetch_next = getenv("SWIFT_NO_PREFETCH_NEXT") == nullptr;
     c->use_pdl = getenv("SWIFT_PDL") != nullptr;   // programmatic dependent launch: measured neutral to slightly negative on whole forwards, so opt-in
     c->fuse = getenv("SWIFT_NO_FUSE") == nullptr && desc->head_dim <= TC_TILE_N;
     c->graphs = new std::vector<FwdGraph>();
