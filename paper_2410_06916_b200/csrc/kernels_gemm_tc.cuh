@@ -34,7 +34,6 @@ constexpr int TC_STAGES = 9;        // 144 KB of weight tiles in flight per SM: 
 constexpr int TC_THREADS = 192;
 constexpr int TC_A_BYTES = TC_TILE_N * TC_BK * 2;   // 16384
 constexpr int TC_B_BYTES = TC_COLS * TC_BK * 2;     // 4096
-constexpr int TC_NEXT_TILES = 2;     // tiles of the next GEMM each CTA prefetches into L2 at the end of its loads
 constexpr int TC_PRE = 1;           // tiles requested before the set-up barrier (see the producer's comment)
 constexpr int TC_STAGE_BYTES = TC_A_BYTES + TC_B_BYTES;
 constexpr int TC_SMEM_BYTES = TC_STAGES * TC_STAGE_BYTES + 1024 /*alignment slack*/ + 256 /*barriers*/;
@@ -186,7 +185,7 @@ struct EpiParams {
     const float2* rope_cs;
     // any epilogue: shape of the GEMM that runs next on this stream (0 = none): each CTA asks for the first
     // weight tiles it will need there to be brought into L2 while this launch drains
-    int next_N, next_K;
+    int next_N, next_K, next_tiles;
 };
 
 template <int EPI, typename TKV>
@@ -388,7 +387,7 @@ gemm_tc_kernel(DevState* st, const __grid_constant__ CUtensorMap mapW, const __g
                 if ((int)blockIdx.x < nk.G) {
                     const long long u0 = nk.start(blockIdx.x), u1 = nk.start(blockIdx.x + 1);
                     int t = (int)(u0 / nk.KB), k = (int)(u0 - (long long)t * nk.KB);
-                    for (int i = 0; i < TC_NEXT_TILES && u0 + i < u1; ++i, (++k == nk.KB ? (k = 0, ++t) : 0))
+                    for (int i = 0; i < ep.next_tiles && u0 + i < u1; ++i, (++k == nk.KB ? (k = 0, ++t) : 0))
                         asm volatile("cp.async.bulk.prefetch.tensor.2d.L2.global [%0, {%1, %2}];"
                                      ::"l"(&mapNext), "r"(k * TC_BK), "r"(t * TC_TILE_N) : "memory");
                 }

@@ -75,7 +75,7 @@ struct swift_ctx {
     cudaEvent_t ev[8];
     // captured forwards; programmatic dependent launch between the kernels of a forward
     bool use_graphs, use_pdl, fuse, fuse_combine, prefetch_next;
-    int attn_rows_per_cta;
+    int attn_rows_per_cta, prefetch_tiles;
     std::vector<FwdGraph>* graphs;
     uint64_t graph_clock;
     // tensor-core GEMM path (bf16 models)
@@ -507,6 +507,7 @@ swift_status forward_chunk_fused(swift_ctx* ctx, int rows, const int* toks_dev, 
             next_map = order[gemm_index].map;
             ep.next_N = order[gemm_index].N;
             ep.next_K = order[gemm_index].K;
+            ep.next_tiles = ctx->prefetch_tiles;
         }
         const GemmSite g{nullptr, N, K, nullptr, mw, mx};
         switch (epi) {
@@ -973,6 +974,10 @@ swift_status swift_load(const swift_model_desc* desc, swift_devbuf weights, swif
     }
     c->fuse_combine = getenv("SWIFT_NO_FUSE_COMBINE") == nullptr;
     c->prefetch_next = getenv("SWIFT_NO_PREFETCH_NEXT") == nullptr;
+    {
+        const char* e = getenv("SWIFT_PREFETCH_TILES");      // 16 KB tiles of the next GEMM each CTA asks L2 for
+        c->prefetch_tiles = e ? std::max(0, std::min(256, atoi(e))) : 16;
+    }
     c->use_pdl = getenv("SWIFT_PDL") != nullptr;   // programmatic dependent launch: measured neutral to slightly negative on whole forwards, so opt-in
     c->fuse = getenv("SWIFT_NO_FUSE") == nullptr && desc->head_dim <= TC_TILE_N;
     c->graphs = new std::vector<FwdGraph>();
