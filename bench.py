@@ -282,7 +282,7 @@ def main():
     achieved = g_bytes / (g_ms * 1e-3) * 1e-9
     # DRAM bytes per launch of that kernel from the ncu capture summarised in profiles/gemm_tc_7b_gate_up_9rows.md
     # (7B widths, 9 rows); other shapes have no capture of their own
-    traffic = 186.2e6 if (cfg.name == "7b" and run.max_draft == 8) else None
+    traffic = 185.9e6 if (cfg.name == "7b" and run.max_draft == 8) else None
     roofline = {"bound": "hbm", "kernel": "skinny GEMM, fused gate/up projection, %d rows" % (run.max_draft + 1),
                 "achieved": achieved, "peak": hbm_peak, "peak_kind": f"{peak_kind} copy bandwidth (burst)", "unit": "GB/s",
                 "frac": achieved / hbm_peak, "traffic": traffic, "bytes_per_launch": g_bytes, "ms_per_launch": g_ms,
