@@ -1,7 +1,10 @@
 // GQA decode attention over the paged KV cache for the <= 16 new rows of one forward chunk, with
-// the causal mask across those rows.  Split-KV: each CTA owns one (query head, 256-position chunk);
-// chunks are anchored at multiples of 256 positions and combined in chunk order, so a row's result
-// does not depend on how many other rows are in flight.
+// the causal mask across those rows.  Split-KV: each CTA owns one (query head, 64-position chunk);
+// chunks are anchored at multiples of 64 positions and merged in chunk order, so a row's result
+// does not depend on how many other rows are in flight.  Two split kernels: attn_stream_kernel
+// (head_dim 128: K and V go straight from the cache into registers) and attn_split_kernel (any
+// head size, K and V staged in shared memory); the merge is attn_combine_kernel, or the tail of
+// attn_stream_kernel itself for one-row forwards.
 #pragma once
 #include "common.cuh"
 #include "kernels_gemm_tc.cuh"

@@ -13,7 +13,15 @@
 // number of bytes whatever N and K are.  A CTA whose range covers only part of a tile writes its
 // partial accumulator to a slab; the last CTA to finish a tile (per-tile arrival counter) adds the
 // slabs in slab order and writes Y, which makes the result independent of arrival order and of the
-// row count.
+// row count.  A CTA that finds all the other segments of its tile already arrived skips its own slab
+// and arrival and adds the others' slabs, fetched early, to its registers in the same order.
+//
+// What surrounds the stream matters as much as the stream at these sizes (tens of microseconds per
+// launch): one weight tile is requested before the set-up barrier and the rest from the producer
+// loop (a full ring from every CTA at once delayed the first tile by 3 us); per-row epilogue loops
+// are rolled over the rows that exist (the last tile's epilogue runs once, from cold instruction
+// caches); and once a CTA has requested all of its own tiles it asks L2 for the first tiles it
+// will stream in the GEMM that follows, which fills the idle HBM time around the kernel boundary.
 //
 // Pipeline per CTA: warp 0 issues TMA loads (weights 128x64 + activations 32x64 per stage, 128-byte
 // swizzle) into a 9-stage shared-memory ring guarded by mbarriers; warp 1 issues tcgen05.mma from
