@@ -423,6 +423,42 @@ def test_cache_fills_to_capacity(small_cfg):
         g.close()
 
 
+def test_launch_options_do_not_change_results(monkeypatch):
+    """The measurement switches read at load time (captured graphs or direct launches, the attention merge fused
+    into one-row launches or not, attention rows grouped over more CTAs, the L2 prefetch of the next GEMM's tiles,
+    programmatic dependent launch) choose how the same arithmetic is launched: logits and generated tokens must be
+    identical bit for bit, at 7B widths (head size 128, the tensor-core path)."""
+    from paper_2410_06916_b200 import GenParams, SwiftModel
+    cfg = synth.MODELS["7b"].with_blocks(2, n_planted=1)
+    toks = synth.prompt(cfg, 210)
+    z = synth.block_mask(cfg, [1])
+
+    def run(env):
+        for k, v in env.items():
+            monkeypatch.setenv(k, v)
+        m = SwiftModel(cfg, max_positions=320, max_draft=8)
+        try:
+            m.load_weights(synth.iter_tensors(cfg))
+            m.prefill(toks[:200])
+            nine, _ = m.forward_rows(toks[200:209], 200, None, write_kv=False)
+            one, _ = m.forward_rows(toks[200:201], 200, z, write_kv=False)
+            van, _, _ = m.generate(toks[:200], GenParams(max_new=20, vanilla=True))
+            sw, st, _ = m.generate(toks[:200], GenParams(max_new=20, max_draft=8, skip_mask=z))
+        finally:
+            m.close()
+            for k in env:
+                monkeypatch.delenv(k)
+        return nine, one, van, sw
+
+    base = run({})
+    assert base[2] == base[3]                                    # lossless on the GPU
+    for env in ({"SWIFT_NO_GRAPHS": "1"}, {"SWIFT_NO_FUSE_COMBINE": "1"}, {"SWIFT_ATTN_ROWS": "4"},
+                {"SWIFT_PREFETCH_TILES": "0"}, {"SWIFT_PREFETCH_TILES": "64"}, {"SWIFT_PDL": "1"}):
+        got = run(env)
+        assert np.array_equal(got[0], base[0]) and np.array_equal(got[1], base[1]), env
+        assert got[2] == base[2] and got[3] == base[3], env
+
+
 @pytest.mark.slow
 def test_full_depth_7b_against_oracle_and_losslessness():
     """Config 2 at full size (32 blocks, 13 GB of weights), in the launch configuration the benchmark times:
