@@ -570,7 +570,19 @@ gemm_tc_kernel(DevState* st, const __grid_constant__ CUtensorMap mapW, const __g
                 if (last_flag_sh) {                             // last arrival: add the slabs in slab order
 #pragma unroll
                     for (int m = 0; m < ROWS; ++m) val[m] = 0.f;
-                    if (n < N) {
+                    if (n < N && n_rows == 1) {                 // one row: eight slabs' loads in flight at a time
+                        float a = 0.f;
+                        for (int j0 = 0; j0 < nseg; j0 += 8) {
+                            float t8[8];
+#pragma unroll
+                            for (int jj = 0; jj < 8; ++jj)
+                                t8[jj] = j0 + jj < nseg ? __ldcg(slabs + (size_t)(j0 + jj) * ROWS * N + n) : 0.f;
+#pragma unroll
+                            for (int jj = 0; jj < 8; ++jj)
+                                if (j0 + jj < nseg) a += t8[jj];
+                        }
+                        val[0] = a;
+                    } else if (n < N) {
                         for (int j0 = 0; j0 < nseg; j0 += 2) {      // two slabs' loads in flight at a time
 #pragma unroll
                             for (int jj = 0; jj < 2; ++jj)
