@@ -259,14 +259,28 @@ def main():
     value, dec_ms, tot_ms, wall = aggregate_replicas(tokens, dec_ms, tot_ms, wall, world, device="cuda")
     e2e = world * sum(s.tokens for s in stats) / wall
 
+    def dist_of(ms, nbytes, keep):
+        """min / median / max over rounds of the achieved fraction of the HBM roofline (first round left out: warm-up)."""
+        f = [b / (t * 1e-3) * 1e-9 / hbm_peak for t, b, k in list(zip(ms, nbytes, keep))[1:] if k and t > 0]
+        if not f:
+            return None
+        return {"min": min(f), "p50": statistics.median(f), "max": max(f), "rounds": len(f)}
+
     # vanilla decoding of the same model for the comparison the metric names
     swift_tokens = model.generate(prompt, gp)[0]
+    md, mv, bd, bv, kd = model.round_times()
+    fdist = {"draft_frac": dist_of(md, bd, kd > 0), "verify_frac": dist_of(mv, bv, kd == run.max_draft)}
+    # expected speedup of Eq. 5 (Appendix B.3) with the measured cost ratio c = one draft forward / one verification
+    full = kd == run.max_draft
+    c_meas = float(np.median(md[full] / kd[full]) / np.median(mv[full])) if full.any() and run.max_draft > 0 else None
     model.generate(prompt[:64], GenParams(max_new=8, vanilla=True))
     if sampling:
         model.set_sampling(False)
     v_tokens, vst, _ = model.generate(prompt, GenParams(max_new=max_new, vanilla=True))
     vanilla = (vst.tokens - 1) / (vst.ms_decode * 1e-3)
     lossless = None if sampling else (swift_tokens == v_tokens)   # greedy SWIFT must reproduce vanilla decoding
+    _, vmv, _, vbv, _ = model.round_times()
+    fdist["vanilla_frac"] = dist_of(vmv, vbv, np.ones(len(vmv), dtype=bool))
 
     s0 = stats[-1]
     n_ctx = run.prompt_len + max_new // 2
@@ -280,9 +294,9 @@ def main():
     g_ms, g_bytes = model.time_gemm(2, run.max_draft + 1, 200)
     g1_ms, _ = model.time_gemm(2, 1, 200)
     achieved = g_bytes / (g_ms * 1e-3) * 1e-9
-    # DRAM bytes per launch of that kernel from the ncu capture summarised in profiles/gemm_tc_7b_gate_up_9rows.md
-    # (7B widths, 9 rows); other shapes have no capture of their own
-    traffic = 185.9e6 if (cfg.name == "7b" and run.max_draft == 8) else None
+    # DRAM bytes per launch of that kernel (read + write, mean of two launches) from the ncu captures summarised in
+    # profiles/gemm_tc_gate_up_9rows.md (7B and 13B widths, 9 rows); other shapes have no capture of their own
+    traffic = {"7b": 186.6e6, "13b": 289.6e6}.get(cfg.name) if run.max_draft == 8 else None
     roofline = {"bound": "hbm", "kernel": "skinny GEMM, fused gate/up projection, %d rows" % (run.max_draft + 1),
                 "achieved": achieved, "peak": hbm_peak, "peak_kind": f"{peak_kind} copy bandwidth (burst)", "unit": "GB/s",
                 "frac": achieved / hbm_peak, "traffic": traffic, "bytes_per_launch": g_bytes, "ms_per_launch": g_ms,
@@ -295,9 +309,14 @@ def main():
                       "e2e_note": "whole swift_generate call incl. prefill and host copies, host clock", "context": PAPER_CONTEXT},
            "vanilla_tokens_per_s": vanilla, "swift_equals_vanilla": lossless, "speedup_vs_vanilla": value / world / vanilla,
            "M": (s0.tokens - 1) / s0.rounds, "alpha": s0.accepted / max(s0.drafted, 1), "rounds": s0.rounds,
-           "ms_prefill": s0.ms_prefill, "forwards": fw, "roofline": roofline,
+           "ms_prefill": s0.ms_prefill, "forwards": fw, "forwards_per_round": fdist, "roofline": roofline,
            "e2e": {"value": e2e, "unit": UNIT, "h2d_bytes_per_step": 4 * run.prompt_len, "d2h_bytes_per_step": 448 * (s0.rounds + 1)},
            "gpu_launches": launches, "clocks": clk.summary()}
+
+    if c_meas is not None:
+        M_, a_ = out["M"], out["alpha"]
+        out["eq5"] = {"c_measured": c_meas, "expected_speedup": M_ * a_ / ((M_ - 1) * c_meas + a_) if a_ > 0 else None,
+                      "achieved_speedup": out["speedup_vs_vanilla"]}
 
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
         small = cfg if weights is not None and cfg.n_blocks * cfg.block_params() < 16e9 else cfg.with_blocks(8)

@@ -202,6 +202,15 @@ int32_t swift_committed_length(const swift_ctx* ctx);               /* n; -1 if 
 int64_t swift_launch_count(const swift_ctx* ctx);                   /* kernels enqueued since load */
 double swift_forward_bytes(const swift_ctx* ctx, const uint8_t* skip_mask_host, int32_t n_rows,
                            int32_t n_context); /* algorithmic HBM bytes of one forward */
+/* Per-round record of the last swift_generate on this context, for judging every forward and not only their sum
+ * (the drafting stage dominates latency, paper Section 5.3; the metrics M and alpha are per round, Appendix B.3).
+ * Round i (a vanilla step counts as a round with no drafts): CUDA-event time on the stream of its drafting phase
+ * (all `drafted[i]` draft forwards together) and of its verification (the full-model forward plus the accept
+ * step), and the algorithmic HBM bytes of those forwards.  Host arrays of `capacity` entries, any of them may be
+ * NULL; returns the number of rounds recorded (which may exceed capacity; only `capacity` entries are written),
+ * -1 if ctx is NULL. */
+int32_t swift_round_times(const swift_ctx* ctx, int32_t capacity, float* ms_draft_host, float* ms_verify_host,
+                          double* bytes_draft_host, double* bytes_verify_host, int32_t* drafted_host);
 /* Times `iters` back-to-back launches of one weight-streaming GEMM of the walk (which: 0 fused QKV,
  * 1 o_proj, 2 fused gate/up, 3 down, 4 output head) with n_rows rows, cycling over the blocks' weights
  * so that successive launches read different memory.  Outputs the average CUDA-event time per launch

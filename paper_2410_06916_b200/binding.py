@@ -52,7 +52,7 @@ class _Stats(C.Structure):
 SYMBOLS = ("swift_weights_bytes", "swift_kv_bytes", "swift_workspace_bytes", "swift_load", "swift_free",
            "swift_last_error", "swift_pack_tensor", "swift_set_sampling", "swift_forward_rows", "swift_prefill",
            "swift_set_pending", "swift_draft", "swift_verify", "swift_accept", "swift_score_skipsets", "swift_generate",
-           "swift_committed_length", "swift_launch_count", "swift_forward_bytes", "swift_read_kv", "swift_time_gemm", "swift_set_gemm_impl", "swift_gemm", "swift_gemm_static",
+           "swift_committed_length", "swift_launch_count", "swift_round_times", "swift_forward_bytes", "swift_read_kv", "swift_time_gemm", "swift_set_gemm_impl", "swift_gemm", "swift_gemm_static",
            "swift_gemm_static_error")
 
 _lib = None
@@ -86,6 +86,8 @@ def load_library(path: Optional[str] = None) -> C.CDLL:
     lib.swift_committed_length.argtypes = [vp]
     lib.swift_launch_count.argtypes = [vp]
     lib.swift_launch_count.restype = C.c_int64
+    lib.swift_round_times.argtypes = [vp, i32, vp, vp, vp, vp, vp]
+    lib.swift_round_times.restype = C.c_int32
     lib.swift_forward_bytes.argtypes = [vp, vp, i32, i32]
     lib.swift_forward_bytes.restype = C.c_double
     lib.swift_set_gemm_impl.argtypes = [vp, i32]
@@ -321,6 +323,15 @@ class SwiftModel:
                                                  _ptr(trace), C.byref(st)))
         stats = GenStats(**{f: getattr(st, f) for f in GenStats.__dataclass_fields__})
         return out[:n_out.value].tolist(), stats, trace[:stats.rounds]
+
+    def round_times(self):
+        """Per round of the last generate(): (ms_draft, ms_verify, bytes_draft, bytes_verify, drafted) arrays."""
+        n = self._lib.swift_round_times(self.ctx, 0, None, None, None, None, None)
+        md, mv = np.zeros(n, dtype=np.float32), np.zeros(n, dtype=np.float32)
+        bd, bv = np.zeros(n, dtype=np.float64), np.zeros(n, dtype=np.float64)
+        k = np.zeros(n, dtype=np.int32)
+        self._lib.swift_round_times(self.ctx, n, _ptr(md), _ptr(mv), _ptr(bd), _ptr(bv), _ptr(k))
+        return md, mv, bd, bv, k
 
     def set_gemm_impl(self, tensor_cores: bool):
         self._check(self._lib.swift_set_gemm_impl(self.ctx, 1 if tensor_cores else 0))

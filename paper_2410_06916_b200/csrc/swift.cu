@@ -78,6 +78,9 @@ struct swift_ctx {
     int attn_rows_per_cta, prefetch_tiles;
     std::vector<FwdGraph>* graphs;
     uint64_t graph_clock;
+    // per-round record of the last swift_generate (swift_round_times)
+    struct RoundTime { float ms_draft, ms_verify; double bytes_draft, bytes_verify; int32_t drafted; };
+    std::vector<RoundTime> round_times;
     // tensor-core GEMM path (bf16 models)
     bool use_tc;
     std::vector<CUtensorMap> tm_wqkv, tm_wo, tm_wgu, tm_wdown;
@@ -1259,6 +1262,21 @@ swift_status swift_set_gemm_impl(swift_ctx* ctx, int32_t impl)
 
 int32_t swift_committed_length(const swift_ctx* ctx) { return ctx ? ctx->n : -1; }
 int64_t swift_launch_count(const swift_ctx* ctx) { return ctx ? ctx->launches : -1; }
+int32_t swift_round_times(const swift_ctx* ctx, int32_t capacity, float* ms_draft, float* ms_verify, double* bytes_draft,
+                          double* bytes_verify, int32_t* drafted)
+{
+    if (!ctx) return -1;
+    const int n = (int)ctx->round_times.size();
+    for (int i = 0; i < n && i < capacity; ++i) {
+        const auto& r = ctx->round_times[i];
+        if (ms_draft) ms_draft[i] = r.ms_draft;
+        if (ms_verify) ms_verify[i] = r.ms_verify;
+        if (bytes_draft) bytes_draft[i] = r.bytes_draft;
+        if (bytes_verify) bytes_verify[i] = r.bytes_verify;
+        if (drafted) drafted[i] = r.drafted;
+    }
+    return n;
+}
 double swift_forward_bytes(const swift_ctx* ctx, const uint8_t* skip, int32_t n_rows, int32_t n_context)
 {
     return ctx ? forward_bytes(ctx, skip, n_rows, n_context) : 0.0;
@@ -1372,6 +1390,7 @@ swift_status swift_generate(swift_ctx* ctx, const swift_gen_params* gp, const in
     memset(&stt, 0, sizeof stt);
     stt.best_matchness = -1.f;
     cudaEvent_t* ev = ctx->ev;
+    ctx->round_times.clear();
 
     CU(cudaEventRecord(ev[0], ctx->stream));
     int first = 0;
@@ -1391,6 +1410,7 @@ swift_status swift_generate(swift_ctx* ctx, const swift_gen_params* gp, const in
         if (gp->vanilla) {
             ctx->round++;
             launch_begin_round(ctx, 0.f);
+            CU(cudaEventRecord(ev[5], ctx->stream));
             ST(enqueue_verify(ctx, 1, 0));
             if (ctx->mode == SWIFT_SAMPLING) {
                 sample_row_kernel<<<1, VOCAB_THREADS, 0, ctx->stream>>>(state_of(ctx), kptr<float>(ctx, ctx->kl.logits), d.vocab, 0,
@@ -1401,9 +1421,15 @@ swift_status swift_generate(swift_ctx* ctx, const swift_gen_params* gp, const in
                 ST(enqueue_accept(ctx));
                 ctx->mode = save;
             }
+            CU(cudaEventRecord(ev[6], ctx->stream));
             ST(read_state(ctx, &hs));
             hs.n_accepted = 0;
-            stt.bytes_verify += forward_bytes(ctx, nullptr, 1, n_start);
+            float mv = 0.f;
+            CU(cudaEventElapsedTime(&mv, ev[5], ev[6]));
+            const double bv = forward_bytes(ctx, nullptr, 1, n_start);
+            stt.ms_verify += mv;
+            stt.bytes_verify += bv;
+            ctx->round_times.push_back({0.f, mv, 0.0, bv, 0});
         } else {
             if (optimising && count >= gp->gamma) {
                 CU(cudaEventRecord(ev[2], ctx->stream));
@@ -1438,8 +1464,12 @@ swift_status swift_generate(swift_ctx* ctx, const swift_gen_params* gp, const in
             CU(cudaEventElapsedTime(&md, ev[4], ev[5]));
             CU(cudaEventElapsedTime(&mv, ev[5], ev[6]));
             stt.ms_draft += md; stt.ms_verify += mv;
-            for (int j = 0; j < hs.n_drafted; ++j) stt.bytes_draft += forward_bytes(ctx, z.data(), 1, n_start + j);
-            stt.bytes_verify += forward_bytes(ctx, nullptr, hs.n_drafted + 1, n_start);
+            double bd = 0.0;
+            for (int j = 0; j < hs.n_drafted; ++j) bd += forward_bytes(ctx, z.data(), 1, n_start + j);
+            const double bv = forward_bytes(ctx, nullptr, hs.n_drafted + 1, n_start);
+            stt.bytes_draft += bd;
+            stt.bytes_verify += bv;
+            ctx->round_times.push_back({md, mv, bd, bv, hs.n_drafted});
             stt.drafted += hs.n_drafted;
             stt.accepted += hs.n_accepted;
         }

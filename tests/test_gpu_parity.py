@@ -219,6 +219,27 @@ def test_config1_generate_matches_oracle(tiny_pair):
         assert st.accepted == o_stats["accepted"] and st.drafted == o_stats["drafted"]
 
 
+def test_round_times_cover_every_round(tiny_pair):
+    """swift_round_times: one record per round of the last generate, consistent with its trace and its totals."""
+    _, g = tiny_pair
+    from paper_2410_06916_b200 import GenParams
+    prompt = synth.prompt(TINY, 32)
+    z = synth.block_mask(TINY, synth.planted_blocks(TINY))
+    _, st, trace = g.generate(prompt, GenParams(max_new=40, max_draft=4, skip_mask=z))
+    md, mv, bd, bv, k = g.round_times()
+    assert len(md) == st.rounds and [int(t[1]) for t in trace] == k.tolist()
+    assert (mv > 0).all() and (md[k > 0] > 0).all()
+    assert abs(md.sum() - st.ms_draft) < 1e-3 * st.ms_draft + 1e-4 and abs(mv.sum() - st.ms_verify) < 1e-3 * st.ms_verify + 1e-4
+    assert abs(bd.sum() - st.bytes_draft) < 1e-6 * st.bytes_draft and abs(bv.sum() - st.bytes_verify) < 1e-6 * st.bytes_verify
+    for i in (0, len(k) - 1):                               # bytes of a round = its forwards' algorithmic bytes
+        n0, ki = int(trace[i][0]), int(k[i])
+        assert bv[i] == g.forward_bytes(None, ki + 1, n0)
+        assert bd[i] == sum(g.forward_bytes(z, 1, n0 + j) for j in range(ki))
+    _, vst, _ = g.generate(prompt, GenParams(max_new=9, vanilla=True))
+    md, mv, bd, bv, k = g.round_times()
+    assert len(mv) == vst.rounds == 8 and (k == 0).all() and (md == 0).all() and (mv > 0).all()
+
+
 def test_gpu_swift_equals_gpu_vanilla_bf16(bf16_pair):
     _, g = bf16_pair
     from paper_2410_06916_b200 import GenParams
