@@ -313,6 +313,15 @@ def main():
            "e2e": {"value": e2e, "unit": UNIT, "h2d_bytes_per_step": 4 * run.prompt_len, "d2h_bytes_per_step": 448 * (s0.rounds + 1)},
            "gpu_launches": launches, "clocks": clk.summary()}
 
+    if run.optimise and s0.opt_rounds > 0:
+        # candidate scoring (Eq. 2-3): every candidate is two 16-row forwards under its own skip set over the gamma context
+        # tokens; bytes = the algorithmic bytes of those forwards at the context length where scoring starts
+        sc_bytes = sum(2 * model.forward_bytes(cands[r][c], 16, run.prompt_len + run.gamma)
+                       for r in range(s0.opt_rounds) for c in range(cands.shape[1]))
+        sc_gbs = sc_bytes / (s0.ms_score * 1e-3) * 1e-9
+        out["scoring"] = {"opt_rounds": s0.opt_rounds, "candidates_per_round": int(cands.shape[1]), "gamma": run.gamma,
+                          "ms_per_round": s0.ms_score / s0.opt_rounds, "best_matchness": s0.best_matchness,
+                          "gbs": sc_gbs, "frac": sc_gbs / hbm_peak, "share_of_decode": s0.ms_score / s0.ms_decode}
     if c_meas is not None:
         M_, a_ = out["M"], out["alpha"]
         out["eq5"] = {"c_measured": c_meas, "expected_speedup": M_ * a_ / ((M_ - 1) * c_meas + a_) if a_ > 0 else None,

@@ -31,6 +31,33 @@ def make_pair(cfg, max_positions=256, page_size=16, max_draft=15, oracle_dtype=N
     return o, gpu
 
 
+class LazyBlocks:
+    """Per-block weights generated from the seed when a block is asked for and dropped afterwards, so that the
+    oracle can walk a model whose widened weights would not fit host memory (its forward takes each block once)."""
+
+    def __init__(self, cfg):
+        self.cfg = cfg
+        self.planted = set(synth.planted_blocks(cfg))
+
+    def __len__(self):
+        return self.cfg.n_blocks
+
+    def __getitem__(self, b):
+        return {name: synth.make_tensor(self.cfg, name, b, planted=b in self.planted) for name in synth._BLOCK_TENSORS}
+
+
+def make_streamed_pair(cfg, max_positions=256, page_size=16, max_draft=15, kv_dtype="f32"):
+    """(oracle, gpu model) over identical synthetic weights, neither side holding a host copy of the blocks:
+    the GPU is filled tensor by tensor, the oracle regenerates a block whenever its forward reaches it."""
+    from paper_2410_06916_b200 import SwiftModel
+    gpu = SwiftModel(cfg, max_positions=max_positions, page_size=page_size, max_draft=max_draft, kv_dtype=kv_dtype)
+    gpu.load_weights(synth.iter_tensors(cfg))
+    w = {name: synth.make_tensor(cfg, name) for name in ("embed", "lm_head", "final_norm")}
+    w["blocks"] = LazyBlocks(cfg)
+    o = so.Oracle(so.Shape.of(cfg), w, dtype=torch.float32, max_positions=max_positions)
+    return o, gpu
+
+
 def logit_err(got: np.ndarray, ref: torch.Tensor) -> float:
     """max over rows of max|got - ref| / std(ref row)."""
     ref = ref.to(torch.float64).numpy()

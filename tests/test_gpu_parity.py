@@ -8,7 +8,8 @@ import torch
 
 import synth
 from oracle import swift_oracle as so
-from tests.helpers import LOGIT_TOL, MARGIN, compare_free_running, logit_err, make_pair, resync, walk_rounds
+from tests.helpers import (LOGIT_TOL, MARGIN, compare_free_running, logit_err, make_pair, make_streamed_pair, resync,
+                           walk_rounds)
 
 pytestmark = pytest.mark.gpu
 
@@ -480,30 +481,54 @@ def test_launch_options_do_not_change_results(monkeypatch):
         assert got[2] == base[2] and got[3] == base[3], env
 
 
+FULL_DEPTH = [("7b", 14, 8, 48, 64), ("13b", 18, 8, 48, 48), ("70b", 36, 12, 29, 48)]
+
+
 @pytest.mark.slow
-def test_full_depth_7b_against_oracle_and_losslessness():
-    """Config 2 at full size (32 blocks, 13 GB of weights), in the launch configuration the benchmark times:
-    teacher-forced logits of the last prompt rows against the oracle, then SWIFT == vanilla on the GPU."""
+@pytest.mark.parametrize("name,n_skip,max_draft,n_prompt,need_gb", FULL_DEPTH, ids=[c[0] for c in FULL_DEPTH])
+def test_full_depth_against_oracle_and_losslessness(name, n_skip, max_draft, n_prompt, need_gb):
+    """Configs 2, 3/4 and 5 at full size (32 / 40 / 80 blocks; 13 / 26 / 138 GB of weights), in the launch
+    configurations the benchmark times: teacher-forced logits of the last prompt rows against the oracle, from
+    16-row chunks, from one verification-shaped forward (max_draft + 1 rows) and from a one-row forward; then
+    SWIFT == vanilla on the GPU.  The oracle regenerates each block from the seed as its forward reaches it, so
+    no widened copy of the weights is held.  The 70B case takes a minute or two (two passes over 138 GB of
+    generated weights); SWIFT_SKIP_70B=1 leaves it out."""
+    import os
     import psutil
-    if psutil.virtual_memory().available < 64 * 2 ** 30:
-        pytest.skip("needs 64 GB of host memory for the oracle's fp32 copy of the weights")
+    if name == "70b" and os.environ.get("SWIFT_SKIP_70B"):
+        pytest.skip("SWIFT_SKIP_70B is set")
+    if psutil.virtual_memory().available < need_gb * 2 ** 30:
+        pytest.skip(f"needs {need_gb} GB of host memory")
+    import gc
+    gc.collect()
+    torch.cuda.empty_cache()                                    # buffers of the earlier tests' models
+    if name == "70b" and torch.cuda.mem_get_info()[0] < 150 * 2 ** 30:
+        pytest.skip("needs 150 GB of free device memory")
     from paper_2410_06916_b200 import GenParams
-    cfg = synth.MODELS["7b"]
-    o, g = make_pair(cfg, max_positions=256, max_draft=8)
+    cfg = synth.MODELS[name]
+    o, g = make_streamed_pair(cfg, max_positions=256, max_draft=max_draft)
     try:
-        prompt = synth.prompt(cfg, 48)
+        prompt = synth.prompt(cfg, n_prompt)
         ref = o.forward_rows(prompt, 0)
         g.prefill(prompt[:1])
         got, am = g.forward_rows(prompt, 0)
-        err = logit_err(got[-8:], ref[-8:])
-        print(f"7B full depth: teacher-forced logits off by {err:.2e} sigma")
+        rows = max_draft + 1
+        err = logit_err(got[-rows:], ref[-rows:])
+        print(f"{name} full depth: teacher-forced logits off by {err:.2e} sigma")
         assert err < LOGIT_TOL
-        for i in range(40, 48):
+        for i in range(n_prompt - rows, n_prompt):
             if so.top2_margin(ref[i]) > MARGIN:
                 assert int(am[i]) == so.argmax_lowest(ref[i])
-        z = synth.block_mask(cfg, synth.draft_blocks(cfg, 14))
-        van, _, _ = g.generate(prompt, GenParams(max_new=48, vanilla=True))
-        out, st, _ = g.generate(prompt, GenParams(max_new=48, max_draft=8, skip_mask=z))
+        # the same rows as one verification-shaped forward and the last one as a one-row forward
+        g.prefill(prompt[:-1])
+        ver, _ = g.forward_rows(prompt[-rows:], n_prompt - rows, None, write_kv=False)
+        one, _ = g.forward_rows(prompt[-1:], n_prompt - 1, None, write_kv=False)
+        assert logit_err(ver, ref[-rows:]) < LOGIT_TOL and logit_err(one, ref[-1:]) < LOGIT_TOL
+        assert np.array_equal(ver, got[-rows:]) and np.array_equal(one[0], got[-1])   # row-count invariance
+        z = synth.block_mask(cfg, synth.draft_blocks(cfg, n_skip))
+        n_new = 2 * (max_draft + 1) + 6
+        van, _, _ = g.generate(prompt, GenParams(max_new=n_new, vanilla=True))
+        out, st, _ = g.generate(prompt, GenParams(max_new=n_new, max_draft=max_draft, skip_mask=z))
         assert out == van and st.accepted > 0
     finally:
         g.close()
