@@ -43,7 +43,17 @@ class LazyBlocks:
         return self.cfg.n_blocks
 
     def __getitem__(self, b):
-        return {name: synth.make_tensor(self.cfg, name, b, planted=b in self.planted) for name in synth._BLOCK_TENSORS}
+        return _LazyBlock(self.cfg, b, b in self.planted)
+
+
+class _LazyBlock:
+    """One block's tensors, each generated when it is asked for (a skipped sub-layer's weights never are)."""
+
+    def __init__(self, cfg, b, planted):
+        self.cfg, self.b, self.planted = cfg, b, planted
+
+    def __getitem__(self, name):
+        return synth.make_tensor(self.cfg, name, self.b, planted=self.planted)
 
 
 def make_streamed_pair(cfg, max_positions=256, page_size=16, max_draft=15, kv_dtype="f32"):

@@ -532,3 +532,41 @@ def test_full_depth_against_oracle_and_losslessness(name, n_skip, max_draft, n_p
         assert out == van and st.accepted > 0
     finally:
         g.close()
+
+
+@pytest.mark.slow
+def test_full_depth_13b_scoring_and_rounds():
+    """Configs 3 and 4 at full size (40 blocks, 26 GB of weights): candidate scoring on 32 context tokens (Eq. 2-3),
+    one greedy round with the planted skip set and one speculative-sampling round with 20 blocks skipped, each step
+    compared with the oracle (which regenerates the weights it needs from the seed)."""
+    import psutil
+    if psutil.virtual_memory().available < 48 * 2 ** 30:
+        pytest.skip("needs 48 GB of host memory")
+    cfg = synth.MODELS["13b"]
+    o, g = make_streamed_pair(cfg, max_positions=256, max_draft=8)
+    try:
+        prompt = synth.prompt(cfg, 40)
+        o.prefill(prompt)
+        g.prefill(prompt)
+        g.set_pending(o.tokens[-1])
+        z18 = synth.block_mask(cfg, synth.draft_blocks(cfg, 18))
+        masks = np.stack([z18, np.zeros_like(z18), synth.candidate_masks(cfg, 18, 1, 0)[0]])
+        ref, _ = o.score_skipsets(masks.tolist(), 32)
+        got = g.score_skipsets(masks, 32)
+        # (the window here is prompt text, not the model's own output, so even the empty set scores low: the point
+        # is that both sides count the same matches)
+        for c in range(len(masks)):
+            if got[c] != pytest.approx(ref[c]):
+                rows = o.forward_rows(o.tokens[o.n - 32:o.n], o.n - 32, masks[c].tolist(), write_kv=False)
+                assert min(so.top2_margin(r) for r in rows) <= MARGIN, (c, got[c], ref[c])
+        st = walk_rounds(o, g, list(z18), n_rounds=1, max_k=4)
+        assert st["max_logit_err"] < LOGIT_TOL and st["rounds"] + st["resyncs"] == 1, st
+        seed = 4
+        g.set_sampling(True, 1.0, seed)
+        resync(g, o, 1)
+        z20 = list(synth.block_mask(cfg, synth.draft_blocks(cfg, 20)))
+        st = walk_rounds(o, g, z20, n_rounds=1, max_k=3, sampling=True, seed=seed, first_round=2, dec_tol=0.06)
+        assert st["max_logit_err"] < LOGIT_TOL, st
+    finally:
+        g.set_sampling(False)
+        g.close()
