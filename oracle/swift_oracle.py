@@ -8,7 +8,8 @@ smoke check and the benchmark's CPU-baseline leg use this file.
 What is pinned by tests independent of this file: the decoder forward against the Huggingface LLaMA
 implementation the paper ran (Appendix B.2) and against torch's fused attention; greedy
 losslessness against vanilla decoding (Section 3.1); sampling acceptance by chi-squared and the
-closed-form acceptance rate; matchness (Eq. 3) by brute force; Eq. 5 against the values printed in
+closed-form acceptance rate; nucleus filtering by a worked example, subset enumeration and the
+Huggingface warper; matchness (Eq. 3) by brute force; Eq. 5 against the values printed in
 Table 5; Philox against an independent library implementation.
 
 Parity unpinned by the paper (readings, fixed by convention only): RMSNorm eps 1e-5, RoPE theta
@@ -73,6 +74,31 @@ def categorical(weights: torch.Tensor, u: float) -> Tuple[int, float]:
 
 
 # =============================================================================== model pieces
+def nucleus(prob: torch.Tensor, top_p: float) -> Tuple[torch.Tensor, float]:
+    """Nucleus (top-p) filter, the sampling setting of Appendix B.2 (temperature 0.6, top_p 0.95).
+
+    Tokens are taken in order of decreasing probability until their total mass first reaches top_p times
+    the whole; every token at least as probable as the last one taken is kept (equal probabilities are
+    kept or dropped together), the others get probability 0, and the kept ones are renormalised.
+    top_p >= 1 returns the distribution unchanged.  Also returns how far the cut was from falling one
+    token earlier or later: min(|mass before the last token - top_p|, |mass with it - top_p|) as a
+    fraction of the whole."""
+    if top_p >= 1.0:
+        return prob, float("inf")
+    p = prob.to(torch.float64)
+    order = torch.sort(p, descending=True, stable=True).indices
+    cs = torch.cumsum(p[order], dim=0)
+    total = float(cs[-1])
+    goal = top_p * total
+    m = int(torch.searchsorted(cs, torch.tensor(goal, dtype=torch.float64)))     # first m with cs[m] >= goal
+    m = min(m, p.numel() - 1)
+    thr = p[order[m]]
+    kept = torch.where(p >= thr, p, torch.zeros_like(p))
+    before = float(cs[m - 1]) if m > 0 else 0.0
+    margin = min(abs(float(cs[m]) - goal), abs(before - goal)) / total
+    return kept / kept.sum(), margin
+
+
 def rmsnorm(x: torch.Tensor, g: torch.Tensor, eps: float) -> torch.Tensor:
     """x * g / sqrt(mean(x^2) + eps), row-wise."""
     return x * torch.rsqrt((x * x).mean(dim=-1, keepdim=True) + eps) * g.to(x.dtype)
@@ -219,12 +245,12 @@ class Oracle:
         return logits
 
     def draft(self, z: Sequence[int], max_k: int, stop_conf: float = 0.0,
-              sampler=None, temperature: float = 1.0) -> Tuple[List[int], List[float], List[torch.Tensor]]:
+              sampler=None, temperature: float = 1.0, top_p: float = 1.0) -> Tuple[List[int], List[float], List[torch.Tensor]]:
         """Autoregressive drafting with the layer-skipped model (Eq. 4) and early stopping.
 
         Step j feeds t* (j = 1) or y'_{j-1} at position n+j-1.  y'_j = argmax of the draft logits,
         p_j = max softmax (T = 1).  The token that falls below epsilon is kept, then drafting stops.
-        With `sampler(j, q_j) -> token`, y'_j is drawn from q_j = softmax(draft logits / T) instead.
+        With `sampler(j, q_j) -> token`, y'_j is drawn from q_j = nucleus(softmax(draft logits / T), top_p) instead.
         Returns (draft tokens, confidences, draft logits rows).
         """
         toks, confs, rows = [], [], []
@@ -235,7 +261,7 @@ class Oracle:
             if sampler is None:
                 y = argmax_lowest(logit)
             else:
-                y = int(sampler(j, torch.softmax(logit.to(torch.float64) / temperature, dim=-1)))
+                y = int(sampler(j, nucleus(torch.softmax(logit.to(torch.float64) / temperature, dim=-1), top_p)[0]))
             toks.append(y)
             confs.append(float(prob.max()))
             rows.append(logit)
@@ -284,16 +310,19 @@ def accept_greedy(draft_tokens: Sequence[int], target_logits: torch.Tensor) -> T
 
 
 def accept_sampling(draft_tokens: Sequence[int], q_rows: Sequence[torch.Tensor], target_logits: torch.Tensor,
-                    temperature: float, seed: int, round_index: int) -> Tuple[int, int, List[dict]]:
+                    temperature: float, seed: int, round_index: int, top_p: float = 1.0) -> Tuple[int, int, List[dict]]:
     """Speculative-sampling verification (the acceptance strategy of Appendix B.2, after Leviathan et al.).
 
-    p_j = softmax(target row j-1 / T); q_j = the distribution y'_j was drawn from.  For j = 1..k draw
+    p_j = nucleus(softmax(target row j-1 / T), top_p): the distribution plain sampling from the target would
+    use; q_j = the distribution y'_j was drawn from.  For j = 1..k draw
     u_j and accept iff u_j * q_j(y'_j) < p_j(y'_j)  (i.e. u < min(1, p/q)).  On the first rejection
     draw the replacement from max(0, p_j - q_j) renormalised; if nothing is rejected draw a bonus token
     from p_{k+1}.  Returns (a, next token, per-decision records for boundary-aware comparison).
     """
     k = len(draft_tokens)
     P = torch.softmax(target_logits.to(torch.float64) / temperature, dim=-1)
+    if top_p < 1.0:
+        P = torch.stack([nucleus(P[i], top_p)[0] for i in range(P.shape[0])])
     log: List[dict] = []
     for j in range(1, k + 1):
         y = int(draft_tokens[j - 1])
@@ -321,6 +350,7 @@ class GenParams:
     stop_conf: float = 0.0        # epsilon
     mode: str = "greedy"          # or "sampling"
     temperature: float = 1.0
+    top_p: float = 1.0
     rng_seed: int = 0
     gamma: int = 32
     stop_matchness: float = 0.95
@@ -343,12 +373,12 @@ class Round:
 
 
 def vanilla_generate(o: Oracle, prompt: Sequence[int], max_new: int, mode: str = "greedy",
-                     temperature: float = 1.0, rng_seed: int = 0) -> Tuple[List[int], List[float]]:
+                     temperature: float = 1.0, rng_seed: int = 0, top_p: float = 1.0) -> Tuple[List[int], List[float]]:
     """Plain autoregressive decoding of the full model: the definition SWIFT must reproduce."""
     logits = o.prefill(prompt)
     margins = [top2_margin(logits[-1])]
     if mode == "sampling":
-        p = torch.softmax(logits[-1].to(torch.float64) / temperature, -1)
+        p = nucleus(torch.softmax(logits[-1].to(torch.float64) / temperature, -1), top_p)[0]
         o.tokens[-1] = categorical(p, uniform(rng_seed, 0, 0, DRAW_BONUS))[0]
     step = 0
     while len(o.tokens) - len(prompt) < max_new:
@@ -356,7 +386,7 @@ def vanilla_generate(o: Oracle, prompt: Sequence[int], max_new: int, mode: str =
         row = o.forward_rows([o.tokens[-1]], o.n)[0]
         margins.append(top2_margin(row))
         if mode == "sampling":
-            p = torch.softmax(row.to(torch.float64) / temperature, -1)
+            p = nucleus(torch.softmax(row.to(torch.float64) / temperature, -1), top_p)[0]
             t = categorical(p, uniform(rng_seed, step, 0, DRAW_BONUS))[0]
         else:
             t = argmax_lowest(row)
@@ -377,7 +407,7 @@ def swift_generate(o: Oracle, prompt: Sequence[int], z0: Sequence[int], gp: GenP
     sampling = gp.mode == "sampling"
     logits = o.prefill(prompt)
     if sampling:
-        p = torch.softmax(logits[-1].to(torch.float64) / gp.temperature, -1)
+        p = nucleus(torch.softmax(logits[-1].to(torch.float64) / gp.temperature, -1), gp.top_p)[0]
         o.tokens[-1] = categorical(p, uniform(gp.rng_seed, 0, 0, DRAW_BONUS))[0]
     z = [int(v) for v in z0]
     best_score, opt_rounds, optimising = -1.0, 0, gp.max_opt_rounds > 0
@@ -404,14 +434,14 @@ def swift_generate(o: Oracle, prompt: Sequence[int], z0: Sequence[int], gp: GenP
                 def sampler(j, prob, _r=r):
                     q_rows.append(prob)
                     return categorical(prob, uniform(gp.rng_seed, _r, j, DRAW_DRAFT))[0]
-                d_tok, d_conf, d_rows = o.draft(z, k_max, gp.stop_conf, sampler, gp.temperature)
+                d_tok, d_conf, d_rows = o.draft(z, k_max, gp.stop_conf, sampler, gp.temperature, gp.top_p)
             else:
                 d_tok, d_conf, d_rows = o.draft(z, k_max, gp.stop_conf)
         else:
             d_tok, d_conf, d_rows = [], [], []
         tl = o.verify(d_tok)
         if sampling:
-            a, nxt, dec = accept_sampling(d_tok, q_rows, tl, gp.temperature, gp.rng_seed, r)
+            a, nxt, dec = accept_sampling(d_tok, q_rows, tl, gp.temperature, gp.rng_seed, r, gp.top_p)
         else:
             (a, nxt), dec = accept_greedy(d_tok, tl), []
         rounds.append(Round(o.n, d_tok, d_conf, [top2_margin(x) for x in d_rows],

@@ -170,6 +170,77 @@ def test_speculative_sampling_reproduces_target_distribution(case):
         assert accepted == trials
 
 
+# ------------------------------------------------------------------------------ nucleus (top-p) filtering
+def test_nucleus_worked_example_and_limits():
+    """By hand: p = (0.5, 0.3, 0.15, 0.05).  top_p 0.9 needs three tokens (0.8 < 0.9 <= 0.95); top_p 0.5 is reached
+    by the first token alone; top_p 1 changes nothing; a tiny top_p leaves the arg max (greedy)."""
+    p = torch.tensor([0.15, 0.5, 0.05, 0.3], dtype=torch.float64)
+    f, margin = so.nucleus(p, 0.9)
+    assert torch.allclose(f, torch.tensor([0.15, 0.5, 0.0, 0.3], dtype=torch.float64) / 0.95)
+    assert margin == pytest.approx(0.05)                      # 0.95 - 0.9; the other side (0.8) is 0.1 away
+    assert torch.allclose(so.nucleus(p, 0.5)[0], torch.tensor([0.0, 1.0, 0.0, 0.0], dtype=torch.float64))
+    assert torch.allclose(so.nucleus(p, 0.51)[0], torch.tensor([0.0, 0.625, 0.0, 0.375], dtype=torch.float64))
+    assert so.nucleus(p, 1.0)[0] is p
+    assert torch.equal(so.nucleus(p, 1e-9)[0], torch.tensor([0.0, 1.0, 0.0, 0.0], dtype=torch.float64))
+    # equal probabilities are kept together
+    t = torch.tensor([0.4, 0.2, 0.2, 0.2], dtype=torch.float64)
+    assert torch.allclose(so.nucleus(t, 0.5)[0], t)
+
+
+def test_nucleus_is_the_smallest_set_of_most_probable_tokens_by_brute_force():
+    """Among all token subsets whose mass reaches top_p, the kept set is one of minimum size, and of those the one
+    of maximum mass (checked by enumerating every subset of a 10-token vocabulary)."""
+    import itertools
+    g = torch.Generator().manual_seed(8)
+    for trial in range(20):
+        p = torch.softmax(torch.randn(10, generator=g, dtype=torch.float64) * 1.3, 0)
+        top_p = float(torch.rand(1, generator=g, dtype=torch.float64)) * 0.98 + 0.01
+        f, _ = so.nucleus(p, top_p)
+        kept = set(torch.nonzero(f).flatten().tolist())
+        best = None
+        for size in range(1, 11):
+            ok = [c for c in itertools.combinations(range(10), size) if float(p[list(c)].sum()) >= top_p]
+            if ok:
+                best = set(max(ok, key=lambda c: float(p[list(c)].sum())))
+                break
+        assert kept == best, (trial, top_p)
+        assert torch.allclose(f[list(kept)], p[list(kept)] / p[list(kept)].sum())
+
+
+def test_nucleus_keeps_the_tokens_huggingface_keeps():
+    """The library the paper ran (Appendix B.2) filters with TopPLogitsWarper: same kept set on random logits."""
+    from transformers.generation.logits_process import TopPLogitsWarper
+    g = torch.Generator().manual_seed(12)
+    for top_p in (0.95, 0.6, 0.3):
+        logits = torch.randn(5, 300, generator=g, dtype=torch.float64) * 2.0
+        warped = TopPLogitsWarper(top_p=top_p)(None, logits.clone())
+        for r in range(5):
+            f, margin = so.nucleus(torch.softmax(logits[r], -1), top_p)
+            if margin > 1e-9:
+                assert torch.equal(f > 0, torch.isfinite(warped[r])), (top_p, r)
+
+
+def test_speculative_sampling_with_nucleus_reproduces_the_filtered_target():
+    """With top_p < 1 the emitted token must follow nucleus(p) (tokens outside it never appear), whatever q."""
+    g = torch.Generator().manual_seed(5)
+    V, top_p, trials, seed = 12, 0.8, 60_000, 23
+    p = torch.softmax(torch.randn(V, generator=g, dtype=torch.float64) * 1.5, 0)
+    q_full = torch.softmax(torch.randn(V, generator=g, dtype=torch.float64) * 1.5, 0)
+    pf, q = so.nucleus(p, top_p)[0], so.nucleus(q_full, top_p)[0]
+    assert 0 < int((pf == 0).sum()) < V - 1
+    tl = torch.log(p)[None].repeat(2, 1)
+    counts = np.zeros(V)
+    for t in range(trials):
+        y = so.categorical(q, so.uniform(seed, t, 1, so.DRAW_DRAFT))[0]
+        a, nxt, _ = so.accept_sampling([y], [q], tl, 1.0, seed, t, top_p)
+        counts[y if a == 1 else nxt] += 1
+    assert counts[(pf == 0).numpy()].sum() == 0
+    live = (pf > 0).numpy()
+    expect = pf.numpy()[live] * trials
+    chi2 = float(((counts[live] - expect) ** 2 / expect).sum())
+    assert chi2 < 40.0, chi2
+
+
 def test_wrong_acceptance_rules_fail_the_chi_squared():
     """Guard on the guard: always accepting the draft gives q, not p, and the statistic explodes."""
     g = torch.Generator().manual_seed(3)
