@@ -170,7 +170,8 @@ def main():
     hbm_peak, peak_kind = peaks()
     sampling = run.mode == "sampling"
     desc = (f"{args.workload}: {cfg.name}-shaped decoder ({cfg.n_blocks} blocks, d {cfg.d_model}, {cfg.dtype}), "
-            f"prompt {run.prompt_len}, {max_new} {run.mode} tokens, {run.n_skip_blocks} blocks skipped, max draft {run.max_draft}")
+            f"prompt {run.prompt_len}, {max_new} {run.mode} tokens, {run.n_skip_blocks} blocks skipped, max draft {run.max_draft}"
+            + (f", temperature {run.temperature}, top_p {run.top_p}" if sampling and (run.temperature != 1.0 or run.top_p != 1.0) else ""))
 
     if args.impl == "reference":
         if rank != 0:
@@ -225,7 +226,7 @@ def main():
     else:
         model.load_weights(synth.iter_tensors(cfg))
     if sampling:
-        model.set_sampling(True, run.temperature, run.rng_seed)
+        model.set_sampling(True, run.temperature, run.rng_seed, run.top_p)
     prompt = synth.prompt(cfg, run.prompt_len, stream=rank)
     cands = None
     if run.optimise:

@@ -100,6 +100,14 @@ swift_status swift_pack_tensor(swift_ctx* ctx, swift_tensor_kind kind, int32_t b
  * by `seed`; temperature scales both the target's and the draft's logits.  Default: greedy. */
 swift_status swift_set_sampling(swift_ctx* ctx, int32_t mode, float temperature, uint64_t seed);
 
+/* Nucleus (top-p) filtering of the distributions sampling mode draws from and compares (the paper samples with
+ * temperature 0.6 and top_p 0.95 on code generation, Appendix B.2).  Both the target's p = softmax(logits / T) and
+ * the draft's q are cut to their most probable tokens whose mass first reaches top_p (every token as probable as
+ * the last one included is kept) and renormalised; acceptance, the residual max(0, p - q) and the bonus draw then
+ * use the cut distributions, so the output follows what plain nucleus sampling from the target would give.
+ * top_p in (0, 1]; 1 (the default) = no filtering.  No effect in greedy mode.  Not allowed inside a round. */
+swift_status swift_set_top_p(swift_ctx* ctx, float top_p);
+
 /*
  * The primitive under all three forms of the forward: M = n_rows new rows at positions
  * pos0 .. pos0+M-1 run through the sub-layers not in `skip_mask` (NULL = full model); every row

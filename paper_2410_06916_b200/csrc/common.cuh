@@ -38,6 +38,7 @@ struct DevState {
     float stop_conf;       // early-stop threshold of this round
     unsigned seed_lo, seed_hi;
     int pad[2];
+    float row_thresh[ROWS]; // nucleus sampling: smallest exp((l - max) / T) a row keeps (0 = everything); row_sum covers the kept ones
 };
 
 // Programmatic dependent launch.  Every kernel of a forward is launched with programmatic stream

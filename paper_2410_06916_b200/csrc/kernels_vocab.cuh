@@ -86,7 +86,8 @@ __device__ int block_categorical(WeightFn w, int n, float u, float* sh)
 // drafting when the confidence is below stop_conf.
 __global__ void __launch_bounds__(VOCAB_THREADS)
 vocab_kernel(DevState* st, const float* __restrict__ part, int n_split, size_t split_stride,
-             float* __restrict__ logits, int vocab, float inv_temp, int mode, int sampling, float* __restrict__ q_rows)
+             float* __restrict__ logits, int vocab, float inv_temp, int mode, int sampling, float* __restrict__ q_rows,
+             float top_p)
 {
     pdl_enter();
     __shared__ float sh[VOCAB_THREADS + 72];
@@ -168,10 +169,36 @@ vocab_kernel(DevState* st, const float* __restrict__ part, int n_split, size_t s
     s1 = block_sum(s1, sh);
     sT = block_sum(sT, sh);
     const float conf = 1.f / s1;
+
+    // Nucleus sampling (top_p < 1): keep the most probable tokens whose mass first reaches top_p of the whole, all
+    // tokens as probable as the last one included.  With w_i = exp((l_i - max) / T) that is {w_i >= theta} for the
+    // largest theta whose kept mass is still >= top_p * sum(w).  Positive floats order like their bit patterns, so
+    // theta is found by bisection on the bit pattern (31 block-wide sums); the kept mass replaces the row sum.
+    float theta = 0.f;
+    if (sampling && top_p < 1.f) {
+        const float goal = top_p * sT;
+        auto mass_from = [&](unsigned bits) {
+            float m = 0.f;                                      // the row as this thread stored it above, same index order
+#pragma unroll 1
+            for (int i = tid; i < vocab; i += VOCAB_THREADS) {
+                const float w = expf((lrow[i] - am.v) * inv_temp);
+                if (__float_as_uint(w) >= bits) m += w;
+            }
+            return block_sum(m, sh);
+        };
+        unsigned lo = 0u, hi = 0x3F800001u;                     // mass_from(lo) >= goal > mass_from(hi) = 0 (w <= 1)
+        while (hi - lo > 1u) {
+            const unsigned mid = lo + (hi - lo) / 2u;
+            if (mass_from(mid) >= goal) lo = mid; else hi = mid;
+        }
+        theta = __uint_as_float(lo);
+        sT = mass_from(lo);
+    }
     if (tid == 0) {
         st->argmax[r] = am.i;
         st->row_max[r] = am.v;
         st->row_sum[r] = sT;
+        st->row_thresh[r] = theta;
     }
     if (mode != VOCAB_DRAFT || r != 0) return;
 
@@ -185,7 +212,10 @@ vocab_kernel(DevState* st, const float* __restrict__ part, int n_split, size_t s
     if (sampling) {
         float* qrow = q_rows + (size_t)(draft_j - 1) * vocab;
         const float inv_sum = 1.f / sT;
-        for (int i = tid; i < vocab; i += VOCAB_THREADS) qrow[i] = expf((lrow[i] - am.v) * inv_temp) * inv_sum;
+        for (int i = tid; i < vocab; i += VOCAB_THREADS) {
+            const float w = expf((lrow[i] - am.v) * inv_temp);
+            qrow[i] = w >= theta ? w * inv_sum : 0.f;
+        }
         __syncthreads();
         const float u = philox_uniform(seed, round, (uint32_t)draft_j, DRAW_DRAFT);
         y = block_categorical([&](int i) { return qrow[i]; }, vocab, u, sh);
@@ -223,7 +253,8 @@ accept_kernel(DevState* st, const float* __restrict__ logits, const float* __res
         int a = 0, rejected = 0;
         for (int j = 1; j <= k; ++j) {
             const int y = st->draft_tok[j];
-            const float p = expf((logits[(size_t)(j - 1) * vocab + y] - st->row_max[j - 1]) * inv_temp) / st->row_sum[j - 1];
+            const float w = expf((logits[(size_t)(j - 1) * vocab + y] - st->row_max[j - 1]) * inv_temp);
+            const float p = w >= st->row_thresh[j - 1] ? w / st->row_sum[j - 1] : 0.f;
             const float q = q_rows[(size_t)(j - 1) * vocab + y];
             const float u = philox_uniform(seed, round, (uint32_t)j, DRAW_ACCEPT);
             if (!(u * q < p)) { rejected = 1; break; }
@@ -235,8 +266,8 @@ accept_kernel(DevState* st, const float* __restrict__ logits, const float* __res
     __syncthreads();
     const int a = sh_a, rejected = sh_rejected;
     const float* lrow = logits + (size_t)a * vocab;          // target row j-1 with j = a+1
-    const float mx = st->row_max[a], inv_sum = 1.f / st->row_sum[a];
-    auto p_of = [&](int i) { return expf((lrow[i] - mx) * inv_temp) * inv_sum; };
+    const float mx = st->row_max[a], inv_sum = 1.f / st->row_sum[a], theta = st->row_thresh[a];
+    auto p_of = [&](int i) { const float w = expf((lrow[i] - mx) * inv_temp); return w >= theta ? w * inv_sum : 0.f; };
     int tok;
     if (rejected) {
         const float* qrow = q_rows + (size_t)a * vocab;
@@ -265,9 +296,10 @@ sample_row_kernel(DevState* st, const float* __restrict__ logits, int vocab, int
 {
     __shared__ float sh[VOCAB_THREADS + 72];
     const float* lrow = logits + (size_t)row * vocab;
-    const float mx = st->row_max[row];
+    const float mx = st->row_max[row], theta = st->row_thresh[row];
     const float u = philox_uniform(seed, round, slot, DRAW_BONUS);
-    const int tok = block_categorical([&](int i) { return expf((lrow[i] - mx) * inv_temp); }, vocab, u, sh);
+    const int tok = block_categorical([&](int i) { const float w = expf((lrow[i] - mx) * inv_temp); return w >= theta ? w : 0.f; },
+                                      vocab, u, sh);
     if (threadIdx.x == 0) {
         st->next_token = tok;
         st->draft_tok[0] = tok;

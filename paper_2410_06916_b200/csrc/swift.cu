@@ -69,7 +69,7 @@ struct swift_ctx {
     int phase, n, pending, n_prompt, round, last_k, last_max_k;
     bool round_open;
     std::vector<int> hist;           // prompt + generated tokens, pending included
-    int mode; float temperature; uint64_t seed;
+    int mode; float temperature, top_p; uint64_t seed;
     int64_t launches;
     std::string err;
     cudaEvent_t ev[8];
@@ -448,7 +448,7 @@ swift_status forward_chunk(swift_ctx* ctx, int rows, const int* toks_dev, const 
         ST(run_gemm<T>(ctx, mr, GemmSite{xn, d.vocab, dm, wptr<T>(ctx, ctx->wl.lm_head), &ctx->tm_lm_head, &ctx->tm_xn}, &S));
         CU(launch_k(vocab_kernel, dim3(rows), dim3(VOCAB_THREADS), 0, ctx, st, (const float*)part, S, (size_t)ROWS * d.vocab,
                     kptr<float>(ctx, ctx->kl.logits), d.vocab, 1.0f / ctx->temperature, head.mode,
-                    ctx->mode == SWIFT_SAMPLING ? 1 : 0, kptr<float>(ctx, ctx->kl.q_rows)));
+                    ctx->mode == SWIFT_SAMPLING ? 1 : 0, kptr<float>(ctx, ctx->kl.q_rows), ctx->top_p));
     }
     CU(cudaGetLastError());
     return SWIFT_OK;
@@ -551,7 +551,7 @@ swift_status forward_chunk_fused(swift_ctx* ctx, int rows, const int* toks_dev, 
         ST(gemm(EPI_PLAIN, &ctx->tm_lm_head, &ctx->tm_xn, d.vocab, dm, ep));
         CU(launch_k(vocab_kernel, dim3(rows), dim3(VOCAB_THREADS), 0, ctx, st, (const float*)kptr<float>(ctx, ctx->kl.part), 1,
                     (size_t)ROWS * d.vocab, kptr<float>(ctx, ctx->kl.logits), d.vocab, 1.0f / ctx->temperature, head.mode,
-                    ctx->mode == SWIFT_SAMPLING ? 1 : 0, kptr<float>(ctx, ctx->kl.q_rows)));
+                    ctx->mode == SWIFT_SAMPLING ? 1 : 0, kptr<float>(ctx, ctx->kl.q_rows), ctx->top_p));
     }
     CU(cudaGetLastError());
     return SWIFT_OK;
@@ -577,14 +577,14 @@ swift_status forward_chunk_any(swift_ctx* ctx, int rows, const int* toks_dev, co
 // hundred kernel launches per forward.
 struct FwdKey {
     int rows, head_run, head_mode, sampling, use_tc, use_pdl, fuse;
-    float temperature;
+    float temperature, top_p;
     const void* toks;
     const void* page_table;
     std::vector<uint8_t> mask;
     bool operator==(const FwdKey& o) const
     {
         return rows == o.rows && head_run == o.head_run && head_mode == o.head_mode && sampling == o.sampling &&
-               use_tc == o.use_tc && use_pdl == o.use_pdl && fuse == o.fuse && temperature == o.temperature && toks == o.toks && page_table == o.page_table && mask == o.mask;
+               use_tc == o.use_tc && use_pdl == o.use_pdl && fuse == o.fuse && temperature == o.temperature && top_p == o.top_p && toks == o.toks && page_table == o.page_table && mask == o.mask;
     }
 };
 struct FwdGraph {
@@ -599,7 +599,7 @@ swift_status forward_cached(swift_ctx* ctx, int rows, const int* toks_dev, const
 {
     if (!ctx->use_graphs) return forward_chunk_any(ctx, rows, toks_dev, skip, page_table, head);
     const int L = 2 * ctx->d.n_blocks;
-    FwdKey key{rows, head.run ? 1 : 0, head.mode, ctx->mode, ctx->use_tc ? 1 : 0, ctx->use_pdl ? 1 : 0, ctx->fuse ? 1 : 0, ctx->temperature, toks_dev, page_table,
+    FwdKey key{rows, head.run ? 1 : 0, head.mode, ctx->mode, ctx->use_tc ? 1 : 0, ctx->use_pdl ? 1 : 0, ctx->fuse ? 1 : 0, ctx->temperature, ctx->top_p, toks_dev, page_table,
                skip ? std::vector<uint8_t>(skip, skip + L) : std::vector<uint8_t>()};
     auto& cache = *ctx->graphs;
     ctx->graph_clock++;
@@ -960,7 +960,7 @@ swift_status swift_load(const swift_model_desc* desc, swift_devbuf weights, swif
     c->max_splits = ceil_div(desc->max_positions, ATTN_CHUNK);
     c->phase = PH_LOADED; c->n = 0; c->pending = 0; c->n_prompt = 0; c->round = 0; c->last_k = 0; c->last_max_k = 0;
     c->round_open = false;
-    c->mode = SWIFT_GREEDY; c->temperature = 1.f; c->seed = 0; c->launches = 0;
+    c->mode = SWIFT_GREEDY; c->temperature = 1.f; c->top_p = 1.f; c->seed = 0; c->launches = 0;
     ctx = c;
     c->use_tc = false;
     if (desc->dtype == SWIFT_BF16) {
@@ -1064,6 +1064,15 @@ swift_status swift_set_sampling(swift_ctx* ctx, int32_t mode, float temperature,
     if (!(temperature > 0.f)) return fail(ctx, SWIFT_EINVAL, "temperature must be positive");
     if (ctx->round_open) return fail(ctx, SWIFT_ESTATE, "cannot change the acceptance strategy inside a round");
     ctx->mode = mode; ctx->temperature = temperature; ctx->seed = seed;
+    return SWIFT_OK;
+}
+
+swift_status swift_set_top_p(swift_ctx* ctx, float top_p)
+{
+    if (!ctx) return SWIFT_EINVAL;
+    if (!(top_p > 0.f) || top_p > 1.f) return fail(ctx, SWIFT_EINVAL, "top_p must be in (0, 1]");
+    if (ctx->round_open) return fail(ctx, SWIFT_ESTATE, "cannot change the sampling distribution inside a round");
+    ctx->top_p = top_p;
     return SWIFT_OK;
 }
 

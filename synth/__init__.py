@@ -94,6 +94,7 @@ class RunConfig:
     n_skip_blocks: int = 0       # blocks skipped by the draft model (both sub-layers)
     mode: str = "greedy"         # "greedy" or "sampling"
     temperature: float = 1.0
+    top_p: float = 1.0           # nucleus filtering of the sampling distributions (1 = none)
     rng_seed: int = 0
     optimise: bool = False       # on-the-fly skip-set optimisation (Section 4.1)
     gamma: int = 32              # context window
@@ -118,6 +119,8 @@ RUNS: Dict[str, Tuple[str, RunConfig]] = {
     "c3": ("13b", RunConfig(1024, 512, 8, n_skip_blocks=18, optimise=True)),
     "c3-fixed": ("13b", RunConfig(1024, 512, 8, n_skip_blocks=18)),     # config 3's shape with the planted set held fixed
     "c4": ("13b", RunConfig(1024, 512, 8, n_skip_blocks=20, mode="sampling", rng_seed=4)),
+    # config 4 with the sampling setting the paper uses on code generation (Appendix B.2)
+    "c4-nucleus": ("13b", RunConfig(1024, 512, 8, n_skip_blocks=20, mode="sampling", temperature=0.6, top_p=0.95, rng_seed=4)),
     "c5": ("70b", RunConfig(2048, 512, 12, n_skip_blocks=36)),
 }
 

@@ -83,7 +83,7 @@ def resync(gpu, o: so.Oracle, rounds_done: int = -1):
 
 
 def walk_rounds(o: so.Oracle, gpu, z, n_rounds: int, max_k: int, stop_conf: float = 0.0, sampling=False,
-                temperature=1.0, seed=0, first_round=1, dec_tol=1e-3):
+                temperature=1.0, seed=0, first_round=1, dec_tol=1e-3, top_p=1.0):
     """Runs n_rounds of draft -> verify -> accept on both sides from the same state and compares every
     intermediate the oracle exposes, exempting only decisions the oracle marks as near a boundary.
     Returns counters for the caller to assert on."""
@@ -99,7 +99,7 @@ def walk_rounds(o: so.Oracle, gpu, z, n_rounds: int, max_k: int, stop_conf: floa
                 tok, dist = so.categorical(q, so.uniform(seed, _r, j, so.DRAW_DRAFT))
                 dec_margins.append(dist)
                 return tok
-            d_tok, d_conf, d_rows = o.draft(z, max_k, stop_conf, sampler, temperature)
+            d_tok, d_conf, d_rows = o.draft(z, max_k, stop_conf, sampler, temperature, top_p)
         else:
             d_tok, d_conf, d_rows = o.draft(z, max_k, stop_conf)
             dec_margins = [so.top2_margin(x) for x in d_rows]
@@ -121,7 +121,7 @@ def walk_rounds(o: so.Oracle, gpu, z, n_rounds: int, max_k: int, stop_conf: floa
         if sampling and not same_draft:
             # the draft distributions kept on the GPU belong to another prefix: start this round over
             tl = o.verify(d_tok)
-            a, nxt, _ = so.accept_sampling(d_tok, q_rows, tl, temperature, seed, r)
+            a, nxt, _ = so.accept_sampling(d_tok, q_rows, tl, temperature, seed, r, top_p)
             o.commit(d_tok[:a], nxt)
             gpu.verify(d_tok); gpu.accept()
             resync(gpu, o, r)
@@ -139,7 +139,7 @@ def walk_rounds(o: so.Oracle, gpu, z, n_rounds: int, max_k: int, stop_conf: floa
             if t_margin[i] > MARGIN:
                 assert int(g_am[i]) == t_am[i], f"round {r} row {i}"
         if sampling:
-            a, nxt, dec = so.accept_sampling(d_tok, q_rows, tl, temperature, seed, r)
+            a, nxt, dec = so.accept_sampling(d_tok, q_rows, tl, temperature, seed, r, top_p)
             exempt = any(d["margin"] <= dec_tol for d in dec)
         else:
             a, nxt = so.accept_greedy(d_tok, tl)

@@ -429,6 +429,47 @@ def test_sampling_with_temperature(tiny_pair):
         g.set_sampling(False)
 
 
+@pytest.mark.parametrize("T,top_p", [(0.6, 0.95), (1.0, 0.5), (0.8, 0.05)])
+def test_sampling_with_nucleus_filter(tiny_pair, T, top_p):
+    """Appendix B.2's sampling setting (temperature 0.6, top_p 0.95) and two sharper cuts: draft draws, accept
+    decisions and resampled tokens follow the oracle's, and no emitted token lies outside the target's nucleus."""
+    o, g = tiny_pair
+    prompt = synth.prompt(TINY, 24)
+    seed = 31
+    g.set_sampling(True, T, seed, top_p)
+    try:
+        logits = o.prefill(prompt)
+        p = so.nucleus(torch.softmax(logits[-1].double() / T, -1), top_p)[0]
+        first, dist = so.categorical(p, so.uniform(seed, 0, 0, so.DRAW_BONUS))
+        o.tokens[-1] = first
+        g_first = g.prefill(prompt)
+        assert g_first == first or dist < 1e-3
+        assert p[g_first] > 0
+        g.set_pending(first)
+        z = list(synth.block_mask(TINY, synth.draft_blocks(TINY, 5)))
+        st = walk_rounds(o, g, z, n_rounds=20, max_k=4, sampling=True, temperature=T, seed=seed, top_p=top_p)
+        assert st["accept_cmp"] >= 15 and st["max_logit_err"] < 1e-4, st
+    finally:
+        g.set_sampling(False)
+
+
+def test_vanilla_sampling_with_nucleus_filter(tiny_pair):
+    """Plain sampling of the full model with temperature and top_p: the same tokens as the oracle's, up to draws
+    that land within 1e-3 of a bracket edge."""
+    o, g = tiny_pair
+    from paper_2410_06916_b200 import GenParams
+    prompt = synth.prompt(TINY, 24)
+    seed, T, top_p = 9, 0.6, 0.9
+    ref, _ = so.vanilla_generate(o, prompt, 24, mode="sampling", temperature=T, rng_seed=seed, top_p=top_p)
+    g.set_sampling(True, T, seed, top_p)
+    try:
+        out, _, _ = g.generate(prompt, GenParams(max_new=24, vanilla=True))
+    finally:
+        g.set_sampling(False)
+    same = next((i for i, (a, b) in enumerate(zip(out, ref)) if a != b), len(ref))
+    assert same >= 12, (same, out, ref)
+
+
 def test_cache_fills_to_capacity(small_cfg):
     """Generation that ends exactly at max_positions, and one token more is refused without side effects."""
     from paper_2410_06916_b200 import GenParams, SwiftError
