@@ -87,7 +87,7 @@ __device__ int block_categorical(WeightFn w, int n, float u, float* sh)
 __global__ void __launch_bounds__(VOCAB_THREADS)
 vocab_kernel(DevState* st, const float* __restrict__ part, int n_split, size_t split_stride,
              float* __restrict__ logits, int vocab, float inv_temp, int mode, int sampling, float* __restrict__ q_rows,
-             float top_p)
+             float top_p, int w_cached)
 {
     pdl_enter();
     __shared__ float sh[VOCAB_THREADS + 72];
@@ -177,11 +177,16 @@ vocab_kernel(DevState* st, const float* __restrict__ part, int n_split, size_t s
     float theta = 0.f;
     if (sampling && top_p < 1.f) {
         const float goal = top_p * sT;
+        // w_cached: the launch provides vocab floats of dynamic shared memory, and every thread keeps the weights
+        // of its own indices there instead of evaluating 31 x vocab exponentials (same values either way)
+        extern __shared__ float w_sh[];
+        if (w_cached)
+            for (int i = tid; i < vocab; i += VOCAB_THREADS) w_sh[i] = expf((lrow[i] - am.v) * inv_temp);
         auto mass_from = [&](unsigned bits) {
             float m = 0.f;                                      // the row as this thread stored it above, same index order
 #pragma unroll 1
             for (int i = tid; i < vocab; i += VOCAB_THREADS) {
-                const float w = expf((lrow[i] - am.v) * inv_temp);
+                const float w = w_cached ? w_sh[i] : expf((lrow[i] - am.v) * inv_temp);
                 if (__float_as_uint(w) >= bits) m += w;
             }
             return block_sum(m, sh);

@@ -251,6 +251,15 @@ DevState* state_of(swift_ctx* c) { return kptr<DevState>(c, c->kl.state); }
 int mr_of(int rows) { return rows <= 1 ? 1 : rows <= 2 ? 2 : rows <= 4 ? 4 : rows <= 8 ? 8 : 16; }
 int attn_mr_of(int rows) { return rows > 8 && rows <= 12 ? 12 : mr_of(rows); }   // 9 rows = a verification of 8 drafts
 
+// Dynamic shared memory of the vocabulary kernel: one float per token while a nucleus cut is searched (sampling with
+// top_p < 1), if the vocabulary fits; nothing otherwise.
+constexpr size_t VOCAB_CACHE_MAX_BYTES = 200 * 1024;
+size_t vocab_cache_bytes(const swift_ctx* ctx)
+{
+    const size_t need = (size_t)ctx->d.vocab * sizeof(float);
+    return (ctx->mode == SWIFT_SAMPLING && ctx->top_p < 1.f && need <= VOCAB_CACHE_MAX_BYTES) ? need : 0;
+}
+
 // ------------------------------------------------------------------------------ launches
 // Launch with programmatic stream serialisation (see pdl_enter in common.cuh).
 template <typename... KArgs, typename... Args>
@@ -446,9 +455,9 @@ swift_status forward_chunk(swift_ctx* ctx, int rows, const int* toks_dev, const 
         CU(launch_k(resid_norm_kernel, dim3(rows), dim3(512), 0, ctx, (const DevState*)st, h, pend, pend_S, (size_t)ROWS * dm,
                     (const float*)wptr<float>(ctx, ctx->wl.final_norm), xn, xn_hl, dm, d.rms_eps));
         ST(run_gemm<T>(ctx, mr, GemmSite{xn, d.vocab, dm, wptr<T>(ctx, ctx->wl.lm_head), &ctx->tm_lm_head, &ctx->tm_xn}, &S));
-        CU(launch_k(vocab_kernel, dim3(rows), dim3(VOCAB_THREADS), 0, ctx, st, (const float*)part, S, (size_t)ROWS * d.vocab,
+        CU(launch_k(vocab_kernel, dim3(rows), dim3(VOCAB_THREADS), vocab_cache_bytes(ctx), ctx, st, (const float*)part, S, (size_t)ROWS * d.vocab,
                     kptr<float>(ctx, ctx->kl.logits), d.vocab, 1.0f / ctx->temperature, head.mode,
-                    ctx->mode == SWIFT_SAMPLING ? 1 : 0, kptr<float>(ctx, ctx->kl.q_rows), ctx->top_p));
+                    ctx->mode == SWIFT_SAMPLING ? 1 : 0, kptr<float>(ctx, ctx->kl.q_rows), ctx->top_p, vocab_cache_bytes(ctx) != 0 ? 1 : 0));
     }
     CU(cudaGetLastError());
     return SWIFT_OK;
@@ -549,9 +558,9 @@ swift_status forward_chunk_fused(swift_ctx* ctx, int rows, const int* toks_dev, 
         EpiParams ep = base;
         ep.n_sumsq_tiles = n_tiles_in;
         ST(gemm(EPI_PLAIN, &ctx->tm_lm_head, &ctx->tm_xn, d.vocab, dm, ep));
-        CU(launch_k(vocab_kernel, dim3(rows), dim3(VOCAB_THREADS), 0, ctx, st, (const float*)kptr<float>(ctx, ctx->kl.part), 1,
+        CU(launch_k(vocab_kernel, dim3(rows), dim3(VOCAB_THREADS), vocab_cache_bytes(ctx), ctx, st, (const float*)kptr<float>(ctx, ctx->kl.part), 1,
                     (size_t)ROWS * d.vocab, kptr<float>(ctx, ctx->kl.logits), d.vocab, 1.0f / ctx->temperature, head.mode,
-                    ctx->mode == SWIFT_SAMPLING ? 1 : 0, kptr<float>(ctx, ctx->kl.q_rows), ctx->top_p));
+                    ctx->mode == SWIFT_SAMPLING ? 1 : 0, kptr<float>(ctx, ctx->kl.q_rows), ctx->top_p, vocab_cache_bytes(ctx) != 0 ? 1 : 0));
     }
     CU(cudaGetLastError());
     return SWIFT_OK;
@@ -863,6 +872,7 @@ cudaError_t init_kernel_attrs()
     if (e == cudaSuccess) e = cudaFuncSetAttribute(gemm_tc_kernel<EPI_SWIGLU, float>, cudaFuncAttributeMaxDynamicSharedMemorySize, TC_SMEM_BYTES);
     if (e == cudaSuccess) e = cudaFuncSetAttribute(gemm_tc_kernel<EPI_QKV, float>, cudaFuncAttributeMaxDynamicSharedMemorySize, TC_SMEM_BYTES);
     if (e == cudaSuccess) e = cudaFuncSetAttribute(gemm_tc_kernel<EPI_QKV, __nv_bfloat16>, cudaFuncAttributeMaxDynamicSharedMemorySize, TC_SMEM_BYTES);
+    if (e == cudaSuccess) e = cudaFuncSetAttribute(vocab_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)VOCAB_CACHE_MAX_BYTES);
     return e;
 }
 
