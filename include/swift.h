@@ -108,6 +108,13 @@ swift_status swift_set_sampling(swift_ctx* ctx, int32_t mode, float temperature,
  * top_p in (0, 1]; 1 (the default) = no filtering.  No effect in greedy mode.  Not allowed inside a round. */
 swift_status swift_set_top_p(swift_ctx* ctx, float top_p);
 
+/* How draft tokens are chosen in sampling mode.  0 (default): y'_j is drawn from the draft's distribution q_j and
+ * accepted with probability min(1, p_j(y') / q_j(y')).  1: y'_j = argmax of the draft's logits, as Eq. 4 of Section 4.2
+ * writes the drafting step; q_j is then the point mass on y'_j, so the draft is accepted with probability p_j(y') and a
+ * rejected one is replaced by a draw from p_j with y'_j removed.  Both leave the output distributed as sampling from the
+ * target.  No effect in greedy mode.  Not allowed inside a round. */
+swift_status swift_set_greedy_draft(swift_ctx* ctx, int32_t on);
+
 /*
  * The primitive under all three forms of the forward: M = n_rows new rows at positions
  * pos0 .. pos0+M-1 run through the sub-layers not in `skip_mask` (NULL = full model); every row

@@ -309,6 +309,13 @@ def accept_greedy(draft_tokens: Sequence[int], target_logits: torch.Tensor) -> T
     return a, argmax_lowest(target_logits[a])
 
 
+def point_mass(n: int, y: int) -> torch.Tensor:
+    """The distribution of a draft token chosen by arg max (Eq. 4): all mass on y."""
+    q = torch.zeros(n, dtype=torch.float64)
+    q[y] = 1.0
+    return q
+
+
 def accept_sampling(draft_tokens: Sequence[int], q_rows: Sequence[torch.Tensor], target_logits: torch.Tensor,
                     temperature: float, seed: int, round_index: int, top_p: float = 1.0) -> Tuple[int, int, List[dict]]:
     """Speculative-sampling verification (the acceptance strategy of Appendix B.2, after Leviathan et al.).
@@ -351,6 +358,7 @@ class GenParams:
     mode: str = "greedy"          # or "sampling"
     temperature: float = 1.0
     top_p: float = 1.0
+    greedy_draft: bool = False    # sampling mode with drafts chosen by arg max (Eq. 4 as written): q_j = point mass on y'_j
     rng_seed: int = 0
     gamma: int = 32
     stop_matchness: float = 0.95
@@ -432,6 +440,10 @@ def swift_generate(o: Oracle, prompt: Sequence[int], z0: Sequence[int], gp: GenP
         if k_max > 0:
             if sampling:
                 def sampler(j, prob, _r=r):
+                    if gp.greedy_draft:
+                        y = argmax_lowest(prob)
+                        q_rows.append(point_mass(prob.numel(), y))
+                        return y
                     q_rows.append(prob)
                     return categorical(prob, uniform(gp.rng_seed, _r, j, DRAW_DRAFT))[0]
                 d_tok, d_conf, d_rows = o.draft(z, k_max, gp.stop_conf, sampler, gp.temperature, gp.top_p)

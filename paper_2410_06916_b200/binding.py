@@ -50,7 +50,7 @@ class _Stats(C.Structure):
 
 # every symbol include/swift.h declares
 SYMBOLS = ("swift_weights_bytes", "swift_kv_bytes", "swift_workspace_bytes", "swift_load", "swift_free",
-           "swift_last_error", "swift_pack_tensor", "swift_set_sampling", "swift_set_top_p", "swift_forward_rows", "swift_prefill",
+           "swift_last_error", "swift_pack_tensor", "swift_set_sampling", "swift_set_top_p", "swift_set_greedy_draft", "swift_forward_rows", "swift_prefill",
            "swift_set_pending", "swift_draft", "swift_verify", "swift_accept", "swift_score_skipsets", "swift_generate",
            "swift_committed_length", "swift_launch_count", "swift_round_times", "swift_forward_bytes", "swift_read_kv", "swift_time_gemm", "swift_set_gemm_impl", "swift_gemm", "swift_gemm_static",
            "swift_gemm_static_error")
@@ -76,6 +76,7 @@ def load_library(path: Optional[str] = None) -> C.CDLL:
     lib.swift_pack_tensor.argtypes = [vp, i32, i32, vp, C.c_size_t]
     lib.swift_set_sampling.argtypes = [vp, i32, f32, u64]
     lib.swift_set_top_p.argtypes = [vp, f32]
+    lib.swift_set_greedy_draft.argtypes = [vp, i32]
     lib.swift_forward_rows.argtypes = [vp, vp, i32, i32, vp, i32, vp, vp]
     lib.swift_prefill.argtypes = [vp, vp, i32, vp]
     lib.swift_set_pending.argtypes = [vp, i32, i32]
@@ -239,9 +240,11 @@ class SwiftModel:
         for name, block, t in tensors:
             self.pack(name, block, t)
 
-    def set_sampling(self, sampling: bool, temperature: float = 1.0, seed: int = 0, top_p: float = 1.0):
+    def set_sampling(self, sampling: bool, temperature: float = 1.0, seed: int = 0, top_p: float = 1.0,
+                     greedy_draft: bool = False):
         self._check(self._lib.swift_set_sampling(self.ctx, 1 if sampling else 0, temperature, seed))
         self._check(self._lib.swift_set_top_p(self.ctx, top_p))
+        self._check(self._lib.swift_set_greedy_draft(self.ctx, 1 if greedy_draft else 0))
 
     @property
     def n(self) -> int:

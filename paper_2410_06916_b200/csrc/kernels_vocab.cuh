@@ -81,9 +81,10 @@ __device__ int block_categorical(WeightFn w, int n, float u, float* sh)
 
 // One CTA per row.  logits[r][i] = sum_s part[s][r][i]; argmax (lowest id on ties), row max,
 // sum exp((l-max)/T); confidence p = max softmax at T = 1.
-// VOCAB_DRAFT (one row, draft step j): y'_j = argmax, or a draw from q_j = softmax(l/T) whose
-// probabilities are kept in q_rows[j-1][:]; records the token and its confidence, and disarms
-// drafting when the confidence is below stop_conf.
+// VOCAB_DRAFT (one row, draft step j): y'_j = argmax, or (sampling == 1) a draw from q_j = softmax(l/T),
+// nucleus-cut, whose probabilities are kept in q_rows[j-1][:], or (sampling == 2) the argmax with the point
+// mass on it as q_j; records the token and its confidence, and disarms drafting when the confidence is
+// below stop_conf.
 __global__ void __launch_bounds__(VOCAB_THREADS)
 vocab_kernel(DevState* st, const float* __restrict__ part, int n_split, size_t split_stride,
              float* __restrict__ logits, int vocab, float inv_temp, int mode, int sampling, float* __restrict__ q_rows,
@@ -214,7 +215,11 @@ vocab_kernel(DevState* st, const float* __restrict__ part, int n_split, size_t s
     const uint64_t seed = ((uint64_t)st->seed_hi << 32) | st->seed_lo;
     const uint32_t round = (uint32_t)st->round;
     int y = am.i;
-    if (sampling) {
+    if (sampling == 2) {
+        // greedy drafts under speculative-sampling acceptance (Eq. 4 taken literally): q_j is the point mass on y'_j
+        float* qrow = q_rows + (size_t)(draft_j - 1) * vocab;
+        for (int i = tid; i < vocab; i += VOCAB_THREADS) qrow[i] = i == y ? 1.f : 0.f;
+    } else if (sampling) {
         float* qrow = q_rows + (size_t)(draft_j - 1) * vocab;
         const float inv_sum = 1.f / sT;
         for (int i = tid; i < vocab; i += VOCAB_THREADS) {

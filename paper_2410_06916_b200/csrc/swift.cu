@@ -69,7 +69,7 @@ struct swift_ctx {
     int phase, n, pending, n_prompt, round, last_k, last_max_k;
     bool round_open;
     std::vector<int> hist;           // prompt + generated tokens, pending included
-    int mode; float temperature, top_p; uint64_t seed;
+    int mode; float temperature, top_p; uint64_t seed; bool greedy_draft;
     int64_t launches;
     std::string err;
     cudaEvent_t ev[8];
@@ -250,6 +250,9 @@ DevState* state_of(swift_ctx* c) { return kptr<DevState>(c, c->kl.state); }
 
 int mr_of(int rows) { return rows <= 1 ? 1 : rows <= 2 ? 2 : rows <= 4 ? 4 : rows <= 8 ? 8 : 16; }
 int attn_mr_of(int rows) { return rows > 8 && rows <= 12 ? 12 : mr_of(rows); }   // 9 rows = a verification of 8 drafts
+
+// What the vocabulary kernel does on a draft row: 0 argmax (greedy mode), 1 draw from q, 2 argmax with q the point mass.
+int sampling_flag(const swift_ctx* ctx) { return ctx->mode == SWIFT_SAMPLING ? (ctx->greedy_draft ? 2 : 1) : 0; }
 
 // Dynamic shared memory of the vocabulary kernel: one float per token while a nucleus cut is searched (sampling with
 // top_p < 1), if the vocabulary fits; nothing otherwise.
@@ -457,7 +460,7 @@ swift_status forward_chunk(swift_ctx* ctx, int rows, const int* toks_dev, const 
         ST(run_gemm<T>(ctx, mr, GemmSite{xn, d.vocab, dm, wptr<T>(ctx, ctx->wl.lm_head), &ctx->tm_lm_head, &ctx->tm_xn}, &S));
         CU(launch_k(vocab_kernel, dim3(rows), dim3(VOCAB_THREADS), vocab_cache_bytes(ctx), ctx, st, (const float*)part, S, (size_t)ROWS * d.vocab,
                     kptr<float>(ctx, ctx->kl.logits), d.vocab, 1.0f / ctx->temperature, head.mode,
-                    ctx->mode == SWIFT_SAMPLING ? 1 : 0, kptr<float>(ctx, ctx->kl.q_rows), ctx->top_p, vocab_cache_bytes(ctx) != 0 ? 1 : 0));
+                    sampling_flag(ctx), kptr<float>(ctx, ctx->kl.q_rows), ctx->top_p, vocab_cache_bytes(ctx) != 0 ? 1 : 0));
     }
     CU(cudaGetLastError());
     return SWIFT_OK;
@@ -560,7 +563,7 @@ swift_status forward_chunk_fused(swift_ctx* ctx, int rows, const int* toks_dev, 
         ST(gemm(EPI_PLAIN, &ctx->tm_lm_head, &ctx->tm_xn, d.vocab, dm, ep));
         CU(launch_k(vocab_kernel, dim3(rows), dim3(VOCAB_THREADS), vocab_cache_bytes(ctx), ctx, st, (const float*)kptr<float>(ctx, ctx->kl.part), 1,
                     (size_t)ROWS * d.vocab, kptr<float>(ctx, ctx->kl.logits), d.vocab, 1.0f / ctx->temperature, head.mode,
-                    ctx->mode == SWIFT_SAMPLING ? 1 : 0, kptr<float>(ctx, ctx->kl.q_rows), ctx->top_p, vocab_cache_bytes(ctx) != 0 ? 1 : 0));
+                    sampling_flag(ctx), kptr<float>(ctx, ctx->kl.q_rows), ctx->top_p, vocab_cache_bytes(ctx) != 0 ? 1 : 0));
     }
     CU(cudaGetLastError());
     return SWIFT_OK;
@@ -608,7 +611,7 @@ swift_status forward_cached(swift_ctx* ctx, int rows, const int* toks_dev, const
 {
     if (!ctx->use_graphs) return forward_chunk_any(ctx, rows, toks_dev, skip, page_table, head);
     const int L = 2 * ctx->d.n_blocks;
-    FwdKey key{rows, head.run ? 1 : 0, head.mode, ctx->mode, ctx->use_tc ? 1 : 0, ctx->use_pdl ? 1 : 0, ctx->fuse ? 1 : 0, ctx->temperature, ctx->top_p, toks_dev, page_table,
+    FwdKey key{rows, head.run ? 1 : 0, head.mode, sampling_flag(ctx), ctx->use_tc ? 1 : 0, ctx->use_pdl ? 1 : 0, ctx->fuse ? 1 : 0, ctx->temperature, ctx->top_p, toks_dev, page_table,
                skip ? std::vector<uint8_t>(skip, skip + L) : std::vector<uint8_t>()};
     auto& cache = *ctx->graphs;
     ctx->graph_clock++;
@@ -970,7 +973,7 @@ swift_status swift_load(const swift_model_desc* desc, swift_devbuf weights, swif
     c->max_splits = ceil_div(desc->max_positions, ATTN_CHUNK);
     c->phase = PH_LOADED; c->n = 0; c->pending = 0; c->n_prompt = 0; c->round = 0; c->last_k = 0; c->last_max_k = 0;
     c->round_open = false;
-    c->mode = SWIFT_GREEDY; c->temperature = 1.f; c->top_p = 1.f; c->seed = 0; c->launches = 0;
+    c->mode = SWIFT_GREEDY; c->temperature = 1.f; c->top_p = 1.f; c->greedy_draft = false; c->seed = 0; c->launches = 0;
     ctx = c;
     c->use_tc = false;
     if (desc->dtype == SWIFT_BF16) {
@@ -1074,6 +1077,14 @@ swift_status swift_set_sampling(swift_ctx* ctx, int32_t mode, float temperature,
     if (!(temperature > 0.f)) return fail(ctx, SWIFT_EINVAL, "temperature must be positive");
     if (ctx->round_open) return fail(ctx, SWIFT_ESTATE, "cannot change the acceptance strategy inside a round");
     ctx->mode = mode; ctx->temperature = temperature; ctx->seed = seed;
+    return SWIFT_OK;
+}
+
+swift_status swift_set_greedy_draft(swift_ctx* ctx, int32_t on)
+{
+    if (!ctx) return SWIFT_EINVAL;
+    if (ctx->round_open) return fail(ctx, SWIFT_ESTATE, "cannot change the drafting rule inside a round");
+    ctx->greedy_draft = on != 0;
     return SWIFT_OK;
 }
 

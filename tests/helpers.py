@@ -83,7 +83,7 @@ def resync(gpu, o: so.Oracle, rounds_done: int = -1):
 
 
 def walk_rounds(o: so.Oracle, gpu, z, n_rounds: int, max_k: int, stop_conf: float = 0.0, sampling=False,
-                temperature=1.0, seed=0, first_round=1, dec_tol=1e-3, top_p=1.0):
+                temperature=1.0, seed=0, first_round=1, dec_tol=1e-3, top_p=1.0, greedy_draft=False):
     """Runs n_rounds of draft -> verify -> accept on both sides from the same state and compares every
     intermediate the oracle exposes, exempting only decisions the oracle marks as near a boundary.
     Returns counters for the caller to assert on."""
@@ -95,6 +95,12 @@ def walk_rounds(o: so.Oracle, gpu, z, n_rounds: int, max_k: int, stop_conf: floa
         dec_margins: List[float] = []
         if sampling:
             def sampler(j, q, _r=r):
+                if greedy_draft:                       # arg max of the draft; q is the point mass on it
+                    tok = so.argmax_lowest(q)
+                    q_rows.append(so.point_mass(q.numel(), tok))
+                    top2 = torch.topk(q, 2).values
+                    dec_margins.append(float(top2[0] - top2[1]) / float(top2[0]))   # relative gap of the two best
+                    return tok
                 q_rows.append(q)
                 tok, dist = so.categorical(q, so.uniform(seed, _r, j, so.DRAW_DRAFT))
                 dec_margins.append(dist)

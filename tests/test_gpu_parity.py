@@ -453,6 +453,26 @@ def test_sampling_with_nucleus_filter(tiny_pair, T, top_p):
         g.set_sampling(False)
 
 
+@pytest.mark.parametrize("T,top_p", [(1.0, 1.0), (0.6, 0.95)])
+def test_sampling_with_greedy_drafts(tiny_pair, T, top_p):
+    """Sampling acceptance with drafts chosen by arg max (Eq. 4 as written; q_j = point mass): draft tokens, accept
+    decisions (u < p_j(y')) and replacement draws follow the oracle's."""
+    o, g = tiny_pair
+    prompt = synth.prompt(TINY, 24)
+    seed = 57
+    g.set_sampling(True, T, seed, top_p, greedy_draft=True)
+    try:
+        o.prefill(prompt)
+        g.prefill(prompt); g.set_pending(o.tokens[-1])
+        z = list(synth.block_mask(TINY, synth.planted_blocks(TINY)))
+        st = walk_rounds(o, g, z, n_rounds=20, max_k=4, sampling=True, temperature=T, seed=seed, top_p=top_p,
+                         greedy_draft=True)
+        assert st["accept_cmp"] >= 15 and st["max_logit_err"] < 1e-4, st
+        assert st["accepted"] < st["drafted"]           # point-mass drafts of a flat model are mostly rejected
+    finally:
+        g.set_sampling(False)
+
+
 def test_vanilla_sampling_with_nucleus_filter(tiny_pair):
     """Plain sampling of the full model with temperature and top_p: the same tokens as the oracle's, up to draws
     that land within 1e-3 of a bracket edge."""

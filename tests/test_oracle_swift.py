@@ -254,8 +254,10 @@ def test_wrong_acceptance_rules_fail_the_chi_squared():
     assert float(((counts - expect) ** 2 / expect).sum()) > 200.0
 
 
-def test_whole_round_sampling_is_lossless_on_a_tiny_model():
-    """Second emitted token of SWIFT in sampling mode: its law, given the first token, is the target's."""
+@pytest.mark.parametrize("greedy_draft", [False, True], ids=["sampled_drafts", "argmax_drafts"])
+def test_whole_round_sampling_is_lossless_on_a_tiny_model(greedy_draft):
+    """Second emitted token of SWIFT in sampling mode: its law, given the first token, is the target's, whether the
+    drafts are drawn from the draft distribution or chosen by arg max (Eq. 4) with a point-mass q."""
     cfg = synth.ModelConfig("micro", n_blocks=2, d_model=16, n_heads=2, n_kv_heads=1, head_dim=8, ffn=24,
                             vocab=6, dtype="f32", seed=5, n_planted=1, init_std=0.6)
     w = synth.make_weights(cfg)
@@ -274,7 +276,8 @@ def test_whole_round_sampling_is_lossless_on_a_tiny_model():
     counts = np.zeros(cfg.vocab)
     for t in range(trials):
         out, _, _ = so.swift_generate(_oracle(cfg, w, 32), prompt, z,
-                                      so.GenParams(max_new=3, max_draft=2, mode="sampling", rng_seed=1000 + t))
+                                      so.GenParams(max_new=3, max_draft=2, mode="sampling", rng_seed=1000 + t,
+                                                   greedy_draft=greedy_draft))
         counts[out[1]] += 1
     expect = law.numpy() * trials
     chi2 = float(((counts - expect) ** 2 / expect).sum())
