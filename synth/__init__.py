@@ -112,6 +112,9 @@ MODELS: Dict[str, ModelConfig] = {
     "7b": ModelConfig("7b", 32, 4096, 32, 32, 128, 11008, 32000, "bf16", seed=2, n_planted=14),
     "13b": ModelConfig("13b", 40, 5120, 40, 40, 128, 13824, 32000, "bf16", seed=3, n_planted=18),
     "70b": ModelConfig("70b", 80, 8192, 64, 8, 128, 28672, 32000, "bf16", seed=6, n_planted=36),
+    # a 34B-class backbone (the paper also runs 33B/34B models, Section 5.2, without giving their shapes): 60 blocks, 56 query
+    # heads on 8 KV heads (7 per group, not a power of two), vocabulary 64000 (twice the others'), skip ratio 0.5
+    "34b": ModelConfig("34b", 60, 7168, 56, 8, 128, 20480, 64000, "bf16", seed=12, n_planted=30),
 }
 RUNS: Dict[str, Tuple[str, RunConfig]] = {
     "c1": ("tiny", RunConfig(32, 64, 4, stop_conf=0.8, n_skip_blocks=4)),
@@ -122,6 +125,7 @@ RUNS: Dict[str, Tuple[str, RunConfig]] = {
     # config 4 with the sampling setting the paper uses on code generation (Appendix B.2)
     "c4-nucleus": ("13b", RunConfig(1024, 512, 8, n_skip_blocks=20, mode="sampling", temperature=0.6, top_p=0.95, rng_seed=4)),
     "c5": ("70b", RunConfig(2048, 512, 12, n_skip_blocks=36)),
+    "w34": ("34b", RunConfig(1024, 512, 8, n_skip_blocks=30)),            # second workload shape: 34B class, r = 0.5
 }
 
 

@@ -133,9 +133,10 @@ def test_weight_streaming_gemm_kernels(shape, rows):
         g.close()
 
 
-@pytest.mark.parametrize("shape,kv", [("7b", "f32"), ("13b", "f32"), ("13b", "bf16"), ("70b", "f32")])
+@pytest.mark.parametrize("shape,kv", [("7b", "f32"), ("13b", "f32"), ("13b", "bf16"), ("70b", "f32"), ("34b", "f32")])
 def test_full_width_bf16_forward(shape, kv):
-    """Two blocks at the real 7B / 13B / 70B (grouped-query, 8 query heads per KV head) widths and vocabulary, in
+    """Two blocks at the real 7B / 13B / 70B (grouped-query, 8 query heads per KV head) / 34B-class (7 query heads per
+    KV head, 64000-token vocabulary) widths and vocabulary, in
     the launch shapes the benchmark uses: one row (drafting, vanilla) and nine rows (verification of 8 drafts),
     behind a prefix that spans several attention chunks, full model and layer-skipped."""
     cfg = synth.MODELS[shape].with_blocks(2, n_planted=1)
@@ -542,13 +543,14 @@ def test_launch_options_do_not_change_results(monkeypatch):
         assert got[2] == base[2] and got[3] == base[3], env
 
 
-FULL_DEPTH = [("7b", 14, 8, 48, 64), ("13b", 18, 8, 48, 48), ("70b", 36, 12, 29, 48)]
+FULL_DEPTH = [("7b", 14, 8, 48, 64), ("13b", 18, 8, 48, 48), ("34b", 30, 8, 48, 48), ("70b", 36, 12, 29, 48)]
 
 
 @pytest.mark.slow
 @pytest.mark.parametrize("name,n_skip,max_draft,n_prompt,need_gb", FULL_DEPTH, ids=[c[0] for c in FULL_DEPTH])
 def test_full_depth_against_oracle_and_losslessness(name, n_skip, max_draft, n_prompt, need_gb):
-    """Configs 2, 3/4 and 5 at full size (32 / 40 / 80 blocks; 13 / 26 / 138 GB of weights), in the launch
+    """Configs 2, 3/4 and 5 and the 34B-class shape at full size (32 / 40 / 80 / 60 blocks; 13 / 26 / 138 / 69 GB of
+    weights), in the launch
     configurations the benchmark times: teacher-forced logits of the last prompt rows against the oracle, from
     16-row chunks, from one verification-shaped forward (max_draft + 1 rows) and from a one-row forward; then
     SWIFT == vanilla on the GPU.  The oracle regenerates each block from the seed as its forward reaches it, so
