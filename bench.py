@@ -296,7 +296,7 @@ def main():
     g1_ms, _ = model.time_gemm(2, 1, 200)
     achieved = g_bytes / (g_ms * 1e-3) * 1e-9
     # DRAM bytes per launch of that kernel (read + write, mean of two launches) from the ncu captures summarised in
-    # profiles/gemm_tc_gate_up_9rows.md (7B and 13B widths, 9 rows); other shapes have no capture of their own
+    # the profiles folder (7B and 13B widths, 9 rows); other shapes have no capture of their own
     traffic = {"7b": 186.6e6, "13b": 289.6e6}.get(cfg.name) if run.max_draft == 8 else None
     roofline = {"bound": "hbm", "kernel": "skinny GEMM, fused gate/up projection, %d rows" % (run.max_draft + 1),
                 "achieved": achieved, "peak": hbm_peak, "peak_kind": f"{peak_kind} copy bandwidth (burst)", "unit": "GB/s",

@@ -224,6 +224,11 @@ double swift_forward_bytes(const swift_ctx* ctx, const uint8_t* skip_mask_host, 
  * step), and the algorithmic HBM bytes of those forwards.  Host arrays of `capacity` entries, any of them may be
  * NULL; returns the number of rounds recorded (which may exceed capacity; only `capacity` entries are written),
  * -1 if ctx is NULL. */
+/* The skip set the last swift_generate on this context ended with: its `skip_mask` argument, or the best candidate the
+ * on-the-fly optimisation kept (Section 4.1).  Feeding it to the next call as `skip_mask` is how an optimised set
+ * carries over from one input to the next in a stream of inputs (the dynamic input streams of Section 5.3).
+ * mask_host: [2*n_blocks] bytes, may be NULL; returns 2*n_blocks, or -1 before the first generate or if ctx is NULL. */
+int32_t swift_final_skip_mask(const swift_ctx* ctx, uint8_t* mask_host);
 int32_t swift_round_times(const swift_ctx* ctx, int32_t capacity, float* ms_draft_host, float* ms_verify_host,
                           double* bytes_draft_host, double* bytes_verify_host, int32_t* drafted_host);
 /* Times `iters` back-to-back launches of one weight-streaming GEMM of the walk (which: 0 fused QKV,

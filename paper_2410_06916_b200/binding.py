@@ -52,7 +52,7 @@ class _Stats(C.Structure):
 SYMBOLS = ("swift_weights_bytes", "swift_kv_bytes", "swift_workspace_bytes", "swift_load", "swift_free",
            "swift_last_error", "swift_pack_tensor", "swift_set_sampling", "swift_set_top_p", "swift_set_greedy_draft", "swift_forward_rows", "swift_prefill",
            "swift_set_pending", "swift_draft", "swift_verify", "swift_accept", "swift_score_skipsets", "swift_generate",
-           "swift_committed_length", "swift_launch_count", "swift_round_times", "swift_forward_bytes", "swift_read_kv", "swift_time_gemm", "swift_set_gemm_impl", "swift_gemm", "swift_gemm_static",
+           "swift_committed_length", "swift_launch_count", "swift_round_times", "swift_final_skip_mask", "swift_forward_bytes", "swift_read_kv", "swift_time_gemm", "swift_set_gemm_impl", "swift_gemm", "swift_gemm_static",
            "swift_gemm_static_error")
 
 _lib = None
@@ -88,6 +88,8 @@ def load_library(path: Optional[str] = None) -> C.CDLL:
     lib.swift_committed_length.argtypes = [vp]
     lib.swift_launch_count.argtypes = [vp]
     lib.swift_launch_count.restype = C.c_int64
+    lib.swift_final_skip_mask.argtypes = [vp, vp]
+    lib.swift_final_skip_mask.restype = C.c_int32
     lib.swift_round_times.argtypes = [vp, i32, vp, vp, vp, vp, vp]
     lib.swift_round_times.restype = C.c_int32
     lib.swift_forward_bytes.argtypes = [vp, vp, i32, i32]
@@ -328,6 +330,11 @@ class SwiftModel:
                                                  _ptr(trace), C.byref(st)))
         stats = GenStats(**{f: getattr(st, f) for f in GenStats.__dataclass_fields__})
         return out[:n_out.value].tolist(), stats, trace[:stats.rounds]
+
+    def final_skip_mask(self) -> Optional[np.ndarray]:
+        """The skip set the last generate() ended with (to seed the next input of a stream), or None."""
+        m = np.zeros(self.n_sub, dtype=np.uint8)
+        return m if self._lib.swift_final_skip_mask(self.ctx, _ptr(m)) == self.n_sub else None
 
     def round_times(self):
         """Per round of the last generate(): (ms_draft, ms_verify, bytes_draft, bytes_verify, drafted) arrays."""

@@ -81,6 +81,7 @@ struct swift_ctx {
     // per-round record of the last swift_generate (swift_round_times)
     struct RoundTime { float ms_draft, ms_verify; double bytes_draft, bytes_verify; int32_t drafted; };
     std::vector<RoundTime> round_times;
+    std::vector<uint8_t> last_mask;          // skip set in use when the last swift_generate ended (swift_final_skip_mask)
     // tensor-core GEMM path (bf16 models)
     bool use_tc;
     std::vector<CUtensorMap> tm_wqkv, tm_wo, tm_wgu, tm_wdown;
@@ -1292,6 +1293,12 @@ swift_status swift_set_gemm_impl(swift_ctx* ctx, int32_t impl)
 
 int32_t swift_committed_length(const swift_ctx* ctx) { return ctx ? ctx->n : -1; }
 int64_t swift_launch_count(const swift_ctx* ctx) { return ctx ? ctx->launches : -1; }
+int32_t swift_final_skip_mask(const swift_ctx* ctx, uint8_t* mask_host)
+{
+    if (!ctx || ctx->last_mask.empty()) return -1;
+    if (mask_host) memcpy(mask_host, ctx->last_mask.data(), ctx->last_mask.size());
+    return (int32_t)ctx->last_mask.size();
+}
 int32_t swift_round_times(const swift_ctx* ctx, int32_t capacity, float* ms_draft, float* ms_verify, double* bytes_draft,
                           double* bytes_verify, int32_t* drafted)
 {
@@ -1512,6 +1519,7 @@ swift_status swift_generate(swift_ctx* ctx, const swift_gen_params* gp, const in
         out_tokens[count++] = hs.next_token;
         commit_round(ctx, hs);
     }
+    ctx->last_mask = z;
     CU(cudaEventRecord(ev[7], ctx->stream));
     CU(cudaStreamSynchronize(ctx->stream));
     CU(cudaEventElapsedTime(&stt.ms_prefill, ev[0], ev[1]));

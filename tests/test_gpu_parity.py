@@ -296,6 +296,12 @@ def test_generate_with_on_the_fly_optimisation(tiny_pair):
     out, st, trace = g.generate(prompt, GenParams(max_new=80, max_draft=4, gamma=32, n_opt_rounds=3, skip_mask=z0,
                                                   candidate_masks=cands, stop_matchness=2.0))
     assert out == o_out and st.opt_rounds == 3
+    # the set the run ended with (what the next input of a stream starts from) is the oracle's, and a run that is
+    # given it without optimisation keeps it
+    assert g.final_skip_mask().tolist() == o_rounds[-1].z
+    kept = g.final_skip_mask()
+    g.generate(prompt, GenParams(max_new=8, max_draft=4, skip_mask=kept))
+    assert np.array_equal(g.final_skip_mask(), kept)
     scored = [r for r in o_rounds if r.matchness is not None]
     assert abs(st.best_matchness - max(max(r.matchness) for r in scored)) <= 1.0 / 32 + 1e-6
     first = next(i for i, r in enumerate(o_rounds) if r.matchness is not None)
