@@ -105,24 +105,25 @@ def workload(name: str):
     return cfg, run, z
 
 
-def oracle_sample(cfg, run, z, weights, n_ctx=16, k=2):
-    """The CPU oracle, as it stands, on a bounded slice of the workload: a short prefill, then one
-    vanilla step and one SWIFT round (k drafts + verify + accept).  Returns tokens/s of both."""
+def oracle_sample(cfg, run, z, weights, n_ctx=16, k=4, n_vanilla=3):
+    """The CPU oracle, as it stands, on a bounded slice of the workload: a short prefill, then n_vanilla
+    vanilla steps and one SWIFT round (k drafts + verify + accept).  Returns tokens/s of both."""
     from oracle import swift_oracle as so
     dtype = torch.float64 if cfg.dtype == "f32" else torch.float32
-    o = so.Oracle(so.Shape.of(cfg), weights, dtype=dtype, max_positions=n_ctx + k + 8)
+    o = so.Oracle(so.Shape.of(cfg), weights, dtype=dtype, max_positions=n_ctx + n_vanilla + k + 8)
     prompt = synth.prompt(cfg, n_ctx)
     o.prefill(prompt)
     t0 = time.perf_counter()
-    row = o.forward_rows([o.tokens[-1]], o.n)[0]
-    o.commit([], so.argmax_lowest(row))
+    for _ in range(n_vanilla):
+        row = o.forward_rows([o.tokens[-1]], o.n)[0]
+        o.commit([], so.argmax_lowest(row))
     t1 = time.perf_counter()
     d_tok, _, _ = o.draft(list(z), k)
     tl = o.verify(d_tok)
     a, nxt = so.accept_greedy(d_tok, tl)
     o.commit(d_tok[:a], nxt)
     t2 = time.perf_counter()
-    return {"vanilla": 1.0 / (t1 - t0), "swift": (a + 1) / (t2 - t1), "seconds": t2 - t0, "accepted": a, "k": k}
+    return {"vanilla": n_vanilla / (t1 - t0), "swift": (a + 1) / (t2 - t1), "seconds": t2 - t0, "accepted": a, "k": k}
 
 
 def micro(cfg, run, args, hbm_peak):
@@ -186,7 +187,7 @@ def main():
             if i >= args.warmup:
                 vals.append(s)
         v = statistics.mean(x["swift"] for x in vals) * (small.n_blocks / cfg.n_blocks if small is not cfg else 1.0)
-        sample = "per step: prefill of 16 tokens, then one vanilla step and one SWIFT round of 2 drafts + verify + accept" + \
+        sample = "per step: prefill of 16 tokens, then 3 vanilla steps and one SWIFT round of 4 drafts + verify + accept" + \
                  ("" if small is cfg else f"; on an 8-block copy of the model, scaled by depth (extrapolated)")
         print(json.dumps({"impl": "reference", "metric": METRIC, "value": v, "unit": UNIT, "n_gpus": 0, "steps": args.steps,
                           "warmup": args.warmup, "ms_per_step": 1e3 * statistics.mean(x["seconds"] for x in vals),
@@ -338,7 +339,7 @@ def main():
         scale = 1.0 if small is cfg else small.n_blocks / cfg.n_blocks
         out["cpu_baseline"] = {"value": s["swift"] * scale, "unit": UNIT, "cores": torch.get_num_threads(), "kind": "oracle",
                                "vanilla_value": s["vanilla"] * scale,
-                               "sample": "prefill of 16 tokens, then one vanilla step and one SWIFT round of 2 drafts + verify "
+                               "sample": "prefill of 16 tokens, then 3 vanilla steps and one SWIFT round of 4 drafts + verify "
                                          "+ accept (%.1f s of CPU work)%s" % (s["seconds"], "" if small is cfg else
                                                                                "; 8-block copy scaled by depth (extrapolated)")}
     if rank == 0:
