@@ -74,7 +74,7 @@ struct swift_ctx {
     std::string err;
     cudaEvent_t ev[8];
     // captured forwards; programmatic dependent launch between the kernels of a forward
-    bool use_graphs, use_pdl, fuse, fuse_combine, prefetch_next;
+    bool use_graphs, use_pdl, pdl_next, pdl_gemms, fuse, fuse_combine, prefetch_next;
     int attn_rows_per_cta, prefetch_tiles;
     std::vector<FwdGraph>* graphs;
     uint64_t graph_clock;
@@ -278,7 +278,8 @@ cudaError_t launch_k(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t sme
     attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
-    cfg.numAttrs = ctx->use_pdl ? 1 : 0;
+    cfg.numAttrs = (ctx->use_pdl || ctx->pdl_next) ? 1 : 0;
+    ctx->pdl_next = false;
     ctx->launches++;
     return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
 }
@@ -320,6 +321,7 @@ template <int EPI, typename TKV>
 swift_status launch_gemm_tc(swift_ctx* ctx, const GemmSite& g, const EpiParams& ep, const CUtensorMap* next_map = nullptr)
 {
     if (ceil_div(g.N, TC_TILE_N) > TC_MAX_TILES) return fail(ctx, SWIFT_EUNSUPPORTED, "GEMM with %d output tiles", ceil_div(g.N, TC_TILE_N));
+    if (ctx->pdl_gemms) ctx->pdl_next = true;     // this launch may begin before its predecessor has finished (see swift_load)
     CU(launch_k(gemm_tc_kernel<EPI, TKV>, dim3(TC_GRID), dim3(TC_THREADS), (size_t)TC_SMEM_BYTES, ctx, state_of(ctx), *g.mapW, *g.mapX,
                 kptr<float>(ctx, ctx->kl.part), kptr<float>(ctx, ctx->kl.slabs), kptr<int>(ctx, ctx->kl.counters), g.N, g.K, ep,
                 next_map ? *next_map : *g.mapW));
@@ -995,7 +997,13 @@ swift_status swift_load(const swift_model_desc* desc, swift_devbuf weights, swif
         const char* e = getenv("SWIFT_PREFETCH_TILES");      // 16 KB tiles of the next GEMM each CTA asks L2 for
         c->prefetch_tiles = e ? std::max(0, std::min(256, atoi(e))) : 16;
     }
-    c->use_pdl = getenv("SWIFT_PDL") != nullptr;   // programmatic dependent launch: measured neutral to slightly negative on whole forwards, so opt-in
+    // Programmatic dependent launch.  On by default for the tensor-core GEMM launches only: a GEMM's CTAs then start during
+    // the tail of whatever precedes them and have their barriers, descriptors and first weight tile under way when its
+    // results become visible (+1.6 to 1.9 % on whole 13B forwards).  As the secondary of such an edge the attention and
+    // split-merge launches lose (their early CTAs sit beside the running GEMM), so SWIFT_PDL=1 (every launch) stays opt-in.
+    c->pdl_next = false;
+    c->pdl_gemms = getenv("SWIFT_NO_PDL_GEMMS") == nullptr;
+    c->use_pdl = getenv("SWIFT_PDL") != nullptr;
     c->fuse = getenv("SWIFT_NO_FUSE") == nullptr && desc->head_dim <= TC_TILE_N;
     c->graphs = new std::vector<FwdGraph>();
     c->graph_clock = 0;

@@ -543,7 +543,7 @@ def test_launch_options_do_not_change_results(monkeypatch):
     base = run({})
     assert base[2] == base[3]                                    # lossless on the GPU
     for env in ({"SWIFT_NO_GRAPHS": "1"}, {"SWIFT_NO_FUSE_COMBINE": "1"}, {"SWIFT_ATTN_ROWS": "4"},
-                {"SWIFT_PREFETCH_TILES": "0"}, {"SWIFT_PREFETCH_TILES": "64"}, {"SWIFT_PDL": "1"}):
+                {"SWIFT_PREFETCH_TILES": "0"}, {"SWIFT_PREFETCH_TILES": "64"}, {"SWIFT_PDL": "1"}, {"SWIFT_NO_PDL_GEMMS": "1"}):
         got = run(env)
         assert np.array_equal(got[0], base[0]) and np.array_equal(got[1], base[1]), env
         assert got[2] == base[2] and got[3] == base[3], env
