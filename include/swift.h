@@ -179,19 +179,25 @@ typedef struct {
     int32_t max_draft;      /* N_D */
     float stop_conf;        /* epsilon; 0 disables early stopping */
     int32_t vanilla;        /* 1 = plain autoregressive decoding of the full model (the baseline) */
-    /* on-the-fly optimisation (Section 4.1); n_opt_rounds = 0 keeps skip_mask fixed */
+    /* on-the-fly optimisation (Section 4.1); n_opt_rounds = 0 keeps skip_mask fixed.  An optimisation round scores the
+     * set in use together with the n_candidates proposals on the last gamma generated tokens and keeps the best of them
+     * (the set in use on ties, then the earliest proposal).  It ends once the kept set scores above stop_matchness,
+     * after n_opt_rounds rounds, or after opt_patience rounds in a row without a replacement (0 = no such rule): the
+     * stop rules of Appendix B.2. */
     int32_t gamma, n_candidates, n_opt_rounds;
     float stop_matchness;
+    int32_t opt_patience;
     const uint8_t* skip_mask;       /* host, [2*n_blocks]: the (initial) draft skip set */
     const uint8_t* candidate_masks; /* host, [n_opt_rounds][n_candidates][2*n_blocks] or NULL */
 } swift_gen_params;
 
 typedef struct {
     int32_t tokens, rounds, drafted, accepted, opt_rounds, reserved;
-    float best_matchness;
+    float best_matchness;   /* matchness of the set the last optimisation round kept (-1 if none ran) */
     float ms_prefill, ms_decode, ms_draft, ms_verify, ms_score; /* CUDA-event times on the stream */
-    double bytes_draft, bytes_verify;  /* algorithmic HBM bytes of all draft / verify forwards */
+    double bytes_draft, bytes_verify;  /* algorithmic HBM bytes of all draft / verify forwards (swift_forward_bytes, 2-byte K,V) */
     int64_t kernel_launches;           /* kernels enqueued by the whole call */
+    int64_t h2d_bytes, d2h_bytes;      /* bytes the call copied host -> device and device -> host (prompt and tokens included) */
 } swift_stats;
 
 /* prefill + rounds until max_new tokens are out.  out_tokens_host[max_new]; *n_out_host = max_new.
@@ -215,8 +221,12 @@ swift_status swift_gemm(swift_ctx* ctx, int32_t which, int32_t block, const floa
 /* Introspection used by tests and the benchmark. */
 int32_t swift_committed_length(const swift_ctx* ctx);               /* n; -1 if ctx is NULL */
 int64_t swift_launch_count(const swift_ctx* ctx);                   /* kernels enqueued since load */
+/* HBM bytes one forward of n_rows rows behind n_context cached positions must move: weights of the kept sub-layers
+ * and the output head, cached K,V of the kept attention sub-layers, embedding rows in, logits out.  kv_elem_bytes =
+ * bytes counted per cached K or V element: 2 is what the method needs (a 16-bit cache) and what the per-round records
+ * and swift_stats use; 0 counts the cache as this context stores it (4 with kv_dtype SWIFT_F32). */
 double swift_forward_bytes(const swift_ctx* ctx, const uint8_t* skip_mask_host, int32_t n_rows,
-                           int32_t n_context); /* algorithmic HBM bytes of one forward */
+                           int32_t n_context, int32_t kv_elem_bytes);
 /* Per-round record of the last swift_generate on this context, for judging every forward and not only their sum
  * (the drafting stage dominates latency, paper Section 5.3; the metrics M and alpha are per round, Appendix B.3).
  * Round i (a vanilla step counts as a round with no drafts): CUDA-event time on the stream of its drafting phase

@@ -363,6 +363,7 @@ class GenParams:
     gamma: int = 32
     stop_matchness: float = 0.95
     max_opt_rounds: int = 0       # 0 = skip set fixed
+    patience: int = 0             # stop optimising after this many rounds in a row that kept the incumbent (0 = never)
 
 
 @dataclass
@@ -411,6 +412,12 @@ def swift_generate(o: Oracle, prompt: Sequence[int], z0: Sequence[int], gp: GenP
     roll the KV cache back.  Emits exactly gp.max_new tokens: the draft length is capped at
     remaining - 1, and with one token left a plain full-model step is taken.
     `candidates(round) -> masks [C, L]` supplies the proposals of one optimisation round.
+
+    An optimisation round scores the set in use together with the proposals on the same window (the set in
+    use is entry 0 of the round's `matchness`) and keeps the highest-scoring one (Section 4.1), the earliest
+    among equals: the set in use is replaced only by a proposal that beats it on the tokens both were scored
+    on.  Optimisation ends once the kept set scores above gp.stop_matchness, after gp.max_opt_rounds rounds,
+    or after gp.patience rounds in a row without a replacement (the stop rules of Appendix B.2).
     """
     sampling = gp.mode == "sampling"
     logits = o.prefill(prompt)
@@ -418,7 +425,7 @@ def swift_generate(o: Oracle, prompt: Sequence[int], z0: Sequence[int], gp: GenP
         p = nucleus(torch.softmax(logits[-1].to(torch.float64) / gp.temperature, -1), gp.top_p)[0]
         o.tokens[-1] = categorical(p, uniform(gp.rng_seed, 0, 0, DRAW_BONUS))[0]
     z = [int(v) for v in z0]
-    best_score, opt_rounds, optimising = -1.0, 0, gp.max_opt_rounds > 0
+    best_score, opt_rounds, optimising, stale = -1.0, 0, gp.max_opt_rounds > 0, 0
     rounds: List[Round] = []
     n_prompt = len(prompt)
     r = 0
@@ -427,13 +434,13 @@ def swift_generate(o: Oracle, prompt: Sequence[int], z0: Sequence[int], gp: GenP
         remaining = gp.max_new - (len(o.tokens) - n_prompt)
         scores = None
         if optimising and len(o.tokens) - n_prompt >= gp.gamma and candidates is not None:
-            masks = candidates(opt_rounds)
+            masks = [list(z)] + [[int(v) for v in m] for m in candidates(opt_rounds)]
             scores, _ = o.score_skipsets(masks, gp.gamma)
-            c_best = max(range(len(scores)), key=lambda c: (scores[c], -c))
-            if scores[c_best] > best_score:               # strictly better only
-                best_score, z = scores[c_best], [int(v) for v in masks[c_best]]
+            c_best = max(range(len(scores)), key=lambda c: (scores[c], -c))   # entry 0, the set in use, wins ties
+            best_score, z = scores[c_best], masks[c_best]
+            stale = 0 if c_best != 0 else stale + 1
             opt_rounds += 1
-            if best_score > gp.stop_matchness or opt_rounds >= gp.max_opt_rounds:
+            if best_score > gp.stop_matchness or opt_rounds >= gp.max_opt_rounds or (gp.patience > 0 and stale >= gp.patience):
                 optimising = False
         k_max = min(gp.max_draft, remaining - 1)
         q_rows: List[torch.Tensor] = []

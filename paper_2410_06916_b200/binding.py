@@ -39,13 +39,15 @@ class _DevBuf(C.Structure):
 class _GenParams(C.Structure):
     _fields_ = [("max_new", C.c_int32), ("max_draft", C.c_int32), ("stop_conf", C.c_float), ("vanilla", C.c_int32),
                 ("gamma", C.c_int32), ("n_candidates", C.c_int32), ("n_opt_rounds", C.c_int32),
-                ("stop_matchness", C.c_float), ("skip_mask", C.c_void_p), ("candidate_masks", C.c_void_p)]
+                ("stop_matchness", C.c_float), ("opt_patience", C.c_int32), ("skip_mask", C.c_void_p),
+                ("candidate_masks", C.c_void_p)]
 
 
 class _Stats(C.Structure):
     _fields_ = [(n, C.c_int32) for n in ("tokens", "rounds", "drafted", "accepted", "opt_rounds", "reserved")] + \
                [(n, C.c_float) for n in ("best_matchness", "ms_prefill", "ms_decode", "ms_draft", "ms_verify", "ms_score")] + \
-               [("bytes_draft", C.c_double), ("bytes_verify", C.c_double), ("kernel_launches", C.c_int64)]
+               [("bytes_draft", C.c_double), ("bytes_verify", C.c_double), ("kernel_launches", C.c_int64),
+                ("h2d_bytes", C.c_int64), ("d2h_bytes", C.c_int64)]
 
 
 # every symbol include/swift.h declares
@@ -92,7 +94,7 @@ def load_library(path: Optional[str] = None) -> C.CDLL:
     lib.swift_final_skip_mask.restype = C.c_int32
     lib.swift_round_times.argtypes = [vp, i32, vp, vp, vp, vp, vp]
     lib.swift_round_times.restype = C.c_int32
-    lib.swift_forward_bytes.argtypes = [vp, vp, i32, i32]
+    lib.swift_forward_bytes.argtypes = [vp, vp, i32, i32, i32]
     lib.swift_forward_bytes.restype = C.c_double
     lib.swift_set_gemm_impl.argtypes = [vp, i32]
     lib.swift_gemm_static.argtypes = [vp, i32, i32, i32, vp, i32, vp, vp]
@@ -123,6 +125,7 @@ class GenParams:
     gamma: int = 32
     n_opt_rounds: int = 0
     stop_matchness: float = 0.95
+    opt_patience: int = 0                             # optimisation rounds without a replacement before it stops (0 = no rule)
     skip_mask: Optional[np.ndarray] = None            # uint8 [2*n_blocks]
     candidate_masks: Optional[np.ndarray] = None      # uint8 [n_opt_rounds, C, 2*n_blocks]
 
@@ -143,6 +146,8 @@ class GenStats:
     bytes_draft: float
     bytes_verify: float
     kernel_launches: int
+    h2d_bytes: int = 0
+    d2h_bytes: int = 0
 
 
 STATIC_SCRATCH_BYTES = 8 * 1024 * 1024
@@ -256,9 +261,10 @@ class SwiftModel:
     def launches(self) -> int:
         return self._lib.swift_launch_count(self.ctx)
 
-    def forward_bytes(self, skip_mask, n_rows: int, n_context: int) -> float:
+    def forward_bytes(self, skip_mask, n_rows: int, n_context: int, kv_elem_bytes: int = 2) -> float:
+        """HBM bytes one forward must move; cached K,V counted at kv_elem_bytes per element (0 = as this context stores them)."""
         m = None if skip_mask is None else _u8(skip_mask)
-        return self._lib.swift_forward_bytes(self.ctx, _ptr(m), n_rows, n_context)
+        return self._lib.swift_forward_bytes(self.ctx, _ptr(m), n_rows, n_context, kv_elem_bytes)
 
     # ------------------------------------------------------------------ the steps
     def forward_rows(self, tokens: Sequence[int], pos0: int, skip_mask=None, write_kv: bool = True,
@@ -320,7 +326,7 @@ class SwiftModel:
         cands = None if gp.candidate_masks is None else _u8(gp.candidate_masks)
         n_cand = 0 if cands is None else cands.reshape(gp.n_opt_rounds, -1, self.n_sub).shape[1]
         cp = _GenParams(gp.max_new, gp.max_draft, gp.stop_conf, 1 if gp.vanilla else 0, gp.gamma, n_cand,
-                        gp.n_opt_rounds if cands is not None else 0, gp.stop_matchness, _ptr(skip), _ptr(cands))
+                        gp.n_opt_rounds if cands is not None else 0, gp.stop_matchness, gp.opt_patience, _ptr(skip), _ptr(cands))
         out = np.zeros(gp.max_new, dtype=np.int32)
         trace = np.zeros((gp.max_new, 4), dtype=np.int32)
         n_out = C.c_int32()

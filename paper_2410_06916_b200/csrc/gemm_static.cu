@@ -30,6 +30,7 @@ namespace {
 constexpr size_t CONTROL_BYTES = 1024;               // DevState at the front of the array
 constexpr int KC = 512;                              // k elements per split: 16 rows x 512 fp32 = 32 KB of shared memory
 constexpr int MAX_DEVICES = 64;
+static_assert(sizeof(DevState) <= CONTROL_BYTES, "the control block must end before the first partial-sum slab");
 
 // The scratch itself.  In host code this name is only a handle for cudaGetSymbolAddress: it is not a
 // device address and must never be passed to a kernel.

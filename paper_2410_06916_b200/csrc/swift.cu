@@ -70,7 +70,7 @@ struct swift_ctx {
     bool round_open;
     std::vector<int> hist;           // prompt + generated tokens, pending included
     int mode; float temperature, top_p; uint64_t seed; bool greedy_draft;
-    int64_t launches;
+    int64_t launches, h2d_bytes, d2h_bytes;
     std::string err;
     cudaEvent_t ev[8];
     // captured forwards; programmatic dependent launch between the kernels of a forward
@@ -99,6 +99,13 @@ swift_status fail(swift_ctx* c, swift_status s, const char* fmt, ...)
     va_end(ap);
     if (c) c->err = buf; else g_load_error = buf;
     return s;
+}
+
+// Host <-> device copy on the context's stream, counted: the totals are what a whole swift_generate call moved.
+cudaError_t copy_async(swift_ctx* c, void* dst, const void* src, size_t bytes, cudaMemcpyKind kind)
+{
+    (kind == cudaMemcpyHostToDevice ? c->h2d_bytes : c->d2h_bytes) += (int64_t)bytes;
+    return cudaMemcpyAsync(dst, src, bytes, kind, c->stream);
 }
 
 #define CU(call)                                                                                   \
@@ -671,7 +678,7 @@ struct HostState { DevState s; };
 
 swift_status read_state(swift_ctx* ctx, DevState* out)
 {
-    CU(cudaMemcpyAsync(out, state_of(ctx), sizeof(DevState), cudaMemcpyDeviceToHost, ctx->stream));
+    CU(copy_async(ctx, out, state_of(ctx), sizeof(DevState), cudaMemcpyDeviceToHost));
     CU(cudaStreamSynchronize(ctx->stream));
     if (out->error) {
         const int code = out->error;
@@ -699,7 +706,7 @@ swift_status prepare_scratch(swift_ctx* ctx, int p_begin, int p_end)
     std::vector<int> pt(ctx->n_pages_main);
     for (int i = 0; i < ctx->n_pages_main; ++i) pt[i] = i;
     for (int p = first; p <= last; ++p) pt[p] = ctx->n_pages_main + (p - first);
-    CU(cudaMemcpyAsync(kptr<int>(ctx, ctx->kl.pt_score), pt.data(), pt.size() * 4, cudaMemcpyHostToDevice, ctx->stream));
+    CU(copy_async(ctx, kptr<int>(ctx, ctx->kl.pt_score), pt.data(), pt.size() * 4, cudaMemcpyHostToDevice));
     if (p_begin % P) {
         const size_t v16 = page_bytes(&ctx->d) / 16;
         page_copy_kernel<<<296, 256, 0, ctx->stream>>>(reinterpret_cast<uint4*>(ctx->kvbase), v16, first, ctx->n_pages_main);
@@ -717,17 +724,17 @@ swift_status run_rows(swift_ctx* ctx, const int32_t* tokens, int n_rows, int pos
     for (int c0 = 0; c0 < n_rows; c0 += ROWS) {
         const int rows = std::min(ROWS, n_rows - c0);
         const bool last = c0 + rows == n_rows;
-        CU(cudaMemcpyAsync(st->row_tok, tokens + c0, rows * 4, cudaMemcpyHostToDevice, ctx->stream));
+        CU(copy_async(ctx, st->row_tok, tokens + c0, rows * 4, cudaMemcpyHostToDevice));
         set_rows_kernel<<<1, 1, 0, ctx->stream>>>(st, pos0 + c0, rows);
         ctx->launches++;
         HeadOpts head;
         head.run = head_mode == 2 || (head_mode == 1 && last);
         ST(forward_cached(ctx, rows, st->row_tok, skip, page_table, head));
         if (head.run && logits_host)
-            CU(cudaMemcpyAsync(logits_host + (size_t)c0 * ctx->d.vocab, kptr<float>(ctx, ctx->kl.logits),
-                               (size_t)rows * ctx->d.vocab * 4, cudaMemcpyDeviceToHost, ctx->stream));
+            CU(copy_async(ctx, logits_host + (size_t)c0 * ctx->d.vocab, kptr<float>(ctx, ctx->kl.logits),
+                               (size_t)rows * ctx->d.vocab * 4, cudaMemcpyDeviceToHost));
         if (head.run && argmax_host)
-            CU(cudaMemcpyAsync(argmax_host + c0, st->argmax, rows * 4, cudaMemcpyDeviceToHost, ctx->stream));
+            CU(copy_async(ctx, argmax_host + c0, st->argmax, rows * 4, cudaMemcpyDeviceToHost));
         if (last && last_chunk_rows) *last_chunk_rows = rows;
     }
     return SWIFT_OK;
@@ -807,8 +814,8 @@ swift_status enqueue_score(swift_ctx* ctx, const uint8_t* masks, int C, int gamm
     int* tok_dev = kptr<int>(ctx, ctx->kl.score_tok);
     int* truth_dev = kptr<int>(ctx, ctx->kl.score_truth);
     int* out_dev = kptr<int>(ctx, ctx->kl.score_out);
-    CU(cudaMemcpyAsync(tok_dev, ctx->hist.data() + (n - gamma), gamma * 4, cudaMemcpyHostToDevice, ctx->stream));
-    CU(cudaMemcpyAsync(truth_dev, ctx->hist.data() + (n - gamma + 1), gamma * 4, cudaMemcpyHostToDevice, ctx->stream));
+    CU(copy_async(ctx, tok_dev, ctx->hist.data() + (n - gamma), gamma * 4, cudaMemcpyHostToDevice));
+    CU(copy_async(ctx, truth_dev, ctx->hist.data() + (n - gamma + 1), gamma * 4, cudaMemcpyHostToDevice));
     ST(prepare_scratch(ctx, n - gamma, n));
     for (int c = 0; c < C; ++c) {
         for (int c0 = 0; c0 < gamma; c0 += ROWS) {
@@ -827,10 +834,13 @@ swift_status enqueue_score(swift_ctx* ctx, const uint8_t* masks, int C, int gamm
     return SWIFT_OK;
 }
 
-double forward_bytes(const swift_ctx* ctx, const uint8_t* skip, int n_rows, int n_context)
+// Bytes one forward must move (weights of the kept sub-layers, output head, cached K,V of the kept attention
+// sub-layers, embedding rows in, logits out).  kv_elem_bytes: size of a cached K or V element to count; 0 = as stored.
+// The records of a run count 2 bytes (a 16-bit cache, what the method needs); an fp32 cache moves twice that.
+double forward_bytes(const swift_ctx* ctx, const uint8_t* skip, int n_rows, int n_context, int kv_elem_bytes = 2)
 {
     const swift_model_desc& d = ctx->d;
-    const double es = (double)ctx->esize, kes = (double)kv_esize_of(&ctx->d);
+    const double es = (double)ctx->esize, kes = kv_elem_bytes > 0 ? (double)kv_elem_bytes : (double)kv_esize_of(&ctx->d);
     const double dm = d.d_model, qd = (double)d.n_heads * d.head_dim, kd = (double)d.n_kv_heads * d.head_dim;
     const double attn_w = (qd + 2 * kd) * dm + dm * qd, mlp_w = 3.0 * d.ffn * dm;
     double bytes = (double)d.vocab * dm * es;                      // output head
@@ -976,7 +986,7 @@ swift_status swift_load(const swift_model_desc* desc, swift_devbuf weights, swif
     c->max_splits = ceil_div(desc->max_positions, ATTN_CHUNK);
     c->phase = PH_LOADED; c->n = 0; c->pending = 0; c->n_prompt = 0; c->round = 0; c->last_k = 0; c->last_max_k = 0;
     c->round_open = false;
-    c->mode = SWIFT_GREEDY; c->temperature = 1.f; c->top_p = 1.f; c->greedy_draft = false; c->seed = 0; c->launches = 0;
+    c->mode = SWIFT_GREEDY; c->temperature = 1.f; c->top_p = 1.f; c->greedy_draft = false; c->seed = 0; c->launches = 0; c->h2d_bytes = 0; c->d2h_bytes = 0;
     ctx = c;
     c->use_tc = false;
     if (desc->dtype == SWIFT_BF16) {
@@ -1191,6 +1201,9 @@ swift_status swift_verify(swift_ctx* ctx, const int32_t* tokens_host, int32_t k,
         if (k < 0 || k > SWIFT_MAX_ROWS - 1) return fail(ctx, SWIFT_ECAPACITY, "k %d outside 0..%d", k, SWIFT_MAX_ROWS - 1);
         if (ctx->mode == SWIFT_SAMPLING && k > 0 && ctx->phase != PH_DRAFTED)
             return fail(ctx, SWIFT_ESTATE, "sampling acceptance needs the draft distributions of swift_draft");
+        // acceptance compares p_j with the distribution q_j kept from draft step j: there are only last_k of those
+        if (ctx->mode == SWIFT_SAMPLING && k > ctx->last_k)
+            return fail(ctx, SWIFT_ECAPACITY, "sampling acceptance of %d tokens, but swift_draft produced %d draft distributions", k, ctx->last_k);
         if (k > 0) ST(check_tokens(ctx, tokens_host, k));
         if (ctx->n + k + 1 > ctx->d.max_positions) return fail(ctx, SWIFT_ECAPACITY, "KV cache too small");
         if (ctx->phase == PH_READY) {
@@ -1198,7 +1211,7 @@ swift_status swift_verify(swift_ctx* ctx, const int32_t* tokens_host, int32_t k,
             launch_begin_round(ctx, 0.f);
             ctx->round_open = true;
         }
-        if (k > 0) CU(cudaMemcpyAsync(state_of(ctx)->draft_tok + 1, tokens_host, k * 4, cudaMemcpyHostToDevice, ctx->stream));
+        if (k > 0) CU(copy_async(ctx, state_of(ctx)->draft_tok + 1, tokens_host, k * 4, cudaMemcpyHostToDevice));
         rows_launch = k + 1; forced_k = k;
     } else {
         if (ctx->phase != PH_DRAFTED) return fail(ctx, SWIFT_ESTATE, "no draft to verify: call swift_draft or pass tokens");
@@ -1212,7 +1225,7 @@ swift_status swift_verify(swift_ctx* ctx, const int32_t* tokens_host, int32_t k,
     const int rows = hs.n_drafted + 1;
     if (target_argmax) for (int r = 0; r < rows; ++r) target_argmax[r] = hs.argmax[r];
     if (logits_host) {
-        CU(cudaMemcpyAsync(logits_host, kptr<float>(ctx, ctx->kl.logits), (size_t)rows * ctx->d.vocab * 4, cudaMemcpyDeviceToHost, ctx->stream));
+        CU(copy_async(ctx, logits_host, kptr<float>(ctx, ctx->kl.logits), (size_t)rows * ctx->d.vocab * 4, cudaMemcpyDeviceToHost));
         CU(cudaStreamSynchronize(ctx->stream));
     }
     return SWIFT_OK;
@@ -1241,7 +1254,7 @@ swift_status swift_score_skipsets(swift_ctx* ctx, const uint8_t* masks, int32_t 
     if (gamma > ctx->n) return fail(ctx, SWIFT_EINVAL, "gamma %d exceeds the %d cached positions", gamma, ctx->n);
     ST(enqueue_score(ctx, masks, C, gamma));
     std::vector<int> counts(C);
-    CU(cudaMemcpyAsync(counts.data(), kptr<int>(ctx, ctx->kl.score_out), C * 4, cudaMemcpyDeviceToHost, ctx->stream));
+    CU(copy_async(ctx, counts.data(), kptr<int>(ctx, ctx->kl.score_out), C * 4, cudaMemcpyDeviceToHost));
     DevState hs;
     ST(read_state(ctx, &hs));
     for (int c = 0; c < C; ++c) matchness[c] = (float)counts[c] / (float)gamma;
@@ -1261,7 +1274,7 @@ swift_status swift_gemm(swift_ctx* ctx, int32_t which, int32_t block, const floa
     float* X = which == 1 ? kptr<float>(ctx, ctx->kl.xa) : which == 3 ? kptr<float>(ctx, ctx->kl.act) : kptr<float>(ctx, ctx->kl.xn);
     const size_t woff = which == 0 ? ctx->wl.wqkv[block] : which == 1 ? ctx->wl.wo[block] : which == 2 ? ctx->wl.wgu[block]
                         : which == 3 ? ctx->wl.wdown[block] : ctx->wl.lm_head;
-    CU(cudaMemcpyAsync(X, x_host, (size_t)n_rows * K * 4, cudaMemcpyHostToDevice, ctx->stream));
+    CU(copy_async(ctx, X, x_host, (size_t)n_rows * K * 4, cudaMemcpyHostToDevice));
     set_rows_kernel<<<1, 1, 0, ctx->stream>>>(state_of(ctx), 0, n_rows);
     ctx->launches++;
     GemmSite g{X, N, K, ctx->wbase + woff, nullptr, nullptr};
@@ -1280,8 +1293,7 @@ swift_status swift_gemm(swift_ctx* ctx, int32_t which, int32_t block, const floa
     std::vector<float> slab((size_t)n_rows * N);
     std::fill(y_host, y_host + (size_t)n_rows * N, 0.f);
     for (int s = 0; s < S; ++s) {          // slabs are added in slab order, as the consumers on the device do
-        CU(cudaMemcpyAsync(slab.data(), kptr<float>(ctx, ctx->kl.part) + (size_t)s * ROWS * N, slab.size() * 4,
-                           cudaMemcpyDeviceToHost, ctx->stream));
+        CU(copy_async(ctx, slab.data(), kptr<float>(ctx, ctx->kl.part) + (size_t)s * ROWS * N, slab.size() * 4, cudaMemcpyDeviceToHost));
         CU(cudaStreamSynchronize(ctx->stream));
         for (size_t i = 0; i < slab.size(); ++i) y_host[i] += slab[i];
     }
@@ -1322,9 +1334,9 @@ int32_t swift_round_times(const swift_ctx* ctx, int32_t capacity, float* ms_draf
     }
     return n;
 }
-double swift_forward_bytes(const swift_ctx* ctx, const uint8_t* skip, int32_t n_rows, int32_t n_context)
+double swift_forward_bytes(const swift_ctx* ctx, const uint8_t* skip, int32_t n_rows, int32_t n_context, int32_t kv_elem_bytes)
 {
-    return ctx ? forward_bytes(ctx, skip, n_rows, n_context) : 0.0;
+    return ctx ? forward_bytes(ctx, skip, n_rows, n_context, kv_elem_bytes) : 0.0;
 }
 
 } // extern "C"
@@ -1349,7 +1361,7 @@ swift_status swift_read_kv(swift_ctx* ctx, int32_t block, int32_t which, int32_t
             kv_read_kernel<float><<<64, 256, 0, ctx->stream>>>(reinterpret_cast<const float*>(ctx->kvbase), pt_main(ctx),
                                                                ctx->kv, block, which, pos0 + c0, cnt, stage);
         ctx->launches++;
-        CU(cudaMemcpyAsync(out_host + (size_t)c0 * per_pos, stage, (size_t)cnt * per_pos * 4, cudaMemcpyDeviceToHost, ctx->stream));
+        CU(copy_async(ctx, out_host + (size_t)c0 * per_pos, stage, (size_t)cnt * per_pos * 4, cudaMemcpyDeviceToHost));
         CU(cudaStreamSynchronize(ctx->stream));
     }
     return SWIFT_OK;
@@ -1425,12 +1437,12 @@ swift_status swift_generate(swift_ctx* ctx, const swift_gen_params* gp, const in
         if (!gp->skip_mask) return fail(ctx, SWIFT_EINVAL, "skip_mask is null");
         if (gp->max_draft < 0 || gp->max_draft > d.max_draft) return fail(ctx, SWIFT_ECAPACITY, "max_draft %d outside 0..%d", gp->max_draft, d.max_draft);
         if (gp->n_opt_rounds > 0) {
-            if (!gp->candidate_masks || gp->n_candidates < 1 || gp->n_candidates > 1024) return fail(ctx, SWIFT_EINVAL, "candidate masks missing");
+            if (!gp->candidate_masks || gp->n_candidates < 1 || gp->n_candidates > 1023) return fail(ctx, SWIFT_EINVAL, "candidate masks missing");
             if (gp->gamma < 1 || gp->gamma > MAX_SCORE_ROWS) return fail(ctx, SWIFT_ECAPACITY, "gamma must be in 1..%d", MAX_SCORE_ROWS);
         }
     }
     const int L = 2 * d.n_blocks;
-    const int64_t launches0 = ctx->launches;
+    const int64_t launches0 = ctx->launches, h2d0 = ctx->h2d_bytes, d2h0 = ctx->d2h_bytes;
     swift_stats stt;
     memset(&stt, 0, sizeof stt);
     stt.best_matchness = -1.f;
@@ -1448,6 +1460,8 @@ swift_status swift_generate(swift_ctx* ctx, const swift_gen_params* gp, const in
     if (!gp->vanilla) memcpy(z.data(), gp->skip_mask, L);
     bool optimising = !gp->vanilla && gp->n_opt_rounds > 0;
     std::vector<int> counts;
+    std::vector<uint8_t> round_masks;
+    int stale_rounds = 0;
     DevState hs;
     while (count < gp->max_new) {
         const int remaining = gp->max_new - count;
@@ -1478,24 +1492,29 @@ swift_status swift_generate(swift_ctx* ctx, const swift_gen_params* gp, const in
         } else {
             if (optimising && count >= gp->gamma) {
                 CU(cudaEventRecord(ev[2], ctx->stream));
-                const uint8_t* masks = gp->candidate_masks + (size_t)stt.opt_rounds * gp->n_candidates * L;
-                ST(enqueue_score(ctx, masks, gp->n_candidates, gp->gamma));
-                counts.resize(gp->n_candidates);
-                CU(cudaMemcpyAsync(counts.data(), kptr<int>(ctx, ctx->kl.score_out), gp->n_candidates * 4, cudaMemcpyDeviceToHost, ctx->stream));
+                // entry 0 is the set in use, scored on the same window as the round's proposals
+                const int n_scored = gp->n_candidates + 1;
+                round_masks.resize((size_t)n_scored * L);
+                memcpy(round_masks.data(), z.data(), L);
+                memcpy(round_masks.data() + L, gp->candidate_masks + (size_t)stt.opt_rounds * gp->n_candidates * L, (size_t)gp->n_candidates * L);
+                const uint8_t* masks = round_masks.data();
+                ST(enqueue_score(ctx, masks, n_scored, gp->gamma));
+                counts.resize(n_scored);
+                CU(copy_async(ctx, counts.data(), kptr<int>(ctx, ctx->kl.score_out), n_scored * 4, cudaMemcpyDeviceToHost));
                 CU(cudaEventRecord(ev[3], ctx->stream));
                 CU(cudaStreamSynchronize(ctx->stream));
                 float ms = 0.f;
                 CU(cudaEventElapsedTime(&ms, ev[2], ev[3]));
                 stt.ms_score += ms;
                 int cb = 0;
-                for (int c = 1; c < gp->n_candidates; ++c) if (counts[c] > counts[cb]) cb = c;   // lowest index among equals
-                const float best = (float)counts[cb] / (float)gp->gamma;
-                if (best > stt.best_matchness) {                                                // strictly better only
-                    stt.best_matchness = best;
-                    memcpy(z.data(), masks + (size_t)cb * L, L);
-                }
+                for (int c = 1; c < n_scored; ++c) if (counts[c] > counts[cb]) cb = c;   // strictly better only: the set in use wins ties
+                stt.best_matchness = (float)counts[cb] / (float)gp->gamma;
+                if (cb != 0) memcpy(z.data(), masks + (size_t)cb * L, L);
+                stale_rounds = cb != 0 ? 0 : stale_rounds + 1;
                 stt.opt_rounds++;
-                if (stt.best_matchness > gp->stop_matchness || stt.opt_rounds >= gp->n_opt_rounds) optimising = false;
+                if (stt.best_matchness > gp->stop_matchness || stt.opt_rounds >= gp->n_opt_rounds ||
+                    (gp->opt_patience > 0 && stale_rounds >= gp->opt_patience))
+                    optimising = false;
             }
             const int k_max = std::min(gp->max_draft, remaining - 1);
             CU(cudaEventRecord(ev[4], ctx->stream));
@@ -1534,6 +1553,8 @@ swift_status swift_generate(swift_ctx* ctx, const swift_gen_params* gp, const in
     CU(cudaEventElapsedTime(&stt.ms_decode, ev[1], ev[7]));
     stt.tokens = count;
     stt.kernel_launches = ctx->launches - launches0;
+    stt.h2d_bytes = ctx->h2d_bytes - h2d0 + (int64_t)n_prompt * 4;     // the prompt itself is read from host memory
+    stt.d2h_bytes = ctx->d2h_bytes - d2h0 + (int64_t)count * 4;        // and the tokens are written there
     if (n_out) *n_out = count;
     if (stats) *stats = stt;
     return SWIFT_OK;

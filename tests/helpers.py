@@ -129,7 +129,7 @@ def walk_rounds(o: so.Oracle, gpu, z, n_rounds: int, max_k: int, stop_conf: floa
             tl = o.verify(d_tok)
             a, nxt, _ = so.accept_sampling(d_tok, q_rows, tl, temperature, seed, r, top_p)
             o.commit(d_tok[:a], nxt)
-            gpu.verify(d_tok); gpu.accept()
+            gpu.verify(); gpu.accept()                  # close the GPU's round on its own drafts, then start over
             resync(gpu, o, r)
             stats["resyncs"] += 1
             continue

@@ -14,6 +14,9 @@ from tests.helpers import (LOGIT_TOL, MARGIN, compare_free_running, logit_err, m
 pytestmark = pytest.mark.gpu
 
 TINY = synth.MODELS["tiny"]
+# Sampling decisions of bf16 models must agree with the oracle wherever its distance to the decision boundary exceeds
+# this: logits agree to about 1e-4 of their spread, so p/q and the running sums agree to a few 1e-4 relative.
+BF16_DEC_TOL = 1e-3
 BF16_SMALL = synth.ModelConfig("bf16-small", n_blocks=3, d_model=512, n_heads=8, n_kv_heads=2, head_dim=64,
                                ffn=1376, vocab=3001, dtype="bf16", seed=21, n_planted=1, gain_std=0.05)
 
@@ -197,7 +200,8 @@ def test_bf16_rounds(bf16_pair):
     o.prefill(prompt); g.prefill(prompt); g.set_pending(o.tokens[-1])
     z = list(synth.block_mask(BF16_SMALL, synth.planted_blocks(BF16_SMALL)))
     st = walk_rounds(o, g, z, n_rounds=8, max_k=8)
-    assert st["max_logit_err"] < LOGIT_TOL and st["accept_cmp"] >= 4, st
+    print("bf16 rounds:", st)
+    assert st["max_logit_err"] < LOGIT_TOL and st["accept_cmp"] >= 6, st      # at most two rounds may sit on a near-tie
 
 
 # ------------------------------------------------------------------------------ whole runs
@@ -303,9 +307,33 @@ def test_generate_with_on_the_fly_optimisation(tiny_pair):
     g.generate(prompt, GenParams(max_new=8, max_draft=4, skip_mask=kept))
     assert np.array_equal(g.final_skip_mask(), kept)
     scored = [r for r in o_rounds if r.matchness is not None]
-    assert abs(st.best_matchness - max(max(r.matchness) for r in scored)) <= 1.0 / 32 + 1e-6
+    assert abs(st.best_matchness - max(scored[-1].matchness)) <= 1.0 / 32 + 1e-6   # score of the set kept by the last round
     first = next(i for i, r in enumerate(o_rounds) if r.matchness is not None)
     assert [int(t[2]) for t in trace[:first]] == [r.accepted for r in o_rounds[:first]]   # same z0 until then
+
+
+def test_optimisation_keeps_a_set_no_proposal_beats(small_cfg):
+    """The set in use is scored with the proposals (Section 4.1: the highest-scoring set is retained): with the planted
+    branches scaled to exactly 0 the planted set scores 1 on every window, so it survives every round; patience and the
+    score threshold end the optimisation as in the oracle."""
+    from paper_2410_06916_b200 import GenParams
+    cfg = synth.ModelConfig(**{**small_cfg.__dict__, "planted_scale": 0.0})
+    o, g = make_pair(cfg, max_positions=96, page_size=8)
+    try:
+        planted = synth.block_mask(cfg, synth.planted_blocks(cfg))
+        prompt = synth.prompt(cfg, 10)
+        cands = np.stack([synth.candidate_masks(cfg, 2, 6, r) for r in range(4)])
+        for patience, stop, want_rounds in ((0, 2.0, 4), (2, 2.0, 2), (0, 0.95, 1)):
+            ogp = so.GenParams(max_new=40, max_draft=3, gamma=8, max_opt_rounds=4, stop_matchness=stop, patience=patience)
+            o2 = so.Oracle(o.s, o.w, dtype=o.dtype, max_positions=96)
+            o_out, o_rounds, _ = so.swift_generate(o2, prompt, list(planted), ogp, lambda r: cands[r])
+            out, st, _ = g.generate(prompt, GenParams(max_new=40, max_draft=3, gamma=8, n_opt_rounds=4, stop_matchness=stop,
+                                                      opt_patience=patience, skip_mask=planted, candidate_masks=cands))
+            assert st.opt_rounds == want_rounds == sum(r.matchness is not None for r in o_rounds)
+            assert out == o_out and st.best_matchness == 1.0
+            assert np.array_equal(g.final_skip_mask(), planted)
+    finally:
+        g.close()
 
 
 # ------------------------------------------------------------------------------ sampling
@@ -339,8 +367,9 @@ def test_sampling_bf16_rounds(bf16_pair):
         o.prefill(prompt)
         g.prefill(prompt); g.set_pending(o.tokens[-1])
         z = list(synth.block_mask(BF16_SMALL, [1]))
-        st = walk_rounds(o, g, z, n_rounds=12, max_k=6, sampling=True, seed=seed, dec_tol=0.06)
-        assert st["accept_cmp"] >= 6, st
+        st = walk_rounds(o, g, z, n_rounds=12, max_k=6, sampling=True, seed=seed, dec_tol=BF16_DEC_TOL)
+        print("bf16 sampling rounds:", st)
+        assert st["accept_cmp"] >= 10, st                                      # at most two rounds may sit on a decision boundary
     finally:
         g.set_sampling(False)
 
@@ -371,6 +400,13 @@ def test_errors_are_statuses_not_crashes(small_cfg):
         g.draft(z, 2)
     g.verify(); g.accept()
     assert g.n >= 4
+    # speculative sampling compares p_j with the q_j kept from drafting: more tokens than were drafted cannot be verified
+    g.set_sampling(True, 1.0, 3)
+    toks, _ = g.draft(z, 2)
+    with pytest.raises(SwiftError, match="ECAPACITY"):
+        g.verify(list(toks) + [1])
+    g.verify(list(toks)); g.accept()
+    g.set_sampling(False)
     g.close()
 
 
@@ -634,7 +670,7 @@ def test_full_depth_13b_scoring_and_rounds():
         g.set_sampling(True, 1.0, seed)
         resync(g, o, 1)
         z20 = list(synth.block_mask(cfg, synth.draft_blocks(cfg, 20)))
-        st = walk_rounds(o, g, z20, n_rounds=1, max_k=3, sampling=True, seed=seed, first_round=2, dec_tol=0.06)
+        st = walk_rounds(o, g, z20, n_rounds=1, max_k=3, sampling=True, seed=seed, first_round=2, dec_tol=BF16_DEC_TOL)
         assert st["max_logit_err"] < LOGIT_TOL, st
     finally:
         g.set_sampling(False)

@@ -111,22 +111,50 @@ def test_matchness_by_brute_force(small_cfg, small_weights):
 
 
 def test_optimisation_keeps_strictly_better_candidates(small_cfg, small_weights):
+    """Section 4.1: the highest-scoring set is retained.  The set in use is scored on the same window as the
+    proposals (entry 0) and is replaced only by a proposal that beats it there; earliest among equals."""
     prompt = synth.prompt(small_cfg, 8)
     cands = lambda r: synth.candidate_masks(small_cfg, 2, 4, r)
-    gp = so.GenParams(max_new=30, max_draft=3, gamma=8, max_opt_rounds=3)
-    out, rounds, _ = so.swift_generate(_oracle(small_cfg, small_weights), prompt,
-                                       list(synth.block_mask(small_cfg, synth.uniform_blocks(4, 2))), gp, cands)
+    gp = so.GenParams(max_new=30, max_draft=3, gamma=8, max_opt_rounds=3, stop_matchness=2.0)
+    z0 = list(synth.block_mask(small_cfg, synth.uniform_blocks(4, 2)))
+    out, rounds, _ = so.swift_generate(_oracle(small_cfg, small_weights), prompt, z0, gp, cands)
     ref, _ = so.vanilla_generate(_oracle(small_cfg, small_weights), prompt, 30)
     assert out == ref
     scored = [r for r in rounds if r.matchness is not None]
-    assert len(scored) == 3 and all(len(r.matchness) == 4 for r in scored)
-    best = -1.0
-    for r in scored:
-        if max(r.matchness) > best:
-            best = max(r.matchness)
-            c = r.matchness.index(best)                           # lowest index among equals
-            assert r.z == list(cands(scored.index(r))[c])
-    assert rounds[-1].z == [x for x in scored if max(x.matchness) == best][0].z
+    assert len(scored) == 3 and all(len(r.matchness) == 5 for r in scored)
+    z = z0
+    for i, r in enumerate(scored):
+        pool = [z] + [list(m) for m in cands(i)]
+        best = max(r.matchness)
+        z = pool[r.matchness.index(best)]                         # lowest index among equals; index 0 = the set in use
+        assert r.z == z
+    assert rounds[-1].z == z
+    first = rounds.index(scored[0])
+    assert all(r.z == z0 for r in rounds[:first])
+
+
+def test_optimisation_never_drops_a_set_no_proposal_beats(small_cfg):
+    """With the planted residual branches scaled to exactly 0 the planted set re-predicts every context token
+    (matchness 1), so no proposal can score strictly higher: it must survive every optimisation round, and a
+    run that starts elsewhere must not end on anything worse than what it held on the way."""
+    cfg = synth.ModelConfig(**{**small_cfg.__dict__, "planted_scale": 0.0})
+    w = synth.make_weights(cfg)
+    planted = list(synth.block_mask(cfg, synth.planted_blocks(cfg)))
+    prompt = synth.prompt(cfg, 10)
+    cands = lambda r: synth.candidate_masks(cfg, 2, 6, r)
+    gp = so.GenParams(max_new=40, max_draft=3, gamma=8, max_opt_rounds=4, stop_matchness=2.0)
+    _, rounds, stats = so.swift_generate(_oracle(cfg, w), prompt, planted, gp, cands)
+    scored = [r for r in rounds if r.matchness is not None]
+    assert len(scored) == 4 and all(r.matchness[0] == 1.0 for r in scored)
+    assert all(r.z == planted for r in rounds) and stats["alpha"] == 1.0
+    # patience: two rounds in a row without a replacement end the optimisation
+    gp2 = so.GenParams(max_new=40, max_draft=3, gamma=8, max_opt_rounds=4, stop_matchness=2.0, patience=2)
+    _, rounds2, _ = so.swift_generate(_oracle(cfg, w), prompt, planted, gp2, cands)
+    assert sum(r.matchness is not None for r in rounds2) == 2
+    # the score threshold ends it after the first round (1.0 > 0.95)
+    gp3 = so.GenParams(max_new=40, max_draft=3, gamma=8, max_opt_rounds=4)
+    _, rounds3, _ = so.swift_generate(_oracle(cfg, w), prompt, planted, gp3, cands)
+    assert sum(r.matchness is not None for r in rounds3) == 1
 
 
 # ------------------------------------------------------------------------------ sampling acceptance

@@ -10,6 +10,7 @@ import pytest
 import torch
 
 import synth
+from oracle import swift_oracle as so
 
 pytestmark = pytest.mark.gpu
 
@@ -45,6 +46,9 @@ def test_static_scratch_gemm_matches_the_context_gemm_twice_in_a_row(dtype):
             scale = float(np.sqrt((ref ** 2).mean()))
             assert np.isfinite(got).all()
             assert np.abs(got - ref).max() < 2e-4 * scale, float(np.abs(got - ref).max() / scale)
+            # ... and against the plain fp64 product, so that a defect both entry points share cannot hide
+            exact = so.linear(x, w).numpy()
+            assert np.abs(got - exact).max() < 2e-4 * scale, float(np.abs(got - exact).max() / scale)
     finally:
         g.close()
 
