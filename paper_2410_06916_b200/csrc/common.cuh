@@ -39,7 +39,21 @@ struct DevState {
     unsigned seed_lo, seed_hi;
     int pad[2];
     float row_thresh[ROWS]; // nucleus sampling: smallest exp((l - max) / T) a row keeps (0 = everything); row_sum covers the kept ones
+    // Shape of the forward's own rows.  Row m is stored at cache slot pos0 + m; it sits at sequence position
+    // pos0 + row_depth[m] (rotary embedding) and sees row j of the forward iff bit j of row_vis[m] is set.  A plain
+    // forward has depth m and bits 0..m (causal order); a verified token tree has a node's depth and its ancestors.
+    unsigned row_vis[ROWS];
+    int row_depth[ROWS];
 };
+
+// Causal order over the forward's rows: the default shape.
+__device__ __forceinline__ void set_causal_rows(DevState* st)
+{
+    for (int m = 0; m < ROWS; ++m) {
+        st->row_vis[m] = (2u << m) - 1u;
+        st->row_depth[m] = m;
+    }
+}
 
 // Programmatic dependent launch.  Every kernel of a forward is launched with programmatic stream
 // serialisation: it may start while its predecessor is still running, so it (a) lets its own successor

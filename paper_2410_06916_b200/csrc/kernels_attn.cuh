@@ -192,7 +192,7 @@ attn_split_kernel(const DevState* st, const float* __restrict__ q, const T* __re
 __device__ __forceinline__ void combine_row(int pos0, int r, int h, const float* __restrict__ o_part,
                                             const float2* __restrict__ ml_part, int max_splits, int n_heads, int dh,
                                             float* __restrict__ out, __nv_bfloat16* __restrict__ planes,
-                                            float* comb_sh, float* wmax_sh)
+                                            float* comb_sh, float* wmax_sh, int part_rows = ROWS)
 {
     const int d = threadIdx.x;
     // row r sees positions <= pos0 + r: later splits hold nothing for it (and, when the rows were processed in
@@ -204,15 +204,15 @@ __device__ __forceinline__ void combine_row(int pos0, int r, int h, const float*
 
     // the first 16 splits' partial outputs are requested before anything else: they do not depend on the weights
     constexpr int CB = 16;
-    const float* op = o_part + (base * ROWS + r) * dh + d;
-    const size_t stride = (size_t)ROWS * dh;
+    const float* op = o_part + (base * part_rows + r) * dh + d;
+    const size_t stride = (size_t)part_rows * dh;
     float o[CB];
 #pragma unroll
     for (int i = 0; i < CB; ++i) o[i] = i < n_splits ? __ldcg(op + (size_t)i * stride) : 0.f;
 
     float mx = -INFINITY;
     for (int s = d; s < n_splits; s += blockDim.x) {
-        const float2 ml = __ldcg(ml_part + (base + s) * ROWS + r);
+        const float2 ml = __ldcg(ml_part + (base + s) * part_rows + r);
         w_sh[s] = ml.x;
         l_sh[s] = ml.y;
         mx = fmaxf(mx, ml.x);

@@ -14,6 +14,7 @@ __global__ void set_rows_kernel(DevState* st, int pos0, int n_rows)
     st->pos0 = pos0;
     st->n_rows = n_rows;
     st->tok_off = 0;
+    set_causal_rows(st);
 }
 
 // Start of a round: pending token into slot 0, drafting armed.
@@ -28,6 +29,7 @@ __global__ void begin_round_kernel(DevState* st, int pending_token, int use_give
     st->active = 1;
     st->n_drafted = 0;
     st->n_accepted = 0;
+    set_causal_rows(st);
 }
 
 // Draft step j (1-based): one row, input y'_{j-1} (slot j-1), position n + j - 1; a stopped draft

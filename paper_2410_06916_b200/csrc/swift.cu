@@ -15,6 +15,7 @@
 
 #include "common.cuh"
 #include "kernels_attn.cuh"
+#include "kernels_attn_mma.cuh"
 #include "kernels_elem.cuh"
 #include "kernels_gemm_simt.cuh"
 #include "kernels_gemm_tc.cuh"
@@ -74,7 +75,7 @@ struct swift_ctx {
     std::string err;
     cudaEvent_t ev[8];
     // captured forwards; programmatic dependent launch between the kernels of a forward
-    bool use_graphs, use_pdl, pdl_next, pdl_gemms, fuse, fuse_combine, prefetch_next;
+    bool use_graphs, use_pdl, pdl_next, pdl_gemms, fuse, fuse_combine, prefetch_next, attn_mma;
     int attn_rows_per_cta, prefetch_tiles;
     std::vector<FwdGraph>* graphs;
     uint64_t graph_clock;
@@ -374,12 +375,46 @@ swift_status launch_attn_mr(swift_ctx* ctx, const int* page_table, int block, in
     return SWIFT_OK;
 }
 
-// Attention of one block for the forward chunk's rows: split kernel + merge of the splits into `out` (fp32 rows)
-// and, when given, the hi/lo planes the next GEMM reads.
-template <typename T>
-swift_status launch_attn(swift_ctx* ctx, int rows, const int* page_table, int block, float* out, __nv_bfloat16* planes)
+#define ST(call)                                   \
+    do {                                           \
+        swift_status s_ = (call);                  \
+        if (s_ != SWIFT_OK) return s_;             \
+    } while (0)
+
+template <typename T, int NT>
+swift_status launch_attn_mma(swift_ctx* ctx, const int* page_table, int block, bool fused, float* out, __nv_bfloat16* planes)
 {
     const swift_model_desc& d = ctx->d;
+    CU(launch_k(attn_mma_kernel<T, NT>, dim3(d.n_kv_heads, ctx->max_splits), dim3(AM_THREADS), attn_mma_smem_bytes(NT, ctx->max_splits), ctx,
+                (const DevState*)state_of(ctx), (const float*)kptr<float>(ctx, ctx->kl.q), reinterpret_cast<const T*>(ctx->kvbase),
+                page_table, ctx->kv, block, d.n_heads, ctx->max_splits, 1.0f / sqrtf((float)d.head_dim),
+                kptr<float>(ctx, ctx->kl.o_part), kptr<float2>(ctx, ctx->kl.ml_part), (int)ROWS,
+                fused ? kptr<int>(ctx, ctx->kl.attn_counters) : (int*)nullptr, fused ? out : (float*)nullptr,
+                fused ? planes : (__nv_bfloat16*)nullptr));
+    return SWIFT_OK;
+}
+
+// Attention of one block for the forward chunk's rows: split kernel + merge of the splits into `out` (fp32 rows)
+// and, when given, the hi/lo planes the next GEMM reads.  `full_model`: no sub-layer of this forward is skipped.  The
+// target model's forwards (verification, vanilla steps, prefill) take the tensor-core kernel, layer-skipped forwards
+// the streaming one; a row's result never depends on the row count within either family, which is what makes a
+// vanilla step and the same row of a verification agree bit for bit.
+template <typename T>
+swift_status launch_attn(swift_ctx* ctx, int rows, const int* page_table, int block, float* out, __nv_bfloat16* planes,
+                         bool full_model)
+{
+    const swift_model_desc& d = ctx->d;
+    if (d.head_dim == 128 && full_model && ctx->attn_mma) {
+        const bool fused = rows == 1 && ctx->fuse_combine;
+        const swift_status ms = (d.n_heads / d.n_kv_heads) * rows <= 8 ? launch_attn_mma<T, 1>(ctx, page_table, block, fused, out, planes)
+                                                                       : launch_attn_mma<T, 2>(ctx, page_table, block, fused, out, planes);
+        if (ms != SWIFT_OK) return ms;
+        if (fused) return SWIFT_OK;
+        CU(launch_k(attn_combine_kernel, dim3(d.n_heads, rows), dim3(d.head_dim), 2 * (size_t)ctx->max_splits * sizeof(float), ctx,
+                    (const DevState*)state_of(ctx), (const float*)kptr<float>(ctx, ctx->kl.o_part),
+                    (const float2*)kptr<float2>(ctx, ctx->kl.ml_part), ctx->max_splits, d.n_heads, d.head_dim, out, planes));
+        return SWIFT_OK;
+    }
     // The streaming kernel (head_dim 128) takes the rows in groups of at most attn_rows_per_cta, one group per
     // grid.z slice: fewer rows per CTA means fewer registers and more CTAs in flight.
     int mr = attn_mr_of(rows), groups = 1;
@@ -412,11 +447,6 @@ struct HeadOpts {
     int mode = VOCAB_PLAIN;
 };
 
-#define ST(call)                                   \
-    do {                                           \
-        swift_status s_ = (call);                  \
-        if (s_ != SWIFT_OK) return s_;             \
-    } while (0)
 
 // Enqueues the kernels of one forward chunk of at most `rows` (<= 16) rows.  The device state
 // (pos0, n_rows, tok_off) must have been set by a preceding kernel on the same stream.
@@ -439,6 +469,8 @@ swift_status forward_chunk(swift_ctx* ctx, int rows, const int* toks_dev, const 
     __nv_bfloat16* act_hl = tc ? kptr<__nv_bfloat16>(ctx, ctx->kl.act_hl) : nullptr;
     const float* pend = nullptr;      // pending residual-branch output (split-K slabs) not yet added to h
     int pend_S = 0, S = 0;
+    bool full_model = true;
+    for (int sl = 0; sl < 2 * d.n_blocks; ++sl) full_model = full_model && !(skip && skip[sl]);
 
     CU(launch_k(embed_kernel<T>, dim3(rows), dim3(256), 0, ctx, st, toks_dev, (const T*)wptr<T>(ctx, ctx->wl.embed), h, dm, d.vocab));
     for (int b = 0; b < d.n_blocks; ++b) {
@@ -450,7 +482,7 @@ swift_status forward_chunk(swift_ctx* ctx, int rows, const int* toks_dev, const 
                         (const DevState*)st, (const float*)part, S, (size_t)ROWS * nqkv, nqkv, kptr<float>(ctx, ctx->kl.q),
                         reinterpret_cast<TKV*>(ctx->kvbase), page_table, ctx->kv, b, d.n_heads,
                         (const float2*)kptr<float2>(ctx, ctx->kl.rope), d.max_positions));
-            ST(launch_attn<TKV>(ctx, rows, page_table, b, xa, xa_hl));
+            ST(launch_attn<TKV>(ctx, rows, page_table, b, xa, xa_hl, full_model));
             ST(run_gemm<T>(ctx, mr, GemmSite{xa, dm, qd, wptr<T>(ctx, ctx->wl.wo[b]), tc ? &ctx->tm_wo[b] : nullptr, &ctx->tm_xa}, &S));
             pend = part; pend_S = S;
         }
@@ -498,6 +530,7 @@ swift_status forward_chunk_fused(swift_ctx* ctx, int rows, const int* toks_dev, 
     std::vector<int> kept;                       // sub-layers that run, in walk order
     for (int sl = 0; sl < 2 * d.n_blocks; ++sl)
         if (!(skip && skip[sl])) kept.push_back(sl);
+    const bool full_model = (int)kept.size() == 2 * d.n_blocks;
     auto gain_of = [&](size_t k) -> const float* {   // gain of the RMSNorm in front of kept[k]; past the end: the final norm
         if (k < kept.size()) return wptr<float>(ctx, (kept[k] & 1) ? ctx->wl.mlp_norm[kept[k] >> 1] : ctx->wl.attn_norm[kept[k] >> 1]);
         return head.run ? wptr<float>(ctx, ctx->wl.final_norm) : nullptr;
@@ -556,7 +589,7 @@ swift_status forward_chunk_fused(swift_ctx* ctx, int rows, const int* toks_dev, 
             ep.q_out = kptr<float>(ctx, ctx->kl.q); ep.kv_pool = ctx->kvbase; ep.page_table = page_table; ep.L = ctx->kv;
             ep.block = b; ep.n_heads = d.n_heads; ep.max_positions = d.max_positions; ep.rope_cs = kptr<float2>(ctx, ctx->kl.rope);
             ST(gemm(EPI_QKV, &ctx->tm_wqkv[b], &ctx->tm_xn, nqkv, dm, ep));
-            ST(launch_attn<TKV>(ctx, rows, page_table, b, xa, xa_hl));
+            ST(launch_attn<TKV>(ctx, rows, page_table, b, xa, xa_hl, full_model));
             ST(gemm(EPI_RESID, &ctx->tm_wo[b], &ctx->tm_xa, dm, qd, resid));
         } else {
             EpiParams ep = base;
@@ -888,6 +921,11 @@ cudaError_t init_kernel_attrs()
     if (e == cudaSuccess) e = cudaFuncSetAttribute(gemm_tc_kernel<EPI_SWIGLU, float>, cudaFuncAttributeMaxDynamicSharedMemorySize, TC_SMEM_BYTES);
     if (e == cudaSuccess) e = cudaFuncSetAttribute(gemm_tc_kernel<EPI_QKV, float>, cudaFuncAttributeMaxDynamicSharedMemorySize, TC_SMEM_BYTES);
     if (e == cudaSuccess) e = cudaFuncSetAttribute(gemm_tc_kernel<EPI_QKV, __nv_bfloat16>, cudaFuncAttributeMaxDynamicSharedMemorySize, TC_SMEM_BYTES);
+    const int am_max = (int)attn_mma_smem_bytes(2, 262144 / ATTN_CHUNK);
+    if (e == cudaSuccess) e = cudaFuncSetAttribute(attn_mma_kernel<float, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, am_max);
+    if (e == cudaSuccess) e = cudaFuncSetAttribute(attn_mma_kernel<float, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, am_max);
+    if (e == cudaSuccess) e = cudaFuncSetAttribute(attn_mma_kernel<__nv_bfloat16, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, am_max);
+    if (e == cudaSuccess) e = cudaFuncSetAttribute(attn_mma_kernel<__nv_bfloat16, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, am_max);
     if (e == cudaSuccess) e = cudaFuncSetAttribute(vocab_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)VOCAB_CACHE_MAX_BYTES);
     return e;
 }
@@ -1002,6 +1040,7 @@ swift_status swift_load(const swift_model_desc* desc, swift_devbuf weights, swif
         c->attn_rows_per_cta = (v == 1 || v == 2 || v == 4 || v == 6 || v == 8 || v == 12) ? v : 16;
     }
     c->fuse_combine = getenv("SWIFT_NO_FUSE_COMBINE") == nullptr;
+    c->attn_mma = getenv("SWIFT_NO_ATTN_MMA") == nullptr;      // full-model forwards on the streaming attention kernel too
     c->prefetch_next = getenv("SWIFT_NO_PREFETCH_NEXT") == nullptr;
     {
         const char* e = getenv("SWIFT_PREFETCH_TILES");      // 16 KB tiles of the next GEMM each CTA asks L2 for
