@@ -166,6 +166,41 @@ def test_full_width_bf16_forward(shape, kv):
         g.close()
 
 
+@pytest.mark.parametrize("shape,n_prefix,max_k", [("13b", 1100, 8), ("70b", 2130, 12), ("7b", 700, 8)])
+def test_benchmark_context_lengths(shape, n_prefix, max_k):
+    """Two blocks at full width behind prefixes as long as the benchmark's contexts (config 3/4: 1024 + up to 512,
+    config 5: 2048 + 512, config 2: 512 + 256): more than 16 attention chunks per row (the merge of the chunks runs
+    its second batch), page tables of more than a hundred pages, the one-row merge inside the attention launch with
+    17 to 34 chunks.  Compared with the oracle: the last prefill rows, a one-row and a (max_draft + 1)-row forward of
+    the full and of a layer-skipped model, then two whole rounds of draft / verify / accept."""
+    cfg = synth.MODELS[shape].with_blocks(2, n_planted=1)
+    o, g = make_pair(cfg, max_positions=n_prefix + 64, max_draft=max_k)
+    try:
+        rows = max_k + 1
+        toks = synth.prompt(cfg, n_prefix + rows)
+        o.prefill(toks[:n_prefix])
+        g.prefill(toks[:n_prefix])
+        assert g.n == n_prefix == o.n
+        ref3 = o.forward_rows(toks[n_prefix - 3:n_prefix], n_prefix - 3, write_kv=False)
+        got3, _ = g.forward_rows(toks[n_prefix - 3:n_prefix], n_prefix - 3, write_kv=False)
+        err = logit_err(got3, ref3)
+        print(f"{shape} at {n_prefix} positions: last prefill rows off by {err:.2e} sigma")
+        assert err < LOGIT_TOL
+        for z in (None, list(synth.block_mask(cfg, [1])), [1, 0, 0, 1]):
+            refm = o.forward_rows(toks[n_prefix:n_prefix + rows], n_prefix, z, write_kv=False)
+            gotm, _ = g.forward_rows(toks[n_prefix:n_prefix + rows], n_prefix, z, write_kv=False)
+            got1, _ = g.forward_rows(toks[n_prefix:n_prefix + 1], n_prefix, z, write_kv=False)
+            errm = logit_err(gotm, refm)
+            assert errm < LOGIT_TOL and logit_err(got1, refm[:1]) < LOGIT_TOL, (z, errm)
+            assert np.array_equal(got1[0], gotm[0])              # row-count invariance, bit for bit
+        g.set_pending(o.tokens[-1])
+        st = walk_rounds(o, g, list(synth.block_mask(cfg, [1])), n_rounds=2, max_k=max_k)
+        print(f"{shape} at {n_prefix} positions: rounds {st}")
+        assert st["max_logit_err"] < LOGIT_TOL and st["rounds"] == 2, st
+    finally:
+        g.close()
+
+
 # ------------------------------------------------------------------------------ rounds
 @pytest.mark.parametrize("stop_conf,max_k", [(0.0, 4), (0.8, 4), (0.0005, 7), (0.0, 15)])
 def test_tiny_rounds_step_by_step(tiny_pair, stop_conf, max_k):
