@@ -197,23 +197,28 @@ class Oracle:
         return x @ W.to(self.dtype).T
 
     def forward_rows(self, row_tokens: Sequence[int], pos0: int, z: Optional[Sequence[int]] = None,
-                     write_kv: bool = True) -> torch.Tensor:
+                     write_kv: bool = True, depth: Optional[Sequence[int]] = None,
+                     sees: Optional[torch.Tensor] = None) -> torch.Tensor:
         """Logits [M, V] for M new rows at positions pos0..pos0+M-1 under skipped sub-layer set z.
 
         Every row attends to cached positions [0, pos0) and causally to the new rows.  A skipped
         sub-layer is the identity on the residual stream (Section 3.1): its norm, projections and,
         for attention, its K,V computation are all left out.  K,V of the new rows are stored in the
         cache for non-skipped attention sub-layers when write_kv is set.
+
+        A token tree (Section 4.2, dynamic verification) is a set of rows that are not one sequence:
+        `depth[i]` puts row i at sequence position pos0 + depth[i] and `sees` [M, M] says which of the
+        new rows row i attends to (its ancestors and itself).  Row i's K,V still go to cache slot pos0 + i.
         """
         s = self.s
         M = len(row_tokens)
         z = [0] * (2 * s.n_blocks) if z is None else [int(v) for v in z]
         assert len(z) == 2 * s.n_blocks and pos0 + M <= self.max_positions
-        pos = torch.arange(pos0, pos0 + M)
+        pos = torch.arange(pos0, pos0 + M) if depth is None else pos0 + torch.tensor(list(depth), dtype=torch.long)
         h = self.w["embed"][torch.tensor(list(row_tokens), dtype=torch.long)].to(self.dtype)
-        # row i may read cache position j < pos0 always, and new row j' <= i
-        allowed = torch.cat([torch.ones(M, pos0, dtype=torch.bool),
-                             torch.tril(torch.ones(M, M, dtype=torch.bool))], dim=1)
+        # row i may read cache position j < pos0 always, and new row j' <= i (or the rows `sees` names)
+        among = torch.tril(torch.ones(M, M, dtype=torch.bool)) if sees is None else sees.to(torch.bool)
+        allowed = torch.cat([torch.ones(M, pos0, dtype=torch.bool), among], dim=1)
         for b in range(s.n_blocks):
             wb = self.w["blocks"][b]
             if not z[2 * b]:
@@ -273,6 +278,23 @@ class Oracle:
     def verify(self, draft_tokens: Sequence[int]) -> torch.Tensor:
         """Full model on rows [t*, y'_1..y'_k] at positions n..n+k; K,V written for every layer."""
         return self.forward_rows([self.tokens[-1]] + list(draft_tokens), self.n)
+
+    def verify_tree(self, tree: "TokenTree") -> torch.Tensor:
+        """Full model on all rows of a token tree at once (Section 4.2, dynamic verification): row i sits at position
+        n + depth[i], attends to the cache and to its own ancestors, and leaves its K,V in slot n + i."""
+        assert tree.tokens[0] == self.tokens[-1]
+        return self.forward_rows(tree.tokens, self.n, depth=tree.depth, sees=tree.sees())
+
+    def commit_path(self, tree: "TokenTree", path: Sequence[int], next_token: int) -> None:
+        """KV rollback after a verified tree: the accepted node of depth j must end up in slot n + j; chain nodes are
+        there already, an accepted alternative is moved there from the slot it was verified in."""
+        for j, row in enumerate(path, start=1):
+            assert tree.depth[row] == j
+            if row != j:
+                for b in range(self.s.n_blocks):
+                    self.K[b][self.n + j] = self.K[b][self.n + row]
+                    self.V[b][self.n + j] = self.V[b][self.n + row]
+        self.commit([tree.tokens[r] for r in path], next_token)
 
     def commit(self, accepted: Sequence[int], next_token: int) -> None:
         """KV rollback: keep positions [0, n + a + 1); positions beyond are dropped (left stale)."""
@@ -349,6 +371,78 @@ def accept_sampling(draft_tokens: Sequence[int], q_rows: Sequence[torch.Tensor],
     return k, tok, log
 
 
+# =============================================================================== dynamic verification (token tree)
+def tree_width(p: float) -> int:
+    """How many of the draft model's top predictions stand in for a draft token of confidence p (Section 4.2):
+    10, 5, 3, 1 for p in (0, 0.5], (0.5, 0.8], (0.8, 0.95], (0.95, 1]."""
+    return 10 if p <= 0.5 else 5 if p <= 0.8 else 3 if p <= 0.95 else 1
+
+
+@dataclass
+class TokenTree:
+    """The draft candidates of one round, linearised: row 0 is the pending token t*, rows 1..k the drafted chain
+    y'_1..y'_k, then, depth by depth, the alternatives of each draft position (the draft model's next-best
+    predictions at that step).  An alternative of depth j hangs off chain row j-1 and has no children: drafting
+    went on from y'_j only."""
+    tokens: List[int]
+    depth: List[int]
+    parent: List[int]
+
+    def sees(self) -> torch.Tensor:
+        """[M, M]: row i attends to its ancestors and itself (the 'special causal attention mask' of Section 4.2)."""
+        M = len(self.tokens)
+        a = torch.zeros(M, M, dtype=torch.bool)
+        for i in range(M):
+            j = i
+            while j >= 0:
+                a[i, j] = True
+                j = self.parent[j]
+        return a
+
+    def children(self, node: int) -> List[int]:
+        return [c for c, p in enumerate(self.parent) if p == node]
+
+
+def ranked_tokens(row: torch.Tensor, n: int) -> List[int]:
+    """The n best token ids of a logits row, best first; equal logits in order of token id."""
+    idx = torch.sort(row.to(torch.float64), descending=True, stable=True).indices   # stable: equal values keep index order
+    return [int(i) for i in idx[:n]]
+
+
+def build_tree(pending: int, draft_tokens: Sequence[int], draft_rows: Sequence[torch.Tensor], conf: Sequence[float],
+               row_budget: int) -> TokenTree:
+    """Extends every draft position j with the draft model's top-k predictions at that step, k = tree_width(p_j).
+    The paper sets no limit on the rows verified at once; here the forward takes row_budget rows, so the chain
+    (1 + k rows) is placed first and the alternatives are handed out from the first draft position on until the
+    rows run out (an earlier position decides whether the later ones matter at all)."""
+    k = len(draft_tokens)
+    assert row_budget >= k + 1
+    tokens, depth, parent = [int(pending)] + [int(t) for t in draft_tokens], list(range(k + 1)), list(range(-1, k))
+    for j in range(1, k + 1):
+        extra = min(tree_width(conf[j - 1]) - 1, row_budget - len(tokens))
+        if extra <= 0:
+            continue
+        best = ranked_tokens(draft_rows[j - 1], extra + 1)
+        alts = [t for t in best if t != tokens[j]][:extra]            # the chain token is the best one under greedy drafting
+        for t in alts:
+            tokens.append(t); depth.append(j); parent.append(j - 1)
+    return TokenTree(tokens, depth, parent)
+
+
+def accept_tree(tree: TokenTree, target_logits: torch.Tensor) -> Tuple[List[int], int]:
+    """Greedy verification of a token tree: from t*, follow the child whose token is the target's arg max at the
+    current node; where no child matches, that arg max is the next token.  Returns (rows of the accepted nodes in
+    order, next token): every emitted token is what vanilla greedy decoding would have produced."""
+    node, path = 0, []
+    while True:
+        gold = argmax_lowest(target_logits[node])
+        hit = [c for c in tree.children(node) if tree.tokens[c] == gold]
+        if not hit:
+            return path, gold
+        node = hit[0]
+        path.append(node)
+
+
 # =============================================================================== whole runs
 @dataclass
 class GenParams:
@@ -364,6 +458,7 @@ class GenParams:
     stop_matchness: float = 0.95
     max_opt_rounds: int = 0       # 0 = skip set fixed
     patience: int = 0             # stop optimising after this many rounds in a row that kept the incumbent (0 = never)
+    tree_rows: int = 0            # dynamic verification: rows one verification may hold (0 = the drafted chain only)
 
 
 @dataclass
@@ -379,6 +474,8 @@ class Round:
     decisions: List[dict] = field(default_factory=list)
     matchness: Optional[List[float]] = None
     z: Optional[List[int]] = None
+    tree: Optional[TokenTree] = None       # dynamic verification: the rows that were verified and the accepted path
+    path: Optional[List[int]] = None
 
 
 def vanilla_generate(o: Oracle, prompt: Sequence[int], max_new: int, mode: str = "greedy",
@@ -458,6 +555,16 @@ def swift_generate(o: Oracle, prompt: Sequence[int], z0: Sequence[int], gp: GenP
                 d_tok, d_conf, d_rows = o.draft(z, k_max, gp.stop_conf)
         else:
             d_tok, d_conf, d_rows = [], [], []
+        if gp.tree_rows > 0 and not sampling:
+            # dynamic verification: the chain plus the draft model's next-best predictions, verified as one tree
+            tree = build_tree(o.tokens[-1], d_tok, d_rows, d_conf, max(gp.tree_rows, len(d_tok) + 1))
+            tl = o.verify_tree(tree)
+            path, nxt = accept_tree(tree, tl)
+            M = len(tree.tokens)
+            rounds.append(Round(o.n, d_tok, d_conf, [top2_margin(x) for x in d_rows], [argmax_lowest(tl[i]) for i in range(M)],
+                                [top2_margin(tl[i]) for i in range(M)], len(path), nxt, [], scores, list(z), tree, list(path)))
+            o.commit_path(tree, path, nxt)
+            continue
         tl = o.verify(d_tok)
         if sampling:
             a, nxt, dec = accept_sampling(d_tok, q_rows, tl, gp.temperature, gp.rng_seed, r, gp.top_p)

@@ -381,3 +381,76 @@ def test_expected_speedup_matches_table_5():
     for *_, M, alpha, c, printed in rows:
         assert abs(so.expected_speedup(float(M), float(alpha), float(c)) - float(printed)) < 0.0051
     assert so.expected_speedup(1.0, 0.7, 0.55) == 1.0            # one token per round: no gain, no loss
+
+
+# ------------------------------------------------------------------------------ dynamic verification (token tree)
+def test_tree_width_bins_are_the_papers():
+    """Section 4.2: k = 10, 5, 3, 1 for p in (0, 0.5], (0.5, 0.8], (0.8, 0.95], (0.95, 1]."""
+    for p, k in ((1e-6, 10), (0.3, 10), (0.5, 10), (0.5000001, 5), (0.8, 5), (0.81, 3), (0.95, 3), (0.9500001, 1), (1.0, 1)):
+        assert so.tree_width(p) == k, p
+
+
+def test_tree_shape_and_row_budget():
+    rows = [torch.tensor([0.0, 5.0, 4.0, 3.0, 2.0, 1.0, 0.5, 0.4, 0.3, 0.2, 0.1, -1.0]),
+            torch.tensor([9.0, 1.0, 8.0, 7.0, 0.0, 0.0, 0.0, 0.0, 0.0, 0.0, 0.0, 0.0])]
+    tree = so.build_tree(7, [1, 0], rows, [0.7, 0.9], row_budget=64)           # widths 5 and 3
+    assert tree.tokens == [7, 1, 0, 2, 3, 4, 5, 2, 3]                           # chain first, then alternatives depth by depth
+    assert tree.depth == [0, 1, 2, 1, 1, 1, 1, 2, 2]
+    assert tree.parent == [-1, 0, 1, 0, 0, 0, 0, 1, 1]
+    sees = tree.sees()
+    assert sees[2].tolist() == [True, True, True] + [False] * 6                 # y'_2 sees t*, y'_1, itself
+    assert sees[4].tolist() == [True, False, False, False, True, False, False, False, False]   # an alternative of y'_1: t* and itself
+    assert sees[8].tolist() == [True, True, False, False, False, False, False, False, True]    # an alternative of y'_2: t*, y'_1, itself
+    tight = so.build_tree(7, [1, 0], rows, [0.7, 0.9], row_budget=5)           # 3 chain rows + 2: the first position takes both
+    assert tight.tokens == [7, 1, 0, 2, 3] and tight.depth == [0, 1, 2, 1, 1]
+    assert so.build_tree(7, [1, 0], rows, [0.99, 0.96], row_budget=64).tokens == [7, 1, 0]     # confident drafts: the chain alone
+    # equal logits rank by token id
+    assert so.ranked_tokens(torch.tensor([1.0, 3.0, 3.0, 2.0, 3.0]), 4) == [1, 2, 4, 3]
+
+
+def test_tree_rows_equal_separate_causal_forwards(small_cfg, small_weights):
+    """Brute force: verifying the linearised tree in one masked forward gives every node the logits a plain causal
+    forward over its root-to-node path gives."""
+    o = _oracle(small_cfg, small_weights)
+    o.prefill(synth.prompt(small_cfg, 11))
+    z = [1, 1, 0, 0, 1, 0, 0, 1]
+    d_tok, d_conf, d_rows = o.draft(z, 4)
+    tree = so.build_tree(o.tokens[-1], d_tok, d_rows, [0.4, 0.7, 0.9, 0.99], row_budget=32)    # widths 10, 5, 3, 1
+    assert len(tree.tokens) == 5 + 9 + 4 + 2
+    tl = o.verify_tree(tree)
+    for node in range(len(tree.tokens)):
+        path = []
+        j = node
+        while j >= 0:
+            path.append(j)
+            j = tree.parent[j]
+        path.reverse()
+        b = _oracle(small_cfg, small_weights)
+        b.forward_rows(o.tokens[:o.n], 0)
+        ref = b.forward_rows([tree.tokens[r] for r in path], o.n, write_kv=False)[-1]
+        assert torch.allclose(tl[node], ref, atol=1e-9, rtol=0), node
+
+
+@pytest.mark.parametrize("stop_conf", [0.0, 0.05])
+def test_tree_verification_is_lossless_and_never_shorter(small_cfg, small_weights, stop_conf):
+    """Section 3.1 / 4.2: with the tree every emitted token is still the target's arg max, so the output equals
+    vanilla greedy decoding for every skip set; and from the same state a tree round accepts at least as many
+    tokens as the chain alone."""
+    prompt = synth.prompt(small_cfg, 9)
+    ref, _ = so.vanilla_generate(_oracle(small_cfg, small_weights), prompt, 30)
+    gains = 0
+    for z in _masks(small_cfg):
+        o = _oracle(small_cfg, small_weights)
+        out, rounds, stats = so.swift_generate(o, prompt, z, so.GenParams(max_new=30, max_draft=4, stop_conf=stop_conf, tree_rows=16))
+        assert out == ref and len(out) == 30, z
+        fresh = _oracle(small_cfg, small_weights)
+        fresh.forward_rows(o.tokens[:o.n], 0)
+        for b in range(small_cfg.n_blocks):                       # accepted alternatives were moved to their slots
+            assert torch.allclose(o.K[b][:o.n], fresh.K[b][:o.n], atol=1e-10) and torch.allclose(o.V[b][:o.n], fresh.V[b][:o.n], atol=1e-10)
+        for r in rounds:
+            assert len(r.tree.tokens) <= max(16, len(r.draft) + 1) and r.tree.tokens[1:len(r.draft) + 1] == r.draft
+            chain_a, _ = so.accept_greedy(r.draft, torch.stack([torch.nn.functional.one_hot(torch.tensor(t), small_cfg.vocab).double()
+                                                                for t in r.target_argmax[:len(r.draft) + 1]]))
+            assert r.accepted >= chain_a
+            gains += r.accepted - chain_a
+    assert gains > 0                                              # some alternative was accepted somewhere
