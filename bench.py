@@ -98,6 +98,27 @@ def aggregate_replicas(tokens: int, decode_ms: float, total_ms: float, wall_s: f
     return world * tokens / (decode_ms * 1e-3), decode_ms, total_ms, wall_s
 
 
+def config_of(desc: str, kv_dtype: str):
+    """The `config` object of the JSON line; both arms (this library, the CPU oracle) print the same keys and values."""
+    return {"workload": desc, "l2": "inputs (weights) far larger than L2; no flush", "parallelism": "replicas only",
+            "kv_cache": kv_dtype, "e2e_note": "whole swift_generate call incl. prefill and host copies, host clock",
+            "context": PAPER_CONTEXT}
+
+
+def profile_traffic(shape: str, rows: int):
+    """DRAM bytes per launch of the gate/up GEMM from the ncu capture summarised under profiles/ (a line
+    `traffic: <shape> <rows> rows = <bytes> bytes per launch` in the summary that names its command), or None."""
+    path = os.path.join(ROOT, "profiles", "gemm_tc_gate_up_9rows.md")
+    try:
+        for line in open(path):
+            parts = line.split()
+            if len(parts) >= 7 and parts[0] == "traffic:" and parts[1] == shape and parts[2] == str(rows):
+                return float(parts[5])
+    except OSError:
+        pass
+    return None
+
+
 def workload(name: str):
     model_name, run = synth.RUNS[name]
     cfg = synth.MODELS[model_name]
@@ -105,14 +126,20 @@ def workload(name: str):
     return cfg, run, z
 
 
-def oracle_sample(cfg, run, z, weights, n_ctx=16, k=4, n_vanilla=3):
-    """The CPU oracle, as it stands, on a bounded slice of the workload: a short prefill, then n_vanilla
-    vanilla steps and one SWIFT round (k drafts + verify + accept).  Returns tokens/s of both."""
+def oracle_sample(cfg, run, z, weights, n_ctx, k=None, n_vanilla=3):
+    """The CPU oracle, as it stands, on a bounded slice of the workload at its final context length n_ctx: n_vanilla
+    vanilla steps and one SWIFT round (k drafts + verify + accept) behind a cache of n_ctx positions.  The cache is
+    filled with seeded random K,V instead of a prefill of n_ctx tokens (a forward's cost does not depend on the cached
+    values; the prefill alone would take minutes on host cores).  Returns tokens/s of both."""
     from oracle import swift_oracle as so
+    k = run.max_draft if k is None else k
     dtype = torch.float64 if cfg.dtype == "f32" else torch.float32
     o = so.Oracle(so.Shape.of(cfg), weights, dtype=dtype, max_positions=n_ctx + n_vanilla + k + 8)
-    prompt = synth.prompt(cfg, n_ctx)
-    o.prefill(prompt)
+    g = torch.Generator().manual_seed(1234)
+    for b in range(cfg.n_blocks):
+        o.K[b][:n_ctx] = torch.randn(n_ctx, cfg.n_kv_heads, cfg.head_dim, generator=g, dtype=dtype)
+        o.V[b][:n_ctx] = torch.randn(n_ctx, cfg.n_kv_heads, cfg.head_dim, generator=g, dtype=dtype)
+    o.n, o.tokens = n_ctx, synth.prompt(cfg, n_ctx + 1)
     t0 = time.perf_counter()
     for _ in range(n_vanilla):
         row = o.forward_rows([o.tokens[-1]], o.n)[0]
@@ -124,6 +151,23 @@ def oracle_sample(cfg, run, z, weights, n_ctx=16, k=4, n_vanilla=3):
     o.commit(d_tok[:a], nxt)
     t2 = time.perf_counter()
     return {"vanilla": n_vanilla / (t1 - t0), "swift": (a + 1) / (t2 - t1), "seconds": t2 - t0, "accepted": a, "k": k}
+
+
+def oracle_model(cfg, run, z, weights=None):
+    """The model the CPU baseline runs: the workload's own when its widened copy fits comfortably in host memory,
+    else an 8-block copy with the same widths (its throughput is scaled by depth and labelled as extrapolated)."""
+    small = cfg if cfg.n_blocks * cfg.block_params() < 8e9 else cfg.with_blocks(8)
+    if small is cfg:
+        return cfg, z, (weights if weights is not None else synth.make_weights(cfg)), 1.0
+    zz = synth.block_mask(small, synth.draft_blocks(small, max(1, run.n_skip_blocks * 8 // cfg.n_blocks)))
+    return small, zz, synth.make_weights(small), small.n_blocks / cfg.n_blocks
+
+
+def sample_text(cfg, small, run, n_ctx, seconds=None):
+    return (f"3 vanilla steps and one SWIFT round of {run.max_draft} drafts + verify + accept behind {n_ctx} cached positions "
+            f"(the workload's final context length; cache filled with seeded random K,V)"
+            + (f", {seconds:.1f} s of CPU work" if seconds is not None else "")
+            + ("" if small is cfg else "; on an 8-block copy of the model, scaled by depth (extrapolated)"))
 
 
 def micro(cfg, run, args, hbm_peak):
@@ -148,7 +192,7 @@ def main():
     ap.add_argument("--steps", type=int, default=3)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--workload", default="c2", choices=sorted(synth.RUNS))
+    ap.add_argument("--workload", default="c3", choices=sorted(synth.RUNS))
     ap.add_argument("--max-new", type=int, default=0, help="override the number of generated tokens")
     ap.add_argument("--prompt-len", type=int, default=0, help="override the prompt length (profiling runs)")
     ap.add_argument("--kv-dtype", default="f32", choices=["f32", "bf16"], help="storage of cached K,V")
@@ -178,21 +222,19 @@ def main():
         if rank != 0:
             return
         torch.set_num_threads(os.cpu_count() or 1)
-        small = cfg if cfg.n_blocks * cfg.block_params() < 16e9 else cfg.with_blocks(8)
-        zz = z if small is cfg else synth.block_mask(small, synth.draft_blocks(small, max(1, run.n_skip_blocks * 8 // cfg.n_blocks)))
-        w = synth.make_weights(small)
+        small, zz, w, scale = oracle_model(cfg, run, z)
+        n_ctx = run.prompt_len + max_new
         vals = []
         for i in range(args.warmup + args.steps):
-            s = oracle_sample(small, run, zz, w)
+            s = oracle_sample(small, run, zz, w, n_ctx)
             if i >= args.warmup:
                 vals.append(s)
-        v = statistics.mean(x["swift"] for x in vals) * (small.n_blocks / cfg.n_blocks if small is not cfg else 1.0)
-        sample = "per step: prefill of 16 tokens, then 3 vanilla steps and one SWIFT round of 4 drafts + verify + accept" + \
-                 ("" if small is cfg else f"; on an 8-block copy of the model, scaled by depth (extrapolated)")
+        v = statistics.mean(x["swift"] for x in vals) * scale
+        sample = "per step: " + sample_text(cfg, small, run, n_ctx)
         print(json.dumps({"impl": "reference", "metric": METRIC, "value": v, "unit": UNIT, "n_gpus": 0, "steps": args.steps,
                           "warmup": args.warmup, "ms_per_step": 1e3 * statistics.mean(x["seconds"] for x in vals),
                           "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
-                          "config": {"workload": desc},
+                          "config": config_of(desc, args.kv_dtype),
                           "cpu_baseline": {"value": v, "unit": UNIT, "cores": torch.get_num_threads(), "kind": "oracle", "sample": sample},
                           "e2e": {"value": v, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}))
         return
@@ -271,7 +313,12 @@ def main():
     # vanilla decoding of the same model for the comparison the metric names
     swift_tokens = model.generate(prompt, gp)[0]
     md, mv, bd, bv, kd = model.round_times()
+    sbd, sbv = model.round_bytes_stored()
     fdist = {"draft_frac": dist_of(md, bd, kd > 0), "verify_frac": dist_of(mv, bv, kd == run.max_draft)}
+    # the same rounds with cached K,V counted as they are stored (fp32 by default): what the implementation moves
+    fdist_stored = {"draft_frac": dist_of(md, sbd, kd > 0), "verify_frac": dist_of(mv, sbv, kd == run.max_draft)}
+    stored_ratio = {"draft": float(sbd[kd > 0].sum() / max(bd[kd > 0].sum(), 1.0)) if (kd > 0).any() else None,
+                    "verify": float(sbv.sum() / max(bv.sum(), 1.0))}
     # expected speedup of Eq. 5 (Appendix B.3) with the measured cost ratio c = one draft forward / one verification
     full = kd == run.max_draft
     c_meas = float(np.median(md[full] / kd[full]) / np.median(mv[full])) if full.any() and run.max_draft > 0 else None
@@ -282,7 +329,10 @@ def main():
     vanilla = (vst.tokens - 1) / (vst.ms_decode * 1e-3)
     lossless = None if sampling else (swift_tokens == v_tokens)   # greedy SWIFT must reproduce vanilla decoding
     _, vmv, _, vbv, _ = model.round_times()
+    _, vsbv = model.round_bytes_stored()
     fdist["vanilla_frac"] = dist_of(vmv, vbv, np.ones(len(vmv), dtype=bool))
+    fdist_stored["vanilla_frac"] = dist_of(vmv, vsbv, np.ones(len(vmv), dtype=bool))
+    stored_ratio["vanilla"] = float(vsbv.sum() / max(vbv.sum(), 1.0))
 
     s0 = stats[-1]
     n_ctx = run.prompt_len + max_new // 2
@@ -291,6 +341,12 @@ def main():
           "vanilla_gbs": vst.bytes_verify / (vst.ms_decode * 1e-3) * 1e-9,
           "draft_bytes": model.forward_bytes(z, 1, n_ctx), "verify_bytes": model.forward_bytes(None, run.max_draft + 1, n_ctx)}
     fw["draft_frac"], fw["verify_frac"], fw["vanilla_frac"] = (fw[k] / hbm_peak for k in ("draft_gbs", "verify_gbs", "vanilla_gbs"))
+    fw["bytes"] = "algorithmic: weights of the kept sub-layers + output head + cached K,V at 2 bytes per element + rows in/out"
+    # the same sums with the cache counted as stored (stored / algorithmic bytes of the same forwards)
+    fw["stored_bytes_ratio"] = stored_ratio
+    fw["draft_frac_stored_bytes"] = fw["draft_frac"] * stored_ratio["draft"] if stored_ratio["draft"] else None
+    fw["verify_frac_stored_bytes"] = fw["verify_frac"] * stored_ratio["verify"]
+    fw["vanilla_frac_stored_bytes"] = fw["vanilla_frac"] * stored_ratio["vanilla"]
 
     # dominant kernel: the weight-streaming GEMM (largest instance: fused gate/up), timed alone with CUDA events
     g_ms, g_bytes = model.time_gemm(2, run.max_draft + 1, 200)
@@ -298,50 +354,62 @@ def main():
     achieved = g_bytes / (g_ms * 1e-3) * 1e-9
     # DRAM bytes per launch of that kernel (read + write, mean of two launches) from the ncu captures summarised in
     # the profiles folder (7B and 13B widths, 9 rows); other shapes have no capture of their own
-    traffic = {"7b": 186.6e6, "13b": 289.6e6}.get(cfg.name) if run.max_draft == 8 else None
+    traffic = profile_traffic(cfg.name, run.max_draft + 1)
     roofline = {"bound": "hbm", "kernel": "skinny GEMM, fused gate/up projection, %d rows" % (run.max_draft + 1),
                 "achieved": achieved, "peak": hbm_peak, "peak_kind": f"{peak_kind} copy bandwidth (burst)", "unit": "GB/s",
                 "frac": achieved / hbm_peak, "traffic": traffic, "bytes_per_launch": g_bytes, "ms_per_launch": g_ms,
-                "one_row_frac": g_bytes / (g1_ms * 1e-3) * 1e-9 / hbm_peak}
+                "one_row_frac": g_bytes / (g1_ms * 1e-3) * 1e-9 / hbm_peak,
+                # whole forwards (every kernel of the walk), worst round of the run, algorithmic bytes: the target quantity
+                "forward_draft_frac": fdist["draft_frac"]["min"] if fdist["draft_frac"] else None,
+                "forward_verify_frac": fdist["verify_frac"]["min"] if fdist["verify_frac"] else None,
+                "forward_draft_frac_stored_bytes": fdist_stored["draft_frac"]["min"] if fdist_stored["draft_frac"] else None,
+                "forward_verify_frac_stored_bytes": fdist_stored["verify_frac"]["min"] if fdist_stored["verify_frac"] else None}
 
     out = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
            "ms_per_step": tot_ms / args.steps, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
            "dtype": "bf16" if cfg.dtype == "bf16" else "f32", "data": "synthetic",
-           "config": {"workload": desc, "l2": "inputs (weights) far larger than L2; no flush", "parallelism": "replicas only", "kv_cache": args.kv_dtype,
-                      "e2e_note": "whole swift_generate call incl. prefill and host copies, host clock", "context": PAPER_CONTEXT},
+           "config": config_of(desc, args.kv_dtype),
            "vanilla_tokens_per_s": vanilla, "swift_equals_vanilla": lossless, "speedup_vs_vanilla": value / world / vanilla,
            "M": (s0.tokens - 1) / s0.rounds, "alpha": s0.accepted / max(s0.drafted, 1), "rounds": s0.rounds,
-           "ms_prefill": s0.ms_prefill, "forwards": fw, "forwards_per_round": fdist, "roofline": roofline,
-           "e2e": {"value": e2e, "unit": UNIT, "h2d_bytes_per_step": 4 * run.prompt_len, "d2h_bytes_per_step": 448 * (s0.rounds + 1)},
+           "ms_prefill": s0.ms_prefill, "forwards": fw, "forwards_per_round": fdist, "forwards_per_round_stored_bytes": fdist_stored, "roofline": roofline,
+           "e2e": {"value": e2e, "unit": UNIT, "h2d_bytes_per_step": s0.h2d_bytes, "d2h_bytes_per_step": s0.d2h_bytes},
            "gpu_launches": launches, "clocks": clk.summary()}
 
+    # Candidate scoring (Eq. 2-3), for every shape: one round of the workload's candidate count on the last gamma generated
+    # tokens of the run that just ended, timed with CUDA events on the library's stream.  Bytes: what the method needs if
+    # every kept sub-layer's weights are streamed once per candidate (each candidate is one draft-model forward of gamma rows).
+    n_cand = run.n_candidates
+    probe = synth.candidate_masks(cfg, max(1, run.n_skip_blocks), n_cand, 0)
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    model.score_skipsets(probe[:2], run.gamma)                       # warm-up
+    with torch.cuda.stream(model.stream):
+        ev0.record(model.stream)
+        model.score_skipsets(probe, run.gamma)
+        ev1.record(model.stream)
+    torch.cuda.synchronize()
+    ms_round = ev0.elapsed_time(ev1)
+    n_end = run.prompt_len + max_new
+    sc_bytes = sum(model.forward_bytes(probe[c], run.gamma, n_end - run.gamma) for c in range(n_cand))
+    sc_gbs = sc_bytes / (ms_round * 1e-3) * 1e-9
+    out["scoring"] = {"candidates_per_round": n_cand, "gamma": run.gamma, "ms_per_round": ms_round, "gbs": sc_gbs,
+                      "frac": sc_gbs / hbm_peak, "bound": "hbm (weights streamed once per candidate)",
+                      "vs_one_vanilla_step": ms_round / (1e3 / vanilla)}
     if run.optimise and s0.opt_rounds > 0:
-        # candidate scoring (Eq. 2-3): every candidate is two 16-row forwards under its own skip set over the gamma context
-        # tokens; bytes = the algorithmic bytes of those forwards at the context length where scoring starts
-        sc_bytes = sum(2 * model.forward_bytes(cands[r][c], 16, run.prompt_len + run.gamma)
-                       for r in range(s0.opt_rounds) for c in range(cands.shape[1]))
-        sc_gbs = sc_bytes / (s0.ms_score * 1e-3) * 1e-9
-        out["scoring"] = {"opt_rounds": s0.opt_rounds, "candidates_per_round": int(cands.shape[1]), "gamma": run.gamma,
-                          "ms_per_round": s0.ms_score / s0.opt_rounds, "best_matchness": s0.best_matchness,
-                          "gbs": sc_gbs, "frac": sc_gbs / hbm_peak, "share_of_decode": s0.ms_score / s0.ms_decode}
+        out["scoring"].update({"opt_rounds": s0.opt_rounds, "ms_per_round_in_run": s0.ms_score / s0.opt_rounds,
+                               "best_matchness": s0.best_matchness, "share_of_decode": s0.ms_score / s0.ms_decode})
     if c_meas is not None:
         M_, a_ = out["M"], out["alpha"]
         out["eq5"] = {"c_measured": c_meas, "expected_speedup": M_ * a_ / ((M_ - 1) * c_meas + a_) if a_ > 0 else None,
                       "achieved_speedup": out["speedup_vs_vanilla"]}
 
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
-        small = cfg if weights is not None and cfg.n_blocks * cfg.block_params() < 16e9 else cfg.with_blocks(8)
-        zz = z if small is cfg else synth.block_mask(small, synth.draft_blocks(small, max(1, run.n_skip_blocks * 8 // cfg.n_blocks)))
-        w = weights if small is cfg else synth.make_weights(small)
         model.close()
+        small, zz, w, scale = oracle_model(cfg, run, z, weights)
         torch.set_num_threads(os.cpu_count() or 1)
-        s = oracle_sample(small, run, zz, w)
-        scale = 1.0 if small is cfg else small.n_blocks / cfg.n_blocks
+        n_ctx = run.prompt_len + max_new
+        s = oracle_sample(small, run, zz, w, n_ctx)
         out["cpu_baseline"] = {"value": s["swift"] * scale, "unit": UNIT, "cores": torch.get_num_threads(), "kind": "oracle",
-                               "vanilla_value": s["vanilla"] * scale,
-                               "sample": "prefill of 16 tokens, then 3 vanilla steps and one SWIFT round of 4 drafts + verify "
-                                         "+ accept (%.1f s of CPU work)%s" % (s["seconds"], "" if small is cfg else
-                                                                               "; 8-block copy scaled by depth (extrapolated)")}
+                               "vanilla_value": s["vanilla"] * scale, "sample": sample_text(cfg, small, run, n_ctx, s["seconds"])}
     if rank == 0:
         print(json.dumps(out))
     if world > 1:

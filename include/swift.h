@@ -241,6 +241,9 @@ double swift_forward_bytes(const swift_ctx* ctx, const uint8_t* skip_mask_host, 
 int32_t swift_final_skip_mask(const swift_ctx* ctx, uint8_t* mask_host);
 int32_t swift_round_times(const swift_ctx* ctx, int32_t capacity, float* ms_draft_host, float* ms_verify_host,
                           double* bytes_draft_host, double* bytes_verify_host, int32_t* drafted_host);
+/* The same rounds' bytes with cached K,V counted as this context stores them (swift_forward_bytes with kv_elem_bytes 0):
+ * what the implementation moves, beside the algorithmic figure above.  Same conventions as swift_round_times. */
+int32_t swift_round_bytes_stored(const swift_ctx* ctx, int32_t capacity, double* bytes_draft_host, double* bytes_verify_host);
 /* Times `iters` back-to-back launches of one weight-streaming GEMM of the walk (which: 0 fused QKV,
  * 1 o_proj, 2 fused gate/up, 3 down, 4 output head) with n_rows rows, cycling over the blocks' weights
  * so that successive launches read different memory.  Outputs the average CUDA-event time per launch

@@ -54,7 +54,7 @@ class _Stats(C.Structure):
 SYMBOLS = ("swift_weights_bytes", "swift_kv_bytes", "swift_workspace_bytes", "swift_load", "swift_free",
            "swift_last_error", "swift_pack_tensor", "swift_set_sampling", "swift_set_top_p", "swift_set_greedy_draft", "swift_forward_rows", "swift_prefill",
            "swift_set_pending", "swift_draft", "swift_verify", "swift_accept", "swift_score_skipsets", "swift_generate",
-           "swift_committed_length", "swift_launch_count", "swift_round_times", "swift_final_skip_mask", "swift_forward_bytes", "swift_read_kv", "swift_time_gemm", "swift_set_gemm_impl", "swift_gemm", "swift_gemm_static",
+           "swift_committed_length", "swift_launch_count", "swift_round_times", "swift_round_bytes_stored", "swift_final_skip_mask", "swift_forward_bytes", "swift_read_kv", "swift_time_gemm", "swift_set_gemm_impl", "swift_gemm", "swift_gemm_static",
            "swift_gemm_static_error")
 
 _lib = None
@@ -94,6 +94,8 @@ def load_library(path: Optional[str] = None) -> C.CDLL:
     lib.swift_final_skip_mask.restype = C.c_int32
     lib.swift_round_times.argtypes = [vp, i32, vp, vp, vp, vp, vp]
     lib.swift_round_times.restype = C.c_int32
+    lib.swift_round_bytes_stored.argtypes = [vp, i32, vp, vp]
+    lib.swift_round_bytes_stored.restype = C.c_int32
     lib.swift_forward_bytes.argtypes = [vp, vp, i32, i32, i32]
     lib.swift_forward_bytes.restype = C.c_double
     lib.swift_set_gemm_impl.argtypes = [vp, i32]
@@ -350,6 +352,13 @@ class SwiftModel:
         k = np.zeros(n, dtype=np.int32)
         self._lib.swift_round_times(self.ctx, n, _ptr(md), _ptr(mv), _ptr(bd), _ptr(bv), _ptr(k))
         return md, mv, bd, bv, k
+
+    def round_bytes_stored(self):
+        """Per round of the last generate(): (bytes_draft, bytes_verify) with cached K,V counted as stored."""
+        n = self._lib.swift_round_bytes_stored(self.ctx, 0, None, None)
+        bd, bv = np.zeros(n, dtype=np.float64), np.zeros(n, dtype=np.float64)
+        self._lib.swift_round_bytes_stored(self.ctx, n, _ptr(bd), _ptr(bv))
+        return bd, bv
 
     def set_gemm_impl(self, tensor_cores: bool):
         self._check(self._lib.swift_set_gemm_impl(self.ctx, 1 if tensor_cores else 0))

@@ -4,7 +4,7 @@
 //
 // One CTA = one KV head x one chunk, for ALL query heads of that KV head's group and all rows of the forward
 // (R = group size x rows "query rows"), so a K/V byte is loaded once per forward however many heads share it.
-// The contraction is issued "swapped", with the streamed operand on the M side of mma.sync.m16n8k8 (tf32):
+// The contraction is issued "swapped", with the streamed operand on the M side of mma.sync.m16n8k16 (bf16):
 //     S^T [16 positions x 8 query rows] = K [16 positions x 128 dims]   . Q^T [128 dims x 8 query rows]
 //     O^T [16 dims      x 8 query rows] = V^T [16 dims x 16 positions]  . P^T [16 positions x 8 query rows]
 // so accumulator registers scale with the number of query rows (one 8-row tile for a one-row forward, two for a
@@ -14,8 +14,11 @@
 // fragment elements are picked out of them, no shuffle and no shared-memory staging.  Warp w owns positions
 // [16w, 16w + 16) of the chunk; the four warps' partial results are merged in warp order.
 //
-// Precision: cached K,V and the queries are fp32.  Each tf32 operand is split into hi = tf32(x) and lo = x - hi and
-// a product is three MMAs (lo*hi, hi*lo, hi*hi), which keeps about 21 mantissa bits; accumulation is fp32.
+// Precision: cached K,V and the queries are fp32.  Every operand is split into two bf16 numbers, hi = bf16(x) and
+// lo = bf16(x - hi) (16 significant bits together, the same treatment the weight-streaming GEMM gives its
+// activations), and a product is three MMAs (lo*hi, hi*lo, hi*hi); accumulation is fp32.  (The tf32 form of the
+// same kernel, m16n8k8 with four times as many MMA instructions, was bound by the issue rate of the legacy tensor
+// path and slower than the FMA kernel it was meant to replace.)
 //
 // Which rows a query row sees among the forward's own rows comes from a bit mask per row in the control block
 // (plain causal order, or the ancestors of a node when a token tree is verified); cached positions below the
@@ -27,29 +30,27 @@
 namespace swk {
 
 constexpr int AM_THREADS = 128;
-constexpr int AM_QSTRIDE = 144;     // floats per staged query row: the 8 rows of a fragment load fall into different banks
+constexpr int AM_QSTRIDE = 144;     // bf16 per staged query row (288 bytes): the rows of a fragment load fall into different banks
 constexpr int AM_OSTRIDE = 132;     // floats per row of a warp's partial output
 constexpr int AM_PSTRIDE = 20;      // floats per row of a warp's probabilities (16 positions)
 
 __host__ __device__ constexpr size_t attn_mma_smem_bytes(int nt, int max_splits)
 {
-    return (size_t)(2 * 8 * nt * AM_QSTRIDE + 4 * 8 * nt * AM_OSTRIDE + 4 * 8 * nt * AM_PSTRIDE + 2 * 4 * 8 * nt + 2 * max_splits) * 4;
+    return (size_t)(2 * 8 * nt * AM_QSTRIDE) * 2 +
+           (size_t)(4 * 8 * nt * AM_OSTRIDE + 4 * 8 * nt * AM_PSTRIDE + 2 * 4 * 8 * nt + 2 * max_splits) * 4;
 }
 
-__device__ __forceinline__ uint32_t tf32_of(float x)
+// Two fp32 numbers -> their bf16 hi parts and lo parts, each pair packed into one register (first number in the
+// low half, as the MMA fragments want it): hi = bf16(x), lo = bf16(x - hi), both rounded to nearest.
+__device__ __forceinline__ void split_pair(float x0, float x1, uint32_t& hi, uint32_t& lo)
 {
-    uint32_t r;
-    asm("cvt.rna.tf32.f32 %0, %1;" : "=r"(r) : "f"(x));
-    return r;
+    asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(hi) : "f"(x1), "f"(x0));
+    const float r0 = x0 - __uint_as_float(hi << 16), r1 = x1 - __uint_as_float(hi & 0xFFFF0000u);
+    asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(lo) : "f"(r1), "f"(r0));
 }
-__device__ __forceinline__ void split_tf32(float x, uint32_t& hi, uint32_t& lo)
+__device__ __forceinline__ void mma_bf16(float (&c)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1)
 {
-    hi = tf32_of(x);
-    lo = __float_as_uint(x - __uint_as_float(hi));
-}
-__device__ __forceinline__ void mma_tf32(float (&c)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1)
-{
-    asm volatile("mma.sync.aligned.m16n8k8.row.col.f32.tf32.tf32.f32 {%0, %1, %2, %3}, {%4, %5, %6, %7}, {%8, %9}, {%0, %1, %2, %3};"
+    asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0, %1, %2, %3}, {%4, %5, %6, %7}, {%8, %9}, {%0, %1, %2, %3};"
                  : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
                  : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
 }
@@ -57,9 +58,9 @@ __device__ __forceinline__ void mma_tf32(float (&c)[4], const uint32_t (&a)[4], 
 __device__ __forceinline__ void mma_split(float (&c)[4], const uint32_t (&ah)[4], const uint32_t (&al)[4], uint32_t bh0,
                                           uint32_t bh1, uint32_t bl0, uint32_t bl1)
 {
-    mma_tf32(c, al, bh0, bh1);
-    mma_tf32(c, ah, bl0, bl1);
-    mma_tf32(c, ah, bh0, bh1);
+    mma_bf16(c, al, bh0, bh1);
+    mma_bf16(c, ah, bl0, bl1);
+    mma_bf16(c, ah, bh0, bh1);
 }
 
 // grid = (n_kv_heads, max_splits), block = 128, dynamic smem = attn_mma_smem_bytes(NT, max_splits).
@@ -88,9 +89,9 @@ attn_mma_kernel(const DevState* st, const float* __restrict__ q, const T* __rest
     const bool live = j0 < len;                             // this warp's 16 positions hold something
 
     extern __shared__ __align__(16) float am_smem[];
-    float* q_hi = am_smem;                                  // [QR][AM_QSTRIDE] (tf32 bit patterns)
-    float* q_lo = q_hi + QR * AM_QSTRIDE;
-    float* part_acc = q_lo + QR * AM_QSTRIDE;               // [4][QR][AM_OSTRIDE]
+    __nv_bfloat16* q_hi = reinterpret_cast<__nv_bfloat16*>(am_smem);   // [QR][AM_QSTRIDE]
+    __nv_bfloat16* q_lo = q_hi + QR * AM_QSTRIDE;
+    float* part_acc = reinterpret_cast<float*>(q_lo + QR * AM_QSTRIDE);   // [4][QR][AM_OSTRIDE]
     float* p_sh = part_acc + 4 * QR * AM_OSTRIDE;           // [4][QR][AM_PSTRIDE]
     float2* part_ml = reinterpret_cast<float2*>(p_sh + 4 * QR * AM_PSTRIDE);   // [4][QR]
     float* comb_sh = reinterpret_cast<float*>(part_ml + 4 * QR);               // [2 * max_splits]
@@ -139,10 +140,11 @@ attn_mma_kernel(const DevState* st, const float* __restrict__ q, const T* __rest
                 v = *reinterpret_cast<const float4*>(q + ((size_t)r * n_heads + kvh * G + hl) * DH + c4 * 4);
                 v.x *= scale; v.y *= scale; v.z *= scale; v.w *= scale;
             }
-            uint4 hi, lo;
-            split_tf32(v.x, hi.x, lo.x); split_tf32(v.y, hi.y, lo.y); split_tf32(v.z, hi.z, lo.z); split_tf32(v.w, hi.w, lo.w);
-            *reinterpret_cast<uint4*>(q_hi + rl * AM_QSTRIDE + c4 * 4) = hi;
-            *reinterpret_cast<uint4*>(q_lo + rl * AM_QSTRIDE + c4 * 4) = lo;
+            uint2 hi, lo;
+            split_pair(v.x, v.y, hi.x, lo.x);
+            split_pair(v.z, v.w, hi.y, lo.y);
+            *reinterpret_cast<uint2*>(q_hi + rl * AM_QSTRIDE + c4 * 4) = hi;
+            *reinterpret_cast<uint2*>(q_lo + rl * AM_QSTRIDE + c4 * 4) = lo;
         }
         __syncthreads();
 
@@ -152,22 +154,16 @@ attn_mma_kernel(const DevState* st, const float* __restrict__ q, const T* __rest
 #pragma unroll
             for (int nt = 0; nt < NT; ++nt) { sacc[nt][0] = sacc[nt][1] = sacc[nt][2] = sacc[nt][3] = 0.f; }
 #pragma unroll
-            for (int j = 0; j < 8; ++j) {
-                uint4 bh[NT], bl[NT];
+            for (int j = 0; j < 8; ++j) {                   // k-step j: dims 16j .. 16j + 15, this lane's share 16j + 4t .. + 3
+                uint32_t ah[4], al[4];
+                split_pair(kA[j].x, kA[j].y, ah[0], al[0]); split_pair(kB[j].x, kB[j].y, ah[1], al[1]);
+                split_pair(kA[j].z, kA[j].w, ah[2], al[2]); split_pair(kB[j].z, kB[j].w, ah[3], al[3]);
 #pragma unroll
                 for (int nt = 0; nt < NT; ++nt) {
-                    bh[nt] = *reinterpret_cast<const uint4*>(q_hi + (8 * nt + g) * AM_QSTRIDE + 16 * j + 4 * t);
-                    bl[nt] = *reinterpret_cast<const uint4*>(q_lo + (8 * nt + g) * AM_QSTRIDE + 16 * j + 4 * t);
+                    const uint2 bh = *reinterpret_cast<const uint2*>(q_hi + (8 * nt + g) * AM_QSTRIDE + 16 * j + 4 * t);
+                    const uint2 bl = *reinterpret_cast<const uint2*>(q_lo + (8 * nt + g) * AM_QSTRIDE + 16 * j + 4 * t);
+                    mma_split(sacc[nt], ah, al, bh.x, bh.y, bl.x, bl.y);
                 }
-                uint32_t ah[4], al[4];
-                split_tf32(kA[j].x, ah[0], al[0]); split_tf32(kB[j].x, ah[1], al[1]);
-                split_tf32(kA[j].y, ah[2], al[2]); split_tf32(kB[j].y, ah[3], al[3]);
-#pragma unroll
-                for (int nt = 0; nt < NT; ++nt) mma_split(sacc[nt], ah, al, bh[nt].x, bh[nt].y, bl[nt].x, bl[nt].y);
-                split_tf32(kA[j].z, ah[0], al[0]); split_tf32(kB[j].z, ah[1], al[1]);
-                split_tf32(kA[j].w, ah[2], al[2]); split_tf32(kB[j].w, ah[3], al[3]);
-#pragma unroll
-                for (int nt = 0; nt < NT; ++nt) mma_split(sacc[nt], ah, al, bh[nt].z, bh[nt].w, bl[nt].z, bl[nt].w);
             }
 
             // ---- soft-max over this warp's 16 positions, per query row (the 8 lanes that share t hold one row's scores)
@@ -214,24 +210,23 @@ attn_mma_kernel(const DevState* st, const float* __restrict__ q, const T* __rest
             for (int nt = 0; nt < NT; ++nt)
 #pragma unroll
                 for (int mt = 0; mt < 8; ++mt) { oacc[nt][mt][0] = oacc[nt][mt][1] = oacc[nt][mt][2] = oacc[nt][mt][3] = 0.f; }
-#pragma unroll
-            for (int step = 0; step < 2; ++step) {          // positions {t, t + 4} + 8 * step of the warp's 16
+            {                                               // one k-step: the warp's 16 positions, this lane's share t, t + 4, t + 8, t + 12
                 uint32_t bh0[NT], bh1[NT], bl0[NT], bl1[NT];
 #pragma unroll
                 for (int nt = 0; nt < NT; ++nt) {
-                    split_tf32(pw[(8 * nt + g) * AM_PSTRIDE + t + 8 * step], bh0[nt], bl0[nt]);
-                    split_tf32(pw[(8 * nt + g) * AM_PSTRIDE + t + 4 + 8 * step], bh1[nt], bl1[nt]);
+                    const float* pr = pw + (8 * nt + g) * AM_PSTRIDE + t;
+                    split_pair(pr[0], pr[4], bh0[nt], bl0[nt]);
+                    split_pair(pr[8], pr[12], bh1[nt], bl1[nt]);
                 }
 #pragma unroll
                 for (int i = 0; i < 4; ++i) {
-                    const float4 va = vv[2 * step][i], vb = vv[2 * step + 1][i];
                     uint32_t ah[4], al[4];
-                    split_tf32(va.x, ah[0], al[0]); split_tf32(va.y, ah[1], al[1]);
-                    split_tf32(vb.x, ah[2], al[2]); split_tf32(vb.y, ah[3], al[3]);
+                    split_pair(vv[0][i].x, vv[1][i].x, ah[0], al[0]); split_pair(vv[0][i].y, vv[1][i].y, ah[1], al[1]);
+                    split_pair(vv[2][i].x, vv[3][i].x, ah[2], al[2]); split_pair(vv[2][i].y, vv[3][i].y, ah[3], al[3]);
 #pragma unroll
                     for (int nt = 0; nt < NT; ++nt) mma_split(oacc[nt][2 * i], ah, al, bh0[nt], bh1[nt], bl0[nt], bl1[nt]);
-                    split_tf32(va.z, ah[0], al[0]); split_tf32(va.w, ah[1], al[1]);
-                    split_tf32(vb.z, ah[2], al[2]); split_tf32(vb.w, ah[3], al[3]);
+                    split_pair(vv[0][i].z, vv[1][i].z, ah[0], al[0]); split_pair(vv[0][i].w, vv[1][i].w, ah[1], al[1]);
+                    split_pair(vv[2][i].z, vv[3][i].z, ah[2], al[2]); split_pair(vv[2][i].w, vv[3][i].w, ah[3], al[3]);
 #pragma unroll
                     for (int nt = 0; nt < NT; ++nt) mma_split(oacc[nt][2 * i + 1], ah, al, bh0[nt], bh1[nt], bl0[nt], bl1[nt]);
                 }

@@ -80,7 +80,7 @@ struct swift_ctx {
     std::vector<FwdGraph>* graphs;
     uint64_t graph_clock;
     // per-round record of the last swift_generate (swift_round_times)
-    struct RoundTime { float ms_draft, ms_verify; double bytes_draft, bytes_verify; int32_t drafted; };
+    struct RoundTime { float ms_draft, ms_verify; double bytes_draft, bytes_verify; int32_t drafted; double stored_draft, stored_verify; };
     std::vector<RoundTime> round_times;
     std::vector<uint8_t> last_mask;          // skip set in use when the last swift_generate ended (swift_final_skip_mask)
     // tensor-core GEMM path (bf16 models)
@@ -1373,6 +1373,16 @@ int32_t swift_round_times(const swift_ctx* ctx, int32_t capacity, float* ms_draf
     }
     return n;
 }
+int32_t swift_round_bytes_stored(const swift_ctx* ctx, int32_t capacity, double* bytes_draft, double* bytes_verify)
+{
+    if (!ctx) return -1;
+    const int n = (int)ctx->round_times.size();
+    for (int i = 0; i < n && i < capacity; ++i) {
+        if (bytes_draft) bytes_draft[i] = ctx->round_times[i].stored_draft;
+        if (bytes_verify) bytes_verify[i] = ctx->round_times[i].stored_verify;
+    }
+    return n;
+}
 double swift_forward_bytes(const swift_ctx* ctx, const uint8_t* skip, int32_t n_rows, int32_t n_context, int32_t kv_elem_bytes)
 {
     return ctx ? forward_bytes(ctx, skip, n_rows, n_context, kv_elem_bytes) : 0.0;
@@ -1527,7 +1537,7 @@ swift_status swift_generate(swift_ctx* ctx, const swift_gen_params* gp, const in
             const double bv = forward_bytes(ctx, nullptr, 1, n_start);
             stt.ms_verify += mv;
             stt.bytes_verify += bv;
-            ctx->round_times.push_back({0.f, mv, 0.0, bv, 0});
+            ctx->round_times.push_back({0.f, mv, 0.0, bv, 0, 0.0, forward_bytes(ctx, nullptr, 1, n_start, 0)});
         } else {
             if (optimising && count >= gp->gamma) {
                 CU(cudaEventRecord(ev[2], ctx->stream));
@@ -1572,7 +1582,9 @@ swift_status swift_generate(swift_ctx* ctx, const swift_gen_params* gp, const in
             const double bv = forward_bytes(ctx, nullptr, hs.n_drafted + 1, n_start);
             stt.bytes_draft += bd;
             stt.bytes_verify += bv;
-            ctx->round_times.push_back({md, mv, bd, bv, hs.n_drafted});
+            double sd = 0.0;                      // the same forwards with the cache counted as it is stored
+            for (int j = 0; j < hs.n_drafted; ++j) sd += forward_bytes(ctx, z.data(), 1, n_start + j, 0);
+            ctx->round_times.push_back({md, mv, bd, bv, hs.n_drafted, sd, forward_bytes(ctx, nullptr, hs.n_drafted + 1, n_start, 0)});
             stt.drafted += hs.n_drafted;
             stt.accepted += hs.n_accepted;
         }
