@@ -586,3 +586,135 @@ def swift_generate(o: Oracle, prompt: Sequence[int], z0: Sequence[int], gp: GenP
 def expected_speedup(M: float, alpha: float, c: float) -> float:
     """Eq. 5: E(Spd.) = M*alpha / ((M-1)*c + alpha), c = 1 - r the draft/target cost ratio."""
     return M * alpha / ((M - 1.0) * c + alpha)
+
+
+# =============================================================================== layer set suggestion (Section 4.1)
+class LayerSetOptimizer:
+    """Proposes skipped-layer sets for the on-the-fly optimisation (Section 4.1, 'Efficient Layer Set Suggestion').
+
+    The input space is all sets of m of the n_blocks blocks (skip ratio r = m / n_blocks fixed).  Optimisation step o
+    (counted from 1) proposes a uniformly random set, except every beta-th step, which asks a Gaussian-process model of
+    matchness over the sets seen so far for the set with the highest upper confidence bound (Bayesian optimisation).
+    The paper delegates that part to a third-party package and prints no formulas; this is the textbook form:
+
+      * a set is its indicator vector x in {0,1}^n_blocks; the squared distance of two sets is their Hamming distance;
+      * prior: zero-mean GP on standardised scores, Matern-5/2 covariance k(d) = (1 + s + s^2/3) exp(-s), s = sqrt(5) d / ell,
+        observation noise `noise`; ell is the one of `ells` with the highest marginal likelihood;
+      * posterior mean and variance by a Cholesky factorisation of K + noise * I;
+      * acquisition mu + kappa * sigma, maximised over a pool: `pool` random sets plus every set one swap away from the
+        best set seen; sets already evaluated are left out.
+
+    Random draws come from Philox4x32-10 keyed by `seed`: counter (index, 0, stream, 0x4F5054), one word per draw.
+    """
+
+    def __init__(self, n_blocks: int, m: int, beta: int = 25, seed: int = 0, pool: int = 512, kappa: float = 2.576,
+                 noise: float = 1e-2, ells: Sequence[float] = (1.0, 2.0, 4.0)):
+        assert 0 < m < n_blocks
+        self.nb, self.m, self.beta, self.seed, self.pool, self.kappa, self.noise, self.ells = n_blocks, m, beta, seed, pool, kappa, noise, tuple(ells)
+        self.step = 0                       # optimisation steps taken (= proposals made)
+        self.draws = 0                      # random words consumed
+        self.X: List[Tuple[int, ...]] = []  # evaluated sets (sorted block tuples) ...
+        self.y: List[float] = []            # ... and their matchness
+
+    # ---- random sets
+    def _word(self) -> int:
+        w = philox4x32_10((self.draws & _MASK32, self.draws >> 32, 7, 0x4F5054), (self.seed & _MASK32, (self.seed >> 32) & _MASK32))[0]
+        self.draws += 1
+        return w
+
+    def random_set(self) -> Tuple[int, ...]:
+        """m blocks by a partial Fisher-Yates shuffle: position i swaps with i + word mod (n - i)."""
+        idx = list(range(self.nb))
+        for i in range(self.m):
+            j = i + self._word() % (self.nb - i)
+            idx[i], idx[j] = idx[j], idx[i]
+        return tuple(sorted(idx[:self.m]))
+
+    # ---- Gaussian process
+    @staticmethod
+    def matern52(d2, ell: float):
+        import numpy as np
+        s = np.sqrt(5.0 * np.asarray(d2, dtype=np.float64)) / ell
+        return (1.0 + s + s * s / 3.0) * np.exp(-s)
+
+    def _indicator(self, sets):
+        import numpy as np
+        X = np.zeros((len(sets), self.nb))
+        for i, s in enumerate(sets):
+            X[i, list(s)] = 1.0
+        return X
+
+    def fit(self):
+        """Standardises the scores and picks ell by marginal likelihood.  Returns what predict() needs."""
+        import numpy as np
+        X = self._indicator(self.X)
+        y = np.asarray(self.y, dtype=np.float64)
+        mu, sd = y.mean(), y.std()
+        sd = sd if sd > 1e-12 else 1.0
+        t = (y - mu) / sd
+        d2 = (X[:, None, :] != X[None, :, :]).sum(-1).astype(np.float64)
+        best = None
+        for ell in self.ells:
+            K = self.matern52(d2, ell) + self.noise * np.eye(len(y))
+            Lc = np.linalg.cholesky(K)
+            a = np.linalg.solve(Lc.T, np.linalg.solve(Lc, t))
+            lml = -0.5 * float(t @ a) - float(np.log(np.diag(Lc)).sum()) - 0.5 * len(y) * math.log(2.0 * math.pi)
+            if best is None or lml > best[0]:
+                best = (lml, ell, Lc, a)
+        return {"X": X, "mu": mu, "sd": sd, "ell": best[1], "L": best[2], "alpha": best[3], "lml": best[0]}
+
+    def predict(self, model, sets):
+        """Posterior mean and standard deviation of matchness at `sets` (in matchness units)."""
+        import numpy as np
+        Z = self._indicator(sets)
+        d2 = (Z[:, None, :] != model["X"][None, :, :]).sum(-1).astype(np.float64)
+        Ks = self.matern52(d2, model["ell"])
+        mean = Ks @ model["alpha"]
+        v = np.linalg.solve(model["L"], Ks.T)
+        var = np.maximum(1.0 - (v * v).sum(0), 0.0)
+        return model["mu"] + model["sd"] * mean, model["sd"] * np.sqrt(var)
+
+    # ---- proposals
+    def best_set(self) -> Optional[Tuple[int, ...]]:
+        """The evaluated set with the highest matchness (the earliest among equals)."""
+        if not self.y:
+            return None
+        return self.X[max(range(len(self.y)), key=lambda i: (self.y[i], -i))]
+
+    def bayesian_set(self) -> Tuple[Tuple[int, ...], dict]:
+        """The unevaluated set with the highest mu + kappa * sigma among `pool` random sets and the one-swap
+        neighbours of the best set seen (pool order, earliest among equals)."""
+        cand: List[Tuple[int, ...]] = [self.random_set() for _ in range(self.pool)]
+        inc = self.best_set()
+        if inc is not None:
+            outside = [b for b in range(self.nb) if b not in inc]
+            for out_b in inc:
+                for in_b in outside:
+                    cand.append(tuple(sorted((set(inc) - {out_b}) | {in_b})))
+        seen = set(self.X)
+        cand = [c for c in dict.fromkeys(cand) if c not in seen]
+        if not cand or not self.X:
+            return (cand[0] if cand else self.random_set()), {}
+        model = self.fit()
+        mean, std = self.predict(model, cand)
+        ucb = mean + self.kappa * std
+        i = max(range(len(cand)), key=lambda j: (float(ucb[j]), -j))
+        return cand[i], {"ucb": float(ucb[i]), "candidates": cand, "ucb_all": ucb, "model": model}
+
+    def suggest(self) -> Tuple[int, ...]:
+        """The next proposal: Bayesian every beta-th step once something has been evaluated, random otherwise."""
+        self.step += 1
+        if self.beta > 0 and self.step % self.beta == 0 and self.X:
+            return self.bayesian_set()[0]
+        return self.random_set()
+
+    def observe(self, blocks: Sequence[int], matchness: float) -> None:
+        self.X.append(tuple(sorted(int(b) for b in blocks)))
+        self.y.append(float(matchness))
+
+    def mask(self, blocks: Sequence[int]) -> List[int]:
+        """Sub-layer mask [attn_0, mlp_0, ...] that skips both sub-layers of every block in `blocks`."""
+        z = [0] * (2 * self.nb)
+        for b in blocks:
+            z[2 * b] = z[2 * b + 1] = 1
+        return z
