@@ -187,6 +187,12 @@ typedef struct {
     int32_t gamma, n_candidates, n_opt_rounds;
     float stop_matchness;
     int32_t opt_patience;
+    /* candidate_masks == NULL with n_opt_rounds > 0: the library proposes the candidates itself ("Efficient Layer Set
+     * Suggestion", Section 4.1): sets of opt_skip_blocks whole blocks, uniformly random except every opt_beta-th
+     * proposal (counted over the whole run), which maximises the upper confidence bound of a Gaussian-process model of
+     * the scores seen so far (opt_beta 0 = random search only; the paper uses 25).  Seeded by opt_seed. */
+    int32_t opt_skip_blocks, opt_beta;
+    uint64_t opt_seed;
     const uint8_t* skip_mask;       /* host, [2*n_blocks]: the (initial) draft skip set */
     const uint8_t* candidate_masks; /* host, [n_opt_rounds][n_candidates][2*n_blocks] or NULL */
 } swift_gen_params;
@@ -206,6 +212,18 @@ typedef struct {
 swift_status swift_generate(swift_ctx* ctx, const swift_gen_params* params, const int32_t* prompt_host,
                             int32_t n_prompt, int32_t* out_tokens_host, int32_t* n_out_host,
                             int32_t* trace_host, swift_stats* stats);
+
+/*
+ * The proposal engine on its own (host only, no device work): "Efficient Layer Set Suggestion" of Section 4.1.
+ * swift_opt_suggest writes the next proposal as a sub-layer mask [2*n_blocks] (both sub-layers of each chosen block)
+ * and, when is_bayesian_host is not NULL, whether it came from the Gaussian-process step; swift_opt_observe records
+ * the matchness a mask obtained (any mask that skips whole blocks).  NULL / SWIFT_EINVAL on bad arguments.
+ */
+typedef struct swift_opt swift_opt;
+swift_opt* swift_opt_create(int32_t n_blocks, int32_t n_skip_blocks, int32_t beta, uint64_t seed, int32_t pool);
+void swift_opt_free(swift_opt* opt);
+swift_status swift_opt_suggest(swift_opt* opt, uint8_t* mask_host, int32_t* is_bayesian_host);
+swift_status swift_opt_observe(swift_opt* opt, const uint8_t* mask_host, float matchness);
 
 /* Selects the kernel behind the weight-streaming GEMMs: 1 = tensor cores (tcgen05 + TMA; default and
  * only sensible choice for bf16 models), 0 = the SIMT kernel (always used for fp32 models; for bf16 it

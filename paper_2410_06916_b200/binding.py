@@ -39,8 +39,8 @@ class _DevBuf(C.Structure):
 class _GenParams(C.Structure):
     _fields_ = [("max_new", C.c_int32), ("max_draft", C.c_int32), ("stop_conf", C.c_float), ("vanilla", C.c_int32),
                 ("gamma", C.c_int32), ("n_candidates", C.c_int32), ("n_opt_rounds", C.c_int32),
-                ("stop_matchness", C.c_float), ("opt_patience", C.c_int32), ("skip_mask", C.c_void_p),
-                ("candidate_masks", C.c_void_p)]
+                ("stop_matchness", C.c_float), ("opt_patience", C.c_int32), ("opt_skip_blocks", C.c_int32),
+                ("opt_beta", C.c_int32), ("opt_seed", C.c_uint64), ("skip_mask", C.c_void_p), ("candidate_masks", C.c_void_p)]
 
 
 class _Stats(C.Structure):
@@ -55,7 +55,7 @@ SYMBOLS = ("swift_weights_bytes", "swift_kv_bytes", "swift_workspace_bytes", "sw
            "swift_last_error", "swift_pack_tensor", "swift_set_sampling", "swift_set_top_p", "swift_set_greedy_draft", "swift_forward_rows", "swift_prefill",
            "swift_set_pending", "swift_draft", "swift_verify", "swift_accept", "swift_score_skipsets", "swift_generate",
            "swift_committed_length", "swift_launch_count", "swift_round_times", "swift_round_bytes_stored", "swift_final_skip_mask", "swift_forward_bytes", "swift_read_kv", "swift_time_gemm", "swift_set_gemm_impl", "swift_gemm", "swift_gemm_static",
-           "swift_gemm_static_error")
+           "swift_gemm_static_error", "swift_opt_create", "swift_opt_free", "swift_opt_suggest", "swift_opt_observe")
 
 _lib = None
 
@@ -94,6 +94,12 @@ def load_library(path: Optional[str] = None) -> C.CDLL:
     lib.swift_final_skip_mask.restype = C.c_int32
     lib.swift_round_times.argtypes = [vp, i32, vp, vp, vp, vp, vp]
     lib.swift_round_times.restype = C.c_int32
+    lib.swift_opt_create.argtypes = [i32, i32, i32, C.c_uint64, i32]
+    lib.swift_opt_create.restype = vp
+    lib.swift_opt_free.argtypes = [vp]
+    lib.swift_opt_free.restype = None
+    lib.swift_opt_suggest.argtypes = [vp, vp, vp]
+    lib.swift_opt_observe.argtypes = [vp, vp, C.c_float]
     lib.swift_round_bytes_stored.argtypes = [vp, i32, vp, vp]
     lib.swift_round_bytes_stored.restype = C.c_int32
     lib.swift_forward_bytes.argtypes = [vp, vp, i32, i32, i32]
@@ -128,6 +134,10 @@ class GenParams:
     n_opt_rounds: int = 0
     stop_matchness: float = 0.95
     opt_patience: int = 0                             # optimisation rounds without a replacement before it stops (0 = no rule)
+    n_candidates: int = 0                             # proposals per round when the library makes them itself (candidate_masks None)
+    opt_skip_blocks: int = 0                          # ... sets of this many whole blocks,
+    opt_beta: int = 25                                # ... a Gaussian-process proposal every opt_beta-th one (0 = random search only)
+    opt_seed: int = 0
     skip_mask: Optional[np.ndarray] = None            # uint8 [2*n_blocks]
     candidate_masks: Optional[np.ndarray] = None      # uint8 [n_opt_rounds, C, 2*n_blocks]
 
@@ -153,6 +163,37 @@ class GenStats:
 
 
 STATIC_SCRATCH_BYTES = 8 * 1024 * 1024
+
+
+class LayerSetOptimizer:
+    """The library's proposal engine for the on-the-fly optimisation (Section 4.1), usable on its own: host code
+    only, no device needed.  suggest() -> (mask uint8[2*n_blocks], came from the Gaussian-process step); observe(mask, score)."""
+
+    def __init__(self, n_blocks: int, n_skip_blocks: int, beta: int = 25, seed: int = 0, pool: int = 512):
+        self._lib = load_library()
+        self.n_sub = 2 * n_blocks
+        self._h = self._lib.swift_opt_create(n_blocks, n_skip_blocks, beta, seed, pool)
+        if not self._h:
+            raise ValueError("swift_opt_create rejected the arguments")
+
+    def suggest(self) -> Tuple[np.ndarray, bool]:
+        m = np.zeros(self.n_sub, dtype=np.uint8)
+        b = C.c_int32()
+        if self._lib.swift_opt_suggest(self._h, _ptr(m), C.byref(b)) != 0:
+            raise SwiftError("swift_opt_suggest failed")
+        return m, bool(b.value)
+
+    def observe(self, mask, matchness: float) -> None:
+        if self._lib.swift_opt_observe(self._h, _ptr(_u8(mask)), float(matchness)) != 0:
+            raise SwiftError("swift_opt_observe failed")
+
+    def close(self) -> None:
+        if self._h:
+            self._lib.swift_opt_free(self._h)
+            self._h = None
+
+    def __del__(self):
+        self.close()
 
 
 def gemm_static(w: torch.Tensor, x: torch.Tensor, y: torch.Tensor, stream: Optional[torch.cuda.Stream] = None) -> None:
@@ -326,9 +367,11 @@ class SwiftModel:
         p = _i32(prompt)
         skip = None if gp.skip_mask is None else _u8(gp.skip_mask)
         cands = None if gp.candidate_masks is None else _u8(gp.candidate_masks)
-        n_cand = 0 if cands is None else cands.reshape(gp.n_opt_rounds, -1, self.n_sub).shape[1]
+        n_cand = gp.n_candidates if cands is None else cands.reshape(gp.n_opt_rounds, -1, self.n_sub).shape[1]
+        own = cands is None and gp.n_candidates > 0 and gp.opt_skip_blocks > 0      # the library proposes the candidates
         cp = _GenParams(gp.max_new, gp.max_draft, gp.stop_conf, 1 if gp.vanilla else 0, gp.gamma, n_cand,
-                        gp.n_opt_rounds if cands is not None else 0, gp.stop_matchness, gp.opt_patience, _ptr(skip), _ptr(cands))
+                        gp.n_opt_rounds if (cands is not None or own) else 0, gp.stop_matchness, gp.opt_patience,
+                        gp.opt_skip_blocks, gp.opt_beta, gp.opt_seed, _ptr(skip), _ptr(cands))
         out = np.zeros(gp.max_new, dtype=np.int32)
         trace = np.zeros((gp.max_new, 4), dtype=np.int32)
         n_out = C.c_int32()

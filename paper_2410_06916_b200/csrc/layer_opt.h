@@ -1,0 +1,222 @@
+// Host-side proposal engine for the on-the-fly layer-set optimisation (Section 4.1, "Efficient Layer Set
+// Suggestion"): random search over the sets of m of n_blocks blocks, with a Gaussian-process (Bayesian
+// optimisation) proposal every beta-th step.  Plain C++, no device code.
+//
+// The paper leaves the Bayesian step to a third-party package; this is the textbook form.  A set is its indicator
+// vector, the squared distance of two sets their Hamming distance.  Scores are standardised; the prior is a
+// zero-mean GP with Matern-5/2 covariance k(d) = (1 + s + s^2/3) exp(-s), s = sqrt(5) d / ell, plus observation
+// noise; ell is the candidate length scale with the highest marginal likelihood; the posterior comes from a
+// Cholesky factorisation; the proposal is the unevaluated set with the highest mean + kappa * deviation among a
+// pool of random sets and all sets one swap away from the best set seen.  Random draws are Philox4x32-10 words.
+#pragma once
+#include <algorithm>
+#include <cmath>
+#include <cstdint>
+#include <set>
+#include <vector>
+
+namespace swopt {
+
+inline void philox_round(uint32_t (&c)[4], uint32_t (&k)[2])
+{
+    const uint64_t p0 = (uint64_t)0xD2511F53u * c[0], p1 = (uint64_t)0xCD9E8D57u * c[2];
+    const uint32_t n0 = (uint32_t)(p1 >> 32) ^ c[1] ^ k[0], n1 = (uint32_t)p1, n2 = (uint32_t)(p0 >> 32) ^ c[3] ^ k[1], n3 = (uint32_t)p0;
+    c[0] = n0; c[1] = n1; c[2] = n2; c[3] = n3;
+    k[0] += 0x9E3779B9u; k[1] += 0xBB67AE85u;
+}
+// first output word of Philox4x32-10 at counter (index lo, index hi, 7, tag), key = seed
+inline uint32_t philox_word(uint64_t seed, uint64_t index)
+{
+    uint32_t c[4] = {(uint32_t)index, (uint32_t)(index >> 32), 7u, 0x4F5054u};
+    uint32_t k[2] = {(uint32_t)seed, (uint32_t)(seed >> 32)};
+    for (int r = 0; r < 10; ++r) philox_round(c, k);
+    return c[0];
+}
+
+typedef std::vector<int> BlockSet;   // sorted block indices
+
+struct GpModel {
+    std::vector<BlockSet> X;
+    std::vector<double> L, alpha;    // Cholesky factor (row-major lower triangle, n x n) and K^-1 t
+    double mu = 0.0, sd = 1.0, ell = 1.0, lml = 0.0;
+    int n = 0;
+};
+
+class LayerOpt {
+public:
+    LayerOpt(int n_blocks, int m, int beta, uint64_t seed, int pool = 512, double kappa = 2.576, double noise = 1e-2)
+        : nb(n_blocks), m(m), beta(beta), pool(pool), seed(seed), kappa(kappa), noise(noise) {}
+
+    int nb, m, beta, pool;
+    uint64_t seed;
+    double kappa, noise;
+    std::vector<double> ells = {1.0, 2.0, 4.0};
+    long long step = 0;              // proposals made
+    uint64_t draws = 0;              // random words consumed
+    std::vector<BlockSet> X;         // evaluated sets ...
+    std::vector<double> y;           // ... and their matchness
+
+    BlockSet random_set()
+    {
+        std::vector<int> idx(nb);
+        for (int i = 0; i < nb; ++i) idx[i] = i;
+        for (int i = 0; i < m; ++i) {               // partial Fisher-Yates shuffle
+            const int j = i + (int)(philox_word(seed, draws++) % (uint32_t)(nb - i));
+            std::swap(idx[i], idx[j]);
+        }
+        BlockSet s(idx.begin(), idx.begin() + m);
+        std::sort(s.begin(), s.end());
+        return s;
+    }
+
+    static int hamming(const BlockSet& a, const BlockSet& b)   // of the indicator vectors
+    {
+        size_t i = 0, j = 0;
+        int common = 0;
+        while (i < a.size() && j < b.size()) {
+            if (a[i] == b[j]) { ++common; ++i; ++j; }
+            else if (a[i] < b[j]) ++i;
+            else ++j;
+        }
+        return (int)a.size() + (int)b.size() - 2 * common;
+    }
+    static double matern52(double d2, double ell)
+    {
+        const double s = std::sqrt(5.0 * d2) / ell;
+        return (1.0 + s + s * s / 3.0) * std::exp(-s);
+    }
+
+    int best_index() const                           // highest matchness, the earliest among equals
+    {
+        int b = -1;
+        for (size_t i = 0; i < y.size(); ++i)
+            if (b < 0 || y[i] > y[b]) b = (int)i;
+        return b;
+    }
+
+    void observe(const BlockSet& s, double matchness)
+    {
+        BlockSet t(s);
+        std::sort(t.begin(), t.end());
+        X.push_back(t);
+        y.push_back(matchness);
+    }
+
+    GpModel fit() const;
+    void predict(const GpModel& g, const BlockSet& s, double* mean, double* dev) const;
+    BlockSet bayesian_set(double* ucb_out = nullptr);
+    BlockSet suggest()
+    {
+        ++step;
+        if (beta > 0 && step % beta == 0 && !X.empty()) return bayesian_set();
+        return random_set();
+    }
+};
+
+inline GpModel LayerOpt::fit() const
+{
+    const int n = (int)y.size();
+    GpModel best;
+    double mu = 0.0, var = 0.0;
+    for (double v : y) mu += v;
+    mu /= n;
+    for (double v : y) var += (v - mu) * (v - mu);
+    double sd = std::sqrt(var / n);
+    if (sd <= 1e-12) sd = 1.0;
+    std::vector<double> t(n), d2((size_t)n * n);
+    for (int i = 0; i < n; ++i) t[i] = (y[i] - mu) / sd;
+    for (int i = 0; i < n; ++i)
+        for (int j = 0; j <= i; ++j) d2[(size_t)i * n + j] = hamming(X[i], X[j]);
+    bool have = false;
+    for (double ell : ells) {
+        std::vector<double> Lc((size_t)n * n, 0.0);
+        bool ok = true;
+        for (int i = 0; i < n && ok; ++i) {           // Cholesky, row by row
+            for (int j = 0; j <= i; ++j) {
+                double acc = matern52(d2[(size_t)i * n + j], ell) + (i == j ? noise : 0.0);
+                for (int k = 0; k < j; ++k) acc -= Lc[(size_t)i * n + k] * Lc[(size_t)j * n + k];
+                if (i == j) {
+                    if (acc <= 0.0) { ok = false; break; }
+                    Lc[(size_t)i * n + i] = std::sqrt(acc);
+                } else {
+                    Lc[(size_t)i * n + j] = acc / Lc[(size_t)j * n + j];
+                }
+            }
+        }
+        if (!ok) continue;
+        std::vector<double> a(t);                     // alpha = K^-1 t by two triangular solves
+        for (int i = 0; i < n; ++i) {
+            for (int k = 0; k < i; ++k) a[i] -= Lc[(size_t)i * n + k] * a[k];
+            a[i] /= Lc[(size_t)i * n + i];
+        }
+        for (int i = n - 1; i >= 0; --i) {
+            for (int k = i + 1; k < n; ++k) a[i] -= Lc[(size_t)k * n + i] * a[k];
+            a[i] /= Lc[(size_t)i * n + i];
+        }
+        double lml = -0.5 * n * std::log(2.0 * 3.14159265358979323846);
+        for (int i = 0; i < n; ++i) lml -= 0.5 * t[i] * a[i] + std::log(Lc[(size_t)i * n + i]);
+        if (!have || lml > best.lml) {
+            have = true;
+            best.L.swap(Lc); best.alpha.swap(a); best.ell = ell; best.lml = lml;
+        }
+    }
+    best.X = X; best.mu = mu; best.sd = sd; best.n = have ? n : 0;
+    return best;
+}
+
+inline void LayerOpt::predict(const GpModel& g, const BlockSet& s, double* mean, double* dev) const
+{
+    const int n = g.n;
+    std::vector<double> ks(n), v(n);
+    double mu = 0.0;
+    for (int i = 0; i < n; ++i) { ks[i] = matern52(hamming(s, g.X[i]), g.ell); mu += ks[i] * g.alpha[i]; }
+    double q = 0.0;                                   // |L^-1 ks|^2
+    for (int i = 0; i < n; ++i) {
+        double acc = ks[i];
+        for (int k = 0; k < i; ++k) acc -= g.L[(size_t)i * n + k] * v[k];
+        v[i] = acc / g.L[(size_t)i * n + i];
+        q += v[i] * v[i];
+    }
+    *mean = g.mu + g.sd * mu;
+    *dev = g.sd * std::sqrt(std::max(1.0 - q, 0.0));
+}
+
+inline BlockSet LayerOpt::bayesian_set(double* ucb_out)
+{
+    std::vector<BlockSet> cand;
+    for (int i = 0; i < pool; ++i) cand.push_back(random_set());
+    const int bi = best_index();
+    if (bi >= 0) {
+        const BlockSet inc = X[bi];
+        std::vector<int> outside;
+        for (int b = 0; b < nb; ++b) if (!std::binary_search(inc.begin(), inc.end(), b)) outside.push_back(b);
+        for (int out_b : inc)
+            for (int in_b : outside) {
+                BlockSet s;
+                for (int b : inc) if (b != out_b) s.push_back(b);
+                s.push_back(in_b);
+                std::sort(s.begin(), s.end());
+                cand.push_back(s);
+            }
+    }
+    std::set<BlockSet> seen(X.begin(), X.end());      // leave out evaluated sets and repeats, keeping pool order
+    std::vector<BlockSet> fresh;
+    for (const BlockSet& c : cand)
+        if (seen.insert(c).second) fresh.push_back(c);
+    if (fresh.empty()) return random_set();
+    if (X.empty()) return fresh[0];
+    const GpModel g = fit();
+    if (g.n == 0) return fresh[0];
+    int pick = 0;
+    double best = 0.0;
+    for (size_t i = 0; i < fresh.size(); ++i) {
+        double mean, dev;
+        predict(g, fresh[i], &mean, &dev);
+        const double u = mean + kappa * dev;
+        if (i == 0 || u > best) { best = u; pick = (int)i; }
+    }
+    if (ucb_out) *ucb_out = best;
+    return fresh[pick];
+}
+
+} // namespace swopt

@@ -14,6 +14,7 @@
 #include <vector>
 
 #include "common.cuh"
+#include "layer_opt.h"
 #include "kernels_attn.cuh"
 #include "kernels_attn_mma.cuh"
 #include "kernels_elem.cuh"
@@ -1390,6 +1391,48 @@ double swift_forward_bytes(const swift_ctx* ctx, const uint8_t* skip, int32_t n_
 
 } // extern "C"
 
+// =============================================================================== proposal engine (host only)
+struct swift_opt { swopt::LayerOpt impl; swift_opt(int nb, int m, int beta, uint64_t seed, int pool) : impl(nb, m, beta, seed, pool) {} };
+
+namespace {
+void blocks_to_mask(const swopt::BlockSet& s, int n_blocks, uint8_t* mask)
+{
+    memset(mask, 0, 2 * (size_t)n_blocks);
+    for (int b : s) mask[2 * b] = mask[2 * b + 1] = 1;
+}
+swopt::BlockSet mask_to_blocks(const uint8_t* mask, int n_blocks)
+{
+    swopt::BlockSet s;
+    for (int b = 0; b < n_blocks; ++b) if (mask[2 * b] && mask[2 * b + 1]) s.push_back(b);
+    return s;
+}
+} // namespace
+
+extern "C" {
+
+swift_opt* swift_opt_create(int32_t n_blocks, int32_t n_skip_blocks, int32_t beta, uint64_t seed, int32_t pool)
+{
+    if (n_blocks < 2 || n_skip_blocks < 1 || n_skip_blocks >= n_blocks || beta < 0 || pool < 1) return nullptr;
+    return new swift_opt(n_blocks, n_skip_blocks, beta, seed, pool);
+}
+void swift_opt_free(swift_opt* opt) { delete opt; }
+swift_status swift_opt_suggest(swift_opt* opt, uint8_t* mask_host, int32_t* is_bayesian_host)
+{
+    if (!opt || !mask_host) return SWIFT_EINVAL;
+    const bool bayes = opt->impl.beta > 0 && (opt->impl.step + 1) % opt->impl.beta == 0 && !opt->impl.X.empty();
+    blocks_to_mask(opt->impl.suggest(), opt->impl.nb, mask_host);
+    if (is_bayesian_host) *is_bayesian_host = bayes ? 1 : 0;
+    return SWIFT_OK;
+}
+swift_status swift_opt_observe(swift_opt* opt, const uint8_t* mask_host, float matchness)
+{
+    if (!opt || !mask_host) return SWIFT_EINVAL;
+    opt->impl.observe(mask_to_blocks(mask_host, opt->impl.nb), (double)matchness);
+    return SWIFT_OK;
+}
+
+} // extern "C"
+
 // =============================================================================== inspection, generate
 extern "C" {
 
@@ -1486,7 +1529,9 @@ swift_status swift_generate(swift_ctx* ctx, const swift_gen_params* gp, const in
         if (!gp->skip_mask) return fail(ctx, SWIFT_EINVAL, "skip_mask is null");
         if (gp->max_draft < 0 || gp->max_draft > d.max_draft) return fail(ctx, SWIFT_ECAPACITY, "max_draft %d outside 0..%d", gp->max_draft, d.max_draft);
         if (gp->n_opt_rounds > 0) {
-            if (!gp->candidate_masks || gp->n_candidates < 1 || gp->n_candidates > 1023) return fail(ctx, SWIFT_EINVAL, "candidate masks missing");
+            if (gp->n_candidates < 1 || gp->n_candidates > 1023) return fail(ctx, SWIFT_EINVAL, "n_candidates must be in 1..1023");
+            if (!gp->candidate_masks && (gp->opt_skip_blocks < 1 || gp->opt_skip_blocks >= d.n_blocks || gp->opt_beta < 0))
+                return fail(ctx, SWIFT_EINVAL, "without candidate masks, opt_skip_blocks must be in 1..n_blocks-1 and opt_beta >= 0");
             if (gp->gamma < 1 || gp->gamma > MAX_SCORE_ROWS) return fail(ctx, SWIFT_ECAPACITY, "gamma must be in 1..%d", MAX_SCORE_ROWS);
         }
     }
@@ -1511,6 +1556,9 @@ swift_status swift_generate(swift_ctx* ctx, const swift_gen_params* gp, const in
     std::vector<int> counts;
     std::vector<uint8_t> round_masks;
     int stale_rounds = 0;
+    // proposals come from the caller, or from the library's own engine (random search + Gaussian-process step)
+    swopt::LayerOpt engine(d.n_blocks, std::max(1, std::min(d.n_blocks - 1, gp->opt_skip_blocks)), gp->opt_beta, gp->opt_seed);
+    const bool own_proposals = !gp->vanilla && gp->n_opt_rounds > 0 && !gp->candidate_masks;
     DevState hs;
     while (count < gp->max_new) {
         const int remaining = gp->max_new - count;
@@ -1545,7 +1593,10 @@ swift_status swift_generate(swift_ctx* ctx, const swift_gen_params* gp, const in
                 const int n_scored = gp->n_candidates + 1;
                 round_masks.resize((size_t)n_scored * L);
                 memcpy(round_masks.data(), z.data(), L);
-                memcpy(round_masks.data() + L, gp->candidate_masks + (size_t)stt.opt_rounds * gp->n_candidates * L, (size_t)gp->n_candidates * L);
+                if (own_proposals)
+                    for (int c = 0; c < gp->n_candidates; ++c) blocks_to_mask(engine.suggest(), d.n_blocks, round_masks.data() + (size_t)(c + 1) * L);
+                else
+                    memcpy(round_masks.data() + L, gp->candidate_masks + (size_t)stt.opt_rounds * gp->n_candidates * L, (size_t)gp->n_candidates * L);
                 const uint8_t* masks = round_masks.data();
                 ST(enqueue_score(ctx, masks, n_scored, gp->gamma));
                 counts.resize(n_scored);
@@ -1555,6 +1606,9 @@ swift_status swift_generate(swift_ctx* ctx, const swift_gen_params* gp, const in
                 float ms = 0.f;
                 CU(cudaEventElapsedTime(&ms, ev[2], ev[3]));
                 stt.ms_score += ms;
+                if (own_proposals)                  // every score of the round goes into the Gaussian-process model
+                    for (int c = 0; c < n_scored; ++c)
+                        engine.observe(mask_to_blocks(masks + (size_t)c * L, d.n_blocks), (double)counts[c] / (double)gp->gamma);
                 int cb = 0;
                 for (int c = 1; c < n_scored; ++c) if (counts[c] > counts[cb]) cb = c;   // strictly better only: the set in use wins ties
                 stt.best_matchness = (float)counts[cb] / (float)gp->gamma;

@@ -65,3 +65,38 @@ def test_product_path_has_no_oracle_or_cpu_fallback():
         import synth
         with pytest.raises(RuntimeError, match="needs a CUDA device"):
             SwiftModel(synth.MODELS["tiny"], 64)
+
+
+def test_proposal_engine_follows_the_oracles():
+    """The library's layer-set proposal engine (host code, Section 4.1) against the oracle's, fed the same scores:
+    random-search proposals are identical (same counter-based draws); a Gaussian-process proposal may differ from the
+    oracle's only where the oracle's own acquisition values tie to rounding."""
+    import numpy as np
+    from oracle import swift_oracle as so
+    from paper_2410_06916_b200 import LayerSetOptimizer
+    nb, m, beta = 24, 9, 5
+    planted = set(range(0, 18, 2))
+    score = lambda blocks: round((1.0 - len(set(blocks) - planted) / m) * 32) / 32
+    ref = so.LayerSetOptimizer(nb, m, beta=beta, seed=11, pool=64)
+    lib = LayerSetOptimizer(nb, m, beta=beta, seed=11, pool=64)
+    n_bayes = 0
+    for step in range(1, 41):
+        draws_before = ref.draws
+        expect_bayes = step % beta == 0
+        mask, bayes = lib.suggest()
+        got = tuple(int(b) for b in range(nb) if mask[2 * b])
+        assert bayes == expect_bayes and len(got) == m and all(mask[2 * b] == mask[2 * b + 1] for b in range(nb))
+        if expect_bayes:
+            ref.step += 1
+            want, info = ref.bayesian_set()
+            if got != want:
+                i = info["candidates"].index(got)
+                assert abs(float(info["ucb_all"][i]) - info["ucb"]) < 1e-9, (step, got, want)
+            n_bayes += 1
+        else:
+            assert got == ref.suggest(), step
+        assert ref.draws > draws_before
+        ref.observe(got, score(got))
+        lib.observe(mask, score(got))
+    assert n_bayes == 8 and max(ref.y) >= 0.75
+    lib.close()
