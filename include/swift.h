@@ -158,6 +158,31 @@ swift_status swift_verify(swift_ctx* ctx, const int32_t* tokens_host, int32_t k,
                           float* logits_host);
 
 /*
+ * Dynamic verification (Section 4.2): with tree_rows > 0, a verification of the device's own drafts (swift_verify with
+ * tokens_host == NULL, and the rounds of swift_generate) holds up to tree_rows rows instead of the drafted chain alone:
+ * every draft position j is extended with the draft model's top-k predictions at that step, k = 10, 5, 3, 1 for a
+ * confidence p_j in (0, 0.5], (0.5, 0.8], (0.8, 0.95], (0.95, 1].  Rows 0..k are the chain [t*, y'_1..y'_k]; the rest
+ * are the alternatives, handed out from the first draft position on until the rows run out (the paper sets no limit;
+ * one forward of this library holds SWIFT_MAX_ROWS rows).  An alternative of depth j sits at sequence position n + j,
+ * attends to the cache, to chain rows 0..j-1 and to itself, and is stored in the cache slot of its row.  swift_accept
+ * then follows, from t*, the child that equals the target's arg max, and moves an accepted alternative's K,V to the
+ * slot of its depth.  Greedy decoding only (in sampling mode the setting has no effect).  tree_rows: 0 (off, the
+ * default) or 2..SWIFT_MAX_ROWS.  Not allowed inside a round.
+ */
+swift_status swift_set_tree(swift_ctx* ctx, int32_t tree_rows);
+
+/* Verifies a token tree the caller spells out: tokens_host[n_rows] with tokens_host[0] the pending token,
+ * parent_host[n_rows] the row each row hangs off (parent_host[0] = -1, parent_host[i] < i).  Row i is stored in cache
+ * slot n + i.  Outputs as swift_verify, n_rows entries.  swift_accept then walks the tree as described above. */
+swift_status swift_verify_tree(swift_ctx* ctx, const int32_t* tokens_host, const int32_t* parent_host, int32_t n_rows,
+                               int32_t* target_argmax_host, float* logits_host);
+
+/* The rows of the tree the last verification held, as read back by that call (call it before swift_accept): tokens,
+ * parent rows and depths, SWIFT_MAX_ROWS entries each (any may be NULL).  Returns the number of rows, 0 when the last
+ * verification held a plain chain, -1 if ctx is NULL. */
+int32_t swift_tree_rows(const swift_ctx* ctx, int32_t* tokens_host, int32_t* parent_host, int32_t* depth_host);
+
+/*
  * Acceptance + KV rollback.  Greedy: a = longest prefix of drafts equal to the target's argmax,
  * next token = target argmax of row a.  Sampling: accept y'_j while u_j * q_j(y'_j) < p_j(y'_j);
  * on the first rejection the next token is drawn from max(0, p_j - q_j) renormalised, after k

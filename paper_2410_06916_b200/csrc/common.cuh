@@ -9,6 +9,7 @@ namespace swk {
 constexpr int ROWS = 16;          // rows of one forward chunk (pending token + up to 15 drafts)
 constexpr int ATTN_CHUNK = 64;    // KV positions per attention split; anchored at multiples of this
 constexpr int MAX_SCORE_ROWS = 128;
+constexpr int TREE_TOPK = 10;        // most predictions one draft position is extended with (Section 4.2)
 
 // purposes of a random draw inside one decoding round (Philox counter word 2)
 enum { DRAW_DRAFT = 0, DRAW_ACCEPT = 1, DRAW_RESAMPLE = 2, DRAW_BONUS = 3 };
@@ -44,6 +45,12 @@ struct DevState {
     // forward has depth m and bits 0..m (causal order); a verified token tree has a node's depth and its ancestors.
     unsigned row_vis[ROWS];
     int row_depth[ROWS];
+    // Token tree of a verification (dynamic verification, Section 4.2): parent row of every row (-1 for row 0), and
+    // after acceptance the rows of the accepted nodes in order (acc_row[j-1] = row of the accepted node of depth j).
+    int row_parent[ROWS];
+    int acc_row[ROWS];
+    int tree_rows;         // rows of the verified tree; 0 = the verification held the drafted chain only
+    int pad2[3];
 };
 
 // Causal order over the forward's rows: the default shape.
@@ -52,7 +59,9 @@ __device__ __forceinline__ void set_causal_rows(DevState* st)
     for (int m = 0; m < ROWS; ++m) {
         st->row_vis[m] = (2u << m) - 1u;
         st->row_depth[m] = m;
+        st->row_parent[m] = m - 1;
     }
+    st->tree_rows = 0;
 }
 
 // Programmatic dependent launch.  Every kernel of a forward is launched with programmatic stream

@@ -137,7 +137,9 @@ attn_split_kernel(const DevState* st, const float* __restrict__ q, const T* __re
     for (int r = warp; r < n_rows; r += ATTN_THREADS / 32) {
         float m = -INFINITY;
         for (int j = lane; j < len; j += 32) {
-            const float v = (c0 + j <= pos0 + r) ? sc[r * ATTN_CHUNK + j] + sc[(MR + r) * ATTN_CHUNK + j] : -INFINITY;
+            const int pj = c0 + j;                          // cached context, or a row of the forward this row may see
+            const bool vis = pj < pos0 || ((st->row_vis[r] >> (pj - pos0)) & 1u) != 0u;
+            const float v = vis ? sc[r * ATTN_CHUNK + j] + sc[(MR + r) * ATTN_CHUNK + j] : -INFINITY;
             ps[r * ATTN_CHUNK + j] = v;
             m = fmaxf(m, v);
         }
@@ -344,6 +346,8 @@ attn_stream_kernel(const DevState* st, const float* __restrict__ q, const T* __r
     __shared__ float2 part_ml[NW][MR];
     __shared__ __align__(16) float p_sh[NW][MR][ATTN_BATCH];
     __shared__ float corr_sh[NW][MR];
+    __shared__ unsigned vis_sh[ROWS];
+    if (tid < ROWS) vis_sh[tid] = st->row_vis[tid];
 
     for (int i = tid; i < MR * 32; i += ATTN_THREADS) {
         const int r = i >> 5, c = i & 31;
@@ -411,7 +415,10 @@ attn_stream_kernel(const DevState* st, const float* __restrict__ q, const T* __r
         for (int t = 0; t < N3; ++t) {
             const int r = row_base + t;
             float x = sc[t];
-            if (c0 + j0 + pi > pos0 + r) x = -INFINITY;                // causal mask; also covers positions past the end
+            {                                                          // visibility among the forward's rows; also covers positions past the end
+                const int dlt = c0 + j0 + pi - pos0 + row0;            // index among the forward's rows; negative = cached context
+                if (dlt >= 0 && (dlt >= ROWS || ((vis_sh[min(row0 + r, ROWS - 1)] >> dlt) & 1u) == 0u)) x = -INFINITY;
+            }
             float bm = x;
             bm = fmaxf(bm, __shfl_xor_sync(0xffffffffu, bm, 4));
             bm = fmaxf(bm, __shfl_xor_sync(0xffffffffu, bm, 8));

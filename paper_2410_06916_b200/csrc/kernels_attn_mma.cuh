@@ -30,6 +30,13 @@
 namespace swk {
 
 constexpr int AM_THREADS = 128;
+#ifndef SWIFT_AM_V_LATE
+#define SWIFT_AM_V_LATE 1
+#endif
+#ifndef SWIFT_AM_CTAS
+#define SWIFT_AM_CTAS 4
+#endif
+constexpr bool AM_V_LATE = SWIFT_AM_V_LATE != 0;   // V loaded after the scores (fewer live registers, more CTAs per SM)
 constexpr int AM_QSTRIDE = 144;     // bf16 per staged query row (288 bytes): the rows of a fragment load fall into different banks
 constexpr int AM_OSTRIDE = 132;     // floats per row of a warp's partial output
 constexpr int AM_PSTRIDE = 20;      // floats per row of a warp's probabilities (16 positions)
@@ -69,7 +76,7 @@ __device__ __forceinline__ void mma_split(float (&c)[4], const uint32_t (&ah)[4]
 // part_rows = row stride of o_part / ml_part: o_part[h][s][part_rows][128] (unnormalised), ml_part[h][s][part_rows].
 // head_counters / out / planes: as in attn_stream_kernel, used for one-row forwards only (merge by the last CTA).
 template <typename T, int NT>
-__global__ void __launch_bounds__(AM_THREADS, 2)
+__global__ void __launch_bounds__(AM_THREADS, SWIFT_AM_CTAS)
 attn_mma_kernel(const DevState* st, const float* __restrict__ q, const T* __restrict__ kv_pool,
                 const int* __restrict__ page_table, KvLayout L, int block, int n_heads, int max_splits, float scale,
                 float* __restrict__ o_part, float2* __restrict__ ml_part, int part_rows, int* __restrict__ head_counters,
@@ -123,11 +130,13 @@ attn_mma_kernel(const DevState* st, const float* __restrict__ q, const T* __rest
             asm volatile("" : "+l"(ka), "+l"(kb));
 #pragma unroll
             for (int j = 0; j < 8; ++j) { kA[j] = load_row4<T>(ka + 16 * j); kB[j] = load_row4<T>(kb + 16 * j); }
+            if (!AM_V_LATE) {
 #pragma unroll
-            for (int u = 0; u < 4; ++u) {
-                asm volatile("" : "+l"(vp[u]));
+                for (int u = 0; u < 4; ++u) {
+                    asm volatile("" : "+l"(vp[u]));
 #pragma unroll
-                for (int i = 0; i < 4; ++i) vv[u][i] = load_row4<T>(vp[u] + 32 * i);
+                    for (int i = 0; i < 4; ++i) vv[u][i] = load_row4<T>(vp[u] + 32 * i);
+                }
             }
         }
         __syncthreads();                                    // the previous pass's merge has read part_acc; vis_sh is set
@@ -166,6 +175,14 @@ attn_mma_kernel(const DevState* st, const float* __restrict__ q, const T* __rest
                 }
             }
 
+            if (AM_V_LATE) {                                // V is requested once K's registers are free: the soft-max covers part of the wait
+#pragma unroll
+                for (int u = 0; u < 4; ++u) {
+                    asm volatile("" : "+l"(vp[u]));
+#pragma unroll
+                    for (int i = 0; i < 4; ++i) vv[u][i] = load_row4<T>(vp[u] + 32 * i);
+                }
+            }
             // ---- soft-max over this warp's 16 positions, per query row (the 8 lanes that share t hold one row's scores)
             float* pw = p_sh + w * QR * AM_PSTRIDE;
 #pragma unroll

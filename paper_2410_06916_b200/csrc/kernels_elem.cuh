@@ -50,9 +50,76 @@ __global__ void begin_draft_step_kernel(DevState* st, int n, int j)
 __global__ void begin_verify_kernel(DevState* st, int n, int forced_k)
 {
     if (forced_k >= 0) st->n_drafted = forced_k;
+    set_causal_rows(st);
     st->pos0 = n;
     st->n_rows = st->n_drafted + 1;
     st->tok_off = 0;
+}
+
+// How many of the draft model's top predictions stand in for a draft token of confidence p (Section 4.2):
+// 10, 5, 3, 1 for p in (0, 0.5], (0.5, 0.8], (0.8, 0.95], (0.95, 1].
+__host__ __device__ inline int tree_width(float p) { return p <= 0.5f ? 10 : p <= 0.8f ? 5 : p <= 0.95f ? 3 : 1; }
+
+// Verification of a token tree built on the device: rows 0..k are the chain [t*, y'_1..y'_k] as in a plain
+// verification; the remaining rows (up to `budget` in all) hold, draft position by draft position from the first on,
+// the next-best predictions the draft model made there (cand[(j-1)*TREE_TOPK + i], i >= 1; cand_n[j-1] of them count,
+// the chain token included).  An alternative of depth j hangs off chain row j-1: it sees rows 0..j-1 and itself.
+__global__ void begin_verify_tree_kernel(DevState* st, int n, const int* __restrict__ cand, const int* __restrict__ cand_n, int budget)
+{
+    const int k = st->n_drafted;
+    set_causal_rows(st);
+    int used = k + 1;
+    for (int j = 1; j <= k; ++j) {
+        int extra = min(cand_n[j - 1] - 1, budget - used);
+        for (int i = 1; i <= extra; ++i) {
+            st->draft_tok[used] = cand[(j - 1) * TREE_TOPK + i];
+            st->row_depth[used] = j;
+            st->row_parent[used] = j - 1;
+            st->row_vis[used] = ((1u << j) - 1u) | (1u << used);
+            ++used;
+        }
+    }
+    st->pos0 = n;
+    st->n_rows = used;
+    st->tok_off = 0;
+    st->tree_rows = used;
+}
+
+// Verification of a tree the caller spelled out: tokens in st->draft_tok[0..rows), parents in st->row_parent (copied
+// there beforehand, parent[i] < i, parent[0] = -1): fills depths and visibility.
+__global__ void begin_verify_given_tree_kernel(DevState* st, int n, int rows)
+{
+    st->row_depth[0] = 0;
+    st->row_vis[0] = 1u;
+    for (int m = 1; m < rows; ++m) {
+        const int p = st->row_parent[m];
+        st->row_depth[m] = st->row_depth[p] + 1;
+        st->row_vis[m] = st->row_vis[p] | (1u << m);
+    }
+    st->pos0 = n;
+    st->n_rows = rows;
+    st->tok_off = 0;
+    st->tree_rows = rows;
+    st->n_drafted = rows - 1;
+}
+
+// After a tree was accepted: the accepted node of depth j belongs in cache slot pos0 + j; one that was verified in
+// another slot (an alternative) is moved there, K and V of every block.  grid = (n_blocks, 2), any block size.
+template <typename T>
+__global__ void kv_move_accepted_kernel(const DevState* st, T* __restrict__ kv_pool, const int* __restrict__ page_table, KvLayout L, int pos0)
+{
+    if (st->tree_rows == 0) return;
+    const int block = blockIdx.x, kv = blockIdx.y, per = L.n_kv_heads * L.head_dim;
+    for (int j = 1; j <= st->n_accepted; ++j) {                  // ascending depth: a slot is never needed after it was overwritten
+        const int src = pos0 + st->acc_row[j - 1], dst = pos0 + j;
+        if (src == dst) continue;
+        const int ps = page_table[src >> L.page_shift], pd = page_table[dst >> L.page_shift];
+        for (int i = threadIdx.x; i < per; i += blockDim.x) {
+            const int h = i / L.head_dim, d = i - h * L.head_dim;
+            kv_pool[L.offset(pd, block, kv, h, dst & (L.page_size - 1)) + d] = kv_pool[L.offset(ps, block, kv, h, src & (L.page_size - 1)) + d];
+        }
+        __syncthreads();
+    }
 }
 
 // Precomputed rotary table: cs[pos][i] = (cos, sin)(pos * theta^(-2i/dh)), evaluated in double.
@@ -180,7 +247,8 @@ __global__ void qkv_post_kernel(const DevState* st, const float* __restrict__ pa
     const int r = blockIdx.x;
     if (r >= st->n_rows) return;
     const int head = blockIdx.y, half = L.head_dim >> 1, i = threadIdx.x;
-    const int pos = st->pos0 + r;
+    const int pos = st->pos0 + r;                       // cache slot of the row; its sequence position follows its depth
+    const int rpos = st->pos0 + st->row_depth[r];
     if (pos >= max_positions) return;
     const size_t col = (size_t)head * L.head_dim + i;
     float a = 0.f, b = 0.f;
@@ -189,7 +257,7 @@ __global__ void qkv_post_kernel(const DevState* st, const float* __restrict__ pa
         a += p[0];
         b += p[half];
     }
-    const float2 cs = rope_cs[(size_t)pos * half + i];
+    const float2 cs = rope_cs[(size_t)rpos * half + i];
     if (head < n_heads) {
         float* q = q_out + (size_t)r * n_heads * L.head_dim + col;
         q[0] = a * cs.x - b * cs.y;

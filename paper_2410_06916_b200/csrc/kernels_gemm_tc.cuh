@@ -451,7 +451,8 @@ gemm_tc_kernel(DevState* st, const __grid_constant__ CUtensorMap mapW, const __g
             const int half = ep.L.head_dim >> 1, pos0 = pos0_epi;
             for (int idx = etid; idx < ROWS * half; idx += 128) {
                 const int m = idx / half, j = idx - m * half, pos = pos0 + m;
-                if (m < n_rows && pos < ep.max_positions) rope_sh[m * (TC_TILE_N / 2) + j] = ep.rope_cs[(size_t)pos * half + j];
+                // the row is stored in cache slot pos; its rotary position follows its depth (they differ in a token tree)
+                if (m < n_rows && pos < ep.max_positions) rope_sh[m * (TC_TILE_N / 2) + j] = ep.rope_cs[(size_t)(pos0 + st->row_depth[m]) * half + j];
             }
             if (etid < ROWS) {
                 const int pos = pos0 + etid;

@@ -88,7 +88,7 @@ __device__ int block_categorical(WeightFn w, int n, float u, float* sh)
 __global__ void __launch_bounds__(VOCAB_THREADS)
 vocab_kernel(DevState* st, const float* __restrict__ part, int n_split, size_t split_stride,
              float* __restrict__ logits, int vocab, float inv_temp, int mode, int sampling, float* __restrict__ q_rows,
-             float top_p, int w_cached)
+             float top_p, int w_cached, int* __restrict__ cand, int* __restrict__ cand_n)
 {
     pdl_enter();
     __shared__ float sh[VOCAB_THREADS + 72];
@@ -236,6 +236,42 @@ vocab_kernel(DevState* st, const float* __restrict__ part, int n_split, size_t s
         st->n_drafted = draft_j;
         if (conf < stop_conf) st->active = 0;
     }
+    // Dynamic verification (Section 4.2): the draft position is extended with the draft model's top-k predictions,
+    // k by the confidence of the position.  cand[(j-1)*TREE_TOPK + i] = the i-th best token (logit descending, token
+    // id ascending among equals; entry 0 is y'_j itself), found by k - 1 further arg-max passes over the row, each
+    // restricted to what ranks after the previous pick.
+    if (cand != nullptr && !sampling) {
+        const int width = conf <= 0.5f ? 10 : conf <= 0.8f ? 5 : conf <= 0.95f ? 3 : 1;
+        if (tid == 0) { cand[(draft_j - 1) * TREE_TOPK] = am.i; cand_n[draft_j - 1] = width; }
+        ArgMax prev = am;
+        for (int rank = 1; rank < width; ++rank) {
+            ArgMax best{-INFINITY, 0x7FFFFFFF};
+            for (int i = tid; i < vocab; i += VOCAB_THREADS) {
+                const float v = lrow[i];
+                if (v < prev.v || (v == prev.v && i > prev.i)) best = better(best, ArgMax{v, i});
+            }
+#pragma unroll
+            for (int o = 16; o > 0; o >>= 1) {
+                ArgMax t2{__shfl_xor_sync(0xFFFFFFFFu, best.v, o), __shfl_xor_sync(0xFFFFFFFFu, best.i, o)};
+                best = better(best, t2);
+            }
+            __syncthreads();
+            if (lane == 0) sh_am[warp] = best;
+            __syncthreads();
+            if (warp == 0) {
+                ArgMax t3 = sh_am[lane];
+#pragma unroll
+                for (int o = 16; o > 0; o >>= 1) {
+                    ArgMax t4{__shfl_xor_sync(0xFFFFFFFFu, t3.v, o), __shfl_xor_sync(0xFFFFFFFFu, t3.i, o)};
+                    t3 = better(t3, t4);
+                }
+                if (lane == 0) sh_am[0] = t3;
+            }
+            __syncthreads();
+            prev = sh_am[0];
+            if (tid == 0) cand[(draft_j - 1) * TREE_TOPK + rank] = prev.i;
+        }
+    }
 }
 
 // Acceptance over the k = st->n_drafted drafts of the round, one CTA.  `logits` holds the k+1
@@ -249,6 +285,28 @@ accept_kernel(DevState* st, const float* __restrict__ logits, const float* __res
     __shared__ int sh_a, sh_rejected;
     const int k = st->n_drafted;
     const int tid = threadIdx.x;
+    if (!sampling && st->tree_rows > 0) {
+        // greedy verification of a token tree: from row 0 follow the child whose token is the target's arg max at the
+        // current node; where no child matches, that arg max is the next token
+        if (tid == 0) {
+            const int rows = st->tree_rows;
+            int node = 0, a = 0, gold = st->argmax[0];
+            for (;;) {
+                gold = st->argmax[node];
+                int hit = -1;
+                for (int r = 1; r < rows; ++r)
+                    if (st->row_parent[r] == node && st->draft_tok[r] == gold) { hit = r; break; }
+                if (hit < 0) break;
+                st->acc_row[a++] = hit;
+                node = hit;
+            }
+            for (int j = 1; j <= a; ++j) st->draft_tok[j] = st->draft_tok[st->acc_row[j - 1]];   // acc_row[j-1] >= j: read before overwritten
+            st->n_accepted = a;
+            st->next_token = gold;
+            st->draft_tok[0] = gold;
+        }
+        return;
+    }
     if (!sampling) {
         if (tid == 0) {
             int a = 0;

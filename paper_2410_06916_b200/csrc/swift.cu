@@ -48,7 +48,7 @@ struct WeightLayout {
 };
 
 struct WorkLayout {
-    size_t state, h, xn, xa, act, q, part, o_part, ml_part, logits, q_rows, rope, pt_main, pt_score, score_tok,
+    size_t state, h, xn, xa, act, q, part, o_part, ml_part, logits, q_rows, rope, pt_main, pt_score, score_tok, cand, cand_n,
         score_truth, score_out, attn_counters, xn_hl, xa_hl, act_hl, slabs, counters, sumsq, total;
     size_t part_floats, slab_floats;
 };
@@ -72,6 +72,8 @@ struct swift_ctx {
     bool round_open;
     std::vector<int> hist;           // prompt + generated tokens, pending included
     int mode; float temperature, top_p; uint64_t seed; bool greedy_draft;
+    int tree_rows;                   // dynamic verification: rows one verification may hold (0 = off)
+    DevState last_state;             // control block as last read back
     int64_t launches, h2d_bytes, d2h_bytes;
     std::string err;
     cudaEvent_t ev[8];
@@ -235,6 +237,8 @@ WorkLayout work_layout(const swift_model_desc* d)
     k.score_tok = c.take(MAX_SCORE_ROWS * 4);
     k.score_truth = c.take(MAX_SCORE_ROWS * 4);
     k.score_out = c.take(1024 * 4);
+    k.cand = c.take((size_t)ROWS * TREE_TOPK * 4);
+    k.cand_n = c.take(ROWS * 4);
     k.attn_counters = c.take((size_t)d->n_heads * 4);
     // tensor-core path (bf16 models): hi/lo bf16 planes of the GEMM inputs, stream-K slabs, tile counters
     k.slab_floats = 0;
@@ -448,6 +452,12 @@ struct HeadOpts {
     int mode = VOCAB_PLAIN;
 };
 
+// Where a draft step leaves its top predictions when dynamic verification is on (greedy decoding only), else null.
+int* tree_cand(swift_ctx* ctx, const HeadOpts& head)
+{
+    return (head.mode == VOCAB_DRAFT && ctx->tree_rows > 0 && ctx->mode == SWIFT_GREEDY) ? kptr<int>(ctx, ctx->kl.cand) : nullptr;
+}
+
 
 // Enqueues the kernels of one forward chunk of at most `rows` (<= 16) rows.  The device state
 // (pos0, n_rows, tok_off) must have been set by a preceding kernel on the same stream.
@@ -503,7 +513,8 @@ swift_status forward_chunk(swift_ctx* ctx, int rows, const int* toks_dev, const 
         ST(run_gemm<T>(ctx, mr, GemmSite{xn, d.vocab, dm, wptr<T>(ctx, ctx->wl.lm_head), &ctx->tm_lm_head, &ctx->tm_xn}, &S));
         CU(launch_k(vocab_kernel, dim3(rows), dim3(VOCAB_THREADS), vocab_cache_bytes(ctx), ctx, st, (const float*)part, S, (size_t)ROWS * d.vocab,
                     kptr<float>(ctx, ctx->kl.logits), d.vocab, 1.0f / ctx->temperature, head.mode,
-                    sampling_flag(ctx), kptr<float>(ctx, ctx->kl.q_rows), ctx->top_p, vocab_cache_bytes(ctx) != 0 ? 1 : 0));
+                    sampling_flag(ctx), kptr<float>(ctx, ctx->kl.q_rows), ctx->top_p, vocab_cache_bytes(ctx) != 0 ? 1 : 0,
+                    tree_cand(ctx, head), kptr<int>(ctx, ctx->kl.cand_n)));
     }
     CU(cudaGetLastError());
     return SWIFT_OK;
@@ -607,7 +618,8 @@ swift_status forward_chunk_fused(swift_ctx* ctx, int rows, const int* toks_dev, 
         ST(gemm(EPI_PLAIN, &ctx->tm_lm_head, &ctx->tm_xn, d.vocab, dm, ep));
         CU(launch_k(vocab_kernel, dim3(rows), dim3(VOCAB_THREADS), vocab_cache_bytes(ctx), ctx, st, (const float*)kptr<float>(ctx, ctx->kl.part), 1,
                     (size_t)ROWS * d.vocab, kptr<float>(ctx, ctx->kl.logits), d.vocab, 1.0f / ctx->temperature, head.mode,
-                    sampling_flag(ctx), kptr<float>(ctx, ctx->kl.q_rows), ctx->top_p, vocab_cache_bytes(ctx) != 0 ? 1 : 0));
+                    sampling_flag(ctx), kptr<float>(ctx, ctx->kl.q_rows), ctx->top_p, vocab_cache_bytes(ctx) != 0 ? 1 : 0,
+                    tree_cand(ctx, head), kptr<int>(ctx, ctx->kl.cand_n)));
     }
     CU(cudaGetLastError());
     return SWIFT_OK;
@@ -632,7 +644,7 @@ swift_status forward_chunk_any(swift_ctx* ctx, int rows, const int* toks_dev, co
 // sequence is captured once into a CUDA graph and replayed: one graph launch instead of several
 // hundred kernel launches per forward.
 struct FwdKey {
-    int rows, head_run, head_mode, sampling, use_tc, use_pdl, fuse;
+    int rows, head_run, head_mode, sampling, use_tc, use_pdl, fuse, tree;
     float temperature, top_p;
     const void* toks;
     const void* page_table;
@@ -640,7 +652,7 @@ struct FwdKey {
     bool operator==(const FwdKey& o) const
     {
         return rows == o.rows && head_run == o.head_run && head_mode == o.head_mode && sampling == o.sampling &&
-               use_tc == o.use_tc && use_pdl == o.use_pdl && fuse == o.fuse && temperature == o.temperature && top_p == o.top_p && toks == o.toks && page_table == o.page_table && mask == o.mask;
+               use_tc == o.use_tc && use_pdl == o.use_pdl && fuse == o.fuse && tree == o.tree && temperature == o.temperature && top_p == o.top_p && toks == o.toks && page_table == o.page_table && mask == o.mask;
     }
 };
 struct FwdGraph {
@@ -655,7 +667,7 @@ swift_status forward_cached(swift_ctx* ctx, int rows, const int* toks_dev, const
 {
     if (!ctx->use_graphs) return forward_chunk_any(ctx, rows, toks_dev, skip, page_table, head);
     const int L = 2 * ctx->d.n_blocks;
-    FwdKey key{rows, head.run ? 1 : 0, head.mode, sampling_flag(ctx), ctx->use_tc ? 1 : 0, ctx->use_pdl ? 1 : 0, ctx->fuse ? 1 : 0, ctx->temperature, ctx->top_p, toks_dev, page_table,
+    FwdKey key{rows, head.run ? 1 : 0, head.mode, sampling_flag(ctx), ctx->use_tc ? 1 : 0, ctx->use_pdl ? 1 : 0, ctx->fuse ? 1 : 0, tree_cand(ctx, head) ? 1 : 0, ctx->temperature, ctx->top_p, toks_dev, page_table,
                skip ? std::vector<uint8_t>(skip, skip + L) : std::vector<uint8_t>()};
     auto& cache = *ctx->graphs;
     ctx->graph_clock++;
@@ -714,6 +726,7 @@ swift_status read_state(swift_ctx* ctx, DevState* out)
 {
     CU(copy_async(ctx, out, state_of(ctx), sizeof(DevState), cudaMemcpyDeviceToHost));
     CU(cudaStreamSynchronize(ctx->stream));
+    ctx->last_state = *out;
     if (out->error) {
         const int code = out->error;
         CU(cudaMemsetAsync(&state_of(ctx)->error, 0, sizeof(int), ctx->stream));
@@ -807,10 +820,20 @@ swift_status enqueue_draft(swift_ctx* ctx, const uint8_t* skip, int max_k, float
     return SWIFT_OK;
 }
 
+// Dynamic verification applies to rounds of greedy decoding that verify what the device drafted.
+bool tree_active(const swift_ctx* ctx) { return ctx->tree_rows > 0 && ctx->mode == SWIFT_GREEDY; }
+
 swift_status enqueue_verify(swift_ctx* ctx, int rows_launch, int forced_k)
 {
     DevState* st = state_of(ctx);
-    begin_verify_kernel<<<1, 1, 0, ctx->stream>>>(st, ctx->n, forced_k);
+    if (forced_k < 0 && tree_active(ctx)) {
+        // the chain plus the draft model's next-best predictions, as many rows as the budget holds
+        const int budget = std::max(ctx->tree_rows, rows_launch);
+        begin_verify_tree_kernel<<<1, 1, 0, ctx->stream>>>(st, ctx->n, kptr<int>(ctx, ctx->kl.cand), kptr<int>(ctx, ctx->kl.cand_n), budget);
+        rows_launch = budget;
+    } else {
+        begin_verify_kernel<<<1, 1, 0, ctx->stream>>>(st, ctx->n, forced_k);
+    }
     ctx->launches++;
     HeadOpts head;
     head.run = true;
@@ -824,6 +847,15 @@ swift_status enqueue_accept(swift_ctx* ctx)
                                                         ctx->mode == SWIFT_SAMPLING ? 1 : 0, 1.0f / ctx->temperature,
                                                         ctx->seed, (uint32_t)ctx->round);
     ctx->launches++;
+    if (ctx->tree_rows > 0) {             // an accepted alternative is moved to the cache slot of its depth (no-op for a chain)
+        if (ctx->d.kv_dtype == SWIFT_BF16)
+            kv_move_accepted_kernel<__nv_bfloat16><<<dim3(ctx->d.n_blocks, 2), 256, 0, ctx->stream>>>(
+                state_of(ctx), reinterpret_cast<__nv_bfloat16*>(ctx->kvbase), pt_main(ctx), ctx->kv, ctx->n);
+        else
+            kv_move_accepted_kernel<float><<<dim3(ctx->d.n_blocks, 2), 256, 0, ctx->stream>>>(
+                state_of(ctx), reinterpret_cast<float*>(ctx->kvbase), pt_main(ctx), ctx->kv, ctx->n);
+        ctx->launches++;
+    }
     CU(cudaGetLastError());
     return SWIFT_OK;
 }
@@ -1025,7 +1057,7 @@ swift_status swift_load(const swift_model_desc* desc, swift_devbuf weights, swif
     c->max_splits = ceil_div(desc->max_positions, ATTN_CHUNK);
     c->phase = PH_LOADED; c->n = 0; c->pending = 0; c->n_prompt = 0; c->round = 0; c->last_k = 0; c->last_max_k = 0;
     c->round_open = false;
-    c->mode = SWIFT_GREEDY; c->temperature = 1.f; c->top_p = 1.f; c->greedy_draft = false; c->seed = 0; c->launches = 0; c->h2d_bytes = 0; c->d2h_bytes = 0;
+    c->mode = SWIFT_GREEDY; c->temperature = 1.f; c->top_p = 1.f; c->greedy_draft = false; c->seed = 0; c->tree_rows = 0; memset(&c->last_state, 0, sizeof(DevState)); c->launches = 0; c->h2d_bytes = 0; c->d2h_bytes = 0;
     ctx = c;
     c->use_tc = false;
     if (desc->dtype == SWIFT_BF16) {
@@ -1256,19 +1288,82 @@ swift_status swift_verify(swift_ctx* ctx, const int32_t* tokens_host, int32_t k,
     } else {
         if (ctx->phase != PH_DRAFTED) return fail(ctx, SWIFT_ESTATE, "no draft to verify: call swift_draft or pass tokens");
         rows_launch = ctx->last_k + 1; forced_k = -1;
+        if (tree_active(ctx) && ctx->n + std::max(ctx->tree_rows, rows_launch) > ctx->d.max_positions)
+            return fail(ctx, SWIFT_ECAPACITY, "KV cache too small for the rows of the token tree");
     }
     ST(enqueue_verify(ctx, rows_launch, forced_k));
     DevState hs;
     ST(read_state(ctx, &hs));
     ctx->last_k = hs.n_drafted;
     ctx->phase = PH_VERIFIED;
-    const int rows = hs.n_drafted + 1;
+    const int rows = hs.tree_rows > 0 ? hs.tree_rows : hs.n_drafted + 1;
     if (target_argmax) for (int r = 0; r < rows; ++r) target_argmax[r] = hs.argmax[r];
     if (logits_host) {
         CU(copy_async(ctx, logits_host, kptr<float>(ctx, ctx->kl.logits), (size_t)rows * ctx->d.vocab * 4, cudaMemcpyDeviceToHost));
         CU(cudaStreamSynchronize(ctx->stream));
     }
     return SWIFT_OK;
+}
+
+swift_status swift_set_tree(swift_ctx* ctx, int32_t tree_rows)
+{
+    if (!ctx) return SWIFT_EINVAL;
+    if (tree_rows != 0 && (tree_rows < 2 || tree_rows > SWIFT_MAX_ROWS)) return fail(ctx, SWIFT_EINVAL, "tree_rows must be 0 or in 2..%d", SWIFT_MAX_ROWS);
+    if (ctx->round_open) return fail(ctx, SWIFT_ESTATE, "cannot change the verification form inside a round");
+    ctx->tree_rows = tree_rows;
+    return SWIFT_OK;
+}
+
+swift_status swift_verify_tree(swift_ctx* ctx, const int32_t* tokens_host, const int32_t* parent_host, int32_t n_rows,
+                               int32_t* target_argmax, float* logits_host)
+{
+    if (!ctx) return SWIFT_EINVAL;
+    if (ctx->phase != PH_READY && ctx->phase != PH_DRAFTED) return fail(ctx, SWIFT_ESTATE, "swift_verify_tree needs a prefilled context");
+    if (ctx->mode != SWIFT_GREEDY) return fail(ctx, SWIFT_EUNSUPPORTED, "token trees are verified under greedy decoding only");
+    if (!tokens_host || !parent_host) return fail(ctx, SWIFT_EINVAL, "null argument");
+    if (n_rows < 1 || n_rows > SWIFT_MAX_ROWS) return fail(ctx, SWIFT_ECAPACITY, "a tree of %d rows; at most %d", n_rows, SWIFT_MAX_ROWS);
+    if (tokens_host[0] != ctx->pending) return fail(ctx, SWIFT_EINVAL, "row 0 of the tree must be the pending token");
+    if (parent_host[0] != -1) return fail(ctx, SWIFT_EINVAL, "row 0 is the root: its parent must be -1");
+    for (int i = 1; i < n_rows; ++i)
+        if (parent_host[i] < 0 || parent_host[i] >= i) return fail(ctx, SWIFT_EINVAL, "parent of row %d must be an earlier row", i);
+    ST(check_tokens(ctx, tokens_host, n_rows));
+    if (ctx->n + n_rows > ctx->d.max_positions) return fail(ctx, SWIFT_ECAPACITY, "KV cache too small");
+    if (ctx->phase == PH_READY) {
+        ctx->round++;
+        launch_begin_round(ctx, 0.f);
+        ctx->round_open = true;
+    }
+    DevState* st = state_of(ctx);
+    CU(copy_async(ctx, st->draft_tok, tokens_host, (size_t)n_rows * 4, cudaMemcpyHostToDevice));
+    CU(copy_async(ctx, st->row_parent, parent_host, (size_t)n_rows * 4, cudaMemcpyHostToDevice));
+    begin_verify_given_tree_kernel<<<1, 1, 0, ctx->stream>>>(st, ctx->n, n_rows);
+    ctx->launches++;
+    HeadOpts head;
+    head.run = true;
+    ST(forward_cached(ctx, n_rows, st->draft_tok, nullptr, pt_main(ctx), head));
+    DevState hs;
+    ST(read_state(ctx, &hs));
+    ctx->last_k = hs.n_drafted;
+    ctx->phase = PH_VERIFIED;
+    if (target_argmax) for (int r = 0; r < n_rows; ++r) target_argmax[r] = hs.argmax[r];
+    if (logits_host) {
+        CU(copy_async(ctx, logits_host, kptr<float>(ctx, ctx->kl.logits), (size_t)n_rows * ctx->d.vocab * 4, cudaMemcpyDeviceToHost));
+        CU(cudaStreamSynchronize(ctx->stream));
+    }
+    return SWIFT_OK;
+}
+
+int32_t swift_tree_rows(const swift_ctx* ctx, int32_t* tokens_host, int32_t* parent_host, int32_t* depth_host)
+{
+    if (!ctx) return -1;
+    const DevState& hs = ctx->last_state;
+    const int rows = hs.tree_rows > 0 ? hs.tree_rows : 0;
+    for (int r = 0; r < rows; ++r) {
+        if (tokens_host) tokens_host[r] = hs.draft_tok[r];
+        if (parent_host) parent_host[r] = hs.row_parent[r];
+        if (depth_host) depth_host[r] = hs.row_depth[r];
+    }
+    return rows;
 }
 
 swift_status swift_accept(swift_ctx* ctx, int32_t* n_accepted, int32_t* next_token)
@@ -1525,6 +1620,8 @@ swift_status swift_generate(swift_ctx* ctx, const swift_gen_params* gp, const in
     const swift_model_desc& d = ctx->d;
     if (gp->max_new < 1) return fail(ctx, SWIFT_EINVAL, "max_new must be >= 1");
     if (n_prompt + gp->max_new + 1 > d.max_positions) return fail(ctx, SWIFT_ECAPACITY, "prompt + max_new exceeds max_positions");
+    if (!gp->vanilla && tree_active(ctx) && n_prompt + gp->max_new + ctx->tree_rows > d.max_positions)
+        return fail(ctx, SWIFT_ECAPACITY, "prompt + max_new + tree_rows exceeds max_positions (the rows of a token tree occupy cache slots)");
     if (!gp->vanilla) {
         if (!gp->skip_mask) return fail(ctx, SWIFT_EINVAL, "skip_mask is null");
         if (gp->max_draft < 0 || gp->max_draft > d.max_draft) return fail(ctx, SWIFT_ECAPACITY, "max_draft %d outside 0..%d", gp->max_draft, d.max_draft);
@@ -1633,12 +1730,13 @@ swift_status swift_generate(swift_ctx* ctx, const swift_gen_params* gp, const in
             stt.ms_draft += md; stt.ms_verify += mv;
             double bd = 0.0;
             for (int j = 0; j < hs.n_drafted; ++j) bd += forward_bytes(ctx, z.data(), 1, n_start + j);
-            const double bv = forward_bytes(ctx, nullptr, hs.n_drafted + 1, n_start);
+            const int v_rows = hs.tree_rows > 0 ? hs.tree_rows : hs.n_drafted + 1;
+            const double bv = forward_bytes(ctx, nullptr, v_rows, n_start);
             stt.bytes_draft += bd;
             stt.bytes_verify += bv;
             double sd = 0.0;                      // the same forwards with the cache counted as it is stored
             for (int j = 0; j < hs.n_drafted; ++j) sd += forward_bytes(ctx, z.data(), 1, n_start + j, 0);
-            ctx->round_times.push_back({md, mv, bd, bv, hs.n_drafted, sd, forward_bytes(ctx, nullptr, hs.n_drafted + 1, n_start, 0)});
+            ctx->round_times.push_back({md, mv, bd, bv, hs.n_drafted, sd, forward_bytes(ctx, nullptr, v_rows, n_start, 0)});
             stt.drafted += hs.n_drafted;
             stt.accepted += hs.n_accepted;
         }

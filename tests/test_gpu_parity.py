@@ -710,3 +710,109 @@ def test_full_depth_13b_scoring_and_rounds():
     finally:
         g.set_sampling(False)
         g.close()
+
+
+# ------------------------------------------------------------------------------ dynamic verification (token tree)
+def _tree_round(o, g, z, max_k, budget, stats):
+    """One round with dynamic verification on both sides from the same state; compares the tree the device built with the
+    oracle's, every row's logits and arg max, the accepted path and the next token (margin rules as elsewhere)."""
+    d_tok, d_conf, d_rows = o.draft(z, max_k)
+    tree = so.build_tree(o.tokens[-1], d_tok, d_rows, d_conf, budget)
+    g_tok, g_conf = g.draft(z, max_k)
+    am, logits = g.verify()
+    t_tok, t_par, t_dep = g.tree_rows()
+    same = list(g_tok) == d_tok and t_tok == tree.tokens
+    if same:
+        assert t_par == tree.parent and t_dep == tree.depth
+        stats["trees_equal"] += 1
+    else:
+        # a different chain or another choice of alternatives is allowed only where the oracle's own ranking of the draft
+        # logits is nearly tied, or a confidence sits on the edge of a bin (another width)
+        near = False
+        for j, row in enumerate(d_rows):
+            width = so.tree_width(d_conf[j])
+            top = torch.sort(row.to(torch.float64), descending=True).values[:width + 1]
+            near = near or float((top[:-1] - top[1:]).min()) <= MARGIN or min(abs(d_conf[j] - e) for e in (0.5, 0.8, 0.95)) < 1e-3
+        assert near, (list(g_tok), d_tok, t_tok, tree.tokens)
+        g.accept()
+        tl = o.verify_tree(tree)
+        path, nxt = so.accept_tree(tree, tl)
+        o.commit_path(tree, path, nxt)
+        resync(g, o)
+        stats["resyncs"] += 1
+        return
+    tl = o.verify_tree(tree)
+    M = len(tree.tokens)
+    err = logit_err(logits[:M], tl)
+    stats["max_logit_err"] = max(stats["max_logit_err"], err)
+    assert err <= LOGIT_TOL, err
+    margins = [so.top2_margin(tl[i]) for i in range(M)]
+    for i in range(M):
+        if margins[i] > MARGIN:
+            assert int(am[i]) == so.argmax_lowest(tl[i]), i
+    path, nxt = so.accept_tree(tree, tl)
+    a, g_next = g.accept()
+    o.commit_path(tree, path, nxt)
+    stats["rounds"] += 1
+    stats["alternatives"] += int(any(r > len(d_tok) for r in path))
+    if (a, g_next) == (len(path), nxt):
+        stats["accept_cmp"] += 1
+    else:
+        assert min(margins[r] for r in [0] + path) <= MARGIN, (a, g_next, path, nxt)
+        resync(g, o)
+        stats["resyncs"] += 1
+
+
+def _tree_stats():
+    return dict(rounds=0, trees_equal=0, accept_cmp=0, resyncs=0, alternatives=0, max_logit_err=0.0)
+
+
+@pytest.mark.parametrize("which,budget,max_k", [("tiny", 16, 4), ("tiny", 9, 6), ("small", 16, 5), ("bf16", 16, 8)])
+def test_tree_rounds_follow_the_oracle(which, budget, max_k, tiny_pair, small_pair, bf16_pair, small_cfg):
+    """Dynamic verification (Section 4.2) round by round against the oracle: the same tree, logits of every row (chain and
+    alternatives, each at its own depth behind its own ancestors), the accepted path, and the cache after an accepted
+    alternative was moved to its slot (the following rounds read it)."""
+    o, g = {"tiny": tiny_pair, "small": small_pair, "bf16": bf16_pair}[which]
+    cfg = {"tiny": TINY, "small": small_cfg, "bf16": BF16_SMALL}[which]
+    prompt = synth.prompt(cfg, 21)
+    z = list(synth.block_mask(cfg, synth.planted_blocks(cfg)[:1])) if which != "small" else [1, 0, 0, 0, 0, 1, 0, 0]
+    o.prefill(prompt); g.prefill(prompt); g.set_pending(o.tokens[-1])
+    g.set_tree(budget)
+    st = _tree_stats()
+    try:
+        for _ in range(10):
+            _tree_round(o, g, z, max_k, budget, st)
+        print(f"tree rounds ({which}, {budget} rows): {st}")
+        assert st["rounds"] >= 8 and st["accept_cmp"] >= st["rounds"] - 2 and st["alternatives"] >= 1, st
+        for b in range(cfg.n_blocks):                      # the cache after the moves is the target's
+            assert np.allclose(g.read_kv(b, 0, 0, g.n), o.K[b][:o.n].numpy(), atol=2e-3 if which == "bf16" else 1e-4)
+            assert np.allclose(g.read_kv(b, 1, 0, g.n), o.V[b][:o.n].numpy(), atol=2e-3 if which == "bf16" else 1e-4)
+    finally:
+        g.set_tree(0)
+
+
+def test_generate_with_dynamic_verification(tiny_pair):
+    """Whole runs with the token tree: the output is still vanilla greedy decoding (Section 3.1), it matches the oracle's run
+    with the same row budget round for round, and a round emits at least as many tokens as the chain alone would."""
+    from paper_2410_06916_b200 import GenParams
+    o, g = tiny_pair
+    prompt = synth.prompt(TINY, 30)
+    z = synth.block_mask(TINY, synth.planted_blocks(TINY)[:3])
+    van, _, _ = g.generate(prompt, GenParams(max_new=60, vanilla=True))
+    chain, st0, _ = g.generate(prompt, GenParams(max_new=60, max_draft=5, skip_mask=z))
+    g.set_tree(16)
+    try:
+        out, st, trace = g.generate(prompt, GenParams(max_new=60, max_draft=5, skip_mask=z))
+    finally:
+        g.set_tree(0)
+    ref, margins = so.vanilla_generate(so.Oracle(o.s, o.w, dtype=o.dtype, max_positions=192), prompt, 60)
+    o2 = so.Oracle(o.s, o.w, dtype=o.dtype, max_positions=192)
+    o_out, o_rounds, o_stats = so.swift_generate(o2, prompt, list(z), so.GenParams(max_new=60, max_draft=5, tree_rows=16))
+    assert o_out == ref
+    n_same = compare_free_running(out, ref, margins)
+    assert chain == van and (out == van or n_same < 60)                 # lossless; a tree round may differ from vanilla only at a near-tie
+    if out == o_out:
+        assert [int(t[2]) for t in trace] == [r.accepted for r in o_rounds]
+        assert st.rounds == o_stats["rounds"]
+    assert st.rounds <= st0.rounds                                       # alternatives only ever add accepted tokens
+    print(f"tree generate: {st.rounds} rounds with the tree, {st0.rounds} without; oracle {o_stats['rounds']}")
