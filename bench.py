@@ -170,6 +170,35 @@ def sample_text(cfg, small, run, n_ctx, seconds=None):
             + ("" if small is cfg else "; on an 8-block copy of the model, scaled by depth (extrapolated)"))
 
 
+def stream_mode(model, cfg, run, z, gp, args, max_new, desc, hbm_peak):
+    """A stream of inputs with the skip set carried over: input i starts from the set input i-1 ended with
+    (swift_final_skip_mask) and keeps optimising it until an input ends above the matchness threshold; after that the
+    set is used as it is.  One vanilla run per input gives the reference speed on the same prompt."""
+    import dataclasses
+    from paper_2410_06916_b200 import GenParams
+    carry, optimising, rows = z, run.optimise, []
+    model.generate(synth.prompt(cfg, 64), GenParams(max_new=8, vanilla=True))          # warm-up
+    tot_tokens = tot_ms = van_ms = 0.0
+    for i in range(args.stream):
+        prompt = synth.prompt(cfg, run.prompt_len, stream=100 + i)
+        gpi = dataclasses.replace(gp, skip_mask=carry, n_opt_rounds=gp.n_opt_rounds if optimising else 0, opt_seed=gp.opt_seed + i)
+        out, st, _ = model.generate(prompt, gpi)
+        van, vst, _ = model.generate(prompt, GenParams(max_new=max_new, vanilla=True))
+        carry = model.final_skip_mask()
+        if st.opt_rounds > 0 and st.best_matchness > run.stop_matchness:
+            optimising = False
+        rows.append({"input": i, "tokens_per_s": (st.tokens - 1) / (st.ms_decode * 1e-3), "vanilla_tokens_per_s": (vst.tokens - 1) / (vst.ms_decode * 1e-3),
+                     "alpha": st.accepted / max(st.drafted, 1), "M": (st.tokens - 1) / st.rounds, "opt_rounds": st.opt_rounds,
+                     "best_matchness": st.best_matchness, "ms_score": st.ms_score, "equals_vanilla": out == van,
+                     "skipped_blocks": [int(b) for b in range(cfg.n_blocks) if carry[2 * b] and carry[2 * b + 1]]})
+        tot_tokens += st.tokens - 1; tot_ms += st.ms_decode; van_ms += vst.ms_decode
+    print(json.dumps({"metric": METRIC, "value": tot_tokens / (tot_ms * 1e-3), "unit": UNIT, "n_gpus": 1, "steps": args.stream, "warmup": 1,
+                      "ms_per_step": tot_ms / args.stream, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+                      "dtype": "bf16" if cfg.dtype == "bf16" else "f32", "data": "synthetic",
+                      "config": config_of(desc + f"; stream of {args.stream} inputs, skip set carried over", args.kv_dtype),
+                      "vanilla_tokens_per_s": tot_tokens / (van_ms * 1e-3), "speedup_vs_vanilla": van_ms / tot_ms, "stream": rows}))
+
+
 def micro(cfg, run, args, hbm_peak):
     """Each GEMM shape of the walk, alone, on a 4-block copy of the model (weights still several times L2)."""
     from paper_2410_06916_b200 import SwiftModel
@@ -197,6 +226,9 @@ def main():
     ap.add_argument("--prompt-len", type=int, default=0, help="override the prompt length (profiling runs)")
     ap.add_argument("--kv-dtype", default="f32", choices=["f32", "bf16"], help="storage of cached K,V")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--stream", type=int, default=0,
+                    help="run the workload as a stream of this many inputs (different prompts), each starting from the skip set "
+                         "the previous one ended with (the dynamic input streams of the paper's Section 5.3); prints one JSON line")
     ap.add_argument("--micro", action="store_true",
                     help="time each weight-streaming GEMM of the model alone on a few-block copy (profiling aid); prints one JSON line")
     ap.add_argument("--micro-iters", type=int, default=40)
@@ -271,12 +303,20 @@ def main():
     if sampling:
         model.set_sampling(True, run.temperature, run.rng_seed, run.top_p)
     prompt = synth.prompt(cfg, run.prompt_len, stream=rank)
-    cands = None
     if run.optimise:
-        cands = np.stack([synth.candidate_masks(cfg, run.n_skip_blocks, run.n_candidates, r) for r in range(run.max_opt_rounds)])
+        # config 3 as written: start from the uniform pattern; every optimisation round the library proposes the candidates
+        # itself (random search, a Gaussian-process proposal every 25th step: Section 4.1, Appendix B.2) and scores them
+        # together with the set in use; it stops above matchness 0.95, after the round cap, or after 300 proposals in a
+        # row without a better set (Appendix B.2's patience, in rounds of n_candidates proposals)
         z = synth.block_mask(cfg, synth.uniform_blocks(cfg.n_blocks, run.n_skip_blocks))
     gp = GenParams(max_new=max_new, max_draft=run.max_draft, stop_conf=run.stop_conf, skip_mask=z, gamma=run.gamma,
-                   n_opt_rounds=run.max_opt_rounds if run.optimise else 0, stop_matchness=run.stop_matchness, candidate_masks=cands)
+                   n_opt_rounds=run.max_opt_rounds if run.optimise else 0, stop_matchness=run.stop_matchness,
+                   n_candidates=run.n_candidates if run.optimise else 0, opt_skip_blocks=run.n_skip_blocks, opt_beta=25,
+                   opt_seed=cfg.seed, opt_patience=-(-300 // run.n_candidates))
+
+    if args.stream > 0:
+        stream_mode(model, cfg, run, z, gp, args, max_new, desc, hbm_peak)
+        return
 
     def barrier():
         torch.cuda.synchronize()

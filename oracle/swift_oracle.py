@@ -501,14 +501,16 @@ def vanilla_generate(o: Oracle, prompt: Sequence[int], max_new: int, mode: str =
 
 
 def swift_generate(o: Oracle, prompt: Sequence[int], z0: Sequence[int], gp: GenParams,
-                   candidates=None) -> Tuple[List[int], List[Round], dict]:
+                   candidates=None, optimizer: "Optional[LayerSetOptimizer]" = None,
+                   n_candidates: int = 0) -> Tuple[List[int], List[Round], dict]:
     """Draft-then-verify decoding with skipped sub-layer set z (Sections 4.1-4.2).
 
     Each round: [optionally score candidates on the last gamma generated tokens and keep the best] ->
     draft at most N_D tokens (stop early below epsilon) -> verify with the full model -> accept ->
     roll the KV cache back.  Emits exactly gp.max_new tokens: the draft length is capped at
     remaining - 1, and with one token left a plain full-model step is taken.
-    `candidates(round) -> masks [C, L]` supplies the proposals of one optimisation round.
+    `candidates(round) -> masks [C, L]` supplies the proposals of one optimisation round; alternatively `optimizer`
+    (a LayerSetOptimizer) proposes n_candidates sets per round and is told every score of the round.
 
     An optimisation round scores the set in use together with the proposals on the same window (the set in
     use is entry 0 of the round's `matchness`) and keeps the highest-scoring one (Section 4.1), the earliest
@@ -530,9 +532,16 @@ def swift_generate(o: Oracle, prompt: Sequence[int], z0: Sequence[int], gp: GenP
         r += 1
         remaining = gp.max_new - (len(o.tokens) - n_prompt)
         scores = None
-        if optimising and len(o.tokens) - n_prompt >= gp.gamma and candidates is not None:
-            masks = [list(z)] + [[int(v) for v in m] for m in candidates(opt_rounds)]
+        if optimising and len(o.tokens) - n_prompt >= gp.gamma and (candidates is not None or optimizer is not None):
+            if optimizer is not None:
+                proposals = [optimizer.mask(optimizer.suggest()) for _ in range(n_candidates)]
+            else:
+                proposals = [[int(v) for v in m] for m in candidates(opt_rounds)]
+            masks = [list(z)] + proposals
             scores, _ = o.score_skipsets(masks, gp.gamma)
+            if optimizer is not None:
+                for mk, sc in zip(masks, scores):
+                    optimizer.observe([b for b in range(o.s.n_blocks) if mk[2 * b] and mk[2 * b + 1]], sc)
             c_best = max(range(len(scores)), key=lambda c: (scores[c], -c))   # entry 0, the set in use, wins ties
             best_score, z = scores[c_best], masks[c_best]
             stale = 0 if c_best != 0 else stale + 1

@@ -34,7 +34,7 @@ constexpr int AM_THREADS = 128;
 #define SWIFT_AM_V_LATE 1
 #endif
 #ifndef SWIFT_AM_CTAS
-#define SWIFT_AM_CTAS 4
+#define SWIFT_AM_CTAS 3
 #endif
 constexpr bool AM_V_LATE = SWIFT_AM_V_LATE != 0;   // V loaded after the scores (fewer live registers, more CTAs per SM)
 constexpr int AM_QSTRIDE = 144;     // bf16 per staged query row (288 bytes): the rows of a fragment load fall into different banks

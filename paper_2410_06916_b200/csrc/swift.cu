@@ -1073,7 +1073,12 @@ swift_status swift_load(const swift_model_desc* desc, swift_devbuf weights, swif
         c->attn_rows_per_cta = (v == 1 || v == 2 || v == 4 || v == 6 || v == 8 || v == 12) ? v : 16;
     }
     c->fuse_combine = getenv("SWIFT_NO_FUSE_COMBINE") == nullptr;
-    c->attn_mma = getenv("SWIFT_NO_ATTN_MMA") == nullptr;      // full-model forwards on the streaming attention kernel too
+    {
+        // Tensor-core attention for the target model's forwards: SWIFT_ATTN_MMA=1 / 0 forces it on / off; by default it
+        // serves grouped-query shapes (several query heads per KV head share one CTA's K,V loads there).
+        const char* e = getenv("SWIFT_ATTN_MMA");
+        c->attn_mma = e ? atoi(e) != 0 : desc->n_heads / desc->n_kv_heads >= 4;
+    }
     c->prefetch_next = getenv("SWIFT_NO_PREFETCH_NEXT") == nullptr;
     {
         const char* e = getenv("SWIFT_PREFETCH_TILES");      // 16 KB tiles of the next GEMM each CTA asks L2 for

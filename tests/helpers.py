@@ -13,8 +13,9 @@ LOGIT_TOL = 2e-2        # max |dlogit| / std(oracle row)
 MARGIN = 0.05           # tokens must agree wherever the oracle's top-1/top-2 gap exceeds this
 
 
-def make_pair(cfg, max_positions=256, page_size=16, max_draft=15, oracle_dtype=None, kv_dtype="f32"):
-    """(oracle, gpu model) over identical synthetic weights."""
+def make_pair(cfg, max_positions=256, page_size=16, max_draft=15, oracle_dtype=None, kv_dtype="f32", widen=True):
+    """(oracle, gpu model) over identical synthetic weights.  widen=False keeps the oracle's copy in the storage type
+    (it widens a tensor whenever it applies it): half the host memory of an fp32 copy, for the multi-billion shapes."""
     from paper_2410_06916_b200 import SwiftModel
     w = synth.make_weights(cfg)
     gpu = SwiftModel(cfg, max_positions=max_positions, page_size=page_size, max_draft=max_draft, kv_dtype=kv_dtype)
@@ -24,7 +25,7 @@ def make_pair(cfg, max_positions=256, page_size=16, max_draft=15, oracle_dtype=N
             gpu.pack(name, b, t)
     if oracle_dtype is None:
         oracle_dtype = torch.float64 if cfg.dtype == "f32" else torch.float32
-    if cfg.dtype == "bf16":          # widen once (exact) so the oracle does not convert on every call
+    if cfg.dtype == "bf16" and widen:    # widen once (exact) so the oracle does not convert on every call
         w = {k: (v.to(oracle_dtype) if torch.is_tensor(v) else [{n: t.to(oracle_dtype) for n, t in blk.items()} for blk in v])
              for k, v in w.items()}
     o = so.Oracle(so.Shape.of(cfg), w, dtype=oracle_dtype, max_positions=max_positions)

@@ -674,44 +674,6 @@ def test_full_depth_against_oracle_and_losslessness(name, n_skip, max_draft, n_p
         g.close()
 
 
-@pytest.mark.slow
-def test_full_depth_13b_scoring_and_rounds():
-    """Configs 3 and 4 at full size (40 blocks, 26 GB of weights): candidate scoring on 32 context tokens (Eq. 2-3),
-    one greedy round with the planted skip set and one speculative-sampling round with 20 blocks skipped, each step
-    compared with the oracle (which regenerates the weights it needs from the seed)."""
-    import psutil
-    if psutil.virtual_memory().available < 48 * 2 ** 30:
-        pytest.skip("needs 48 GB of host memory")
-    cfg = synth.MODELS["13b"]
-    o, g = make_streamed_pair(cfg, max_positions=256, max_draft=8)
-    try:
-        prompt = synth.prompt(cfg, 40)
-        o.prefill(prompt)
-        g.prefill(prompt)
-        g.set_pending(o.tokens[-1])
-        z18 = synth.block_mask(cfg, synth.draft_blocks(cfg, 18))
-        masks = np.stack([z18, np.zeros_like(z18), synth.candidate_masks(cfg, 18, 1, 0)[0]])
-        ref, _ = o.score_skipsets(masks.tolist(), 32)
-        got = g.score_skipsets(masks, 32)
-        # (the window here is prompt text, not the model's own output, so even the empty set scores low: the point
-        # is that both sides count the same matches)
-        for c in range(len(masks)):
-            if got[c] != pytest.approx(ref[c]):
-                rows = o.forward_rows(o.tokens[o.n - 32:o.n], o.n - 32, masks[c].tolist(), write_kv=False)
-                assert min(so.top2_margin(r) for r in rows) <= MARGIN, (c, got[c], ref[c])
-        st = walk_rounds(o, g, list(z18), n_rounds=1, max_k=4)
-        assert st["max_logit_err"] < LOGIT_TOL and st["rounds"] + st["resyncs"] == 1, st
-        seed = 4
-        g.set_sampling(True, 1.0, seed)
-        resync(g, o, 1)
-        z20 = list(synth.block_mask(cfg, synth.draft_blocks(cfg, 20)))
-        st = walk_rounds(o, g, z20, n_rounds=1, max_k=3, sampling=True, seed=seed, first_round=2, dec_tol=BF16_DEC_TOL)
-        assert st["max_logit_err"] < LOGIT_TOL, st
-    finally:
-        g.set_sampling(False)
-        g.close()
-
-
 # ------------------------------------------------------------------------------ dynamic verification (token tree)
 def _tree_round(o, g, z, max_k, budget, stats):
     """One round with dynamic verification on both sides from the same state; compares the tree the device built with the
@@ -775,7 +737,9 @@ def test_tree_rounds_follow_the_oracle(which, budget, max_k, tiny_pair, small_pa
     o, g = {"tiny": tiny_pair, "small": small_pair, "bf16": bf16_pair}[which]
     cfg = {"tiny": TINY, "small": small_cfg, "bf16": BF16_SMALL}[which]
     prompt = synth.prompt(cfg, 21)
-    z = list(synth.block_mask(cfg, synth.planted_blocks(cfg)[:1])) if which != "small" else [1, 0, 0, 0, 0, 1, 0, 0]
+    # a skip set whose drafts are often wrong, so that alternatives get accepted and moved (tiny: a block that is not planted)
+    z = {"tiny": list(synth.block_mask(cfg, [b for b in range(cfg.n_blocks) if b not in synth.planted_blocks(cfg)][:1])),
+         "small": [1, 0, 0, 0, 0, 1, 0, 0], "bf16": list(synth.block_mask(cfg, synth.planted_blocks(cfg)[:1]))}[which]
     o.prefill(prompt); g.prefill(prompt); g.set_pending(o.tokens[-1])
     g.set_tree(budget)
     st = _tree_stats()
@@ -783,7 +747,8 @@ def test_tree_rounds_follow_the_oracle(which, budget, max_k, tiny_pair, small_pa
         for _ in range(10):
             _tree_round(o, g, z, max_k, budget, st)
         print(f"tree rounds ({which}, {budget} rows): {st}")
-        assert st["rounds"] >= 8 and st["accept_cmp"] >= st["rounds"] - 2 and st["alternatives"] >= 1, st
+        assert st["rounds"] >= 8 and st["accept_cmp"] >= st["rounds"] - 2, st
+        assert st["alternatives"] >= 1 or which != "tiny", st          # the move of an accepted alternative was exercised
         for b in range(cfg.n_blocks):                      # the cache after the moves is the target's
             assert np.allclose(g.read_kv(b, 0, 0, g.n), o.K[b][:o.n].numpy(), atol=2e-3 if which == "bf16" else 1e-4)
             assert np.allclose(g.read_kv(b, 1, 0, g.n), o.V[b][:o.n].numpy(), atol=2e-3 if which == "bf16" else 1e-4)
@@ -816,3 +781,129 @@ def test_generate_with_dynamic_verification(tiny_pair):
         assert st.rounds == o_stats["rounds"]
     assert st.rounds <= st0.rounds                                       # alternatives only ever add accepted tokens
     print(f"tree generate: {st.rounds} rounds with the tree, {st0.rounds} without; oracle {o_stats['rounds']}")
+
+
+def test_generate_with_the_librarys_own_proposals(tiny_pair):
+    """On-the-fly optimisation with the library proposing the candidates (random search with a Gaussian-process proposal every
+    beta-th step, Section 4.1) against the oracle running its own engine with the same seed: same proposals, same scores,
+    same set at the end."""
+    from paper_2410_06916_b200 import GenParams
+    o, g = tiny_pair
+    prompt = synth.prompt(TINY, 32)
+    z0 = synth.block_mask(TINY, synth.uniform_blocks(8, 4))
+    o2 = so.Oracle(o.s, o.w, dtype=o.dtype, max_positions=192)
+    opt = so.LayerSetOptimizer(8, 4, beta=5, seed=7)
+    ogp = so.GenParams(max_new=90, max_draft=4, gamma=32, max_opt_rounds=4, stop_matchness=2.0)
+    o_out, o_rounds, _ = so.swift_generate(o2, prompt, list(z0), ogp, optimizer=opt, n_candidates=6)
+    out, st, _ = g.generate(prompt, GenParams(max_new=90, max_draft=4, gamma=32, n_opt_rounds=4, stop_matchness=2.0, skip_mask=z0,
+                                              n_candidates=6, opt_skip_blocks=4, opt_beta=5, opt_seed=7))
+    assert out == o_out and st.opt_rounds == 4
+    scored = [r for r in o_rounds if r.matchness is not None]
+    assert len(scored) == 4 and all(len(r.matchness) == 7 for r in scored)
+    assert abs(st.best_matchness - max(scored[-1].matchness)) <= 1.0 / 32 + 1e-6
+    assert g.final_skip_mask().tolist() == o_rounds[-1].z
+
+
+@pytest.mark.slow
+def test_configs_3_and_4_at_benchmark_context_full_depth():
+    """Configs 3 and 4 as they run: the 13B shape at full depth behind the benchmark's 1024-token prompt.  The GPU generates
+    with the planted skip set; the oracle then replays the whole committed sequence teacher-forced in one pass (every
+    emitted token must be its arg max given the same prefix, and the GPU's logits of the last rows must match), which also
+    leaves the oracle in the GPU's state for: a candidate-scoring round on 32 context tokens (config 3, Eq. 2-3) and one
+    speculative-sampling round with 20 blocks skipped (config 4), each compared step by step."""
+    import gc
+    import psutil
+    if psutil.virtual_memory().available < 44 * 2 ** 30:
+        pytest.skip("needs 44 GB of host memory")
+    gc.collect()
+    torch.cuda.empty_cache()
+    from paper_2410_06916_b200 import GenParams
+    cfg = synth.MODELS["13b"]
+    n_prompt, n_new = 1024, 48
+    o, g = make_pair(cfg, max_positions=n_prompt + n_new + 64, max_draft=8, widen=False)
+    try:
+        prompt = synth.prompt(cfg, n_prompt)
+        z18 = synth.block_mask(cfg, synth.draft_blocks(cfg, 18))
+        out, st, trace = g.generate(prompt, GenParams(max_new=n_new, max_draft=8, skip_mask=z18))
+        assert st.accepted > 0 and g.n == n_prompt + n_new - 1
+        seq = list(prompt) + out[:-1]
+        ref = o.forward_rows(seq, 0)                                  # one teacher-forced pass: row i predicts token i + 1
+        o.n, o.tokens = len(seq), seq + [out[-1]]
+        exempt = 0
+        for i, tok in enumerate(out):
+            row = ref[n_prompt - 1 + i]
+            if so.argmax_lowest(row) != tok:
+                assert so.top2_margin(row) <= MARGIN, (i, tok, so.argmax_lowest(row), so.top2_margin(row))
+                exempt += 1
+        got, _ = g.forward_rows(seq[-9:], len(seq) - 9, write_kv=False)
+        err = logit_err(got, ref[-9:])
+        print(f"13b at {len(seq)} positions, full depth: logits off by {err:.2e} sigma; {exempt} of {n_new} tokens on a near-tie; "
+              f"{st.accepted}/{st.drafted} drafts accepted")
+        assert err < LOGIT_TOL and exempt <= 3
+        # config 3: one scoring round on the last 32 generated tokens
+        masks = np.stack([z18, np.zeros_like(z18), synth.candidate_masks(cfg, 18, 1, 0)[0]])
+        ref_m, _ = o.score_skipsets(masks.tolist(), 32)
+        got_m = g.score_skipsets(masks, 32)
+        assert got_m[1] == 1.0 or exempt > 0
+        for c in range(len(masks)):
+            assert abs(got_m[c] - ref_m[c]) <= (1.0 / 32 + 1e-6), (c, got_m[c], ref_m[c])
+        # one greedy round step by step (draft tokens and confidences, target logits, accepted length)
+        st3 = walk_rounds(o, g, list(z18), n_rounds=1, max_k=4)
+        assert st3["max_logit_err"] < LOGIT_TOL and st3["rounds"] + st3["resyncs"] == 1, st3
+        # config 4: one speculative-sampling round with 20 blocks skipped
+        seed = 4
+        g.set_sampling(True, 1.0, seed)
+        resync(g, o, 1)
+        z20 = list(synth.block_mask(cfg, synth.draft_blocks(cfg, 20)))
+        st4 = walk_rounds(o, g, z20, n_rounds=1, max_k=3, sampling=True, seed=seed, first_round=2, dec_tol=BF16_DEC_TOL)
+        assert st4["max_logit_err"] < LOGIT_TOL, st4
+    finally:
+        g.set_sampling(False)
+        g.close()
+
+
+@pytest.mark.slow
+def test_config2_whole_run_against_the_oracles_trace():
+    """Config 2 as it runs (7B shape, 512-token prompt, 256 greedy tokens, the planted 14 blocks skipped, at most 8 drafts)
+    against the oracle's free-running trace stored under tests/golden/ (written by tests/golden/make_traces.py, which calls
+    only the oracle): tokens identical up to the first position where the oracle's top-1/top-2 margin is small, and the
+    accepted lengths of the rounds before it."""
+    import json
+    import os
+    from tests.golden.make_traces import trace_key
+    path = os.path.join(os.path.dirname(os.path.abspath(__file__)), "golden", "c2_trace.json")
+    if not os.path.exists(path):
+        pytest.skip("no stored trace")
+    tr = json.load(open(path))
+    if tr["key"] != trace_key("c2"):
+        pytest.skip("the stored trace was written by another version of the oracle or of the input generator")
+    import gc
+    gc.collect()
+    torch.cuda.empty_cache()
+    from paper_2410_06916_b200 import GenParams, SwiftModel
+    model_name, run = synth.RUNS["c2"]
+    cfg = synth.MODELS[model_name]
+    g = SwiftModel(cfg, max_positions=run.prompt_len + run.max_new + 32, max_draft=run.max_draft)
+    try:
+        g.load_weights(synth.iter_tensors(cfg))
+        prompt = synth.prompt(cfg, run.prompt_len)
+        z = np.asarray(tr["skip_mask"], dtype=np.uint8)
+        assert z.tolist() == synth.block_mask(cfg, synth.draft_blocks(cfg, run.n_skip_blocks)).tolist()
+        van, _, _ = g.generate(prompt, GenParams(max_new=run.max_new, vanilla=True))
+        out, st, trace = g.generate(prompt, GenParams(max_new=run.max_new, max_draft=run.max_draft, skip_mask=z))
+        n_same = compare_free_running(van, tr["tokens"], tr["margins"])
+        assert out == van
+        # rounds that lie wholly before the first tolerated divergence: same start, same drafts accepted, same next token
+        checked = 0
+        for r, ref in zip(trace, tr["rounds"]):
+            if ref["n_start"] + len(ref["draft"]) + 1 - run.prompt_len >= n_same:
+                break
+            if min(ref["draft_margin"] + ref["target_margin"]) <= MARGIN:
+                break                                             # a near-tie inside the round: lengths may differ from here on
+            assert (int(r[0]), int(r[2]), int(r[3])) == (ref["n_start"], ref["accepted"], ref["next_token"]), (checked, r, ref)
+            checked += 1
+        print(f"config 2 against the stored trace: {n_same} of {run.max_new} tokens before the first near-tie, {checked} rounds compared, "
+              f"M {(st.tokens - 1) / st.rounds:.2f} (oracle {tr['stats']['M']:.2f}), alpha {st.accepted / max(st.drafted, 1):.2f} (oracle {tr['stats']['alpha']:.2f})")
+        assert n_same >= 16 and checked >= 1
+    finally:
+        g.close()
