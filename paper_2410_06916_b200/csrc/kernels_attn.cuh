@@ -194,8 +194,9 @@ attn_split_kernel(const DevState* st, const float* __restrict__ q, const T* __re
 __device__ __forceinline__ void combine_row(int pos0, int r, int h, const float* __restrict__ o_part,
                                             const float2* __restrict__ ml_part, int max_splits, int n_heads, int dh,
                                             float* __restrict__ out, __nv_bfloat16* __restrict__ planes,
-                                            float* comb_sh, float* wmax_sh, int part_rows = ROWS)
+                                            float* comb_sh, float* wmax_sh, int part_rows = ROWS, int row_shift = 0)
 {
+    // row_shift: where row r of this sequence sits in the partial-result and output buffers (a sequence inside a larger chunk)
     const int d = threadIdx.x;
     // row r sees positions <= pos0 + r: later splits hold nothing for it (and, when the rows were processed in
     // groups, were not written for it at all)
@@ -206,7 +207,7 @@ __device__ __forceinline__ void combine_row(int pos0, int r, int h, const float*
 
     // the first 16 splits' partial outputs are requested before anything else: they do not depend on the weights
     constexpr int CB = 16;
-    const float* op = o_part + (base * part_rows + r) * dh + d;
+    const float* op = o_part + (base * part_rows + r + row_shift) * dh + d;
     const size_t stride = (size_t)part_rows * dh;
     float o[CB];
 #pragma unroll
@@ -214,7 +215,7 @@ __device__ __forceinline__ void combine_row(int pos0, int r, int h, const float*
 
     float mx = -INFINITY;
     for (int s = d; s < n_splits; s += blockDim.x) {
-        const float2 ml = __ldcg(ml_part + (base + s) * part_rows + r);
+        const float2 ml = __ldcg(ml_part + (base + s) * part_rows + r + row_shift);
         w_sh[s] = ml.x;
         l_sh[s] = ml.y;
         mx = fmaxf(mx, ml.x);
@@ -245,8 +246,8 @@ __device__ __forceinline__ void combine_row(int pos0, int r, int h, const float*
         }
     }
     const float v = num / den;
-    out[((size_t)r * n_heads + h) * dh + d] = v;
-    if (planes) store_hi_lo(planes, r, n_heads * dh, h * dh + d, v);
+    out[((size_t)(r + row_shift) * n_heads + h) * dh + d] = v;
+    if (planes) store_hi_lo(planes, r + row_shift, n_heads * dh, h * dh + d, v);
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -509,14 +510,17 @@ attn_stream_kernel(const DevState* st, const float* __restrict__ q, const T* __r
 // order (combine_row above).
 __global__ void attn_combine_kernel(const DevState* st, const float* __restrict__ o_part,
                                     const float2* __restrict__ ml_part, int max_splits, int n_heads, int dh,
-                                    float* __restrict__ out, __nv_bfloat16* __restrict__ planes)
+                                    float* __restrict__ out, __nv_bfloat16* __restrict__ planes, int part_rows,
+                                    int row_base, int n_rows_fixed, int pos0_fixed)
 {
+    // row_base / n_rows_fixed / pos0_fixed: as in attn_mma_kernel (one sequence inside a larger chunk), 0 / 0 / 0 otherwise
     pdl_enter();
     const int r = blockIdx.y;
-    if (r >= st->n_rows) return;
+    if (r >= (n_rows_fixed > 0 ? n_rows_fixed : st->n_rows)) return;
     extern __shared__ float comb_sh[];
     __shared__ float wmax_sh[32];
-    combine_row(st->pos0, r, blockIdx.x, o_part, ml_part, max_splits, n_heads, dh, out, planes, comb_sh, wmax_sh);
+    combine_row(n_rows_fixed > 0 ? pos0_fixed : st->pos0, r, blockIdx.x, o_part, ml_part, max_splits, n_heads, dh, out, planes, comb_sh,
+                wmax_sh, part_rows, row_base);
 }
 
 } // namespace swk

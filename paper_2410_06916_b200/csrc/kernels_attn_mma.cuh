@@ -80,13 +80,16 @@ __global__ void __launch_bounds__(AM_THREADS, SWIFT_AM_CTAS)
 attn_mma_kernel(const DevState* st, const float* __restrict__ q, const T* __restrict__ kv_pool,
                 const int* __restrict__ page_table, KvLayout L, int block, int n_heads, int max_splits, float scale,
                 float* __restrict__ o_part, float2* __restrict__ ml_part, int part_rows, int* __restrict__ head_counters,
-                float* __restrict__ out, __nv_bfloat16* __restrict__ planes)
+                float* __restrict__ out, __nv_bfloat16* __restrict__ planes, int row_base, int n_rows_fixed, int pos0_fixed)
 {
+    // n_rows_fixed > 0: the rows [row_base, row_base + n_rows_fixed) of a larger chunk form one sequence of their own, whose
+    // first row sits at cache slot pos0_fixed (candidate scoring); otherwise the whole forward is the sequence.
     pdl_enter();
     constexpr int DH = 128, QR = 8 * NT;                    // query rows per pass
-    const int n_rows = st->n_rows;
+    const int n_rows = n_rows_fixed > 0 ? n_rows_fixed : st->n_rows;
     if (n_rows <= 0) return;
-    const int pos0 = st->pos0, total = pos0 + n_rows;
+    const int pos0 = n_rows_fixed > 0 ? pos0_fixed : st->pos0, total = pos0 + n_rows;
+    q += (size_t)row_base * n_heads * 128;
     const int kvh = blockIdx.x, s = blockIdx.y, c0 = s * ATTN_CHUNK;
     if (c0 >= total) return;
     const int len = min(ATTN_CHUNK, total - c0);
@@ -277,7 +280,7 @@ attn_mma_kernel(const DevState* st, const float* __restrict__ q, const T* __rest
                 num = fmaf(wt, part_acc[((size_t)ww * QR + rl) * AM_OSTRIDE + tid], num);
                 den = fmaf(wt, ml.y, den);
             }
-            const size_t slot = ((size_t)(kvh * G + hl) * max_splits + s) * part_rows + r;
+            const size_t slot = ((size_t)(kvh * G + hl) * max_splits + s) * part_rows + row_base + r;
             o_part[slot * DH + tid] = num;
             if (tid == 0) ml_part[slot] = make_float2(M, den);
         }

@@ -46,6 +46,24 @@ constexpr int TC_PRE = 1;           // tiles requested before the set-up barrier
 constexpr int TC_STAGE_BYTES = TC_A_BYTES + TC_B_BYTES;
 constexpr int TC_SMEM_BYTES = TC_STAGES * TC_STAGE_BYTES + 1024 /*alignment slack*/ + 256 /*barriers*/;
 constexpr long long TC_WAIT_CYCLES = 3000000000LL;  // ~1.5 s of SM clocks before a wait is declared dead
+
+// The same kernel serves forwards of up to 16 rows (NB = 1: decoding) and of up to 16 * NB rows (NB = 2, 4, 8: prefill
+// chunks and candidate scoring).  Rows come in blocks of 16; block rb occupies operand rows / accumulator columns
+// [32 rb, 32 rb + 32): its 16 hi rows, then its 16 lo rows.  More rows per weight tile mean a wider MMA (N = 32 NB), a
+// larger activation tile per stage and fewer stages in the same shared memory.
+template <int NB>
+struct TcShape {
+    static constexpr int COLS = TC_COLS * NB;                        // MMA N
+    static constexpr int B_BYTES = COLS * TC_BK * 2;
+    static constexpr int STAGE_BYTES = TC_A_BYTES + B_BYTES;
+    static constexpr int STAGES = NB == 1 ? TC_STAGES : (196 * 1024) / STAGE_BYTES;   // 8, 6, 4 stages for NB = 2, 4, 8
+    static constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + 1024 + 256;
+    static constexpr int TMEM_COLS = 2 * COLS;                       // two accumulator buffers; 64 .. 512, a power of two
+    static constexpr uint32_t IDESC = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(COLS >> 3) << 17) | ((uint32_t)(TC_TILE_N >> 4) << 24);
+    static constexpr int ROWS_MAX = ROWS * NB;
+};
+constexpr int TC_NB_MAX = 8;
+constexpr int TC_ROWS_MAX = ROWS * TC_NB_MAX;       // rows of the largest forward chunk
 constexpr int TC_ERR_TIMEOUT = 2;
 
 // ------------------------------------------------------------------------------ PTX wrappers
@@ -152,12 +170,14 @@ struct StreamK {
     }
 };
 
-// fp32 rows -> the two bf16 planes the tensor-core GEMM reads: plane[r] = bf16(x), plane[16 + r] = bf16(x - hi).
+// fp32 rows -> the two bf16 planes the tensor-core GEMM reads, in blocks of 16 rows: row r of the forward sits in block
+// r / 16; a block is 32 operand rows, hi = bf16(x) in its first 16 and lo = bf16(x - hi) in its last 16.
 __device__ __forceinline__ void store_hi_lo(__nv_bfloat16* planes, int r, int K, int i, float x)
 {
     const __nv_bfloat16 hi = __float2bfloat16_rn(x);
-    planes[(size_t)r * K + i] = hi;
-    planes[(size_t)(ROWS + r) * K + i] = __float2bfloat16_rn(x - __bfloat162float(hi));
+    const size_t row = (size_t)(r >> 4) * (2 * ROWS) + (r & (ROWS - 1));
+    planes[row * K + i] = hi;
+    planes[(row + ROWS) * K + i] = __float2bfloat16_rn(x - __bfloat162float(hi));
 }
 
 // What the epilogue does with a finished output tile.  The element-wise steps of the decoder walk are
@@ -191,16 +211,24 @@ struct EpiParams {
     KvLayout L;
     int block, n_heads, max_positions;
     const float2* rope_cs;
+    int sum_rows;                   // rows per tile in sumsq_in / sumsq_out: 16 for decoding, 16 * NB for chunks of many rows
+    // EPI_QKV on a chunk that holds several sequences side by side (candidate scoring: every candidate's window rows, each
+    // with its own scratch pages): per 16-row block, the cache slot of its first row and the page table of its sequence
+    int per_block;
+    int rb_pos0[8];
+    const int* rb_page_table[8];
     // any epilogue: shape of the GEMM that runs next on this stream (0 = none): each CTA asks for the first
     // weight tiles it will need there to be brought into L2 while this launch drains
     int next_N, next_K, next_tiles;
 };
 
+// row0: first row of the 16-row block this call finishes (0 when decoding); n_rows: rows of that block that exist;
+// pos0: cache slot of row row0; rstd_sh / rope_sh / page_sh are indexed by the row within the block.
 template <int EPI, typename TKV>
 __device__ __forceinline__ void tc_finalize(const EpiParams& ep, int pos0, float (&val)[ROWS], int n_rows, int tile,
                                             int quarter, int lane, int etid, int N, float* Y, const float* rstd_sh,
                                             float* stage_sh, const float (&h_pre)[ROWS], float gain_pre,
-                                            const float2* rope_sh, const int* page_sh)
+                                            const float2* rope_sh, const int* page_sh, int row0 = 0)
 {
     // h_pre / gain_pre (EPI_RESID) and rope_sh / page_sh (EPI_QKV) were fetched while the accumulator was still
     // being computed, so that nothing here waits for a round trip to L2 before it can store.
@@ -214,7 +242,7 @@ __device__ __forceinline__ void tc_finalize(const EpiParams& ep, int pos0, float
         if (n < N) {
 #pragma unroll
             for (int m = 0; m < ROWS; ++m)
-                if (m < n_rows) Y[(size_t)m * N + n] = val[m];
+                if (m < n_rows) Y[(size_t)(row0 + m) * N + n] = val[m];
         }
     } else if (EPI == EPI_SWIGLU) {
         // rows come in groups of 32: 16 gate rows then the 16 matching up rows (same warp); staged through shared
@@ -227,7 +255,7 @@ __device__ __forceinline__ void tc_finalize(const EpiParams& ep, int pos0, float
 #pragma unroll 1
             for (int m = 0; m < n_rows; ++m) {
                 const float g = stage_sh[m * TC_TILE_N + l], up = stage_sh[m * TC_TILE_N + l + 16];
-                store_hi_lo(ep.act_planes, m, ep.ffn, i, g / (1.f + expf(-g)) * up);
+                store_hi_lo(ep.act_planes, row0 + m, ep.ffn, i, g / (1.f + expf(-g)) * up);
             }
         }
         __syncwarp();                                  // the staging rows are rewritten by the next tile
@@ -242,8 +270,8 @@ __device__ __forceinline__ void tc_finalize(const EpiParams& ep, int pos0, float
             float hn = 0.f;
             if (n < N) {
                 hn = stage_sh[m * TC_TILE_N + l];
-                ep.h[(size_t)m * N + n] = hn;
-                if (ep.gain_next) store_hi_lo(ep.planes_out, m, N, n, hn * gain_pre);
+                ep.h[(size_t)(row0 + m) * N + n] = hn;
+                if (ep.gain_next) store_hi_lo(ep.planes_out, row0 + m, N, n, hn * gain_pre);
             }
             if (ep.gain_next) {                        // uniform over the grid
                 const float w = warp_sum(hn * hn);
@@ -253,7 +281,7 @@ __device__ __forceinline__ void tc_finalize(const EpiParams& ep, int pos0, float
         if (ep.gain_next) {
             asm volatile("bar.sync 1, 128;" ::: "memory");
             if (etid < ROWS)
-                ep.sumsq_out[(size_t)tile * ROWS + etid] = etid < n_rows ?
+                ep.sumsq_out[(size_t)tile * ep.sum_rows + row0 + etid] = etid < n_rows ?
                     (sums_sh[etid] + sums_sh[ROWS + etid]) + (sums_sh[2 * ROWS + etid] + sums_sh[3 * ROWS + etid]) : 0.f;
             asm volatile("bar.sync 1, 128;" ::: "memory");
         }
@@ -278,7 +306,7 @@ __device__ __forceinline__ void tc_finalize(const EpiParams& ep, int pos0, float
                         out = i < half ? a * cs.x - b * cs.y : a * cs.x + b * cs.y;
                     }
                     if (gh < ep.n_heads) {
-                        ep.q_out[(size_t)m * ep.n_heads * dh + n] = out;
+                        ep.q_out[(size_t)(row0 + m) * ep.n_heads * dh + n] = out;
                     } else {
                         const int hk = gh - ep.n_heads;
                         const int kv = hk >= ep.L.n_kv_heads ? 1 : 0;
@@ -295,12 +323,13 @@ __device__ __forceinline__ void tc_finalize(const EpiParams& ep, int pos0, float
 // grid = G persistent CTAs, block = 192 threads, dynamic smem = TC_SMEM_BYTES.
 // mapW: bf16 [N][K], box {64, 128}; mapX: bf16 [32][K] (rows 0-15 hi, 16-31 lo), box {64, 32}; both
 // 128-byte swizzled.  slabs: [S_max][ROWS][N] fp32; counters: one int per tile, zero on entry and on exit.
-template <int EPI, typename TKV>
+template <int EPI, typename TKV, int NB = 1>
 __global__ void __launch_bounds__(TC_THREADS, 1)
 gemm_tc_kernel(DevState* st, const __grid_constant__ CUtensorMap mapW, const __grid_constant__ CUtensorMap mapX,
                float* __restrict__ Y, float* __restrict__ slabs, int* __restrict__ counters, int N, int K,
                const __grid_constant__ EpiParams ep, const __grid_constant__ CUtensorMap mapNext)
 {
+    typedef TcShape<NB> S;
     pdl_trigger();
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int n_tiles = (N + TC_TILE_N - 1) / TC_TILE_N;
@@ -313,15 +342,15 @@ gemm_tc_kernel(DevState* st, const __grid_constant__ CUtensorMap mapW, const __g
 
     extern __shared__ unsigned char smem_raw[];
     const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;        // swizzled tiles need 1024-byte alignment
-    const uint32_t bars = base + TC_STAGES * TC_STAGE_BYTES;            // full[8], empty[8], tfull[2], tempty[2]
+    const uint32_t bars = base + S::STAGES * S::STAGE_BYTES;            // full[8], empty[8], tfull[2], tempty[2]
     auto full_bar = [&](int s) { return bars + 8u * s; };
-    auto empty_bar = [&](int s) { return bars + 8u * (TC_STAGES + s); };
-    auto tfull_bar = [&](int b) { return bars + 8u * (2 * TC_STAGES + b); };
-    auto tempty_bar = [&](int b) { return bars + 8u * (2 * TC_STAGES + 2 + b); };
+    auto empty_bar = [&](int s) { return bars + 8u * (S::STAGES + s); };
+    auto tfull_bar = [&](int b) { return bars + 8u * (2 * S::STAGES + b); };
+    auto tempty_bar = [&](int b) { return bars + 8u * (2 * S::STAGES + 2 + b); };
     __shared__ uint32_t tmem_base_sh;
     __shared__ int last_flag_sh, peek_sh;
     __shared__ int abort_sh, epi_abort_sh;
-    __shared__ float rstd_sh[ROWS];
+    __shared__ float rstd_sh[ROWS * NB];
     __shared__ float stage_sh[EPI == EPI_PLAIN ? 4 * ROWS : ROWS * TC_TILE_N + 4 * ROWS];
     __shared__ float2 rope_sh[EPI == EPI_QKV ? ROWS * (TC_TILE_N / 2) : 1];   // (cos, sin) of the rows' positions
     __shared__ int page_sh[ROWS];                                              // KV page of each row's position
@@ -342,17 +371,17 @@ gemm_tc_kernel(DevState* st, const __grid_constant__ CUtensorMap mapW, const __g
         const int n_pre0 = (int)((u_end - u_begin) < TC_PRE ? (u_end - u_begin) : TC_PRE);
         int tile0 = (int)(u_begin / sk.KB), kb0 = (int)(u_begin - (long long)tile0 * sk.KB);
         for (int i = 0, t = tile0, k = kb0; i < n_pre0; ++i, (++k == sk.KB ? (k = 0, ++t) : 0)) {
-            mbar_expect_tx(full_bar(i), TC_STAGE_BYTES);
-            tma_load_2d(base + i * TC_STAGE_BYTES, &mapW, k * TC_BK, t * TC_TILE_N, full_bar(i));
+            mbar_expect_tx(full_bar(i), S::STAGE_BYTES);
+            tma_load_2d(base + i * S::STAGE_BYTES, &mapW, k * TC_BK, t * TC_TILE_N, full_bar(i));
         }
         pdl_wait();
         n_rows_early = st->n_rows;
         for (int i = 0, k = kb0; i < n_pre0; ++i, (++k == sk.KB ? (k = 0) : 0))
-            tma_load_2d(base + i * TC_STAGE_BYTES + TC_A_BYTES, &mapX, k * TC_BK, 0, full_bar(i));
+            tma_load_2d(base + i * S::STAGE_BYTES + TC_A_BYTES, &mapX, k * TC_BK, 0, full_bar(i));
     }
     if (warp == 1) {   // this warp sets up the remaining barriers and allocates 64 TMEM columns: two accumulator buffers of 32
         if (lane == 0) {
-            for (int s = 0; s < TC_STAGES; ++s) { if (s >= TC_PRE) mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
+            for (int s = 0; s < S::STAGES; ++s) { if (s >= TC_PRE) mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
             for (int b = 0; b < 2; ++b) { mbar_init(tfull_bar(b), 1); mbar_init(tempty_bar(b), 4); }
             abort_sh = 0;
             epi_abort_sh = 0;
@@ -361,7 +390,7 @@ gemm_tc_kernel(DevState* st, const __grid_constant__ CUtensorMap mapW, const __g
         __syncwarp();
         pdl_wait();
         n_rows_early = st->n_rows;
-        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&tmem_base_sh)), "r"(64));
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&tmem_base_sh)), "r"(S::TMEM_COLS));
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;");
     }
     tc_fence_before();
@@ -379,10 +408,10 @@ gemm_tc_kernel(DevState* st, const __grid_constant__ CUtensorMap mapW, const __g
             int it = n_pre;
             int tile = (int)((u_begin + n_pre) / sk.KB), kb = (int)((u_begin + n_pre) % sk.KB);
             for (long long u = u_begin + n_pre; u < u_end; ++u, ++it, (++kb == sk.KB ? (kb = 0, ++tile) : 0)) {
-                const int s = it % TC_STAGES;
-                if (!mbar_wait(empty_bar(s), ((it / TC_STAGES) & 1) ^ 1)) { abort_sh = 1; break; }
-                const uint32_t a_dst = base + s * TC_STAGE_BYTES, b_dst = a_dst + TC_A_BYTES;
-                mbar_expect_tx(full_bar(s), TC_STAGE_BYTES);
+                const int s = it % S::STAGES;
+                if (!mbar_wait(empty_bar(s), ((it / S::STAGES) & 1) ^ 1)) { abort_sh = 1; break; }
+                const uint32_t a_dst = base + s * S::STAGE_BYTES, b_dst = a_dst + TC_A_BYTES;
+                mbar_expect_tx(full_bar(s), S::STAGE_BYTES);
                 tma_load_2d(a_dst, &mapW, kb * TC_BK, tile * TC_TILE_N, full_bar(s));
                 tma_load_2d(b_dst, &mapX, kb * TC_BK, 0, full_bar(s));
             }
@@ -417,14 +446,14 @@ gemm_tc_kernel(DevState* st, const __grid_constant__ CUtensorMap mapW, const __g
                     if (!mbar_wait(tempty_bar(buf), ((seg >> 1) & 1) ^ 1)) { abort_sh = 1; break; }
                     tc_fence_after();
                 }
-                const int s = it % TC_STAGES;
-                if (!mbar_wait(full_bar(s), (it / TC_STAGES) & 1)) { abort_sh = 1; break; }
+                const int s = it % S::STAGES;
+                if (!mbar_wait(full_bar(s), (it / S::STAGES) & 1)) { abort_sh = 1; break; }
                 tc_fence_after();
-                const uint32_t a_addr = base + s * TC_STAGE_BYTES, b_addr = a_addr + TC_A_BYTES;
+                const uint32_t a_addr = base + s * S::STAGE_BYTES, b_addr = a_addr + TC_A_BYTES;
                 const uint64_t a_desc = tc_smem_desc(a_addr), b_desc = tc_smem_desc(b_addr);
 #pragma unroll
                 for (int k = 0; k < TC_BK / 16; ++k)   // 16 bf16 = 32 bytes further along the swizzled row
-                    tc_mma(tmem_base + buf * TC_COLS, a_desc + 2 * k, b_desc + 2 * k, TC_IDESC, (seg_first && k == 0) ? 0u : 1u);
+                    tc_mma(tmem_base + buf * S::COLS, a_desc + 2 * k, b_desc + 2 * k, S::IDESC, (seg_first && k == 0) ? 0u : 1u);
                 tc_commit(empty_bar(s));               // smem stage reusable once these MMAs have read it
                 if (seg_last) { tc_commit(tfull_bar(buf)); ++seg; }
             }
@@ -438,16 +467,16 @@ gemm_tc_kernel(DevState* st, const __grid_constant__ CUtensorMap mapW, const __g
         const int etid = tid - 64;                     // 0..127
         int seg = 0;
         long long u = n_rows != 0 ? u_begin : u_end;
-        if (etid < ROWS) {                             // rstd of the RMSNorm in front of this GEMM (1 when there is none)
+        if (etid < ROWS * NB) {                        // rstd of the RMSNorm in front of this GEMM (1 when there is none)
             float r = 1.f;
             if (EPI != EPI_RESID && ep.sumsq_in) {
                 float ss = 0.f;
-                for (int t = 0; t < ep.n_sumsq_tiles; ++t) ss += ep.sumsq_in[(size_t)t * ROWS + etid];
+                for (int t = 0; t < ep.n_sumsq_tiles; ++t) ss += ep.sumsq_in[(size_t)t * ep.sum_rows + etid];
                 r = rsqrtf(ss * ep.inv_d + ep.eps);
             }
             rstd_sh[etid] = r;
         }
-        if (EPI == EPI_QKV) {
+        if (EPI == EPI_QKV && NB == 1) {
             const int half = ep.L.head_dim >> 1, pos0 = pos0_epi;
             for (int idx = etid; idx < ROWS * half; idx += 128) {
                 const int m = idx / half, j = idx - m * half, pos = pos0 + m;
@@ -460,7 +489,112 @@ gemm_tc_kernel(DevState* st, const __grid_constant__ CUtensorMap mapW, const __g
             }
         }
         asm volatile("bar.sync 1, 128;" ::: "memory");
-        while (u < u_end) {
+        if constexpr (NB > 1) {
+            // Chunks of many rows: the accumulator holds NB blocks of 16 rows side by side; each is drained, finished
+            // (or parked in this CTA's slab) in turn with the code of the 16-row case.  No early fetches and no
+            // fast path here: these launches are long enough for their tails not to matter.
+            constexpr int RT = ROWS * NB;
+            const int live_blocks = (n_rows + ROWS - 1) / ROWS;
+            auto finish_block = [&](int rb, float (&val)[ROWS], int tile, int n) {
+                const int row0 = rb * ROWS, rows_here = min(ROWS, n_rows - row0);
+                const int pos_b = (EPI == EPI_QKV && ep.per_block) ? ep.rb_pos0[rb] : pos0_epi + row0;   // cache slot of the block's first row
+                if (EPI == EPI_QKV) {                      // rotary factors and cache pages of this block's rows
+                    const int* pt = ep.per_block ? ep.rb_page_table[rb] : ep.page_table;
+                    asm volatile("bar.sync 1, 128;" ::: "memory");
+                    const int half = ep.L.head_dim >> 1;
+                    for (int idx = etid; idx < ROWS * half; idx += 128) {
+                        const int m = idx / half, j = idx - m * half, pos = pos_b + m;
+                        if (m < rows_here && pos < ep.max_positions) rope_sh[m * (TC_TILE_N / 2) + j] = ep.rope_cs[(size_t)pos * half + j];
+                    }
+                    if (etid < ROWS) {
+                        const int pos = pos_b + etid;
+                        page_sh[etid] = (etid < rows_here && pos < ep.max_positions) ? pt[pos >> ep.L.page_shift] : 0;
+                    }
+                    asm volatile("bar.sync 1, 128;" ::: "memory");
+                }
+                float h_pre[ROWS];
+                float gain_pre = 0.f;
+                if (EPI == EPI_RESID) {
+#pragma unroll
+                    for (int m = 0; m < ROWS; ++m) h_pre[m] = (n < N && m < rows_here) ? __ldcg(ep.h + (size_t)(row0 + m) * N + n) : 0.f;
+                    if (ep.gain_next && n < N) gain_pre = ep.gain_next[n];
+                }
+                tc_finalize<EPI, TKV>(ep, pos_b, val, rows_here, tile, quarter, lane, etid, N, Y, rstd_sh + row0, stage_sh,
+                                      h_pre, gain_pre, rope_sh, page_sh, row0);
+            };
+            while (u < u_end) {
+                const int tile = (int)(u / sk.KB), kb0 = (int)(u % sk.KB);
+                const long long tile_end = (long long)(tile + 1) * sk.KB;
+                const long long seg_end = tile_end < u_end ? tile_end : u_end;
+                const int buf = seg & 1;
+                const int n = tile * TC_TILE_N + quarter * 32 + lane;
+                const bool whole = (kb0 == 0) && (seg_end == tile_end);
+                int slab = 0, nseg = 1;
+                if (!whole) {
+                    const int g_first = sk.owner((long long)tile * sk.KB), g_last = sk.owner(tile_end - 1);
+                    slab = blockIdx.x - g_first;
+                    nseg = g_last - g_first + 1;
+                }
+                if (!mbar_wait(tfull_bar(buf), (seg >> 1) & 1)) epi_abort_sh = 1;
+                asm volatile("bar.sync 1, 128;" ::: "memory");
+                if (epi_abort_sh) { abort_sh = 1; break; }
+                tc_fence_after();
+                for (int rb = 0; rb < live_blocks; ++rb) {
+                    uint32_t v[32];
+                    const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(buf * S::COLS + rb * TC_COLS);
+                    asm volatile(
+                        "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+                        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+                        "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+                        : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]),
+                          "=r"(v[8]), "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15]),
+                          "=r"(v[16]), "=r"(v[17]), "=r"(v[18]), "=r"(v[19]), "=r"(v[20]), "=r"(v[21]), "=r"(v[22]), "=r"(v[23]),
+                          "=r"(v[24]), "=r"(v[25]), "=r"(v[26]), "=r"(v[27]), "=r"(v[28]), "=r"(v[29]), "=r"(v[30]), "=r"(v[31])
+                        : "r"(taddr));
+                    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+                    float val[ROWS];
+#pragma unroll
+                    for (int m = 0; m < ROWS; ++m) val[m] = __uint_as_float(v[m]) + __uint_as_float(v[16 + m]);
+                    if (whole) {
+                        finish_block(rb, val, tile, n);
+                    } else if (n < N) {
+                        float* mine = slabs + ((size_t)slab * RT + rb * ROWS) * N;
+                        const int rows_here = min(ROWS, n_rows - rb * ROWS);
+#pragma unroll
+                        for (int m = 0; m < ROWS; ++m)
+                            if (m < rows_here) mine[(size_t)m * N + n] = val[m];
+                    }
+                }
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(tempty_bar(buf));   // accumulator buffer free again (4 warps arrive)
+                if (!whole) {
+                    asm volatile("bar.sync 1, 128;" ::: "memory");
+                    if (etid == 0) last_flag_sh = (atom_add_acq_rel_gpu(&counters[tile], 1) == nseg - 1) ? 1 : 0;
+                    asm volatile("bar.sync 1, 128;" ::: "memory");
+                    if (last_flag_sh) {                         // last arrival: add the slabs in slab order, block by block
+                        for (int rb = 0; rb < live_blocks; ++rb) {
+                            const int rows_here = min(ROWS, n_rows - rb * ROWS);
+                            float val[ROWS];
+#pragma unroll
+                            for (int m = 0; m < ROWS; ++m) val[m] = 0.f;
+                            if (n < N)
+                                for (int j = 0; j < nseg; ++j) {
+#pragma unroll
+                                    for (int m = 0; m < ROWS; ++m)
+                                        if (m < rows_here) val[m] += __ldcg(slabs + (((size_t)j * RT + rb * ROWS + m) * N + n));
+                                }
+                            finish_block(rb, val, tile, n);
+                        }
+                        if (etid == 0) counters[tile] = 0;
+                    }
+                    asm volatile("bar.sync 1, 128;" ::: "memory");
+                }
+                ++seg;
+                u = seg_end;
+            }
+        }
+        while (NB == 1 && u < u_end) {
             const int tile = (int)(u / sk.KB), kb0 = (int)(u % sk.KB);
             const long long tile_end = (long long)(tile + 1) * sk.KB;
             const long long seg_end = tile_end < u_end ? tile_end : u_end;
@@ -497,7 +631,7 @@ gemm_tc_kernel(DevState* st, const __grid_constant__ CUtensorMap mapW, const __g
                     if ((n >> 5) * 16 + (lane & 15) < ep.ffn) touch_global(ep.act_planes + (n >> 5) * 16 + (lane & 15));
                 } else if (EPI == EPI_RESID) {
                     if (ep.gain_next) touch_global(ep.planes_out + n);
-                    if (ep.gain_next && lane == 0) touch_global(ep.sumsq_out + (size_t)tile * ROWS);
+                    if (ep.gain_next && lane == 0) touch_global(ep.sumsq_out + (size_t)tile * ep.sum_rows);
                 } else {
                     const int dh = ep.L.head_dim;
                     const int gh = n / dh, i = n - gh * dh;
@@ -525,7 +659,7 @@ gemm_tc_kernel(DevState* st, const __grid_constant__ CUtensorMap mapW, const __g
             if (epi_abort_sh) { abort_sh = 1; break; }
             tc_fence_after();
             uint32_t v[32];
-            const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(buf * TC_COLS);
+            const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(buf * S::COLS);
             asm volatile(
                 "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
                 "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
@@ -613,7 +747,7 @@ gemm_tc_kernel(DevState* st, const __grid_constant__ CUtensorMap mapW, const __g
     if (abort_sh && tid == 0) st->error = TC_ERR_TIMEOUT;
     if (warp == 1) {
         tc_fence_after();
-        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(64));
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(S::TMEM_COLS));
     }
 }
 

@@ -48,7 +48,7 @@ struct WeightLayout {
 };
 
 struct WorkLayout {
-    size_t state, h, xn, xa, act, q, part, o_part, ml_part, logits, q_rows, rope, pt_main, pt_score, score_tok, cand, cand_n,
+    size_t state, h, xn, xa, act, q, part, o_part, ml_part, logits, q_rows, rope, pt_main, pt_score, score_tok, cand, cand_n, big_tok,
         score_truth, score_out, attn_counters, xn_hl, xa_hl, act_hl, slabs, counters, sumsq, total;
     size_t part_floats, slab_floats;
 };
@@ -78,7 +78,7 @@ struct swift_ctx {
     std::string err;
     cudaEvent_t ev[8];
     // captured forwards; programmatic dependent launch between the kernels of a forward
-    bool use_graphs, use_pdl, pdl_next, pdl_gemms, fuse, fuse_combine, prefetch_next, attn_mma;
+    bool use_graphs, use_pdl, pdl_next, pdl_gemms, fuse, fuse_combine, prefetch_next, attn_mma, big_chunks;
     int attn_rows_per_cta, prefetch_tiles;
     std::vector<FwdGraph>* graphs;
     uint64_t graph_clock;
@@ -90,6 +90,7 @@ struct swift_ctx {
     bool use_tc;
     std::vector<CUtensorMap> tm_wqkv, tm_wo, tm_wgu, tm_wdown;
     CUtensorMap tm_lm_head, tm_embed, tm_xn, tm_xa, tm_act;
+    CUtensorMap tm_xn_big, tm_xa_big, tm_act_big;      // the same planes seen as 2 * TC_ROWS_MAX operand rows (chunks of many rows)
 };
 
 namespace {
@@ -207,6 +208,9 @@ size_t page_bytes(const swift_model_desc* d)
     return (size_t)d->n_blocks * 2 * d->n_kv_heads * d->page_size * d->head_dim * kv_esize_of(d);
 }
 
+// Rows of the largest forward chunk: TC_ROWS_MAX where the tensor-core walk with many-row chunks applies, else 16.
+size_t big_rows_of(const swift_model_desc* d) { return (d->dtype == SWIFT_BF16 && d->head_dim == 128) ? (size_t)TC_ROWS_MAX : (size_t)ROWS; }
+
 WorkLayout work_layout(const swift_model_desc* d)
 {
     WorkLayout k;
@@ -219,15 +223,18 @@ WorkLayout work_layout(const swift_model_desc* d)
     need((int)(qd + 2 * kd), (int)dm); need((int)dm, (int)qd); need(2 * d->ffn, (int)dm); need((int)dm, d->ffn);
     need(d->vocab, (int)dm);
     k.part_floats = pf;
+    // bf16 models with head size 128 also run chunks of up to TC_ROWS_MAX rows (prefill): their row buffers are that tall
+    const size_t RB = big_rows_of(d);
     k.state = c.take(sizeof(DevState));
-    k.h = c.take(ROWS * dm * 4);
+    k.h = c.take(RB * dm * 4);
     k.xn = c.take(ROWS * dm * 4);
-    k.xa = c.take(ROWS * qd * 4);
+    k.xa = c.take(RB * qd * 4);
     k.act = c.take(ROWS * (size_t)d->ffn * 4);
-    k.q = c.take(ROWS * qd * 4);
+    k.q = c.take(RB * qd * 4);
     k.part = c.take(pf * 4);
-    k.o_part = c.take((size_t)d->n_heads * max_splits * ROWS * d->head_dim * 4);
-    k.ml_part = c.take((size_t)d->n_heads * max_splits * ROWS * 8);
+    k.o_part = c.take((size_t)d->n_heads * max_splits * RB * d->head_dim * 4);
+    k.ml_part = c.take((size_t)d->n_heads * max_splits * RB * 8);
+    k.big_tok = c.take(RB * 4);
     k.logits = c.take((size_t)ROWS * d->vocab * 4);
     k.q_rows = c.take((size_t)std::max(1, d->max_draft) * d->vocab * 4);
     k.rope = c.take((size_t)d->max_positions * (d->head_dim / 2) * 8);
@@ -244,15 +251,15 @@ WorkLayout work_layout(const swift_model_desc* d)
     k.slab_floats = 0;
     k.xn_hl = k.xa_hl = k.act_hl = k.slabs = k.counters = k.sumsq = 0;
     if (d->dtype == SWIFT_BF16) {
-        auto slab_need = [&](int N, int K) { k.slab_floats = std::max(k.slab_floats, (size_t)max_segments(N, K) * ROWS * (size_t)N); };
+        auto slab_need = [&](int N, int K) { k.slab_floats = std::max(k.slab_floats, (size_t)max_segments(N, K) * RB * (size_t)N); };
         slab_need((int)(qd + 2 * kd), (int)dm); slab_need((int)dm, (int)qd); slab_need(2 * d->ffn, (int)dm);
         slab_need((int)dm, d->ffn); slab_need(d->vocab, (int)dm);
-        k.xn_hl = c.take(2 * ROWS * dm * 2);
-        k.xa_hl = c.take(2 * ROWS * qd * 2);
-        k.act_hl = c.take(2 * ROWS * (size_t)d->ffn * 2);
+        k.xn_hl = c.take(2 * RB * dm * 2);
+        k.xa_hl = c.take(2 * RB * qd * 2);
+        k.act_hl = c.take(2 * RB * (size_t)d->ffn * 2);
         k.slabs = c.take(k.slab_floats * 4);
         k.counters = c.take(TC_MAX_TILES * 4);
-        k.sumsq = c.take((size_t)std::max(1, ceil_div((int)dm, TC_TILE_N)) * ROWS * 4);
+        k.sumsq = c.take((size_t)std::max(1, ceil_div((int)dm, TC_TILE_N)) * RB * 4);
     }
     k.total = c.off;
     return k;
@@ -330,12 +337,12 @@ struct GemmSite {
     const CUtensorMap* mapX;
 };
 
-template <int EPI, typename TKV>
+template <int EPI, typename TKV, int NB = 1>
 swift_status launch_gemm_tc(swift_ctx* ctx, const GemmSite& g, const EpiParams& ep, const CUtensorMap* next_map = nullptr)
 {
     if (ceil_div(g.N, TC_TILE_N) > TC_MAX_TILES) return fail(ctx, SWIFT_EUNSUPPORTED, "GEMM with %d output tiles", ceil_div(g.N, TC_TILE_N));
     if (ctx->pdl_gemms) ctx->pdl_next = true;     // this launch may begin before its predecessor has finished (see swift_load)
-    CU(launch_k(gemm_tc_kernel<EPI, TKV>, dim3(TC_GRID), dim3(TC_THREADS), (size_t)TC_SMEM_BYTES, ctx, state_of(ctx), *g.mapW, *g.mapX,
+    CU(launch_k(gemm_tc_kernel<EPI, TKV, NB>, dim3(TC_GRID), dim3(TC_THREADS), (size_t)TcShape<NB>::SMEM_BYTES, ctx, state_of(ctx), *g.mapW, *g.mapX,
                 kptr<float>(ctx, ctx->kl.part), kptr<float>(ctx, ctx->kl.slabs), kptr<int>(ctx, ctx->kl.counters), g.N, g.K, ep,
                 next_map ? *next_map : *g.mapW));
     return SWIFT_OK;
@@ -349,6 +356,7 @@ swift_status run_gemm(swift_ctx* ctx, int mr, const GemmSite& g, int* n_split)
         *n_split = 1;
         EpiParams ep;
         memset(&ep, 0, sizeof ep);
+        ep.sum_rows = ROWS;
         return launch_gemm_tc<EPI_PLAIN, float>(ctx, g, ep);
     }
     GemmPlan p;
@@ -387,13 +395,14 @@ swift_status launch_attn_mr(swift_ctx* ctx, const int* page_table, int block, in
     } while (0)
 
 template <typename T, int NT>
-swift_status launch_attn_mma(swift_ctx* ctx, const int* page_table, int block, bool fused, float* out, __nv_bfloat16* planes)
+swift_status launch_attn_mma(swift_ctx* ctx, const int* page_table, int block, bool fused, float* out, __nv_bfloat16* planes,
+                             int part_rows = ROWS)
 {
     const swift_model_desc& d = ctx->d;
     CU(launch_k(attn_mma_kernel<T, NT>, dim3(d.n_kv_heads, ctx->max_splits), dim3(AM_THREADS), attn_mma_smem_bytes(NT, ctx->max_splits), ctx,
                 (const DevState*)state_of(ctx), (const float*)kptr<float>(ctx, ctx->kl.q), reinterpret_cast<const T*>(ctx->kvbase),
                 page_table, ctx->kv, block, d.n_heads, ctx->max_splits, 1.0f / sqrtf((float)d.head_dim),
-                kptr<float>(ctx, ctx->kl.o_part), kptr<float2>(ctx, ctx->kl.ml_part), (int)ROWS,
+                kptr<float>(ctx, ctx->kl.o_part), kptr<float2>(ctx, ctx->kl.ml_part), part_rows,
                 fused ? kptr<int>(ctx, ctx->kl.attn_counters) : (int*)nullptr, fused ? out : (float*)nullptr,
                 fused ? planes : (__nv_bfloat16*)nullptr));
     return SWIFT_OK;
@@ -417,7 +426,7 @@ swift_status launch_attn(swift_ctx* ctx, int rows, const int* page_table, int bl
         if (fused) return SWIFT_OK;
         CU(launch_k(attn_combine_kernel, dim3(d.n_heads, rows), dim3(d.head_dim), 2 * (size_t)ctx->max_splits * sizeof(float), ctx,
                     (const DevState*)state_of(ctx), (const float*)kptr<float>(ctx, ctx->kl.o_part),
-                    (const float2*)kptr<float2>(ctx, ctx->kl.ml_part), ctx->max_splits, d.n_heads, d.head_dim, out, planes));
+                    (const float2*)kptr<float2>(ctx, ctx->kl.ml_part), ctx->max_splits, d.n_heads, d.head_dim, out, planes, (int)ROWS));
         return SWIFT_OK;
     }
     // The streaming kernel (head_dim 128) takes the rows in groups of at most attn_rows_per_cta, one group per
@@ -443,7 +452,7 @@ swift_status launch_attn(swift_ctx* ctx, int rows, const int* page_table, int bl
     if (s != SWIFT_OK || fused) return s;
     CU(launch_k(attn_combine_kernel, dim3(d.n_heads, rows), dim3(d.head_dim), 2 * (size_t)ctx->max_splits * sizeof(float), ctx,
                 (const DevState*)state_of(ctx), (const float*)kptr<float>(ctx, ctx->kl.o_part),
-                (const float2*)kptr<float2>(ctx, ctx->kl.ml_part), ctx->max_splits, d.n_heads, d.head_dim, out, planes));
+                (const float2*)kptr<float2>(ctx, ctx->kl.ml_part), ctx->max_splits, d.n_heads, d.head_dim, out, planes, (int)ROWS));
     return SWIFT_OK;
 }
 
@@ -552,6 +561,7 @@ swift_status forward_chunk_fused(swift_ctx* ctx, int rows, const int* toks_dev, 
     base.inv_d = 1.0f / (float)dm;
     base.eps = d.rms_eps;
     base.sumsq_in = sumsq;
+    base.sum_rows = ROWS;
     int n_tiles_in = 1;                          // the embedding gather writes one "tile" of sums
 
     // the weight matrices in the order this forward streams them: each GEMM prefetches the start of the next one
@@ -620,6 +630,60 @@ swift_status forward_chunk_fused(swift_ctx* ctx, int rows, const int* toks_dev, 
                     (size_t)ROWS * d.vocab, kptr<float>(ctx, ctx->kl.logits), d.vocab, 1.0f / ctx->temperature, head.mode,
                     sampling_flag(ctx), kptr<float>(ctx, ctx->kl.q_rows), ctx->top_p, vocab_cache_bytes(ctx) != 0 ? 1 : 0,
                     tree_cand(ctx, head), kptr<int>(ctx, ctx->kl.cand_n)));
+    }
+    CU(cudaGetLastError());
+    return SWIFT_OK;
+}
+
+// The full model over a chunk of up to TC_ROWS_MAX rows (prefill): the same walk as forward_chunk_fused with every weight
+// tile applied to all rows at once (the GEMM in its NB = 8 form, tensor-core attention over all rows of a chunk per K,V
+// load), no output head.  Tokens in the big_tok device array; the control block holds pos0 and the row count.
+template <typename TKV>
+swift_status forward_chunk_big(swift_ctx* ctx, int rows, const int* page_table)
+{
+    typedef __nv_bfloat16 T;
+    constexpr int NB = TC_NB_MAX;
+    const swift_model_desc& d = ctx->d;
+    DevState* st = state_of(ctx);
+    const int dm = d.d_model, qd = d.n_heads * d.head_dim, kd = d.n_kv_heads * d.head_dim, nqkv = qd + 2 * kd;
+    float* h = kptr<float>(ctx, ctx->kl.h);
+    float* xa = kptr<float>(ctx, ctx->kl.xa);
+    __nv_bfloat16* xn_hl = kptr<__nv_bfloat16>(ctx, ctx->kl.xn_hl);
+    __nv_bfloat16* xa_hl = kptr<__nv_bfloat16>(ctx, ctx->kl.xa_hl);
+    __nv_bfloat16* act_hl = kptr<__nv_bfloat16>(ctx, ctx->kl.act_hl);
+    float* sumsq = kptr<float>(ctx, ctx->kl.sumsq);
+    EpiParams base;
+    memset(&base, 0, sizeof base);
+    base.inv_d = 1.0f / (float)dm;
+    base.eps = d.rms_eps;
+    base.sumsq_in = sumsq;
+    base.sum_rows = TC_ROWS_MAX;
+    const int d_tiles = ceil_div(dm, TC_TILE_N);
+    int n_tiles_in = 1;
+    CU(launch_k(embed_fused_kernel<T>, dim3(rows), dim3(1024), 0, ctx, st, (const int*)kptr<int>(ctx, ctx->kl.big_tok),
+                (const T*)wptr<T>(ctx, ctx->wl.embed), h, (const float*)wptr<float>(ctx, ctx->wl.attn_norm[0]), xn_hl, sumsq, dm, d.vocab));
+    for (int b = 0; b < d.n_blocks; ++b) {
+        EpiParams ep = base;
+        ep.n_sumsq_tiles = n_tiles_in;
+        ep.q_out = kptr<float>(ctx, ctx->kl.q); ep.kv_pool = ctx->kvbase; ep.page_table = page_table; ep.L = ctx->kv;
+        ep.block = b; ep.n_heads = d.n_heads; ep.max_positions = d.max_positions; ep.rope_cs = kptr<float2>(ctx, ctx->kl.rope);
+        ST((launch_gemm_tc<EPI_QKV, TKV, NB>(ctx, GemmSite{nullptr, nqkv, dm, nullptr, &ctx->tm_wqkv[b], &ctx->tm_xn_big}, ep)));
+        ST((launch_attn_mma<TKV, 2>(ctx, page_table, b, false, xa, xa_hl, TC_ROWS_MAX)));
+        CU(launch_k(attn_combine_kernel, dim3(d.n_heads, rows), dim3(d.head_dim), 2 * (size_t)ctx->max_splits * sizeof(float), ctx,
+                    (const DevState*)st, (const float*)kptr<float>(ctx, ctx->kl.o_part), (const float2*)kptr<float2>(ctx, ctx->kl.ml_part),
+                    ctx->max_splits, d.n_heads, d.head_dim, xa, xa_hl, (int)TC_ROWS_MAX));
+        EpiParams resid = base;
+        resid.h = h; resid.planes_out = xn_hl; resid.sumsq_out = sumsq;
+        resid.gain_next = wptr<float>(ctx, ctx->wl.mlp_norm[b]);
+        ST((launch_gemm_tc<EPI_RESID, float, NB>(ctx, GemmSite{nullptr, dm, qd, nullptr, &ctx->tm_wo[b], &ctx->tm_xa_big}, resid)));
+        EpiParams sw = base;
+        sw.n_sumsq_tiles = d_tiles;
+        sw.act_planes = act_hl; sw.ffn = d.ffn;
+        ST((launch_gemm_tc<EPI_SWIGLU, float, NB>(ctx, GemmSite{nullptr, 2 * d.ffn, dm, nullptr, &ctx->tm_wgu[b], &ctx->tm_xn_big}, sw)));
+        // nothing reads the residual stream of a prefill chunk after its last block: no planes, no sums there
+        resid.gain_next = b + 1 < d.n_blocks ? wptr<float>(ctx, ctx->wl.attn_norm[b + 1]) : nullptr;
+        ST((launch_gemm_tc<EPI_RESID, float, NB>(ctx, GemmSite{nullptr, dm, d.ffn, nullptr, &ctx->tm_wdown[b], &ctx->tm_act_big}, resid)));
+        n_tiles_in = d_tiles;
     }
     CU(cudaGetLastError());
     return SWIFT_OK;
@@ -954,6 +1018,11 @@ cudaError_t init_kernel_attrs()
     if (e == cudaSuccess) e = cudaFuncSetAttribute(gemm_tc_kernel<EPI_SWIGLU, float>, cudaFuncAttributeMaxDynamicSharedMemorySize, TC_SMEM_BYTES);
     if (e == cudaSuccess) e = cudaFuncSetAttribute(gemm_tc_kernel<EPI_QKV, float>, cudaFuncAttributeMaxDynamicSharedMemorySize, TC_SMEM_BYTES);
     if (e == cudaSuccess) e = cudaFuncSetAttribute(gemm_tc_kernel<EPI_QKV, __nv_bfloat16>, cudaFuncAttributeMaxDynamicSharedMemorySize, TC_SMEM_BYTES);
+    constexpr int big_smem = TcShape<TC_NB_MAX>::SMEM_BYTES;
+    if (e == cudaSuccess) e = cudaFuncSetAttribute(gemm_tc_kernel<EPI_RESID, float, TC_NB_MAX>, cudaFuncAttributeMaxDynamicSharedMemorySize, big_smem);
+    if (e == cudaSuccess) e = cudaFuncSetAttribute(gemm_tc_kernel<EPI_SWIGLU, float, TC_NB_MAX>, cudaFuncAttributeMaxDynamicSharedMemorySize, big_smem);
+    if (e == cudaSuccess) e = cudaFuncSetAttribute(gemm_tc_kernel<EPI_QKV, float, TC_NB_MAX>, cudaFuncAttributeMaxDynamicSharedMemorySize, big_smem);
+    if (e == cudaSuccess) e = cudaFuncSetAttribute(gemm_tc_kernel<EPI_QKV, __nv_bfloat16, TC_NB_MAX>, cudaFuncAttributeMaxDynamicSharedMemorySize, big_smem);
     const int am_max = (int)attn_mma_smem_bytes(2, 262144 / ATTN_CHUNK);
     if (e == cudaSuccess) e = cudaFuncSetAttribute(attn_mma_kernel<float, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, am_max);
     if (e == cudaSuccess) e = cudaFuncSetAttribute(attn_mma_kernel<float, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, am_max);
@@ -1002,6 +1071,11 @@ swift_status make_all_maps(swift_ctx* ctx)
     ST(make_map(ctx, &ctx->tm_xn, ctx->ws + ctx->kl.xn_hl, 2 * ROWS, dm, TC_COLS));
     ST(make_map(ctx, &ctx->tm_xa, ctx->ws + ctx->kl.xa_hl, 2 * ROWS, qd, TC_COLS));
     ST(make_map(ctx, &ctx->tm_act, ctx->ws + ctx->kl.act_hl, 2 * ROWS, d.ffn, TC_COLS));
+    if (big_rows_of(&d) == (size_t)TC_ROWS_MAX) {
+        ST(make_map(ctx, &ctx->tm_xn_big, ctx->ws + ctx->kl.xn_hl, 2 * TC_ROWS_MAX, dm, TcShape<TC_NB_MAX>::COLS));
+        ST(make_map(ctx, &ctx->tm_xa_big, ctx->ws + ctx->kl.xa_hl, 2 * TC_ROWS_MAX, qd, TcShape<TC_NB_MAX>::COLS));
+        ST(make_map(ctx, &ctx->tm_act_big, ctx->ws + ctx->kl.act_hl, 2 * TC_ROWS_MAX, d.ffn, TcShape<TC_NB_MAX>::COLS));
+    }
     return SWIFT_OK;
 }
 
@@ -1074,10 +1148,12 @@ swift_status swift_load(const swift_model_desc* desc, swift_devbuf weights, swif
     }
     c->fuse_combine = getenv("SWIFT_NO_FUSE_COMBINE") == nullptr;
     {
-        // Tensor-core attention for the target model's forwards: SWIFT_ATTN_MMA=1 / 0 forces it on / off; by default it
-        // serves grouped-query shapes (several query heads per KV head share one CTA's K,V loads there).
+        // Tensor-core attention for the target model's decode forwards (verification, vanilla steps): opt-in with
+        // SWIFT_ATTN_MMA=1.  Measured on the same box it lost to the streaming kernel at every shape tried (13B widths:
+        // verification 0.648 against 0.662 of the roofline, vanilla steps 0.747 against 0.779); prefill chunks of many
+        // rows always use it.
         const char* e = getenv("SWIFT_ATTN_MMA");
-        c->attn_mma = e ? atoi(e) != 0 : desc->n_heads / desc->n_kv_heads >= 4;
+        c->attn_mma = e != nullptr && atoi(e) != 0;
     }
     c->prefetch_next = getenv("SWIFT_NO_PREFETCH_NEXT") == nullptr;
     {
@@ -1092,6 +1168,8 @@ swift_status swift_load(const swift_model_desc* desc, swift_devbuf weights, swif
     c->pdl_gemms = getenv("SWIFT_NO_PDL_GEMMS") == nullptr;
     c->use_pdl = getenv("SWIFT_PDL") != nullptr;
     c->fuse = getenv("SWIFT_NO_FUSE") == nullptr && desc->head_dim <= TC_TILE_N;
+    // prefill in chunks of up to TC_ROWS_MAX rows (SWIFT_NO_BIG_CHUNKS: 16 rows at a time, as decoding does)
+    c->big_chunks = c->use_tc && c->fuse && big_rows_of(desc) == (size_t)TC_ROWS_MAX && getenv("SWIFT_NO_BIG_CHUNKS") == nullptr;
     c->graphs = new std::vector<FwdGraph>();
     c->graph_clock = 0;
     cudaError_t e = init_kernel_attrs();
@@ -1219,7 +1297,24 @@ swift_status swift_prefill(swift_ctx* ctx, const int32_t* tokens, int32_t n, int
     ctx->round_open = false;
     ctx->n = 0;
     int last_rows = 0;
-    ST(run_rows(ctx, tokens, n, 0, nullptr, pt_main(ctx), 1, nullptr, nullptr, &last_rows));
+    // All but the last (up to 16) rows go through in chunks of up to TC_ROWS_MAX rows where that path exists: every weight
+    // is then streamed once per 128 rows instead of once per 16.  The last rows take the decoding path, which ends in
+    // the output head.
+    int done = 0;
+    if (ctx->big_chunks && n > 2 * ROWS) {
+        const int big_total = ((n - 1) / ROWS) * ROWS;           // leaves 1..16 rows
+        DevState* st = state_of(ctx);
+        for (int c0 = 0; c0 < big_total; c0 += TC_ROWS_MAX) {
+            const int rows = std::min((int)TC_ROWS_MAX, big_total - c0);
+            CU(copy_async(ctx, kptr<int>(ctx, ctx->kl.big_tok), tokens + c0, (size_t)rows * 4, cudaMemcpyHostToDevice));
+            set_rows_kernel<<<1, 1, 0, ctx->stream>>>(st, c0, rows);
+            ctx->launches++;
+            if (ctx->d.kv_dtype == SWIFT_BF16) ST(forward_chunk_big<__nv_bfloat16>(ctx, rows, pt_main(ctx)));
+            else ST(forward_chunk_big<float>(ctx, rows, pt_main(ctx)));
+        }
+        done = big_total;
+    }
+    ST(run_rows(ctx, tokens + done, n - done, done, nullptr, pt_main(ctx), 1, nullptr, nullptr, &last_rows));
     if (ctx->mode == SWIFT_SAMPLING) {
         sample_row_kernel<<<1, VOCAB_THREADS, 0, ctx->stream>>>(state_of(ctx), kptr<float>(ctx, ctx->kl.logits), ctx->d.vocab,
                                                                 last_rows - 1, 1.0f / ctx->temperature, ctx->seed, 0u, 0u);

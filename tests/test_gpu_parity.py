@@ -166,13 +166,16 @@ def test_full_width_bf16_forward(shape, kv):
         g.close()
 
 
-@pytest.mark.parametrize("shape,n_prefix,max_k", [("13b", 1100, 8), ("70b", 2130, 12), ("7b", 700, 8)])
-def test_benchmark_context_lengths(shape, n_prefix, max_k):
+@pytest.mark.parametrize("shape,n_prefix,max_k,attn_mma", [("13b", 1100, 8, 0), ("70b", 2130, 12, 0), ("7b", 700, 8, 0), ("70b", 1300, 12, 1),
+                                                           ("13b", 400, 8, 1)])
+def test_benchmark_context_lengths(shape, n_prefix, max_k, attn_mma, monkeypatch):
     """Two blocks at full width behind prefixes as long as the benchmark's contexts (config 3/4: 1024 + up to 512,
     config 5: 2048 + 512, config 2: 512 + 256): more than 16 attention chunks per row (the merge of the chunks runs
     its second batch), page tables of more than a hundred pages, the one-row merge inside the attention launch with
     17 to 34 chunks.  Compared with the oracle: the last prefill rows, a one-row and a (max_draft + 1)-row forward of
     the full and of a layer-skipped model, then two whole rounds of draft / verify / accept."""
+    if attn_mma:                    # the opt-in tensor-core attention for the target model's forwards (read at load)
+        monkeypatch.setenv("SWIFT_ATTN_MMA", "1")
     cfg = synth.MODELS[shape].with_blocks(2, n_planted=1)
     o, g = make_pair(cfg, max_positions=n_prefix + 64, max_draft=max_k)
     try:
@@ -664,7 +667,9 @@ def test_full_depth_against_oracle_and_losslessness(name, n_skip, max_draft, n_p
         ver, _ = g.forward_rows(prompt[-rows:], n_prompt - rows, None, write_kv=False)
         one, _ = g.forward_rows(prompt[-1:], n_prompt - 1, None, write_kv=False)
         assert logit_err(ver, ref[-rows:]) < LOGIT_TOL and logit_err(one, ref[-1:]) < LOGIT_TOL
-        assert np.array_equal(ver, got[-rows:]) and np.array_equal(one[0], got[-1])   # row-count invariance
+        assert np.array_equal(one[0], ver[-1])                      # row-count invariance, bit for bit (same cached prefix)
+        # `got` came from 16-row chunks, the prefix under `ver` from prefill's 128-row chunks: another order of additions
+        assert logit_err(ver, torch.from_numpy(got[-rows:])) < 1e-3
         z = synth.block_mask(cfg, synth.draft_blocks(cfg, n_skip))
         n_new = 2 * (max_draft + 1) + 6
         van, _, _ = g.generate(prompt, GenParams(max_new=n_new, vanilla=True))
@@ -898,12 +903,13 @@ def test_config2_whole_run_against_the_oracles_trace():
         for r, ref in zip(trace, tr["rounds"]):
             if ref["n_start"] + len(ref["draft"]) + 1 - run.prompt_len >= n_same:
                 break
-            if min(ref["draft_margin"] + ref["target_margin"]) <= MARGIN:
-                break                                             # a near-tie inside the round: lengths may differ from here on
-            assert (int(r[0]), int(r[2]), int(r[3])) == (ref["n_start"], ref["accepted"], ref["next_token"]), (checked, r, ref)
+            if (int(r[0]), int(r[2]), int(r[3])) != (ref["n_start"], ref["accepted"], ref["next_token"]):
+                # the rounds may part ways only where the oracle itself sits on a near-tie (a draft or a target arg max)
+                assert min(ref["draft_margin"] + ref["target_margin"]) <= MARGIN, (checked, r, ref)
+                break
             checked += 1
         print(f"config 2 against the stored trace: {n_same} of {run.max_new} tokens before the first near-tie, {checked} rounds compared, "
               f"M {(st.tokens - 1) / st.rounds:.2f} (oracle {tr['stats']['M']:.2f}), alpha {st.accepted / max(st.drafted, 1):.2f} (oracle {tr['stats']['alpha']:.2f})")
-        assert n_same >= 16 and checked >= 1
+        assert n_same >= 16 and checked >= 4
     finally:
         g.close()
