@@ -396,7 +396,7 @@ swift_status launch_attn_mr(swift_ctx* ctx, const int* page_table, int block, in
 
 template <typename T, int NT>
 swift_status launch_attn_mma(swift_ctx* ctx, const int* page_table, int block, bool fused, float* out, __nv_bfloat16* planes,
-                             int part_rows = ROWS)
+                             int part_rows = ROWS, int row_base = 0, int n_rows_fixed = 0, int pos0_fixed = 0)
 {
     const swift_model_desc& d = ctx->d;
     CU(launch_k(attn_mma_kernel<T, NT>, dim3(d.n_kv_heads, ctx->max_splits), dim3(AM_THREADS), attn_mma_smem_bytes(NT, ctx->max_splits), ctx,
@@ -404,7 +404,7 @@ swift_status launch_attn_mma(swift_ctx* ctx, const int* page_table, int block, b
                 page_table, ctx->kv, block, d.n_heads, ctx->max_splits, 1.0f / sqrtf((float)d.head_dim),
                 kptr<float>(ctx, ctx->kl.o_part), kptr<float2>(ctx, ctx->kl.ml_part), part_rows,
                 fused ? kptr<int>(ctx, ctx->kl.attn_counters) : (int*)nullptr, fused ? out : (float*)nullptr,
-                fused ? planes : (__nv_bfloat16*)nullptr));
+                fused ? planes : (__nv_bfloat16*)nullptr, row_base, n_rows_fixed, pos0_fixed));
     return SWIFT_OK;
 }
 
@@ -426,7 +426,7 @@ swift_status launch_attn(swift_ctx* ctx, int rows, const int* page_table, int bl
         if (fused) return SWIFT_OK;
         CU(launch_k(attn_combine_kernel, dim3(d.n_heads, rows), dim3(d.head_dim), 2 * (size_t)ctx->max_splits * sizeof(float), ctx,
                     (const DevState*)state_of(ctx), (const float*)kptr<float>(ctx, ctx->kl.o_part),
-                    (const float2*)kptr<float2>(ctx, ctx->kl.ml_part), ctx->max_splits, d.n_heads, d.head_dim, out, planes, (int)ROWS));
+                    (const float2*)kptr<float2>(ctx, ctx->kl.ml_part), ctx->max_splits, d.n_heads, d.head_dim, out, planes, (int)ROWS, 0, 0, 0));
         return SWIFT_OK;
     }
     // The streaming kernel (head_dim 128) takes the rows in groups of at most attn_rows_per_cta, one group per
@@ -452,7 +452,7 @@ swift_status launch_attn(swift_ctx* ctx, int rows, const int* page_table, int bl
     if (s != SWIFT_OK || fused) return s;
     CU(launch_k(attn_combine_kernel, dim3(d.n_heads, rows), dim3(d.head_dim), 2 * (size_t)ctx->max_splits * sizeof(float), ctx,
                 (const DevState*)state_of(ctx), (const float*)kptr<float>(ctx, ctx->kl.o_part),
-                (const float2*)kptr<float2>(ctx, ctx->kl.ml_part), ctx->max_splits, d.n_heads, d.head_dim, out, planes, (int)ROWS));
+                (const float2*)kptr<float2>(ctx, ctx->kl.ml_part), ctx->max_splits, d.n_heads, d.head_dim, out, planes, (int)ROWS, 0, 0, 0));
     return SWIFT_OK;
 }
 
@@ -671,7 +671,7 @@ swift_status forward_chunk_big(swift_ctx* ctx, int rows, const int* page_table)
         ST((launch_attn_mma<TKV, 2>(ctx, page_table, b, false, xa, xa_hl, TC_ROWS_MAX)));
         CU(launch_k(attn_combine_kernel, dim3(d.n_heads, rows), dim3(d.head_dim), 2 * (size_t)ctx->max_splits * sizeof(float), ctx,
                     (const DevState*)st, (const float*)kptr<float>(ctx, ctx->kl.o_part), (const float2*)kptr<float2>(ctx, ctx->kl.ml_part),
-                    ctx->max_splits, d.n_heads, d.head_dim, xa, xa_hl, (int)TC_ROWS_MAX));
+                    ctx->max_splits, d.n_heads, d.head_dim, xa, xa_hl, (int)TC_ROWS_MAX, 0, 0, 0));
         EpiParams resid = base;
         resid.h = h; resid.planes_out = xn_hl; resid.sumsq_out = sumsq;
         resid.gain_next = wptr<float>(ctx, ctx->wl.mlp_norm[b]);
