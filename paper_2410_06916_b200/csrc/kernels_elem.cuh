@@ -302,3 +302,95 @@ __global__ void swiglu_kernel(const DevState* st, const float* __restrict__ part
 }
 
 } // namespace swk
+
+namespace swk {
+
+// ------------------------------------------------------------------------------ candidate scoring, all candidates at once
+// Every candidate skip set keeps its own copy of the window's residual rows in H_all[c * gamma + i]; a sub-layer is
+// applied to the candidates that keep it, gathered into chunks of up to 128 rows, and scattered back (Eq. 2 evaluates
+// all candidates on the same gamma context tokens, "Parallel Candidate Evaluation", Section 4.1).
+
+// H_all[row] = embedding of the window token row % gamma.  grid = rows, any block size.
+template <typename T>
+__global__ void embed_rows_kernel(DevState* st, const int* __restrict__ toks, const T* __restrict__ embed, float* __restrict__ H_all,
+                                  int d, int vocab, int gamma)
+{
+    const int row = blockIdx.x;
+    int tok = toks[row % gamma];
+    if (tok < 0 || tok >= vocab) {
+        if (threadIdx.x == 0) st->error = 1;
+        tok = 0;
+    }
+    const T* src = embed + (size_t)tok * d;
+    for (int i = threadIdx.x; i < d; i += blockDim.x) H_all[(size_t)row * d + i] = to_float(src[i]);
+}
+
+// Chunk row r <- H_all[rowmap[r]]: copies the residual row into the chunk's h, stores the hi/lo planes of h * gain (the
+// input of the sub-layer's first GEMM) and the row's sum of squares as "tile 0".  grid = chunk rows, block = 1024.
+__global__ void gather_norm_kernel(const int* __restrict__ rowmap, const float* __restrict__ H_all, float* __restrict__ h,
+                                   const float* __restrict__ gain, __nv_bfloat16* __restrict__ planes, float* __restrict__ sumsq_out, int d)
+{
+    __shared__ float red[33];
+    const int r = blockIdx.x;
+    const float* src = H_all + (size_t)rowmap[r] * d;
+    float ss = 0.f;
+    for (int i = threadIdx.x; i < d; i += blockDim.x) {
+        const float v = src[i];
+        h[(size_t)r * d + i] = v;
+        store_hi_lo(planes, r, d, i, v * gain[i]);
+        ss += v * v;
+    }
+    const float total = block_sum(ss, red);
+    if (threadIdx.x == 0) sumsq_out[r] = total;
+}
+
+// H_all[rowmap[r]] <- chunk row r.  grid = chunk rows.
+__global__ void scatter_rows_kernel(const int* __restrict__ rowmap, const float* __restrict__ h, float* __restrict__ H_all, int d)
+{
+    const int r = blockIdx.x;
+    float* dst = H_all + (size_t)rowmap[r] * d;
+    for (int i = threadIdx.x; i < d; i += blockDim.x) dst[i] = h[(size_t)r * d + i];
+}
+
+// out[row] = arg max of logits[row][:], lowest token id among equals.  grid = rows, block = 1024.
+__global__ void __launch_bounds__(1024) argmax_rows_kernel(const float* __restrict__ logits, int vocab, int* __restrict__ out)
+{
+    __shared__ float sv[32];
+    __shared__ int si[32];
+    const float* row = logits + (size_t)blockIdx.x * vocab;
+    float bv = -INFINITY;
+    int bi = 0x7FFFFFFF;
+    for (int i = threadIdx.x; i < vocab; i += blockDim.x) {
+        const float v = row[i];
+        if (v > bv || (v == bv && i < bi)) { bv = v; bi = i; }
+    }
+    for (int o = 16; o > 0; o >>= 1) {
+        const float ov = __shfl_xor_sync(0xFFFFFFFFu, bv, o);
+        const int oi = __shfl_xor_sync(0xFFFFFFFFu, bi, o);
+        if (ov > bv || (ov == bv && oi < bi)) { bv = ov; bi = oi; }
+    }
+    if ((threadIdx.x & 31) == 0) { sv[threadIdx.x >> 5] = bv; si[threadIdx.x >> 5] = bi; }
+    __syncthreads();
+    if (threadIdx.x < 32) {
+        bv = threadIdx.x < (blockDim.x >> 5) ? sv[threadIdx.x] : -INFINITY;
+        bi = threadIdx.x < (blockDim.x >> 5) ? si[threadIdx.x] : 0x7FFFFFFF;
+        for (int o = 16; o > 0; o >>= 1) {
+            const float ov = __shfl_xor_sync(0xFFFFFFFFu, bv, o);
+            const int oi = __shfl_xor_sync(0xFFFFFFFFu, bi, o);
+            if (ov > bv || (ov == bv && oi < bi)) { bv = ov; bi = oi; }
+        }
+        if (threadIdx.x == 0) out[blockIdx.x] = bi;
+    }
+}
+
+// counts[c] = #{ i < gamma : pred[c * gamma + i] == truth[i] } (the numerator of Eq. 3).  One thread per candidate.
+__global__ void match_rows_kernel(const int* __restrict__ pred, const int* __restrict__ truth, int gamma, int n_cand, int* __restrict__ counts)
+{
+    const int c = blockIdx.x * blockDim.x + threadIdx.x;
+    if (c >= n_cand) return;
+    int m = 0;
+    for (int i = 0; i < gamma; ++i) m += pred[c * gamma + i] == truth[i] ? 1 : 0;
+    counts[c] = m;
+}
+
+} // namespace swk

@@ -48,7 +48,7 @@ struct WeightLayout {
 };
 
 struct WorkLayout {
-    size_t state, h, xn, xa, act, q, part, o_part, ml_part, logits, q_rows, rope, pt_main, pt_score, score_tok, cand, cand_n, big_tok,
+    size_t state, h, xn, xa, act, q, part, o_part, ml_part, logits, q_rows, rope, pt_main, pt_score, score_tok, cand, cand_n, big_tok, score_H, score_logits, score_pred, score_maps, pt_slots,
         score_truth, score_out, attn_counters, xn_hl, xa_hl, act_hl, slabs, counters, sumsq, total;
     size_t part_floats, slab_floats;
 };
@@ -78,7 +78,7 @@ struct swift_ctx {
     std::string err;
     cudaEvent_t ev[8];
     // captured forwards; programmatic dependent launch between the kernels of a forward
-    bool use_graphs, use_pdl, pdl_next, pdl_gemms, fuse, fuse_combine, prefetch_next, attn_mma, big_chunks;
+    bool use_graphs, use_pdl, pdl_next, pdl_gemms, fuse, fuse_combine, prefetch_next, attn_mma, big_chunks, batched_scoring;
     int attn_rows_per_cta, prefetch_tiles;
     std::vector<FwdGraph>* graphs;
     uint64_t graph_clock;
@@ -201,11 +201,21 @@ int max_segments(int N, int K)
     return worst;
 }
 
-int scratch_pages(const swift_model_desc* d) { return MAX_SCORE_ROWS / d->page_size + 2; }
+// Scratch KV pages beyond the sequence's own: the window of one candidate (copy-on-write start page included), or the
+// windows of the several candidates of one chunk when candidates are scored side by side.
+int scratch_pages(const swift_model_desc* d) { return MAX_SCORE_ROWS / d->page_size + 8; }
 
 size_t page_bytes(const swift_model_desc* d)
 {
     return (size_t)d->n_blocks * 2 * d->n_kv_heads * d->page_size * d->head_dim * kv_esize_of(d);
+}
+
+constexpr int SCORE_ROWS_MAX = 4096;     // candidates x window rows scored side by side (beyond that: one candidate at a time)
+constexpr int SCORE_SLOTS_MAX = 8;       // candidates per chunk of TC_ROWS_MAX rows (window of 16 rows)
+// Row-map entries of one scoring round: one map of TC_ROWS_MAX rows per (sub-layer or output head, chunk of candidates).
+size_t score_map_ints(const swift_model_desc* d)
+{
+    return (size_t)(2 * d->n_blocks + 1) * (SCORE_ROWS_MAX / TC_ROWS_MAX + SCORE_ROWS_MAX / ROWS / 2) * TC_ROWS_MAX;
 }
 
 // Rows of the largest forward chunk: TC_ROWS_MAX where the tensor-core walk with many-row chunks applies, else 16.
@@ -235,6 +245,16 @@ WorkLayout work_layout(const swift_model_desc* d)
     k.o_part = c.take((size_t)d->n_heads * max_splits * RB * d->head_dim * 4);
     k.ml_part = c.take((size_t)d->n_heads * max_splits * RB * 8);
     k.big_tok = c.take(RB * 4);
+    // candidate scoring with all candidates side by side (chunks of many rows only): every candidate's window rows, one
+    // chunk of logits, the predictions, the row maps of a whole scoring round, one page table per candidate of a chunk
+    k.score_H = k.score_logits = k.score_pred = k.score_maps = k.pt_slots = 0;
+    if (RB > ROWS) {
+        k.score_H = c.take((size_t)SCORE_ROWS_MAX * dm * 4);
+        k.score_logits = c.take(RB * (size_t)d->vocab * 4);
+        k.score_pred = c.take((size_t)SCORE_ROWS_MAX * 4);
+        k.score_maps = c.take(score_map_ints(d) * 4);
+        k.pt_slots = c.take((size_t)SCORE_SLOTS_MAX * (d->max_positions / d->page_size) * 4);
+    }
     k.logits = c.take((size_t)ROWS * d->vocab * 4);
     k.q_rows = c.take((size_t)std::max(1, d->max_draft) * d->vocab * 4);
     k.rope = c.take((size_t)d->max_positions * (d->head_dim / 2) * 8);
@@ -937,8 +957,16 @@ void commit_round(swift_ctx* ctx, const DevState& hs)
 }
 
 // Scores C candidates; results (match counts) land in the score_out device array.
+template <typename TKV>
+swift_status enqueue_score_batched(swift_ctx* ctx, const uint8_t* masks, int C, int gamma);
+
 swift_status enqueue_score(swift_ctx* ctx, const uint8_t* masks, int C, int gamma)
 {
+    if (ctx->batched_scoring) {                        // all candidates side by side where the shape allows it
+        const swift_status bs = ctx->d.kv_dtype == SWIFT_BF16 ? enqueue_score_batched<__nv_bfloat16>(ctx, masks, C, gamma)
+                                                              : enqueue_score_batched<float>(ctx, masks, C, gamma);
+        if (bs != SWIFT_EUNSUPPORTED) return bs;
+    }
     const int n = ctx->n, L = 2 * ctx->d.n_blocks;
     DevState* st = state_of(ctx);
     int* tok_dev = kptr<int>(ctx, ctx->kl.score_tok);
@@ -967,6 +995,137 @@ swift_status enqueue_score(swift_ctx* ctx, const uint8_t* masks, int C, int gamm
 // Bytes one forward must move (weights of the kept sub-layers, output head, cached K,V of the kept attention
 // sub-layers, embedding rows in, logits out).  kv_elem_bytes: size of a cached K or V element to count; 0 = as stored.
 // The records of a run count 2 bytes (a 16-bit cache, what the method needs); an fp32 cache moves twice that.
+// All candidates side by side ("Parallel Candidate Evaluation", Section 4.1): every candidate keeps its own copy of the
+// window's gamma residual rows; the sub-layers are walked once, and each is applied to the candidates that keep it,
+// gathered into chunks of up to TC_ROWS_MAX rows, so its weights are streamed once per chunk of candidates instead of
+// once per 16 rows of every candidate.  Each candidate of a chunk has its own scratch KV pages for the window.  Results
+// (match counts) land in the score_out device array.  Returns SWIFT_EUNSUPPORTED when the shape does not fit this form.
+template <typename TKV>
+swift_status enqueue_score_batched(swift_ctx* ctx, const uint8_t* masks, int C, int gamma)
+{
+    typedef __nv_bfloat16 T;
+    constexpr int NB = TC_NB_MAX;
+    const swift_model_desc& d = ctx->d;
+    const int n = ctx->n, L = 2 * d.n_blocks, P = d.page_size, pos_w = n - gamma;
+    if (!ctx->big_chunks || gamma % ROWS || gamma > TC_ROWS_MAX || C * gamma > SCORE_ROWS_MAX) return SWIFT_EUNSUPPORTED;
+    const int pages_per_slot = ceil_div(gamma, P) + 1;
+    const int cpg = std::min(std::min(TC_ROWS_MAX / gamma, ctx->n_pages_scratch / pages_per_slot), (int)SCORE_SLOTS_MAX);   // candidates per chunk
+    if (cpg < 1) return SWIFT_EUNSUPPORTED;
+    // ---- row maps of the whole round: per sub-layer, the candidates that keep it in chunks of cpg; then the output head
+    struct Chunk { int sub; int n_cand; size_t map_off; };
+    std::vector<Chunk> chunks;
+    std::vector<int> maps;
+    for (int sub = 0; sub <= L; ++sub) {
+        std::vector<int> keep;
+        for (int c = 0; c < C; ++c) if (sub == L || !masks[(size_t)c * L + sub]) keep.push_back(c);
+        for (size_t g0 = 0; g0 < keep.size(); g0 += cpg) {
+            const int nc = (int)std::min<size_t>(cpg, keep.size() - g0);
+            chunks.push_back({sub, nc, maps.size()});
+            for (int j = 0; j < nc; ++j)
+                for (int i = 0; i < gamma; ++i) maps.push_back(keep[g0 + j] * gamma + i);
+            maps.resize(chunks.back().map_off + TC_ROWS_MAX, 0);
+        }
+    }
+    if (maps.size() > score_map_ints(&d)) return SWIFT_EUNSUPPORTED;
+    DevState* st = state_of(ctx);
+    int* tok_dev = kptr<int>(ctx, ctx->kl.score_tok);
+    int* truth_dev = kptr<int>(ctx, ctx->kl.score_truth);
+    int* maps_dev = kptr<int>(ctx, ctx->kl.score_maps);
+    float* H_all = kptr<float>(ctx, ctx->kl.score_H);
+    CU(copy_async(ctx, tok_dev, ctx->hist.data() + (n - gamma), (size_t)gamma * 4, cudaMemcpyHostToDevice));
+    CU(copy_async(ctx, truth_dev, ctx->hist.data() + (n - gamma + 1), (size_t)gamma * 4, cudaMemcpyHostToDevice));
+    CU(copy_async(ctx, maps_dev, maps.data(), maps.size() * 4, cudaMemcpyHostToDevice));
+    // ---- one page table per candidate slot of a chunk: the window's pages go to the slot's scratch pages
+    const int first = pos_w / P, last = (n - 1) / P, np = ctx->n_pages_main;
+    std::vector<int> pts((size_t)cpg * np);
+    for (int j = 0; j < cpg; ++j) {
+        for (int i = 0; i < np; ++i) pts[(size_t)j * np + i] = i;
+        for (int p = first; p <= last; ++p) pts[(size_t)j * np + p] = np + j * pages_per_slot + (p - first);
+    }
+    int* pt_dev = kptr<int>(ctx, ctx->kl.pt_slots);
+    CU(copy_async(ctx, pt_dev, pts.data(), pts.size() * 4, cudaMemcpyHostToDevice));
+    if (pos_w % P) {                                  // the window starts inside a page: every slot starts from a copy of it
+        const size_t v16 = page_bytes(&d) / 16;
+        for (int j = 0; j < cpg; ++j) {
+            page_copy_kernel<<<296, 256, 0, ctx->stream>>>(reinterpret_cast<uint4*>(ctx->kvbase), v16, first, np + j * pages_per_slot);
+            ctx->launches++;
+        }
+    }
+    // ---- the walk
+    const int dm = d.d_model, qd = d.n_heads * d.head_dim, kd = d.n_kv_heads * d.head_dim, nqkv = qd + 2 * kd;
+    float* h = kptr<float>(ctx, ctx->kl.h);
+    float* xa = kptr<float>(ctx, ctx->kl.xa);
+    __nv_bfloat16* xn_hl = kptr<__nv_bfloat16>(ctx, ctx->kl.xn_hl);
+    __nv_bfloat16* xa_hl = kptr<__nv_bfloat16>(ctx, ctx->kl.xa_hl);
+    __nv_bfloat16* act_hl = kptr<__nv_bfloat16>(ctx, ctx->kl.act_hl);
+    float* sumsq = kptr<float>(ctx, ctx->kl.sumsq);
+    float* logits = kptr<float>(ctx, ctx->kl.score_logits);
+    int* pred = kptr<int>(ctx, ctx->kl.score_pred);
+    EpiParams base;
+    memset(&base, 0, sizeof base);
+    base.inv_d = 1.0f / (float)dm;
+    base.eps = d.rms_eps;
+    base.sumsq_in = sumsq;
+    base.sum_rows = TC_ROWS_MAX;
+    base.n_sumsq_tiles = 1;                           // gather_norm_kernel leaves each row's sum of squares as tile 0
+    embed_rows_kernel<T><<<C * gamma, 256, 0, ctx->stream>>>(st, tok_dev, (const T*)wptr<T>(ctx, ctx->wl.embed), H_all, dm, d.vocab, gamma);
+    ctx->launches++;
+    for (const Chunk& ch : chunks) {
+        const int rows = ch.n_cand * gamma;
+        const int* map = maps_dev + ch.map_off;
+        set_rows_kernel<<<1, 1, 0, ctx->stream>>>(st, pos_w, rows);
+        ctx->launches++;
+        if (ch.sub == L) {                            // output head: final norm, logits, arg max per row
+            gather_norm_kernel<<<rows, 1024, 0, ctx->stream>>>(map, H_all, h, wptr<float>(ctx, ctx->wl.final_norm), xn_hl, sumsq, dm);
+            ctx->launches++;
+            CU(launch_k(gemm_tc_kernel<EPI_PLAIN, float, NB>, dim3(TC_GRID), dim3(TC_THREADS), (size_t)TcShape<NB>::SMEM_BYTES, ctx, st,
+                        ctx->tm_lm_head, ctx->tm_xn_big, logits, kptr<float>(ctx, ctx->kl.slabs), kptr<int>(ctx, ctx->kl.counters), d.vocab, dm,
+                        base, ctx->tm_lm_head));
+            // the head's chunks hold consecutive candidates: their predictions go where their rows are in H_all
+            argmax_rows_kernel<<<rows, 1024, 0, ctx->stream>>>(logits, d.vocab, pred + maps[ch.map_off]);
+            ctx->launches++;
+            continue;
+        }
+        const int b = ch.sub >> 1;
+        EpiParams resid = base;
+        resid.h = h;                                  // h += branch output; nothing chained: the next sub-layer regroups the rows
+        if (!(ch.sub & 1)) {
+            gather_norm_kernel<<<rows, 1024, 0, ctx->stream>>>(map, H_all, h, wptr<float>(ctx, ctx->wl.attn_norm[b]), xn_hl, sumsq, dm);
+            ctx->launches++;
+            EpiParams ep = base;
+            ep.q_out = kptr<float>(ctx, ctx->kl.q); ep.kv_pool = ctx->kvbase; ep.page_table = pt_dev; ep.L = ctx->kv;
+            ep.block = b; ep.n_heads = d.n_heads; ep.max_positions = d.max_positions; ep.rope_cs = kptr<float2>(ctx, ctx->kl.rope);
+            ep.per_block = 1;
+            for (int rb = 0; rb < NB; ++rb) {
+                const int j = std::min((rb * ROWS) / gamma, ch.n_cand - 1);
+                ep.rb_pos0[rb] = pos_w + (rb * ROWS) % gamma;
+                ep.rb_page_table[rb] = pt_dev + (size_t)j * np;
+            }
+            ST((launch_gemm_tc<EPI_QKV, TKV, NB>(ctx, GemmSite{nullptr, nqkv, dm, nullptr, &ctx->tm_wqkv[b], &ctx->tm_xn_big}, ep)));
+            for (int j = 0; j < ch.n_cand; ++j) {     // each candidate of the chunk is a sequence of its own
+                ST((launch_attn_mma<TKV, 2>(ctx, pt_dev + (size_t)j * np, b, false, xa, xa_hl, TC_ROWS_MAX, j * gamma, gamma, pos_w)));
+                CU(launch_k(attn_combine_kernel, dim3(d.n_heads, gamma), dim3(d.head_dim), 2 * (size_t)ctx->max_splits * sizeof(float), ctx,
+                            (const DevState*)st, (const float*)kptr<float>(ctx, ctx->kl.o_part), (const float2*)kptr<float2>(ctx, ctx->kl.ml_part),
+                            ctx->max_splits, d.n_heads, d.head_dim, xa, xa_hl, (int)TC_ROWS_MAX, j * gamma, gamma, pos_w));
+            }
+            ST((launch_gemm_tc<EPI_RESID, float, NB>(ctx, GemmSite{nullptr, dm, qd, nullptr, &ctx->tm_wo[b], &ctx->tm_xa_big}, resid)));
+        } else {
+            gather_norm_kernel<<<rows, 1024, 0, ctx->stream>>>(map, H_all, h, wptr<float>(ctx, ctx->wl.mlp_norm[b]), xn_hl, sumsq, dm);
+            ctx->launches++;
+            EpiParams sw = base;
+            sw.act_planes = act_hl; sw.ffn = d.ffn;
+            ST((launch_gemm_tc<EPI_SWIGLU, float, NB>(ctx, GemmSite{nullptr, 2 * d.ffn, dm, nullptr, &ctx->tm_wgu[b], &ctx->tm_xn_big}, sw)));
+            ST((launch_gemm_tc<EPI_RESID, float, NB>(ctx, GemmSite{nullptr, dm, d.ffn, nullptr, &ctx->tm_wdown[b], &ctx->tm_act_big}, resid)));
+        }
+        scatter_rows_kernel<<<rows, 256, 0, ctx->stream>>>(map, h, H_all, dm);
+        ctx->launches++;
+    }
+    match_rows_kernel<<<ceil_div(C, 128), 128, 0, ctx->stream>>>(pred, truth_dev, gamma, C, kptr<int>(ctx, ctx->kl.score_out));
+    ctx->launches++;
+    CU(cudaGetLastError());
+    return SWIFT_OK;
+}
+
 double forward_bytes(const swift_ctx* ctx, const uint8_t* skip, int n_rows, int n_context, int kv_elem_bytes = 2)
 {
     const swift_model_desc& d = ctx->d;
@@ -1019,6 +1178,7 @@ cudaError_t init_kernel_attrs()
     if (e == cudaSuccess) e = cudaFuncSetAttribute(gemm_tc_kernel<EPI_QKV, float>, cudaFuncAttributeMaxDynamicSharedMemorySize, TC_SMEM_BYTES);
     if (e == cudaSuccess) e = cudaFuncSetAttribute(gemm_tc_kernel<EPI_QKV, __nv_bfloat16>, cudaFuncAttributeMaxDynamicSharedMemorySize, TC_SMEM_BYTES);
     constexpr int big_smem = TcShape<TC_NB_MAX>::SMEM_BYTES;
+    if (e == cudaSuccess) e = cudaFuncSetAttribute(gemm_tc_kernel<EPI_PLAIN, float, TC_NB_MAX>, cudaFuncAttributeMaxDynamicSharedMemorySize, big_smem);
     if (e == cudaSuccess) e = cudaFuncSetAttribute(gemm_tc_kernel<EPI_RESID, float, TC_NB_MAX>, cudaFuncAttributeMaxDynamicSharedMemorySize, big_smem);
     if (e == cudaSuccess) e = cudaFuncSetAttribute(gemm_tc_kernel<EPI_SWIGLU, float, TC_NB_MAX>, cudaFuncAttributeMaxDynamicSharedMemorySize, big_smem);
     if (e == cudaSuccess) e = cudaFuncSetAttribute(gemm_tc_kernel<EPI_QKV, float, TC_NB_MAX>, cudaFuncAttributeMaxDynamicSharedMemorySize, big_smem);
@@ -1170,6 +1330,7 @@ swift_status swift_load(const swift_model_desc* desc, swift_devbuf weights, swif
     c->fuse = getenv("SWIFT_NO_FUSE") == nullptr && desc->head_dim <= TC_TILE_N;
     // prefill in chunks of up to TC_ROWS_MAX rows (SWIFT_NO_BIG_CHUNKS: 16 rows at a time, as decoding does)
     c->big_chunks = c->use_tc && c->fuse && big_rows_of(desc) == (size_t)TC_ROWS_MAX && getenv("SWIFT_NO_BIG_CHUNKS") == nullptr;
+    c->batched_scoring = c->big_chunks && getenv("SWIFT_NO_BATCHED_SCORING") == nullptr;
     c->graphs = new std::vector<FwdGraph>();
     c->graph_clock = 0;
     cudaError_t e = init_kernel_attrs();

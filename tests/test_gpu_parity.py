@@ -200,6 +200,18 @@ def test_benchmark_context_lengths(shape, n_prefix, max_k, attn_mma, monkeypatch
         st = walk_rounds(o, g, list(synth.block_mask(cfg, [1])), n_rounds=2, max_k=max_k)
         print(f"{shape} at {n_prefix} positions: rounds {st}")
         assert st["max_logit_err"] < LOGIT_TOL and st["rounds"] == 2, st
+        # candidate scoring at this context (Eq. 2-3): six skip sets side by side (more than one chunk of candidates), each
+        # with its own scratch pages for the 32-token window, against the oracle's one-by-one scores
+        masks = np.array([[0, 0, 0, 0], [1, 1, 0, 0], [1, 0, 0, 1], [0, 1, 1, 0], [0, 0, 1, 1], [0, 0, 0, 1]], dtype=np.uint8)
+        ref_m, _ = o.score_skipsets(masks.tolist(), 32)
+        got_m = g.score_skipsets(masks, 32)
+        for c in range(len(masks)):
+            if got_m[c] != pytest.approx(ref_m[c]):
+                win = o.forward_rows(o.tokens[o.n - 32:o.n], o.n - 32, masks[c].tolist(), write_kv=False)
+                assert min(so.top2_margin(r) for r in win) <= MARGIN and abs(got_m[c] - ref_m[c]) <= 2.0 / 32, (c, got_m[c], ref_m[c])
+        # the scratch pages left the sequence's own cache alone: the next round still follows the oracle
+        st = walk_rounds(o, g, list(synth.block_mask(cfg, [1])), n_rounds=1, max_k=max_k)
+        assert st["max_logit_err"] < LOGIT_TOL, st
     finally:
         g.close()
 
