@@ -250,6 +250,13 @@ void swift_opt_free(swift_opt* opt);
 swift_status swift_opt_suggest(swift_opt* opt, uint8_t* mask_host, int32_t* is_bayesian_host);
 swift_status swift_opt_observe(swift_opt* opt, const uint8_t* mask_host, float matchness);
 
+/* Every device-side wait of this library (on a shared-memory barrier that a bulk copy or a tensor-core instruction
+ * completes) is bounded: when its limit runs out the kernel records it, winds down and the next call that reads the
+ * control block returns SWIFT_ETIMEOUT, with the context still usable.  This call exercises exactly that path in a
+ * harmless form: one thread waits limit_us microseconds on a barrier nothing arrives on.  Returns SWIFT_ETIMEOUT
+ * (that is the expected outcome); the call after it works normally. */
+swift_status swift_probe_wait_limit(swift_ctx* ctx, int32_t limit_us);
+
 /* Selects the kernel behind the weight-streaming GEMMs: 1 = tensor cores (tcgen05 + TMA; default and
  * only sensible choice for bf16 models), 0 = the SIMT kernel (always used for fp32 models; for bf16 it
  * exists so that tests can check one kernel against the other).  No open round. */

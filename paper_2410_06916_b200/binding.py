@@ -55,7 +55,7 @@ SYMBOLS = ("swift_weights_bytes", "swift_kv_bytes", "swift_workspace_bytes", "sw
            "swift_last_error", "swift_pack_tensor", "swift_set_sampling", "swift_set_top_p", "swift_set_greedy_draft", "swift_forward_rows", "swift_prefill",
            "swift_set_pending", "swift_draft", "swift_verify", "swift_accept", "swift_score_skipsets", "swift_generate",
            "swift_committed_length", "swift_launch_count", "swift_round_times", "swift_round_bytes_stored", "swift_final_skip_mask", "swift_forward_bytes", "swift_read_kv", "swift_time_gemm", "swift_set_gemm_impl", "swift_gemm", "swift_gemm_static",
-           "swift_gemm_static_error", "swift_set_tree", "swift_verify_tree", "swift_tree_rows", "swift_opt_create", "swift_opt_free", "swift_opt_suggest", "swift_opt_observe")
+           "swift_gemm_static_error", "swift_probe_wait_limit", "swift_set_tree", "swift_verify_tree", "swift_tree_rows", "swift_opt_create", "swift_opt_free", "swift_opt_suggest", "swift_opt_observe")
 
 _lib = None
 
@@ -94,6 +94,7 @@ def load_library(path: Optional[str] = None) -> C.CDLL:
     lib.swift_final_skip_mask.restype = C.c_int32
     lib.swift_round_times.argtypes = [vp, i32, vp, vp, vp, vp, vp]
     lib.swift_round_times.restype = C.c_int32
+    lib.swift_probe_wait_limit.argtypes = [vp, i32]
     lib.swift_set_tree.argtypes = [vp, i32]
     lib.swift_verify_tree.argtypes = [vp, vp, vp, i32, vp, vp]
     lib.swift_tree_rows.argtypes = [vp, vp, vp, vp]
@@ -353,6 +354,11 @@ class SwiftModel:
         with torch.cuda.device(self.device):
             self._check(self._lib.swift_verify(self.ctx, tp, k, _ptr(am), _ptr(logits)))
         return am, logits
+
+    def probe_wait_limit(self, limit_us: int = 1000) -> None:
+        """Lets one bounded device-side wait run out (harmlessly); raises SwiftError(ETIMEOUT), after which the model works on."""
+        with torch.cuda.device(self.device):
+            self._check(self._lib.swift_probe_wait_limit(self.ctx, limit_us))
 
     def set_tree(self, tree_rows: int) -> None:
         """Dynamic verification (Section 4.2): rows one verification of the device's own drafts may hold (0 = the chain only)."""

@@ -82,7 +82,7 @@ __device__ __forceinline__ void mbar_arrive(uint32_t bar)
     asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
 }
 // Bounded wait on a phase parity.  Returns false when the limit ran out.
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity)
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, long long limit_cycles = TC_WAIT_CYCLES)
 {
     const long long t0 = clock64();
     for (uint32_t it = 0;; ++it) {
@@ -93,7 +93,7 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity)
             "selp.u32 %0, 1, 0, p;\n\t}"
             : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
         if (ok) return true;
-        if ((it & 63u) == 63u && clock64() - t0 > TC_WAIT_CYCLES) return false;
+        if ((it & 63u) == 63u && clock64() - t0 > limit_cycles) return false;
     }
 }
 __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, int c0, int c1, uint32_t bar)
@@ -748,6 +748,20 @@ gemm_tc_kernel(DevState* st, const __grid_constant__ CUtensorMap mapW, const __g
     if (warp == 1) {
         tc_fence_after();
         asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(S::TMEM_COLS));
+    }
+}
+
+// What happens when a bounded wait runs out, in its harmless form: one thread waits, with the given limit, on a barrier
+// nothing ever arrives on; the wait gives up, and the kernel reports it the way the GEMM does (the error word of the
+// control block) and returns normally.  No fault, no trap: the context stays usable.
+__global__ void wait_probe_kernel(DevState* st, long long limit_cycles)
+{
+    __shared__ __align__(8) unsigned long long bar_storage;
+    if (threadIdx.x == 0) {
+        const uint32_t bar = smem_u32(&bar_storage);
+        mbar_init(bar, 1);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        if (!mbar_wait(bar, 0, limit_cycles)) st->error = TC_ERR_TIMEOUT;
     }
 }
 

@@ -1697,6 +1697,18 @@ swift_status swift_gemm(swift_ctx* ctx, int32_t which, int32_t block, const floa
     return read_state(ctx, &hs);
 }
 
+swift_status swift_probe_wait_limit(swift_ctx* ctx, int32_t limit_us)
+{
+    if (!ctx) return SWIFT_EINVAL;
+    if (limit_us < 1 || limit_us > 100000) return fail(ctx, SWIFT_EINVAL, "limit_us must be in 1..100000");
+    if (ctx->round_open) return fail(ctx, SWIFT_ESTATE, "a round is open");
+    wait_probe_kernel<<<1, 32, 0, ctx->stream>>>(state_of(ctx), (long long)limit_us * 2000LL);   // about 2 cycles per nanosecond
+    ctx->launches++;
+    CU(cudaGetLastError());
+    DevState hs;
+    return read_state(ctx, &hs);
+}
+
 swift_status swift_set_gemm_impl(swift_ctx* ctx, int32_t impl)
 {
     if (!ctx) return SWIFT_EINVAL;

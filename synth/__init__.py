@@ -49,6 +49,8 @@ class ModelConfig:
     planted_scale: float = 0.01
     init_std: float = 0.02
     gain_std: float = 0.0  # norm gains = 1 + gain_std * N(0,1); the paper-shaped configs use 1
+    embed_std: float = 0.0      # standard deviation of the token embedding; 0 = init_std
+    branch_scale: float = 1.0   # factor on every block's residual-branch output projections (wo, wdown), planted or not
     rope_theta: float = 10000.0
     rms_eps: float = 1e-5
 
@@ -115,11 +117,20 @@ MODELS: Dict[str, ModelConfig] = {
     # a 34B-class backbone (the paper also runs 33B/34B models, Section 5.2, without giving their shapes): 60 blocks, 56 query
     # heads on 8 KV heads (7 per group, not a power of two), vocabulary 64000 (twice the others'), skip ratio 0.5
     "34b": ModelConfig("34b", 60, 7168, 56, 8, 128, 20480, 64000, "bf16", seed=12, n_planted=30),
+    # The 13B shape with layers that behave like a trained model's for the purposes of layer skipping: with N(0, 0.02)
+    # everywhere a block's output is as large as the whole residual stream, and skipping any single block that is not
+    # planted already destroys the prediction (measured: matchness <= 0.16), so no search over skip sets can be
+    # guided by matchness.  Here the token embedding carries the stream (std 0.9) and every block adds a modest
+    # increment (output projections x 0.05, planted ones x 0.01 on top): matchness then falls gradually with every
+    # non-planted block skipped, as the paper's models do.  Config 3 (on-the-fly optimisation) runs on this one.
+    "13b-graded": ModelConfig("13b-graded", 40, 5120, 40, 40, 128, 13824, 32000, "bf16", seed=3, n_planted=18,
+                              embed_std=0.9, branch_scale=0.05),
 }
 RUNS: Dict[str, Tuple[str, RunConfig]] = {
     "c1": ("tiny", RunConfig(32, 64, 4, stop_conf=0.8, n_skip_blocks=4)),
     "c2": ("7b", RunConfig(512, 256, 8, n_skip_blocks=14)),
-    "c3": ("13b", RunConfig(1024, 512, 8, n_skip_blocks=18, optimise=True)),
+    "c3": ("13b-graded", RunConfig(1024, 512, 8, n_skip_blocks=18, optimise=True)),
+    "c3-flat": ("13b", RunConfig(1024, 512, 8, n_skip_blocks=18, optimise=True)),     # the same on the all-N(0, 0.02) model
     "c3-fixed": ("13b", RunConfig(1024, 512, 8, n_skip_blocks=18)),     # config 3's shape with the planted set held fixed
     "c4": ("13b", RunConfig(1024, 512, 8, n_skip_blocks=20, mode="sampling", rng_seed=4)),
     # config 4 with the sampling setting the paper uses on code generation (Appendix B.2)
@@ -240,8 +251,11 @@ def make_tensor(cfg: ModelConfig, name: str, block: int = -1, planted: bool | No
         return 1.0 + fill(shape, cfg.seed, tid, cfg.gain_std, "f32")
     if planted is None:
         planted = block in planted_blocks(cfg)
-    s2 = cfg.planted_scale if (planted and name in ("wo", "wdown")) else 1.0
-    return fill(shape, cfg.seed, tid, cfg.init_std, cfg.dtype, s2, out=out)
+    s2 = 1.0
+    if name in ("wo", "wdown"):
+        s2 = cfg.branch_scale * (cfg.planted_scale if planted else 1.0)
+    std = cfg.embed_std if (name == "embed" and cfg.embed_std > 0.0) else cfg.init_std
+    return fill(shape, cfg.seed, tid, std, cfg.dtype, s2, out=out)
 
 
 def iter_tensors(cfg: ModelConfig) -> Iterator[Tuple[str, int, torch.Tensor]]:

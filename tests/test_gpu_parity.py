@@ -925,3 +925,28 @@ def test_config2_whole_run_against_the_oracles_trace():
         assert n_same >= 16 and checked >= 4
     finally:
         g.close()
+
+
+def test_a_wait_that_runs_out_is_a_status(small_cfg):
+    """A bounded device-side wait whose limit runs out (here: one thread waiting a millisecond on a barrier nothing arrives
+    on) comes back as SWIFT_ETIMEOUT from the call that reads the control block, and the context works on afterwards."""
+    from paper_2410_06916_b200 import SwiftError, SwiftModel
+    g = SwiftModel(small_cfg, max_positions=32, page_size=8, max_draft=4)
+    try:
+        w = synth.make_weights(small_cfg)
+        g.pack("embed", -1, w["embed"]); g.pack("lm_head", -1, w["lm_head"]); g.pack("final_norm", -1, w["final_norm"])
+        for b, wb in enumerate(w["blocks"]):
+            for name, t in wb.items():
+                g.pack(name, b, t)
+        first = g.prefill([1, 2, 3])
+        with pytest.raises(SwiftError, match="ETIMEOUT"):
+            g.probe_wait_limit(1000)
+        assert g.n == 3
+        assert g.prefill([1, 2, 3]) == first                    # the same context, the same answer
+        with pytest.raises(SwiftError, match="ETIMEOUT"):
+            g.probe_wait_limit(200)
+        toks, _ = g.draft(np.zeros(8, np.uint8), 2)
+        g.verify(); g.accept()
+        assert g.n >= 4
+    finally:
+        g.close()
