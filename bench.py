@@ -181,10 +181,10 @@ def stream_mode(model, cfg, run, z, gp, args, max_new, desc, hbm_peak):
     tot_tokens = tot_ms = van_ms = 0.0
     for i in range(args.stream):
         prompt = synth.prompt(cfg, run.prompt_len, stream=100 + i)
-        gpi = dataclasses.replace(gp, skip_mask=carry, n_opt_rounds=gp.n_opt_rounds if optimising else 0, opt_seed=gp.opt_seed + i)
+        gpi = dataclasses.replace(gp, skip_mask=carry, n_opt_rounds=gp.n_opt_rounds if optimising else 0)
         out, st, _ = model.generate(prompt, gpi)
+        carry = model.final_skip_mask()                  # (before the vanilla run, which ends with the empty set)
         van, vst, _ = model.generate(prompt, GenParams(max_new=max_new, vanilla=True))
-        carry = model.final_skip_mask()
         if st.opt_rounds > 0 and st.best_matchness > run.stop_matchness:
             optimising = False
         rows.append({"input": i, "tokens_per_s": (st.tokens - 1) / (st.ms_decode * 1e-3), "vanilla_tokens_per_s": (vst.tokens - 1) / (vst.ms_decode * 1e-3),
@@ -352,6 +352,7 @@ def main():
 
     # vanilla decoding of the same model for the comparison the metric names
     swift_tokens = model.generate(prompt, gp)[0]
+    z_final = model.final_skip_mask()
     md, mv, bd, bv, kd = model.round_times()
     sbd, sbv = model.round_bytes_stored()
     fdist = {"draft_frac": dist_of(md, bd, kd > 0), "verify_frac": dist_of(mv, bv, kd == run.max_draft)}
@@ -414,6 +415,21 @@ def main():
            "ms_prefill": s0.ms_prefill, "forwards": fw, "forwards_per_round": fdist, "forwards_per_round_stored_bytes": fdist_stored, "roofline": roofline,
            "e2e": {"value": e2e, "unit": UNIT, "h2d_bytes_per_step": s0.h2d_bytes, "d2h_bytes_per_step": s0.d2h_bytes},
            "gpu_launches": launches, "clocks": clk.summary()}
+
+    # Dynamic verification (Section 4.2): the same run with the skip set the main run ended with, verifying the chain alone
+    # and verifying a token tree of up to 16 rows (greedy decoding only)
+    if not sampling and run.max_draft > 0:
+        import dataclasses
+        gp_fix = dataclasses.replace(gp, skip_mask=z_final, n_opt_rounds=0)
+        c_tok, c_st, _ = model.generate(prompt, gp_fix)
+        model.set_tree(16)
+        t_tok, t_st, _ = model.generate(prompt, gp_fix)
+        model.set_tree(0)
+        out["dynamic_verification"] = {
+            "tree_rows": 16, "M_chain": (c_st.tokens - 1) / c_st.rounds, "M_tree": (t_st.tokens - 1) / t_st.rounds,
+            "tokens_per_s_chain": (c_st.tokens - 1) / (c_st.ms_decode * 1e-3), "tokens_per_s_tree": (t_st.tokens - 1) / (t_st.ms_decode * 1e-3),
+            "alpha_chain": c_st.accepted / max(c_st.drafted, 1), "tree_equals_vanilla": t_tok == v_tokens,
+            "tokens_differing_from_vanilla": sum(int(a != b) for a, b in zip(t_tok, v_tokens))}
 
     # Candidate scoring (Eq. 2-3), for every shape: one round of the workload's candidate count on the last gamma generated
     # tokens of the run that just ended, timed with CUDA events on the library's stream.  Bytes: what the method needs if

@@ -215,7 +215,9 @@ typedef struct {
     /* candidate_masks == NULL with n_opt_rounds > 0: the library proposes the candidates itself ("Efficient Layer Set
      * Suggestion", Section 4.1): sets of opt_skip_blocks whole blocks, uniformly random except every opt_beta-th
      * proposal (counted over the whole run), which maximises the upper confidence bound of a Gaussian-process model of
-     * the scores seen so far (opt_beta 0 = random search only; the paper uses 25).  Seeded by opt_seed. */
+     * the scores seen so far (opt_beta 0 = random search only; the paper uses 25).  Seeded by opt_seed.  The engine and
+     * what it has learnt stay with the context across calls (a stream of inputs keeps optimising one model of the
+     * scores); calling with another opt_skip_blocks, opt_beta or opt_seed starts afresh. */
     int32_t opt_skip_blocks, opt_beta;
     uint64_t opt_seed;
     const uint8_t* skip_mask;       /* host, [2*n_blocks]: the (initial) draft skip set */

@@ -607,19 +607,23 @@ class LayerSetOptimizer:
     The paper delegates that part to a third-party package and prints no formulas; this is the textbook form:
 
       * a set is its indicator vector x in {0,1}^n_blocks; the squared distance of two sets is their Hamming distance;
-      * prior: zero-mean GP on standardised scores, Matern-5/2 covariance k(d) = (1 + s + s^2/3) exp(-s), s = sqrt(5) d / ell,
-        observation noise `noise`; ell is the one of `ells` with the highest marginal likelihood;
-      * posterior mean and variance by a Cholesky factorisation of K + noise * I;
-      * acquisition mu + kappa * sigma, maximised over a pool: `pool` random sets plus every set one swap away from the
-        best set seen; sets already evaluated are left out.
+      * mean function: ridge regression of the standardised scores on the indicators, w = (X^T X + ridge I)^-1 X^T t, over
+        all evaluated sets (how much each block costs when skipped: the additive part of matchness);
+      * on the residuals of the `gp_window` most recent evaluations: zero-mean GP, Matern-5/2 covariance
+        k(d) = (1 + s + s^2/3) exp(-s), s = sqrt(5) d / ell, observation noise `noise`; ell is the one of `ells` with the
+        highest marginal likelihood; posterior mean and variance by a Cholesky factorisation of K + noise * I;
+      * acquisition mu + kappa * sigma, maximised over a pool: `pool` random sets, every set one swap away from the best
+        set seen, the m blocks with the smallest regression cost, and every set one swap away from that; sets already
+        evaluated are left out.
 
     Random draws come from Philox4x32-10 keyed by `seed`: counter (index, 0, stream, 0x4F5054), one word per draw.
     """
 
     def __init__(self, n_blocks: int, m: int, beta: int = 25, seed: int = 0, pool: int = 512, kappa: float = 2.576,
-                 noise: float = 1e-2, ells: Sequence[float] = (1.0, 2.0, 4.0)):
+                 noise: float = 1e-2, ells: Sequence[float] = (1.0, 2.0, 4.0), ridge: float = 1.0, gp_window: int = 256):
         assert 0 < m < n_blocks
         self.nb, self.m, self.beta, self.seed, self.pool, self.kappa, self.noise, self.ells = n_blocks, m, beta, seed, pool, kappa, noise, tuple(ells)
+        self.ridge, self.gp_window = ridge, gp_window
         self.step = 0                       # optimisation steps taken (= proposals made)
         self.draws = 0                      # random words consumed
         self.X: List[Tuple[int, ...]] = []  # evaluated sets (sorted block tuples) ...
@@ -656,21 +660,24 @@ class LayerSetOptimizer:
     def fit(self):
         """Standardises the scores and picks ell by marginal likelihood.  Returns what predict() needs."""
         import numpy as np
-        X = self._indicator(self.X)
+        Xall = self._indicator(self.X)
         y = np.asarray(self.y, dtype=np.float64)
         mu, sd = y.mean(), y.std()
         sd = sd if sd > 1e-12 else 1.0
-        t = (y - mu) / sd
+        t_all = (y - mu) / sd
+        w = np.linalg.solve(Xall.T @ Xall + self.ridge * np.eye(self.nb), Xall.T @ t_all)     # mean function
+        X = Xall[-self.gp_window:]
+        t = (t_all - Xall @ w)[-self.gp_window:]                                              # the GP models what is left
         d2 = (X[:, None, :] != X[None, :, :]).sum(-1).astype(np.float64)
         best = None
         for ell in self.ells:
-            K = self.matern52(d2, ell) + self.noise * np.eye(len(y))
+            K = self.matern52(d2, ell) + self.noise * np.eye(len(t))
             Lc = np.linalg.cholesky(K)
             a = np.linalg.solve(Lc.T, np.linalg.solve(Lc, t))
-            lml = -0.5 * float(t @ a) - float(np.log(np.diag(Lc)).sum()) - 0.5 * len(y) * math.log(2.0 * math.pi)
+            lml = -0.5 * float(t @ a) - float(np.log(np.diag(Lc)).sum()) - 0.5 * len(t) * math.log(2.0 * math.pi)
             if best is None or lml > best[0]:
                 best = (lml, ell, Lc, a)
-        return {"X": X, "mu": mu, "sd": sd, "ell": best[1], "L": best[2], "alpha": best[3], "lml": best[0]}
+        return {"X": X, "mu": mu, "sd": sd, "ell": best[1], "L": best[2], "alpha": best[3], "lml": best[0], "w": w, "resid": t}
 
     def predict(self, model, sets):
         """Posterior mean and standard deviation of matchness at `sets` (in matchness units)."""
@@ -678,7 +685,7 @@ class LayerSetOptimizer:
         Z = self._indicator(sets)
         d2 = (Z[:, None, :] != model["X"][None, :, :]).sum(-1).astype(np.float64)
         Ks = self.matern52(d2, model["ell"])
-        mean = Ks @ model["alpha"]
+        mean = Z @ model["w"] + Ks @ model["alpha"]
         v = np.linalg.solve(model["L"], Ks.T)
         var = np.maximum(1.0 - (v * v).sum(0), 0.0)
         return model["mu"] + model["sd"] * mean, model["sd"] * np.sqrt(var)
@@ -694,17 +701,27 @@ class LayerSetOptimizer:
         """The unevaluated set with the highest mu + kappa * sigma among `pool` random sets and the one-swap
         neighbours of the best set seen (pool order, earliest among equals)."""
         cand: List[Tuple[int, ...]] = [self.random_set() for _ in range(self.pool)]
-        inc = self.best_set()
-        if inc is not None:
-            outside = [b for b in range(self.nb) if b not in inc]
-            for out_b in inc:
+
+        def with_swaps(base):
+            out = [tuple(base)]
+            outside = [b for b in range(self.nb) if b not in base]
+            for out_b in base:
                 for in_b in outside:
-                    cand.append(tuple(sorted((set(inc) - {out_b}) | {in_b})))
+                    out.append(tuple(sorted((set(base) - {out_b}) | {in_b})))
+            return out
+
+        inc = self.best_set()
+        model = self.fit() if self.X else None
+        if inc is not None:
+            cand += with_swaps(inc)[1:]
+            # the m blocks that cost least to skip according to the regression: largest weights, compared to six decimals
+            # (blocks that were always skipped together get the same weight up to rounding), lowest index among equals
+            order = sorted(range(self.nb), key=lambda b: (-math.floor(float(model["w"][b]) * 1e6 + 0.5), b))
+            cand += with_swaps(tuple(sorted(order[:self.m])))
         seen = set(self.X)
         cand = [c for c in dict.fromkeys(cand) if c not in seen]
         if not cand or not self.X:
             return (cand[0] if cand else self.random_set()), {}
-        model = self.fit()
         mean, std = self.predict(model, cand)
         ucb = mean + self.kappa * std
         i = max(range(len(cand)), key=lambda j: (float(ucb[j]), -j))

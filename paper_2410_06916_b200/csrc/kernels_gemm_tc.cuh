@@ -143,6 +143,7 @@ __device__ __forceinline__ void touch_global(const void* p)
     unsigned v;
     const unsigned long long a = reinterpret_cast<unsigned long long>(p) & ~3ull;   // the word that holds *p
     asm volatile("ld.global.cg.b32 %0, [%1];" : "=r"(v) : "l"(a) : "memory");
+    (void)v;
 }
 
 __device__ __forceinline__ int ld_acquire_gpu(const int* p)

@@ -3,11 +3,13 @@
 // optimisation) proposal every beta-th step.  Plain C++, no device code.
 //
 // The paper leaves the Bayesian step to a third-party package; this is the textbook form.  A set is its indicator
-// vector, the squared distance of two sets their Hamming distance.  Scores are standardised; the prior is a
-// zero-mean GP with Matern-5/2 covariance k(d) = (1 + s + s^2/3) exp(-s), s = sqrt(5) d / ell, plus observation
-// noise; ell is the candidate length scale with the highest marginal likelihood; the posterior comes from a
-// Cholesky factorisation; the proposal is the unevaluated set with the highest mean + kappa * deviation among a
-// pool of random sets and all sets one swap away from the best set seen.  Random draws are Philox4x32-10 words.
+// vector, the squared distance of two sets their Hamming distance.  Scores are standardised.  Mean function: ridge
+// regression of the scores on the indicators over all evaluated sets (what each block costs when skipped).  On the
+// residuals of the most recent evaluations: a zero-mean GP with Matern-5/2 covariance
+// k(d) = (1 + s + s^2/3) exp(-s), s = sqrt(5) d / ell, plus observation noise; ell is the candidate length scale with the
+// highest marginal likelihood; the posterior comes from a Cholesky factorisation.  The proposal is the unevaluated set with
+// the highest mean + kappa * deviation among a pool: random sets, all sets one swap away from the best set seen, the m
+// blocks with the smallest regression cost and all sets one swap away from that.  Random draws are Philox4x32-10 words.
 #pragma once
 #include <algorithm>
 #include <cmath>
@@ -38,6 +40,7 @@ typedef std::vector<int> BlockSet;   // sorted block indices
 struct GpModel {
     std::vector<BlockSet> X;
     std::vector<double> L, alpha;    // Cholesky factor (row-major lower triangle, n x n) and K^-1 t
+    std::vector<double> w;           // mean function: regression weight of every block
     double mu = 0.0, sd = 1.0, ell = 1.0, lml = 0.0;
     int n = 0;
 };
@@ -51,6 +54,8 @@ public:
     uint64_t seed;
     double kappa, noise;
     std::vector<double> ells = {1.0, 2.0, 4.0};
+    double ridge = 1.0;              // regularisation of the mean function
+    int gp_window = 256;             // the GP sees the residuals of this many most recent evaluations
     long long step = 0;              // proposals made
     uint64_t draws = 0;              // random words consumed
     std::vector<BlockSet> X;         // evaluated sets ...
@@ -115,18 +120,48 @@ public:
 
 inline GpModel LayerOpt::fit() const
 {
-    const int n = (int)y.size();
+    const int n_all = (int)y.size();
     GpModel best;
     double mu = 0.0, var = 0.0;
     for (double v : y) mu += v;
-    mu /= n;
+    mu /= n_all;
     for (double v : y) var += (v - mu) * (v - mu);
-    double sd = std::sqrt(var / n);
+    double sd = std::sqrt(var / n_all);
     if (sd <= 1e-12) sd = 1.0;
+    std::vector<double> t_all(n_all);
+    for (int i = 0; i < n_all; ++i) t_all[i] = (y[i] - mu) / sd;
+    // mean function: (X^T X + ridge I) w = X^T t over all evaluations, by Cholesky of the n_blocks x n_blocks matrix
+    std::vector<double> A((size_t)nb * nb, 0.0), w(nb, 0.0);
+    for (int i = 0; i < n_all; ++i)
+        for (int p : X[i]) {
+            w[p] += t_all[i];
+            for (int q : X[i]) A[(size_t)p * nb + q] += 1.0;
+        }
+    for (int p = 0; p < nb; ++p) A[(size_t)p * nb + p] += ridge;
+    for (int i = 0; i < nb; ++i)
+        for (int j = 0; j <= i; ++j) {
+            double acc = A[(size_t)i * nb + j];
+            for (int k = 0; k < j; ++k) acc -= A[(size_t)i * nb + k] * A[(size_t)j * nb + k];
+            A[(size_t)i * nb + j] = i == j ? std::sqrt(acc) : acc / A[(size_t)j * nb + j];
+        }
+    for (int i = 0; i < nb; ++i) {
+        for (int k = 0; k < i; ++k) w[i] -= A[(size_t)i * nb + k] * w[k];
+        w[i] /= A[(size_t)i * nb + i];
+    }
+    for (int i = nb - 1; i >= 0; --i) {
+        for (int k = i + 1; k < nb; ++k) w[i] -= A[(size_t)k * nb + i] * w[k];
+        w[i] /= A[(size_t)i * nb + i];
+    }
+    // the GP models the residuals of the most recent evaluations
+    const int n = std::min(n_all, gp_window), first = n_all - n;
     std::vector<double> t(n), d2((size_t)n * n);
-    for (int i = 0; i < n; ++i) t[i] = (y[i] - mu) / sd;
+    for (int i = 0; i < n; ++i) {
+        double r = t_all[first + i];
+        for (int p : X[first + i]) r -= w[p];
+        t[i] = r;
+    }
     for (int i = 0; i < n; ++i)
-        for (int j = 0; j <= i; ++j) d2[(size_t)i * n + j] = hamming(X[i], X[j]);
+        for (int j = 0; j <= i; ++j) d2[(size_t)i * n + j] = hamming(X[first + i], X[first + j]);
     bool have = false;
     for (double ell : ells) {
         std::vector<double> Lc((size_t)n * n, 0.0);
@@ -160,7 +195,8 @@ inline GpModel LayerOpt::fit() const
             best.L.swap(Lc); best.alpha.swap(a); best.ell = ell; best.lml = lml;
         }
     }
-    best.X = X; best.mu = mu; best.sd = sd; best.n = have ? n : 0;
+    best.X.assign(X.begin() + first, X.end());
+    best.w = w; best.mu = mu; best.sd = sd; best.n = have ? n : 0;
     return best;
 }
 
@@ -177,6 +213,7 @@ inline void LayerOpt::predict(const GpModel& g, const BlockSet& s, double* mean,
         v[i] = acc / g.L[(size_t)i * n + i];
         q += v[i] * v[i];
     }
+    for (int p : s) mu += g.w[p];                     // mean function
     *mean = g.mu + g.sd * mu;
     *dev = g.sd * std::sqrt(std::max(1.0 - q, 0.0));
 }
@@ -185,28 +222,40 @@ inline BlockSet LayerOpt::bayesian_set(double* ucb_out)
 {
     std::vector<BlockSet> cand;
     for (int i = 0; i < pool; ++i) cand.push_back(random_set());
-    const int bi = best_index();
-    if (bi >= 0) {
-        const BlockSet inc = X[bi];
+    auto add_swaps = [&](const BlockSet& base) {      // every set one swap away from `base`
         std::vector<int> outside;
-        for (int b = 0; b < nb; ++b) if (!std::binary_search(inc.begin(), inc.end(), b)) outside.push_back(b);
-        for (int out_b : inc)
+        for (int b = 0; b < nb; ++b) if (!std::binary_search(base.begin(), base.end(), b)) outside.push_back(b);
+        for (int out_b : base)
             for (int in_b : outside) {
                 BlockSet s;
-                for (int b : inc) if (b != out_b) s.push_back(b);
+                for (int b : base) if (b != out_b) s.push_back(b);
                 s.push_back(in_b);
                 std::sort(s.begin(), s.end());
                 cand.push_back(s);
             }
+    };
+    const int bi = best_index();
+    GpModel g;
+    if (!X.empty()) g = fit();
+    if (bi >= 0) {
+        add_swaps(X[bi]);
+        // the m blocks that cost least to skip according to the regression: largest weights, compared to six decimals
+        // (blocks that were always skipped together get the same weight up to rounding), lowest index among equals
+        std::vector<int> order(nb);
+        std::vector<long long> key(nb);
+        for (int b = 0; b < nb; ++b) { order[b] = b; key[b] = (long long)std::floor(g.w[b] * 1e6 + 0.5); }
+        std::stable_sort(order.begin(), order.end(), [&](int p, int q) { return key[p] > key[q]; });
+        BlockSet cheapest(order.begin(), order.begin() + m);
+        std::sort(cheapest.begin(), cheapest.end());
+        cand.push_back(cheapest);
+        add_swaps(cheapest);
     }
     std::set<BlockSet> seen(X.begin(), X.end());      // leave out evaluated sets and repeats, keeping pool order
     std::vector<BlockSet> fresh;
     for (const BlockSet& c : cand)
         if (seen.insert(c).second) fresh.push_back(c);
     if (fresh.empty()) return random_set();
-    if (X.empty()) return fresh[0];
-    const GpModel g = fit();
-    if (g.n == 0) return fresh[0];
+    if (X.empty() || g.n == 0) return fresh[0];
     int pick = 0;
     double best = 0.0;
     for (size_t i = 0; i < fresh.size(); ++i) {

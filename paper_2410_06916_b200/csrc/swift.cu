@@ -72,6 +72,7 @@ struct swift_ctx {
     bool round_open;
     std::vector<int> hist;           // prompt + generated tokens, pending included
     int mode; float temperature, top_p; uint64_t seed; bool greedy_draft;
+    swopt::LayerOpt* engine;         // proposal engine of swift_generate's own optimisation, kept across calls
     int tree_rows;                   // dynamic verification: rows one verification may hold (0 = off)
     DevState last_state;             // control block as last read back
     int64_t launches, h2d_bytes, d2h_bytes;
@@ -1291,7 +1292,7 @@ swift_status swift_load(const swift_model_desc* desc, swift_devbuf weights, swif
     c->max_splits = ceil_div(desc->max_positions, ATTN_CHUNK);
     c->phase = PH_LOADED; c->n = 0; c->pending = 0; c->n_prompt = 0; c->round = 0; c->last_k = 0; c->last_max_k = 0;
     c->round_open = false;
-    c->mode = SWIFT_GREEDY; c->temperature = 1.f; c->top_p = 1.f; c->greedy_draft = false; c->seed = 0; c->tree_rows = 0; memset(&c->last_state, 0, sizeof(DevState)); c->launches = 0; c->h2d_bytes = 0; c->d2h_bytes = 0;
+    c->mode = SWIFT_GREEDY; c->temperature = 1.f; c->top_p = 1.f; c->greedy_draft = false; c->seed = 0; c->engine = nullptr; c->tree_rows = 0; memset(&c->last_state, 0, sizeof(DevState)); c->launches = 0; c->h2d_bytes = 0; c->d2h_bytes = 0;
     ctx = c;
     c->use_tc = false;
     if (desc->dtype == SWIFT_BF16) {
@@ -1366,6 +1367,7 @@ swift_status swift_free(swift_ctx* ctx)
     for (auto& ev : ctx->ev) if (ev) cudaEventDestroy(ev);
     for (auto& g : *ctx->graphs) cudaGraphExecDestroy(g.exec);
     delete ctx->graphs;
+    delete ctx->engine;
     delete ctx;
     return SWIFT_OK;
 }
@@ -1927,8 +1929,17 @@ swift_status swift_generate(swift_ctx* ctx, const swift_gen_params* gp, const in
     std::vector<uint8_t> round_masks;
     int stale_rounds = 0;
     // proposals come from the caller, or from the library's own engine (random search + Gaussian-process step)
-    swopt::LayerOpt engine(d.n_blocks, std::max(1, std::min(d.n_blocks - 1, gp->opt_skip_blocks)), gp->opt_beta, gp->opt_seed);
+    // The engine and everything it has learnt stay with the context from one call to the next (the paper optimises over a
+    // stream of inputs, Section 4.1's timeline); other settings (blocks to skip, beta, seed) start a new one.
     const bool own_proposals = !gp->vanilla && gp->n_opt_rounds > 0 && !gp->candidate_masks;
+    if (own_proposals) {
+        const int m_skip = std::max(1, std::min(d.n_blocks - 1, gp->opt_skip_blocks));
+        if (!ctx->engine || ctx->engine->m != m_skip || ctx->engine->beta != gp->opt_beta || ctx->engine->seed != gp->opt_seed) {
+            delete ctx->engine;
+            ctx->engine = new swopt::LayerOpt(d.n_blocks, m_skip, gp->opt_beta, gp->opt_seed);
+        }
+    }
+    swopt::LayerOpt* engine_p = ctx->engine;
     DevState hs;
     while (count < gp->max_new) {
         const int remaining = gp->max_new - count;
@@ -1964,7 +1975,7 @@ swift_status swift_generate(swift_ctx* ctx, const swift_gen_params* gp, const in
                 round_masks.resize((size_t)n_scored * L);
                 memcpy(round_masks.data(), z.data(), L);
                 if (own_proposals)
-                    for (int c = 0; c < gp->n_candidates; ++c) blocks_to_mask(engine.suggest(), d.n_blocks, round_masks.data() + (size_t)(c + 1) * L);
+                    for (int c = 0; c < gp->n_candidates; ++c) blocks_to_mask(engine_p->suggest(), d.n_blocks, round_masks.data() + (size_t)(c + 1) * L);
                 else
                     memcpy(round_masks.data() + L, gp->candidate_masks + (size_t)stt.opt_rounds * gp->n_candidates * L, (size_t)gp->n_candidates * L);
                 const uint8_t* masks = round_masks.data();
@@ -1978,7 +1989,7 @@ swift_status swift_generate(swift_ctx* ctx, const swift_gen_params* gp, const in
                 stt.ms_score += ms;
                 if (own_proposals)                  // every score of the round goes into the Gaussian-process model
                     for (int c = 0; c < n_scored; ++c)
-                        engine.observe(mask_to_blocks(masks + (size_t)c * L, d.n_blocks), (double)counts[c] / (double)gp->gamma);
+                        engine_p->observe(mask_to_blocks(masks + (size_t)c * L, d.n_blocks), (double)counts[c] / (double)gp->gamma);
                 int cb = 0;
                 for (int c = 1; c < n_scored; ++c) if (counts[c] > counts[cb]) cb = c;   // strictly better only: the set in use wins ties
                 stt.best_matchness = (float)counts[cb] / (float)gp->gamma;

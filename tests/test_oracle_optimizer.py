@@ -41,11 +41,30 @@ def test_gaussian_process_matches_scikit_learn(ell):
     mean, std = opt.predict(model, probe)
     X = opt._indicator(opt.X)
     y = np.asarray(opt.y)
-    gp = GaussianProcessRegressor(kernel=Matern(length_scale=ell, nu=2.5), alpha=1e-2, optimizer=None, normalize_y=True)
-    gp.fit(X, y)                                        # Euclidean distance of indicator vectors = sqrt(Hamming distance)
-    ref_mean, ref_std = gp.predict(opt._indicator(probe), return_std=True)
-    assert np.allclose(mean, ref_mean, atol=1e-9) and np.allclose(std, ref_std, atol=1e-7)
+    # mean function: ridge regression of the standardised scores on the indicators, here by an augmented least-squares solve
+    t = (y - y.mean()) / y.std()
+    w = np.linalg.lstsq(np.vstack([X, np.sqrt(opt.ridge) * np.eye(12)]), np.concatenate([t, np.zeros(12)]), rcond=None)[0]
+    assert np.allclose(model["w"], w, atol=1e-10)
+    # the Gaussian process models the residuals (all 30 evaluations fit its window)
+    gp = GaussianProcessRegressor(kernel=Matern(length_scale=ell, nu=2.5), alpha=1e-2, optimizer=None, normalize_y=False)
+    gp.fit(X, t - X @ w)                                # Euclidean distance of indicator vectors = sqrt(Hamming distance)
+    P = opt._indicator(probe)
+    ref_mean, ref_std = gp.predict(P, return_std=True)
+    assert np.allclose(mean, y.mean() + y.std() * (P @ w + ref_mean), atol=1e-9) and np.allclose(std, y.std() * ref_std, atol=1e-7)
     assert model["lml"] == pytest.approx(gp.log_marginal_likelihood_value_, abs=1e-8)
+
+
+def test_gaussian_process_window_takes_the_most_recent_evaluations():
+    opt = so.LayerSetOptimizer(12, 5, seed=4, gp_window=10, ells=(2.0,))
+    f = _planted_objective({0, 2, 4, 6, 8}, 5)
+    for _ in range(25):
+        s = opt.random_set()
+        opt.observe(s, f(s))
+    model = opt.fit()
+    assert model["X"].shape == (10, 12) and np.array_equal(model["X"], opt._indicator(opt.X[-10:]))
+    y = np.asarray(opt.y)
+    t = (y - y.mean()) / y.std()
+    assert np.allclose(model["resid"], (t - opt._indicator(opt.X) @ model["w"])[-10:])
 
 
 def test_length_scale_is_chosen_by_marginal_likelihood():
@@ -82,6 +101,8 @@ def test_every_beta_th_step_is_bayesian_and_maximises_the_bound():
     inc = opt.best_set()
     swaps = {tuple(sorted((set(inc) - {a}) | {b})) for a in inc for b in range(16) if b not in inc}
     assert swaps - set(opt.X) <= set(info["candidates"])                           # every one-swap neighbour is considered
+    cheapest = tuple(sorted(sorted(range(16), key=lambda b: (-round(float(info["model"]["w"][b]), 6), b))[:6]))
+    assert cheapest in set(info["candidates"]) | set(opt.X)                        # and the regression's own best guess
 
 
 def test_finds_a_planted_set_that_random_search_misses():
@@ -97,6 +118,6 @@ def test_finds_a_planted_set_that_random_search_misses():
         if f(s) >= 0.9 and best_at is None:
             best_at = step
             break
-    assert best_at is not None and best_at <= 600, best_at
+    assert best_at is not None and best_at <= 300, best_at
     rs = so.LayerSetOptimizer(40, 18, beta=0, seed=0)
     assert max(f(rs.suggest()) for _ in range(1000)) < 0.9
