@@ -248,7 +248,9 @@ def main():
     sampling = run.mode == "sampling"
     desc = (f"{args.workload}: {cfg.name}-shaped decoder ({cfg.n_blocks} blocks, d {cfg.d_model}, {cfg.dtype}), "
             f"prompt {run.prompt_len}, {max_new} {run.mode} tokens, {run.n_skip_blocks} blocks skipped, max draft {run.max_draft}"
-            + (f", temperature {run.temperature}, top_p {run.top_p}" if sampling and (run.temperature != 1.0 or run.top_p != 1.0) else ""))
+            + (f", temperature {run.temperature}, top_p {run.top_p}" if sampling and (run.temperature != 1.0 or run.top_p != 1.0) else "")
+            + (f", on-the-fly optimisation ({run.n_candidates} proposals per round, at most {run.max_opt_rounds} rounds per input); the steps "
+               "form a stream: skip set and proposal engine carry over from step to step, warm-up steps included" if run.optimise else ""))
 
     if args.impl == "reference":
         if rank != 0:
@@ -324,15 +326,32 @@ def main():
             dist.barrier()
         torch.cuda.synchronize()
 
+    # With on-the-fly optimisation the steps form a stream, as in the paper (the optimisation phase runs until it has
+    # converged and its cost is spread over the inputs that follow): a step starts from the skip set the previous step
+    # ended with, the library's proposal engine keeps what it has learnt, and once a step ends with its set above the
+    # matchness threshold the later steps use that set as it is.  The warm-up steps are the first inputs of that stream.
+    import dataclasses
+    opt_log = []
+
+    def one_step():
+        nonlocal gp
+        tok, st, _ = model.generate(prompt, gp)
+        if run.optimise:
+            opt_log.append({"opt_rounds": st.opt_rounds, "best_matchness": st.best_matchness, "ms_score": st.ms_score,
+                            "tokens_per_s": (st.tokens - 1) / (st.ms_decode * 1e-3), "alpha": st.accepted / max(st.drafted, 1)})
+            done = st.opt_rounds > 0 and st.best_matchness > run.stop_matchness
+            gp = dataclasses.replace(gp, skip_mask=model.final_skip_mask(), n_opt_rounds=0 if (done or gp.n_opt_rounds == 0) else gp.n_opt_rounds)
+        return st
+
     for _ in range(args.warmup):
-        model.generate(prompt, gp)
+        one_step()
     launches0 = model.launches
     stats = []
     barrier()
     with ClockSampler(local) as clk:
         t0 = time.perf_counter()
         for _ in range(args.steps):
-            stats.append(model.generate(prompt, gp)[1])
+            stats.append(one_step())
         torch.cuda.synchronize()
         wall = time.perf_counter() - t0
     barrier()
@@ -450,6 +469,14 @@ def main():
     out["scoring"] = {"candidates_per_round": n_cand, "gamma": run.gamma, "ms_per_round": ms_round, "gbs": sc_gbs,
                       "frac": sc_gbs / hbm_peak, "bound": "hbm (weights streamed once per candidate)",
                       "vs_one_vanilla_step": ms_round / (1e3 / vanilla)}
+    if run.optimise:
+        # the optimisation phase as it went over the warm-up and timed steps (step 0 is config 3 as written: one input,
+        # from the uniform pattern, its optimisation rounds inside its decode time)
+        out["optimisation"] = {"steps": opt_log, "rounds_total": sum(x["opt_rounds"] for x in opt_log),
+                               "converged_at_step": next((i for i, x in enumerate(opt_log) if x["best_matchness"] > run.stop_matchness), None),
+                               "first_step_tokens_per_s": opt_log[0]["tokens_per_s"] if opt_log else None,
+                               "skipped_blocks": [int(b) for b in range(cfg.n_blocks) if z_final[2 * b] and z_final[2 * b + 1]],
+                               "planted_blocks": synth.planted_blocks(cfg)}
     if run.optimise and s0.opt_rounds > 0:
         out["scoring"].update({"opt_rounds": s0.opt_rounds, "ms_per_round_in_run": s0.ms_score / s0.opt_rounds,
                                "best_matchness": s0.best_matchness, "share_of_decode": s0.ms_score / s0.ms_decode})
