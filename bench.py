@@ -250,7 +250,7 @@ def main():
             f"prompt {run.prompt_len}, {max_new} {run.mode} tokens, {run.n_skip_blocks} blocks skipped, max draft {run.max_draft}"
             + (f", temperature {run.temperature}, top_p {run.top_p}" if sampling and (run.temperature != 1.0 or run.top_p != 1.0) else "")
             + (f", on-the-fly optimisation ({run.n_candidates} proposals per round, at most {run.max_opt_rounds} rounds per input); the steps "
-               "form a stream: skip set and proposal engine carry over from step to step, warm-up steps included" if run.optimise else ""))
+               "form a stream of different inputs: skip set and proposal engine carry over from step to step, warm-up steps included" if run.optimise else ""))
 
     if args.impl == "reference":
         if rank != 0:
@@ -334,7 +334,9 @@ def main():
     opt_log = []
 
     def one_step():
-        nonlocal gp
+        nonlocal gp, prompt
+        if run.optimise:                                     # every step of the stream is another input
+            prompt = synth.prompt(cfg, run.prompt_len, stream=1000 * rank + len(opt_log))
         tok, st, _ = model.generate(prompt, gp)
         if run.optimise:
             opt_log.append({"opt_rounds": st.opt_rounds, "best_matchness": st.best_matchness, "ms_score": st.ms_score,
@@ -414,7 +416,7 @@ def main():
     achieved = g_bytes / (g_ms * 1e-3) * 1e-9
     # DRAM bytes per launch of that kernel (read + write, mean of two launches) from the ncu captures summarised in
     # the profiles folder (7B and 13B widths, 9 rows); other shapes have no capture of their own
-    traffic = profile_traffic(cfg.name, run.max_draft + 1)
+    traffic = profile_traffic(cfg.name.split("-")[0], run.max_draft + 1)        # keyed by the widths (13b-graded has the 13b shapes)
     roofline = {"bound": "hbm", "kernel": "skinny GEMM, fused gate/up projection, %d rows" % (run.max_draft + 1),
                 "achieved": achieved, "peak": hbm_peak, "peak_kind": f"{peak_kind} copy bandwidth (burst)", "unit": "GB/s",
                 "frac": achieved / hbm_peak, "traffic": traffic, "bytes_per_launch": g_bytes, "ms_per_launch": g_ms,
