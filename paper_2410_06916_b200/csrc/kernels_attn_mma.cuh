@@ -122,9 +122,18 @@ attn_mma_kernel(const DevState* st, const float* __restrict__ q, const T* __rest
     }
 
     const int n_pass = (R + QR - 1) / QR;
+    // gridDim.z > 1: the passes are spread over the grid's z dimension, one per CTA (chunks of many rows: the first
+    // chunks of a prompt have few K,V chunks and would otherwise leave most SMs idle)
+    const int pass_begin = gridDim.z > 1 ? (int)blockIdx.z : 0;
+    const int pass_end = gridDim.z > 1 ? min(n_pass, (int)blockIdx.z + 1) : n_pass;
 #pragma unroll 1
-    for (int pass = 0; pass < n_pass; ++pass) {
+    for (int pass = pass_begin; pass < pass_end; ++pass) {
         const int rho0 = pass * QR;
+        {   // a pass none of whose rows sees this chunk yet (causal order) has nothing to add: the merge never reads it
+            const int rho1 = min(R, rho0 + QR) - 1;
+            const int r_last = (rho0 / n_rows == rho1 / n_rows) ? rho1 % n_rows : n_rows - 1;
+            if (n_rows > ROWS && c0 > pos0 + r_last) continue;
+        }
         // K and V go from memory straight into fragment order, once per pass: a forward with more query rows than one
         // pass takes (grouped-query models) reads them again from L1/L2 rather than holding 128 registers of them
         // across the loop.  The empty asm keeps the compiler from hoisting the loads (and their hi/lo splits) out of it.

@@ -79,7 +79,7 @@ struct swift_ctx {
     std::string err;
     cudaEvent_t ev[8];
     // captured forwards; programmatic dependent launch between the kernels of a forward
-    bool use_graphs, use_pdl, pdl_next, pdl_gemms, fuse, fuse_combine, prefetch_next, attn_mma, big_chunks, batched_scoring;
+    bool use_graphs, use_pdl, pdl_next, pdl_gemms, fuse, fuse_combine, prefetch_next, attn_mma, big_chunks, batched_scoring, whole_tiles;
     int attn_rows_per_cta, prefetch_tiles;
     std::vector<FwdGraph>* graphs;
     uint64_t graph_clock;
@@ -189,13 +189,13 @@ constexpr int TC_GRID = 148;        // persistent CTAs of the tensor-core GEMM: 
 constexpr int TC_MAX_TILES = 1024;
 
 // Largest number of CTAs that share one output tile under the stream-K schedule (= slabs needed).
-int max_segments(int N, int K)
+int max_segments(int N, int K, int grid = TC_GRID)
 {
     StreamK sk;
     sk.KB = ceil_div(K, TC_BK);
     const int tiles = ceil_div(N, TC_TILE_N);
     sk.U = (long long)tiles * sk.KB;
-    sk.G = (int)std::min<long long>(TC_GRID, sk.U);
+    sk.G = (int)std::min<long long>(grid, sk.U);
     int worst = 1;
     for (int t = 0; t < tiles; ++t)
         worst = std::max(worst, sk.owner((long long)(t + 1) * sk.KB - 1) - sk.owner((long long)t * sk.KB) + 1);
@@ -363,7 +363,15 @@ swift_status launch_gemm_tc(swift_ctx* ctx, const GemmSite& g, const EpiParams& 
 {
     if (ceil_div(g.N, TC_TILE_N) > TC_MAX_TILES) return fail(ctx, SWIFT_EUNSUPPORTED, "GEMM with %d output tiles", ceil_div(g.N, TC_TILE_N));
     if (ctx->pdl_gemms) ctx->pdl_next = true;     // this launch may begin before its predecessor has finished (see swift_load)
-    CU(launch_k(gemm_tc_kernel<EPI, TKV, NB>, dim3(TC_GRID), dim3(TC_THREADS), (size_t)TcShape<NB>::SMEM_BYTES, ctx, state_of(ctx), *g.mapW, *g.mapX,
+    // Decoding streams each weight once and wants every SM to stream the same bytes: 148 CTAs, tiles cut where the ranges
+    // fall.  A chunk of many rows is bound by its tensor work and its epilogues (128 rows per tile to finish, a 64 KB slab
+    // per partial tile), so there every CTA takes whole tiles: the fewest CTAs that need the same number of waves.
+    int grid = TC_GRID;
+    if (NB > 1 && ctx->whole_tiles) {
+        const int tiles = ceil_div(g.N, TC_TILE_N), waves = ceil_div(tiles, TC_GRID), even = ceil_div(tiles, waves);
+        if (max_segments(g.N, g.K, even) <= max_segments(g.N, g.K)) grid = even;      // slabs are sized for the 148-CTA schedule
+    }
+    CU(launch_k(gemm_tc_kernel<EPI, TKV, NB>, dim3(grid), dim3(TC_THREADS), (size_t)TcShape<NB>::SMEM_BYTES, ctx, state_of(ctx), *g.mapW, *g.mapX,
                 kptr<float>(ctx, ctx->kl.part), kptr<float>(ctx, ctx->kl.slabs), kptr<int>(ctx, ctx->kl.counters), g.N, g.K, ep,
                 next_map ? *next_map : *g.mapW));
     return SWIFT_OK;
@@ -417,10 +425,10 @@ swift_status launch_attn_mr(swift_ctx* ctx, const int* page_table, int block, in
 
 template <typename T, int NT>
 swift_status launch_attn_mma(swift_ctx* ctx, const int* page_table, int block, bool fused, float* out, __nv_bfloat16* planes,
-                             int part_rows = ROWS, int row_base = 0, int n_rows_fixed = 0, int pos0_fixed = 0)
+                             int part_rows = ROWS, int row_base = 0, int n_rows_fixed = 0, int pos0_fixed = 0, int z_passes = 1)
 {
     const swift_model_desc& d = ctx->d;
-    CU(launch_k(attn_mma_kernel<T, NT>, dim3(d.n_kv_heads, ctx->max_splits), dim3(AM_THREADS), attn_mma_smem_bytes(NT, ctx->max_splits), ctx,
+    CU(launch_k(attn_mma_kernel<T, NT>, dim3(d.n_kv_heads, ctx->max_splits, z_passes), dim3(AM_THREADS), attn_mma_smem_bytes(NT, ctx->max_splits), ctx,
                 (const DevState*)state_of(ctx), (const float*)kptr<float>(ctx, ctx->kl.q), reinterpret_cast<const T*>(ctx->kvbase),
                 page_table, ctx->kv, block, d.n_heads, ctx->max_splits, 1.0f / sqrtf((float)d.head_dim),
                 kptr<float>(ctx, ctx->kl.o_part), kptr<float2>(ctx, ctx->kl.ml_part), part_rows,
@@ -689,7 +697,8 @@ swift_status forward_chunk_big(swift_ctx* ctx, int rows, const int* page_table)
         ep.q_out = kptr<float>(ctx, ctx->kl.q); ep.kv_pool = ctx->kvbase; ep.page_table = page_table; ep.L = ctx->kv;
         ep.block = b; ep.n_heads = d.n_heads; ep.max_positions = d.max_positions; ep.rope_cs = kptr<float2>(ctx, ctx->kl.rope);
         ST((launch_gemm_tc<EPI_QKV, TKV, NB>(ctx, GemmSite{nullptr, nqkv, dm, nullptr, &ctx->tm_wqkv[b], &ctx->tm_xn_big}, ep)));
-        ST((launch_attn_mma<TKV, 2>(ctx, page_table, b, false, xa, xa_hl, TC_ROWS_MAX)));
+        ST((launch_attn_mma<TKV, 2>(ctx, page_table, b, false, xa, xa_hl, TC_ROWS_MAX, 0, 0, 0,
+                                    ceil_div((d.n_heads / d.n_kv_heads) * rows, 16))));
         CU(launch_k(attn_combine_kernel, dim3(d.n_heads, rows), dim3(d.head_dim), 2 * (size_t)ctx->max_splits * sizeof(float), ctx,
                     (const DevState*)st, (const float*)kptr<float>(ctx, ctx->kl.o_part), (const float2*)kptr<float2>(ctx, ctx->kl.ml_part),
                     ctx->max_splits, d.n_heads, d.head_dim, xa, xa_hl, (int)TC_ROWS_MAX, 0, 0, 0));
@@ -1104,7 +1113,8 @@ swift_status enqueue_score_batched(swift_ctx* ctx, const uint8_t* masks, int C, 
             }
             ST((launch_gemm_tc<EPI_QKV, TKV, NB>(ctx, GemmSite{nullptr, nqkv, dm, nullptr, &ctx->tm_wqkv[b], &ctx->tm_xn_big}, ep)));
             for (int j = 0; j < ch.n_cand; ++j) {     // each candidate of the chunk is a sequence of its own
-                ST((launch_attn_mma<TKV, 2>(ctx, pt_dev + (size_t)j * np, b, false, xa, xa_hl, TC_ROWS_MAX, j * gamma, gamma, pos_w)));
+                ST((launch_attn_mma<TKV, 2>(ctx, pt_dev + (size_t)j * np, b, false, xa, xa_hl, TC_ROWS_MAX, j * gamma, gamma, pos_w,
+                                            ceil_div((d.n_heads / d.n_kv_heads) * gamma, 16))));
                 CU(launch_k(attn_combine_kernel, dim3(d.n_heads, gamma), dim3(d.head_dim), 2 * (size_t)ctx->max_splits * sizeof(float), ctx,
                             (const DevState*)st, (const float*)kptr<float>(ctx, ctx->kl.o_part), (const float2*)kptr<float2>(ctx, ctx->kl.ml_part),
                             ctx->max_splits, d.n_heads, d.head_dim, xa, xa_hl, (int)TC_ROWS_MAX, j * gamma, gamma, pos_w));
@@ -1331,6 +1341,7 @@ swift_status swift_load(const swift_model_desc* desc, swift_devbuf weights, swif
     c->fuse = getenv("SWIFT_NO_FUSE") == nullptr && desc->head_dim <= TC_TILE_N;
     // prefill in chunks of up to TC_ROWS_MAX rows (SWIFT_NO_BIG_CHUNKS: 16 rows at a time, as decoding does)
     c->big_chunks = c->use_tc && c->fuse && big_rows_of(desc) == (size_t)TC_ROWS_MAX && getenv("SWIFT_NO_BIG_CHUNKS") == nullptr;
+    c->whole_tiles = getenv("SWIFT_NO_WHOLE_TILES") == nullptr;
     c->batched_scoring = c->big_chunks && getenv("SWIFT_NO_BATCHED_SCORING") == nullptr;
     c->graphs = new std::vector<FwdGraph>();
     c->graph_clock = 0;
