@@ -17,6 +17,7 @@
 #include "layer_opt.h"
 #include "kernels_attn.cuh"
 #include "kernels_attn_mma.cuh"
+#include "kernels_attn_tile.cuh"
 #include "kernels_elem.cuh"
 #include "kernels_gemm_simt.cuh"
 #include "kernels_gemm_tc.cuh"
@@ -79,7 +80,7 @@ struct swift_ctx {
     std::string err;
     cudaEvent_t ev[8];
     // captured forwards; programmatic dependent launch between the kernels of a forward
-    bool use_graphs, use_pdl, pdl_next, pdl_gemms, fuse, fuse_combine, prefetch_next, attn_mma, big_chunks, batched_scoring, whole_tiles;
+    bool use_graphs, use_pdl, pdl_next, pdl_gemms, fuse, fuse_combine, prefetch_next, attn_mma, big_chunks, batched_scoring, whole_tiles, attn_tile;
     int attn_rows_per_cta, prefetch_tiles;
     std::vector<FwdGraph>* graphs;
     uint64_t graph_clock;
@@ -423,6 +424,20 @@ swift_status launch_attn_mr(swift_ctx* ctx, const int* page_table, int block, in
         if (s_ != SWIFT_OK) return s_;             \
     } while (0)
 
+// Attention of a chunk of many rows (or of one sequence inside it): tiles of 64 query rows against 64-position chunks.
+template <typename T>
+swift_status launch_attn_tile(swift_ctx* ctx, const int* page_table, int block, int rows, int part_rows, int row_base, int n_rows_fixed,
+                              int pos0_fixed)
+{
+    const swift_model_desc& d = ctx->d;
+    const int q_rows = (d.n_heads / d.n_kv_heads) * rows;
+    CU(launch_k(attn_tile_kernel<T>, dim3(d.n_kv_heads, ctx->max_splits, ceil_div(q_rows, AT_QROWS)), dim3(AT_THREADS), AT_SMEM_BYTES, ctx,
+                (const DevState*)state_of(ctx), (const float*)kptr<float>(ctx, ctx->kl.q), reinterpret_cast<const T*>(ctx->kvbase),
+                page_table, ctx->kv, block, d.n_heads, ctx->max_splits, 1.0f / sqrtf((float)d.head_dim),
+                kptr<float>(ctx, ctx->kl.o_part), kptr<float2>(ctx, ctx->kl.ml_part), part_rows, row_base, n_rows_fixed, pos0_fixed));
+    return SWIFT_OK;
+}
+
 template <typename T, int NT>
 swift_status launch_attn_mma(swift_ctx* ctx, const int* page_table, int block, bool fused, float* out, __nv_bfloat16* planes,
                              int part_rows = ROWS, int row_base = 0, int n_rows_fixed = 0, int pos0_fixed = 0, int z_passes = 1)
@@ -697,8 +712,9 @@ swift_status forward_chunk_big(swift_ctx* ctx, int rows, const int* page_table)
         ep.q_out = kptr<float>(ctx, ctx->kl.q); ep.kv_pool = ctx->kvbase; ep.page_table = page_table; ep.L = ctx->kv;
         ep.block = b; ep.n_heads = d.n_heads; ep.max_positions = d.max_positions; ep.rope_cs = kptr<float2>(ctx, ctx->kl.rope);
         ST((launch_gemm_tc<EPI_QKV, TKV, NB>(ctx, GemmSite{nullptr, nqkv, dm, nullptr, &ctx->tm_wqkv[b], &ctx->tm_xn_big}, ep)));
-        ST((launch_attn_mma<TKV, 2>(ctx, page_table, b, false, xa, xa_hl, TC_ROWS_MAX, 0, 0, 0,
-                                    ceil_div((d.n_heads / d.n_kv_heads) * rows, 16))));
+        if (ctx->attn_tile) ST((launch_attn_tile<TKV>(ctx, page_table, b, rows, TC_ROWS_MAX, 0, 0, 0)));
+        else ST((launch_attn_mma<TKV, 2>(ctx, page_table, b, false, xa, xa_hl, TC_ROWS_MAX, 0, 0, 0,
+                                         ceil_div((d.n_heads / d.n_kv_heads) * rows, 16))));
         CU(launch_k(attn_combine_kernel, dim3(d.n_heads, rows), dim3(d.head_dim), 2 * (size_t)ctx->max_splits * sizeof(float), ctx,
                     (const DevState*)st, (const float*)kptr<float>(ctx, ctx->kl.o_part), (const float2*)kptr<float2>(ctx, ctx->kl.ml_part),
                     ctx->max_splits, d.n_heads, d.head_dim, xa, xa_hl, (int)TC_ROWS_MAX, 0, 0, 0));
@@ -1113,8 +1129,9 @@ swift_status enqueue_score_batched(swift_ctx* ctx, const uint8_t* masks, int C, 
             }
             ST((launch_gemm_tc<EPI_QKV, TKV, NB>(ctx, GemmSite{nullptr, nqkv, dm, nullptr, &ctx->tm_wqkv[b], &ctx->tm_xn_big}, ep)));
             for (int j = 0; j < ch.n_cand; ++j) {     // each candidate of the chunk is a sequence of its own
-                ST((launch_attn_mma<TKV, 2>(ctx, pt_dev + (size_t)j * np, b, false, xa, xa_hl, TC_ROWS_MAX, j * gamma, gamma, pos_w,
-                                            ceil_div((d.n_heads / d.n_kv_heads) * gamma, 16))));
+                if (ctx->attn_tile) ST((launch_attn_tile<TKV>(ctx, pt_dev + (size_t)j * np, b, gamma, TC_ROWS_MAX, j * gamma, gamma, pos_w)));
+                else ST((launch_attn_mma<TKV, 2>(ctx, pt_dev + (size_t)j * np, b, false, xa, xa_hl, TC_ROWS_MAX, j * gamma, gamma, pos_w,
+                                                 ceil_div((d.n_heads / d.n_kv_heads) * gamma, 16))));
                 CU(launch_k(attn_combine_kernel, dim3(d.n_heads, gamma), dim3(d.head_dim), 2 * (size_t)ctx->max_splits * sizeof(float), ctx,
                             (const DevState*)st, (const float*)kptr<float>(ctx, ctx->kl.o_part), (const float2*)kptr<float2>(ctx, ctx->kl.ml_part),
                             ctx->max_splits, d.n_heads, d.head_dim, xa, xa_hl, (int)TC_ROWS_MAX, j * gamma, gamma, pos_w));
@@ -1194,6 +1211,8 @@ cudaError_t init_kernel_attrs()
     if (e == cudaSuccess) e = cudaFuncSetAttribute(gemm_tc_kernel<EPI_SWIGLU, float, TC_NB_MAX>, cudaFuncAttributeMaxDynamicSharedMemorySize, big_smem);
     if (e == cudaSuccess) e = cudaFuncSetAttribute(gemm_tc_kernel<EPI_QKV, float, TC_NB_MAX>, cudaFuncAttributeMaxDynamicSharedMemorySize, big_smem);
     if (e == cudaSuccess) e = cudaFuncSetAttribute(gemm_tc_kernel<EPI_QKV, __nv_bfloat16, TC_NB_MAX>, cudaFuncAttributeMaxDynamicSharedMemorySize, big_smem);
+    if (e == cudaSuccess) e = cudaFuncSetAttribute(attn_tile_kernel<float>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)AT_SMEM_BYTES);
+    if (e == cudaSuccess) e = cudaFuncSetAttribute(attn_tile_kernel<__nv_bfloat16>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)AT_SMEM_BYTES);
     const int am_max = (int)attn_mma_smem_bytes(2, 262144 / ATTN_CHUNK);
     if (e == cudaSuccess) e = cudaFuncSetAttribute(attn_mma_kernel<float, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, am_max);
     if (e == cudaSuccess) e = cudaFuncSetAttribute(attn_mma_kernel<float, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, am_max);
@@ -1342,6 +1361,7 @@ swift_status swift_load(const swift_model_desc* desc, swift_devbuf weights, swif
     // prefill in chunks of up to TC_ROWS_MAX rows (SWIFT_NO_BIG_CHUNKS: 16 rows at a time, as decoding does)
     c->big_chunks = c->use_tc && c->fuse && big_rows_of(desc) == (size_t)TC_ROWS_MAX && getenv("SWIFT_NO_BIG_CHUNKS") == nullptr;
     c->whole_tiles = getenv("SWIFT_NO_WHOLE_TILES") == nullptr;
+    c->attn_tile = getenv("SWIFT_NO_ATTN_TILE") == nullptr;      // chunks of many rows: 64-row query tiles with K,V staged in shared memory
     c->batched_scoring = c->big_chunks && getenv("SWIFT_NO_BATCHED_SCORING") == nullptr;
     c->graphs = new std::vector<FwdGraph>();
     c->graph_clock = 0;
