@@ -41,6 +41,15 @@ def peaks():
     return 6650.0, "fallback"
 
 
+def tensor_peak_tflops():
+    """Dense bf16 throughput sustained over a long loop (the many-row GEMMs run inside long steps)."""
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        d = json.load(open(p))
+        return float(d.get("bf16_tflops_sustained", d.get("bf16_tflops", 1400.0)))
+    return 1400.0
+
+
 class ClockSampler:
     """Samples SM clocks and throttle reasons with nvidia-smi while the timed region runs."""
     Q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
@@ -199,7 +208,7 @@ def stream_mode(model, cfg, run, z, gp, args, max_new, desc, hbm_peak):
                       "vanilla_tokens_per_s": tot_tokens / (van_ms * 1e-3), "speedup_vs_vanilla": van_ms / tot_ms, "stream": rows}))
 
 
-def micro(cfg, run, args, hbm_peak):
+def micro(cfg, run, args, hbm_peak, tensor_peak):
     """Each GEMM shape of the walk, alone, on a 4-block copy of the model (weights still several times L2)."""
     from paper_2410_06916_b200 import SwiftModel
     small = cfg.with_blocks(4)
@@ -212,6 +221,12 @@ def micro(cfg, run, args, hbm_peak):
             ms, nbytes = model.time_gemm(which, rows, args.micro_iters)
             out["gemms"][f"{name}/{rows}"] = {"us": round(ms * 1e3, 2), "MB": round(nbytes / 1e6, 1),
                                               "gbs": round(nbytes / ms * 1e-6, 1), "frac": round(nbytes / ms * 1e-6 / hbm_peak, 3)}
+        if args.micro_many_rows and (which != 2 or 2 * small.ffn <= small.vocab):
+            # the many-row form: tensor-bound; two bf16 products per weight (hi and lo activation planes)
+            ms, nbytes = model.time_gemm(which, 128, args.micro_iters)
+            tflops = 2 * 2.0 * 128 * (nbytes / 2) / ms * 1e-9
+            out["gemms"][f"{name}/128"] = {"us": round(ms * 1e3, 2), "MB": round(nbytes / 1e6, 1), "tflops_hi_lo": round(tflops, 1),
+                                           "frac_tensor": round(tflops / tensor_peak, 3)}
     print(json.dumps(out))
 
 
@@ -232,6 +247,7 @@ def main():
     ap.add_argument("--micro", action="store_true",
                     help="time each weight-streaming GEMM of the model alone on a few-block copy (profiling aid); prints one JSON line")
     ap.add_argument("--micro-iters", type=int, default=40)
+    ap.add_argument("--micro-many-rows", action="store_true", help="with --micro: also the 128-row form of each GEMM")
     ap.add_argument("--micro-forward", action="store_true",
                     help="a few decode rounds on a 4-block copy of the model at the workload's context length (profiling aid)")
     args = ap.parse_args()
@@ -245,6 +261,7 @@ def main():
         run = dataclasses.replace(run, prompt_len=args.prompt_len)
     max_new = args.max_new or run.max_new
     hbm_peak, peak_kind = peaks()
+    tensor_peak = tensor_peak_tflops()
     sampling = run.mode == "sampling"
     desc = (f"{args.workload}: {cfg.name}-shaped decoder ({cfg.n_blocks} blocks, d {cfg.d_model}, {cfg.dtype}), "
             f"prompt {run.prompt_len}, {max_new} {run.mode} tokens, {run.n_skip_blocks} blocks skipped, max draft {run.max_draft}"
@@ -276,7 +293,7 @@ def main():
     from paper_2410_06916_b200 import GenParams, SwiftModel
     torch.cuda.set_device(local)
     if args.micro:
-        micro(cfg, run, args, hbm_peak)
+        micro(cfg, run, args, hbm_peak, tensor_peak)
         return
     if args.micro_forward:
         small = cfg.with_blocks(4)

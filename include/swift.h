@@ -297,8 +297,10 @@ int32_t swift_round_times(const swift_ctx* ctx, int32_t capacity, float* ms_draf
  * what the implementation moves, beside the algorithmic figure above.  Same conventions as swift_round_times. */
 int32_t swift_round_bytes_stored(const swift_ctx* ctx, int32_t capacity, double* bytes_draft_host, double* bytes_verify_host);
 /* Times `iters` back-to-back launches of one weight-streaming GEMM of the walk (which: 0 fused QKV,
- * 1 o_proj, 2 fused gate/up, 3 down, 4 output head) with n_rows rows, cycling over the blocks' weights
- * so that successive launches read different memory.  Outputs the average CUDA-event time per launch
+ * 1 o_proj, 2 fused gate/up, 3 down, 4 output head) with n_rows rows (1..16, or 128: the many-row form that
+ * prefill chunks and side-by-side candidate scoring use, with the plain epilogue; SWIFT_EUNSUPPORTED where the
+ * model has no such form, SWIFT_ECAPACITY if the output is wider than the vocabulary), cycling over the blocks'
+ * weights so that successive launches read different memory.  Outputs the average CUDA-event time per launch
  * on the stream and the weight bytes one launch streams.  Clobbers the workspace of an open round. */
 swift_status swift_time_gemm(swift_ctx* ctx, int32_t which, int32_t n_rows, int32_t iters,
                              float* ms_per_launch_host, double* bytes_per_launch_host);

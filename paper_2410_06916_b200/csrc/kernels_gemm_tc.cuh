@@ -323,7 +323,8 @@ __device__ __forceinline__ void tc_finalize(const EpiParams& ep, int pos0, float
 
 // grid = G persistent CTAs, block = 192 threads, dynamic smem = TC_SMEM_BYTES.
 // mapW: bf16 [N][K], box {64, 128}; mapX: bf16 [32][K] (rows 0-15 hi, 16-31 lo), box {64, 32}; both
-// 128-byte swizzled.  slabs: [S_max][ROWS][N] fp32; counters: one int per tile, zero on entry and on exit.
+// 128-byte swizzled.  slabs: [S_max][ROWS][N] fp32 (many rows: [S_max][tile][block][row of tile][16], the 16 values a
+// thread holds side by side); counters: one int per tile, zero on entry and on exit.
 template <int EPI, typename TKV, int NB = 1>
 __global__ void __launch_bounds__(TC_THREADS, 1)
 gemm_tc_kernel(DevState* st, const __grid_constant__ CUtensorMap mapW, const __grid_constant__ CUtensorMap mapX,
@@ -352,8 +353,8 @@ gemm_tc_kernel(DevState* st, const __grid_constant__ CUtensorMap mapW, const __g
     __shared__ int last_flag_sh, peek_sh;
     __shared__ int abort_sh, epi_abort_sh;
     __shared__ float rstd_sh[ROWS * NB];
-    __shared__ float stage_sh[EPI == EPI_PLAIN ? 4 * ROWS : ROWS * TC_TILE_N + 4 * ROWS];
-    __shared__ float2 rope_sh[EPI == EPI_QKV ? ROWS * (TC_TILE_N / 2) : 1];   // (cos, sin) of the rows' positions
+    __shared__ float stage_sh[EPI == EPI_PLAIN ? 4 * ROWS : (NB > 1 && EPI == EPI_QKV ? 2 : 1) * ROWS * TC_TILE_N + 8 * ROWS];
+    __shared__ float2 rope_sh[EPI == EPI_QKV && NB == 1 ? ROWS * (TC_TILE_N / 2) : 1];   // (cos, sin) of the rows' positions
     __shared__ int page_sh[ROWS];                                              // KV page of each row's position
 
     // The producer and the MMA warp need the row count before they can start; they read it here, ahead of the
@@ -491,44 +492,125 @@ gemm_tc_kernel(DevState* st, const __grid_constant__ CUtensorMap mapW, const __g
         }
         asm volatile("bar.sync 1, 128;" ::: "memory");
         if constexpr (NB > 1) {
-            // Chunks of many rows: the accumulator holds NB blocks of 16 rows side by side; each is drained, finished
-            // (or parked in this CTA's slab) in turn with the code of the 16-row case.  No early fetches and no
-            // fast path here: these launches are long enough for their tails not to matter.
+            // Chunks of many rows: the accumulator holds NB blocks of 16 rows side by side; each is drained and finished
+            // (or parked in this CTA's slab) in turn.  Everything a block's finish needs from global memory (its slice
+            // of the residual stream, or its rows' rotary factors and cache pages) is requested one block ahead, the
+            // row loops are unrolled (this code runs NB times per tile: it is warm), and the staging buffers alternate
+            // between blocks so that one barrier per block suffices.
             constexpr int RT = ROWS * NB;
             const int live_blocks = (n_rows + ROWS - 1) / ROWS;
-            auto finish_block = [&](int rb, float (&val)[ROWS], int tile, int n) {
+            const int l = quarter * 32 + lane;
+            const size_t slab_stride = (size_t)n_tiles * TC_TILE_N * RT;     // one CTA's parked partial tiles
+            float* sums_sh = stage_sh + (EPI == EPI_QKV ? 2 : 1) * ROWS * TC_TILE_N;      // [2][4 * ROWS]
+            struct ManyPre { float h[ROWS]; float2 cs[ROWS]; int page[ROWS]; };
+            auto prefetch = [&](int rb, int n, ManyPre& p) {
                 const int row0 = rb * ROWS, rows_here = min(ROWS, n_rows - row0);
-                const int pos_b = (EPI == EPI_QKV && ep.per_block) ? ep.rb_pos0[rb] : pos0_epi + row0;   // cache slot of the block's first row
-                if (EPI == EPI_QKV) {                      // rotary factors and cache pages of this block's rows
-                    const int* pt = ep.per_block ? ep.rb_page_table[rb] : ep.page_table;
-                    asm volatile("bar.sync 1, 128;" ::: "memory");
-                    const int half = ep.L.head_dim >> 1;
-                    for (int idx = etid; idx < ROWS * half; idx += 128) {
-                        const int m = idx / half, j = idx - m * half, pos = pos_b + m;
-                        if (m < rows_here && pos < ep.max_positions) rope_sh[m * (TC_TILE_N / 2) + j] = ep.rope_cs[(size_t)pos * half + j];
-                    }
-                    if (etid < ROWS) {
-                        const int pos = pos_b + etid;
-                        page_sh[etid] = (etid < rows_here && pos < ep.max_positions) ? pt[pos >> ep.L.page_shift] : 0;
-                    }
-                    asm volatile("bar.sync 1, 128;" ::: "memory");
-                }
-                float h_pre[ROWS];
-                float gain_pre = 0.f;
                 if (EPI == EPI_RESID) {
 #pragma unroll
-                    for (int m = 0; m < ROWS; ++m) h_pre[m] = (n < N && m < rows_here) ? __ldcg(ep.h + (size_t)(row0 + m) * N + n) : 0.f;
-                    if (ep.gain_next && n < N) gain_pre = ep.gain_next[n];
+                    for (int m = 0; m < ROWS; ++m) p.h[m] = (n < N && m < rows_here) ? __ldcg(ep.h + (size_t)(row0 + m) * N + n) : 0.f;
+                } else if (EPI == EPI_QKV) {
+                    const int pos_b = ep.per_block ? ep.rb_pos0[rb] : pos0_epi + row0;     // cache slot of the block's first row
+                    const int* pt = ep.per_block ? ep.rb_page_table[rb] : ep.page_table;
+                    const int dh = ep.L.head_dim, half = dh >> 1, i = n % dh, j = i < half ? i : i - half;
+#pragma unroll
+                    for (int m = 0; m < ROWS; ++m) {
+                        const int pos = pos_b + m;
+                        const bool ok = m < rows_here && pos < ep.max_positions;
+                        p.cs[m] = ok ? __ldg(ep.rope_cs + (size_t)pos * half + j) : make_float2(1.f, 0.f);
+                        p.page[m] = ok ? __ldg(pt + (pos >> ep.L.page_shift)) : -1;
+                    }
                 }
-                tc_finalize<EPI, TKV>(ep, pos_b, val, rows_here, tile, quarter, lane, etid, N, Y, rstd_sh + row0, stage_sh,
-                                      h_pre, gain_pre, rope_sh, page_sh, row0);
+            };
+            auto finish_many = [&](int rb, float (&val)[ROWS], int tile, int n, const ManyPre& p, float gain) {
+                const int row0 = rb * ROWS, rows_here = min(ROWS, n_rows - row0);
+                if (EPI != EPI_RESID) {
+#pragma unroll
+                    for (int m = 0; m < ROWS; ++m) val[m] *= rstd_sh[row0 + m];
+                }
+                if (EPI == EPI_PLAIN) {
+                    if (n < N) {
+#pragma unroll
+                        for (int m = 0; m < ROWS; ++m)
+                            if (m < rows_here) Y[(size_t)(row0 + m) * N + n] = val[m];
+                    }
+                } else if (EPI == EPI_SWIGLU) {
+                    // lanes 0-15 hold gate rows, lanes 16-31 the matching up rows: the lower half finishes the block's
+                    // rows 0-7, the upper half rows 8-15, after one exchange per row pair
+                    const int i = (n >> 5) * 16 + (lane & 15);
+                    const bool upper = lane >= 16;
+#pragma unroll
+                    for (int m = 0; m < ROWS / 2; ++m) {
+                        const float recv = __shfl_xor_sync(0xffffffffu, upper ? val[m] : val[m + ROWS / 2], 16);
+                        const float g = upper ? recv : val[m], up = upper ? val[m + ROWS / 2] : recv;
+                        const int row = upper ? m + ROWS / 2 : m;
+                        if (i < ep.ffn && row < rows_here) store_hi_lo(ep.act_planes, row0 + row, ep.ffn, i, g / (1.f + expf(-g)) * up);
+                    }
+                } else if (EPI == EPI_RESID) {
+                    float sq[ROWS];
+#pragma unroll
+                    for (int m = 0; m < ROWS; ++m) {
+                        const float hn = p.h[m] + val[m];
+                        const bool ok = n < N && m < rows_here;
+                        if (ok) {
+                            ep.h[(size_t)(row0 + m) * N + n] = hn;
+                            if (ep.gain_next) store_hi_lo(ep.planes_out, row0 + m, N, n, hn * gain);
+                        }
+                        sq[m] = ok ? hn * hn : 0.f;
+                    }
+                    if (ep.gain_next) {                    // uniform over the grid
+                        // sums of squares per row over the warp's 32 columns: halve the rows a lane carries at every
+                        // exchange; lane pair (2r, 2r + 1) ends with row r
+#pragma unroll
+                        for (int s = 16, len = ROWS; s >= 2; s >>= 1, len >>= 1) {
+                            const bool up_half = (lane & s) != 0;
+#pragma unroll
+                            for (int i = 0; i < ROWS / 2; ++i)
+                                if (i < len / 2) {
+                                    const float keep = up_half ? sq[i + len / 2] : sq[i], send = up_half ? sq[i] : sq[i + len / 2];
+                                    sq[i] = keep + __shfl_xor_sync(0xffffffffu, send, s);
+                                }
+                        }
+                        const float tot = sq[0] + __shfl_xor_sync(0xffffffffu, sq[0], 1);
+                        float* ss = sums_sh + (rb & 1) * 4 * ROWS;
+                        if (!(lane & 1)) ss[quarter * ROWS + (lane >> 1)] = tot;
+                        asm volatile("bar.sync 1, 128;" ::: "memory");
+                        if (etid < ROWS)
+                            ep.sumsq_out[(size_t)tile * ep.sum_rows + row0 + etid] = etid < rows_here ?
+                                (ss[etid] + ss[ROWS + etid]) + (ss[2 * ROWS + etid] + ss[3 * ROWS + etid]) : 0.f;
+                    }
+                } else {   // EPI_QKV: the RoPE partner of row l sits dh/2 rows away in the same tile, in another warp
+                    float* stg = stage_sh + (rb & 1) * ROWS * TC_TILE_N;
+#pragma unroll
+                    for (int m = 0; m < ROWS; ++m) stg[m * TC_TILE_N + l] = val[m];
+                    asm volatile("bar.sync 1, 128;" ::: "memory");
+                    const int dh = ep.L.head_dim, half = dh >> 1;
+                    const int gh = n / dh, i = n - gh * dh;
+                    const int lp = i < half ? l + half : l - half;
+                    const int pos_b = ep.per_block ? ep.rb_pos0[rb] : pos0_epi + row0;
+                    TKV* pool = reinterpret_cast<TKV*>(ep.kv_pool);
+                    const int hk = gh - ep.n_heads;
+                    const int kv = hk >= ep.L.n_kv_heads ? 1 : 0;
+                    const int kh = kv ? hk - ep.L.n_kv_heads : hk;
+                    if (n < N) {
+#pragma unroll
+                        for (int m = 0; m < ROWS; ++m) {
+                            if (p.page[m] >= 0) {           // the row exists and its position fits the cache
+                                const float a = val[m], b = stg[m * TC_TILE_N + lp];
+                                float out = a;
+                                if (gh < ep.n_heads + ep.L.n_kv_heads) out = i < half ? a * p.cs[m].x - b * p.cs[m].y : a * p.cs[m].x + b * p.cs[m].y;
+                                if (gh < ep.n_heads) ep.q_out[(size_t)(row0 + m) * ep.n_heads * dh + n] = out;
+                                else store_val(pool + ep.L.offset(p.page[m], ep.block, kv, kh, (pos_b + m) & (ep.L.page_size - 1)) + i, out);
+                            }
+                        }
+                    }
+                }
             };
             while (u < u_end) {
                 const int tile = (int)(u / sk.KB), kb0 = (int)(u % sk.KB);
                 const long long tile_end = (long long)(tile + 1) * sk.KB;
                 const long long seg_end = tile_end < u_end ? tile_end : u_end;
                 const int buf = seg & 1;
-                const int n = tile * TC_TILE_N + quarter * 32 + lane;
+                const int n = tile * TC_TILE_N + l;
                 const bool whole = (kb0 == 0) && (seg_end == tile_end);
                 int slab = 0, nseg = 1;
                 if (!whole) {
@@ -536,11 +618,19 @@ gemm_tc_kernel(DevState* st, const __grid_constant__ CUtensorMap mapW, const __g
                     slab = blockIdx.x - g_first;
                     nseg = g_last - g_first + 1;
                 }
+                ManyPre pre;
+                float gain = 0.f;
+                if (whole) {
+                    prefetch(0, n, pre);
+                    if (EPI == EPI_RESID && ep.gain_next && n < N) gain = ep.gain_next[n];
+                }
                 if (!mbar_wait(tfull_bar(buf), (seg >> 1) & 1)) epi_abort_sh = 1;
                 asm volatile("bar.sync 1, 128;" ::: "memory");
                 if (epi_abort_sh) { abort_sh = 1; break; }
                 tc_fence_after();
                 for (int rb = 0; rb < live_blocks; ++rb) {
+                    ManyPre nxt;
+                    if (whole && rb + 1 < live_blocks) prefetch(rb + 1, n, nxt);
                     uint32_t v[32];
                     const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(buf * S::COLS + rb * TC_COLS);
                     asm volatile(
@@ -557,13 +647,12 @@ gemm_tc_kernel(DevState* st, const __grid_constant__ CUtensorMap mapW, const __g
 #pragma unroll
                     for (int m = 0; m < ROWS; ++m) val[m] = __uint_as_float(v[m]) + __uint_as_float(v[16 + m]);
                     if (whole) {
-                        finish_block(rb, val, tile, n);
-                    } else if (n < N) {
-                        float* mine = slabs + ((size_t)slab * RT + rb * ROWS) * N;
-                        const int rows_here = min(ROWS, n_rows - rb * ROWS);
+                        finish_many(rb, val, tile, n, pre, gain);
+                        pre = nxt;
+                    } else {                                   // parked as this thread's 16 values side by side
+                        float4* mine = reinterpret_cast<float4*>(slabs + (size_t)slab * slab_stride + (((size_t)tile * NB + rb) * TC_TILE_N + l) * ROWS);
 #pragma unroll
-                        for (int m = 0; m < ROWS; ++m)
-                            if (m < rows_here) mine[(size_t)m * N + n] = val[m];
+                        for (int q4 = 0; q4 < ROWS / 4; ++q4) mine[q4] = make_float4(val[4 * q4], val[4 * q4 + 1], val[4 * q4 + 2], val[4 * q4 + 3]);
                     }
                 }
                 tc_fence_before();
@@ -574,18 +663,55 @@ gemm_tc_kernel(DevState* st, const __grid_constant__ CUtensorMap mapW, const __g
                     if (etid == 0) last_flag_sh = (atom_add_acq_rel_gpu(&counters[tile], 1) == nseg - 1) ? 1 : 0;
                     asm volatile("bar.sync 1, 128;" ::: "memory");
                     if (last_flag_sh) {                         // last arrival: add the slabs in slab order, block by block
+                        constexpr int SJ = EPI == EPI_QKV ? 2 : 3;   // slabs fetched side by side (more than that: one after another)
+                        float cur[SJ][ROWS], nxs[SJ][ROWS];
+                        auto fetch = [&](int rb, float (&t)[SJ][ROWS]) {
+#pragma unroll
+                            for (int j = 0; j < SJ; ++j) {
+                                const float4* src = reinterpret_cast<const float4*>(slabs + (size_t)j * slab_stride + (((size_t)tile * NB + rb) * TC_TILE_N + l) * ROWS);
+#pragma unroll
+                                for (int q4 = 0; q4 < ROWS / 4; ++q4) {
+                                    const float4 x = j < nseg ? __ldcg(src + q4) : make_float4(0.f, 0.f, 0.f, 0.f);
+                                    t[j][4 * q4] = x.x; t[j][4 * q4 + 1] = x.y; t[j][4 * q4 + 2] = x.z; t[j][4 * q4 + 3] = x.w;
+                                }
+                            }
+                        };
+                        constexpr bool AHEAD = EPI != EPI_QKV;    // the next block's slabs are requested before this block is finished
+                        if (AHEAD) fetch(0, cur);
+                        prefetch(0, n, pre);
+                        if (EPI == EPI_RESID && ep.gain_next && n < N) gain = ep.gain_next[n];
                         for (int rb = 0; rb < live_blocks; ++rb) {
-                            const int rows_here = min(ROWS, n_rows - rb * ROWS);
+                            ManyPre nxt;
+                            if (!AHEAD) fetch(rb, cur);
+                            if (rb + 1 < live_blocks) {
+                                if (AHEAD) fetch(rb + 1, nxs);
+                                prefetch(rb + 1, n, nxt);
+                            }
                             float val[ROWS];
 #pragma unroll
                             for (int m = 0; m < ROWS; ++m) val[m] = 0.f;
-                            if (n < N)
-                                for (int j = 0; j < nseg; ++j) {
 #pragma unroll
-                                    for (int m = 0; m < ROWS; ++m)
-                                        if (m < rows_here) val[m] += __ldcg(slabs + (((size_t)j * RT + rb * ROWS + m) * N + n));
+                            for (int j = 0; j < SJ; ++j)
+                                if (j < nseg) {
+#pragma unroll
+                                    for (int m = 0; m < ROWS; ++m) val[m] += cur[j][m];
                                 }
-                            finish_block(rb, val, tile, n);
+                            for (int j = SJ; j < nseg; ++j) {
+                                const float4* src = reinterpret_cast<const float4*>(slabs + (size_t)j * slab_stride + (((size_t)tile * NB + rb) * TC_TILE_N + l) * ROWS);
+#pragma unroll
+                                for (int q4 = 0; q4 < ROWS / 4; ++q4) {
+                                    const float4 x = __ldcg(src + q4);
+                                    val[4 * q4] += x.x; val[4 * q4 + 1] += x.y; val[4 * q4 + 2] += x.z; val[4 * q4 + 3] += x.w;
+                                }
+                            }
+                            finish_many(rb, val, tile, n, pre, gain);
+                            pre = nxt;
+                            if (AHEAD) {
+#pragma unroll
+                                for (int j = 0; j < SJ; ++j)
+#pragma unroll
+                                    for (int m = 0; m < ROWS; ++m) cur[j][m] = nxs[j][m];
+                            }
                         }
                         if (etid == 0) counters[tile] = 0;
                     }

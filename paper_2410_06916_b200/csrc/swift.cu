@@ -11,6 +11,8 @@
 #include <cstdio>
 #include <cstring>
 #include <string>
+#include <map>
+#include <mutex>
 #include <vector>
 
 #include "common.cuh"
@@ -203,6 +205,45 @@ int max_segments(int N, int K, int grid = TC_GRID)
     return worst;
 }
 
+// Grid of a many-row GEMM launch.  Such a launch is bound by tensor work, and a tile that is shared between CTAs costs
+// each of them a 64 KB slab to write and the last one the others' slabs to add, so the stream-K cut is chosen per shape:
+// among the grids that the slabs were sized for, the one whose busiest CTA has the least to do, counting a shared
+// segment as PART_COST extra K steps and the final merge as MERGE_COST.  (40 tiles of a long K: 120 CTAs, three to a
+// tile; 120 tiles: one each; 216 tiles: 144 CTAs, three tiles to a pair.)
+int many_row_grid(int N, int K)
+{
+    static const int forced = getenv("SWIFT_MANY_GRID") ? atoi(getenv("SWIFT_MANY_GRID")) : 0;
+    constexpr long long PART_COST = 10, MERGE_COST = 14;
+    static std::mutex mu;
+    static std::map<std::pair<int, int>, int> memo;         // the search below is far too slow for a launch path
+    std::lock_guard<std::mutex> lock(mu);
+    auto it = memo.find({N, K});
+    if (it != memo.end()) return it->second;
+    const int tiles = ceil_div(N, TC_TILE_N), cap = max_segments(N, K);
+    if (forced > 0 && forced <= TC_GRID && max_segments(N, K, forced) <= cap) return memo[{N, K}] = forced;
+    StreamK sk;
+    sk.KB = ceil_div(K, TC_BK);
+    sk.U = (long long)tiles * sk.KB;
+    int best = TC_GRID;
+    long long best_cost = -1;
+    for (int G = TC_GRID; G >= TC_GRID / 2; --G) {
+        sk.G = (int)std::min<long long>(G, sk.U);
+        if (max_segments(N, K, G) > cap) continue;
+        long long worst = 0;
+        bool shared = false;
+        for (int g = 0; g < sk.G; ++g) {
+            const long long u0 = sk.start(g), u1 = sk.start(g + 1);
+            long long cost = u1 - u0;
+            if (u0 % sk.KB) { cost += PART_COST; shared = true; }
+            if (u1 % sk.KB && (u1 / sk.KB != u0 / sk.KB || !(u0 % sk.KB))) { cost += PART_COST; shared = true; }
+            worst = std::max(worst, cost);
+        }
+        if (shared) worst += MERGE_COST;
+        if (best_cost < 0 || worst < best_cost) { best_cost = worst; best = G; }
+    }
+    return memo[{N, K}] = best;
+}
+
 // Scratch KV pages beyond the sequence's own: the window of one candidate (copy-on-write start page included), or the
 // windows of the several candidates of one chunk when candidates are scored side by side.
 int scratch_pages(const swift_model_desc* d) { return MAX_SCORE_ROWS / d->page_size + 8; }
@@ -273,7 +314,9 @@ WorkLayout work_layout(const swift_model_desc* d)
     k.slab_floats = 0;
     k.xn_hl = k.xa_hl = k.act_hl = k.slabs = k.counters = k.sumsq = 0;
     if (d->dtype == SWIFT_BF16) {
-        auto slab_need = [&](int N, int K) { k.slab_floats = std::max(k.slab_floats, (size_t)max_segments(N, K) * RB * (size_t)N); };
+        auto slab_need = [&](int N, int K) {      // whole tiles: the many-row form parks 128 x RB values per tile
+            k.slab_floats = std::max(k.slab_floats, (size_t)max_segments(N, K) * RB * (size_t)ceil_div(N, TC_TILE_N) * TC_TILE_N);
+        };
         slab_need((int)(qd + 2 * kd), (int)dm); slab_need((int)dm, (int)qd); slab_need(2 * d->ffn, (int)dm);
         slab_need((int)dm, d->ffn); slab_need(d->vocab, (int)dm);
         k.xn_hl = c.take(2 * RB * dm * 2);
@@ -365,16 +408,23 @@ swift_status launch_gemm_tc(swift_ctx* ctx, const GemmSite& g, const EpiParams& 
     if (ceil_div(g.N, TC_TILE_N) > TC_MAX_TILES) return fail(ctx, SWIFT_EUNSUPPORTED, "GEMM with %d output tiles", ceil_div(g.N, TC_TILE_N));
     if (ctx->pdl_gemms) ctx->pdl_next = true;     // this launch may begin before its predecessor has finished (see swift_load)
     // Decoding streams each weight once and wants every SM to stream the same bytes: 148 CTAs, tiles cut where the ranges
-    // fall.  A chunk of many rows is bound by its tensor work and its epilogues (128 rows per tile to finish, a 64 KB slab
-    // per partial tile), so there every CTA takes whole tiles: the fewest CTAs that need the same number of waves.
+    // fall.  A chunk of many rows is bound by its tensor work and its epilogues: see many_row_grid.
     int grid = TC_GRID;
-    if (NB > 1 && ctx->whole_tiles) {
-        const int tiles = ceil_div(g.N, TC_TILE_N), waves = ceil_div(tiles, TC_GRID), even = ceil_div(tiles, waves);
-        if (max_segments(g.N, g.K, even) <= max_segments(g.N, g.K)) grid = even;      // slabs are sized for the 148-CTA schedule
-    }
+    if (NB > 1 && ctx->whole_tiles) grid = many_row_grid(g.N, g.K);
     CU(launch_k(gemm_tc_kernel<EPI, TKV, NB>, dim3(grid), dim3(TC_THREADS), (size_t)TcShape<NB>::SMEM_BYTES, ctx, state_of(ctx), *g.mapW, *g.mapX,
                 kptr<float>(ctx, ctx->kl.part), kptr<float>(ctx, ctx->kl.slabs), kptr<int>(ctx, ctx->kl.counters), g.N, g.K, ep,
                 next_map ? *next_map : *g.mapW));
+    return SWIFT_OK;
+}
+
+// The plain-epilogue GEMM of a chunk of many rows with its output at Y ([rows][N]).
+template <int NB>
+swift_status launch_gemm_tc_y(swift_ctx* ctx, const GemmSite& g, const EpiParams& ep, float* Y)
+{
+    int grid = TC_GRID;
+    if (ctx->whole_tiles) grid = many_row_grid(g.N, g.K);
+    CU(launch_k(gemm_tc_kernel<EPI_PLAIN, float, NB>, dim3(grid), dim3(TC_THREADS), (size_t)TcShape<NB>::SMEM_BYTES, ctx, state_of(ctx), *g.mapW,
+                *g.mapX, Y, kptr<float>(ctx, ctx->kl.slabs), kptr<int>(ctx, ctx->kl.counters), g.N, g.K, ep, *g.mapW));
     return SWIFT_OK;
 }
 
@@ -1104,9 +1154,7 @@ swift_status enqueue_score_batched(swift_ctx* ctx, const uint8_t* masks, int C, 
         if (ch.sub == L) {                            // output head: final norm, logits, arg max per row
             gather_norm_kernel<<<rows, 1024, 0, ctx->stream>>>(map, H_all, h, wptr<float>(ctx, ctx->wl.final_norm), xn_hl, sumsq, dm);
             ctx->launches++;
-            CU(launch_k(gemm_tc_kernel<EPI_PLAIN, float, NB>, dim3(TC_GRID), dim3(TC_THREADS), (size_t)TcShape<NB>::SMEM_BYTES, ctx, st,
-                        ctx->tm_lm_head, ctx->tm_xn_big, logits, kptr<float>(ctx, ctx->kl.slabs), kptr<int>(ctx, ctx->kl.counters), d.vocab, dm,
-                        base, ctx->tm_lm_head));
+            ST((launch_gemm_tc_y<NB>(ctx, GemmSite{nullptr, d.vocab, dm, nullptr, &ctx->tm_lm_head, &ctx->tm_xn_big}, base, logits)));
             // the head's chunks hold consecutive candidates: their predictions go where their rows are in H_all
             argmax_rows_kernel<<<rows, 1024, 0, ctx->stream>>>(logits, d.vocab, pred + maps[ch.map_off]);
             ctx->launches++;
@@ -1894,6 +1942,29 @@ static swift_status time_gemm_t(swift_ctx* ctx, int which, int n_rows, int iters
     };
     int S = 0;
     (void)p;
+    if (n_rows > ROWS) {   // the many-row form (prefill chunks, side-by-side scoring): plain epilogue into the scoring logits buffer
+        if (!ctx->big_chunks) return fail(ctx, SWIFT_EUNSUPPORTED, "no many-row GEMM for this model");
+        if (N > d.vocab) return fail(ctx, SWIFT_ECAPACITY, "output of %d columns does not fit the buffer used for timing", N);
+        EpiParams ep;
+        memset(&ep, 0, sizeof ep);
+        ep.sum_rows = TC_ROWS_MAX;
+        auto big = [&](int i) -> swift_status {
+            GemmSite g = site(i);
+            g.mapX = which == 1 ? &ctx->tm_xa_big : which == 3 ? &ctx->tm_act_big : &ctx->tm_xn_big;
+            return launch_gemm_tc_y<TC_NB_MAX>(ctx, g, ep, kptr<float>(ctx, ctx->kl.score_logits));
+        };
+        for (int i = 0; i < 3; ++i) ST(big(i));
+        CU(cudaEventRecord(ctx->ev[0], ctx->stream));
+        for (int i = 0; i < iters; ++i) ST(big(i + 3));
+        CU(cudaEventRecord(ctx->ev[1], ctx->stream));
+        CU(cudaStreamSynchronize(ctx->stream));
+        float t = 0.f;
+        CU(cudaEventElapsedTime(&t, ctx->ev[0], ctx->ev[1]));
+        *ms = t / (float)iters;
+        *bytes = (double)N * K * sizeof(T);
+        DevState hs;
+        return read_state(ctx, &hs);
+    }
     for (int i = 0; i < 3; ++i) ST(run_gemm<T>(ctx, mr_of(n_rows), site(i), &S));
     CU(cudaEventRecord(ctx->ev[0], ctx->stream));
     for (int i = 0; i < iters; ++i) ST(run_gemm<T>(ctx, mr_of(n_rows), site(i + 3), &S));
@@ -1913,7 +1984,7 @@ swift_status swift_time_gemm(swift_ctx* ctx, int32_t which, int32_t n_rows, int3
 {
     if (!ctx || !ms || !bytes) return fail(ctx, SWIFT_EINVAL, "null argument");
     if (ctx->round_open) return fail(ctx, SWIFT_ESTATE, "a round is open");
-    if (which < 0 || which > 4 || n_rows < 1 || n_rows > ROWS || iters < 1) return fail(ctx, SWIFT_EINVAL, "bad which / n_rows / iters");
+    if (which < 0 || which > 4 || n_rows < 1 || (n_rows > ROWS && n_rows != TC_ROWS_MAX) || iters < 1) return fail(ctx, SWIFT_EINVAL, "bad which / n_rows / iters");
     if (ctx->d.dtype == SWIFT_BF16) return time_gemm_t<__nv_bfloat16>(ctx, which, n_rows, iters, ms, bytes);
     return time_gemm_t<float>(ctx, which, n_rows, iters, ms, bytes);
 }
