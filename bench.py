@@ -247,6 +247,7 @@ def main():
     ap.add_argument("--micro", action="store_true",
                     help="time each weight-streaming GEMM of the model alone on a few-block copy (profiling aid); prints one JSON line")
     ap.add_argument("--micro-iters", type=int, default=40)
+    ap.add_argument("--micro-score", action="store_true", help="with --micro-forward: also two rounds of candidate scoring")
     ap.add_argument("--micro-many-rows", action="store_true", help="with --micro: also the 128-row form of each GEMM")
     ap.add_argument("--micro-forward", action="store_true",
                     help="a few decode rounds on a 4-block copy of the model at the workload's context length (profiling aid)")
@@ -306,6 +307,16 @@ def main():
                          ("swift", GenParams(max_new=2 * (run.max_draft + 1) + 1, max_draft=run.max_draft, skip_mask=zz))):
             _, st, _ = model.generate(prompt, gp)
             outs[name] = {"ms_decode": st.ms_decode, "tokens": st.tokens, "rounds": st.rounds, "launches": st.kernel_launches}
+        if args.micro_score:          # plus two rounds of candidate scoring (32 proposals, half of the sub-layers skipped)
+            rng = np.random.default_rng(5)
+            masks = (rng.random((32, 2 * small.n_blocks)) < 0.45).astype(np.uint8)
+            ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            for _ in range(2):
+                ev0.record(model.stream)
+                model.score_skipsets(masks, 32)
+                ev1.record(model.stream)
+                torch.cuda.synchronize()
+            outs["scoring_round_ms"] = ev0.elapsed_time(ev1)
         print(json.dumps({"micro_forward": small.name, "prompt": run.prompt_len, **outs}))
         return
     if world > 1:

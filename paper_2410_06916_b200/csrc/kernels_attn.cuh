@@ -511,11 +511,18 @@ attn_stream_kernel(const DevState* st, const float* __restrict__ q, const T* __r
 __global__ void attn_combine_kernel(const DevState* st, const float* __restrict__ o_part,
                                     const float2* __restrict__ ml_part, int max_splits, int n_heads, int dh,
                                     float* __restrict__ out, __nv_bfloat16* __restrict__ planes, int part_rows,
-                                    int row_base, int n_rows_fixed, int pos0_fixed)
+                                    int row_base, int n_rows_fixed, int pos0_fixed, int n_seq)
 {
-    // row_base / n_rows_fixed / pos0_fixed: as in attn_mma_kernel (one sequence inside a larger chunk), 0 / 0 / 0 otherwise
+    // row_base / n_rows_fixed / pos0_fixed: as in attn_mma_kernel (one sequence inside a larger chunk), 0 / 0 / 0 otherwise;
+    // n_seq > 1: grid.y covers that many such sequences, one after another
     pdl_enter();
-    const int r = blockIdx.y;
+    int r = blockIdx.y;
+    if (n_seq > 1) {
+        const int seq = r / n_rows_fixed;
+        if (seq >= n_seq) return;
+        r -= seq * n_rows_fixed;
+        row_base += seq * n_rows_fixed;
+    }
     if (r >= (n_rows_fixed > 0 ? n_rows_fixed : st->n_rows)) return;
     extern __shared__ float comb_sh[];
     __shared__ float wmax_sh[32];

@@ -25,23 +25,42 @@ __device__ __forceinline__ void ldmatrix_x2_trans(uint32_t& r0, uint32_t& r1, co
 
 // grid = (n_kv_heads, max_splits, query tiles), block = 128, dynamic smem = AT_SMEM_BYTES.
 // row_base / n_rows_fixed / pos0_fixed: as in attn_mma_kernel (a sequence inside a larger chunk), else 0 / 0 / 0.
+// n_seq > 1: that many such sequences in one launch (grid.z covers the larger of the batch's and the sequences' tiles),
+// page tables pt_stride ints apart.
 template <typename T>
 __global__ void __launch_bounds__(AT_THREADS, 2)
 attn_tile_kernel(const DevState* st, const float* __restrict__ q, const T* __restrict__ kv_pool,
                  const int* __restrict__ page_table, KvLayout L, int block, int n_heads, int max_splits, float scale,
                  float* __restrict__ o_part, float2* __restrict__ ml_part, int part_rows, int row_base, int n_rows_fixed,
-                 int pos0_fixed)
+                 int pos0_fixed, int n_seq, int pt_stride)
 {
     pdl_enter();
     constexpr int DH = 128;
-    const int n_rows = n_rows_fixed > 0 ? n_rows_fixed : st->n_rows;
+    int n_rows = n_rows_fixed > 0 ? n_rows_fixed : st->n_rows;
     if (n_rows <= 0) return;
     const int pos0 = n_rows_fixed > 0 ? pos0_fixed : st->pos0, total = pos0 + n_rows;
     const int kvh = blockIdx.x, s = blockIdx.y, c0 = s * ATTN_CHUNK;
     if (c0 >= total) return;
     const int len = min(ATTN_CHUNK, total - c0);
-    const int G = n_heads / L.n_kv_heads, R = G * n_rows;
-    const int rho_tile = blockIdx.z * AT_QROWS;
+    const int G = n_heads / L.n_kv_heads;
+    int z = blockIdx.z;
+    if (n_seq > 1) {
+        // n_seq sequences of n_rows rows side by side (rows row_base + seq * n_rows ..), all continuing the same cached
+        // context, each with its own page table for its own rows.  A chunk that lies inside the context is the same for
+        // all of them and fully visible to every row: it is staged once per 64 rows of the whole batch.  A chunk that
+        // reaches into the sequences' own rows is handled per sequence.
+        if (c0 + ATTN_CHUNK <= pos0) {
+            n_rows *= n_seq;
+        } else {
+            const int tiles_per = (G * n_rows + AT_QROWS - 1) / AT_QROWS, seq = z / tiles_per;
+            if (seq >= n_seq) return;
+            z -= seq * tiles_per;
+            row_base += seq * n_rows;
+            page_table += (size_t)seq * pt_stride;
+        }
+    }
+    const int R = G * n_rows;
+    const int rho_tile = z * AT_QROWS;
     if (rho_tile >= R) return;
     {   // a tile none of whose rows sees this chunk yet has nothing to add: the merge never reads it
         const int rho1 = min(R, rho_tile + AT_QROWS) - 1;
@@ -57,24 +76,11 @@ attn_tile_kernel(const DevState* st, const float* __restrict__ q, const T* __res
     __nv_bfloat16* v_hi = k_lo + ATTN_CHUNK * AT_KSTRIDE;
     __nv_bfloat16* v_lo = v_hi + ATTN_CHUNK * AT_KSTRIDE;
 
-    // ---- stage the chunk: thread i takes 16-byte pieces (4 dims of one position); positions past the end are zero
-    for (int i = tid; i < ATTN_CHUNK * 32; i += AT_THREADS) {
-        const int p = i >> 5, c4 = (i & 31) * 4;
-        float4 kk = make_float4(0.f, 0.f, 0.f, 0.f), vv = kk;
-        if (p < len) {
-            const int pos = c0 + p;
-            const int page = __ldg(page_table + (pos >> L.page_shift)), slot = pos & (L.page_size - 1);
-            kk = load_row4<T>(kv_pool + L.offset(page, block, 0, kvh, slot) + c4);
-            vv = load_row4<T>(kv_pool + L.offset(page, block, 1, kvh, slot) + c4);
-        }
-        uint2 hi, lo;
-        split_pair(kk.x, kk.y, hi.x, lo.x); split_pair(kk.z, kk.w, hi.y, lo.y);
-        *reinterpret_cast<uint2*>(k_hi + p * AT_KSTRIDE + c4) = hi;
-        *reinterpret_cast<uint2*>(k_lo + p * AT_KSTRIDE + c4) = lo;
-        split_pair(vv.x, vv.y, hi.x, lo.x); split_pair(vv.z, vv.w, hi.y, lo.y);
-        *reinterpret_cast<uint2*>(v_hi + p * AT_KSTRIDE + c4) = hi;
-        *reinterpret_cast<uint2*>(v_lo + p * AT_KSTRIDE + c4) = lo;
-    }
+    // ---- stage the chunk: thread i takes 16-byte pieces (4 dims of one position); positions past the end are zero.
+    // The pages of the chunk's positions are looked up first and the loads of eight pieces are issued together, so that
+    // a CTA waits for two or three trips to memory rather than for one per piece.
+    __shared__ int page_of[ATTN_CHUNK];
+    if (tid < ATTN_CHUNK) page_of[tid] = tid < len ? __ldg(page_table + ((c0 + tid) >> L.page_shift)) : 0;
 
     // ---- this warp's 16 query rows as A fragments (hi, lo), scaled: rows rho_w + g and rho_w + g + 8
     const int rho_w = rho_tile + 16 * w;
@@ -94,6 +100,33 @@ attn_tile_kernel(const DevState* st, const float* __restrict__ q, const T* __res
         split_pair(a1.x * scale, a1.y * scale, qh[ks][1], ql[ks][1]);
         split_pair(a2.x * scale, a2.y * scale, qh[ks][2], ql[ks][2]);
         split_pair(a3.x * scale, a3.y * scale, qh[ks][3], ql[ks][3]);
+    }
+    __syncthreads();
+#pragma unroll
+    for (int part = 0; part < ATTN_CHUNK * 32 / (8 * AT_THREADS); ++part) {
+        float4 kk[8], vv[8];
+#pragma unroll
+        for (int it = 0; it < 8; ++it) {
+            const int i = tid + (part * 8 + it) * AT_THREADS, p = i >> 5, c4 = (i & 31) * 4;
+            kk[it] = make_float4(0.f, 0.f, 0.f, 0.f);
+            vv[it] = kk[it];
+            if (p < len) {
+                const int slot = (c0 + p) & (L.page_size - 1);
+                kk[it] = load_row4<T>(kv_pool + L.offset(page_of[p], block, 0, kvh, slot) + c4);
+                vv[it] = load_row4<T>(kv_pool + L.offset(page_of[p], block, 1, kvh, slot) + c4);
+            }
+        }
+#pragma unroll
+        for (int it = 0; it < 8; ++it) {
+            const int i = tid + (part * 8 + it) * AT_THREADS, p = i >> 5, c4 = (i & 31) * 4;
+            uint2 hi, lo;
+            split_pair(kk[it].x, kk[it].y, hi.x, lo.x); split_pair(kk[it].z, kk[it].w, hi.y, lo.y);
+            *reinterpret_cast<uint2*>(k_hi + p * AT_KSTRIDE + c4) = hi;
+            *reinterpret_cast<uint2*>(k_lo + p * AT_KSTRIDE + c4) = lo;
+            split_pair(vv[it].x, vv[it].y, hi.x, lo.x); split_pair(vv[it].z, vv[it].w, hi.y, lo.y);
+            *reinterpret_cast<uint2*>(v_hi + p * AT_KSTRIDE + c4) = hi;
+            *reinterpret_cast<uint2*>(v_lo + p * AT_KSTRIDE + c4) = lo;
+        }
     }
     __syncthreads();
     if (rho_w >= R) return;                                 // (after the barrier: every warp helped staging)

@@ -477,14 +477,16 @@ swift_status launch_attn_mr(swift_ctx* ctx, const int* page_table, int block, in
 // Attention of a chunk of many rows (or of one sequence inside it): tiles of 64 query rows against 64-position chunks.
 template <typename T>
 swift_status launch_attn_tile(swift_ctx* ctx, const int* page_table, int block, int rows, int part_rows, int row_base, int n_rows_fixed,
-                              int pos0_fixed)
+                              int pos0_fixed, int n_seq = 1, int pt_stride = 0)
 {
     const swift_model_desc& d = ctx->d;
-    const int q_rows = (d.n_heads / d.n_kv_heads) * rows;
-    CU(launch_k(attn_tile_kernel<T>, dim3(d.n_kv_heads, ctx->max_splits, ceil_div(q_rows, AT_QROWS)), dim3(AT_THREADS), AT_SMEM_BYTES, ctx,
+    const int G = d.n_heads / d.n_kv_heads;
+    const int z = std::max(ceil_div(G * rows * n_seq, AT_QROWS), n_seq * ceil_div(G * rows, AT_QROWS));
+    CU(launch_k(attn_tile_kernel<T>, dim3(d.n_kv_heads, ctx->max_splits, z), dim3(AT_THREADS), AT_SMEM_BYTES, ctx,
                 (const DevState*)state_of(ctx), (const float*)kptr<float>(ctx, ctx->kl.q), reinterpret_cast<const T*>(ctx->kvbase),
                 page_table, ctx->kv, block, d.n_heads, ctx->max_splits, 1.0f / sqrtf((float)d.head_dim),
-                kptr<float>(ctx, ctx->kl.o_part), kptr<float2>(ctx, ctx->kl.ml_part), part_rows, row_base, n_rows_fixed, pos0_fixed));
+                kptr<float>(ctx, ctx->kl.o_part), kptr<float2>(ctx, ctx->kl.ml_part), part_rows, row_base, n_rows_fixed, pos0_fixed, n_seq,
+                pt_stride));
     return SWIFT_OK;
 }
 
@@ -520,7 +522,7 @@ swift_status launch_attn(swift_ctx* ctx, int rows, const int* page_table, int bl
         if (fused) return SWIFT_OK;
         CU(launch_k(attn_combine_kernel, dim3(d.n_heads, rows), dim3(d.head_dim), 2 * (size_t)ctx->max_splits * sizeof(float), ctx,
                     (const DevState*)state_of(ctx), (const float*)kptr<float>(ctx, ctx->kl.o_part),
-                    (const float2*)kptr<float2>(ctx, ctx->kl.ml_part), ctx->max_splits, d.n_heads, d.head_dim, out, planes, (int)ROWS, 0, 0, 0));
+                    (const float2*)kptr<float2>(ctx, ctx->kl.ml_part), ctx->max_splits, d.n_heads, d.head_dim, out, planes, (int)ROWS, 0, 0, 0, 1));
         return SWIFT_OK;
     }
     // The streaming kernel (head_dim 128) takes the rows in groups of at most attn_rows_per_cta, one group per
@@ -546,7 +548,7 @@ swift_status launch_attn(swift_ctx* ctx, int rows, const int* page_table, int bl
     if (s != SWIFT_OK || fused) return s;
     CU(launch_k(attn_combine_kernel, dim3(d.n_heads, rows), dim3(d.head_dim), 2 * (size_t)ctx->max_splits * sizeof(float), ctx,
                 (const DevState*)state_of(ctx), (const float*)kptr<float>(ctx, ctx->kl.o_part),
-                (const float2*)kptr<float2>(ctx, ctx->kl.ml_part), ctx->max_splits, d.n_heads, d.head_dim, out, planes, (int)ROWS, 0, 0, 0));
+                (const float2*)kptr<float2>(ctx, ctx->kl.ml_part), ctx->max_splits, d.n_heads, d.head_dim, out, planes, (int)ROWS, 0, 0, 0, 1));
     return SWIFT_OK;
 }
 
@@ -767,7 +769,7 @@ swift_status forward_chunk_big(swift_ctx* ctx, int rows, const int* page_table)
                                          ceil_div((d.n_heads / d.n_kv_heads) * rows, 16))));
         CU(launch_k(attn_combine_kernel, dim3(d.n_heads, rows), dim3(d.head_dim), 2 * (size_t)ctx->max_splits * sizeof(float), ctx,
                     (const DevState*)st, (const float*)kptr<float>(ctx, ctx->kl.o_part), (const float2*)kptr<float2>(ctx, ctx->kl.ml_part),
-                    ctx->max_splits, d.n_heads, d.head_dim, xa, xa_hl, (int)TC_ROWS_MAX, 0, 0, 0));
+                    ctx->max_splits, d.n_heads, d.head_dim, xa, xa_hl, (int)TC_ROWS_MAX, 0, 0, 0, 1));
         EpiParams resid = base;
         resid.h = h; resid.planes_out = xn_hl; resid.sumsq_out = sumsq;
         resid.gain_next = wptr<float>(ctx, ctx->wl.mlp_norm[b]);
@@ -1176,14 +1178,17 @@ swift_status enqueue_score_batched(swift_ctx* ctx, const uint8_t* masks, int C, 
                 ep.rb_page_table[rb] = pt_dev + (size_t)j * np;
             }
             ST((launch_gemm_tc<EPI_QKV, TKV, NB>(ctx, GemmSite{nullptr, nqkv, dm, nullptr, &ctx->tm_wqkv[b], &ctx->tm_xn_big}, ep)));
-            for (int j = 0; j < ch.n_cand; ++j) {     // each candidate of the chunk is a sequence of its own
-                if (ctx->attn_tile) ST((launch_attn_tile<TKV>(ctx, pt_dev + (size_t)j * np, b, gamma, TC_ROWS_MAX, j * gamma, gamma, pos_w)));
-                else ST((launch_attn_mma<TKV, 2>(ctx, pt_dev + (size_t)j * np, b, false, xa, xa_hl, TC_ROWS_MAX, j * gamma, gamma, pos_w,
-                                                 ceil_div((d.n_heads / d.n_kv_heads) * gamma, 16))));
-                CU(launch_k(attn_combine_kernel, dim3(d.n_heads, gamma), dim3(d.head_dim), 2 * (size_t)ctx->max_splits * sizeof(float), ctx,
-                            (const DevState*)st, (const float*)kptr<float>(ctx, ctx->kl.o_part), (const float2*)kptr<float2>(ctx, ctx->kl.ml_part),
-                            ctx->max_splits, d.n_heads, d.head_dim, xa, xa_hl, (int)TC_ROWS_MAX, j * gamma, gamma, pos_w));
+            // each candidate of the chunk is a sequence of its own behind the context they share
+            if (ctx->attn_tile) {
+                ST((launch_attn_tile<TKV>(ctx, pt_dev, b, gamma, TC_ROWS_MAX, 0, gamma, pos_w, ch.n_cand, np)));
+            } else {
+                for (int j = 0; j < ch.n_cand; ++j)
+                    ST((launch_attn_mma<TKV, 2>(ctx, pt_dev + (size_t)j * np, b, false, xa, xa_hl, TC_ROWS_MAX, j * gamma, gamma, pos_w,
+                                                ceil_div((d.n_heads / d.n_kv_heads) * gamma, 16))));
             }
+            CU(launch_k(attn_combine_kernel, dim3(d.n_heads, ch.n_cand * gamma), dim3(d.head_dim), 2 * (size_t)ctx->max_splits * sizeof(float), ctx,
+                        (const DevState*)st, (const float*)kptr<float>(ctx, ctx->kl.o_part), (const float2*)kptr<float2>(ctx, ctx->kl.ml_part),
+                        ctx->max_splits, d.n_heads, d.head_dim, xa, xa_hl, (int)TC_ROWS_MAX, 0, gamma, pos_w, ch.n_cand));
             ST((launch_gemm_tc<EPI_RESID, float, NB>(ctx, GemmSite{nullptr, dm, qd, nullptr, &ctx->tm_wo[b], &ctx->tm_xa_big}, resid)));
         } else {
             gather_norm_kernel<<<rows, 1024, 0, ctx->stream>>>(map, H_all, h, wptr<float>(ctx, ctx->wl.mlp_norm[b]), xn_hl, sumsq, dm);
