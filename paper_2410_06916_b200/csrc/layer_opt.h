@@ -15,6 +15,7 @@
 #include <cmath>
 #include <cstdint>
 #include <set>
+#include <thread>
 #include <vector>
 
 namespace swopt {
@@ -118,6 +119,22 @@ public:
     }
 };
 
+// fn(i) for i in [0, n) on up to eight host threads (contiguous ranges); the calls must not depend on one another.
+template <typename F>
+inline void parallel_for(int n, F fn)
+{
+    const int hw = (int)std::thread::hardware_concurrency();
+    const int T = std::max(1, std::min(std::min(8, hw > 0 ? hw : 1), n));
+    if (T == 1) {
+        for (int i = 0; i < n; ++i) fn(i);
+        return;
+    }
+    std::vector<std::thread> th;
+    for (int k = 0; k < T; ++k)
+        th.emplace_back([&, k] { for (int i = (int)((long long)n * k / T); i < (int)((long long)n * (k + 1) / T); ++i) fn(i); });
+    for (std::thread& x : th) x.join();
+}
+
 inline GpModel LayerOpt::fit() const
 {
     const int n_all = (int)y.size();
@@ -162,8 +179,12 @@ inline GpModel LayerOpt::fit() const
     }
     for (int i = 0; i < n; ++i)
         for (int j = 0; j <= i; ++j) d2[(size_t)i * n + j] = hamming(X[first + i], X[first + j]);
-    bool have = false;
-    for (double ell : ells) {
+    // one factorisation per length scale, side by side on host threads; the choice among them is made in the scales' order
+    struct Trial { std::vector<double> L, a; double lml = 0.0; bool ok = false; };
+    std::vector<Trial> trials(ells.size());
+    parallel_for((int)ells.size(), [&](int e) {
+        const double ell = ells[e];
+        Trial& tr = trials[e];
         std::vector<double> Lc((size_t)n * n, 0.0);
         bool ok = true;
         for (int i = 0; i < n && ok; ++i) {           // Cholesky, row by row
@@ -178,7 +199,7 @@ inline GpModel LayerOpt::fit() const
                 }
             }
         }
-        if (!ok) continue;
+        if (!ok) return;
         std::vector<double> a(t);                     // alpha = K^-1 t by two triangular solves
         for (int i = 0; i < n; ++i) {
             for (int k = 0; k < i; ++k) a[i] -= Lc[(size_t)i * n + k] * a[k];
@@ -190,9 +211,14 @@ inline GpModel LayerOpt::fit() const
         }
         double lml = -0.5 * n * std::log(2.0 * 3.14159265358979323846);
         for (int i = 0; i < n; ++i) lml -= 0.5 * t[i] * a[i] + std::log(Lc[(size_t)i * n + i]);
-        if (!have || lml > best.lml) {
+        tr.L.swap(Lc); tr.a.swap(a); tr.lml = lml; tr.ok = true;
+    });
+    bool have = false;
+    for (size_t e = 0; e < ells.size(); ++e) {
+        Trial& tr = trials[e];
+        if (tr.ok && (!have || tr.lml > best.lml)) {
             have = true;
-            best.L.swap(Lc); best.alpha.swap(a); best.ell = ell; best.lml = lml;
+            best.L.swap(tr.L); best.alpha.swap(tr.a); best.ell = ells[e]; best.lml = tr.lml;
         }
     }
     best.X.assign(X.begin() + first, X.end());
@@ -256,14 +282,16 @@ inline BlockSet LayerOpt::bayesian_set(double* ucb_out)
         if (seen.insert(c).second) fresh.push_back(c);
     if (fresh.empty()) return random_set();
     if (X.empty() || g.n == 0) return fresh[0];
-    int pick = 0;
-    double best = 0.0;
-    for (size_t i = 0; i < fresh.size(); ++i) {
+    std::vector<double> ucb(fresh.size());             // each prediction is independent: host threads, same values as in turn
+    parallel_for((int)fresh.size(), [&](int i) {
         double mean, dev;
         predict(g, fresh[i], &mean, &dev);
-        const double u = mean + kappa * dev;
-        if (i == 0 || u > best) { best = u; pick = (int)i; }
-    }
+        ucb[i] = mean + kappa * dev;
+    });
+    int pick = 0;
+    double best = 0.0;
+    for (size_t i = 0; i < fresh.size(); ++i)
+        if (i == 0 || ucb[i] > best) { best = ucb[i]; pick = (int)i; }
     if (ucb_out) *ucb_out = best;
     return fresh[pick];
 }
