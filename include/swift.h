@@ -266,7 +266,10 @@ swift_status swift_set_gemm_impl(swift_ctx* ctx, int32_t impl);
 
 /* One weight-streaming GEMM of the walk on caller data: y[r][n] = sum_k x[r][k] * W[n][k] with W the
  * stored weight `which` (0 fused QKV, 1 o_proj, 2 fused gate/up in its interleaved row order, 3 down,
- * 4 output head) of `block`.  x_host: fp32 [n_rows][K], y_host: fp32 [n_rows][N], n_rows <= 16. */
+ * 4 output head) of `block`.  x_host: fp32 [n_rows][K], y_host: fp32 [n_rows][N].  n_rows <= 16: the kernel
+ * decoding uses.  17 <= n_rows <= 128: the many-row form of the tensor-core kernel that prefill chunks and
+ * side-by-side candidate scoring use (bf16 models with head_dim 128 and the tensor-core kernel selected, else
+ * SWIFT_EUNSUPPORTED; SWIFT_ECAPACITY if N exceeds the vocabulary size). */
 swift_status swift_gemm(swift_ctx* ctx, int32_t which, int32_t block, const float* x_host, int32_t n_rows,
                         float* y_host);
 

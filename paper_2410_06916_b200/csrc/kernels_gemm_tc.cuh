@@ -893,10 +893,11 @@ __global__ void wait_probe_kernel(DevState* st, long long limit_cycles)
 }
 
 // grid = (ceil(K/256), rows): splits fp32 rows [rows][K] into the planes (used when a caller supplies X directly)
-__global__ void split_planes_kernel(const float* __restrict__ x, __nv_bfloat16* __restrict__ planes, int K)
+// row0: row of the planes that x's first row goes to
+__global__ void split_planes_kernel(const float* __restrict__ x, __nv_bfloat16* __restrict__ planes, int K, int row0)
 {
     const int r = blockIdx.y, i = blockIdx.x * blockDim.x + threadIdx.x;
-    if (i < K) store_hi_lo(planes, r, K, i, x[(size_t)r * K + i]);
+    if (i < K) store_hi_lo(planes, row0 + r, K, i, x[(size_t)r * K + i]);
 }
 
 } // namespace swk

@@ -1748,14 +1748,40 @@ swift_status swift_gemm(swift_ctx* ctx, int32_t which, int32_t block, const floa
     if (!ctx || !x_host || !y_host) return fail(ctx, SWIFT_EINVAL, "null argument");
     if (ctx->round_open) return fail(ctx, SWIFT_ESTATE, "a round is open");
     const swift_model_desc& d = ctx->d;
-    if (which < 0 || which > 4 || n_rows < 1 || n_rows > ROWS || block < 0 || block >= d.n_blocks)
+    if (which < 0 || which > 4 || n_rows < 1 || n_rows > TC_ROWS_MAX || block < 0 || block >= d.n_blocks)
         return fail(ctx, SWIFT_EINVAL, "bad which / block / n_rows");
+    if (n_rows > ROWS && !(ctx->use_tc && ctx->big_chunks)) return fail(ctx, SWIFT_EUNSUPPORTED, "no many-row GEMM for this model or kernel choice");
     const int dm = d.d_model, qd = d.n_heads * d.head_dim, kd = d.n_kv_heads * d.head_dim;
     const int N = which == 0 ? qd + 2 * kd : which == 1 ? dm : which == 2 ? 2 * d.ffn : which == 3 ? dm : d.vocab;
     const int K = which == 1 ? qd : which == 3 ? d.ffn : dm;
     float* X = which == 1 ? kptr<float>(ctx, ctx->kl.xa) : which == 3 ? kptr<float>(ctx, ctx->kl.act) : kptr<float>(ctx, ctx->kl.xn);
     const size_t woff = which == 0 ? ctx->wl.wqkv[block] : which == 1 ? ctx->wl.wo[block] : which == 2 ? ctx->wl.wgu[block]
                         : which == 3 ? ctx->wl.wdown[block] : ctx->wl.lm_head;
+    if (n_rows > ROWS) {   // the many-row form (prefill chunks, side-by-side scoring), plain epilogue
+        if (N > d.vocab) return fail(ctx, SWIFT_ECAPACITY, "output of %d columns does not fit the buffer used for this call", N);
+        __nv_bfloat16* planes = which == 1 ? kptr<__nv_bfloat16>(ctx, ctx->kl.xa_hl) : which == 3 ? kptr<__nv_bfloat16>(ctx, ctx->kl.act_hl)
+                                           : kptr<__nv_bfloat16>(ctx, ctx->kl.xn_hl);
+        for (int r0 = 0; r0 < n_rows; r0 += ROWS) {            // rows reach their planes 16 at a time through the 16-row buffer
+            const int nr = std::min((int)ROWS, n_rows - r0);
+            CU(copy_async(ctx, X, x_host + (size_t)r0 * K, (size_t)nr * K * 4, cudaMemcpyHostToDevice));
+            split_planes_kernel<<<dim3(ceil_div(K, 256), nr), 256, 0, ctx->stream>>>(X, planes, K, r0);
+            ctx->launches++;
+        }
+        set_rows_kernel<<<1, 1, 0, ctx->stream>>>(state_of(ctx), 0, n_rows);
+        ctx->launches++;
+        EpiParams ep;
+        memset(&ep, 0, sizeof ep);
+        ep.sum_rows = TC_ROWS_MAX;
+        GemmSite g{nullptr, N, K, nullptr,
+                   which == 0 ? &ctx->tm_wqkv[block] : which == 1 ? &ctx->tm_wo[block] : which == 2 ? &ctx->tm_wgu[block]
+                   : which == 3 ? &ctx->tm_wdown[block] : &ctx->tm_lm_head,
+                   which == 1 ? &ctx->tm_xa_big : which == 3 ? &ctx->tm_act_big : &ctx->tm_xn_big};
+        float* Y = kptr<float>(ctx, ctx->kl.score_logits);
+        ST(launch_gemm_tc_y<TC_NB_MAX>(ctx, g, ep, Y));
+        CU(copy_async(ctx, y_host, Y, (size_t)n_rows * N * 4, cudaMemcpyDeviceToHost));
+        DevState hs;
+        return read_state(ctx, &hs);
+    }
     CU(copy_async(ctx, X, x_host, (size_t)n_rows * K * 4, cudaMemcpyHostToDevice));
     set_rows_kernel<<<1, 1, 0, ctx->stream>>>(state_of(ctx), 0, n_rows);
     ctx->launches++;
@@ -1763,7 +1789,7 @@ swift_status swift_gemm(swift_ctx* ctx, int32_t which, int32_t block, const floa
     if (ctx->use_tc) {
         __nv_bfloat16* planes = which == 1 ? kptr<__nv_bfloat16>(ctx, ctx->kl.xa_hl) : which == 3 ? kptr<__nv_bfloat16>(ctx, ctx->kl.act_hl)
                                            : kptr<__nv_bfloat16>(ctx, ctx->kl.xn_hl);
-        split_planes_kernel<<<dim3(ceil_div(K, 256), n_rows), 256, 0, ctx->stream>>>(X, planes, K);
+        split_planes_kernel<<<dim3(ceil_div(K, 256), n_rows), 256, 0, ctx->stream>>>(X, planes, K, 0);
         ctx->launches++;
         g.mapW = which == 0 ? &ctx->tm_wqkv[block] : which == 1 ? &ctx->tm_wo[block] : which == 2 ? &ctx->tm_wgu[block]
                  : which == 3 ? &ctx->tm_wdown[block] : &ctx->tm_lm_head;

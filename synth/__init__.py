@@ -129,8 +129,9 @@ MODELS: Dict[str, ModelConfig] = {
 RUNS: Dict[str, Tuple[str, RunConfig]] = {
     "c1": ("tiny", RunConfig(32, 64, 4, stop_conf=0.8, n_skip_blocks=4)),
     "c2": ("7b", RunConfig(512, 256, 8, n_skip_blocks=14)),
-    "c3": ("13b-graded", RunConfig(1024, 512, 8, n_skip_blocks=18, optimise=True)),
-    "c3-flat": ("13b", RunConfig(1024, 512, 8, n_skip_blocks=18, optimise=True)),     # the same on the all-N(0, 0.02) model
+    # (up to 32 optimisation rounds per input: Appendix B.2's S = 1000 proposals at 32 proposals per round)
+    "c3": ("13b-graded", RunConfig(1024, 512, 8, n_skip_blocks=18, optimise=True, max_opt_rounds=32)),
+    "c3-flat": ("13b", RunConfig(1024, 512, 8, n_skip_blocks=18, optimise=True, max_opt_rounds=32)),     # the same on the all-N(0, 0.02) model
     "c3-fixed": ("13b", RunConfig(1024, 512, 8, n_skip_blocks=18)),     # config 3's shape with the planted set held fixed
     "c4": ("13b", RunConfig(1024, 512, 8, n_skip_blocks=20, mode="sampling", rng_seed=4)),
     # config 4 with the sampling setting the paper uses on code generation (Appendix B.2)

@@ -136,6 +136,39 @@ def test_weight_streaming_gemm_kernels(shape, rows):
         g.close()
 
 
+@pytest.mark.parametrize("shape,rows", [("13b", 128), ("13b", 100), ("7b", 77), ("70b", 33)])
+def test_many_row_gemm_against_the_oracle(shape, rows):
+    """The many-row form of the tensor-core GEMM (prefill chunks, side-by-side scoring) alone, at the real projection
+    shapes: whole tiles per CTA (QKV, gate/up, head) and tiles shared between three or four CTAs (o_proj, down), full and
+    ragged row counts (a last block of 4, 13 or 1 rows), against the oracle's fp64 projection."""
+    cfg = synth.MODELS[shape].with_blocks(1, n_planted=0)
+    from paper_2410_06916_b200 import SwiftModel
+    g = SwiftModel(cfg, max_positions=64)
+    try:
+        w = {n: synth.make_tensor(cfg, n, 0, planted=False) for n in ("wq", "wk", "wv", "wo", "wgate", "wup", "wdown")}
+        w["lm_head"] = synth.make_tensor(cfg, "lm_head")
+        for n, t in w.items():
+            g.pack(n, 0 if n != "lm_head" else -1, t)
+        F = cfg.ffn
+        il = torch.stack([w["wgate"].view(F // 16, 16, -1), w["wup"].view(F // 16, 16, -1)], 1).reshape(2 * F, -1)
+        mats = [torch.cat([w["wq"], w["wk"], w["wv"]]), w["wo"], il, w["wdown"], w["lm_head"]]
+        gen = torch.Generator().manual_seed(1000 + rows)
+        for which, W in enumerate(mats):
+            if W.shape[0] > cfg.vocab:
+                continue                                         # wider than the buffer this call writes to (70B gate/up)
+            x = torch.randn(rows, W.shape[1], generator=gen) * (1.0 + which)
+            ref = so.linear(x, W).numpy()
+            scale = float(np.sqrt((ref ** 2).mean()))
+            y = g.gemm(which, 0, x.numpy())
+            assert np.abs(y - ref).max() < 1e-4 * scale, (which, float(np.abs(y - ref).max()), scale)
+            y16 = g.gemm(which, 0, x.numpy()[:16])               # the decoding kernel on the first 16 rows: same products, other order
+            assert np.abs(y16 - y[:16]).max() < 2e-5 * scale, which
+        ms, nbytes = g.time_gemm(2 if 2 * F <= cfg.vocab else 0, 128, 3)
+        assert ms > 0 and nbytes > 0
+    finally:
+        g.close()
+
+
 @pytest.mark.parametrize("shape,kv", [("7b", "f32"), ("13b", "f32"), ("13b", "bf16"), ("70b", "f32"), ("34b", "f32")])
 def test_full_width_bf16_forward(shape, kv):
     """Two blocks at the real 7B / 13B / 70B (grouped-query, 8 query heads per KV head) / 34B-class (7 query heads per
