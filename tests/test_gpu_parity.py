@@ -162,7 +162,7 @@ def test_many_row_gemm_against_the_oracle(shape, rows):
             y = g.gemm(which, 0, x.numpy())
             assert np.abs(y - ref).max() < 1e-4 * scale, (which, float(np.abs(y - ref).max()), scale)
             y16 = g.gemm(which, 0, x.numpy()[:16])               # the decoding kernel on the first 16 rows: same products, other order
-            assert np.abs(y16 - y[:16]).max() < 2e-5 * scale, which
+            assert np.abs(y16 - y[:16]).max() < 1e-4 * scale, which
         ms, nbytes = g.time_gemm(2 if 2 * F <= cfg.vocab else 0, 128, 3)
         assert ms > 0 and nbytes > 0
     finally:
