@@ -82,7 +82,8 @@ struct swift_ctx {
     std::string err;
     cudaEvent_t ev[8];
     // captured forwards; programmatic dependent launch between the kernels of a forward
-    bool use_graphs, use_pdl, pdl_next, pdl_gemms, fuse, fuse_combine, prefetch_next, attn_mma, big_chunks, batched_scoring, whole_tiles, attn_tile;
+    bool use_graphs, use_pdl, pdl_next, pdl_gemms, fuse, fuse_combine, prefetch_next, attn_mma, big_chunks, batched_scoring, whole_tiles, attn_tile, attn_tile_decode;
+    bool tree_forward = false;      // the forward being enqueued verifies a token tree (rows see their ancestors, not all earlier rows)
     int attn_rows_per_cta, prefetch_tiles;
     std::vector<FwdGraph>* graphs;
     uint64_t graph_clock;
@@ -505,15 +506,22 @@ swift_status launch_attn_mma(swift_ctx* ctx, const int* page_table, int block, b
 }
 
 // Attention of one block for the forward chunk's rows: split kernel + merge of the splits into `out` (fp32 rows)
-// and, when given, the hi/lo planes the next GEMM reads.  `full_model`: no sub-layer of this forward is skipped.  The
-// target model's forwards (verification, vanilla steps, prefill) take the tensor-core kernel, layer-skipped forwards
-// the streaming one; a row's result never depends on the row count within either family, which is what makes a
+// and, when given, the hi/lo planes the next GEMM reads.  `full_model`: no sub-layer of this forward is skipped.  Where
+// a tensor-core kernel is in use for decoding (grouped-query models by default, any model with SWIFT_ATTN_MMA=1), the target
+// model's forwards (verification of a chain, vanilla steps) take it and layer-skipped forwards the streaming one; a row's result never depends on the row count within either family, which is what makes a
 // vanilla step and the same row of a verification agree bit for bit.
 template <typename T>
 swift_status launch_attn(swift_ctx* ctx, int rows, const int* page_table, int block, float* out, __nv_bfloat16* planes,
                          bool full_model)
 {
     const swift_model_desc& d = ctx->d;
+    if (full_model && ctx->attn_tile_decode && !ctx->tree_forward) {
+        ST(launch_attn_tile<T>(ctx, page_table, block, rows, (int)ROWS, 0, 0, 0));
+        CU(launch_k(attn_combine_kernel, dim3(d.n_heads, rows), dim3(d.head_dim), 2 * (size_t)ctx->max_splits * sizeof(float), ctx,
+                    (const DevState*)state_of(ctx), (const float*)kptr<float>(ctx, ctx->kl.o_part),
+                    (const float2*)kptr<float2>(ctx, ctx->kl.ml_part), ctx->max_splits, d.n_heads, d.head_dim, out, planes, (int)ROWS, 0, 0, 0, 1));
+        return SWIFT_OK;
+    }
     if (d.head_dim == 128 && full_model && ctx->attn_mma) {
         const bool fused = rows == 1 && ctx->fuse_combine;
         const swift_status ms = (d.n_heads / d.n_kv_heads) * rows <= 8 ? launch_attn_mma<T, 1>(ctx, page_table, block, fused, out, planes)
@@ -829,7 +837,7 @@ swift_status forward_cached(swift_ctx* ctx, int rows, const int* toks_dev, const
 {
     if (!ctx->use_graphs) return forward_chunk_any(ctx, rows, toks_dev, skip, page_table, head);
     const int L = 2 * ctx->d.n_blocks;
-    FwdKey key{rows, head.run ? 1 : 0, head.mode, sampling_flag(ctx), ctx->use_tc ? 1 : 0, ctx->use_pdl ? 1 : 0, ctx->fuse ? 1 : 0, tree_cand(ctx, head) ? 1 : 0, ctx->temperature, ctx->top_p, toks_dev, page_table,
+    FwdKey key{rows, head.run ? 1 : 0, head.mode, sampling_flag(ctx), ctx->use_tc ? 1 : 0, ctx->use_pdl ? 1 : 0, ctx->fuse ? 1 : 0, (tree_cand(ctx, head) ? 1 : 0) | (ctx->tree_forward ? 2 : 0), ctx->temperature, ctx->top_p, toks_dev, page_table,
                skip ? std::vector<uint8_t>(skip, skip + L) : std::vector<uint8_t>()};
     auto& cache = *ctx->graphs;
     ctx->graph_clock++;
@@ -993,13 +1001,16 @@ swift_status enqueue_verify(swift_ctx* ctx, int rows_launch, int forced_k)
         const int budget = std::max(ctx->tree_rows, rows_launch);
         begin_verify_tree_kernel<<<1, 1, 0, ctx->stream>>>(st, ctx->n, kptr<int>(ctx, ctx->kl.cand), kptr<int>(ctx, ctx->kl.cand_n), budget);
         rows_launch = budget;
+        ctx->tree_forward = true;
     } else {
         begin_verify_kernel<<<1, 1, 0, ctx->stream>>>(st, ctx->n, forced_k);
     }
     ctx->launches++;
     HeadOpts head;
     head.run = true;
-    return forward_cached(ctx, rows_launch, st->draft_tok, nullptr, pt_main(ctx), head);
+    const swift_status fs = forward_cached(ctx, rows_launch, st->draft_tok, nullptr, pt_main(ctx), head);
+    ctx->tree_forward = false;
+    return fs;
 }
 
 swift_status enqueue_accept(swift_ctx* ctx)
@@ -1415,6 +1426,10 @@ swift_status swift_load(const swift_model_desc* desc, swift_devbuf weights, swif
     c->big_chunks = c->use_tc && c->fuse && big_rows_of(desc) == (size_t)TC_ROWS_MAX && getenv("SWIFT_NO_BIG_CHUNKS") == nullptr;
     c->whole_tiles = getenv("SWIFT_NO_WHOLE_TILES") == nullptr;
     c->attn_tile = getenv("SWIFT_NO_ATTN_TILE") == nullptr;      // chunks of many rows: 64-row query tiles with K,V staged in shared memory
+    // Grouped-query models: the target model's decoding forwards (verification, vanilla steps) take that kernel too, one
+    // CTA serving all query heads of a KV group, so that a K,V chunk is fetched and converted once per group
+    c->attn_tile_decode = c->attn_tile && desc->head_dim == 128 && desc->n_heads / desc->n_kv_heads >= 4 &&
+                          getenv("SWIFT_NO_ATTN_TILE_DECODE") == nullptr;
     c->batched_scoring = c->big_chunks && getenv("SWIFT_NO_BATCHED_SCORING") == nullptr;
     c->graphs = new std::vector<FwdGraph>();
     c->graph_clock = 0;
@@ -1687,7 +1702,10 @@ swift_status swift_verify_tree(swift_ctx* ctx, const int32_t* tokens_host, const
     ctx->launches++;
     HeadOpts head;
     head.run = true;
-    ST(forward_cached(ctx, n_rows, st->draft_tok, nullptr, pt_main(ctx), head));
+    ctx->tree_forward = true;
+    const swift_status fs = forward_cached(ctx, n_rows, st->draft_tok, nullptr, pt_main(ctx), head);
+    ctx->tree_forward = false;
+    ST(fs);
     DevState hs;
     ST(read_state(ctx, &hs));
     ctx->last_k = hs.n_drafted;
