@@ -259,6 +259,13 @@ swift_status swift_opt_observe(swift_opt* opt, const uint8_t* mask_host, float m
  * (that is the expected outcome); the call after it works normally. */
 swift_status swift_probe_wait_limit(swift_ctx* ctx, int32_t limit_us);
 
+/* Host-only query (no device is touched): the launch schedule of the many-row form of the tensor-core GEMM for an
+ * [N][K] weight: the grid (number of persistent CTAs, at most 148) into *grid_host and the largest number of CTAs that
+ * share one 128-row output tile into *max_share_host.  A chunk of many rows is bound by tensor work, so the stream-K cut
+ * is chosen per shape: whole tiles per CTA where the shape has enough tiles, tiles shared between CTAs where it has few.
+ * Returns SWIFT_EINVAL for null pointers or N, K < 1. */
+swift_status swift_many_row_schedule(int32_t N, int32_t K, int32_t* grid_host, int32_t* max_share_host);
+
 /* Selects the kernel behind the weight-streaming GEMMs: 1 = tensor cores (tcgen05 + TMA; default and
  * only sensible choice for bf16 models), 0 = the SIMT kernel (always used for fp32 models; for bf16 it
  * exists so that tests can check one kernel against the other).  No open round. */

@@ -55,7 +55,7 @@ SYMBOLS = ("swift_weights_bytes", "swift_kv_bytes", "swift_workspace_bytes", "sw
            "swift_last_error", "swift_pack_tensor", "swift_set_sampling", "swift_set_top_p", "swift_set_greedy_draft", "swift_forward_rows", "swift_prefill",
            "swift_set_pending", "swift_draft", "swift_verify", "swift_accept", "swift_score_skipsets", "swift_generate",
            "swift_committed_length", "swift_launch_count", "swift_round_times", "swift_round_bytes_stored", "swift_final_skip_mask", "swift_forward_bytes", "swift_read_kv", "swift_time_gemm", "swift_set_gemm_impl", "swift_gemm", "swift_gemm_static",
-           "swift_gemm_static_error", "swift_probe_wait_limit", "swift_set_tree", "swift_verify_tree", "swift_tree_rows", "swift_opt_create", "swift_opt_free", "swift_opt_suggest", "swift_opt_observe")
+           "swift_gemm_static_error", "swift_probe_wait_limit", "swift_many_row_schedule", "swift_set_tree", "swift_verify_tree", "swift_tree_rows", "swift_opt_create", "swift_opt_free", "swift_opt_suggest", "swift_opt_observe")
 
 _lib = None
 
@@ -95,6 +95,7 @@ def load_library(path: Optional[str] = None) -> C.CDLL:
     lib.swift_round_times.argtypes = [vp, i32, vp, vp, vp, vp, vp]
     lib.swift_round_times.restype = C.c_int32
     lib.swift_probe_wait_limit.argtypes = [vp, i32]
+    lib.swift_many_row_schedule.argtypes = [i32, i32, C.POINTER(C.c_int32), C.POINTER(C.c_int32)]
     lib.swift_set_tree.argtypes = [vp, i32]
     lib.swift_verify_tree.argtypes = [vp, vp, vp, i32, vp, vp]
     lib.swift_tree_rows.argtypes = [vp, vp, vp, vp]
@@ -199,6 +200,15 @@ class LayerSetOptimizer:
 
     def __del__(self):
         self.close()
+
+
+def many_row_schedule(n: int, k: int) -> Tuple[int, int]:
+    """(grid, largest number of CTAs sharing one output tile) of the many-row GEMM for an [n][k] weight; host only."""
+    grid, share = C.c_int32(), C.c_int32()
+    st = lib().swift_many_row_schedule(n, k, C.byref(grid), C.byref(share))
+    if st != 0:
+        raise SwiftError(f"swift_many_row_schedule({n}, {k}): status {st}")
+    return grid.value, share.value
 
 
 def gemm_static(w: torch.Tensor, x: torch.Tensor, y: torch.Tensor, stream: Optional[torch.cuda.Stream] = None) -> None:

@@ -1827,6 +1827,15 @@ swift_status swift_gemm(swift_ctx* ctx, int32_t which, int32_t block, const floa
     return read_state(ctx, &hs);
 }
 
+swift_status swift_many_row_schedule(int32_t N, int32_t K, int32_t* grid_host, int32_t* max_share_host)
+{
+    if (!grid_host || !max_share_host || N < 1 || K < 1) return SWIFT_EINVAL;
+    const int grid = many_row_grid(N, K);
+    *grid_host = grid;
+    *max_share_host = max_segments(N, K, grid);
+    return SWIFT_OK;
+}
+
 swift_status swift_probe_wait_limit(swift_ctx* ctx, int32_t limit_us)
 {
     if (!ctx) return SWIFT_EINVAL;

@@ -100,3 +100,32 @@ def test_proposal_engine_follows_the_oracles():
         lib.observe(mask, score(got))
     assert n_bayes == 8 and max(ref.y) >= 0.75
     lib.close()
+
+
+def test_many_row_gemm_schedule_on_the_host():
+    """The stream-K cut of the many-row GEMM (host logic, no device): never more than 148 CTAs; a shape with at least as
+    many tiles as fit takes whole tiles per CTA; a shape with few tiles and a long K shares each tile between CTAs, within
+    the number of slabs the workspace was sized for; every unit of work is covered exactly once by construction of the
+    cut, so what is checked here is the choice."""
+    from paper_2410_06916_b200 import many_row_schedule
+    import synth
+    tiles = lambda n: -(-n // 128)
+    for name in ("7b", "13b", "34b", "70b"):
+        c = synth.MODELS[name]
+        shapes = {"qkv": (c.q_dim + 2 * c.kv_dim, c.d_model), "o_proj": (c.d_model, c.q_dim), "gate_up": (2 * c.ffn, c.d_model),
+                  "down": (c.d_model, c.ffn), "head": (c.vocab, c.d_model)}
+        for what, (n, k) in shapes.items():
+            grid, share = many_row_schedule(n, k)
+            assert 74 <= grid <= 148 and share >= 1, (name, what, grid, share)
+            per_cta = tiles(n) / grid                      # tiles of work per CTA
+            if tiles(n) % grid == 0:
+                assert share == 1, (name, what)            # whole tiles: nothing shared
+            if tiles(n) <= 64:
+                assert share >= 2 and grid >= 2 * tiles(n) - 1, (name, what, grid, share)     # few tiles: cut along K
+            assert share <= 8 and per_cta <= 4, (name, what, grid, share)
+    assert many_row_schedule(15360, 5120) == (120, 1)      # 120 tiles: one each
+    assert many_row_schedule(5120, 5120) == (120, 3)       # 40 tiles: three CTAs to a tile
+    g, s = many_row_schedule(27648, 5120)                  # 216 tiles: three tiles to a pair of CTAs
+    assert (g, s) == (144, 2)
+    lib = __import__("paper_2410_06916_b200").load_library()
+    assert lib.swift_many_row_schedule(0, 64, None, None) == 1
