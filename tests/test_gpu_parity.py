@@ -21,6 +21,11 @@ BF16_SMALL = synth.ModelConfig("bf16-small", n_blocks=3, d_model=512, n_heads=8,
                                ffn=1376, vocab=3001, dtype="bf16", seed=21, n_planted=1, gain_std=0.05)
 
 
+# grouped-query attention with head_dim 128: the shape class whose target-model forwards decode on the tile attention kernel
+GQA128 = synth.ModelConfig("gqa128", n_blocks=3, d_model=1024, n_heads=8, n_kv_heads=2, head_dim=128,
+                           ffn=2816, vocab=3001, dtype="bf16", seed=23, n_planted=1, gain_std=0.05)
+
+
 @pytest.fixture(scope="module")
 def tiny_pair():
     o, g = make_pair(TINY, max_positions=192)
@@ -346,6 +351,42 @@ def test_gpu_swift_equals_gpu_vanilla_bf16(bf16_pair):
     kv2 = [g.read_kv(b, w, 0, n) for b in range(BF16_SMALL.n_blocks) for w in (0, 1)]
     for a, b in zip(kv, kv2):
         assert np.array_equal(a, b)
+
+
+def test_grouped_query_decoding_on_the_tile_kernel():
+    """A grouped-query model with head_dim 128 (four query heads per KV head): chain verifications and vanilla steps run
+    their attention on the tile kernel (one CTA per KV head and chunk for the whole group), layer-skipped drafts and
+    token-tree verifications on the streaming kernel.  Rounds against the oracle step by step behind a 270-token prompt
+    (several chunks, a ragged last one), token-tree rounds after them, and whole runs: greedy SWIFT equals greedy vanilla
+    decoding on the GPU for every skip set."""
+    from paper_2410_06916_b200 import GenParams
+    cfg = GQA128
+    o, g = make_pair(cfg, max_positions=640)
+    try:
+        prompt = synth.prompt(cfg, 270)
+        o.prefill(prompt); g.prefill(prompt); g.set_pending(o.tokens[-1])
+        z = list(synth.block_mask(cfg, synth.planted_blocks(cfg)))
+        st = walk_rounds(o, g, z, n_rounds=8, max_k=8)
+        print("grouped-query rounds:", st)
+        assert st["max_logit_err"] < LOGIT_TOL and st["accept_cmp"] >= 6, st
+        g.set_tree(16)
+        ts = _tree_stats()
+        try:
+            for _ in range(6):
+                _tree_round(o, g, z, 8, 16, ts)
+        finally:
+            g.set_tree(0)
+        print("grouped-query tree rounds:", ts)
+        assert ts["rounds"] >= 5 and ts["accept_cmp"] >= ts["rounds"] - 2, ts
+        prompt = synth.prompt(cfg, 64)
+        van, _, _ = g.generate(prompt, GenParams(max_new=40, vanilla=True))
+        for blocks, k in (([1], 8), ([0, 2], 5), ([], 15)):
+            out, gst, _ = g.generate(prompt, GenParams(max_new=40, max_draft=k, skip_mask=synth.block_mask(cfg, blocks)))
+            assert out == van, blocks
+            if not blocks:
+                assert gst.accepted == gst.drafted
+    finally:
+        g.close()
 
 
 # ------------------------------------------------------------------------------ scoring
