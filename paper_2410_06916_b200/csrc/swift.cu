@@ -1428,7 +1428,8 @@ swift_status swift_load(const swift_model_desc* desc, swift_devbuf weights, swif
     c->attn_tile = getenv("SWIFT_NO_ATTN_TILE") == nullptr;      // chunks of many rows: 64-row query tiles with K,V staged in shared memory
     // Grouped-query models: the target model's decoding forwards (verification, vanilla steps) take that kernel too, one
     // CTA serving all query heads of a KV group, so that a K,V chunk is fetched and converted once per group
-    c->attn_tile_decode = c->attn_tile && desc->head_dim == 128 && desc->n_heads / desc->n_kv_heads >= 4 &&
+    c->attn_tile_decode = c->attn_tile && desc->head_dim == 128 &&
+                          (desc->n_heads / desc->n_kv_heads >= 4 || getenv("SWIFT_ATTN_TILE_DECODE") != nullptr) &&
                           getenv("SWIFT_NO_ATTN_TILE_DECODE") == nullptr;
     c->batched_scoring = c->big_chunks && getenv("SWIFT_NO_BATCHED_SCORING") == nullptr;
     c->graphs = new std::vector<FwdGraph>();
