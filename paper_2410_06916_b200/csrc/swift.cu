@@ -82,7 +82,7 @@ struct swift_ctx {
     std::string err;
     cudaEvent_t ev[8];
     // captured forwards; programmatic dependent launch between the kernels of a forward
-    bool use_graphs, use_pdl, pdl_next, pdl_gemms, fuse, fuse_combine, prefetch_next, attn_mma, big_chunks, batched_scoring, whole_tiles, attn_tile, attn_tile_decode;
+    bool use_graphs, use_pdl, pdl_next, pdl_gemms, fuse, fuse_combine, prefetch_next, attn_mma, big_chunks, batched_scoring, whole_tiles, attn_tile, attn_tile_decode, attn_tile_drafts;
     bool tree_forward = false;      // the forward being enqueued verifies a token tree (rows see their ancestors, not all earlier rows)
     int attn_rows_per_cta, prefetch_tiles;
     std::vector<FwdGraph>* graphs;
@@ -507,15 +507,16 @@ swift_status launch_attn_mma(swift_ctx* ctx, const int* page_table, int block, b
 
 // Attention of one block for the forward chunk's rows: split kernel + merge of the splits into `out` (fp32 rows)
 // and, when given, the hi/lo planes the next GEMM reads.  `full_model`: no sub-layer of this forward is skipped.  Where
-// a tensor-core kernel is in use for decoding (grouped-query models by default, any model with SWIFT_ATTN_MMA=1), the target
-// model's forwards (verification of a chain, vanilla steps) take it and layer-skipped forwards the streaming one; a row's result never depends on the row count within either family, which is what makes a
+// a tensor-core kernel is in use for decoding, the target model's forwards (verification of a chain, vanilla steps) all take
+// the same one (grouped-query models: the tile kernel, which their layer-skipped forwards take as well; SWIFT_ATTN_MMA=1: the
+// swapped kernel, layer-skipped forwards on the streaming one); a row's result never depends on the row count within either family, which is what makes a
 // vanilla step and the same row of a verification agree bit for bit.
 template <typename T>
 swift_status launch_attn(swift_ctx* ctx, int rows, const int* page_table, int block, float* out, __nv_bfloat16* planes,
                          bool full_model)
 {
     const swift_model_desc& d = ctx->d;
-    if (full_model && ctx->attn_tile_decode && !ctx->tree_forward) {
+    if ((full_model || ctx->attn_tile_drafts) && ctx->attn_tile_decode && !ctx->tree_forward) {
         ST(launch_attn_tile<T>(ctx, page_table, block, rows, (int)ROWS, 0, 0, 0));
         CU(launch_k(attn_combine_kernel, dim3(d.n_heads, rows), dim3(d.head_dim), 2 * (size_t)ctx->max_splits * sizeof(float), ctx,
                     (const DevState*)state_of(ctx), (const float*)kptr<float>(ctx, ctx->kl.o_part),
@@ -1431,6 +1432,7 @@ swift_status swift_load(const swift_model_desc* desc, swift_devbuf weights, swif
     c->attn_tile_decode = c->attn_tile && desc->head_dim == 128 &&
                           (desc->n_heads / desc->n_kv_heads >= 4 || getenv("SWIFT_ATTN_TILE_DECODE") != nullptr) &&
                           getenv("SWIFT_NO_ATTN_TILE_DECODE") == nullptr;
+    c->attn_tile_drafts = getenv("SWIFT_NO_ATTN_TILE_DRAFTS") == nullptr;   // and so do its layer-skipped forwards (70B shape: +2 %)
     c->batched_scoring = c->big_chunks && getenv("SWIFT_NO_BATCHED_SCORING") == nullptr;
     c->graphs = new std::vector<FwdGraph>();
     c->graph_clock = 0;
