@@ -50,7 +50,11 @@ constexpr long long TC_WAIT_CYCLES = 3000000000LL;  // ~1.5 s of SM clocks befor
 // The same kernel serves forwards of up to 16 rows (NB = 1: decoding) and of up to 16 * NB rows (NB = 2, 4, 8: prefill
 // chunks and candidate scoring).  Rows come in blocks of 16; block rb occupies operand rows / accumulator columns
 // [32 rb, 32 rb + 32): its 16 hi rows, then its 16 lo rows.  More rows per weight tile mean a wider MMA (N = 32 NB), a
-// larger activation tile per stage and fewer stages in the same shared memory.
+// larger activation tile per stage and fewer stages in the same shared memory.  With many rows the kernel is bound by
+// tensor work, not by HBM: the host then picks the grid per shape (whole tiles per CTA where a shape has enough tiles,
+// tiles shared between a few CTAs where it has too few to occupy the SMs), a shared tile's partial accumulators are
+// parked as the 16 values each epilogue thread holds, and the epilogue finishes one 16-row block at a time with the
+// global-memory operands of the next block already requested.
 template <int NB>
 struct TcShape {
     static constexpr int COLS = TC_COLS * NB;                        // MMA N
