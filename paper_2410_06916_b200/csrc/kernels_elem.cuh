@@ -307,8 +307,9 @@ namespace swk {
 
 // ------------------------------------------------------------------------------ candidate scoring, all candidates at once
 // Every candidate skip set keeps its own copy of the window's residual rows in H_all[c * gamma + i]; a sub-layer is
-// applied to the candidates that keep it, gathered into chunks of up to 128 rows, and scattered back (Eq. 2 evaluates
-// all candidates on the same gamma context tokens, "Parallel Candidate Evaluation", Section 4.1).
+// applied to the candidates that keep it, their rows taken in chunks of up to 128 through a row map: the norm's planes
+// are gathered, the sub-layer's last GEMM adds to the residual rows in place (Eq. 2 evaluates all candidates on the same
+// gamma context tokens, "Parallel Candidate Evaluation", Section 4.1).
 
 // H_all[row] = embedding of the window token row % gamma.  grid = rows, any block size.
 template <typename T>
@@ -325,9 +326,10 @@ __global__ void embed_rows_kernel(DevState* st, const int* __restrict__ toks, co
     for (int i = threadIdx.x; i < d; i += blockDim.x) H_all[(size_t)row * d + i] = to_float(src[i]);
 }
 
-// Chunk row r <- H_all[rowmap[r]]: copies the residual row into the chunk's h, stores the hi/lo planes of h * gain (the
-// input of the sub-layer's first GEMM) and the row's sum of squares as "tile 0".  grid = chunk rows, block = 1024.
-__global__ void gather_norm_kernel(const int* __restrict__ rowmap, const float* __restrict__ H_all, float* __restrict__ h,
+// Chunk row r = H_all[rowmap[r]]: stores the hi/lo planes of that residual row * gain (the input of the sub-layer's
+// first GEMM) and the row's sum of squares as "tile 0"; the residual row itself stays where it is (the sub-layer's last
+// GEMM adds to it in place, through the same map).  grid = chunk rows, block = 1024.
+__global__ void gather_norm_kernel(const int* __restrict__ rowmap, const float* __restrict__ H_all,
                                    const float* __restrict__ gain, __nv_bfloat16* __restrict__ planes, float* __restrict__ sumsq_out, int d)
 {
     __shared__ float red[33];
@@ -336,20 +338,11 @@ __global__ void gather_norm_kernel(const int* __restrict__ rowmap, const float* 
     float ss = 0.f;
     for (int i = threadIdx.x; i < d; i += blockDim.x) {
         const float v = src[i];
-        h[(size_t)r * d + i] = v;
         store_hi_lo(planes, r, d, i, v * gain[i]);
         ss += v * v;
     }
     const float total = block_sum(ss, red);
     if (threadIdx.x == 0) sumsq_out[r] = total;
-}
-
-// H_all[rowmap[r]] <- chunk row r.  grid = chunk rows.
-__global__ void scatter_rows_kernel(const int* __restrict__ rowmap, const float* __restrict__ h, float* __restrict__ H_all, int d)
-{
-    const int r = blockIdx.x;
-    float* dst = H_all + (size_t)rowmap[r] * d;
-    for (int i = threadIdx.x; i < d; i += blockDim.x) dst[i] = h[(size_t)r * d + i];
 }
 
 // out[row] = arg max of logits[row][:], lowest token id among equals.  grid = rows, block = 1024.

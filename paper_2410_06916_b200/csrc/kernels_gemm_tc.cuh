@@ -203,6 +203,8 @@ struct EpiParams {
     float inv_d, eps;
     // EPI_RESID
     float* h;                       // [ROWS][N] residual stream
+    const int* h_rows;              // many-row form only: the 16-row block that starts at chunk row r lives in rows h_rows[r] ..
+                                    // h_rows[r] + 15 of h (only multiples of 16 are looked up; null: rows r .. r + 15)
     const float* gain_next;         // [N] gain of the next RMSNorm, or null when nothing follows
     __nv_bfloat16* planes_out;      // [2*ROWS][N]
     float* sumsq_out;               // [n_tiles][ROWS]
@@ -510,8 +512,9 @@ gemm_tc_kernel(DevState* st, const __grid_constant__ CUtensorMap mapW, const __g
             auto prefetch = [&](int rb, int n, ManyPre& p) {
                 const int row0 = rb * ROWS, rows_here = min(ROWS, n_rows - row0);
                 if (EPI == EPI_RESID) {
+                    const float* hb = ep.h + (size_t)(ep.h_rows ? __ldg(ep.h_rows + row0) : row0) * N + n;
 #pragma unroll
-                    for (int m = 0; m < ROWS; ++m) p.h[m] = (n < N && m < rows_here) ? __ldcg(ep.h + (size_t)(row0 + m) * N + n) : 0.f;
+                    for (int m = 0; m < ROWS; ++m) p.h[m] = (n < N && m < rows_here) ? __ldcg(hb + (size_t)m * N) : 0.f;
                 } else if (EPI == EPI_QKV) {
                     const int pos_b = ep.per_block ? ep.rb_pos0[rb] : pos0_epi + row0;     // cache slot of the block's first row
                     const int* pt = ep.per_block ? ep.rb_page_table[rb] : ep.page_table;
@@ -551,12 +554,13 @@ gemm_tc_kernel(DevState* st, const __grid_constant__ CUtensorMap mapW, const __g
                     }
                 } else if (EPI == EPI_RESID) {
                     float sq[ROWS];
+                    float* hb = ep.h + (size_t)(ep.h_rows ? __ldg(ep.h_rows + row0) : row0) * N + n;
 #pragma unroll
                     for (int m = 0; m < ROWS; ++m) {
                         const float hn = p.h[m] + val[m];
                         const bool ok = n < N && m < rows_here;
                         if (ok) {
-                            ep.h[(size_t)(row0 + m) * N + n] = hn;
+                            hb[(size_t)m * N] = hn;
                             if (ep.gain_next) store_hi_lo(ep.planes_out, row0 + m, N, n, hn * gain);
                         }
                         sq[m] = ok ? hn * hn : 0.f;

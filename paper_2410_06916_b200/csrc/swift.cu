@@ -1143,7 +1143,6 @@ swift_status enqueue_score_batched(swift_ctx* ctx, const uint8_t* masks, int C, 
     }
     // ---- the walk
     const int dm = d.d_model, qd = d.n_heads * d.head_dim, kd = d.n_kv_heads * d.head_dim, nqkv = qd + 2 * kd;
-    float* h = kptr<float>(ctx, ctx->kl.h);
     float* xa = kptr<float>(ctx, ctx->kl.xa);
     __nv_bfloat16* xn_hl = kptr<__nv_bfloat16>(ctx, ctx->kl.xn_hl);
     __nv_bfloat16* xa_hl = kptr<__nv_bfloat16>(ctx, ctx->kl.xa_hl);
@@ -1166,7 +1165,7 @@ swift_status enqueue_score_batched(swift_ctx* ctx, const uint8_t* masks, int C, 
         set_rows_kernel<<<1, 1, 0, ctx->stream>>>(st, pos_w, rows);
         ctx->launches++;
         if (ch.sub == L) {                            // output head: final norm, logits, arg max per row
-            gather_norm_kernel<<<rows, 1024, 0, ctx->stream>>>(map, H_all, h, wptr<float>(ctx, ctx->wl.final_norm), xn_hl, sumsq, dm);
+            gather_norm_kernel<<<rows, 1024, 0, ctx->stream>>>(map, H_all, wptr<float>(ctx, ctx->wl.final_norm), xn_hl, sumsq, dm);
             ctx->launches++;
             ST((launch_gemm_tc_y<NB>(ctx, GemmSite{nullptr, d.vocab, dm, nullptr, &ctx->tm_lm_head, &ctx->tm_xn_big}, base, logits)));
             // the head's chunks hold consecutive candidates: their predictions go where their rows are in H_all
@@ -1176,9 +1175,10 @@ swift_status enqueue_score_batched(swift_ctx* ctx, const uint8_t* masks, int C, 
         }
         const int b = ch.sub >> 1;
         EpiParams resid = base;
-        resid.h = h;                                  // h += branch output; nothing chained: the next sub-layer regroups the rows
+        resid.h = H_all;                              // the rows' residual stream, in place through the map; nothing chained:
+        resid.h_rows = map;                           // the next sub-layer regroups the rows
         if (!(ch.sub & 1)) {
-            gather_norm_kernel<<<rows, 1024, 0, ctx->stream>>>(map, H_all, h, wptr<float>(ctx, ctx->wl.attn_norm[b]), xn_hl, sumsq, dm);
+            gather_norm_kernel<<<rows, 1024, 0, ctx->stream>>>(map, H_all, wptr<float>(ctx, ctx->wl.attn_norm[b]), xn_hl, sumsq, dm);
             ctx->launches++;
             EpiParams ep = base;
             ep.q_out = kptr<float>(ctx, ctx->kl.q); ep.kv_pool = ctx->kvbase; ep.page_table = pt_dev; ep.L = ctx->kv;
@@ -1203,15 +1203,13 @@ swift_status enqueue_score_batched(swift_ctx* ctx, const uint8_t* masks, int C, 
                         ctx->max_splits, d.n_heads, d.head_dim, xa, xa_hl, (int)TC_ROWS_MAX, 0, gamma, pos_w, ch.n_cand));
             ST((launch_gemm_tc<EPI_RESID, float, NB>(ctx, GemmSite{nullptr, dm, qd, nullptr, &ctx->tm_wo[b], &ctx->tm_xa_big}, resid)));
         } else {
-            gather_norm_kernel<<<rows, 1024, 0, ctx->stream>>>(map, H_all, h, wptr<float>(ctx, ctx->wl.mlp_norm[b]), xn_hl, sumsq, dm);
+            gather_norm_kernel<<<rows, 1024, 0, ctx->stream>>>(map, H_all, wptr<float>(ctx, ctx->wl.mlp_norm[b]), xn_hl, sumsq, dm);
             ctx->launches++;
             EpiParams sw = base;
             sw.act_planes = act_hl; sw.ffn = d.ffn;
             ST((launch_gemm_tc<EPI_SWIGLU, float, NB>(ctx, GemmSite{nullptr, 2 * d.ffn, dm, nullptr, &ctx->tm_wgu[b], &ctx->tm_xn_big}, sw)));
             ST((launch_gemm_tc<EPI_RESID, float, NB>(ctx, GemmSite{nullptr, dm, d.ffn, nullptr, &ctx->tm_wdown[b], &ctx->tm_act_big}, resid)));
         }
-        scatter_rows_kernel<<<rows, 256, 0, ctx->stream>>>(map, h, H_all, dm);
-        ctx->launches++;
     }
     match_rows_kernel<<<ceil_div(C, 128), 128, 0, ctx->stream>>>(pred, truth_dev, gamma, C, kptr<int>(ctx, ctx->kl.score_out));
     ctx->launches++;
