@@ -466,6 +466,14 @@ def main():
            "e2e": {"value": e2e, "unit": UNIT, "h2d_bytes_per_step": s0.h2d_bytes, "d2h_bytes_per_step": s0.d2h_bytes},
            "gpu_launches": launches, "clocks": clk.summary()}
 
+    if cfg.dtype == "bf16" and cfg.head_dim == 128:
+        # Prefill runs in 128-row chunks through the many-row form of the GEMM: tensor work, two bf16 products (hi and lo
+        # activation planes) per weight of every block per prompt token (the output head sees one row only).
+        pf_flops = 2 * 2.0 * run.prompt_len * cfg.n_blocks * cfg.block_params()
+        pf_tflops = pf_flops / (s0.ms_prefill * 1e-3) * 1e-12
+        out["prefill"] = {"ms": s0.ms_prefill, "tokens": run.prompt_len, "bound": "tensor (128 rows per weight tile, hi and lo bf16 products)",
+                          "tflops_hi_lo": pf_tflops, "peak_tflops": tensor_peak, "frac": pf_tflops / tensor_peak}
+
     # Dynamic verification (Section 4.2): the same run with the skip set the main run ended with, verifying the chain alone
     # and verifying a token tree of up to 16 rows (greedy decoding only)
     if not sampling and run.max_draft > 0:
