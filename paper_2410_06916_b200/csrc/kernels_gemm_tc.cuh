@@ -67,7 +67,10 @@ struct TcShape {
     static constexpr int ROWS_MAX = ROWS * NB;
 };
 constexpr int TC_NB_MAX = 8;
-constexpr int TC_ROWS_MAX = ROWS * TC_NB_MAX;       // rows of the largest forward chunk
+constexpr int TC_ROWS_MAX = ROWS * TC_NB_MAX;       // rows one accumulator tile covers (the wide form's "problem")
+constexpr int TC_PROBS_MAX = 2;                     // problems a launch of the wide form may hold: row ranges of TC_ROWS_MAX rows that share
+                                                    // the weights but nothing else; work tile T = weight tile T / n_prob of problem T % n_prob
+constexpr int TC_BIG_ROWS = TC_ROWS_MAX * TC_PROBS_MAX;   // rows of the largest forward chunk
 constexpr int TC_ERR_TIMEOUT = 2;
 
 // ------------------------------------------------------------------------------ PTX wrappers
@@ -222,8 +225,8 @@ struct EpiParams {
     // EPI_QKV on a chunk that holds several sequences side by side (candidate scoring: every candidate's window rows, each
     // with its own scratch pages): per 16-row block, the cache slot of its first row and the page table of its sequence
     int per_block;
-    int rb_pos0[8];
-    const int* rb_page_table[8];
+    int rb_pos0[8 * TC_PROBS_MAX];
+    const int* rb_page_table[8 * TC_PROBS_MAX];
     // any epilogue: shape of the GEMM that runs next on this stream (0 = none): each CTA asks for the first
     // weight tiles it will need there to be brought into L2 while this launch drains
     int next_N, next_K, next_tiles;
@@ -335,18 +338,22 @@ template <int EPI, typename TKV, int NB = 1>
 __global__ void __launch_bounds__(TC_THREADS, 1)
 gemm_tc_kernel(DevState* st, const __grid_constant__ CUtensorMap mapW, const __grid_constant__ CUtensorMap mapX,
                float* __restrict__ Y, float* __restrict__ slabs, int* __restrict__ counters, int N, int K,
-               const __grid_constant__ EpiParams ep, const __grid_constant__ CUtensorMap mapNext)
+               const __grid_constant__ EpiParams ep, const __grid_constant__ CUtensorMap mapNext, int n_prob_arg)
 {
     typedef TcShape<NB> S;
     pdl_trigger();
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-    const int n_tiles = (N + TC_TILE_N - 1) / TC_TILE_N;
+    const int n_prob = NB > 1 ? n_prob_arg : 1;                     // problems of this launch (wide form only)
+    const int n_tiles = ((N + TC_TILE_N - 1) / TC_TILE_N) * n_prob; // work tiles
     StreamK sk;
     sk.KB = (K + TC_BK - 1) / TC_BK;
     sk.U = (long long)n_tiles * sk.KB;
     sk.G = (int)(sk.U < (long long)gridDim.x ? sk.U : (long long)gridDim.x);   // never more CTAs than units: no empty ranges
     if ((int)blockIdx.x >= sk.G) { pdl_wait(); return; }
     const long long u_begin = sk.start(blockIdx.x), u_end = sk.start(blockIdx.x + 1);
+    // weight rows and activation-plane rows of work tile t (the wide form: problem t % n_prob reads the plane rows of its own row range)
+    auto w_row = [&](int t) { return (NB > 1 ? t / n_prob : t) * TC_TILE_N; };
+    auto x_row = [&](int t) { return NB > 1 ? (t % n_prob) * S::COLS : 0; };
 
     extern __shared__ unsigned char smem_raw[];
     const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;        // swizzled tiles need 1024-byte alignment
@@ -358,7 +365,7 @@ gemm_tc_kernel(DevState* st, const __grid_constant__ CUtensorMap mapW, const __g
     __shared__ uint32_t tmem_base_sh;
     __shared__ int last_flag_sh, peek_sh;
     __shared__ int abort_sh, epi_abort_sh;
-    __shared__ float rstd_sh[ROWS * NB];
+    __shared__ float rstd_sh[ROWS * NB * (NB > 1 ? TC_PROBS_MAX : 1)];
     __shared__ float stage_sh[EPI == EPI_PLAIN ? 4 * ROWS : (NB > 1 && EPI == EPI_QKV ? 2 : 1) * ROWS * TC_TILE_N + 8 * ROWS];
     __shared__ float2 rope_sh[EPI == EPI_QKV && NB == 1 ? ROWS * (TC_TILE_N / 2) : 1];   // (cos, sin) of the rows' positions
     __shared__ int page_sh[ROWS];                                              // KV page of each row's position
@@ -380,12 +387,12 @@ gemm_tc_kernel(DevState* st, const __grid_constant__ CUtensorMap mapW, const __g
         int tile0 = (int)(u_begin / sk.KB), kb0 = (int)(u_begin - (long long)tile0 * sk.KB);
         for (int i = 0, t = tile0, k = kb0; i < n_pre0; ++i, (++k == sk.KB ? (k = 0, ++t) : 0)) {
             mbar_expect_tx(full_bar(i), S::STAGE_BYTES);
-            tma_load_2d(base + i * S::STAGE_BYTES, &mapW, k * TC_BK, t * TC_TILE_N, full_bar(i));
+            tma_load_2d(base + i * S::STAGE_BYTES, &mapW, k * TC_BK, w_row(t), full_bar(i));
         }
         pdl_wait();
         n_rows_early = st->n_rows;
-        for (int i = 0, k = kb0; i < n_pre0; ++i, (++k == sk.KB ? (k = 0) : 0))
-            tma_load_2d(base + i * S::STAGE_BYTES + TC_A_BYTES, &mapX, k * TC_BK, 0, full_bar(i));
+        for (int i = 0, t = tile0, k = kb0; i < n_pre0; ++i, (++k == sk.KB ? (k = 0, ++t) : 0))
+            tma_load_2d(base + i * S::STAGE_BYTES + TC_A_BYTES, &mapX, k * TC_BK, x_row(t), full_bar(i));
     }
     if (warp == 1) {   // this warp sets up the remaining barriers and allocates 64 TMEM columns: two accumulator buffers of 32
         if (lane == 0) {
@@ -420,8 +427,8 @@ gemm_tc_kernel(DevState* st, const __grid_constant__ CUtensorMap mapW, const __g
                 if (!mbar_wait(empty_bar(s), ((it / S::STAGES) & 1) ^ 1)) { abort_sh = 1; break; }
                 const uint32_t a_dst = base + s * S::STAGE_BYTES, b_dst = a_dst + TC_A_BYTES;
                 mbar_expect_tx(full_bar(s), S::STAGE_BYTES);
-                tma_load_2d(a_dst, &mapW, kb * TC_BK, tile * TC_TILE_N, full_bar(s));
-                tma_load_2d(b_dst, &mapX, kb * TC_BK, 0, full_bar(s));
+                tma_load_2d(a_dst, &mapW, kb * TC_BK, w_row(tile), full_bar(s));
+                tma_load_2d(b_dst, &mapX, kb * TC_BK, x_row(tile), full_bar(s));
             }
             }
             if (ep.next_K > 0) {                        // everything of this launch is requested: now the next one's start
@@ -475,14 +482,14 @@ gemm_tc_kernel(DevState* st, const __grid_constant__ CUtensorMap mapW, const __g
         const int etid = tid - 64;                     // 0..127
         int seg = 0;
         long long u = n_rows != 0 ? u_begin : u_end;
-        if (etid < ROWS * NB) {                        // rstd of the RMSNorm in front of this GEMM (1 when there is none)
+        for (int i = etid; i < ROWS * NB * n_prob; i += 128) {   // rstd of the RMSNorm in front of this GEMM (1 when there is none)
             float r = 1.f;
             if (EPI != EPI_RESID && ep.sumsq_in) {
                 float ss = 0.f;
-                for (int t = 0; t < ep.n_sumsq_tiles; ++t) ss += ep.sumsq_in[(size_t)t * ep.sum_rows + etid];
+                for (int t = 0; t < ep.n_sumsq_tiles; ++t) ss += ep.sumsq_in[(size_t)t * ep.sum_rows + i];
                 r = rsqrtf(ss * ep.inv_d + ep.eps);
             }
-            rstd_sh[etid] = r;
+            rstd_sh[i] = r;
         }
         if (EPI == EPI_QKV && NB == 1) {
             const int half = ep.L.head_dim >> 1, pos0 = pos0_epi;
@@ -504,20 +511,21 @@ gemm_tc_kernel(DevState* st, const __grid_constant__ CUtensorMap mapW, const __g
             // row loops are unrolled (this code runs NB times per tile: it is warm), and the staging buffers alternate
             // between blocks so that one barrier per block suffices.
             constexpr int RT = ROWS * NB;
-            const int live_blocks = (n_rows + ROWS - 1) / ROWS;
+            int R0 = 0;                                   // first row of the problem the current work tile belongs to
+            int live_blocks = 0;                          // 16-row blocks of that problem that hold rows
             const int l = quarter * 32 + lane;
             const size_t slab_stride = (size_t)n_tiles * TC_TILE_N * RT;     // one CTA's parked partial tiles
             float* sums_sh = stage_sh + (EPI == EPI_QKV ? 2 : 1) * ROWS * TC_TILE_N;      // [2][4 * ROWS]
             struct ManyPre { float h[ROWS]; float2 cs[ROWS]; int page[ROWS]; };
             auto prefetch = [&](int rb, int n, ManyPre& p) {
-                const int row0 = rb * ROWS, rows_here = min(ROWS, n_rows - row0);
+                const int row0 = R0 + rb * ROWS, rows_here = min(ROWS, n_rows - row0);
                 if (EPI == EPI_RESID) {
                     const float* hb = ep.h + (size_t)(ep.h_rows ? __ldg(ep.h_rows + row0) : row0) * N + n;
 #pragma unroll
                     for (int m = 0; m < ROWS; ++m) p.h[m] = (n < N && m < rows_here) ? __ldcg(hb + (size_t)m * N) : 0.f;
                 } else if (EPI == EPI_QKV) {
-                    const int pos_b = ep.per_block ? ep.rb_pos0[rb] : pos0_epi + row0;     // cache slot of the block's first row
-                    const int* pt = ep.per_block ? ep.rb_page_table[rb] : ep.page_table;
+                    const int pos_b = ep.per_block ? ep.rb_pos0[row0 / ROWS] : pos0_epi + row0;     // cache slot of the block's first row
+                    const int* pt = ep.per_block ? ep.rb_page_table[row0 / ROWS] : ep.page_table;
                     const int dh = ep.L.head_dim, half = dh >> 1, i = n % dh, j = i < half ? i : i - half;
 #pragma unroll
                     for (int m = 0; m < ROWS; ++m) {
@@ -528,8 +536,8 @@ gemm_tc_kernel(DevState* st, const __grid_constant__ CUtensorMap mapW, const __g
                     }
                 }
             };
-            auto finish_many = [&](int rb, float (&val)[ROWS], int tile, int n, const ManyPre& p, float gain) {
-                const int row0 = rb * ROWS, rows_here = min(ROWS, n_rows - row0);
+            auto finish_many = [&](int rb, float (&val)[ROWS], int tile, int n, const ManyPre& p, float gain) {   // tile: the weight tile
+                const int row0 = R0 + rb * ROWS, rows_here = min(ROWS, n_rows - row0);
                 if (EPI != EPI_RESID) {
 #pragma unroll
                     for (int m = 0; m < ROWS; ++m) val[m] *= rstd_sh[row0 + m];
@@ -594,7 +602,7 @@ gemm_tc_kernel(DevState* st, const __grid_constant__ CUtensorMap mapW, const __g
                     const int dh = ep.L.head_dim, half = dh >> 1;
                     const int gh = n / dh, i = n - gh * dh;
                     const int lp = i < half ? l + half : l - half;
-                    const int pos_b = ep.per_block ? ep.rb_pos0[rb] : pos0_epi + row0;
+                    const int pos_b = ep.per_block ? ep.rb_pos0[row0 / ROWS] : pos0_epi + row0;
                     TKV* pool = reinterpret_cast<TKV*>(ep.kv_pool);
                     const int hk = gh - ep.n_heads;
                     const int kv = hk >= ep.L.n_kv_heads ? 1 : 0;
@@ -618,7 +626,10 @@ gemm_tc_kernel(DevState* st, const __grid_constant__ CUtensorMap mapW, const __g
                 const long long tile_end = (long long)(tile + 1) * sk.KB;
                 const long long seg_end = tile_end < u_end ? tile_end : u_end;
                 const int buf = seg & 1;
-                const int n = tile * TC_TILE_N + l;
+                const int wt = tile / n_prob;              // weight tile; the problem is tile % n_prob
+                R0 = (tile - wt * n_prob) * RT;
+                live_blocks = (min(n_rows - R0, RT) + ROWS - 1) / ROWS;
+                const int n = wt * TC_TILE_N + l;
                 const bool whole = (kb0 == 0) && (seg_end == tile_end);
                 int slab = 0, nseg = 1;
                 if (!whole) {
@@ -655,7 +666,7 @@ gemm_tc_kernel(DevState* st, const __grid_constant__ CUtensorMap mapW, const __g
 #pragma unroll
                     for (int m = 0; m < ROWS; ++m) val[m] = __uint_as_float(v[m]) + __uint_as_float(v[16 + m]);
                     if (whole) {
-                        finish_many(rb, val, tile, n, pre, gain);
+                        finish_many(rb, val, wt, n, pre, gain);
                         pre = nxt;
                     } else {                                   // parked as this thread's 16 values side by side
                         float4* mine = reinterpret_cast<float4*>(slabs + (size_t)slab * slab_stride + (((size_t)tile * NB + rb) * TC_TILE_N + l) * ROWS);
@@ -712,7 +723,7 @@ gemm_tc_kernel(DevState* st, const __grid_constant__ CUtensorMap mapW, const __g
                                     val[4 * q4] += x.x; val[4 * q4 + 1] += x.y; val[4 * q4 + 2] += x.z; val[4 * q4 + 3] += x.w;
                                 }
                             }
-                            finish_many(rb, val, tile, n, pre, gain);
+                            finish_many(rb, val, wt, n, pre, gain);
                             pre = nxt;
                             if (AHEAD) {
 #pragma unroll

@@ -12,6 +12,7 @@
 #include <cstring>
 #include <string>
 #include <map>
+#include <tuple>
 #include <mutex>
 #include <vector>
 
@@ -82,7 +83,7 @@ struct swift_ctx {
     std::string err;
     cudaEvent_t ev[8];
     // captured forwards; programmatic dependent launch between the kernels of a forward
-    bool use_graphs, use_pdl, pdl_next, pdl_gemms, fuse, fuse_combine, prefetch_next, attn_mma, big_chunks, batched_scoring, whole_tiles, attn_tile, attn_tile_decode, attn_tile_drafts;
+    bool use_graphs, use_pdl, pdl_next, pdl_gemms, fuse, fuse_combine, prefetch_next, attn_mma, big_chunks, batched_scoring, whole_tiles, attn_tile, attn_tile_decode, attn_tile_drafts, two_problems;
     bool tree_forward = false;      // the forward being enqueued verifies a token tree (rows see their ancestors, not all earlier rows)
     int attn_rows_per_cta, prefetch_tiles;
     std::vector<FwdGraph>* graphs;
@@ -95,7 +96,7 @@ struct swift_ctx {
     bool use_tc;
     std::vector<CUtensorMap> tm_wqkv, tm_wo, tm_wgu, tm_wdown;
     CUtensorMap tm_lm_head, tm_embed, tm_xn, tm_xa, tm_act;
-    CUtensorMap tm_xn_big, tm_xa_big, tm_act_big;      // the same planes seen as 2 * TC_ROWS_MAX operand rows (chunks of many rows)
+    CUtensorMap tm_xn_big, tm_xa_big, tm_act_big;      // the same planes seen as 2 * TC_BIG_ROWS operand rows, boxes of 2 * TC_ROWS_MAX (chunks of many rows)
 };
 
 namespace {
@@ -193,11 +194,11 @@ constexpr int TC_GRID = 148;        // persistent CTAs of the tensor-core GEMM: 
 constexpr int TC_MAX_TILES = 1024;
 
 // Largest number of CTAs that share one output tile under the stream-K schedule (= slabs needed).
-int max_segments(int N, int K, int grid = TC_GRID)
+int max_segments(int N, int K, int grid = TC_GRID, int n_prob = 1)
 {
     StreamK sk;
     sk.KB = ceil_div(K, TC_BK);
-    const int tiles = ceil_div(N, TC_TILE_N);
+    const int tiles = ceil_div(N, TC_TILE_N) * n_prob;      // work tiles
     sk.U = (long long)tiles * sk.KB;
     sk.G = (int)std::min<long long>(grid, sk.U);
     int worst = 1;
@@ -211,17 +212,18 @@ int max_segments(int N, int K, int grid = TC_GRID)
 // among the grids that the slabs were sized for, the one whose busiest CTA has the least to do, counting a shared
 // segment as PART_COST extra K steps and the final merge as MERGE_COST.  (40 tiles of a long K: 120 CTAs, three to a
 // tile; 120 tiles: one each; 216 tiles: 144 CTAs, three tiles to a pair.)
-int many_row_grid(int N, int K)
+int many_row_grid(int N, int K, int n_prob = 1)
 {
     static const int forced = getenv("SWIFT_MANY_GRID") ? atoi(getenv("SWIFT_MANY_GRID")) : 0;
     constexpr long long PART_COST = 10, MERGE_COST = 14;
     static std::mutex mu;
-    static std::map<std::pair<int, int>, int> memo;         // the search below is far too slow for a launch path
+    static std::map<std::tuple<int, int, int>, int> memo;   // the search below is far too slow for a launch path
     std::lock_guard<std::mutex> lock(mu);
-    auto it = memo.find({N, K});
+    const std::tuple<int, int, int> key{N, K, n_prob};
+    auto it = memo.find(key);
     if (it != memo.end()) return it->second;
-    const int tiles = ceil_div(N, TC_TILE_N), cap = max_segments(N, K);
-    if (forced > 0 && forced <= TC_GRID && max_segments(N, K, forced) <= cap) return memo[{N, K}] = forced;
+    const int tiles = ceil_div(N, TC_TILE_N) * n_prob, cap = max_segments(N, K, TC_GRID, n_prob);
+    if (forced > 0 && forced <= TC_GRID && max_segments(N, K, forced, n_prob) <= cap) return memo[key] = forced;
     StreamK sk;
     sk.KB = ceil_div(K, TC_BK);
     sk.U = (long long)tiles * sk.KB;
@@ -229,7 +231,7 @@ int many_row_grid(int N, int K)
     long long best_cost = -1;
     for (int G = TC_GRID; G >= TC_GRID / 2; --G) {
         sk.G = (int)std::min<long long>(G, sk.U);
-        if (max_segments(N, K, G) > cap) continue;
+        if (max_segments(N, K, G, n_prob) > cap) continue;
         long long worst = 0;
         bool shared = false;
         for (int g = 0; g < sk.G; ++g) {
@@ -242,7 +244,7 @@ int many_row_grid(int N, int K)
         if (shared) worst += MERGE_COST;
         if (best_cost < 0 || worst < best_cost) { best_cost = worst; best = G; }
     }
-    return memo[{N, K}] = best;
+    return memo[key] = best;
 }
 
 // Scratch KV pages beyond the sequence's own: the window of one candidate (copy-on-write start page included), or the
@@ -262,8 +264,8 @@ size_t score_map_ints(const swift_model_desc* d)
     return (size_t)(2 * d->n_blocks + 1) * (SCORE_ROWS_MAX / TC_ROWS_MAX + SCORE_ROWS_MAX / ROWS / 2) * TC_ROWS_MAX;
 }
 
-// Rows of the largest forward chunk: TC_ROWS_MAX where the tensor-core walk with many-row chunks applies, else 16.
-size_t big_rows_of(const swift_model_desc* d) { return (d->dtype == SWIFT_BF16 && d->head_dim == 128) ? (size_t)TC_ROWS_MAX : (size_t)ROWS; }
+// Rows of the largest forward chunk: TC_BIG_ROWS where the tensor-core walk with many-row chunks applies, else 16.
+size_t big_rows_of(const swift_model_desc* d) { return (d->dtype == SWIFT_BF16 && d->head_dim == 128) ? (size_t)TC_BIG_ROWS : (size_t)ROWS; }
 
 WorkLayout work_layout(const swift_model_desc* d)
 {
@@ -316,7 +318,9 @@ WorkLayout work_layout(const swift_model_desc* d)
     k.xn_hl = k.xa_hl = k.act_hl = k.slabs = k.counters = k.sumsq = 0;
     if (d->dtype == SWIFT_BF16) {
         auto slab_need = [&](int N, int K) {      // whole tiles: the many-row form parks 128 x RB values per tile
-            k.slab_floats = std::max(k.slab_floats, (size_t)max_segments(N, K) * RB * (size_t)ceil_div(N, TC_TILE_N) * TC_TILE_N);
+            int segs = max_segments(N, K);
+            for (int np = 2; np <= TC_PROBS_MAX; ++np) segs = std::max(segs, max_segments(N, K, TC_GRID, np));
+            k.slab_floats = std::max(k.slab_floats, (size_t)segs * RB * (size_t)ceil_div(N, TC_TILE_N) * TC_TILE_N);
         };
         slab_need((int)(qd + 2 * kd), (int)dm); slab_need((int)dm, (int)qd); slab_need(2 * d->ffn, (int)dm);
         slab_need((int)dm, d->ffn); slab_need(d->vocab, (int)dm);
@@ -404,28 +408,29 @@ struct GemmSite {
 };
 
 template <int EPI, typename TKV, int NB = 1>
-swift_status launch_gemm_tc(swift_ctx* ctx, const GemmSite& g, const EpiParams& ep, const CUtensorMap* next_map = nullptr)
+swift_status launch_gemm_tc(swift_ctx* ctx, const GemmSite& g, const EpiParams& ep, const CUtensorMap* next_map = nullptr, int n_prob = 1)
 {
-    if (ceil_div(g.N, TC_TILE_N) > TC_MAX_TILES) return fail(ctx, SWIFT_EUNSUPPORTED, "GEMM with %d output tiles", ceil_div(g.N, TC_TILE_N));
+    if (ceil_div(g.N, TC_TILE_N) * n_prob > TC_MAX_TILES) return fail(ctx, SWIFT_EUNSUPPORTED, "GEMM with %d output tiles", ceil_div(g.N, TC_TILE_N) * n_prob);
     if (ctx->pdl_gemms) ctx->pdl_next = true;     // this launch may begin before its predecessor has finished (see swift_load)
     // Decoding streams each weight once and wants every SM to stream the same bytes: 148 CTAs, tiles cut where the ranges
     // fall.  A chunk of many rows is bound by its tensor work and its epilogues: see many_row_grid.
     int grid = TC_GRID;
-    if (NB > 1 && ctx->whole_tiles) grid = many_row_grid(g.N, g.K);
+    if (NB > 1 && ctx->whole_tiles) grid = many_row_grid(g.N, g.K, n_prob);
     CU(launch_k(gemm_tc_kernel<EPI, TKV, NB>, dim3(grid), dim3(TC_THREADS), (size_t)TcShape<NB>::SMEM_BYTES, ctx, state_of(ctx), *g.mapW, *g.mapX,
                 kptr<float>(ctx, ctx->kl.part), kptr<float>(ctx, ctx->kl.slabs), kptr<int>(ctx, ctx->kl.counters), g.N, g.K, ep,
-                next_map ? *next_map : *g.mapW));
+                next_map ? *next_map : *g.mapW, n_prob));
     return SWIFT_OK;
 }
 
 // The plain-epilogue GEMM of a chunk of many rows with its output at Y ([rows][N]).
 template <int NB>
-swift_status launch_gemm_tc_y(swift_ctx* ctx, const GemmSite& g, const EpiParams& ep, float* Y)
+swift_status launch_gemm_tc_y(swift_ctx* ctx, const GemmSite& g, const EpiParams& ep, float* Y, int n_prob = 1)
 {
+    if (ceil_div(g.N, TC_TILE_N) * n_prob > TC_MAX_TILES) return fail(ctx, SWIFT_EUNSUPPORTED, "GEMM with %d output tiles", ceil_div(g.N, TC_TILE_N) * n_prob);
     int grid = TC_GRID;
-    if (ctx->whole_tiles) grid = many_row_grid(g.N, g.K);
+    if (ctx->whole_tiles) grid = many_row_grid(g.N, g.K, n_prob);
     CU(launch_k(gemm_tc_kernel<EPI_PLAIN, float, NB>, dim3(grid), dim3(TC_THREADS), (size_t)TcShape<NB>::SMEM_BYTES, ctx, state_of(ctx), *g.mapW,
-                *g.mapX, Y, kptr<float>(ctx, ctx->kl.slabs), kptr<int>(ctx, ctx->kl.counters), g.N, g.K, ep, *g.mapW));
+                *g.mapX, Y, kptr<float>(ctx, ctx->kl.slabs), kptr<int>(ctx, ctx->kl.counters), g.N, g.K, ep, *g.mapW, n_prob));
     return SWIFT_OK;
 }
 
@@ -740,7 +745,7 @@ swift_status forward_chunk_fused(swift_ctx* ctx, int rows, const int* toks_dev, 
     return SWIFT_OK;
 }
 
-// The full model over a chunk of up to TC_ROWS_MAX rows (prefill): the same walk as forward_chunk_fused with every weight
+// The full model over a chunk of up to TC_BIG_ROWS rows (prefill): the same walk as forward_chunk_fused with every weight
 // tile applied to all rows at once (the GEMM in its NB = 8 form, tensor-core attention over all rows of a chunk per K,V
 // load), no output head.  Tokens in the big_tok device array; the control block holds pos0 and the row count.
 template <typename TKV>
@@ -762,7 +767,8 @@ swift_status forward_chunk_big(swift_ctx* ctx, int rows, const int* page_table)
     base.inv_d = 1.0f / (float)dm;
     base.eps = d.rms_eps;
     base.sumsq_in = sumsq;
-    base.sum_rows = TC_ROWS_MAX;
+    base.sum_rows = TC_BIG_ROWS;
+    const int n_prob = ceil_div(rows, TC_ROWS_MAX);      // row ranges of 128 that each GEMM launch runs as separate problems
     const int d_tiles = ceil_div(dm, TC_TILE_N);
     int n_tiles_in = 1;
     CU(launch_k(embed_fused_kernel<T>, dim3(rows), dim3(1024), 0, ctx, st, (const int*)kptr<int>(ctx, ctx->kl.big_tok),
@@ -772,24 +778,24 @@ swift_status forward_chunk_big(swift_ctx* ctx, int rows, const int* page_table)
         ep.n_sumsq_tiles = n_tiles_in;
         ep.q_out = kptr<float>(ctx, ctx->kl.q); ep.kv_pool = ctx->kvbase; ep.page_table = page_table; ep.L = ctx->kv;
         ep.block = b; ep.n_heads = d.n_heads; ep.max_positions = d.max_positions; ep.rope_cs = kptr<float2>(ctx, ctx->kl.rope);
-        ST((launch_gemm_tc<EPI_QKV, TKV, NB>(ctx, GemmSite{nullptr, nqkv, dm, nullptr, &ctx->tm_wqkv[b], &ctx->tm_xn_big}, ep)));
-        if (ctx->attn_tile) ST((launch_attn_tile<TKV>(ctx, page_table, b, rows, TC_ROWS_MAX, 0, 0, 0)));
-        else ST((launch_attn_mma<TKV, 2>(ctx, page_table, b, false, xa, xa_hl, TC_ROWS_MAX, 0, 0, 0,
+        ST((launch_gemm_tc<EPI_QKV, TKV, NB>(ctx, GemmSite{nullptr, nqkv, dm, nullptr, &ctx->tm_wqkv[b], &ctx->tm_xn_big}, ep, nullptr, n_prob)));
+        if (ctx->attn_tile) ST((launch_attn_tile<TKV>(ctx, page_table, b, rows, TC_BIG_ROWS, 0, 0, 0)));
+        else ST((launch_attn_mma<TKV, 2>(ctx, page_table, b, false, xa, xa_hl, TC_BIG_ROWS, 0, 0, 0,
                                          ceil_div((d.n_heads / d.n_kv_heads) * rows, 16))));
         CU(launch_k(attn_combine_kernel, dim3(d.n_heads, rows), dim3(d.head_dim), 2 * (size_t)ctx->max_splits * sizeof(float), ctx,
                     (const DevState*)st, (const float*)kptr<float>(ctx, ctx->kl.o_part), (const float2*)kptr<float2>(ctx, ctx->kl.ml_part),
-                    ctx->max_splits, d.n_heads, d.head_dim, xa, xa_hl, (int)TC_ROWS_MAX, 0, 0, 0, 1));
+                    ctx->max_splits, d.n_heads, d.head_dim, xa, xa_hl, (int)TC_BIG_ROWS, 0, 0, 0, 1));
         EpiParams resid = base;
         resid.h = h; resid.planes_out = xn_hl; resid.sumsq_out = sumsq;
         resid.gain_next = wptr<float>(ctx, ctx->wl.mlp_norm[b]);
-        ST((launch_gemm_tc<EPI_RESID, float, NB>(ctx, GemmSite{nullptr, dm, qd, nullptr, &ctx->tm_wo[b], &ctx->tm_xa_big}, resid)));
+        ST((launch_gemm_tc<EPI_RESID, float, NB>(ctx, GemmSite{nullptr, dm, qd, nullptr, &ctx->tm_wo[b], &ctx->tm_xa_big}, resid, nullptr, n_prob)));
         EpiParams sw = base;
         sw.n_sumsq_tiles = d_tiles;
         sw.act_planes = act_hl; sw.ffn = d.ffn;
-        ST((launch_gemm_tc<EPI_SWIGLU, float, NB>(ctx, GemmSite{nullptr, 2 * d.ffn, dm, nullptr, &ctx->tm_wgu[b], &ctx->tm_xn_big}, sw)));
+        ST((launch_gemm_tc<EPI_SWIGLU, float, NB>(ctx, GemmSite{nullptr, 2 * d.ffn, dm, nullptr, &ctx->tm_wgu[b], &ctx->tm_xn_big}, sw, nullptr, n_prob)));
         // nothing reads the residual stream of a prefill chunk after its last block: no planes, no sums there
         resid.gain_next = b + 1 < d.n_blocks ? wptr<float>(ctx, ctx->wl.attn_norm[b + 1]) : nullptr;
-        ST((launch_gemm_tc<EPI_RESID, float, NB>(ctx, GemmSite{nullptr, dm, d.ffn, nullptr, &ctx->tm_wdown[b], &ctx->tm_act_big}, resid)));
+        ST((launch_gemm_tc<EPI_RESID, float, NB>(ctx, GemmSite{nullptr, dm, d.ffn, nullptr, &ctx->tm_wdown[b], &ctx->tm_act_big}, resid, nullptr, n_prob)));
         n_tiles_in = d_tiles;
     }
     CU(cudaGetLastError());
@@ -1324,10 +1330,10 @@ swift_status make_all_maps(swift_ctx* ctx)
     ST(make_map(ctx, &ctx->tm_xn, ctx->ws + ctx->kl.xn_hl, 2 * ROWS, dm, TC_COLS));
     ST(make_map(ctx, &ctx->tm_xa, ctx->ws + ctx->kl.xa_hl, 2 * ROWS, qd, TC_COLS));
     ST(make_map(ctx, &ctx->tm_act, ctx->ws + ctx->kl.act_hl, 2 * ROWS, d.ffn, TC_COLS));
-    if (big_rows_of(&d) == (size_t)TC_ROWS_MAX) {
-        ST(make_map(ctx, &ctx->tm_xn_big, ctx->ws + ctx->kl.xn_hl, 2 * TC_ROWS_MAX, dm, TcShape<TC_NB_MAX>::COLS));
-        ST(make_map(ctx, &ctx->tm_xa_big, ctx->ws + ctx->kl.xa_hl, 2 * TC_ROWS_MAX, qd, TcShape<TC_NB_MAX>::COLS));
-        ST(make_map(ctx, &ctx->tm_act_big, ctx->ws + ctx->kl.act_hl, 2 * TC_ROWS_MAX, d.ffn, TcShape<TC_NB_MAX>::COLS));
+    if (big_rows_of(&d) == (size_t)TC_BIG_ROWS) {
+        ST(make_map(ctx, &ctx->tm_xn_big, ctx->ws + ctx->kl.xn_hl, 2 * TC_BIG_ROWS, dm, TcShape<TC_NB_MAX>::COLS));
+        ST(make_map(ctx, &ctx->tm_xa_big, ctx->ws + ctx->kl.xa_hl, 2 * TC_BIG_ROWS, qd, TcShape<TC_NB_MAX>::COLS));
+        ST(make_map(ctx, &ctx->tm_act_big, ctx->ws + ctx->kl.act_hl, 2 * TC_BIG_ROWS, d.ffn, TcShape<TC_NB_MAX>::COLS));
     }
     return SWIFT_OK;
 }
@@ -1422,8 +1428,9 @@ swift_status swift_load(const swift_model_desc* desc, swift_devbuf weights, swif
     c->use_pdl = getenv("SWIFT_PDL") != nullptr;
     c->fuse = getenv("SWIFT_NO_FUSE") == nullptr && desc->head_dim <= TC_TILE_N;
     // prefill in chunks of up to TC_ROWS_MAX rows (SWIFT_NO_BIG_CHUNKS: 16 rows at a time, as decoding does)
-    c->big_chunks = c->use_tc && c->fuse && big_rows_of(desc) == (size_t)TC_ROWS_MAX && getenv("SWIFT_NO_BIG_CHUNKS") == nullptr;
+    c->big_chunks = c->use_tc && c->fuse && big_rows_of(desc) == (size_t)TC_BIG_ROWS && getenv("SWIFT_NO_BIG_CHUNKS") == nullptr;
     c->whole_tiles = getenv("SWIFT_NO_WHOLE_TILES") == nullptr;
+    c->two_problems = getenv("SWIFT_NO_TWO_PROBLEMS") == nullptr;    // prefill chunks of 256 rows: two 128-row problems per GEMM launch
     c->attn_tile = getenv("SWIFT_NO_ATTN_TILE") == nullptr;      // chunks of many rows: 64-row query tiles with K,V staged in shared memory
     // Grouped-query models: the target model's decoding forwards (verification, vanilla steps) take that kernel too, one
     // CTA serving all query heads of a KV group, so that a K,V chunk is fetched and converted once per group
@@ -1560,15 +1567,16 @@ swift_status swift_prefill(swift_ctx* ctx, const int32_t* tokens, int32_t n, int
     ctx->round_open = false;
     ctx->n = 0;
     int last_rows = 0;
-    // All but the last (up to 16) rows go through in chunks of up to TC_ROWS_MAX rows where that path exists: every weight
+    // All but the last (up to 16) rows go through in chunks of up to TC_BIG_ROWS rows where that path exists: every weight
     // is then streamed once per 128 rows instead of once per 16.  The last rows take the decoding path, which ends in
     // the output head.
     int done = 0;
     if (ctx->big_chunks && n > 2 * ROWS) {
         const int big_total = ((n - 1) / ROWS) * ROWS;           // leaves 1..16 rows
         DevState* st = state_of(ctx);
-        for (int c0 = 0; c0 < big_total; c0 += TC_ROWS_MAX) {
-            const int rows = std::min((int)TC_ROWS_MAX, big_total - c0);
+        const int chunk = ctx->two_problems ? (int)TC_BIG_ROWS : (int)TC_ROWS_MAX;
+        for (int c0 = 0; c0 < big_total; c0 += chunk) {
+            const int rows = std::min(chunk, big_total - c0);
             CU(copy_async(ctx, kptr<int>(ctx, ctx->kl.big_tok), tokens + c0, (size_t)rows * 4, cudaMemcpyHostToDevice));
             set_rows_kernel<<<1, 1, 0, ctx->stream>>>(st, c0, rows);
             ctx->launches++;
@@ -1767,7 +1775,7 @@ swift_status swift_gemm(swift_ctx* ctx, int32_t which, int32_t block, const floa
     if (!ctx || !x_host || !y_host) return fail(ctx, SWIFT_EINVAL, "null argument");
     if (ctx->round_open) return fail(ctx, SWIFT_ESTATE, "a round is open");
     const swift_model_desc& d = ctx->d;
-    if (which < 0 || which > 4 || n_rows < 1 || n_rows > TC_ROWS_MAX || block < 0 || block >= d.n_blocks)
+    if (which < 0 || which > 4 || n_rows < 1 || n_rows > TC_BIG_ROWS || block < 0 || block >= d.n_blocks)
         return fail(ctx, SWIFT_EINVAL, "bad which / block / n_rows");
     if (n_rows > ROWS && !(ctx->use_tc && ctx->big_chunks)) return fail(ctx, SWIFT_EUNSUPPORTED, "no many-row GEMM for this model or kernel choice");
     const int dm = d.d_model, qd = d.n_heads * d.head_dim, kd = d.n_kv_heads * d.head_dim;
@@ -1790,13 +1798,13 @@ swift_status swift_gemm(swift_ctx* ctx, int32_t which, int32_t block, const floa
         ctx->launches++;
         EpiParams ep;
         memset(&ep, 0, sizeof ep);
-        ep.sum_rows = TC_ROWS_MAX;
+        ep.sum_rows = TC_BIG_ROWS;
         GemmSite g{nullptr, N, K, nullptr,
                    which == 0 ? &ctx->tm_wqkv[block] : which == 1 ? &ctx->tm_wo[block] : which == 2 ? &ctx->tm_wgu[block]
                    : which == 3 ? &ctx->tm_wdown[block] : &ctx->tm_lm_head,
                    which == 1 ? &ctx->tm_xa_big : which == 3 ? &ctx->tm_act_big : &ctx->tm_xn_big};
         float* Y = kptr<float>(ctx, ctx->kl.score_logits);
-        ST(launch_gemm_tc_y<TC_NB_MAX>(ctx, g, ep, Y));
+        ST(launch_gemm_tc_y<TC_NB_MAX>(ctx, g, ep, Y, ceil_div(n_rows, TC_ROWS_MAX)));
         CU(copy_async(ctx, y_host, Y, (size_t)n_rows * N * 4, cudaMemcpyDeviceToHost));
         DevState hs;
         return read_state(ctx, &hs);
@@ -2006,11 +2014,11 @@ static swift_status time_gemm_t(swift_ctx* ctx, int which, int n_rows, int iters
         if (N > d.vocab) return fail(ctx, SWIFT_ECAPACITY, "output of %d columns does not fit the buffer used for timing", N);
         EpiParams ep;
         memset(&ep, 0, sizeof ep);
-        ep.sum_rows = TC_ROWS_MAX;
+        ep.sum_rows = TC_BIG_ROWS;
         auto big = [&](int i) -> swift_status {
             GemmSite g = site(i);
             g.mapX = which == 1 ? &ctx->tm_xa_big : which == 3 ? &ctx->tm_act_big : &ctx->tm_xn_big;
-            return launch_gemm_tc_y<TC_NB_MAX>(ctx, g, ep, kptr<float>(ctx, ctx->kl.score_logits));
+            return launch_gemm_tc_y<TC_NB_MAX>(ctx, g, ep, kptr<float>(ctx, ctx->kl.score_logits), ceil_div(n_rows, TC_ROWS_MAX));
         };
         for (int i = 0; i < 3; ++i) ST(big(i));
         CU(cudaEventRecord(ctx->ev[0], ctx->stream));
@@ -2043,7 +2051,7 @@ swift_status swift_time_gemm(swift_ctx* ctx, int32_t which, int32_t n_rows, int3
 {
     if (!ctx || !ms || !bytes) return fail(ctx, SWIFT_EINVAL, "null argument");
     if (ctx->round_open) return fail(ctx, SWIFT_ESTATE, "a round is open");
-    if (which < 0 || which > 4 || n_rows < 1 || (n_rows > ROWS && n_rows != TC_ROWS_MAX) || iters < 1) return fail(ctx, SWIFT_EINVAL, "bad which / n_rows / iters");
+    if (which < 0 || which > 4 || n_rows < 1 || (n_rows > ROWS && n_rows != TC_ROWS_MAX && n_rows != TC_BIG_ROWS) || iters < 1) return fail(ctx, SWIFT_EINVAL, "bad which / n_rows / iters");
     if (ctx->d.dtype == SWIFT_BF16) return time_gemm_t<__nv_bfloat16>(ctx, which, n_rows, iters, ms, bytes);
     return time_gemm_t<float>(ctx, which, n_rows, iters, ms, bytes);
 }

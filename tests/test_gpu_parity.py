@@ -141,11 +141,12 @@ def test_weight_streaming_gemm_kernels(shape, rows):
         g.close()
 
 
-@pytest.mark.parametrize("shape,rows", [("13b", 128), ("13b", 100), ("7b", 77), ("70b", 33)])
+@pytest.mark.parametrize("shape,rows", [("13b", 128), ("13b", 100), ("7b", 77), ("70b", 33), ("13b", 256), ("7b", 200), ("70b", 145)])
 def test_many_row_gemm_against_the_oracle(shape, rows):
     """The many-row form of the tensor-core GEMM (prefill chunks, side-by-side scoring) alone, at the real projection
     shapes: whole tiles per CTA (QKV, gate/up, head) and tiles shared between three or four CTAs (o_proj, down), full and
-    ragged row counts (a last block of 4, 13 or 1 rows), against the oracle's fp64 projection."""
+    ragged row counts (a last block of 4, 13 or 1 rows), one and two 128-row problems per launch (more than 128 rows),
+    against the oracle's fp64 projection."""
     cfg = synth.MODELS[shape].with_blocks(1, n_planted=0)
     from paper_2410_06916_b200 import SwiftModel
     g = SwiftModel(cfg, max_positions=64)
@@ -165,9 +166,12 @@ def test_many_row_gemm_against_the_oracle(shape, rows):
             ref = so.linear(x, W).numpy()
             scale = float(np.sqrt((ref ** 2).mean()))
             y = g.gemm(which, 0, x.numpy())
-            assert np.abs(y - ref).max() < 1e-4 * scale, (which, float(np.abs(y - ref).max()), scale)
+            # fp32 accumulation over K terms in one chain (a tile that one CTA takes whole) walks about sqrt(K) * 2^-24 of the
+            # result's scale: measured rms 1.3e-5 (two half-length chains) to 2.1e-5 (one chain) at K = 28672, maxima 7e-5 / 1.3e-4
+            tol = 1e-4 * scale * max(1.0, float(np.sqrt(W.shape[1] / 8192)))
+            assert np.abs(y - ref).max() < tol, (which, float(np.abs(y - ref).max()), scale)
             y16 = g.gemm(which, 0, x.numpy()[:16])               # the decoding kernel on the first 16 rows: same products, other order
-            assert np.abs(y16 - y[:16]).max() < 1e-4 * scale, which
+            assert np.abs(y16 - y[:16]).max() < tol, which
         ms, nbytes = g.time_gemm(2 if 2 * F <= cfg.vocab else 0, 128, 3)
         assert ms > 0 and nbytes > 0
     finally:
