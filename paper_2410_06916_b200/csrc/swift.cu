@@ -249,7 +249,7 @@ int many_row_grid(int N, int K, int n_prob = 1)
 
 // Scratch KV pages beyond the sequence's own: the window of one candidate (copy-on-write start page included), or the
 // windows of the several candidates of one chunk when candidates are scored side by side.
-int scratch_pages(const swift_model_desc* d) { return MAX_SCORE_ROWS / d->page_size + 8; }
+int scratch_pages(const swift_model_desc* d) { return 2 * MAX_SCORE_ROWS / d->page_size + 16; }
 
 size_t page_bytes(const swift_model_desc* d)
 {
@@ -257,11 +257,11 @@ size_t page_bytes(const swift_model_desc* d)
 }
 
 constexpr int SCORE_ROWS_MAX = 4096;     // candidates x window rows scored side by side (beyond that: one candidate at a time)
-constexpr int SCORE_SLOTS_MAX = 8;       // candidates per chunk of TC_ROWS_MAX rows (window of 16 rows)
-// Row-map entries of one scoring round: one map of TC_ROWS_MAX rows per (sub-layer or output head, chunk of candidates).
+constexpr int SCORE_SLOTS_MAX = TC_BIG_ROWS / ROWS;       // candidates per chunk of TC_BIG_ROWS rows (window of 16 rows)
+// Row-map entries of one scoring round: one map of a chunk's rows (128 or 256) per (sub-layer or output head, chunk of candidates).
 size_t score_map_ints(const swift_model_desc* d)
 {
-    return (size_t)(2 * d->n_blocks + 1) * (SCORE_ROWS_MAX / TC_ROWS_MAX + SCORE_ROWS_MAX / ROWS / 2) * TC_ROWS_MAX;
+    return (size_t)(2 * d->n_blocks + 1) * (SCORE_ROWS_MAX / TC_ROWS_MAX + SCORE_ROWS_MAX / ROWS / 2) * TC_BIG_ROWS;
 }
 
 // Rows of the largest forward chunk: TC_BIG_ROWS where the tensor-core walk with many-row chunks applies, else 16.
@@ -1093,7 +1093,7 @@ swift_status enqueue_score(swift_ctx* ctx, const uint8_t* masks, int C, int gamm
 // The records of a run count 2 bytes (a 16-bit cache, what the method needs); an fp32 cache moves twice that.
 // All candidates side by side ("Parallel Candidate Evaluation", Section 4.1): every candidate keeps its own copy of the
 // window's gamma residual rows; the sub-layers are walked once, and each is applied to the candidates that keep it,
-// gathered into chunks of up to TC_ROWS_MAX rows, so its weights are streamed once per chunk of candidates instead of
+// gathered into chunks of up to TC_BIG_ROWS rows, so its weights are streamed once per chunk of candidates instead of
 // once per 16 rows of every candidate.  Each candidate of a chunk has its own scratch KV pages for the window.  Results
 // (match counts) land in the score_out device array.  Returns SWIFT_EUNSUPPORTED when the shape does not fit this form.
 template <typename TKV>
@@ -1105,7 +1105,8 @@ swift_status enqueue_score_batched(swift_ctx* ctx, const uint8_t* masks, int C, 
     const int n = ctx->n, L = 2 * d.n_blocks, P = d.page_size, pos_w = n - gamma;
     if (!ctx->big_chunks || gamma % ROWS || gamma > TC_ROWS_MAX || C * gamma > SCORE_ROWS_MAX) return SWIFT_EUNSUPPORTED;
     const int pages_per_slot = ceil_div(gamma, P) + 1;
-    const int cpg = std::min(std::min(TC_ROWS_MAX / gamma, ctx->n_pages_scratch / pages_per_slot), (int)SCORE_SLOTS_MAX);   // candidates per chunk
+    const int chunk_rows = ctx->two_problems ? (int)TC_BIG_ROWS : (int)TC_ROWS_MAX;      // 256: two 128-row problems per GEMM launch
+    const int cpg = std::min(std::min(chunk_rows / gamma, ctx->n_pages_scratch / pages_per_slot), (int)SCORE_SLOTS_MAX);   // candidates per chunk
     if (cpg < 1) return SWIFT_EUNSUPPORTED;
     // ---- row maps of the whole round: per sub-layer, the candidates that keep it in chunks of cpg; then the output head
     struct Chunk { int sub; int n_cand; size_t map_off; };
@@ -1119,7 +1120,7 @@ swift_status enqueue_score_batched(swift_ctx* ctx, const uint8_t* masks, int C, 
             chunks.push_back({sub, nc, maps.size()});
             for (int j = 0; j < nc; ++j)
                 for (int i = 0; i < gamma; ++i) maps.push_back(keep[g0 + j] * gamma + i);
-            maps.resize(chunks.back().map_off + TC_ROWS_MAX, 0);
+            maps.resize(chunks.back().map_off + chunk_rows, 0);
         }
     }
     if (maps.size() > score_map_ints(&d)) return SWIFT_EUNSUPPORTED;
@@ -1161,19 +1162,19 @@ swift_status enqueue_score_batched(swift_ctx* ctx, const uint8_t* masks, int C, 
     base.inv_d = 1.0f / (float)dm;
     base.eps = d.rms_eps;
     base.sumsq_in = sumsq;
-    base.sum_rows = TC_ROWS_MAX;
+    base.sum_rows = TC_BIG_ROWS;
     base.n_sumsq_tiles = 1;                           // gather_norm_kernel leaves each row's sum of squares as tile 0
     embed_rows_kernel<T><<<C * gamma, 256, 0, ctx->stream>>>(st, tok_dev, (const T*)wptr<T>(ctx, ctx->wl.embed), H_all, dm, d.vocab, gamma);
     ctx->launches++;
     for (const Chunk& ch : chunks) {
-        const int rows = ch.n_cand * gamma;
+        const int rows = ch.n_cand * gamma, n_prob = ceil_div(rows, TC_ROWS_MAX);
         const int* map = maps_dev + ch.map_off;
         set_rows_kernel<<<1, 1, 0, ctx->stream>>>(st, pos_w, rows);
         ctx->launches++;
         if (ch.sub == L) {                            // output head: final norm, logits, arg max per row
             gather_norm_kernel<<<rows, 1024, 0, ctx->stream>>>(map, H_all, wptr<float>(ctx, ctx->wl.final_norm), xn_hl, sumsq, dm);
             ctx->launches++;
-            ST((launch_gemm_tc_y<NB>(ctx, GemmSite{nullptr, d.vocab, dm, nullptr, &ctx->tm_lm_head, &ctx->tm_xn_big}, base, logits)));
+            ST((launch_gemm_tc_y<NB>(ctx, GemmSite{nullptr, d.vocab, dm, nullptr, &ctx->tm_lm_head, &ctx->tm_xn_big}, base, logits, n_prob)));
             // the head's chunks hold consecutive candidates: their predictions go where their rows are in H_all
             argmax_rows_kernel<<<rows, 1024, 0, ctx->stream>>>(logits, d.vocab, pred + maps[ch.map_off]);
             ctx->launches++;
@@ -1190,31 +1191,31 @@ swift_status enqueue_score_batched(swift_ctx* ctx, const uint8_t* masks, int C, 
             ep.q_out = kptr<float>(ctx, ctx->kl.q); ep.kv_pool = ctx->kvbase; ep.page_table = pt_dev; ep.L = ctx->kv;
             ep.block = b; ep.n_heads = d.n_heads; ep.max_positions = d.max_positions; ep.rope_cs = kptr<float2>(ctx, ctx->kl.rope);
             ep.per_block = 1;
-            for (int rb = 0; rb < NB; ++rb) {
+            for (int rb = 0; rb < NB * n_prob; ++rb) {
                 const int j = std::min((rb * ROWS) / gamma, ch.n_cand - 1);
                 ep.rb_pos0[rb] = pos_w + (rb * ROWS) % gamma;
                 ep.rb_page_table[rb] = pt_dev + (size_t)j * np;
             }
-            ST((launch_gemm_tc<EPI_QKV, TKV, NB>(ctx, GemmSite{nullptr, nqkv, dm, nullptr, &ctx->tm_wqkv[b], &ctx->tm_xn_big}, ep)));
+            ST((launch_gemm_tc<EPI_QKV, TKV, NB>(ctx, GemmSite{nullptr, nqkv, dm, nullptr, &ctx->tm_wqkv[b], &ctx->tm_xn_big}, ep, nullptr, n_prob)));
             // each candidate of the chunk is a sequence of its own behind the context they share
             if (ctx->attn_tile) {
-                ST((launch_attn_tile<TKV>(ctx, pt_dev, b, gamma, TC_ROWS_MAX, 0, gamma, pos_w, ch.n_cand, np)));
+                ST((launch_attn_tile<TKV>(ctx, pt_dev, b, gamma, TC_BIG_ROWS, 0, gamma, pos_w, ch.n_cand, np)));
             } else {
                 for (int j = 0; j < ch.n_cand; ++j)
-                    ST((launch_attn_mma<TKV, 2>(ctx, pt_dev + (size_t)j * np, b, false, xa, xa_hl, TC_ROWS_MAX, j * gamma, gamma, pos_w,
+                    ST((launch_attn_mma<TKV, 2>(ctx, pt_dev + (size_t)j * np, b, false, xa, xa_hl, TC_BIG_ROWS, j * gamma, gamma, pos_w,
                                                 ceil_div((d.n_heads / d.n_kv_heads) * gamma, 16))));
             }
             CU(launch_k(attn_combine_kernel, dim3(d.n_heads, ch.n_cand * gamma), dim3(d.head_dim), 2 * (size_t)ctx->max_splits * sizeof(float), ctx,
                         (const DevState*)st, (const float*)kptr<float>(ctx, ctx->kl.o_part), (const float2*)kptr<float2>(ctx, ctx->kl.ml_part),
-                        ctx->max_splits, d.n_heads, d.head_dim, xa, xa_hl, (int)TC_ROWS_MAX, 0, gamma, pos_w, ch.n_cand));
-            ST((launch_gemm_tc<EPI_RESID, float, NB>(ctx, GemmSite{nullptr, dm, qd, nullptr, &ctx->tm_wo[b], &ctx->tm_xa_big}, resid)));
+                        ctx->max_splits, d.n_heads, d.head_dim, xa, xa_hl, (int)TC_BIG_ROWS, 0, gamma, pos_w, ch.n_cand));
+            ST((launch_gemm_tc<EPI_RESID, float, NB>(ctx, GemmSite{nullptr, dm, qd, nullptr, &ctx->tm_wo[b], &ctx->tm_xa_big}, resid, nullptr, n_prob)));
         } else {
             gather_norm_kernel<<<rows, 1024, 0, ctx->stream>>>(map, H_all, wptr<float>(ctx, ctx->wl.mlp_norm[b]), xn_hl, sumsq, dm);
             ctx->launches++;
             EpiParams sw = base;
             sw.act_planes = act_hl; sw.ffn = d.ffn;
-            ST((launch_gemm_tc<EPI_SWIGLU, float, NB>(ctx, GemmSite{nullptr, 2 * d.ffn, dm, nullptr, &ctx->tm_wgu[b], &ctx->tm_xn_big}, sw)));
-            ST((launch_gemm_tc<EPI_RESID, float, NB>(ctx, GemmSite{nullptr, dm, d.ffn, nullptr, &ctx->tm_wdown[b], &ctx->tm_act_big}, resid)));
+            ST((launch_gemm_tc<EPI_SWIGLU, float, NB>(ctx, GemmSite{nullptr, 2 * d.ffn, dm, nullptr, &ctx->tm_wgu[b], &ctx->tm_xn_big}, sw, nullptr, n_prob)));
+            ST((launch_gemm_tc<EPI_RESID, float, NB>(ctx, GemmSite{nullptr, dm, d.ffn, nullptr, &ctx->tm_wdown[b], &ctx->tm_act_big}, resid, nullptr, n_prob)));
         }
     }
     match_rows_kernel<<<ceil_div(C, 128), 128, 0, ctx->stream>>>(pred, truth_dev, gamma, C, kptr<int>(ctx, ctx->kl.score_out));
