@@ -274,9 +274,9 @@ swift_status swift_set_gemm_impl(swift_ctx* ctx, int32_t impl);
 /* One weight-streaming GEMM of the walk on caller data: y[r][n] = sum_k x[r][k] * W[n][k] with W the
  * stored weight `which` (0 fused QKV, 1 o_proj, 2 fused gate/up in its interleaved row order, 3 down,
  * 4 output head) of `block`.  x_host: fp32 [n_rows][K], y_host: fp32 [n_rows][N].  n_rows <= 16: the kernel
- * decoding uses.  17 <= n_rows <= 256: the many-row form of the tensor-core kernel that prefill chunks and
- * side-by-side candidate scoring use, more than 128 rows as two row ranges ("problems") that share each weight tile
- * within one launch (bf16 models with head_dim 128 and the tensor-core kernel selected, else SWIFT_EUNSUPPORTED;
+ * decoding uses.  17 <= n_rows <= 512: the many-row form of the tensor-core kernel that prefill chunks and
+ * side-by-side candidate scoring use, more than 128 rows as up to four row ranges ("problems") that share each weight
+ * tile within one launch (bf16 models with head_dim 128 and the tensor-core kernel selected, else SWIFT_EUNSUPPORTED;
  * SWIFT_ECAPACITY if N exceeds the vocabulary size). */
 swift_status swift_gemm(swift_ctx* ctx, int32_t which, int32_t block, const float* x_host, int32_t n_rows,
                         float* y_host);
@@ -308,7 +308,7 @@ int32_t swift_round_times(const swift_ctx* ctx, int32_t capacity, float* ms_draf
  * what the implementation moves, beside the algorithmic figure above.  Same conventions as swift_round_times. */
 int32_t swift_round_bytes_stored(const swift_ctx* ctx, int32_t capacity, double* bytes_draft_host, double* bytes_verify_host);
 /* Times `iters` back-to-back launches of one weight-streaming GEMM of the walk (which: 0 fused QKV,
- * 1 o_proj, 2 fused gate/up, 3 down, 4 output head) with n_rows rows (1..16, or 128 or 256: the many-row form that
+ * 1 o_proj, 2 fused gate/up, 3 down, 4 output head) with n_rows rows (1..16, or 128, 256, 384 or 512: the many-row form that
  * prefill chunks and side-by-side candidate scoring use, with the plain epilogue; SWIFT_EUNSUPPORTED where the
  * model has no such form, SWIFT_ECAPACITY if the output is wider than the vocabulary), cycling over the blocks'
  * weights so that successive launches read different memory.  Outputs the average CUDA-event time per launch

@@ -68,7 +68,7 @@ struct TcShape {
 };
 constexpr int TC_NB_MAX = 8;
 constexpr int TC_ROWS_MAX = ROWS * TC_NB_MAX;       // rows one accumulator tile covers (the wide form's "problem")
-constexpr int TC_PROBS_MAX = 2;                     // problems a launch of the wide form may hold: row ranges of TC_ROWS_MAX rows that share
+constexpr int TC_PROBS_MAX = 4;                     // problems a launch of the wide form may hold: row ranges of TC_ROWS_MAX rows that share
                                                     // the weights but nothing else; work tile T = weight tile T / n_prob of problem T % n_prob
 constexpr int TC_BIG_ROWS = TC_ROWS_MAX * TC_PROBS_MAX;   // rows of the largest forward chunk
 constexpr int TC_ERR_TIMEOUT = 2;

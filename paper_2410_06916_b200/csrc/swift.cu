@@ -83,7 +83,8 @@ struct swift_ctx {
     std::string err;
     cudaEvent_t ev[8];
     // captured forwards; programmatic dependent launch between the kernels of a forward
-    bool use_graphs, use_pdl, pdl_next, pdl_gemms, fuse, fuse_combine, prefetch_next, attn_mma, big_chunks, batched_scoring, whole_tiles, attn_tile, attn_tile_decode, attn_tile_drafts, two_problems;
+    bool use_graphs, use_pdl, pdl_next, pdl_gemms, fuse, fuse_combine, prefetch_next, attn_mma, big_chunks, batched_scoring, whole_tiles, attn_tile, attn_tile_decode, attn_tile_drafts;
+    int many_problems;              // 128-row problems per many-row GEMM launch (chunks of prefill and of candidate scoring hold that many)
     bool tree_forward = false;      // the forward being enqueued verifies a token tree (rows see their ancestors, not all earlier rows)
     int attn_rows_per_cta, prefetch_tiles;
     std::vector<FwdGraph>* graphs;
@@ -191,7 +192,7 @@ WeightLayout weight_layout(const swift_model_desc* d)
 }
 
 constexpr int TC_GRID = 148;        // persistent CTAs of the tensor-core GEMM: one per SM of a B200
-constexpr int TC_MAX_TILES = 1024;
+constexpr int TC_MAX_TILES = 2048;       // work tiles of one launch (70B gate/up: 448 weight tiles x 4 problems)
 
 // Largest number of CTAs that share one output tile under the stream-K schedule (= slabs needed).
 int max_segments(int N, int K, int grid = TC_GRID, int n_prob = 1)
@@ -249,7 +250,7 @@ int many_row_grid(int N, int K, int n_prob = 1)
 
 // Scratch KV pages beyond the sequence's own: the window of one candidate (copy-on-write start page included), or the
 // windows of the several candidates of one chunk when candidates are scored side by side.
-int scratch_pages(const swift_model_desc* d) { return 2 * MAX_SCORE_ROWS / d->page_size + 16; }
+int scratch_pages(const swift_model_desc* d) { return TC_PROBS_MAX * (MAX_SCORE_ROWS / d->page_size + 8); }
 
 size_t page_bytes(const swift_model_desc* d)
 {
@@ -1105,7 +1106,7 @@ swift_status enqueue_score_batched(swift_ctx* ctx, const uint8_t* masks, int C, 
     const int n = ctx->n, L = 2 * d.n_blocks, P = d.page_size, pos_w = n - gamma;
     if (!ctx->big_chunks || gamma % ROWS || gamma > TC_ROWS_MAX || C * gamma > SCORE_ROWS_MAX) return SWIFT_EUNSUPPORTED;
     const int pages_per_slot = ceil_div(gamma, P) + 1;
-    const int chunk_rows = ctx->two_problems ? (int)TC_BIG_ROWS : (int)TC_ROWS_MAX;      // 256: two 128-row problems per GEMM launch
+    const int chunk_rows = ctx->many_problems * TC_ROWS_MAX;      // several 128-row problems per GEMM launch
     const int cpg = std::min(std::min(chunk_rows / gamma, ctx->n_pages_scratch / pages_per_slot), (int)SCORE_SLOTS_MAX);   // candidates per chunk
     if (cpg < 1) return SWIFT_EUNSUPPORTED;
     // ---- row maps of the whole round: per sub-layer, the candidates that keep it in chunks of cpg; then the output head
@@ -1431,7 +1432,10 @@ swift_status swift_load(const swift_model_desc* desc, swift_devbuf weights, swif
     // prefill in chunks of up to TC_ROWS_MAX rows (SWIFT_NO_BIG_CHUNKS: 16 rows at a time, as decoding does)
     c->big_chunks = c->use_tc && c->fuse && big_rows_of(desc) == (size_t)TC_BIG_ROWS && getenv("SWIFT_NO_BIG_CHUNKS") == nullptr;
     c->whole_tiles = getenv("SWIFT_NO_WHOLE_TILES") == nullptr;
-    c->two_problems = getenv("SWIFT_NO_TWO_PROBLEMS") == nullptr;    // prefill chunks of 256 rows: two 128-row problems per GEMM launch
+    {   // chunks of 512 rows: four 128-row problems per GEMM launch (SWIFT_MANY_PROBLEMS=1..4 for measurement)
+        const char* e = getenv("SWIFT_MANY_PROBLEMS");
+        c->many_problems = e ? std::max(1, std::min((int)TC_PROBS_MAX, atoi(e))) : (int)TC_PROBS_MAX;
+    }
     c->attn_tile = getenv("SWIFT_NO_ATTN_TILE") == nullptr;      // chunks of many rows: 64-row query tiles with K,V staged in shared memory
     // Grouped-query models: the target model's decoding forwards (verification, vanilla steps) take that kernel too, one
     // CTA serving all query heads of a KV group, so that a K,V chunk is fetched and converted once per group
@@ -1575,7 +1579,7 @@ swift_status swift_prefill(swift_ctx* ctx, const int32_t* tokens, int32_t n, int
     if (ctx->big_chunks && n > 2 * ROWS) {
         const int big_total = ((n - 1) / ROWS) * ROWS;           // leaves 1..16 rows
         DevState* st = state_of(ctx);
-        const int chunk = ctx->two_problems ? (int)TC_BIG_ROWS : (int)TC_ROWS_MAX;
+        const int chunk = ctx->many_problems * TC_ROWS_MAX;
         for (int c0 = 0; c0 < big_total; c0 += chunk) {
             const int rows = std::min(chunk, big_total - c0);
             CU(copy_async(ctx, kptr<int>(ctx, ctx->kl.big_tok), tokens + c0, (size_t)rows * 4, cudaMemcpyHostToDevice));
@@ -2052,7 +2056,7 @@ swift_status swift_time_gemm(swift_ctx* ctx, int32_t which, int32_t n_rows, int3
 {
     if (!ctx || !ms || !bytes) return fail(ctx, SWIFT_EINVAL, "null argument");
     if (ctx->round_open) return fail(ctx, SWIFT_ESTATE, "a round is open");
-    if (which < 0 || which > 4 || n_rows < 1 || (n_rows > ROWS && n_rows != TC_ROWS_MAX && n_rows != TC_BIG_ROWS) || iters < 1) return fail(ctx, SWIFT_EINVAL, "bad which / n_rows / iters");
+    if (which < 0 || which > 4 || n_rows < 1 || (n_rows > ROWS && (n_rows % TC_ROWS_MAX || n_rows > TC_BIG_ROWS)) || iters < 1) return fail(ctx, SWIFT_EINVAL, "bad which / n_rows / iters");
     if (ctx->d.dtype == SWIFT_BF16) return time_gemm_t<__nv_bfloat16>(ctx, which, n_rows, iters, ms, bytes);
     return time_gemm_t<float>(ctx, which, n_rows, iters, ms, bytes);
 }

@@ -34,7 +34,7 @@ def test_size_queries_and_layout_invariants():
         assert params * es + gains <= wb <= params * es + gains + 256 * (6 * cfg.n_blocks + 4), name
         kv = lib.swift_kv_bytes(C.byref(d))
         per_pos = cfg.n_blocks * 2 * cfg.n_kv_heads * cfg.head_dim * 4      # kv_dtype 0 = fp32
-        assert kv == (4096 + 16 * (2 * 128 // 16 + 16)) * per_pos      # the sequence + scratch pages (windows of the candidates of one chunk)
+        assert kv == (4096 + 16 * 4 * (128 // 16 + 8)) * per_pos       # the sequence + scratch pages (windows of the candidates of one chunk)
         assert lib.swift_workspace_bytes(C.byref(d)) > 0
     bad = binding._Desc(4, 64, 4, 3, 16, 96, 97, 0, 1e4, 1e-5, 64, 16, 4, 0)     # heads not a multiple of kv heads
     assert lib.swift_weights_bytes(C.byref(bad)) == 0

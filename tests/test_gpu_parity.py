@@ -141,11 +141,11 @@ def test_weight_streaming_gemm_kernels(shape, rows):
         g.close()
 
 
-@pytest.mark.parametrize("shape,rows", [("13b", 128), ("13b", 100), ("7b", 77), ("70b", 33), ("13b", 256), ("7b", 200), ("70b", 145)])
+@pytest.mark.parametrize("shape,rows", [("13b", 128), ("13b", 100), ("7b", 77), ("70b", 33), ("13b", 256), ("7b", 200), ("70b", 145), ("13b", 512), ("7b", 400)])
 def test_many_row_gemm_against_the_oracle(shape, rows):
     """The many-row form of the tensor-core GEMM (prefill chunks, side-by-side scoring) alone, at the real projection
     shapes: whole tiles per CTA (QKV, gate/up, head) and tiles shared between three or four CTAs (o_proj, down), full and
-    ragged row counts (a last block of 4, 13 or 1 rows), one and two 128-row problems per launch (more than 128 rows),
+    ragged row counts (a last block of 4, 13 or 1 rows), one to four 128-row problems per launch (more than 128 rows),
     against the oracle's fp64 projection."""
     cfg = synth.MODELS[shape].with_blocks(1, n_planted=0)
     from paper_2410_06916_b200 import SwiftModel
