@@ -1,6 +1,6 @@
 // Attention for chunks of many rows (prefill chunks, the window rows of a scored candidate): one CTA = one KV head x one
-// 64-position chunk of the cache x one tile of 64 query rows (query row rho = hl * n_rows + r: head hl of the KV head's
-// group, row r of the sequence).  The chunk's K and V are loaded from the paged cache once per 64 query rows, split into
+// 64-position chunk of the cache x up to four tiles of 64 query rows, taken in turn (query row rho = hl * n_rows + r: head hl of the KV head's
+// group, row r of the sequence).  The chunk's K and V are loaded from the paged cache once per CTA, split into
 // bf16 hi / lo planes (16 significant bits together, as everywhere else) and kept in shared memory; each of the four
 // warps owns 16 query rows and runs S = Q K^T and O = P V on mma.sync.m16n8k16 with three MMAs per product
 // (lo*hi, hi*lo, hi*hi), fp32 accumulation, a soft-max over the chunk per row in registers.  Outputs are the same
@@ -13,7 +13,8 @@
 namespace swk {
 
 constexpr int AT_THREADS = 128;
-constexpr int AT_QROWS = 64;            // query rows per CTA
+constexpr int AT_QROWS = 64;            // query rows per tile (16 per warp)
+constexpr int AT_TPC = 4;               // tiles a CTA takes in turn on one staged chunk
 constexpr int AT_KSTRIDE = 136;         // bf16 per staged K or V row (128 + 8: rows of a fragment load fall into different banks)
 constexpr size_t AT_SMEM_BYTES = (size_t)4 * ATTN_CHUNK * AT_KSTRIDE * 2;   // K hi, K lo, V hi, V lo
 
@@ -23,7 +24,7 @@ __device__ __forceinline__ void ldmatrix_x2_trans(uint32_t& r0, uint32_t& r1, co
     asm volatile("ldmatrix.sync.aligned.m8n8.x2.trans.shared.b16 {%0, %1}, [%2];" : "=r"(r0), "=r"(r1) : "r"(a));
 }
 
-// grid = (n_kv_heads, max_splits, query tiles), block = 128, dynamic smem = AT_SMEM_BYTES.
+// grid = (n_kv_heads, max_splits, ceil(query tiles / AT_TPC)), block = 128, dynamic smem = AT_SMEM_BYTES.
 // row_base / n_rows_fixed / pos0_fixed: as in attn_mma_kernel (a sequence inside a larger chunk), else 0 / 0 / 0.
 // n_seq > 1: that many such sequences in one launch (grid.z covers the larger of the batch's and the sequences' tiles),
 // page tables pt_stride ints apart.
@@ -44,6 +45,7 @@ attn_tile_kernel(const DevState* st, const float* __restrict__ q, const T* __res
     const int len = min(ATTN_CHUNK, total - c0);
     const int G = n_heads / L.n_kv_heads;
     int z = blockIdx.z;
+    bool per_seq = false;
     if (n_seq > 1) {
         // n_seq sequences of n_rows rows side by side (rows row_base + seq * n_rows ..), all continuing the same cached
         // context, each with its own page table for its own rows.  A chunk that lies inside the context is the same for
@@ -54,17 +56,20 @@ attn_tile_kernel(const DevState* st, const float* __restrict__ q, const T* __res
         } else {
             const int tiles_per = (G * n_rows + AT_QROWS - 1) / AT_QROWS, seq = z / tiles_per;
             if (seq >= n_seq) return;
+            per_seq = true;
             z -= seq * tiles_per;
             row_base += seq * n_rows;
             page_table += (size_t)seq * pt_stride;
         }
     }
     const int R = G * n_rows;
-    const int rho_tile = z * AT_QROWS;
-    if (rho_tile >= R) return;
-    {   // a tile none of whose rows sees this chunk yet has nothing to add: the merge never reads it
-        const int rho1 = min(R, rho_tile + AT_QROWS) - 1;
-        const int r_last = (rho_tile / n_rows == rho1 / n_rows) ? rho1 % n_rows : n_rows - 1;
+    // the CTA stages its chunk once and then takes up to AT_TPC tiles of 64 query rows in turn (one tile where every sequence
+    // has a chunk of its own)
+    const int tile_first = per_seq ? z : z * AT_TPC, tile_count = per_seq ? 1 : AT_TPC;
+    if (tile_first * AT_QROWS >= R) return;
+    {   // tiles none of whose rows sees this chunk yet have nothing to add: the merge never reads them
+        const int rho0 = tile_first * AT_QROWS, rho1 = min(R, (tile_first + tile_count) * AT_QROWS) - 1;
+        const int r_last = (rho0 / n_rows == rho1 / n_rows) ? rho1 % n_rows : n_rows - 1;
         if (c0 > pos0 + r_last) return;
     }
     const int tid = threadIdx.x, lane = tid & 31, w = tid >> 5, g = lane >> 2, t = lane & 3;
@@ -82,25 +87,6 @@ attn_tile_kernel(const DevState* st, const float* __restrict__ q, const T* __res
     __shared__ int page_of[ATTN_CHUNK];
     if (tid < ATTN_CHUNK) page_of[tid] = tid < len ? __ldg(page_table + ((c0 + tid) >> L.page_shift)) : 0;
 
-    // ---- this warp's 16 query rows as A fragments (hi, lo), scaled: rows rho_w + g and rho_w + g + 8
-    const int rho_w = rho_tile + 16 * w;
-    const int rho_a = rho_w + g, rho_b = rho_w + g + 8;
-    const bool live_a = rho_a < R, live_b = rho_b < R;
-    const int hl_a = live_a ? rho_a / n_rows : 0, r_a = live_a ? rho_a - hl_a * n_rows : 0;
-    const int hl_b = live_b ? rho_b / n_rows : 0, r_b = live_b ? rho_b - hl_b * n_rows : 0;
-    const float* qa = q + ((size_t)r_a * n_heads + kvh * G + hl_a) * DH;
-    const float* qb = q + ((size_t)r_b * n_heads + kvh * G + hl_b) * DH;
-    uint32_t qh[8][4], ql[8][4];
-#pragma unroll
-    for (int ks = 0; ks < 8; ++ks) {                        // k-step ks: dims 16 ks .. 16 ks + 15
-        float2 a0 = make_float2(0.f, 0.f), a1 = a0, a2 = a0, a3 = a0;
-        if (live_a) { a0 = *reinterpret_cast<const float2*>(qa + 16 * ks + 2 * t); a2 = *reinterpret_cast<const float2*>(qa + 16 * ks + 8 + 2 * t); }
-        if (live_b) { a1 = *reinterpret_cast<const float2*>(qb + 16 * ks + 2 * t); a3 = *reinterpret_cast<const float2*>(qb + 16 * ks + 8 + 2 * t); }
-        split_pair(a0.x * scale, a0.y * scale, qh[ks][0], ql[ks][0]);
-        split_pair(a1.x * scale, a1.y * scale, qh[ks][1], ql[ks][1]);
-        split_pair(a2.x * scale, a2.y * scale, qh[ks][2], ql[ks][2]);
-        split_pair(a3.x * scale, a3.y * scale, qh[ks][3], ql[ks][3]);
-    }
     __syncthreads();
 #pragma unroll
     for (int part = 0; part < ATTN_CHUNK * 32 / (8 * AT_THREADS); ++part) {
@@ -129,7 +115,35 @@ attn_tile_kernel(const DevState* st, const float* __restrict__ q, const T* __res
         }
     }
     __syncthreads();
-    if (rho_w >= R) return;                                 // (after the barrier: every warp helped staging)
+
+    for (int ti = 0; ti < tile_count; ++ti) {              // no barrier below: the warps go through their tiles on their own
+    const int rho_tile = (tile_first + ti) * AT_QROWS;
+    if (rho_tile >= R) break;
+    {
+        const int rho1 = min(R, rho_tile + AT_QROWS) - 1;
+        const int r_last = (rho_tile / n_rows == rho1 / n_rows) ? rho1 % n_rows : n_rows - 1;
+        if (c0 > pos0 + r_last) continue;                   // this tile sees nothing of the chunk
+    }
+    // ---- this warp's 16 query rows as A fragments (hi, lo), scaled: rows rho_w + g and rho_w + g + 8
+    const int rho_w = rho_tile + 16 * w;
+    if (rho_w >= R) break;
+    const int rho_a = rho_w + g, rho_b = rho_w + g + 8;
+    const bool live_a = rho_a < R, live_b = rho_b < R;
+    const int hl_a = live_a ? rho_a / n_rows : 0, r_a = live_a ? rho_a - hl_a * n_rows : 0;
+    const int hl_b = live_b ? rho_b / n_rows : 0, r_b = live_b ? rho_b - hl_b * n_rows : 0;
+    const float* qa = q + ((size_t)r_a * n_heads + kvh * G + hl_a) * DH;
+    const float* qb = q + ((size_t)r_b * n_heads + kvh * G + hl_b) * DH;
+    uint32_t qh[8][4], ql[8][4];
+#pragma unroll
+    for (int ks = 0; ks < 8; ++ks) {                        // k-step ks: dims 16 ks .. 16 ks + 15
+        float2 a0 = make_float2(0.f, 0.f), a1 = a0, a2 = a0, a3 = a0;
+        if (live_a) { a0 = *reinterpret_cast<const float2*>(qa + 16 * ks + 2 * t); a2 = *reinterpret_cast<const float2*>(qa + 16 * ks + 8 + 2 * t); }
+        if (live_b) { a1 = *reinterpret_cast<const float2*>(qb + 16 * ks + 2 * t); a3 = *reinterpret_cast<const float2*>(qb + 16 * ks + 8 + 2 * t); }
+        split_pair(a0.x * scale, a0.y * scale, qh[ks][0], ql[ks][0]);
+        split_pair(a1.x * scale, a1.y * scale, qh[ks][1], ql[ks][1]);
+        split_pair(a2.x * scale, a2.y * scale, qh[ks][2], ql[ks][2]);
+        split_pair(a3.x * scale, a3.y * scale, qh[ks][3], ql[ks][3]);
+    }
 
     // ---- scores of the warp's 16 rows against the chunk's 64 positions: 8 tiles of 8 positions
     float sacc[8][4];
@@ -209,6 +223,7 @@ attn_tile_kernel(const DevState* st, const float* __restrict__ q, const T* __res
         for (int nt = 0; nt < 16; ++nt)
             *reinterpret_cast<float2*>(o_part + slot * DH + 8 * nt + 2 * t) = make_float2(oacc[nt][2], oacc[nt][3]);
         if (t == 0) ml_part[slot] = make_float2(m_b, l_b);
+    }
     }
 }
 

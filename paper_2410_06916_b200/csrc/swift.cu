@@ -488,7 +488,10 @@ swift_status launch_attn_tile(swift_ctx* ctx, const int* page_table, int block, 
 {
     const swift_model_desc& d = ctx->d;
     const int G = d.n_heads / d.n_kv_heads;
-    const int z = std::max(ceil_div(G * rows * n_seq, AT_QROWS), n_seq * ceil_div(G * rows, AT_QROWS));
+    // a CTA takes up to AT_TPC query tiles on one staged chunk; with several sequences the chunks that reach into their own
+    // rows take one tile per CTA and sequence
+    const int z = n_seq > 1 ? std::max(ceil_div(ceil_div(G * rows * n_seq, AT_QROWS), AT_TPC), n_seq * ceil_div(G * rows, AT_QROWS))
+                            : ceil_div(ceil_div(G * rows, AT_QROWS), AT_TPC);
     CU(launch_k(attn_tile_kernel<T>, dim3(d.n_kv_heads, ctx->max_splits, z), dim3(AT_THREADS), AT_SMEM_BYTES, ctx,
                 (const DevState*)state_of(ctx), (const float*)kptr<float>(ctx, ctx->kl.q), reinterpret_cast<const T*>(ctx->kvbase),
                 page_table, ctx->kv, block, d.n_heads, ctx->max_splits, 1.0f / sqrtf((float)d.head_dim),
