@@ -919,4 +919,15 @@ __global__ void split_planes_kernel(const float* __restrict__ x, __nv_bfloat16* 
     if (i < K) store_hi_lo(planes, row0 + r, K, i, x[(size_t)r * K + i]);
 }
 
+// Deterministic non-trivial contents for operand planes that a timing run would otherwise read as they happen to be
+// (zeros toggle no bits in the tensor pipe and understate its power draw): values in [-0.5, 0.5), lo planes included.
+__global__ void fill_planes_kernel(__nv_bfloat16* __restrict__ planes, size_t n)
+{
+    for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (size_t)gridDim.x * blockDim.x) {
+        unsigned h = (unsigned)i * 2654435761u;
+        h ^= h >> 15; h *= 2246822519u; h ^= h >> 13;
+        planes[i] = __float2bfloat16_rn((float)(h & 0xFFFF) * (1.0f / 65536.0f) - 0.5f);
+    }
+}
+
 } // namespace swk
