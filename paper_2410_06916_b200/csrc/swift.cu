@@ -2046,6 +2046,12 @@ static swift_status time_gemm_t(swift_ctx* ctx, int which, int n_rows, int iters
         DevState hs;
         return read_state(ctx, &hs);
     }
+    if (ctx->use_tc) {     // defined, non-trivial operand planes (see fill_planes_kernel)
+        __nv_bfloat16* planes = which == 1 ? kptr<__nv_bfloat16>(ctx, ctx->kl.xa_hl) : which == 3 ? kptr<__nv_bfloat16>(ctx, ctx->kl.act_hl)
+                                           : kptr<__nv_bfloat16>(ctx, ctx->kl.xn_hl);
+        fill_planes_kernel<<<64, 256, 0, ctx->stream>>>(planes, (size_t)2 * ROWS * K);
+        ctx->launches++;
+    }
     for (int i = 0; i < 3; ++i) ST(run_gemm<T>(ctx, mr_of(n_rows), site(i), &S));
     CU(cudaEventRecord(ctx->ev[0], ctx->stream));
     for (int i = 0; i < iters; ++i) ST(run_gemm<T>(ctx, mr_of(n_rows), site(i + 3), &S));
